@@ -1,0 +1,97 @@
+"""Seeded synthetic inputs shared by the tests, the benchmark and the oracle checks.
+
+This module holds no arithmetic of the method: it only draws numbers and rounds them once
+to the storage type, so that the fp64 oracle and the CUDA path receive identical values.
+
+Recipe (stands in for the paper's C4-token workloads; only shapes and distributions are
+taken): numpy Generator(PCG64(seed)).standard_normal in fp64, drawn in the fixed order
+x (or ids), then per layer W_q, W_k, W_v, W_o, W_up, W_down, then the embedding E;
+weights scaled by 1/sqrt(fan_in); E ~ N(0,1); gains are ones (None).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional
+
+import numpy as np
+
+BASE_SEED = 20260421
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    n_layers: int
+    B: int
+    N: int
+    d_model: int
+    n_heads: int
+    d_ff: int
+    dtype: str              # "f32" or "bf16" (storage; accumulation is always fp32 on the GPU)
+    vocab: int = 0          # 0 = single layer fed with x directly
+    residual_scale: float = 1.0
+    head_dim: int = 64
+
+
+# The five configurations the benchmark definition names (c5 is the N sweep: see sweep()).
+WORKLOADS: Dict[str, Workload] = {
+    "c1": Workload("c1", 1, 1, 256, 128, 2, 512, "f32"),
+    "c2": Workload("c2", 1, 4, 2048, 768, 12, 3072, "bf16"),
+    "c3": Workload("c3", 1, 8, 4096, 1024, 16, 4096, "bf16"),
+    "c4": Workload("c4", 8, 16, 2048, 1024, 16, 4096, "bf16", vocab=32000,
+                   residual_scale=1.0 / np.sqrt(8.0)),
+}
+CONFIG_INDEX = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+
+
+def sweep(N: int) -> Workload:
+    """One point of the sequence-length sweep (B=1, d=1024, bf16)."""
+    return Workload(f"c5_N{N}", 1, 1, N, 1024, 16, 4096, "bf16")
+
+
+def seed_for(wl: Workload) -> int:
+    if wl.name.startswith("c5_N"):
+        return BASE_SEED + 4 + int(np.log2(wl.N))
+    return BASE_SEED + CONFIG_INDEX.get(wl.name, 99)
+
+
+def round_to(a: np.ndarray, dtype: str) -> np.ndarray:
+    """Round fp64 values once to the storage type and return them as fp64 again."""
+    if dtype == "f32":
+        return a.astype(np.float32).astype(np.float64)
+    if dtype == "bf16":
+        import torch
+        return torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    if dtype == "f64":
+        return np.asarray(a, dtype=np.float64)
+    raise ValueError(dtype)
+
+
+WEIGHT_NAMES = ("w_q", "w_k", "w_v", "w_o", "w_up", "w_down")
+
+
+def make_inputs(wl: Workload, seed: Optional[int] = None, B: Optional[int] = None,
+                N: Optional[int] = None) -> dict:
+    """Returns {"x" or "ids", "layers": [ {w_q..w_down} ], "emb"}; every float array is fp64
+    holding values already rounded to wl.dtype.  B / N override the workload's sizes (the
+    draw order is fixed, so a smaller B is NOT a prefix of the full draw)."""
+    rng = np.random.Generator(np.random.PCG64(seed_for(wl) if seed is None else seed))
+    B = wl.B if B is None else B
+    N = wl.N if N is None else N
+    d, f = wl.d_model, wl.d_ff
+    out: dict = {}
+    if wl.vocab:
+        out["ids"] = rng.integers(0, wl.vocab, size=(B, N)).astype(np.int32)
+    else:
+        out["x"] = round_to(rng.standard_normal((B, N, d)), wl.dtype)
+    layers: List[dict] = []
+    for _ in range(wl.n_layers):
+        lw = {}
+        for name, shape, fan_in in (("w_q", (d, d), d), ("w_k", (d, d), d), ("w_v", (d, d), d),
+                                    ("w_o", (d, d), d), ("w_up", (f, d), d), ("w_down", (d, f), f)):
+            lw[name] = round_to(rng.standard_normal(shape) / np.sqrt(fan_in), wl.dtype)
+        layers.append(lw)
+    out["layers"] = layers
+    if wl.vocab:
+        out["emb"] = round_to(rng.standard_normal((wl.vocab, d)), wl.dtype)
+    return out

@@ -1,0 +1,347 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+
+None of these re-uses the oracle's own formulas as the expected value: the expected values
+are closed forms (Sec. 4's theorem), textbook dense attention (App. A's construction),
+the paper's worked schedule examples (tests/golden), combinatorial identities of
+Algorithm 1, scalar math.erf, or relations between independent oracle variants.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import (RTConfig, RTWeights, alg1_tiles, gelu, layer_blk, layer_decode,
+                    layer_fixed_point, layer_seq, rms, stack_decode, stack_prefill, update_tile)
+from oracle.rt_oracle import NORM_PRE, NORM_QK, NORM_QK_FULL, NORM_SKIP_Z
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rand_layer(rng, d, H, dff, flags=NORM_PRE | NORM_QK, alpha=1.0, scale=None, gains=False):
+    cfg = RTConfig(d, H, d // H, dff, norm_flags=flags, residual_scale=alpha, softmax_scale=scale)
+    mk = lambda o, i: rng.standard_normal((o, i)) / np.sqrt(i)
+    w = RTWeights(mk(d, d), mk(d, d), mk(d, d), mk(d, d), mk(dff, d), mk(d, dff))
+    if gains:
+        for g in ("g_attn", "g_mlp", "g_kv", "g_q", "g_k"):
+            setattr(w, g, 1.0 + 0.3 * rng.standard_normal(d))
+    return cfg, w
+
+
+# ------------------------------------------------------------------ schedule (Algorithm 1)
+
+def test_schedule_worked_examples_from_the_paper():
+    rows = [tuple(int(v) for v in ln.split()) for ln in open(os.path.join(GOLDEN, "alg1_worked_examples.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    tiles = {t: (s, e, u, v) for (t, u, v, s, e) in alg1_tiles(8)}
+    assert len(rows) == 2
+    for t, s, e, u, v in rows:
+        assert tiles[t] == (s, e, u, v)
+
+
+@pytest.mark.parametrize("leaf", [1, 2, 3, 4, 8, 16])
+def test_schedule_covers_every_pair_exactly_once(leaf):
+    # App. C: every query accumulates every earlier pair exactly once.  The pairs of a
+    # query's own block come from the in-block step, the rest from the cross tiles.
+    for N in list(range(1, 70)) + [127, 128, 129, 200, 255, 300]:
+        cnt = np.zeros((N + 1, N + 1), dtype=np.int32)
+        for (t, u, v, s, e) in alg1_tiles(N, leaf):
+            assert e == t and u == t + 1 and v <= N and s >= 1
+            cnt[u:v + 1, s:e + 1] += 1
+        for i in range(1, N + 1):
+            start = ((i - 1) // leaf) * leaf + 1
+            cnt[i, start:i] += 1
+        want = np.tril(np.ones((N + 1, N + 1), dtype=np.int32), -1)
+        want[0, :] = 0; want[:, 0] = 0
+        assert np.array_equal(cnt, want), (N, leaf)
+
+
+def test_schedule_total_tile_size_closed_form():
+    # Sum over t of the largest power of two dividing t is (N/2) log2 N + N for N = 2^k
+    # (the O(log N) average slice of Sec. 6, "Cache locality").
+    for k in range(0, 12):
+        N = 1 << k
+        total = sum(e - s + 1 for (t, u, v, s, e) in alg1_tiles(2 * N) if t <= N)
+        assert total == (N // 2) * k + N
+
+
+# ------------------------------------------------------------------ primitives
+
+def test_rms_is_sqrtD_times_unit_vector():
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((5, 48))
+    y = rms(x, np.ones(48), 0.0)
+    assert np.allclose(np.linalg.norm(y, axis=-1), math.sqrt(48), rtol=1e-14)
+    assert np.allclose(y / np.linalg.norm(y, axis=-1, keepdims=True),
+                       x / np.linalg.norm(x, axis=-1, keepdims=True), rtol=1e-13)
+
+
+def test_gelu_is_x_times_normal_cdf():
+    for a in (-6.0, -2.5, -1.0, -0.1, 0.0, 0.3, 1.0, 2.0, 7.0):
+        want = a * 0.5 * math.erfc(-a / math.sqrt(2.0))
+        assert abs(float(gelu(np.array([a]))[0]) - want) <= 1e-15 * max(1.0, abs(want))
+    assert abs(float(gelu(np.array([1.0]))[0]) - 0.8413447460685429) < 1e-15   # Phi(1)
+
+
+def test_update_tile_two_halves_equal_plain_softmax():
+    rng = np.random.default_rng(1)
+    q = rng.standard_normal((3, 8)); K = rng.standard_normal((10, 8)); V = rng.standard_normal((10, 8))
+    m = np.full(3, -np.inf); l = np.zeros(3); o = np.zeros((3, 8))
+    m, l, o = update_tile(q, K[:4], V[:4], m, l, o, 0.7)
+    m, l, o = update_tile(q, K[4:], V[4:], m, l, o, 0.7)
+    S = 0.7 * q @ K.T
+    P = np.exp(S) / np.exp(S).sum(axis=1, keepdims=True)
+    assert np.allclose(o / l[:, None], P @ V, rtol=1e-13, atol=1e-14)
+    assert np.allclose(m, S.max(axis=1))
+
+
+# ------------------------------------------------------------------ pin: closed-form Jacobian (Sec. 4 theorem)
+
+def stirling_first_unsigned(n):
+    c = [[0] * (n + 1) for _ in range(n + 1)]
+    c[0][0] = 1
+    for i in range(1, n + 1):
+        for r in range(1, i + 1):
+            c[i][r] = (i - 1) * c[i - 1][r] + c[i - 1][r - 1]
+    return c
+
+
+@pytest.mark.parametrize("alpha", [1.0, 0.5])
+def test_uniform_attention_layer_matches_closed_form_jacobian(alpha):
+    # Norms off, W_q = 0 (uniform attention), W_o = I, W_down = 0, one head: the layer is
+    # z_k = x_k + (alpha/k)(V x_k + V sum_{j<k} z_j), a linear map whose derivative with
+    # respect to x_1 is (1/k!) sum_r [k r] alpha^r V^r  (k >= 2) and I + alpha V (k = 1).
+    d, N = 6, 9
+    rng = np.random.default_rng(2)
+    V = rng.standard_normal((d, d)) / np.sqrt(d)
+    cfg = RTConfig(d, 1, d, 4, norm_flags=0, residual_scale=alpha, softmax_scale=1.0)
+    w = RTWeights(np.zeros((d, d)), rng.standard_normal((d, d)), V, np.eye(d),
+                  rng.standard_normal((4, d)), np.zeros((d, 4)))
+    X = np.zeros((d, N, d))
+    for j in range(d):
+        X[j, 0, j] = 1.0                         # sequence j feeds x_1 = e_j, zeros elsewhere
+    z, _, _ = layer_seq(cfg, w, X)
+    st = stirling_first_unsigned(N)
+    aV = alpha * V
+    for k in range(1, N + 1):
+        J = z[:, k - 1, :].T                      # column j = response of z_k to e_j
+        if k == 1:
+            want = np.eye(d) + aV
+        else:
+            want = sum(st[k][r] * np.linalg.matrix_power(aV, r) for r in range(1, k + 1)) / math.factorial(k)
+            prod = np.eye(d)
+            for m in range(k):
+                prod = prod @ (aV + m * np.eye(d))
+            assert np.allclose(want, prod / math.factorial(k), rtol=1e-12, atol=1e-14)
+        assert np.allclose(J, want, rtol=1e-12, atol=1e-14), k
+
+
+# ------------------------------------------------------------------ pin: reduces to textbook causal attention (App. A)
+
+@pytest.mark.parametrize("H,qk", [(1, False), (3, False), (3, True)])
+def test_two_block_construction_equals_textbook_causal_attention(H, qk):
+    # Each head's slice splits into a carry half (read by Q, K, V; never written) and a
+    # scratch half (written by V through W_o = I).  With x = (c ; 0), W_down = 0 and no
+    # pre-norm, z = (c ; a): the persistent pair of a position equals its temporary pair,
+    # so the layer is plain causal softmax attention over (Q c, K c, V c).
+    e, N, B = 4, 11, 2
+    dh, d = 2 * e, 2 * e * H
+    rng = np.random.default_rng(3)
+    carry = np.array([h * dh + j for h in range(H) for j in range(e)])
+    scratch = carry + e
+    QT, KT, VT = (rng.standard_normal((H * e, H * e)) for _ in range(3))
+    Wq = np.zeros((d, d)); Wk = np.zeros((d, d)); Wv = np.zeros((d, d))
+    Wq[np.ix_(carry, carry)] = QT
+    Wk[np.ix_(carry, carry)] = KT
+    Wv[np.ix_(scratch, carry)] = VT
+    flags = NORM_QK if qk else 0
+    scale = 0.37
+    cfg = RTConfig(d, H, dh, 5, norm_flags=flags, softmax_scale=scale)
+    w = RTWeights(Wq, Wk, Wv, np.eye(d), rng.standard_normal((5, d)), np.zeros((d, 5)))
+    if qk:   # distinct learnable gains for queries and keys
+        w.g_q = 1.0 + 0.3 * rng.standard_normal(d)
+        w.g_k = 1.0 + 0.3 * rng.standard_normal(d)
+    c = rng.standard_normal((B, N, H * e))
+    x = np.zeros((B, N, d)); x[..., carry] = c
+    z, k, v = layer_seq(cfg, w, x)
+
+    # textbook: per head, softmax(mask(s Q K^T)) V on dense matrices
+    Q = c @ QT.T; K = c @ KT.T; Vv = c @ VT.T
+    want = np.zeros((B, N, H * e))
+    for b in range(B):
+        for h in range(H):
+            sl = slice(h * e, (h + 1) * e)
+            Qh, Kh = Q[b, :, sl], K[b, :, sl]
+            if qk:   # per-head unit-RMS rows; the zero scratch half counts in the mean (width 2e)
+                Qh = Qh / np.sqrt((Qh ** 2).sum(-1, keepdims=True) / dh + cfg.rms_eps) * w.g_q[carry[sl]]
+                Kh = Kh / np.sqrt((Kh ** 2).sum(-1, keepdims=True) / dh + cfg.rms_eps) * w.g_k[carry[sl]]
+            S = scale * Qh @ Kh.T
+            S[np.triu_indices(N, 1)] = -np.inf
+            P = np.exp(S - S.max(axis=1, keepdims=True))
+            P /= P.sum(axis=1, keepdims=True)
+            want[b, :, sl] = P @ Vv[b, :, sl]
+    assert np.allclose(z[..., carry], c, rtol=0, atol=0)
+    assert np.allclose(z[..., scratch], want, rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ pin: W_q = 0 -> running mean of the values
+
+def test_zero_query_projection_gives_uniform_mean():
+    rng = np.random.default_rng(4)
+    cfg, w = rand_layer(rng, 16, 2, 24, alpha=0.7)
+    w.w_q = np.zeros_like(w.w_q)
+    w.w_down = np.zeros_like(w.w_down)            # z_i = x_i + alpha W_o c_i exposes c_i
+    x = rng.standard_normal((2, 12, 16))
+    z, k, v = layer_seq(cfg, w, x)
+    n = x / np.sqrt((x ** 2).mean(-1, keepdims=True) + cfg.rms_eps)
+    vt = n @ w.w_v.T
+    for i in range(12):
+        c = (v[:, :i].sum(axis=1) + vt[:, i]) / (i + 1)
+        assert np.allclose((z[:, i] - x[:, i]) / 0.7, c @ w.w_o.T, rtol=1e-11, atol=1e-12)
+
+
+# ------------------------------------------------------------------ pin: N = 1 and the MLP branch in closed form
+
+@pytest.mark.parametrize("pre", [False, True])
+def test_single_token_elementwise_mlp_closed_form(pre):
+    # N = 1 with W_v = 0: a = 0, h = x.  W_up = I, W_down = I (d_ff = d) make the MLP the
+    # elementwise GELU, so z = x + alpha GELU(RMS(x)) with RMS(x) = sqrt(D) x/||x|| (eps = 0).
+    d, alpha = 8, 0.6
+    rng = np.random.default_rng(5)
+    cfg = RTConfig(d, 2, 4, d, norm_flags=(NORM_PRE if pre else 0) | NORM_QK, rms_eps=0.0, residual_scale=alpha)
+    w = RTWeights(rng.standard_normal((d, d)), rng.standard_normal((d, d)), np.zeros((d, d)),
+                  rng.standard_normal((d, d)), np.eye(d), np.eye(d))
+    x = rng.standard_normal((1, 1, d))
+    z, _, v = layer_seq(cfg, w, x)
+    u = x[0, 0] * (math.sqrt(d) / math.sqrt(sum(t * t for t in x[0, 0]))) if pre else x[0, 0]
+    want = [xi + alpha * ui * 0.5 * (1.0 + math.erf(ui / math.sqrt(2.0))) for xi, ui in zip(x[0, 0], u)]
+    assert np.allclose(z[0, 0], want, rtol=1e-13, atol=1e-14)
+    assert np.all(v == 0)
+
+
+def test_single_token_attention_is_the_temporary_value():
+    # N = 1: softmax over one entry is 1, so c_1 = v~_1 whatever the logit is.
+    rng = np.random.default_rng(6)
+    cfg, w = rand_layer(rng, 12, 3, 20, alpha=0.9, gains=True)
+    w.w_down = np.zeros_like(w.w_down)
+    x = rng.standard_normal((3, 1, 12))
+    z, _, _ = layer_seq(cfg, w, x)
+    n = x[:, 0] * w.g_attn / np.sqrt((x[:, 0] ** 2).mean(-1, keepdims=True) + cfg.rms_eps)
+    assert np.allclose(z[:, 0], x[:, 0] + 0.9 * (n @ w.w_v.T) @ w.w_o.T, rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ pin: blocked == sequential, any block size / order
+
+@pytest.mark.parametrize("N", [1, 2, 7, 16, 21])
+def test_blocked_equals_sequential_for_every_block_size(N):
+    rng = np.random.default_rng(7)
+    cfg, w = rand_layer(rng, 16, 2, 24, alpha=0.8, gains=True)
+    x = rng.standard_normal((2, N, 16))
+    ref = layer_seq(cfg, w, x)
+    for leaf in [1, 2, 3, 4, 5, 8, 16, 32]:
+        got = layer_blk(cfg, w, x, leaf=leaf)
+        for a, b in zip(got, ref):
+            assert np.allclose(a, b, rtol=1e-11, atol=1e-12), (N, leaf)
+
+
+def test_result_is_invariant_to_tiling_order():
+    rng = np.random.default_rng(8)
+    cfg, w = rand_layer(rng, 8, 2, 12, scale=1.0)        # scale 1.0 = the literal Attn of Sec. 2
+    x = rng.standard_normal((1, 13, 8))
+    ref = layer_seq(cfg, w, x)
+    for leaf in (1, 4):
+        for self_first in (True, False):
+            for eager in (False, True):
+                got = layer_blk(cfg, w, x, leaf=leaf, self_first=self_first, eager_leaf=eager)
+                for a, b in zip(got, ref):
+                    assert np.allclose(a, b, rtol=1e-11, atol=1e-12)
+
+
+@pytest.mark.parametrize("flags", [0, NORM_PRE, NORM_QK, NORM_PRE | NORM_QK | NORM_QK_FULL,
+                                   NORM_PRE | NORM_QK | NORM_SKIP_Z])
+def test_blocked_equals_sequential_for_every_norm_flag(flags):
+    rng = np.random.default_rng(9)
+    cfg, w = rand_layer(rng, 8, 2, 12, flags=flags, alpha=0.5, gains=True)
+    x = 0.5 * rng.standard_normal((1, 10, 8))
+    ref = layer_seq(cfg, w, x)
+    got = layer_blk(cfg, w, x, leaf=4)
+    for a, b in zip(got, ref):
+        assert np.allclose(a, b, rtol=1e-11, atol=1e-12)
+
+
+# ------------------------------------------------------------------ pin: fixed point, decode, causality
+
+def test_fixed_point_verifier_accepts_truth_and_rejects_perturbation():
+    rng = np.random.default_rng(10)
+    cfg, w = rand_layer(rng, 16, 2, 24)
+    x = rng.standard_normal((2, 9, 16))
+    z, k, v = layer_seq(cfg, w, x)
+    z2, k2, v2 = layer_fixed_point(cfg, w, x, z)
+    assert np.allclose(z2, z, rtol=1e-11, atol=1e-12)
+    assert np.allclose(k2, k, rtol=1e-11, atol=1e-12) and np.allclose(v2, v, rtol=1e-11, atol=1e-12)
+    zp = z.copy(); zp[0, 3, 5] += 1e-3
+    z3, _, _ = layer_fixed_point(cfg, w, x, zp)
+    assert np.abs(z3 - zp).max() > 1e-5            # a wrong claim is not a fixed point
+    assert np.allclose(z3[:, :4], z[:, :4], rtol=1e-11, atol=1e-12)   # positions before the fault are unaffected
+
+
+def test_prefill_then_decode_equals_longer_prefill():
+    rng = np.random.default_rng(11)
+    cfg, w = rand_layer(rng, 16, 2, 24, alpha=0.7)
+    x = rng.standard_normal((2, 8, 16))
+    z, k, v = layer_seq(cfg, w, x)
+    zs, ks, vs = layer_seq(cfg, w, x[:, :7])
+    kc = np.zeros_like(k); vc = np.zeros_like(v)
+    kc[:, :7], vc[:, :7] = ks, vs
+    zn = layer_decode(cfg, w, x[:, 7], kc, vc, 7)
+    assert np.allclose(zn, z[:, 7], rtol=1e-11, atol=1e-12)
+    assert np.allclose(kc, k, rtol=1e-11, atol=1e-12) and np.allclose(vc, v, rtol=1e-11, atol=1e-12)
+
+
+def test_causality_prefix_and_batch_independence():
+    rng = np.random.default_rng(12)
+    cfg, w = rand_layer(rng, 16, 2, 24)
+    x = rng.standard_normal((3, 10, 16))
+    z, k, v = layer_seq(cfg, w, x)
+    x2 = x.copy(); x2[:, 6:] = rng.standard_normal((3, 4, 16))
+    z2, k2, v2 = layer_seq(cfg, w, x2)
+    assert np.array_equal(z2[:, :6], z[:, :6]) and np.array_equal(k2[:, :6], k[:, :6])
+    assert not np.allclose(z2[:, 6:], z[:, 6:])
+    zp, _, _ = layer_seq(cfg, w, x[:, :6])
+    assert np.allclose(zp, z[:, :6], rtol=1e-13, atol=1e-14)
+    perm = [2, 0, 1]
+    zq, _, _ = layer_seq(cfg, w, x[perm])
+    assert np.allclose(zq, z[perm], rtol=1e-13, atol=1e-14)
+    # later positions do read earlier persistent pairs (the recurrence is real)
+    x3 = x.copy(); x3[:, 0] += 0.5
+    z3, _, _ = layer_seq(cfg, w, x3)
+    assert np.abs(z3[:, 9] - z[:, 9]).max() > 1e-6
+
+
+def test_stack_prefill_then_decode_and_tied_head():
+    rng = np.random.default_rng(13)
+    d, V, L = 16, 37, 3
+    cfg = RTConfig(d, 2, 8, 24, residual_scale=1 / math.sqrt(L))
+    layers = [rand_layer(rng, d, 2, 24)[1] for _ in range(L)]
+    emb = rng.standard_normal((V, d))
+    ids = rng.integers(0, V, size=(2, 6))
+    hid, logits, caches = stack_prefill(cfg, layers, emb, None, ids)
+    # the stack is the composition of single layers fed with each other's z
+    xcur = emb[ids]
+    for wl in layers:
+        xcur, _, _ = layer_blk(cfg, wl, xcur, leaf=2)
+    assert np.allclose(hid, xcur, rtol=1e-10, atol=1e-11)
+    last = hid[:, -1]
+    want = (last * math.sqrt(d) / np.sqrt((last ** 2).sum(-1, keepdims=True) + d * cfg.rms_eps)) @ emb.T
+    assert np.allclose(logits, want, rtol=1e-11, atol=1e-12)
+    # prefill of 5 tokens + one decode step == prefill of 6
+    hid5, _, c5 = stack_prefill(cfg, layers, emb, None, ids[:, :5])
+    caches5 = []
+    for (k, v) in c5:
+        kk = np.zeros((2, 6, d)); vv = np.zeros((2, 6, d))
+        kk[:, :5], vv[:, :5] = k, v
+        caches5.append((kk, vv))
+    lg = stack_decode(cfg, layers, emb, None, ids[:, 5], caches5, 5)
+    assert np.allclose(lg, logits, rtol=1e-10, atol=1e-11)
+    for (k, v), (kk, vv) in zip(caches, caches5):
+        assert np.allclose(k, kk, rtol=1e-10, atol=1e-11) and np.allclose(v, vv, rtol=1e-10, atol=1e-11)
