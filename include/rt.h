@@ -1,0 +1,152 @@
+/*
+ * rt.h -- C ABI of the B200 (sm_100a) Recurrent Transformer prefill library.
+ *
+ * The library evaluates, exactly, the Recurrent Transformer (RT) layer of Sec. 2.2 of
+ * "The Recurrent Transformer" (arXiv 2604.21215): at position i the query and a TEMPORARY
+ * key/value pair come from the layer input x_i, the attention runs over the PERSISTENT
+ * pairs of earlier positions plus that temporary pair, the layer output is
+ *     z_i = x_i + alpha (a_i + MLP[RMS(x_i + alpha a_i)]),
+ * and the persistent pair of position i is computed from z_i (Eqs. 1-2).  Prefill uses
+ * the exact tiling schedule of Sec. 5 / Algorithms 1-2 (App. C).
+ *
+ * Conventions for every entry point
+ *  - All tensor pointers are DEVICE pointers unless a comment says "host".  The caller owns
+ *    every buffer, including the workspace; the library allocates no device memory and keeps
+ *    no global mutable state.  Pointers must be 16-byte aligned.
+ *  - Storage type (rt_dtype) applies to x, weights, gains, z, the K/V caches and the
+ *    embedding.  Accumulation is always fp32.  Logits are fp32.
+ *  - Weights are row-major [out, in]:  y = W u.
+ *  - x and z are [B, N, d_model] row-major.  z must not alias x.
+ *  - A K/V cache is POSITION-MAJOR [N_max, B, d_model] (Sec. 6, "Cache locality"): row t
+ *    holds the persistent pair of position t for all sequences.  Prefill writes rows [0, N),
+ *    decode appends row pos.  All sequences of a batch share the same length.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
+ *    stream) and return without synchronising.  Argument, shape, alignment and workspace
+ *    errors are detected on the host before anything is enqueued.  A device-side bounded
+ *    wait that runs out is recorded in the workspace and read with rt_get_status after the
+ *    caller has synchronised the stream.  Nothing aborts, traps or throws.
+ *  - The same workspace must not be used by two calls that overlap in time.
+ */
+#ifndef RT_B200_H
+#define RT_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RT_OK = 0,
+  RT_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, misaligned pointer, inconsistent shape */
+  RT_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for (e.g. head_dim != 64) */
+  RT_ERR_WORKSPACE = 3,     /* workspace_bytes < rt_workspace_bytes(...) */
+  RT_ERR_CUDA = 4,          /* a CUDA runtime call failed (launch, attribute query) */
+  RT_ERR_TIMEOUT = 5        /* a bounded device-side wait expired; outputs are invalid */
+} rt_status;
+
+typedef enum { RT_F32 = 0, RT_BF16 = 1 } rt_dtype;
+
+/* RT_SCHED_TILED: Algorithm 1's schedule at leaf granularity (each K/V row is streamed
+ * O(log N) times).  RT_SCHED_NAIVE: the token-sequential evaluation of Sec. 5 ("What makes
+ * naive evaluation slow"): every position reads its whole prefix, Theta(N^2) traffic; kept
+ * as the comparison path.  Both give the same result up to rounding order. */
+typedef enum { RT_SCHED_TILED = 0, RT_SCHED_NAIVE = 1 } rt_sched;
+
+enum {                      /* rt_config.norm_flags */
+  RT_NORM_PRE = 1,          /* RMS(x_i), RMS before the MLP and RMS(z_i) are applied (Sec. 2.2) */
+  RT_NORM_QK = 2,           /* qkRMS on queries and keys, per head */
+  RT_NORM_QK_FULL = 4,      /* qkRMS over the full width: oracle only, RT_ERR_UNSUPPORTED here */
+  RT_NORM_SKIP_Z = 8        /* persistent pair from z_i itself (the RMSNorm-ablation appendix) */
+};
+
+typedef struct {
+  int32_t d_model, n_heads, head_dim, d_ff; /* n_heads*head_dim == d_model; head_dim must be 64 */
+  int32_t dtype;            /* rt_dtype */
+  int32_t sched;            /* rt_sched */
+  int32_t leaf;             /* leaf block size of the tiled schedule: power of two in [16, 256]; 0 = auto */
+  int32_t norm_flags;       /* RT_NORM_*; the paper's layer is RT_NORM_PRE | RT_NORM_QK */
+  float rms_eps;            /* added to the mean square inside the root (the paper gives none; 1e-6) */
+  float softmax_scale;      /* logits = scale * <q, k>.  Sec. 2's Attn has scale 1; 1/sqrt(head_dim) is customary */
+  float residual_scale;     /* alpha = 1/sqrt(L) of Sec. 2; 1 for a single layer */
+} rt_config;
+
+typedef struct {            /* device pointers; read-only */
+  const void *w_q, *w_k, *w_v, *w_o;   /* [d_model, d_model]; w_k and w_v serve the temporary AND the persistent pair */
+  const void *w_up;                    /* [d_ff, d_model] */
+  const void *w_down;                  /* [d_model, d_ff]   MLP(u) = w_down GELU(w_up u), exact (erf) GELU, no biases */
+  const void *g_attn, *g_mlp, *g_kv;   /* [d_model] RMS gains of RMS(x), the MLP pre-norm and RMS(z); NULL = ones; g_kv NULL = g_attn */
+  const void *g_q, *g_k;               /* [d_model] qkRMS gains; NULL = ones */
+} rt_layer_weights;
+
+/* Bytes of workspace a call with these shapes needs (N = positions per call: the prefill
+ * length, or 1 for decode).  n_layers >= 1.  Returns 0 for an invalid configuration. */
+size_t rt_workspace_bytes(const rt_config *cfg, int32_t B, int32_t N, int32_t n_layers);
+
+/* One RT layer over x[B,N,d] (Sec. 2.2; Algorithm 1).  Writes z[B,N,d] and rows [0,N) of
+ * k_cache / v_cache [N_max,B,d] (Eqs. 1-2).  N_max >= N. */
+rt_status rt_layer_prefill(const rt_config *cfg, const rt_layer_weights *w,
+                           const void *x, int32_t B, int32_t N,
+                           void *z, void *k_cache, void *v_cache, int32_t N_max,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* A stack of n_layers RT layers with token embedding and tied output head:
+ * x^0 = emb[ids], x^l = layer_l(x^{l-1}), logits = emb . RMS_{g_final}(x^L at the last position).
+ * `layers`, `k_caches`, `v_caches` are HOST arrays of n_layers entries (device pointers inside).
+ * hidden [B,N,d] (storage type) and logits_last [B,vocab] (fp32) may each be NULL. */
+rt_status rt_stack_prefill(const rt_config *cfg, int32_t n_layers, const rt_layer_weights *layers,
+                           const void *emb, const void *g_final, int32_t vocab,
+                           const int32_t *ids, int32_t B, int32_t N,
+                           void *hidden, float *logits_last,
+                           void *const *k_caches, void *const *v_caches, int32_t N_max,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* One decode step of the stack: one new token id per sequence at position `pos` (the
+ * number of positions already in the caches).  A forward pass of RT is a sequence of such
+ * steps (Sec. 5), so this equals prefill of pos+1 tokens at its last position.  Appends row
+ * pos to every cache; writes logits [B,vocab] (fp32). */
+rt_status rt_decode_step(const rt_config *cfg, int32_t n_layers, const rt_layer_weights *layers,
+                         const void *emb, const void *g_final, int32_t vocab,
+                         const int32_t *ids, int32_t B, int32_t pos,
+                         float *logits, void *const *k_caches, void *const *v_caches, int32_t N_max,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Decode step of a single layer: x[B,d] at position pos -> z[B,d]; appends row pos. */
+rt_status rt_layer_decode_step(const rt_config *cfg, const rt_layer_weights *w,
+                               const void *x, int32_t B, int32_t pos,
+                               void *z, void *k_cache, void *v_cache, int32_t N_max,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* After the caller synchronised the stream: copies the device status word of `workspace`
+ * back (a blocking 4-byte copy) and returns it (RT_OK or RT_ERR_TIMEOUT). */
+rt_status rt_get_status(const void *workspace);
+
+const char *rt_status_string(rt_status s);
+
+/* Modelled work of the schedule that a prefill with these shapes runs (pure host function,
+ * no CUDA call): bytes each launch is designed to move between HBM and the SMs, and flops.
+ * vocab = 0 for a single layer fed with x. */
+typedef struct {
+  uint64_t model_bytes_read, model_bytes_written;
+  uint64_t flops_tile;      /* cross-block tiles: 4 * queries * keys * head_dim per head */
+  uint64_t flops_leaf;      /* per-token chain and in-leaf attention */
+  uint64_t flops_gemm;      /* Q / temporary K,V projection (and the head, if vocab > 0) */
+  uint64_t kv_bytes_read;   /* part of model_bytes_read: K/V cache rows streamed by the cross tiles (or, naive, by every position) */
+  uint64_t leaf_kv_bytes_l2; /* NOT in model_bytes_read: rows of a position's own leaf, re-read while still L2-resident */
+  uint64_t n_tiles, n_leaves;
+} rt_counters;
+rt_status rt_plan_counters(const rt_config *cfg, int32_t B, int32_t N, int32_t n_layers, int32_t vocab,
+                           rt_counters *out);
+
+/* The cross tiles of the tiled schedule for a length-N prefill with leaf size `leaf`
+ * (Algorithm 1 applied to blocks of `leaf` positions), 0-based half-open:
+ * tile i lets queries [q0,q1) attend to the pairs [k0,k1) right after position k1-1 is
+ * revealed.  Writes up to `cap` entries of 4 int32 each to `out` (host) and returns the
+ * number of tiles (call with cap = 0 to size the buffer).  Pure host function. */
+int32_t rt_plan_tiles(int32_t N, int32_t leaf, int32_t *out, int32_t cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RT_B200_H */

@@ -261,11 +261,12 @@ def layer_blk(cfg: RTConfig, w: RTWeights, x: np.ndarray, leaf: int = 1,
 
 # ----------------------------------------------------------------------------- O-fix
 
-def layer_fixed_point(cfg: RTConfig, w: RTWeights, x: np.ndarray, z_claim: np.ndarray):
+def layer_fixed_point(cfg: RTConfig, w: RTWeights, x: np.ndarray, z_claim: np.ndarray, rows=None):
     """One parallel sweep (Sec. 6, activation checkpointing): rebuild every persistent pair
     from the claimed outputs z, then recompute every a_i and z_i independently of each other.
     Because z_i depends only on z_j, j < i, the true z is the unique fixed point: the claim
-    is right iff the returned z' equals it.  Returns z', k, v with (k, v) rebuilt from z_claim."""
+    is right iff the returned z' equals it.  Returns z', k, v with (k, v) rebuilt from z_claim.
+    rows: optional iterable of positions to recompute (the other rows of z' stay zero)."""
     x = np.asarray(x, dtype=np.float64)
     zc = np.asarray(z_claim, dtype=np.float64)
     B, N, d = x.shape
@@ -276,7 +277,7 @@ def layer_fixed_point(cfg: RTConfig, w: RTWeights, x: np.ndarray, z_claim: np.nd
     q, kt, vt = _temp_qkv(x, w, cfg)                     # all positions at once
     z2 = np.zeros_like(x)
     for b in range(B):
-        for i in range(N):
+        for i in (range(N) if rows is None else rows):
             c = np.zeros(d)
             for h in range(H):
                 sl = slice(h * dh, (h + 1) * dh)

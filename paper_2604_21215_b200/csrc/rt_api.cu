@@ -1,0 +1,356 @@
+// C ABI of the library (see include/rt.h): argument checks, workspace layout, and the
+// schedule of Algorithm 1 at leaf granularity -- solve a leaf, then let the next query block
+// attend to the block of pairs that just became complete.
+#include <math.h>
+#include <string.h>
+
+#include "rt_kernels.h"
+
+using namespace rt;
+
+namespace {
+
+constexpr int kMaxChunks = 32;
+constexpr int kAutoLeaf = 64;
+
+struct WsLayout {
+  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, hid0, hid1, total;
+};
+
+size_t esize_of(int dtype) { return dtype == RT_BF16 ? 2 : 4; }
+
+bool config_ok(const rt_config* c) {
+  if (!c) return false;
+  if (c->d_model <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->d_ff <= 0) return false;
+  if ((long long)c->n_heads * c->head_dim != c->d_model) return false;
+  if (c->dtype != RT_F32 && c->dtype != RT_BF16) return false;
+  if (c->sched != RT_SCHED_TILED && c->sched != RT_SCHED_NAIVE) return false;
+  if (c->leaf != 0 && (c->leaf < 16 || c->leaf > 256 || (c->leaf & (c->leaf - 1)))) return false;
+  if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
+  if (c->norm_flags & ~15) return false;
+  return true;
+}
+
+rt_status config_supported(const rt_config* c, int B) {
+  if (c->head_dim != kHeadDim) return RT_ERR_UNSUPPORTED;
+  if (c->norm_flags & RT_NORM_QK_FULL) return RT_ERR_UNSUPPORTED;
+  if (c->d_ff % 4) return RT_ERR_UNSUPPORTED;
+  if (B > 64) return RT_ERR_UNSUPPORTED;                 // the per-token chain is written for small batches
+  return RT_OK;
+}
+
+WsLayout ws_layout(const rt_config* c, int B, int N) {
+  WsLayout L;
+  const size_t e = esize_of(c->dtype), d = c->d_model, H = c->n_heads, f = c->d_ff;
+  const size_t tok = (size_t)B * N;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes, 256); return at; };
+  L.sync = take(sizeof(SyncArea));
+  L.q = take(tok * d * e);
+  L.kt = take(tok * d * e);
+  L.vt = take(tok * d * e);
+  L.n = take(tok * d * e);
+  L.st_o = take(tok * d * 4);
+  L.st_m = take(tok * H * 4);
+  L.st_l = take(tok * H * 4);
+  L.ex_h = take((size_t)B * d * 4);
+  L.ex_g = take((size_t)B * f * 4);
+  L.ex_z = take((size_t)B * d * 4);
+  L.ex_k = take((size_t)B * d * 4);
+  L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
+  L.hid0 = take(tok * d * e);
+  L.hid1 = take(tok * d * e);
+  L.total = o;
+  return L;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+bool weights_ok(const rt_layer_weights* w) {
+  if (!w) return false;
+  const void* req[] = {w->w_q, w->w_k, w->w_v, w->w_o, w->w_up, w->w_down};
+  for (const void* p : req) if (!p || !aligned16(p)) return false;
+  const void* opt[] = {w->g_attn, w->g_mlp, w->g_kv, w->g_q, w->g_k};
+  for (const void* p : opt) if (p && !aligned16(p)) return false;
+  return true;
+}
+
+int leaf_size(const rt_config* c) { return c->leaf ? c->leaf : kAutoLeaf; }
+
+// One layer on position-major scratch; x / z given with explicit strides.
+rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x, long long x_bs, long long x_ts,
+                    void* z, long long z_bs, long long z_ts, int B, int n_rows, int pos0, void* k_cache,
+                    void* v_cache, unsigned char* ws, const WsLayout& L, cudaStream_t s) {
+  // n_rows positions starting at cache position pos0 (prefill: pos0 = 0; decode: n_rows = 1)
+  const float scale_log2 = c->softmax_scale * kLog2e;
+  PrepassParams pp;
+  memset(&pp, 0, sizeof(pp));
+  pp.B = B; pp.N = n_rows; pp.d = c->d_model; pp.H = c->n_heads;
+  pp.norm_flags = c->norm_flags; pp.eps = c->rms_eps; pp.scale_log2 = scale_log2;
+  pp.x = x; pp.x_bs = x_bs; pp.x_ts = x_ts;
+  pp.w_q = w->w_q; pp.w_k = w->w_k; pp.w_v = w->w_v;
+  pp.g_attn = w->g_attn; pp.g_q = w->g_q; pp.g_k = w->g_k;
+  pp.n = ws + L.n; pp.q = ws + L.q; pp.kt = ws + L.kt; pp.vt = ws + L.vt;
+  pp.st_o = (float*)(ws + L.st_o); pp.st_m = (float*)(ws + L.st_m); pp.st_l = (float*)(ws + L.st_l);
+  if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
+
+  LeafLaunch ll;
+  if (leaf_plan(c->dtype, B, c->d_model, c->d_ff, &ll) != cudaSuccess) return RT_ERR_CUDA;
+  LeafParams lp;
+  memset(&lp, 0, sizeof(lp));
+  lp.B = B; lp.d = c->d_model; lp.H = c->n_heads; lp.dff = c->d_ff;
+  lp.norm_flags = c->norm_flags; lp.eps = c->rms_eps; lp.scale_log2 = scale_log2; lp.alpha = c->residual_scale;
+  lp.w_o = w->w_o; lp.w_up = w->w_up; lp.w_down = w->w_down; lp.w_k = w->w_k; lp.w_v = w->w_v;
+  lp.g_mlp = w->g_mlp; lp.g_kv = w->g_kv ? w->g_kv : w->g_attn; lp.g_k = w->g_k;
+  lp.x = x; lp.x_bs = x_bs; lp.x_ts = x_ts;
+  lp.z = z; lp.z_bs = z_bs; lp.z_ts = z_ts;
+  lp.k_cache = k_cache; lp.v_cache = v_cache;
+  lp.q = ws + L.q;
+  lp.st_o = pp.st_o; lp.st_m = pp.st_m; lp.st_l = pp.st_l;
+  lp.row_off = pos0;
+  lp.ex_h = (float*)(ws + L.ex_h); lp.ex_g = (float*)(ws + L.ex_g);
+  lp.ex_z = (float*)(ws + L.ex_z); lp.ex_k = (float*)(ws + L.ex_k);
+  lp.ex_part = (float*)(ws + L.ex_part);
+  lp.max_chunks = kMaxChunks;
+  lp.sync = (SyncArea*)(ws + L.sync);
+
+  if (c->sched == RT_SCHED_NAIVE || pos0 > 0) {
+    // token-sequential: every position reads its whole prefix from the cache
+    lp.t0 = pos0; lp.t1 = pos0 + n_rows; lp.attn_begin = 0;
+    if (leaf_launch(c->dtype, lp, ll, s) != cudaSuccess) return RT_ERR_CUDA;
+    return RT_OK;
+  }
+  TileParams tp;
+  memset(&tp, 0, sizeof(tp));
+  tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2;
+  tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
+  tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
+  const int Lf = leaf_size(c), N = n_rows;
+  for (int s0 = 0; s0 < N; s0 += Lf) {
+    const int e0 = s0 + Lf < N ? s0 + Lf : N;
+    lp.t0 = s0; lp.t1 = e0; lp.attn_begin = s0;
+    if (leaf_launch(c->dtype, lp, ll, s) != cudaSuccess) return RT_ERR_CUDA;
+    if (e0 < N) {
+      const int P = e0 & -e0;                              // largest power of two dividing the block end
+      tp.q0 = e0; tp.q1 = e0 + P < N ? e0 + P : N; tp.k0 = e0 - P; tp.k1 = e0;
+      if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    }
+  }
+  return RT_OK;
+}
+
+rt_status common_checks(const rt_config* c, int B, int N, int n_layers, void* ws, size_t ws_bytes) {
+  if (!config_ok(c) || B <= 0 || N <= 0 || n_layers <= 0 || !ws || !aligned16(ws)) return RT_ERR_INVALID_ARG;
+  const rt_status st = config_supported(c, B);
+  if (st != RT_OK) return st;
+  if (ws_bytes < ws_layout(c, B, N).total) return RT_ERR_WORKSPACE;
+  return RT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rt_workspace_bytes(const rt_config* cfg, int32_t B, int32_t N, int32_t n_layers) {
+  if (!config_ok(cfg) || B <= 0 || N <= 0 || n_layers <= 0) return 0;
+  return ws_layout(cfg, B, N).total;
+}
+
+rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t N,
+                           void* z, void* k_cache, void* v_cache, int32_t N_max, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+  rt_status st = common_checks(cfg, B, N, 1, workspace, workspace_bytes);
+  if (st != RT_OK) return st;
+  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || x == z || N_max < N) return RT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(z) || !aligned16(k_cache) || !aligned16(v_cache)) return RT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)workspace;
+  const WsLayout L = ws_layout(cfg, B, N);
+  if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  const long long d = cfg->d_model;
+  return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, ws, L, s);
+}
+
+rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t pos,
+                               void* z, void* k_cache, void* v_cache, int32_t N_max, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+  rt_status st = common_checks(cfg, B, 1, 1, workspace, workspace_bytes);
+  if (st != RT_OK) return st;
+  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || x == z || pos < 0 || pos >= N_max) return RT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(z) || !aligned16(k_cache) || !aligned16(v_cache)) return RT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)workspace;
+  const WsLayout L = ws_layout(cfg, B, 1);
+  if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  const long long d = cfg->d_model;
+  rt_config c = *cfg;
+  c.sched = RT_SCHED_NAIVE;
+  return run_layer(&c, w, x, d, d, z, d, d, B, 1, pos, k_cache, v_cache, ws, L, s);
+}
+
+rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_layer_weights* layers, const void* emb,
+                           const void* g_final, int32_t vocab, const int32_t* ids, int32_t B, int32_t N, void* hidden,
+                           float* logits_last, void* const* k_caches, void* const* v_caches, int32_t N_max,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  rt_status st = common_checks(cfg, B, N, n_layers, workspace, workspace_bytes);
+  if (st != RT_OK) return st;
+  if (!layers || !emb || !ids || !k_caches || !v_caches || vocab <= 0 || N_max < N) return RT_ERR_INVALID_ARG;
+  if (!aligned16(emb) || (hidden && !aligned16(hidden)) || (g_final && !aligned16(g_final))) return RT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!weights_ok(&layers[l]) || !k_caches[l] || !v_caches[l] || !aligned16(k_caches[l]) || !aligned16(v_caches[l]))
+      return RT_ERR_INVALID_ARG;
+  }
+  if ((size_t)B * cfg->d_model * 4 > 200 * 1024) return RT_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)workspace;
+  const WsLayout L = ws_layout(cfg, B, N);
+  if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  const long long d = cfg->d_model;
+  void* bufs[2] = {ws + L.hid0, ws + L.hid1};
+  if (embed_launch(cfg->dtype, emb, ids, B, N, (int)d, vocab, bufs[0], s) != cudaSuccess) return RT_ERR_CUDA;
+  const void* cur = bufs[0];
+  for (int l = 0; l < n_layers; ++l) {
+    void* out = (l == n_layers - 1 && hidden) ? hidden : bufs[(l + 1) & 1];
+    st = run_layer(cfg, &layers[l], cur, (long long)N * d, d, out, (long long)N * d, d, B, N, 0, k_caches[l],
+                   v_caches[l], ws, L, s);
+    if (st != RT_OK) return st;
+    cur = out;
+  }
+  if (logits_last) {
+    const unsigned char* last = (const unsigned char*)cur + (size_t)(N - 1) * d * esize_of(cfg->dtype);
+    if (head_launch(cfg->dtype, emb, g_final, last, (long long)N * d, B, (int)d, vocab, cfg->norm_flags, cfg->rms_eps,
+                    logits_last, s) != cudaSuccess)
+      return RT_ERR_CUDA;
+  }
+  return RT_OK;
+}
+
+rt_status rt_decode_step(const rt_config* cfg, int32_t n_layers, const rt_layer_weights* layers, const void* emb,
+                         const void* g_final, int32_t vocab, const int32_t* ids, int32_t B, int32_t pos, float* logits,
+                         void* const* k_caches, void* const* v_caches, int32_t N_max, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  rt_status st = common_checks(cfg, B, 1, n_layers, workspace, workspace_bytes);
+  if (st != RT_OK) return st;
+  if (!layers || !emb || !ids || !logits || !k_caches || !v_caches || vocab <= 0 || pos < 0 || pos >= N_max)
+    return RT_ERR_INVALID_ARG;
+  if (!aligned16(emb) || (g_final && !aligned16(g_final))) return RT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!weights_ok(&layers[l]) || !k_caches[l] || !v_caches[l] || !aligned16(k_caches[l]) || !aligned16(v_caches[l]))
+      return RT_ERR_INVALID_ARG;
+  }
+  if ((size_t)B * cfg->d_model * 4 > 200 * 1024) return RT_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)workspace;
+  const WsLayout L = ws_layout(cfg, B, 1);
+  if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  const long long d = cfg->d_model;
+  rt_config c = *cfg;
+  c.sched = RT_SCHED_NAIVE;
+  void* bufs[2] = {ws + L.hid0, ws + L.hid1};
+  if (embed_launch(c.dtype, emb, ids, B, 1, (int)d, vocab, bufs[0], s) != cudaSuccess) return RT_ERR_CUDA;
+  const void* cur = bufs[0];
+  for (int l = 0; l < n_layers; ++l) {
+    void* out = bufs[(l + 1) & 1];
+    st = run_layer(&c, &layers[l], cur, d, d, out, d, d, B, 1, pos, k_caches[l], v_caches[l], ws, L, s);
+    if (st != RT_OK) return st;
+    cur = out;
+  }
+  if (head_launch(c.dtype, emb, g_final, cur, d, B, (int)d, vocab, c.norm_flags, c.rms_eps, logits, s) != cudaSuccess)
+    return RT_ERR_CUDA;
+  return RT_OK;
+}
+
+rt_status rt_get_status(const void* workspace) {
+  if (!workspace) return RT_ERR_INVALID_ARG;
+  int st = 0;
+  if (cudaMemcpy(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RT_ERR_CUDA;
+  return (rt_status)st;
+}
+
+const char* rt_status_string(rt_status s) {
+  switch (s) {
+    case RT_OK: return "ok";
+    case RT_ERR_INVALID_ARG: return "invalid argument";
+    case RT_ERR_UNSUPPORTED: return "unsupported configuration";
+    case RT_ERR_WORKSPACE: return "workspace too small";
+    case RT_ERR_CUDA: return "CUDA runtime error";
+    case RT_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int32_t rt_plan_tiles(int32_t N, int32_t leaf, int32_t* out, int32_t cap) {
+  if (N <= 0 || leaf <= 0) return 0;
+  int32_t n = 0;
+  for (int s0 = 0; s0 < N; s0 += leaf) {
+    const int e0 = s0 + leaf < N ? s0 + leaf : N;
+    if (e0 >= N) break;
+    const int blocks = e0 / leaf;
+    const int P = leaf * (blocks & -blocks);
+    if (out && n < cap) {
+      out[4 * n + 0] = e0; out[4 * n + 1] = e0 + P < N ? e0 + P : N;
+      out[4 * n + 2] = e0 - P; out[4 * n + 3] = e0;
+    }
+    ++n;
+  }
+  return n;
+}
+
+rt_status rt_plan_counters(const rt_config* cfg, int32_t B, int32_t N, int32_t n_layers, int32_t vocab,
+                           rt_counters* out) {
+  if (!config_ok(cfg) || B <= 0 || N <= 0 || n_layers <= 0 || vocab < 0 || !out) return RT_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  const uint64_t e = esize_of(cfg->dtype), d = cfg->d_model, H = cfg->n_heads, f = cfg->d_ff, b = B, n = N;
+  const uint64_t tok = b * n;
+  uint64_t rd = 0, wr = 0, kv = 0, kv_leaf = 0, fl_tile = 0, fl_leaf = 0, tiles = 0, leaves = 0;
+  // pre-pass: RMS (x -> n), projection (n, W -> q, k~, v~), state seed (q, k~, v~ -> o, m, l)
+  rd += tok * d * e + tok * d * e + 3 * d * d * e + 3 * tok * d * e;
+  wr += tok * d * e + 3 * tok * d * e + tok * d * 4 + 2 * tok * H * 4;
+  const uint64_t chain_w = (3 * d * d + 2 * d * f) * e;
+  // per token: q row, carried state, x row in; z, k, v rows out
+  rd += tok * d * e + tok * (d + 2 * H) * 4 + tok * d * e;
+  wr += 3 * tok * d * e;
+  fl_leaf += tok * 2 * (3 * d * d + 2 * d * f);
+  if (cfg->sched == RT_SCHED_NAIVE) {
+    leaves = 1;
+    rd += chain_w;
+    kv = b * d * e * n * (n - 1);                        // K and V rows of the whole prefix, every position
+    fl_leaf += 4 * d * b * (n * (n - 1) / 2);
+  } else {
+    const uint64_t Lf = leaf_size(cfg);
+    for (uint64_t s0 = 0; s0 < n; s0 += Lf) {
+      const uint64_t e0 = s0 + Lf < n ? s0 + Lf : n, len = e0 - s0;
+      ++leaves;
+      rd += chain_w;                                     // each launch stages its weight rows once
+      kv_leaf += 2 * b * d * e * (len * (len - 1) / 2);  // in-leaf pairs: written a few steps earlier, L2-resident
+      fl_leaf += 4 * d * b * (len * (len - 1) / 2);
+      if (e0 < n) {
+        const uint64_t P = e0 & (~e0 + 1);
+        const uint64_t nq = (e0 + P < n ? e0 + P : n) - e0;
+        ++tiles;
+        kv += 2 * P * b * d * e;
+        rd += nq * b * d * e + nq * b * (d + 2 * H) * 4;
+        wr += nq * b * (d + 2 * H) * 4;
+        fl_tile += 4 * nq * P * d * b;
+      }
+    }
+  }
+  rd += kv;
+  out->model_bytes_read = rd * n_layers;
+  out->model_bytes_written = wr * n_layers;
+  out->kv_bytes_read = kv * n_layers;
+  out->leaf_kv_bytes_l2 = kv_leaf * n_layers;
+  out->flops_tile = fl_tile * n_layers;
+  out->flops_leaf = fl_leaf * n_layers;
+  out->flops_gemm = tok * 2 * d * 3 * d * n_layers;
+  out->n_tiles = tiles * n_layers;
+  out->n_leaves = leaves * n_layers;
+  if (vocab > 0) {
+    out->model_bytes_read += tok * d * e + (uint64_t)vocab * d * e;
+    out->model_bytes_written += tok * d * e + b * (uint64_t)vocab * 4;
+    out->flops_gemm += 2 * b * d * (uint64_t)vocab;
+  }
+  return RT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,70 @@
+// Host-side launch interface of the RT kernels (internal; the public ABI is include/rt.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "rt_common.cuh"
+
+namespace rt {
+
+// Everything the per-token chain needs.  Position-major buffers are [row, B, d] with
+// row = t - row_off (prefill: row_off = 0; decode: the single row 0 stands for position pos).
+struct LeafParams {
+  int B, d, H, dff;
+  int norm_flags;
+  float eps, scale_log2, alpha;
+  const void *w_o, *w_up, *w_down, *w_k, *w_v;   // storage type
+  const void *g_mlp, *g_kv, *g_k;                // storage type or NULL
+  const void* x;  long long x_bs, x_ts;          // x[b, t, :] = x + b*x_bs + (t-row_off)*x_ts   (elements)
+  void* z;        long long z_bs, z_ts;
+  void *k_cache, *v_cache;                       // [N_max, B, d] storage type
+  const void* q;                                 // [rows, B, d] storage type
+  float *st_o, *st_m, *st_l;                     // online-softmax state: o [rows,B,d], m,l [rows,B,H] (m in log2 units)
+  int t0, t1;                                    // positions [t0, t1) are processed by this launch
+  int row_off;
+  int attn_begin;                                // first key position the in-launch attention covers (0 = whole prefix)
+  float *ex_h, *ex_g, *ex_z, *ex_k;              // exchange vectors [B,d], [B,dff], [B,d], [B,d]
+  float* ex_part;                                // partial attention states [B*H, max_chunks, 66]
+  int max_chunks;
+  int weights_in_smem;                           // 1: each CTA keeps its weight rows in shared memory
+  SyncArea* sync;
+};
+
+struct LeafLaunch { int grid, block; size_t smem; int weights_in_smem; };
+
+// Chooses grid / shared memory for the leaf kernel on the current device.
+cudaError_t leaf_plan(int dtype, int B, int d, int dff, LeafLaunch* out);
+cudaError_t leaf_launch(int dtype, const LeafParams& p, const LeafLaunch& l, cudaStream_t s);
+
+// Pre-pass (Algorithm 1, line 1 and the temporary pair of line 7, hoisted out of the loop).
+struct PrepassParams {
+  int B, N, d, H;
+  int norm_flags;
+  float eps, scale_log2;
+  const void* x; long long x_bs, x_ts;           // x[b, r, :]
+  const void *w_q, *w_k, *w_v, *g_attn, *g_q, *g_k;
+  void* n;                                       // [N*B, d] normalised input (scratch)
+  void *q, *kt, *vt;                             // [N, B, d]
+  float *st_o, *st_m, *st_l;
+};
+cudaError_t prepass_launch(int dtype, const PrepassParams& p, cudaStream_t s);
+
+// Cross-block tile (Algorithm 2 on a [q0,q1) x [k0,k1) block for every sequence and head).
+struct TileParams {
+  int B, d, H;
+  float scale_log2;
+  const void* q;                                 // [N, B, d]
+  const void *k_cache, *v_cache;                 // [N_max, B, d]
+  float *st_o, *st_m, *st_l;
+  int q0, q1, k0, k1;
+};
+cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s);
+
+// Stack helpers.
+cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,
+                         void* x, cudaStream_t s);
+cudaError_t head_launch(int dtype, const void* emb, const void* g_final, const void* hidden, long long h_bs,
+                        int B, int d, int vocab, int norm_flags, float eps, float* logits, cudaStream_t s);
+
+}  // namespace rt

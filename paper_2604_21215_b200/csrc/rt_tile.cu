@@ -1,0 +1,99 @@
+// Cross-block tile: Algorithm 2 (UpdateTile) applied to queries [q0,q1) against the revealed
+// pairs [k0,k1), for every sequence and head, with the running stats (m, l, o) carried in
+// fp32 between tiles.  This file holds the SIMT version (fp32 mode, and any shape the
+// tensor-core version does not take).  m is kept in log2 units: p = 2^(s*log2e*<q,k> - m).
+#include "rt_kernels.h"
+
+namespace rt {
+
+constexpr int kTQ = 16;    // query rows per CTA
+constexpr int kTK = 32;    // keys per shared-memory chunk
+
+template <typename T>
+__global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
+  __shared__ float Qs[kTQ][kHeadDim];
+  __shared__ float Ks[kTK][kHeadDim + 1];
+  __shared__ float Vs[kTK][kHeadDim];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
+  const int qb = p.q0 + blockIdx.x * kTQ;
+  const T* Q = reinterpret_cast<const T*>(p.q);
+  const T* Kc = reinterpret_cast<const T*>(p.k_cache);
+  const T* Vc = reinterpret_cast<const T*>(p.v_cache);
+  const size_t col0 = (size_t)b * p.d + h * kHeadDim;
+  const size_t rstride = (size_t)p.B * p.d;
+
+  for (int i = tid; i < kTQ * kHeadDim; i += 128) {
+    const int r = i / kHeadDim, e = i % kHeadDim;
+    Qs[r][e] = (qb + r < p.q1) ? to_f(Q[(size_t)(qb + r) * rstride + col0 + e]) : 0.f;
+  }
+  // each warp owns 4 query rows; lane holds dims lane and lane+32 of o
+  float m[4], l[4], oa[4], ob[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int qi = qb + warp * 4 + i;
+    if (qi < p.q1) {
+      const size_t sidx = (size_t)qi * p.B + b;
+      m[i] = p.st_m[sidx * p.H + h];
+      l[i] = p.st_l[sidx * p.H + h];
+      oa[i] = p.st_o[sidx * p.d + h * kHeadDim + lane];
+      ob[i] = p.st_o[sidx * p.d + h * kHeadDim + lane + 32];
+    } else { m[i] = 0.f; l[i] = 0.f; oa[i] = 0.f; ob[i] = 0.f; }
+  }
+  for (int kb = p.k0; kb < p.k1; kb += kTK) {
+    __syncthreads();
+    for (int i = tid; i < kTK * kHeadDim; i += 128) {
+      const int r = i / kHeadDim, e = i % kHeadDim;
+      const bool ok = kb + r < p.k1;
+      Ks[r][e] = ok ? to_f(Kc[(size_t)(kb + r) * rstride + col0 + e]) : 0.f;
+      Vs[r][e] = ok ? to_f(Vc[(size_t)(kb + r) * rstride + col0 + e]) : 0.f;
+    }
+    __syncthreads();
+    const bool valid = kb + lane < p.k1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int qr = warp * 4 + i;
+      float s = 0.f;
+#pragma unroll 16
+      for (int e = 0; e < kHeadDim; ++e) s += Qs[qr][e] * Ks[lane][e];
+      const float s2 = valid ? s * p.scale_log2 : -INFINITY;
+      const float m_new = fmaxf(m[i], warp_max(s2));
+      const float pj = valid ? exp2f(s2 - m_new) : 0.f;
+      const float corr = exp2f(m[i] - m_new);
+      l[i] = l[i] * corr + warp_sum(pj);
+      float a = oa[i] * corr, c = ob[i] * corr;
+#pragma unroll 8
+      for (int jj = 0; jj < kTK; ++jj) {
+        const float pw = __shfl_sync(0xffffffffu, pj, jj);
+        a += pw * Vs[jj][lane];
+        c += pw * Vs[jj][lane + 32];
+      }
+      oa[i] = a; ob[i] = c; m[i] = m_new;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int qi = qb + warp * 4 + i;
+    if (qi < p.q1) {
+      const size_t sidx = (size_t)qi * p.B + b;
+      if (lane == 0) { p.st_m[sidx * p.H + h] = m[i]; p.st_l[sidx * p.H + h] = l[i]; }
+      p.st_o[sidx * p.d + h * kHeadDim + lane] = oa[i];
+      p.st_o[sidx * p.d + h * kHeadDim + lane + 32] = ob[i];
+    }
+  }
+}
+
+cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  const int nq = p.q1 - p.q0;
+  if (nq <= 0 || p.k1 <= p.k0) return cudaSuccess;
+  dim3 grid(ceil_div(nq, kTQ), p.B * p.H);
+  if (dtype == RT_BF16) tile_simt_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(p);
+  else tile_simt_kernel<float><<<grid, 128, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  return tile_simt_launch(dtype, p, s);
+}
+
+}  // namespace rt

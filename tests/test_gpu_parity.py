@@ -1,0 +1,183 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle on identical seeded
+inputs.  Error metric per output tensor T in {z, K, V, logits}: max|T_gpu - T_ref| / max|T_ref|.
+Bounds: 1e-4 in fp32 mode, 2e-2 for bf16 storage with fp32 accumulation."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def rel_err(got, ref):
+    return float(np.abs(got - ref).max() / np.abs(ref).max())
+
+
+def make_case(d, H, dff, B, N, dtype, seed, gains=False):
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("case", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=seed)
+    lw = data["layers"][0]
+    if gains:
+        rng = np.random.default_rng(seed + 1)
+        for g in ("g_attn", "g_mlp", "g_kv", "g_q", "g_k"):
+            lw[g] = inputs.round_to(1.0 + 0.2 * rng.standard_normal(d), dtype)
+    return data["x"], lw
+
+
+def run_layer(x, lw, d, H, dff, dtype, **kw):
+    from paper_2604_21215_b200 import rt
+    layer = rt.Layer(d, H, dff, dtype=dtype, **kw)
+    layer.set_weights(lw)
+    return layer, layer.prefill(x)
+
+
+def oracle_layer(x, lw, d, H, dff, **kw):
+    from oracle import RTConfig, RTWeights, layer_seq
+    cfg = RTConfig(d, H, 64, dff, **kw)
+    return layer_seq(cfg, RTWeights(**lw), x)
+
+
+def check(got, ref, tol, what):
+    for name, g, r in zip(("z", "k", "v"), got, ref):
+        e = rel_err(g, r)
+        assert np.isfinite(g).all(), f"{what}: non-finite {name}"
+        assert e <= tol, f"{what}: {name} rel err {e:.3e} > {tol}"
+
+
+# ---------------------------------------------------------------- config 1 (fp32), tiled and naive
+
+@pytest.mark.parametrize("sched,leaf", [("tiled", 16), ("tiled", 32), ("tiled", 64), ("naive", 0)])
+def test_c1_fp32_matches_oracle(sched, leaf):
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.WORKLOADS["c1"]
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    ref = oracle_layer(data["x"], lw, wl.d_model, wl.n_heads, wl.d_ff)
+    _, got = run_layer(data["x"], lw, wl.d_model, wl.n_heads, wl.d_ff, "f32", sched=sched, leaf=leaf)
+    check(got, ref, TOL["f32"], f"c1 {sched} leaf={leaf}")
+
+
+# ---------------------------------------------------------------- ragged sizes, batches, flags (fp32, small)
+
+@pytest.mark.parametrize("B,N,leaf", [(1, 1, 16), (2, 2, 16), (3, 17, 16), (5, 65, 32), (2, 100, 16), (9, 33, 16),
+                                      (1, 130, 64), (16, 40, 16)])
+def test_ragged_sizes_fp32(B, N, leaf):
+    d, H, dff = 128, 2, 256
+    x, lw = make_case(d, H, dff, B, N, "f32", seed=100 + N)
+    ref = oracle_layer(x, lw, d, H, dff)
+    _, got = run_layer(x, lw, d, H, dff, "f32", leaf=leaf)
+    check(got, ref, TOL["f32"], f"B={B} N={N} leaf={leaf}")
+    _, got_n = run_layer(x, lw, d, H, dff, "f32", sched="naive")
+    check(got_n, ref, TOL["f32"], f"naive B={B} N={N}")
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 3 | 8])
+def test_norm_flags_gains_scale_alpha_fp32(flags):
+    d, H, dff, B, N = 192, 3, 320, 2, 50
+    x, lw = make_case(d, H, dff, B, N, "f32", seed=200 + flags, gains=True)
+    x = 0.5 * x
+    kw = dict(norm_flags=flags, softmax_scale=(1.0 if flags & 2 else 0.05), residual_scale=0.6, rms_eps=1e-5)
+    ref = oracle_layer(x, lw, d, H, dff, **kw)
+    _, got = run_layer(x, lw, d, H, dff, "f32", leaf=16, **kw)
+    check(got, ref, 2e-4 if flags & 2 else 1e-4, f"flags={flags}")
+
+
+def test_qk_full_width_is_reported_unsupported():
+    from paper_2604_21215_b200 import rt
+    x, lw = make_case(128, 2, 256, 1, 8, "f32", seed=5)
+    with pytest.raises(rt.RtError) as ei:
+        run_layer(x, lw, 128, 2, 256, "f32", norm_flags=7)
+    assert ei.value.status == rt.RT_ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------- bf16 storage, several tiles and a ragged tail
+
+@pytest.mark.parametrize("B,N,leaf,sched", [(4, 200, 32, "tiled"), (8, 300, 64, "tiled"), (3, 150, 16, "naive"),
+                                            (16, 96, 32, "tiled")])
+def test_bf16_small_matches_oracle(B, N, leaf, sched):
+    d, H, dff = 256, 4, 1024
+    x, lw = make_case(d, H, dff, B, N, "bf16", seed=300 + N)
+    ref = oracle_layer(x, lw, d, H, dff)
+    _, got = run_layer(x, lw, d, H, dff, "bf16", leaf=leaf, sched=sched)
+    check(got, ref, TOL["bf16"], f"bf16 B={B} N={N} leaf={leaf} {sched}")
+
+
+# ---------------------------------------------------------------- decode == one more prefill position
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_prefill_then_decode_matches_oracle(dtype):
+    d, H, dff, B, N = 128, 2, 256, 3, 41
+    x, lw = make_case(d, H, dff, B, N + 2, dtype, seed=400)
+    ref = oracle_layer(x, lw, d, H, dff)
+    from paper_2604_21215_b200 import rt
+    layer = rt.Layer(d, H, dff, dtype=dtype, leaf=16)
+    layer.set_weights(lw)
+    got = layer.prefill(x[:, :N], N_max=N + 2)
+    check(got, tuple(r[:, :N] for r in ref), TOL[dtype], "prefill part")
+    for step in range(2):
+        zn = layer.decode(x[:, N + step], N + step)
+        assert rel_err(zn, ref[0][:, N + step]) <= TOL[dtype]
+    import torch
+    k = layer.k_cache.permute(1, 0, 2).to(torch.float64).cpu().numpy()
+    v = layer.v_cache.permute(1, 0, 2).to(torch.float64).cpu().numpy()
+    assert rel_err(k, ref[1]) <= TOL[dtype] and rel_err(v, ref[2]) <= TOL[dtype]
+
+
+# ---------------------------------------------------------------- stack: embedding, layers, tied head, decode
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stack_prefill_and_decode_match_oracle(dtype):
+    from oracle import RTConfig, RTWeights, stack_prefill, stack_decode
+    from paper_2604_21215_b200 import inputs, rt
+    L, d, H, dff, V, B, N = 3, 128, 2, 256, 500, 3, 37
+    wl = inputs.Workload("stack", L, B, N + 1, d, H, dff, dtype, vocab=V, residual_scale=1 / np.sqrt(L))
+    data = inputs.make_inputs(wl, seed=500)
+    ocfg = RTConfig(d, H, 64, dff, residual_scale=wl.residual_scale)
+    ow = [RTWeights(**lw) for lw in data["layers"]]
+    hid_ref, logits_ref, caches_ref = stack_prefill(ocfg, ow, data["emb"], None, data["ids"])
+    st = rt.Stack(L, d, H, dff, V, dtype=dtype, leaf=16, residual_scale=wl.residual_scale)
+    st.set_weights(data["layers"], data["emb"])
+    hid, logits = st.prefill(data["ids"])
+    tol = TOL[dtype]
+    assert rel_err(hid, hid_ref) <= tol and rel_err(logits, logits_ref) <= tol
+    for (k, v), (kr, vr) in zip(st.caches_numpy(N + 1), caches_ref):
+        assert rel_err(k, kr) <= tol and rel_err(v, vr) <= tol
+    # prefill N, then one decode step, equals prefill N+1 at its last position
+    hid2, _ = st.prefill(data["ids"][:, :N], N_max=N + 1)
+    assert rel_err(hid2, hid_ref[:, :N]) <= tol
+    lg = st.decode(data["ids"][:, N], N)
+    assert rel_err(lg, logits_ref) <= tol
+
+
+# ---------------------------------------------------------------- full-size configs in the benchmark's launch configuration
+
+def test_c2_full_size_bf16_matches_oracle():
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.WORKLOADS["c2"]
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    ref = oracle_layer(data["x"], lw, wl.d_model, wl.n_heads, wl.d_ff)
+    _, got = run_layer(data["x"], lw, wl.d_model, wl.n_heads, wl.d_ff, "bf16")
+    check(got, ref, TOL["bf16"], "c2")
+
+
+def test_c3_full_size_bf16_prefix_and_fixed_point():
+    # The oracle replays the first 384 positions (causality makes them independent of the
+    # rest); the whole length is checked with the fixed-point property on one sequence: feeding
+    # the GPU's z back through one parallel sweep of the oracle must reproduce it.
+    from oracle import RTConfig, RTWeights, layer_fixed_point
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.WORKLOADS["c3"]
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    _, got = run_layer(data["x"], lw, wl.d_model, wl.n_heads, wl.d_ff, "bf16")
+    ref = oracle_layer(data["x"][:, :384], lw, wl.d_model, wl.n_heads, wl.d_ff)
+    check(tuple(g[:, :384] for g in got), ref, TOL["bf16"], "c3 prefix")
+    cfg = RTConfig(wl.d_model, wl.n_heads, 64, wl.d_ff)
+    sel = slice(5, 6)
+    rows = np.r_[0:64, 2040:2056, 4032:4096]     # positions sampled for the re-computation
+    z2, k2, v2 = layer_fixed_point(cfg, RTWeights(**lw), data["x"][sel], got[0][sel], rows=rows)
+    zmax = np.abs(got[0][sel]).max()
+    assert np.abs(z2[:, rows] - got[0][sel][:, rows]).max() / zmax <= TOL["bf16"]
+    assert rel_err(got[1][sel], k2) <= TOL["bf16"] and rel_err(got[2][sel], v2) <= TOL["bf16"]
