@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the RT prefill hot path on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5_N<len>] [--sched tiled|naive]
+    python bench.py --impl reference ...          # times the fp64 CPU oracle instead
+
+A step is one pass of the whole hot path (pre-pass, every leaf launch, every cross tile) over
+one batch.  `value` counts tokens/s with inputs resident in HBM; `e2e` runs the same call with
+the batch coming from pinned host memory and the layer output read back, copies inside the
+timed region.  With N > 1 (torchrun) every rank runs an independent replica of the workload on
+its own GPU -- the path shards over the batch only, so there is no collective on the data
+path -- and the line reports all ranks' tokens over the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rt_prefill_tokens_per_s"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# DRAM bytes (read + write) per leaf launch from the ncu captures summarised under profiles/.
+NCU_LEAF_TRAFFIC = {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def get_workload(name):
+    from paper_2604_21215_b200 import inputs
+    if name.startswith("c5_N"):
+        return inputs.sweep(int(name[4:]))
+    return inputs.WORKLOADS[name]
+
+
+def config_dict(wl, sched, extra=None):
+    c = {"workload": wl.name, "n_layers": wl.n_layers, "B": wl.B, "N": wl.N, "d_model": wl.d_model,
+         "n_heads": wl.n_heads, "d_ff": wl.d_ff, "vocab": wl.vocab, "sched": sched,
+         "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ------------------------------------------------------------------------------------ oracle arm
+
+def oracle_sample(wl, data, n_pos):
+    """Runs the oracle, as it stands, on the first n_pos positions of the workload; returns seconds."""
+    from oracle import RTConfig, RTWeights, layer_seq, stack_prefill
+    cfg = RTConfig(wl.d_model, wl.n_heads, wl.head_dim, wl.d_ff, residual_scale=wl.residual_scale)
+    layers = [RTWeights(**lw) for lw in data["layers"]]
+    t0 = time.perf_counter()
+    if wl.vocab:
+        stack_prefill(cfg, layers, data["emb"], None, data["ids"][:, :n_pos])
+    else:
+        layer_seq(cfg, layers[0], data["x"][:, :n_pos])
+    return time.perf_counter() - t0
+
+
+def oracle_cores():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def sample_positions(wl):
+    # about 10-30 s of CPU work: the first positions of every sequence of the batch
+    n = 1024 if wl.d_model <= 768 else 512
+    if wl.n_layers > 1:
+        n = max(32, n // wl.n_layers)
+    return min(wl.N, n)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2604_21215_b200 import inputs
+    wl = get_workload(args.workload)
+    data = inputs.make_inputs(wl)
+    n_pos = sample_positions(wl)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(wl, data, min(n_pos, 64))
+    times = [oracle_sample(wl, data, n_pos) for _ in range(args.steps)]
+    tot = sum(times)
+    value = wl.B * n_pos * args.steps / tot
+    cores = oracle_cores()
+    sample = (f"fp64 oracle (numpy) on the first {n_pos} of {wl.N} positions of all {wl.B} sequences per step; "
+              "later positions cost more (longer prefixes), so the full workload would be slower per token")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(wl, "oracle", {"l2": "n/a (CPU)"}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------ CUDA arm
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_21215_b200 import inputs, rt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = get_workload(args.workload)
+    data = inputs.make_inputs(wl)
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    leaf_kw = {"leaf": args.leaf} if args.leaf else {}
+    stream = torch.cuda.current_stream(dev)
+
+    if wl.vocab:
+        model = rt.Stack(wl.n_layers, wl.d_model, wl.n_heads, wl.d_ff, wl.vocab, dtype=wl.dtype, device=str(dev),
+                         sched=args.sched, residual_scale=wl.residual_scale, **leaf_kw)
+        model.set_weights(data["layers"], data["emb"])
+        model.reserve(wl.B, wl.N)
+        host_in = torch.from_numpy(data["ids"]).pin_memory()
+        dev_in = host_in.to(dev)
+        dev_out = torch.empty((wl.B, wl.N, wl.d_model), dtype=tdt, device=dev)
+        logits = torch.empty((wl.B, wl.vocab), dtype=torch.float32, device=dev)
+        host_out = torch.empty((wl.B, wl.vocab), dtype=torch.float32).pin_memory()
+        call = lambda inp: model.prefill_device(inp, dev_out, logits)
+        result = logits
+    else:
+        model = rt.Layer(wl.d_model, wl.n_heads, wl.d_ff, dtype=wl.dtype, device=str(dev), sched=args.sched,
+                         residual_scale=wl.residual_scale, **leaf_kw)
+        model.set_weights(data["layers"][0])
+        model.reserve(wl.B, wl.N)
+        host_in = torch.from_numpy(data["x"]).to(tdt).pin_memory()
+        dev_in = host_in.to(dev)
+        dev_out = torch.empty((wl.B, wl.N, wl.d_model), dtype=tdt, device=dev)
+        host_out = torch.empty((wl.B, wl.N, wl.d_model), dtype=tdt).pin_memory()
+        call = lambda inp: model.prefill_device(inp, dev_out)
+        result = dev_out
+    dev_in2 = torch.empty_like(dev_in)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    tokens = wl.B * wl.N
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        """Each step bracketed by its own pair of CUDA events on the launching stream; L2 flushed between."""
+        evs = []
+        for _ in range(steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def e2e_step():
+        dev_in2.copy_(host_in, non_blocking=True)
+        call(dev_in2)
+        host_out.copy_(result, non_blocking=True)
+
+    for _ in range(max(args.warmup, 3)):
+        call(dev_in)
+    torch.cuda.synchronize(dev)
+    if model.status() != rt.RT_OK:
+        raise SystemExit("device status after warm-up: " + rt.rt_status_string(model.status()))
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    rt.rt_profile_enable(True)
+    rt.rt_profile_read()
+    wall0 = time.perf_counter()
+    ms = timed(lambda: call(dev_in), args.steps)
+    barrier()
+    wall = time.perf_counter() - wall0
+    prof = rt.rt_profile_read()
+    rt.rt_profile_enable(False)
+    total_ms = sum(ms)
+    # end to end: pinned host input -> device, the call, result -> pinned host
+    e2e_step(); torch.cuda.synchronize(dev)
+    barrier()
+    e2e_ms = timed(e2e_step, args.steps)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    e2e_total = sum(e2e_ms)
+    if model.status() != rt.RT_OK:
+        raise SystemExit("device status after the timed region: " + rt.rt_status_string(model.status()))
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total = float(t[0]), float(t[1])
+
+    if rank == 0:
+        counters = rt.rt_plan_counters(model.cfg, wl.B, wl.N, wl.n_layers, wl.vocab)
+        peaks = measured_peaks()
+        e = 2 if wl.dtype == "bf16" else 4
+        d, f, B = wl.d_model, wl.d_ff, wl.B
+        # dominant kernel: the leaf recurrence.  Algorithmic bytes per token step = the chain
+        # weights once (shared by the B sequences) + activation rows; per launch x the leaf length.
+        chain_w = (3 * d * d + 2 * d * f) * e
+        act = (7 * e + 4) * d * B
+        n_leaf = max(prof["leaf"]["launches"], 1)
+        tok_steps_per_launch = wl.N * wl.n_layers * args.steps / n_leaf
+        leaf_ms = prof["leaf"]["ms"] / n_leaf
+        alg_bytes = (chain_w + act) * tok_steps_per_launch
+        achieved = alg_bytes / (leaf_ms * 1e-3) / 1e9 if leaf_ms > 0 else 0.0
+        roofline = {"kernel": "leaf_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                    "traffic": NCU_LEAF_TRAFFIC.get(wl.name),
+                    "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": leaf_ms,
+                    "us_per_token_step": 1e3 * leaf_ms / max(tok_steps_per_launch, 1),
+                    "note": "weights stay in shared memory for a whole launch, so the kernel is bound by "
+                            "grid-barrier latency and shared-memory reads, not by HBM; the fraction is the "
+                            "effective weight+activation stream against the HBM copy peak"}
+        tile_ms = prof["tile"]["ms"]
+        tile_tflops = (counters["flops_tile"] * args.steps / (tile_ms * 1e-3) / 1e12) if tile_ms > 0 else None
+        n_pos = sample_positions(wl)
+        t_cpu = oracle_sample(wl, data, n_pos)
+        cpu = {"value": wl.B * n_pos / t_cpu, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle",
+               "sample": f"first {n_pos} of {wl.N} positions, all {wl.B} sequences, one run ({t_cpu:.1f} s)"}
+        launches = sum(v["launches"] for v in prof.values())
+        # the pre-pass group is three kernels, every other group one
+        gpu_launches = int(launches + 2 * prof["prepass"]["launches"])
+        h2d = host_in.numel() * host_in.element_size()
+        d2h = host_out.numel() * host_out.element_size()
+        line = {"metric": METRIC, "value": world * tokens * args.steps / (total_ms * 1e-3), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16/f32-accumulate" if wl.dtype == "bf16" else "f32",
+                "data": "synthetic", "config": config_dict(wl, args.sched, {"leaf": int(model.cfg.leaf) or 64,
+                                                                            "parallelism": f"replicas x{world}"}),
+                "clocks": clocks,
+                "e2e": {"value": world * tokens * args.steps / (e2e_total * 1e-3), "unit": UNIT,
+                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "gpu_launches": gpu_launches,
+                "roofline": roofline, "cpu_baseline": cpu,
+                "kernels": {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps}
+                            for k, v in prof.items()},
+                "tile_tflops": tile_tflops,
+                "model": {"hbm_bytes_per_step": counters["model_bytes_read"] + counters["model_bytes_written"],
+                          "kv_bytes_read_per_step": counters["kv_bytes_read"],
+                          "flops_tile": counters["flops_tile"], "flops_leaf": counters["flops_leaf"],
+                          "flops_gemm": counters["flops_gemm"]},
+                "wall_s_timed_region": wall}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--sched", default="tiled", choices=["tiled", "naive"])
+    ap.add_argument("--leaf", type=int, default=0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

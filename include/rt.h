@@ -139,6 +139,17 @@ typedef struct {
 rt_status rt_plan_counters(const rt_config *cfg, int32_t B, int32_t N, int32_t n_layers, int32_t vocab,
                            rt_counters *out);
 
+/* Per-kernel-class timing for benchmarks.  While enabled (a process-wide switch, off by
+ * default, and the one piece of global state in the library) every call brackets its launches
+ * with CUDA events on the caller's stream: class 0 = pre-pass, 1 = leaf recurrence launches,
+ * 2 = cross-block tiles, 3 = embedding / head.  rt_profile_read waits for the recorded events
+ * (so call it after the work was enqueued), returns the summed milliseconds and the number of
+ * bracketed launch groups per class since the last read, and forgets them.  The paper has no
+ * counterpart; its latency protocol (Sec. 6, "The setup") times whole layers only. */
+typedef struct { double ms[4]; uint64_t launches[4]; } rt_profile;
+rt_status rt_profile_enable(int32_t on);
+rt_status rt_profile_read(rt_profile *out);
+
 /* The cross tiles of the tiled schedule for a length-N prefill with leaf size `leaf`
  * (Algorithm 1 applied to blocks of `leaf` positions), 0-based half-open:
  * tile i lets queries [q0,q1) attend to the pairs [k0,k1) right after position k1-1 is

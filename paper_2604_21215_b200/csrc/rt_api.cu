@@ -4,6 +4,9 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+#include <vector>
+
 #include "rt_kernels.h"
 
 using namespace rt;
@@ -77,11 +80,42 @@ bool weights_ok(const rt_layer_weights* w) {
 
 int leaf_size(const rt_config* c) { return c->leaf ? c->leaf : kAutoLeaf; }
 
+// ---- optional per-kernel-class timing (rt_profile_enable / rt_profile_read) -----------------
+enum ProfClass { kProfPrepass = 0, kProfLeaf = 1, kProfTile = 2, kProfOther = 3, kProfClasses = 4 };
+struct ProfSpan { cudaEvent_t a, b; int cls; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+std::vector<ProfSpan> g_prof_spans;
+constexpr size_t kProfMaxSpans = 1u << 20;
+
+// Records an event pair around the launches issued inside its scope when profiling is on.
+struct ProfScope {
+  cudaStream_t s; int cls; cudaEvent_t a = nullptr, b = nullptr; bool on = false;
+  ProfScope(cudaStream_t s_, int cls_) : s(s_), cls(cls_) {
+    std::lock_guard<std::mutex> g(g_prof_mu);
+    if (!g_prof_on || g_prof_spans.size() >= kProfMaxSpans) return;
+    if (cudaEventCreate(&a) != cudaSuccess) return;
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
+    on = cudaEventRecord(a, s) == cudaSuccess;
+  }
+  ~ProfScope() {
+    if (!a) return;
+    if (on && cudaEventRecord(b, s) == cudaSuccess) {
+      std::lock_guard<std::mutex> g(g_prof_mu);
+      g_prof_spans.push_back({a, b, cls});
+    } else { cudaEventDestroy(a); cudaEventDestroy(b); }
+  }
+};
+
+// State of one API call: the stream and the barrier arrivals enqueued so far.
+struct CallCtx { cudaStream_t s; unsigned bar_base = 0; };
+
 // One layer on position-major scratch; x / z given with explicit strides.
 rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x, long long x_bs, long long x_ts,
                     void* z, long long z_bs, long long z_ts, int B, int n_rows, int pos0, void* k_cache,
-                    void* v_cache, unsigned char* ws, const WsLayout& L, cudaStream_t s) {
+                    void* v_cache, unsigned char* ws, const WsLayout& L, CallCtx& ctx) {
   // n_rows positions starting at cache position pos0 (prefill: pos0 = 0; decode: n_rows = 1)
+  cudaStream_t s = ctx.s;
   const float scale_log2 = c->softmax_scale * kLog2e;
   PrepassParams pp;
   memset(&pp, 0, sizeof(pp));
@@ -92,7 +126,10 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   pp.g_attn = w->g_attn; pp.g_q = w->g_q; pp.g_k = w->g_k;
   pp.n = ws + L.n; pp.q = ws + L.q; pp.kt = ws + L.kt; pp.vt = ws + L.vt;
   pp.st_o = (float*)(ws + L.st_o); pp.st_m = (float*)(ws + L.st_m); pp.st_l = (float*)(ws + L.st_l);
-  if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
+  {
+    ProfScope ps(s, kProfPrepass);
+    if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
+  }
 
   LeafLaunch ll;
   if (leaf_plan(c->dtype, B, c->d_model, c->d_ff, &ll) != cudaSuccess) return RT_ERR_CUDA;
@@ -114,11 +151,17 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   lp.max_chunks = kMaxChunks;
   lp.sync = (SyncArea*)(ws + L.sync);
 
+  auto leaf = [&](int t0, int t1, int attn_begin) -> bool {
+    lp.t0 = t0; lp.t1 = t1; lp.attn_begin = attn_begin; lp.bar_base = ctx.bar_base;
+    ProfScope ps(s, kProfLeaf);
+    if (leaf_launch(c->dtype, lp, ll, s) != cudaSuccess) return false;
+    ctx.bar_base += leaf_barrier_arrivals(t0, t1, ll.grid);
+    return true;
+  };
+
   if (c->sched == RT_SCHED_NAIVE || pos0 > 0) {
     // token-sequential: every position reads its whole prefix from the cache
-    lp.t0 = pos0; lp.t1 = pos0 + n_rows; lp.attn_begin = 0;
-    if (leaf_launch(c->dtype, lp, ll, s) != cudaSuccess) return RT_ERR_CUDA;
-    return RT_OK;
+    return leaf(pos0, pos0 + n_rows, 0) ? RT_OK : RT_ERR_CUDA;
   }
   TileParams tp;
   memset(&tp, 0, sizeof(tp));
@@ -128,11 +171,11 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   const int Lf = leaf_size(c), N = n_rows;
   for (int s0 = 0; s0 < N; s0 += Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
-    lp.t0 = s0; lp.t1 = e0; lp.attn_begin = s0;
-    if (leaf_launch(c->dtype, lp, ll, s) != cudaSuccess) return RT_ERR_CUDA;
+    if (!leaf(s0, e0, s0)) return RT_ERR_CUDA;
     if (e0 < N) {
       const int P = e0 & -e0;                              // largest power of two dividing the block end
       tp.q0 = e0; tp.q1 = e0 + P < N ? e0 + P : N; tp.k0 = e0 - P; tp.k1 = e0;
+      ProfScope ps(s, kProfTile);
       if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
     }
   }
@@ -168,7 +211,8 @@ rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, cons
   const WsLayout L = ws_layout(cfg, B, N);
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
-  return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, ws, L, s);
+  CallCtx ctx{s};
+  return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, ws, L, ctx);
 }
 
 rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t pos,
@@ -185,7 +229,8 @@ rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, 
   const long long d = cfg->d_model;
   rt_config c = *cfg;
   c.sched = RT_SCHED_NAIVE;
-  return run_layer(&c, w, x, d, d, z, d, d, B, 1, pos, k_cache, v_cache, ws, L, s);
+  CallCtx ctx{s};
+  return run_layer(&c, w, x, d, d, z, d, d, B, 1, pos, k_cache, v_cache, ws, L, ctx);
 }
 
 rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_layer_weights* layers, const void* emb,
@@ -207,16 +252,21 @@ rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_laye
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   void* bufs[2] = {ws + L.hid0, ws + L.hid1};
-  if (embed_launch(cfg->dtype, emb, ids, B, N, (int)d, vocab, bufs[0], s) != cudaSuccess) return RT_ERR_CUDA;
+  CallCtx ctx{s};
+  {
+    ProfScope ps(s, kProfOther);
+    if (embed_launch(cfg->dtype, emb, ids, B, N, (int)d, vocab, bufs[0], s) != cudaSuccess) return RT_ERR_CUDA;
+  }
   const void* cur = bufs[0];
   for (int l = 0; l < n_layers; ++l) {
     void* out = (l == n_layers - 1 && hidden) ? hidden : bufs[(l + 1) & 1];
     st = run_layer(cfg, &layers[l], cur, (long long)N * d, d, out, (long long)N * d, d, B, N, 0, k_caches[l],
-                   v_caches[l], ws, L, s);
+                   v_caches[l], ws, L, ctx);
     if (st != RT_OK) return st;
     cur = out;
   }
   if (logits_last) {
+    ProfScope ps(s, kProfOther);
     const unsigned char* last = (const unsigned char*)cur + (size_t)(N - 1) * d * esize_of(cfg->dtype);
     if (head_launch(cfg->dtype, emb, g_final, last, (long long)N * d, B, (int)d, vocab, cfg->norm_flags, cfg->rms_eps,
                     logits_last, s) != cudaSuccess)
@@ -247,11 +297,12 @@ rt_status rt_decode_step(const rt_config* cfg, int32_t n_layers, const rt_layer_
   rt_config c = *cfg;
   c.sched = RT_SCHED_NAIVE;
   void* bufs[2] = {ws + L.hid0, ws + L.hid1};
+  CallCtx ctx{s};
   if (embed_launch(c.dtype, emb, ids, B, 1, (int)d, vocab, bufs[0], s) != cudaSuccess) return RT_ERR_CUDA;
   const void* cur = bufs[0];
   for (int l = 0; l < n_layers; ++l) {
     void* out = bufs[(l + 1) & 1];
-    st = run_layer(&c, &layers[l], cur, d, d, out, d, d, B, 1, pos, k_caches[l], v_caches[l], ws, L, s);
+    st = run_layer(&c, &layers[l], cur, d, d, out, d, d, B, 1, pos, k_caches[l], v_caches[l], ws, L, ctx);
     if (st != RT_OK) return st;
     cur = out;
   }
@@ -265,6 +316,31 @@ rt_status rt_get_status(const void* workspace) {
   int st = 0;
   if (cudaMemcpy(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RT_ERR_CUDA;
   return (rt_status)st;
+}
+
+rt_status rt_profile_enable(int32_t on) {
+  std::lock_guard<std::mutex> g(g_prof_mu);
+  g_prof_on = on != 0;
+  return RT_OK;
+}
+
+rt_status rt_profile_read(rt_profile* out) {
+  if (!out) return RT_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  std::vector<ProfSpan> spans;
+  {
+    std::lock_guard<std::mutex> g(g_prof_mu);
+    spans.swap(g_prof_spans);
+  }
+  rt_status st = RT_OK;
+  for (const ProfSpan& sp : spans) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(sp.b) != cudaSuccess || cudaEventElapsedTime(&ms, sp.a, sp.b) != cudaSuccess) st = RT_ERR_CUDA;
+    else { out->ms[sp.cls] += ms; out->launches[sp.cls] += 1; }
+    cudaEventDestroy(sp.a);
+    cudaEventDestroy(sp.b);
+  }
+  return st;
 }
 
 const char* rt_status_string(rt_status s) {

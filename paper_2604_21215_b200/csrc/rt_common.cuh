@@ -15,7 +15,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct SyncArea {
   int status;               // rt_status written by a kernel whose bounded wait ran out
   unsigned int abort_flag;  // set together with status; every waiter leaves when it sees it
-  unsigned int bar_count;   // arrivals of the running cooperative kernel (zeroed by the host before a launch)
+  unsigned int bar_count;   // barrier arrivals since the start of the API call (zeroed once per call)
   unsigned int pad[61];
 };
 static_assert(sizeof(SyncArea) == 256, "SyncArea is one 256-byte block");
@@ -103,7 +103,7 @@ __device__ __forceinline__ void red_release_add_u32(unsigned* p, unsigned v) {
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 // Barrier over all CTAs of a cooperative launch.  `target` is this CTA's running arrival
-// target (starts at 0; the host zeroes bar_count before the launch).  Returns false when
+// target (starts at the arrivals counted before this launch).  Returns false when
 // the wait ran out or another CTA reported a failure: the caller must then return at once.
 __device__ __forceinline__ bool grid_barrier(SyncArea* s, unsigned& target, unsigned n_ctas, int* s_flag) {
   __syncthreads();

@@ -28,6 +28,8 @@ struct LeafParams {
   float* ex_part;                                // partial attention states [B*H, max_chunks, 66]
   int max_chunks;
   int weights_in_smem;                           // 1: each CTA keeps its weight rows in shared memory
+  unsigned bar_base;                             // arrivals counted by earlier launches of the same call (bar_count is
+                                                 // zeroed once per API call and only ever grows)
   SyncArea* sync;
 };
 
@@ -36,6 +38,8 @@ struct LeafLaunch { int grid, block; size_t smem; int weights_in_smem; };
 // Chooses grid / shared memory for the leaf kernel on the current device.
 cudaError_t leaf_plan(int dtype, int B, int d, int dff, LeafLaunch* out);
 cudaError_t leaf_launch(int dtype, const LeafParams& p, const LeafLaunch& l, cudaStream_t s);
+// Barrier arrivals one launch over [t0,t1) adds to bar_count.
+inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsigned)(t1 - t0) * 5u * (unsigned)grid; }
 
 // Pre-pass (Algorithm 1, line 1 and the temporary pair of line 7, hoisted out of the loop).
 struct PrepassParams {

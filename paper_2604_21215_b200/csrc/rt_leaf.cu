@@ -154,6 +154,8 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
   const int B = p.B, d = p.d, H = p.H, dff = p.dff;
+  // an earlier launch of this call gave up: its barrier count is short, do not wait on it
+  if (*reinterpret_cast<volatile unsigned*>(&p.sync->abort_flag)) return;
   const int d_lo = (int)((long long)d * cta / G), d_hi = (int)((long long)d * (cta + 1) / G);
   const int f_lo = (int)((long long)dff * cta / G), f_hi = (int)((long long)dff * (cta + 1) / G);
   const int nd = d_hi - d_lo, nf = f_hi - f_lo;
@@ -197,7 +199,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   T* kc = reinterpret_cast<T*>(p.k_cache);
   T* vc = reinterpret_cast<T*>(p.v_cache);
   const float inv_d = 1.0f / (float)d;
-  unsigned bar_target = 0;
+  unsigned bar_target = p.bar_base;
   const int n_bg = (B + NB - 1) / NB;
 
   for (int t = p.t0; t < p.t1; ++t) {
@@ -432,9 +434,6 @@ cudaError_t leaf_launch(int dtype, const LeafParams& p_in, const LeafLaunch& l, 
   LeafSmemLayout L = leaf_smem_layout(p.B, p.d, p.dff, l.grid, NB, esize);
   const void* fn = dtype == RT_BF16 ? leaf_fn<__nv_bfloat16>(NB) : leaf_fn<float>(NB);
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
-  if (e != cudaSuccess) return e;
-  // the barrier counter starts from zero in every launch
-  e = cudaMemsetAsync(&p.sync->bar_count, 0, sizeof(unsigned), s);
   if (e != cudaSuccess) return e;
   void* args[] = {(void*)&p, (void*)&L};
   return cudaLaunchCooperativeKernel(fn, dim3(l.grid), dim3(l.block), args, l.smem, s);

@@ -24,7 +24,8 @@ RT_SCHED_TILED, RT_SCHED_NAIVE = 0, 1
 RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
-           "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles")
+           "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
+           "rt_profile_enable", "rt_profile_read")
 
 
 class RtConfig(C.Structure):
@@ -41,6 +42,13 @@ class RtLayerWeights(C.Structure):
 class RtCounters(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("model_bytes_read", "model_bytes_written", "flops_tile", "flops_leaf",
                                            "flops_gemm", "kv_bytes_read", "leaf_kv_bytes_l2", "n_tiles", "n_leaves")]
+
+
+class RtProfile(C.Structure):
+    _fields_ = [("ms", C.c_double * 4), ("launches", C.c_uint64 * 4)]
+
+
+PROFILE_CLASSES = ("prepass", "leaf", "tile", "other")
 
 
 def _load():
@@ -72,6 +80,10 @@ def _load():
     lib.rt_plan_counters.argtypes = [C.POINTER(RtConfig), I, I, I, I, C.POINTER(RtCounters)]
     lib.rt_plan_tiles.restype = I
     lib.rt_plan_tiles.argtypes = [I, I, C.POINTER(I), I]
+    lib.rt_profile_enable.restype = C.c_int
+    lib.rt_profile_enable.argtypes = [I]
+    lib.rt_profile_read.restype = C.c_int
+    lib.rt_profile_read.argtypes = [C.POINTER(RtProfile)]
     return lib
 
 
@@ -136,6 +148,16 @@ def rt_plan_tiles(N: int, leaf: int) -> List[tuple]:
     buf = (C.c_int32 * (4 * max(n, 1)))()
     _lib.rt_plan_tiles(N, leaf, buf, n)
     return [tuple(buf[4 * i:4 * i + 4]) for i in range(n)]
+
+
+def rt_profile_enable(on: bool) -> None:
+    _check(_lib.rt_profile_enable(1 if on else 0), "rt_profile_enable")
+
+
+def rt_profile_read() -> Dict[str, Dict[str, float]]:
+    out = RtProfile()
+    _check(_lib.rt_profile_read(C.byref(out)), "rt_profile_read")
+    return {n: {"ms": float(out.ms[i]), "launches": int(out.launches[i])} for i, n in enumerate(PROFILE_CLASSES)}
 
 
 def make_config(d_model: int, n_heads: int, d_ff: int, dtype: str = "bf16", sched: str = "tiled", leaf: int = 0,
