@@ -17,7 +17,7 @@ constexpr int kMaxChunks = 32;
 constexpr int kAutoLeaf = 64;
 
 struct WsLayout {
-  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, hid0, hid1, total;
+  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, ll, ll_bytes, hid0, hid1, total;
 };
 
 size_t esize_of(int dtype) { return dtype == RT_BF16 ? 2 : 4; }
@@ -61,6 +61,9 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_z = take((size_t)B * d * 4);
   L.ex_k = take((size_t)B * d * 4);
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
+  // flag-carrying exchange words of the bf16 leaf kernel: c, h, z [B,d/2], g [B,dff/2], raw k|v [B,2d]
+  L.ll_bytes = (size_t)B * (3 * (d / 2) + f / 2 + 2 * d) * 8;
+  L.ll = take(L.ll_bytes);
   L.hid0 = take(tok * d * e);
   L.hid1 = take(tok * d * e);
   L.total = o;
@@ -108,7 +111,7 @@ struct ProfScope {
 };
 
 // State of one API call: the stream and the barrier arrivals enqueued so far.
-struct CallCtx { cudaStream_t s; unsigned bar_base = 0; };
+struct CallCtx { cudaStream_t s; unsigned bar_base = 0; unsigned seq_base = 0; };
 
 // One layer on position-major scratch; x / z given with explicit strides.
 rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x, long long x_bs, long long x_ts,
@@ -159,6 +162,25 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     return true;
   };
 
+  // bf16 tiled prefill takes the tensor-core leaf kernel when the shape fits it
+  LeafMmaLaunch ml;
+  const bool use_mma = c->dtype == RT_BF16 && c->sched == RT_SCHED_TILED && pos0 == 0 &&
+                       leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
+  LeafMmaBuffers mb;
+  {
+    unsigned long long* w = (unsigned long long*)(ws + L.ll);
+    const size_t bd2 = (size_t)B * (c->d_model / 2);
+    mb.ll_c = w; mb.ll_h = w + bd2; mb.ll_z = w + 2 * bd2; mb.ll_g = w + 3 * bd2;
+    mb.ll_kv = mb.ll_g + (size_t)B * (c->d_ff / 2);
+  }
+  auto leaf_mma = [&](int t0, int t1) -> bool {
+    lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base;
+    ProfScope ps(s, kProfLeaf);
+    if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return false;
+    ctx.seq_base += (unsigned)(t1 - t0);
+    return true;
+  };
+
   if (c->sched == RT_SCHED_NAIVE || pos0 > 0) {
     // token-sequential: every position reads its whole prefix from the cache
     return leaf(pos0, pos0 + n_rows, 0) ? RT_OK : RT_ERR_CUDA;
@@ -168,10 +190,10 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2;
   tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
   tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
-  const int Lf = leaf_size(c), N = n_rows;
+  const int Lf = use_mma ? ml.leaf : leaf_size(c), N = n_rows;
   for (int s0 = 0; s0 < N; s0 += Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
-    if (!leaf(s0, e0, s0)) return RT_ERR_CUDA;
+    if (!(use_mma ? leaf_mma(s0, e0) : leaf(s0, e0, s0))) return RT_ERR_CUDA;
     if (e0 < N) {
       const int P = e0 & -e0;                              // largest power of two dividing the block end
       tp.q0 = e0; tp.q1 = e0 + P < N ? e0 + P : N; tp.k0 = e0 - P; tp.k1 = e0;
@@ -210,6 +232,7 @@ rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, cons
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, N);
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  if (cudaMemsetAsync(ws + L.ll, 0, L.ll_bytes, s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   CallCtx ctx{s};
   return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, ws, L, ctx);
@@ -226,6 +249,7 @@ rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, 
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, 1);
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  if (cudaMemsetAsync(ws + L.ll, 0, L.ll_bytes, s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   rt_config c = *cfg;
   c.sched = RT_SCHED_NAIVE;
@@ -250,6 +274,7 @@ rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_laye
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, N);
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  if (cudaMemsetAsync(ws + L.ll, 0, L.ll_bytes, s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   void* bufs[2] = {ws + L.hid0, ws + L.hid1};
   CallCtx ctx{s};
@@ -293,6 +318,7 @@ rt_status rt_decode_step(const rt_config* cfg, int32_t n_layers, const rt_layer_
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, 1);
   if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  if (cudaMemsetAsync(ws + L.ll, 0, L.ll_bytes, s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   rt_config c = *cfg;
   c.sched = RT_SCHED_NAIVE;

@@ -16,7 +16,11 @@ struct SyncArea {
   int status;               // rt_status written by a kernel whose bounded wait ran out
   unsigned int abort_flag;  // set together with status; every waiter leaves when it sees it
   unsigned int bar_count;   // barrier arrivals since the start of the API call (zeroed once per call)
-  unsigned int pad[61];
+  unsigned int pad0;
+  // time CTA 0 spent in each phase of the leaf kernel since the start of the API call, in ns:
+  // [2*i] = work of phase i (A..E), [2*i+1] = wait at the barrier that ends it
+  unsigned long long phase_ns[10];
+  unsigned int pad[40];
 };
 static_assert(sizeof(SyncArea) == 256, "SyncArea is one 256-byte block");
 

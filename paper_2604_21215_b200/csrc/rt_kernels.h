@@ -30,6 +30,7 @@ struct LeafParams {
   int weights_in_smem;                           // 1: each CTA keeps its weight rows in shared memory
   unsigned bar_base;                             // arrivals counted by earlier launches of the same call (bar_count is
                                                  // zeroed once per API call and only ever grows)
+  unsigned seq_base;                             // token steps enqueued before this launch in the same call (flag values)
   SyncArea* sync;
 };
 
@@ -40,6 +41,12 @@ cudaError_t leaf_plan(int dtype, int B, int d, int dff, LeafLaunch* out);
 cudaError_t leaf_launch(int dtype, const LeafParams& p, const LeafLaunch& l, cudaStream_t s);
 // Barrier arrivals one launch over [t0,t1) adds to bar_count.
 inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsigned)(t1 - t0) * 5u * (unsigned)grid; }
+
+// bf16 / tiled-schedule leaf kernel (tensor-core mat-vecs, flag-carrying exchange words).
+struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
+struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [B,d/2] x3, [B,dff/2], [B,2d] words
+bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out);
+cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s);
 
 // Pre-pass (Algorithm 1, line 1 and the temporary pair of line 7, hoisted out of the loop).
 struct PrepassParams {

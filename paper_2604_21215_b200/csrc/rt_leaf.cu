@@ -202,6 +202,24 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   unsigned bar_target = p.bar_base;
   const int n_bg = (B + NB - 1) / NB;
 
+  // phase timing by one thread of CTA 0 (two timer reads per phase)
+  const bool timing = (cta == 0 && tid == 0);
+  unsigned long long t_prev = timing ? globaltimer_ns() : 0ull, acc_ns[10];
+#pragma unroll
+  for (int i = 0; i < 10; ++i) acc_ns[i] = 0ull;
+#define LEAF_PHASE_END(i)                                                   \
+  {                                                                         \
+    unsigned long long t_a = timing ? globaltimer_ns() : 0ull;              \
+    const bool ok_ = grid_barrier(p.sync, bar_target, G, s_flag);           \
+    if (timing) {                                                           \
+      const unsigned long long t_b = globaltimer_ns();                      \
+      acc_ns[2 * (i)] += t_a - t_prev;                                      \
+      acc_ns[2 * (i) + 1] += t_b - t_a;                                     \
+      t_prev = t_b;                                                         \
+    }                                                                       \
+    if (!ok_) return;                                                       \
+  }
+
   for (int t = p.t0; t < p.t1; ++t) {
     const int row = t - p.row_off;
     // ---------------- phase A: partial attention over the pairs [attn_begin, t) ----------------
@@ -280,7 +298,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
         *reinterpret_cast<float2*>(part + 4 + 2 * lane) = make_float2(o0, o1);
       }
     }
-    if (!grid_barrier(p.sync, bar_target, G, s_flag)) return;
+    LEAF_PHASE_END(0);
 
     // ---------------- phase B: c_t = merged state / l, a = W_o c, h = x_t + alpha a ----------------
     for (int bg = 0; bg < n_bg; ++bg) {
@@ -317,7 +335,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
       cta_matvec<T, NB>(nd, d, [&](int r) { return Wo + (size_t)r * d; }, load_c, (const T*)nullptr, false, epi,
                         red, ssq_red, L.n_rg_max);
     }
-    if (!grid_barrier(p.sync, bar_target, G, s_flag)) return;
+    LEAF_PHASE_END(1);
 
     // ---------------- phase C: g = GELU(W_up RMS(h)) ----------------
     for (int bg = 0; bg < n_bg; ++bg) {
@@ -335,7 +353,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
       cta_matvec<T, NB>(nf, d, [&](int r) { return Wup + (size_t)r * d; }, load_h, pre ? g_mlp : (const T*)nullptr,
                         pre, epi, red, ssq_red, L.n_rg_max);
     }
-    if (!grid_barrier(p.sync, bar_target, G, s_flag)) return;
+    LEAF_PHASE_END(2);
 
     // ---------------- phase D: z_t = h + alpha W_down g ----------------
     for (int bg = 0; bg < n_bg; ++bg) {
@@ -355,7 +373,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
       cta_matvec<T, NB>(nd, dff, [&](int r) { return Wdn + (size_t)r * dff; }, load_g, (const T*)nullptr, false, epi,
                         red, ssq_red, L.n_rg_max);
     }
-    if (!grid_barrier(p.sync, bar_target, G, s_flag)) return;
+    LEAF_PHASE_END(3);
 
     // ---------------- phase E: raw k_t = W_k RMS(z_t), v_t = W_v RMS(z_t) ----------------
     for (int bg = 0; bg < n_bg; ++bg) {
@@ -375,8 +393,14 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
                         [&](int r) { return r < nd ? Wk + (size_t)r * d : Wv + (size_t)(r - nd) * d; }, load_z,
                         kv_norm ? g_kv : (const T*)nullptr, kv_norm, epi, red, ssq_red, L.n_rg_max);
     }
-    if (!grid_barrier(p.sync, bar_target, G, s_flag)) return;
+    LEAF_PHASE_END(4);
   }
+
+  if (timing) {
+#pragma unroll
+    for (int i = 0; i < 10; ++i) atomicAdd(&p.sync->phase_ns[i], acc_ns[i]);
+  }
+#undef LEAF_PHASE_END
 
   // ---------------- qkRMS and cache write of the last key of this launch ----------------
   if (p.t1 > p.t0) {

@@ -1,0 +1,566 @@
+// Leaf recurrence kernel, bf16 / tiled-schedule version: the sequential part of Algorithm 1
+// for the positions [t0, t1) of one leaf, all B <= 16 sequences at once.
+//
+// Same decomposition as the generic leaf kernel (one persistent CTA per SM, each CTA owning a
+// fixed slice of the output rows of W_o, W_up, W_down, W_k, W_v in shared memory), but built
+// for latency, because a token step is a chain of five all-to-all exchanges of small vectors:
+//   * exchange words carry their own validity flag.  Every published 64-bit word holds a
+//     payload (two bf16, or one fp32) and the 32-bit sequence number of the token step.
+//     A consumer polls the payload words themselves: one L2 round trip per exchange, no
+//     separate fence + counter + reload.  Flags are unique per step of an API call and the
+//     buffers are zeroed at the start of the call.
+//   * the mat-vec products run on the tensor cores as m16n8k16 MMAs with the B sequences as
+//     the M dimension (rows >= B are zero) and 8 weight rows as the N dimension, K split over
+//     the 8 MMA warps of the CTA and reduced through shared memory.  The fragments of the
+//     activations are exactly the polled words; weight fragments are 8-byte shared loads.
+//   * two extra warps per CTA do the in-leaf attention (Algorithm 2 with one key at a time):
+//     each owns one (sequence, head) pair and keeps the running stats (m, l, o) of every query
+//     of the leaf in shared memory.  When the pair (k_j, v_j) arrives it first finishes query
+//     j+1 (the only one on the critical path) and publishes c_{j+1} = o/l, and only then folds
+//     the new pair into the later queries of the leaf, while the rest of the chip is busy with
+//     the mat-vecs of step j+1.  These warps also apply qkRMS to k_j and write the caches.
+#include <cuda_bf16.h>
+
+#include "rt_kernels.h"
+
+namespace rt {
+
+constexpr int kMmaWarps = 8;
+constexpr int kMmaThreads = kMmaWarps * 32;
+constexpr int kAttnSlots = 2;
+constexpr int kLeafMmaThreads = kMmaThreads + 32 * kAttnSlots;
+constexpr int kNT = 4;                  // n-tiles (8 weight rows each) per pass
+constexpr int kQStride = kHeadDim + 2;  // bf16 elements per query row in shared memory
+constexpr int kOStride = kHeadDim + 1;  // floats per o row in shared memory
+
+struct LeafMmaLayout {
+  int max_nd, max_nf;          // weight rows per CTA (upper bounds): d-row matrices, W_up
+  int stride_d, stride_f;      // shared-memory row strides in elements (K + 16)
+  int lf;                      // leaf capacity of the attention state
+  size_t off_wo, off_wup, off_wdn, off_wk, off_wv, off_red, off_ssq, off_hown, off_attn, attn_bytes, total;
+};
+
+LeafMmaLayout leaf_mma_layout(int d, int dff, int grid, int lf, int slots) {
+  LeafMmaLayout L;
+  L.max_nd = 2 * ceil_div(d / 2, grid);
+  L.max_nf = 2 * ceil_div(dff / 2, grid);
+  L.stride_d = d + 16;
+  L.stride_f = dff + 16;
+  L.lf = lf;
+  size_t o = 64;                                             // abort flag
+  L.off_red = o;   o += sizeof(float4) * kMmaWarps * kNT * 32;
+  L.off_ssq = o;   o += sizeof(float) * kMmaWarps * 16;
+  L.off_hown = o;  o += align_up(sizeof(float) * 16 * (size_t)L.max_nd, 16);
+  L.attn_bytes = align_up((size_t)lf * kQStride * 2 + (size_t)lf * kOStride * 4 + (size_t)lf * 8 + 2 * kHeadDim * 4, 16);
+  L.off_attn = o;  o += L.attn_bytes * slots;
+  o = align_up(o, 128);
+  L.off_wo = o;    o += (size_t)L.max_nd * L.stride_d * 2;
+  L.off_wup = o;   o += (size_t)L.max_nf * L.stride_d * 2;
+  L.off_wdn = o;   o += (size_t)L.max_nd * L.stride_f * 2;
+  L.off_wk = o;    o += (size_t)L.max_nd * L.stride_d * 2;
+  L.off_wv = o;    o += (size_t)L.max_nd * L.stride_d * 2;
+  L.total = o;
+  return L;
+}
+
+// ---- small device helpers -------------------------------------------------------------------
+__device__ __forceinline__ float gelu_erf_f(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+__device__ __forceinline__ float bf_lo(unsigned u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(unsigned u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ unsigned pack_bf2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const unsigned*>(&v);
+}
+// Every published word is one 64-bit scalar (payload in the low half, step number in the high
+// half), so a reader never sees a payload without its flag.  Loads fetch two adjacent words.
+__device__ __forceinline__ uint4 ld_relaxed_v4(const void* p) {
+  unsigned long long w0, w1;
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
+  return make_uint4((unsigned)w0, (unsigned)(w0 >> 32), (unsigned)w1, (unsigned)(w1 >> 32));
+}
+__device__ __forceinline__ void st_relaxed_u64(void* p, unsigned lo, unsigned hi) {
+  const unsigned long long w = ((unsigned long long)hi << 32) | lo;
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_v4(void* p, unsigned a, unsigned b, unsigned c, unsigned d) {
+  const unsigned long long w0 = ((unsigned long long)b << 32) | a, w1 = ((unsigned long long)d << 32) | c;
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1,%2};" ::"l"(p), "l"(w0), "l"(w1) : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory"); }
+
+// A wait that ran out: record it for the host and tell every other waiter to leave.
+__device__ __noinline__ void report_timeout(SyncArea* s) {
+  s->status = RT_ERR_TIMEOUT;
+  __threadfence();
+  atomicExch(&s->abort_flag, 1u);
+}
+// Called every few polls: true when the wait must be abandoned.
+__device__ __forceinline__ bool wait_expired(SyncArea* s, unsigned long long& t_start) {
+  if (*reinterpret_cast<volatile unsigned*>(&s->abort_flag)) return true;
+  const unsigned long long now = globaltimer_ns();
+  if (t_start == 0) { t_start = now; return false; }
+  if (now - t_start > kWaitLimitNs) { report_timeout(s); return true; }
+  return false;
+}
+
+struct NTile { const __nv_bfloat16* w; int valid; };   // first row of the tile in shared memory, rows that exist (1..8)
+
+// One mat-vec phase of the MMA warps: y[b, row] = sum_k W[row, k] act[b, k] for up to kNT
+// n-tiles, activations polled from the flag-carrying words `ll` ([B][K/2] u64).
+// On return warp nt (< n_tiles) holds in acc the sums of n-tile nt:
+//   acc[0], acc[1] = rows 2c, 2c+1 of sequence g;  acc[2], acc[3] = the same rows of sequence g+8,
+// and ssq_lo / ssq_hi = sum_k act[g, k]^2 / act[g+8, k]^2 (when want_ssq).
+// MB = 1: B <= 8, MB = 2: B <= 16.  Returns false when the wait was abandoned.
+template <int MB>
+__device__ __forceinline__ bool mma_phase(const unsigned long long* ll, int K, int stride, unsigned seq, int B,
+                                          const NTile (&tiles)[kNT], int n_tiles, const __nv_bfloat16* gain,
+                                          bool want_ssq, float4* red, float* ssq_red, volatile int* s_abort,
+                                          SyncArea* sync, float (&acc_out)[4], float& ssq_lo, float& ssq_hi) {
+  constexpr int KC = 16 / MB;                                 // k-steps per chunk
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, c = lane & 3;
+  const int n_ks = K / 16;
+  const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
+  const int ks0 = warp * ks_per_warp;
+  const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
+  float acc[kNT][4];
+#pragma unroll
+  for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+  float sq0 = 0.f, sq1 = 0.f;
+  const bool row0 = g < B, row1 = (MB == 2) && (g + 8 < B);
+  const unsigned long long* base0 = ll + (size_t)g * (K / 2) + 2 * c;
+  const unsigned long long* base1 = ll + (size_t)(g + 8) * (K / 2) + 2 * c;
+  bool alive = true;
+
+  for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
+    unsigned a[KC][4];
+#pragma unroll
+    for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
+    // ---- poll the words of this chunk: a k-step is 8 words per sequence, this thread takes 2 ----
+    unsigned need0 = 0, need1 = 0;
+#pragma unroll
+    for (int i = 0; i < KC; ++i) {
+      if (kc0 + i < ks1) { if (row0) need0 |= 1u << i; if (row1) need1 |= 1u << i; }
+    }
+    unsigned spins = 0;
+    unsigned long long t_start = 0;
+    while (alive) {
+#pragma unroll
+      for (int i = 0; i < KC; ++i) {
+        if (need0 & (1u << i)) {
+          const uint4 w = ld_relaxed_v4(base0 + (size_t)(kc0 + i) * 8);
+          if (w.y == seq && w.w == seq) { a[i][0] = w.x; a[i][2] = w.z; need0 &= ~(1u << i); }
+        }
+      }
+      if (MB == 2) {
+#pragma unroll
+        for (int i = 0; i < KC; ++i) {
+          if (need1 & (1u << i)) {
+            const uint4 w = ld_relaxed_v4(base1 + (size_t)(kc0 + i) * 8);
+            if (w.y == seq && w.w == seq) { a[i][1] = w.x; a[i][3] = w.z; need1 &= ~(1u << i); }
+          }
+        }
+      }
+      if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
+      if ((++spins & 63u) == 0u) {
+        int bad = 0;
+        if (lane == 0) bad = wait_expired(sync, t_start) ? 1 : 0;
+        if (__shfl_sync(0xffffffffu, bad, 0)) { *s_abort = 1; alive = false; }
+      }
+    }
+    // ---- sum of squares and gain on the raw activations ----
+    if (want_ssq || gain) {
+#pragma unroll
+      for (int i = 0; i < KC; ++i) {
+        if (kc0 + i < ks1) {
+          const int k = (kc0 + i) * 16 + 4 * c;
+          float gn[4] = {1.f, 1.f, 1.f, 1.f};
+          if (gain) {
+            const uint2 gw = *reinterpret_cast<const uint2*>(gain + k);
+            gn[0] = bf_lo(gw.x); gn[1] = bf_hi(gw.x); gn[2] = bf_lo(gw.y); gn[3] = bf_hi(gw.y);
+          }
+#pragma unroll
+          for (int r = 0; r < MB; ++r) {
+            const float v0 = bf_lo(a[i][r]), v1 = bf_hi(a[i][r]), v2 = bf_lo(a[i][2 + r]), v3 = bf_hi(a[i][2 + r]);
+            const float s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+            if (r == 0) sq0 += s; else sq1 += s;
+            if (gain) { a[i][r] = pack_bf2(v0 * gn[0], v1 * gn[1]); a[i][2 + r] = pack_bf2(v2 * gn[2], v3 * gn[3]); }
+          }
+        }
+      }
+    }
+    // ---- tensor-core products: weights are the B operand (8 rows per n-tile) ----
+#pragma unroll
+    for (int i = 0; i < KC; ++i) {
+      if (kc0 + i < ks1) {
+        const int k = (kc0 + i) * 16 + 4 * c;
+#pragma unroll
+        for (int nt = 0; nt < kNT; ++nt) {
+          if (nt < n_tiles) {
+            const int r = g < tiles[nt].valid ? g : tiles[nt].valid - 1;
+            const uint2 b = *reinterpret_cast<const uint2*>(tiles[nt].w + (size_t)r * stride + k);
+            mma_bf16(acc[nt], a[i], b.x, b.y);
+          }
+        }
+      }
+    }
+  }
+  // ---- reduce over the 8 warps (K split) ----
+#pragma unroll
+  for (int nt = 0; nt < kNT; ++nt)
+    if (nt < n_tiles) red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+  if (want_ssq) {
+    sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
+    sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
+    if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
+  }
+  mma_warps_sync();
+  const bool ok = (*s_abort == 0);
+  acc_out[0] = acc_out[1] = acc_out[2] = acc_out[3] = 0.f;
+  ssq_lo = ssq_hi = 0.f;
+  if (warp < n_tiles) {
+#pragma unroll
+    for (int w = 0; w < kMmaWarps; ++w) {
+      const float4 v = red[(w * kNT + warp) * 32 + lane];
+      acc_out[0] += v.x; acc_out[1] += v.y; acc_out[2] += v.z; acc_out[3] += v.w;
+    }
+    if (want_ssq) {
+#pragma unroll
+      for (int w = 0; w < kMmaWarps; ++w) { ssq_lo += ssq_red[w * 16 + g]; ssq_hi += ssq_red[w * 16 + 8 + g]; }
+    }
+  }
+  mma_warps_sync();       // red / ssq_red may be overwritten by the next phase from here on
+  return ok;
+}
+
+// ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
+__device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsigned char* smem_slot, int pair,
+                               const unsigned long long* ll_kv, unsigned long long* ll_c) {
+  const int lane = threadIdx.x & 31;
+  const int B = p.B, d = p.d, H = p.H;
+  const int b = pair / H, h = pair % H;
+  const int n = p.t1 - p.t0;
+  __nv_bfloat16* qs = reinterpret_cast<__nv_bfloat16*>(smem_slot);
+  float* os = reinterpret_cast<float*>(smem_slot + (size_t)L.lf * kQStride * 2);
+  float* ms = os + (size_t)L.lf * kOStride;
+  float* ls = ms + L.lf;
+  float* kbuf = ls + L.lf;
+  float* vbuf = kbuf + kHeadDim;
+  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(p.q);
+  const __nv_bfloat16* g_k = reinterpret_cast<const __nv_bfloat16*>(p.g_k);
+  __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(p.k_cache);
+  __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(p.v_cache);
+  const bool qkn = (p.norm_flags & RT_NORM_QK) != 0;
+
+  // queries and carried stats of the leaf (written by earlier kernels of this call)
+  for (int i = 0; i < n; ++i) {
+    const size_t row = (size_t)(p.t0 + i) * B + b;
+    *reinterpret_cast<unsigned*>(qs + i * kQStride + 2 * lane) =
+        *reinterpret_cast<const unsigned*>(q + row * d + h * kHeadDim + 2 * lane);
+    os[i * kOStride + lane] = p.st_o[row * d + h * kHeadDim + lane];
+    os[i * kOStride + lane + 32] = p.st_o[row * d + h * kHeadDim + lane + 32];
+  }
+  for (int i = lane; i < n; i += 32) {
+    const size_t row = (size_t)(p.t0 + i) * B + b;
+    ms[i] = p.st_m[row * H + h];
+    ls[i] = p.st_l[row * H + h];
+  }
+  __syncwarp();
+  const float gk0 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane) : 1.0f;
+  const float gk1 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane + 1) : 1.0f;
+  unsigned long long* c_word = ll_c + (size_t)b * (d / 2) + h * (kHeadDim / 2) + lane;
+  // c of the first position: nothing of this leaf to fold in
+  {
+    const float il = 1.0f / ls[0];
+    st_relaxed_u64(c_word, pack_bf2(os[2 * lane] * il, os[2 * lane + 1] * il), p.seq_base + 1u);
+  }
+  const unsigned long long* k_words = ll_kv + (size_t)b * (2 * d) + h * kHeadDim + 2 * lane;
+  const unsigned long long* v_words = k_words + d;
+  for (int j = 0; j < n; ++j) {
+    const unsigned seq = p.seq_base + (unsigned)j + 1u;      // step that reveals position t0 + j
+    uint4 kw, vw;
+    unsigned spins = 0;
+    unsigned long long t_start = 0;
+    while (true) {
+      kw = ld_relaxed_v4(k_words);
+      vw = ld_relaxed_v4(v_words);
+      const bool ok = kw.y == seq && kw.w == seq && vw.y == seq && vw.w == seq;
+      if (__all_sync(0xffffffffu, ok)) break;
+      if ((++spins & 63u) == 0u) {
+        int bad = 0;
+        if (lane == 0) bad = wait_expired(p.sync, t_start) ? 1 : 0;
+        if (__shfl_sync(0xffffffffu, bad, 0)) return;
+      }
+    }
+    // Eq. (1): qkRMS over the head, then the storage rounding the cache applies
+    const float k0 = __uint_as_float(kw.x), k1 = __uint_as_float(kw.z);
+    const float ss = warp_sum(k0 * k0 + k1 * k1);
+    const float rs = qkn ? rsqrtf(ss * (1.0f / kHeadDim) + p.eps) : 1.0f;
+    const unsigned kq = pack_bf2(k0 * rs * gk0, k1 * rs * gk1);
+    const unsigned vq = pack_bf2(__uint_as_float(vw.x), __uint_as_float(vw.z));
+    const size_t crow = ((size_t)(p.t0 + j) * B + b) * d + h * kHeadDim + 2 * lane;
+    *reinterpret_cast<unsigned*>(kc + crow) = kq;
+    *reinterpret_cast<unsigned*>(vc + crow) = vq;
+    if (j + 1 >= n) break;
+    const float kf0 = bf_lo(kq), kf1 = bf_hi(kq), vf0 = bf_lo(vq), vf1 = bf_hi(vq);
+    {
+      // critical path: finish query j+1 and publish c_{j+1}
+      const int i = j + 1;
+      const unsigned qw = *reinterpret_cast<const unsigned*>(qs + i * kQStride + 2 * lane);
+      const float s = warp_sum(bf_lo(qw) * kf0 + bf_hi(qw) * kf1) * p.scale_log2;
+      const float m_old = ms[i], l_old = ls[i];
+      const float m_new = fmaxf(m_old, s);
+      const float corr = exp2f(m_old - m_new), pj = exp2f(s - m_new);
+      const float il = 1.0f / (l_old * corr + pj);
+      const float o0 = os[i * kOStride + 2 * lane] * corr + pj * vf0;
+      const float o1 = os[i * kOStride + 2 * lane + 1] * corr + pj * vf1;
+      st_relaxed_u64(c_word, pack_bf2(o0 * il, o1 * il), seq + 1u);
+    }
+    // off the critical path: fold (k_j, v_j) into the later queries of the leaf, one query per lane
+    kbuf[2 * lane] = kf0; kbuf[2 * lane + 1] = kf1;
+    vbuf[2 * lane] = vf0; vbuf[2 * lane + 1] = vf1;
+    __syncwarp();
+    for (int i = j + 2 + lane; i < n; i += 32) {
+      const __nv_bfloat16* qi = qs + i * kQStride;
+      float s = 0.f;
+#pragma unroll 8
+      for (int e = 0; e < kHeadDim; e += 2) {
+        const unsigned qw = *reinterpret_cast<const unsigned*>(qi + e);
+        s += bf_lo(qw) * kbuf[e] + bf_hi(qw) * kbuf[e + 1];
+      }
+      s *= p.scale_log2;
+      const float m_old = ms[i];
+      const float m_new = fmaxf(m_old, s);
+      const float corr = exp2f(m_old - m_new), pj = exp2f(s - m_new);
+      ms[i] = m_new;
+      ls[i] = ls[i] * corr + pj;
+      float* oi = os + i * kOStride;
+#pragma unroll 8
+      for (int e = 0; e < kHeadDim; ++e) oi[e] = oi[e] * corr + pj * vbuf[e];
+    }
+    __syncwarp();
+  }
+}
+
+template <int MB>
+__global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
+                                                                      unsigned long long* ll_c, unsigned long long* ll_h,
+                                                                      unsigned long long* ll_g, unsigned long long* ll_z,
+                                                                      unsigned long long* ll_kv) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem);
+  float4* red = reinterpret_cast<float4*>(smem + L.off_red);
+  float* ssq_red = reinterpret_cast<float*>(smem + L.off_ssq);
+  float* hown = reinterpret_cast<float*>(smem + L.off_hown);
+  __nv_bfloat16* s_wo = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wo);
+  __nv_bfloat16* s_wup = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wup);
+  __nv_bfloat16* s_wdn = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wdn);
+  __nv_bfloat16* s_wk = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wk);
+  __nv_bfloat16* s_wv = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wv);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int B = p.B, d = p.d, H = p.H, dff = p.dff;
+  if (*reinterpret_cast<volatile unsigned*>(&p.sync->abort_flag)) return;
+  // rows are dealt out in pairs so that a published word (two consecutive rows) has one owner
+  const int d_lo = 2 * (int)((long long)(d / 2) * cta / G), d_hi = 2 * (int)((long long)(d / 2) * (cta + 1) / G);
+  const int f_lo = 2 * (int)((long long)(dff / 2) * cta / G), f_hi = 2 * (int)((long long)(dff / 2) * (cta + 1) / G);
+  const int nd = d_hi - d_lo, nf = f_hi - f_lo;
+
+  if (tid == 0) *s_abort = 0;
+  {
+    auto stage = [&](__nv_bfloat16* dst, int dst_stride, const void* src_base, int row_lo, int nrows, int K) {
+      const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(src_base) + (size_t)row_lo * K);
+      const int per_row = K / 8;
+      for (int i = tid; i < nrows * per_row; i += kLeafMmaThreads) {
+        const int r = i / per_row, v = i % per_row;
+        *reinterpret_cast<uint4*>(dst + (size_t)r * dst_stride + v * 8) = src[(size_t)r * per_row + v];
+      }
+    };
+    stage(s_wo, L.stride_d, p.w_o, d_lo, nd, d);
+    stage(s_wup, L.stride_d, p.w_up, f_lo, nf, d);
+    stage(s_wdn, L.stride_f, p.w_down, d_lo, nd, dff);
+    stage(s_wk, L.stride_d, p.w_k, d_lo, nd, d);
+    stage(s_wv, L.stride_d, p.w_v, d_lo, nd, d);
+  }
+  __syncthreads();
+
+  if (warp >= kMmaWarps) {
+    const int slot = warp - kMmaWarps;
+    const int pair = cta + slot * G;
+    if (pair < B * H) attention_role(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
+    return;
+  }
+
+  // ------------------------------ MMA warps ------------------------------
+  const int g = lane >> 2, c = lane & 3;
+  const bool pre = (p.norm_flags & RT_NORM_PRE) != 0;
+  const bool kv_norm = pre && !(p.norm_flags & RT_NORM_SKIP_Z);
+  const __nv_bfloat16* g_mlp = reinterpret_cast<const __nv_bfloat16*>(p.g_mlp);
+  const __nv_bfloat16* g_kv = reinterpret_cast<const __nv_bfloat16*>(p.g_kv);
+  const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(p.x);
+  __nv_bfloat16* z = reinterpret_cast<__nv_bfloat16*>(p.z);
+  const float inv_d = 1.0f / (float)d;
+  const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
+  const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
+
+  auto make_tiles = [&](NTile (&tl)[kNT], const __nv_bfloat16* w, int stride, int nrows, int first_tile) {
+#pragma unroll
+    for (int i = 0; i < kNT; ++i) {
+      const int r0 = (first_tile + i) * 8;
+      tl[i].w = w + (size_t)(r0 < nrows ? r0 : 0) * stride;
+      tl[i].valid = nrows - r0 < 8 ? (nrows - r0 > 0 ? nrows - r0 : 1) : 8;
+    }
+  };
+
+  for (int t = p.t0; t < p.t1; ++t) {
+    const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
+    float acc[4], sl, sh;
+
+    // ---------------- W_o: a = W_o c_t, h = x_t + alpha a ----------------
+    for (int t0n = 0; t0n < nt_d; t0n += kNT) {
+      NTile tl[kNT];
+      make_tiles(tl, s_wo, L.stride_d, nd, t0n);
+      const int ntl = nt_d - t0n < kNT ? nt_d - t0n : kNT;
+      // x of this step for the rows this thread finishes
+      const int rl = (t0n + warp) * 8 + 2 * c;                 // local row pair of the epilogue thread
+      unsigned xw0 = 0, xw1 = 0;
+      if (warp < ntl && rl < nd) {
+        if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+        if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+      }
+      if (!mma_phase<MB>(ll_c, d, L.stride_d, seq, B, tl, ntl, nullptr, false, red, ssq_red, s_abort, p.sync, acc, sl, sh))
+        return;
+      if (warp < ntl && rl < nd) {
+        if (has0) {
+          const float h0 = bf_lo(xw0) + p.alpha * acc[0], h1 = bf_hi(xw0) + p.alpha * acc[1];
+          hown[g * L.max_nd + rl] = h0; hown[g * L.max_nd + rl + 1] = h1;
+          st_relaxed_u64(ll_h + (size_t)g * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
+        }
+        if (has1) {
+          const float h0 = bf_lo(xw1) + p.alpha * acc[2], h1 = bf_hi(xw1) + p.alpha * acc[3];
+          hown[(g + 8) * L.max_nd + rl] = h0; hown[(g + 8) * L.max_nd + rl + 1] = h1;
+          st_relaxed_u64(ll_h + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
+        }
+      }
+    }
+    // ---------------- W_up: g = GELU(W_up RMS(h)) ----------------
+    for (int t0n = 0; t0n < nt_f; t0n += kNT) {
+      NTile tl[kNT];
+      make_tiles(tl, s_wup, L.stride_d, nf, t0n);
+      const int ntl = nt_f - t0n < kNT ? nt_f - t0n : kNT;
+      const int rl = (t0n + warp) * 8 + 2 * c;
+      if (!mma_phase<MB>(ll_h, d, L.stride_d, seq, B, tl, ntl, pre ? g_mlp : nullptr, pre, red, ssq_red, s_abort, p.sync,
+                         acc, sl, sh))
+        return;
+      if (warp < ntl && rl < nf) {
+        if (has0) {
+          const float rs = pre ? rsqrtf(sl * inv_d + p.eps) : 1.0f;
+          st_relaxed_u64(ll_g + (size_t)g * (dff / 2) + (f_lo + rl) / 2,
+                         pack_bf2(gelu_erf_f(acc[0] * rs), gelu_erf_f(acc[1] * rs)), seq);
+        }
+        if (has1) {
+          const float rs = pre ? rsqrtf(sh * inv_d + p.eps) : 1.0f;
+          st_relaxed_u64(ll_g + (size_t)(g + 8) * (dff / 2) + (f_lo + rl) / 2,
+                         pack_bf2(gelu_erf_f(acc[2] * rs), gelu_erf_f(acc[3] * rs)), seq);
+        }
+      }
+    }
+    // ---------------- W_down: z_t = h + alpha W_down g ----------------
+    for (int t0n = 0; t0n < nt_d; t0n += kNT) {
+      NTile tl[kNT];
+      make_tiles(tl, s_wdn, L.stride_f, nd, t0n);
+      const int ntl = nt_d - t0n < kNT ? nt_d - t0n : kNT;
+      const int rl = (t0n + warp) * 8 + 2 * c;
+      if (!mma_phase<MB>(ll_g, dff, L.stride_f, seq, B, tl, ntl, nullptr, false, red, ssq_red, s_abort, p.sync, acc, sl, sh))
+        return;
+      if (warp < ntl && rl < nd) {
+        if (has0) {
+          const float z0 = hown[g * L.max_nd + rl] + p.alpha * acc[0], z1 = hown[g * L.max_nd + rl + 1] + p.alpha * acc[1];
+          const unsigned zw = pack_bf2(z0, z1);
+          *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+          st_relaxed_u64(ll_z + (size_t)g * (d / 2) + (d_lo + rl) / 2, zw, seq);
+        }
+        if (has1) {
+          const float z0 = hown[(g + 8) * L.max_nd + rl] + p.alpha * acc[2];
+          const float z1 = hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * acc[3];
+          const unsigned zw = pack_bf2(z0, z1);
+          *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+          st_relaxed_u64(ll_z + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, zw, seq);
+        }
+      }
+    }
+    // ---------------- W_k, W_v: raw k_t and v_t from RMS(z_t) (Eqs. 1-2; qkRMS is applied by the attention warp) ----
+    for (int t0n = 0; t0n < 2 * nt_d; t0n += kNT) {
+      NTile tl[kNT];
+#pragma unroll
+      for (int i = 0; i < kNT; ++i) {
+        const int ti = t0n + i;
+        const bool is_v = ti >= nt_d;
+        const int r0 = (is_v ? ti - nt_d : ti) * 8;
+        tl[i].w = (is_v ? s_wv : s_wk) + (size_t)(r0 < nd ? r0 : 0) * L.stride_d;
+        tl[i].valid = nd - r0 < 8 ? (nd - r0 > 0 ? nd - r0 : 1) : 8;
+      }
+      const int ntl = 2 * nt_d - t0n < kNT ? 2 * nt_d - t0n : kNT;
+      if (!mma_phase<MB>(ll_z, d, L.stride_d, seq, B, tl, ntl, kv_norm ? g_kv : nullptr, kv_norm, red, ssq_red, s_abort,
+                         p.sync, acc, sl, sh))
+        return;
+      const int ti = t0n + warp;
+      const bool is_v = ti >= nt_d;
+      const int rl = (is_v ? ti - nt_d : ti) * 8 + 2 * c;
+      if (warp < ntl && rl < nd) {
+        const size_t col = (size_t)(is_v ? d : 0) + d_lo + rl;
+        if (has0) {
+          const float rs = kv_norm ? rsqrtf(sl * inv_d + p.eps) : 1.0f;
+          st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(acc[0] * rs), seq, __float_as_uint(acc[1] * rs), seq);
+        }
+        if (has1) {
+          const float rs = kv_norm ? rsqrtf(sh * inv_d + p.eps) : 1.0f;
+          st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(acc[2] * rs), seq,
+                        __float_as_uint(acc[3] * rs), seq);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ host
+
+// Picks the leaf capacity and the launch shape; returns false when this kernel does not take
+// the shape (the generic leaf kernel does).
+bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out) {
+  int dev = 0, sms = 0, max_smem = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+  if (B > 16 || (d % 64) || (dff % 16) || B * H > kAttnSlots * sms) return false;
+  const int cands[3] = {64, 32, 16};
+  for (int lf : cands) {
+    if (want_leaf && lf != want_leaf) continue;
+    const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms));
+    if (L.total <= (size_t)max_smem) {
+      out->grid = sms; out->block = kLeafMmaThreads; out->smem = L.total; out->leaf = lf;
+      return true;
+    }
+  }
+  return false;
+}
+
+cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {
+  LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid));
+  const void* fn = p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2>)
+                           : reinterpret_cast<const void*>(&leaf_mma_kernel<1>);
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
+  if (e != cudaSuccess) return e;
+  LeafParams pp = p;
+  LeafMmaBuffers b = buf;
+  void* args[] = {(void*)&pp, (void*)&L, (void*)&b.ll_c, (void*)&b.ll_h, (void*)&b.ll_g, (void*)&b.ll_z, (void*)&b.ll_kv};
+  return cudaLaunchCooperativeKernel(fn, dim3(l.grid), dim3(l.block), args, l.smem, s);
+}
+
+}  // namespace rt
