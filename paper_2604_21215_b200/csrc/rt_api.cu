@@ -174,10 +174,11 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     mb.ll_kv = mb.ll_g + (size_t)B * (c->d_ff / 2);
   }
   auto leaf_mma = [&](int t0, int t1) -> bool {
-    lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base;
+    lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
     ProfScope ps(s, kProfLeaf);
     if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return false;
     ctx.seq_base += (unsigned)(t1 - t0);
+    ctx.bar_base += (unsigned)(t1 - t0) * (unsigned)ml.grid;      // one grid barrier per token step
     return true;
   };
 

@@ -108,22 +108,93 @@ __device__ __forceinline__ bool wait_expired(SyncArea* s, unsigned long long& t_
   return false;
 }
 
-struct NTile { const __nv_bfloat16* w; int valid; };   // first row of the tile in shared memory, rows that exist (1..8)
+// What one mat-vec phase works on.  Tiles are groups of 8 weight rows in shared memory.
+struct PhaseDesc {
+  const void* act;                 // LL mode: [B][K/2] flag-carrying words; packed mode: [B][K] bf16
+  int K, stride;                   // reduction length, shared-memory row stride of the weights (elements)
+  unsigned seq;                    // flag value of this step (LL mode)
+  int B, n_tiles;
+  const __nv_bfloat16* w[kNT];     // first row of each tile
+  int valid[kNT];                  // rows that exist in each tile (1..8); the rest repeat the last one
+  const __nv_bfloat16* gain;       // optional per-k gain
+  int want_ssq;
+};
+struct PhaseOut { float acc[4]; float ssq_lo, ssq_hi; int ok; };
+struct PhaseShared { float4* red; float* ssq_red; volatile int* s_abort; SyncArea* sync; };
 
-// One mat-vec phase of the MMA warps: y[b, row] = sum_k W[row, k] act[b, k] for up to kNT
-// n-tiles, activations polled from the flag-carrying words `ll` ([B][K/2] u64).
-// On return warp nt (< n_tiles) holds in acc the sums of n-tile nt:
-//   acc[0], acc[1] = rows 2c, 2c+1 of sequence g;  acc[2], acc[3] = the same rows of sequence g+8,
-// and ssq_lo / ssq_hi = sum_k act[g, k]^2 / act[g+8, k]^2 (when want_ssq).
-// MB = 1: B <= 8, MB = 2: B <= 16.  Returns false when the wait was abandoned.
+// Sum of squares (of the raw values) and optional gain for one k-step of fragments; gp points
+// at this thread's 4 gains of the k-step (or is null).
 template <int MB>
-__device__ __forceinline__ bool mma_phase(const unsigned long long* ll, int K, int stride, unsigned seq, int B,
-                                          const NTile (&tiles)[kNT], int n_tiles, const __nv_bfloat16* gain,
-                                          bool want_ssq, float4* red, float* ssq_red, volatile int* s_abort,
-                                          SyncArea* sync, float (&acc_out)[4], float& ssq_lo, float& ssq_hi) {
-  constexpr int KC = 16 / MB;                                 // k-steps per chunk
+__device__ __forceinline__ void frag_ssq_gain(unsigned (&a)[4], const __nv_bfloat16* gp, float& sq0, float& sq1) {
+  float gn[4] = {1.f, 1.f, 1.f, 1.f};
+  if (gp) {
+    const uint2 gw = *reinterpret_cast<const uint2*>(gp);
+    gn[0] = bf_lo(gw.x); gn[1] = bf_hi(gw.x); gn[2] = bf_lo(gw.y); gn[3] = bf_hi(gw.y);
+  }
+#pragma unroll
+  for (int r = 0; r < MB; ++r) {
+    const float v0 = bf_lo(a[r]), v1 = bf_hi(a[r]), v2 = bf_lo(a[2 + r]), v3 = bf_hi(a[2 + r]);
+    const float s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+    if (r == 0) sq0 += s; else sq1 += s;
+    if (gp) { a[r] = pack_bf2(v0 * gn[0], v1 * gn[1]); a[2 + r] = pack_bf2(v2 * gn[2], v3 * gn[3]); }
+  }
+}
+
+// Per-thread shared-memory address of its 8 bytes of weight row g (clamped) of each tile at k = 4c.
+__device__ __forceinline__ void weight_ptrs(const PhaseDesc& ds, int g, int c, const unsigned char* (&wp)[kNT]) {
+#pragma unroll
+  for (int nt = 0; nt < kNT; ++nt) {
+    const int v = ds.valid[nt];
+    const int r = g < v ? g : v - 1;
+    wp[nt] = reinterpret_cast<const unsigned char*>(ds.w[nt < ds.n_tiles ? nt : 0] + (size_t)r * ds.stride + 4 * c);
+  }
+}
+
+// Tail shared by both input modes: reduce the K split over the 8 MMA warps.  Afterwards warp nt
+// (< n_tiles) holds the sums of n-tile nt: acc[0], acc[1] = weight rows 2c, 2c+1 for sequence g,
+// acc[2], acc[3] = the same rows for sequence g+8; ssq_lo / ssq_hi = sum_k act[g or g+8, k]^2.
+__device__ __noinline__ PhaseOut mma_reduce(const float (&acc)[kNT][4], float sq0, float sq1, int n_tiles, int want_ssq,
+                                            const PhaseShared sh) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, c = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < kNT; ++nt)
+    if (nt < n_tiles) sh.red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+  if (want_ssq) {
+    sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
+    sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
+    if (c == 0) { sh.ssq_red[warp * 16 + g] = sq0; sh.ssq_red[warp * 16 + 8 + g] = sq1; }
+  }
+  mma_warps_sync();
+  PhaseOut o;
+  o.ok = (*sh.s_abort == 0);
+  o.acc[0] = o.acc[1] = o.acc[2] = o.acc[3] = 0.f;
+  o.ssq_lo = o.ssq_hi = 0.f;
+  if (warp < n_tiles) {
+#pragma unroll
+    for (int w = 0; w < kMmaWarps; ++w) {
+      const float4 v = sh.red[(w * kNT + warp) * 32 + lane];
+      o.acc[0] += v.x; o.acc[1] += v.y; o.acc[2] += v.z; o.acc[3] += v.w;
+    }
+    if (want_ssq) {
+#pragma unroll
+      for (int w = 0; w < kMmaWarps; ++w) { o.ssq_lo += sh.ssq_red[w * 16 + g]; o.ssq_hi += sh.ssq_red[w * 16 + 8 + g]; }
+    }
+  }
+  mma_warps_sync();       // red / ssq_red may be overwritten by the next phase from here on
+  return o;
+}
+
+// One mat-vec phase, activations polled from flag-carrying words: y[b, row] = sum_k W[row, k] act[b, k].
+// MB = 1: B <= 8, MB = 2: B <= 16.  Kept out of line so that the four phases of a token step share
+// one copy of the code (the step runs once per token: straight-line copies thrash the instruction cache).
+template <int MB>
+__device__ __noinline__ PhaseOut mma_phase_ll(const PhaseDesc& ds, const PhaseShared sh, unsigned long long* wait_ns) {
+  constexpr int KC = 8;                                       // k-steps per chunk
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, c = lane & 3;
+  const int K = ds.K, B = ds.B;
+  const unsigned seq = ds.seq;
   const int n_ks = K / 16;
   const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
   const int ks0 = warp * ks_per_warp;
@@ -133,15 +204,20 @@ __device__ __forceinline__ bool mma_phase(const unsigned long long* ll, int K, i
   for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
   float sq0 = 0.f, sq1 = 0.f;
   const bool row0 = g < B, row1 = (MB == 2) && (g + 8 < B);
+  const unsigned long long* ll = reinterpret_cast<const unsigned long long*>(ds.act);
   const unsigned long long* base0 = ll + (size_t)g * (K / 2) + 2 * c;
   const unsigned long long* base1 = ll + (size_t)(g + 8) * (K / 2) + 2 * c;
   bool alive = true;
+  const unsigned char* wp[kNT];
+  weight_ptrs(ds, g, c, wp);
+  const __nv_bfloat16* gp = ds.gain ? ds.gain + 4 * c : nullptr;
+  const int n_tiles = ds.n_tiles, want_ssq = ds.want_ssq;
 
   for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
     unsigned a[KC][4];
 #pragma unroll
     for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
-    // ---- poll the words of this chunk: a k-step is 8 words per sequence, this thread takes 2 ----
+    // a k-step is 8 words per sequence; this thread takes the 2 adjacent ones at 4c
     unsigned need0 = 0, need1 = 0;
 #pragma unroll
     for (int i = 0; i < KC; ++i) {
@@ -149,6 +225,7 @@ __device__ __forceinline__ bool mma_phase(const unsigned long long* ll, int K, i
     }
     unsigned spins = 0;
     unsigned long long t_start = 0;
+    const unsigned long long t_poll = wait_ns ? globaltimer_ns() : 0ull;
     while (alive) {
 #pragma unroll
       for (int i = 0; i < KC; ++i) {
@@ -169,73 +246,100 @@ __device__ __forceinline__ bool mma_phase(const unsigned long long* ll, int K, i
       if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
       if ((++spins & 63u) == 0u) {
         int bad = 0;
-        if (lane == 0) bad = wait_expired(sync, t_start) ? 1 : 0;
-        if (__shfl_sync(0xffffffffu, bad, 0)) { *s_abort = 1; alive = false; }
+        if (lane == 0) bad = wait_expired(sh.sync, t_start) ? 1 : 0;
+        if (__shfl_sync(0xffffffffu, bad, 0)) { *sh.s_abort = 1; alive = false; }
       }
     }
-    // ---- sum of squares and gain on the raw activations ----
-    if (want_ssq || gain) {
+    if (wait_ns) *wait_ns += globaltimer_ns() - t_poll;
+    const unsigned char* wc[kNT];
 #pragma unroll
-      for (int i = 0; i < KC; ++i) {
-        if (kc0 + i < ks1) {
-          const int k = (kc0 + i) * 16 + 4 * c;
-          float gn[4] = {1.f, 1.f, 1.f, 1.f};
-          if (gain) {
-            const uint2 gw = *reinterpret_cast<const uint2*>(gain + k);
-            gn[0] = bf_lo(gw.x); gn[1] = bf_hi(gw.x); gn[2] = bf_lo(gw.y); gn[3] = bf_hi(gw.y);
-          }
-#pragma unroll
-          for (int r = 0; r < MB; ++r) {
-            const float v0 = bf_lo(a[i][r]), v1 = bf_hi(a[i][r]), v2 = bf_lo(a[i][2 + r]), v3 = bf_hi(a[i][2 + r]);
-            const float s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
-            if (r == 0) sq0 += s; else sq1 += s;
-            if (gain) { a[i][r] = pack_bf2(v0 * gn[0], v1 * gn[1]); a[i][2 + r] = pack_bf2(v2 * gn[2], v3 * gn[3]); }
-          }
-        }
-      }
-    }
-    // ---- tensor-core products: weights are the B operand (8 rows per n-tile) ----
+    for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
+    const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
 #pragma unroll
     for (int i = 0; i < KC; ++i) {
       if (kc0 + i < ks1) {
-        const int k = (kc0 + i) * 16 + 4 * c;
+        if (want_ssq || gp) frag_ssq_gain<MB>(a[i], gc ? gc + i * 16 : nullptr, sq0, sq1);
 #pragma unroll
         for (int nt = 0; nt < kNT; ++nt) {
           if (nt < n_tiles) {
-            const int r = g < tiles[nt].valid ? g : tiles[nt].valid - 1;
-            const uint2 b = *reinterpret_cast<const uint2*>(tiles[nt].w + (size_t)r * stride + k);
+            const uint2 b = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
             mma_bf16(acc[nt], a[i], b.x, b.y);
           }
         }
       }
     }
   }
-  // ---- reduce over the 8 warps (K split) ----
+  return mma_reduce(acc, sq0, sq1, n_tiles, want_ssq, sh);
+}
+
+// The same product with the activations read as plain packed bf16 ([B][K]) after a grid barrier:
+// used for the wide vector (K = d_ff), where doubling the bytes with flags costs more than it saves.
+// No norm or gain on this input (it is the GELU output).
+// All loads of a round are issued before the first product.
+template <int MB>
+__device__ __noinline__ PhaseOut mma_phase_packed(const PhaseDesc& ds, const PhaseShared sh) {
+  constexpr int KC = 32 / MB;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, c = lane & 3;
+  const int K = ds.K, B = ds.B;
+  const int n_ks = K / 16;
+  const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
+  const int ks0 = warp * ks_per_warp;
+  const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
+  float acc[kNT][4];
 #pragma unroll
-  for (int nt = 0; nt < kNT; ++nt)
-    if (nt < n_tiles) red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
-  if (want_ssq) {
-    sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
-    sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
-    if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
+  for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+  const bool row0 = g < B, row1 = (MB == 2) && (g + 8 < B);
+  const __nv_bfloat16* act = reinterpret_cast<const __nv_bfloat16*>(ds.act);
+  const __nv_bfloat16* base0 = act + (size_t)g * K + 4 * c;
+  const __nv_bfloat16* base1 = act + (size_t)(g + 8) * K + 4 * c;
+  const unsigned char* wp[kNT];
+  weight_ptrs(ds, g, c, wp);
+  const int n_tiles = ds.n_tiles;
+  for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
+    unsigned a[KC][4];
+#pragma unroll
+    for (int i = 0; i < KC; ++i) {
+      a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u;
+      if (kc0 + i < ks1) {
+        if (row0) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(base0 + (size_t)(kc0 + i) * 16)); a[i][0] = w.x; a[i][2] = w.y; }
+        if (row1) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(base1 + (size_t)(kc0 + i) * 16)); a[i][1] = w.x; a[i][3] = w.y; }
+      }
+    }
+    const unsigned char* wc[kNT];
+#pragma unroll
+    for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
+#pragma unroll
+    for (int i = 0; i < KC; ++i) {
+      if (kc0 + i < ks1) {
+#pragma unroll
+        for (int nt = 0; nt < kNT; ++nt) {
+          if (nt < n_tiles) {
+            const uint2 b = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
+            mma_bf16(acc[nt], a[i], b.x, b.y);
+          }
+        }
+      }
+    }
+  }
+  return mma_reduce(acc, 0.f, 0.f, n_tiles, 0, sh);
+}
+
+// Barrier over all CTAs, run by the MMA warps only (the attention warps never wait on it).
+__device__ __noinline__ bool mma_grid_barrier(const PhaseShared sh, unsigned target) {
+  mma_warps_sync();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    red_release_add_u32(&sh.sync->bar_count, 1u);
+    unsigned spins = 0;
+    unsigned long long t_start = 0;
+    while (ld_acquire_u32(&sh.sync->bar_count) < target) {
+      if ((++spins & 255u) == 0u && wait_expired(sh.sync, t_start)) { *sh.s_abort = 1; break; }
+    }
+    __threadfence();
   }
   mma_warps_sync();
-  const bool ok = (*s_abort == 0);
-  acc_out[0] = acc_out[1] = acc_out[2] = acc_out[3] = 0.f;
-  ssq_lo = ssq_hi = 0.f;
-  if (warp < n_tiles) {
-#pragma unroll
-    for (int w = 0; w < kMmaWarps; ++w) {
-      const float4 v = red[(w * kNT + warp) * 32 + lane];
-      acc_out[0] += v.x; acc_out[1] += v.y; acc_out[2] += v.z; acc_out[3] += v.w;
-    }
-    if (want_ssq) {
-#pragma unroll
-      for (int w = 0; w < kMmaWarps; ++w) { ssq_lo += ssq_red[w * 16 + g]; ssq_hi += ssq_red[w * 16 + 8 + g]; }
-    }
-  }
-  mma_warps_sync();       // red / ssq_red may be overwritten by the next phase from here on
-  return ok;
+  return *sh.s_abort == 0;
 }
 
 // ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
@@ -281,9 +385,12 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   }
   const unsigned long long* k_words = ll_kv + (size_t)b * (2 * d) + h * kHeadDim + 2 * lane;
   const unsigned long long* v_words = k_words + d;
+  const bool timing = (pair == 0 && lane == 0);
+  unsigned long long a_work = 0, a_wait = 0, t_mark = timing ? globaltimer_ns() : 0ull;
   for (int j = 0; j < n; ++j) {
     const unsigned seq = p.seq_base + (unsigned)j + 1u;      // step that reveals position t0 + j
     uint4 kw, vw;
+    if (timing) { const unsigned long long now = globaltimer_ns(); a_work += now - t_mark; t_mark = now; }
     unsigned spins = 0;
     unsigned long long t_start = 0;
     while (true) {
@@ -297,6 +404,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
         if (__shfl_sync(0xffffffffu, bad, 0)) return;
       }
     }
+    if (timing) { const unsigned long long now = globaltimer_ns(); a_wait += now - t_mark; t_mark = now; }
     // Eq. (1): qkRMS over the head, then the storage rounding the cache applies
     const float k0 = __uint_as_float(kw.x), k1 = __uint_as_float(kw.z);
     const float ss = warp_sum(k0 * k0 + k1 * k1);
@@ -345,6 +453,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     }
     __syncwarp();
   }
+  if (timing) { atomicAdd(&p.sync->phase_ns[0], a_work); atomicAdd(&p.sync->phase_ns[1], a_wait); }
 }
 
 template <int MB>
@@ -401,131 +510,158 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   const int g = lane >> 2, c = lane & 3;
   const bool pre = (p.norm_flags & RT_NORM_PRE) != 0;
   const bool kv_norm = pre && !(p.norm_flags & RT_NORM_SKIP_Z);
-  const __nv_bfloat16* g_mlp = reinterpret_cast<const __nv_bfloat16*>(p.g_mlp);
-  const __nv_bfloat16* g_kv = reinterpret_cast<const __nv_bfloat16*>(p.g_kv);
   const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(p.x);
   __nv_bfloat16* z = reinterpret_cast<__nv_bfloat16*>(p.z);
+  __nv_bfloat16* g_pk = reinterpret_cast<__nv_bfloat16*>(ll_g);      // packed bf16 [B][dff]
   const float inv_d = 1.0f / (float)d;
   const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
   const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
+  const PhaseShared sh{red, ssq_red, s_abort, p.sync};
+  unsigned bar_target = p.bar_base;
 
-  auto make_tiles = [&](NTile (&tl)[kNT], const __nv_bfloat16* w, int stride, int nrows, int first_tile) {
+  PhaseDesc ds;
+  ds.B = B;
+  auto set_tiles = [&](const __nv_bfloat16* w, int stride, int nrows, int first_tile) {
 #pragma unroll
     for (int i = 0; i < kNT; ++i) {
       const int r0 = (first_tile + i) * 8;
-      tl[i].w = w + (size_t)(r0 < nrows ? r0 : 0) * stride;
-      tl[i].valid = nrows - r0 < 8 ? (nrows - r0 > 0 ? nrows - r0 : 1) : 8;
+      ds.w[i] = w + (size_t)(r0 < nrows ? r0 : 0) * stride;
+      ds.valid[i] = nrows - r0 < 8 ? (nrows - r0 > 0 ? nrows - r0 : 1) : 8;
+    }
+  };
+  const bool timing = (cta == 0 && tid == 0);
+  unsigned long long ph_ns[10], wait_ns = 0;
+#pragma unroll
+  for (int i = 0; i < 10; ++i) ph_ns[i] = 0ull;
+  unsigned long long t_ph = timing ? globaltimer_ns() : 0ull;
+  auto phase_done = [&](int i) {
+    if (timing) {
+      const unsigned long long now = globaltimer_ns();
+      ph_ns[2 * i] += now - t_ph - wait_ns; ph_ns[2 * i + 1] += wait_ns;
+      t_ph = now; wait_ns = 0;
     }
   };
 
   for (int t = p.t0; t < p.t1; ++t) {
-    const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
-    float acc[4], sl, sh;
+    ds.seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
+    const unsigned seq = ds.seq;
 
     // ---------------- W_o: a = W_o c_t, h = x_t + alpha a ----------------
     for (int t0n = 0; t0n < nt_d; t0n += kNT) {
-      NTile tl[kNT];
-      make_tiles(tl, s_wo, L.stride_d, nd, t0n);
-      const int ntl = nt_d - t0n < kNT ? nt_d - t0n : kNT;
-      // x of this step for the rows this thread finishes
-      const int rl = (t0n + warp) * 8 + 2 * c;                 // local row pair of the epilogue thread
+      set_tiles(s_wo, L.stride_d, nd, t0n);
+      ds.act = ll_c; ds.K = d; ds.stride = L.stride_d; ds.gain = nullptr; ds.want_ssq = 0;
+      ds.n_tiles = nt_d - t0n < kNT ? nt_d - t0n : kNT;
+      const int rl = (t0n + warp) * 8 + 2 * c;                 // local row pair this thread finishes
       unsigned xw0 = 0, xw1 = 0;
-      if (warp < ntl && rl < nd) {
+      const bool mine = warp < ds.n_tiles && rl < nd;
+      if (mine) {
         if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
         if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
       }
-      if (!mma_phase<MB>(ll_c, d, L.stride_d, seq, B, tl, ntl, nullptr, false, red, ssq_red, s_abort, p.sync, acc, sl, sh))
-        return;
-      if (warp < ntl && rl < nd) {
+      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
+      if (!o.ok) return;
+      if (mine) {
         if (has0) {
-          const float h0 = bf_lo(xw0) + p.alpha * acc[0], h1 = bf_hi(xw0) + p.alpha * acc[1];
+          const float h0 = bf_lo(xw0) + p.alpha * o.acc[0], h1 = bf_hi(xw0) + p.alpha * o.acc[1];
           hown[g * L.max_nd + rl] = h0; hown[g * L.max_nd + rl + 1] = h1;
           st_relaxed_u64(ll_h + (size_t)g * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
         }
         if (has1) {
-          const float h0 = bf_lo(xw1) + p.alpha * acc[2], h1 = bf_hi(xw1) + p.alpha * acc[3];
+          const float h0 = bf_lo(xw1) + p.alpha * o.acc[2], h1 = bf_hi(xw1) + p.alpha * o.acc[3];
           hown[(g + 8) * L.max_nd + rl] = h0; hown[(g + 8) * L.max_nd + rl + 1] = h1;
           st_relaxed_u64(ll_h + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
         }
       }
     }
-    // ---------------- W_up: g = GELU(W_up RMS(h)) ----------------
+    phase_done(1);
+    // ---------------- W_up: g = GELU(W_up RMS(h)), published as packed bf16 ----------------
     for (int t0n = 0; t0n < nt_f; t0n += kNT) {
-      NTile tl[kNT];
-      make_tiles(tl, s_wup, L.stride_d, nf, t0n);
-      const int ntl = nt_f - t0n < kNT ? nt_f - t0n : kNT;
+      set_tiles(s_wup, L.stride_d, nf, t0n);
+      ds.act = ll_h; ds.K = d; ds.stride = L.stride_d;
+      ds.gain = pre ? reinterpret_cast<const __nv_bfloat16*>(p.g_mlp) : nullptr; ds.want_ssq = pre ? 1 : 0;
+      ds.n_tiles = nt_f - t0n < kNT ? nt_f - t0n : kNT;
       const int rl = (t0n + warp) * 8 + 2 * c;
-      if (!mma_phase<MB>(ll_h, d, L.stride_d, seq, B, tl, ntl, pre ? g_mlp : nullptr, pre, red, ssq_red, s_abort, p.sync,
-                         acc, sl, sh))
-        return;
-      if (warp < ntl && rl < nf) {
+      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
+      if (!o.ok) return;
+      if (warp < ds.n_tiles && rl < nf) {
         if (has0) {
-          const float rs = pre ? rsqrtf(sl * inv_d + p.eps) : 1.0f;
-          st_relaxed_u64(ll_g + (size_t)g * (dff / 2) + (f_lo + rl) / 2,
-                         pack_bf2(gelu_erf_f(acc[0] * rs), gelu_erf_f(acc[1] * rs)), seq);
+          const float rs = pre ? rsqrtf(o.ssq_lo * inv_d + p.eps) : 1.0f;
+          *reinterpret_cast<unsigned*>(g_pk + (size_t)g * dff + f_lo + rl) =
+              pack_bf2(gelu_erf_f(o.acc[0] * rs), gelu_erf_f(o.acc[1] * rs));
         }
         if (has1) {
-          const float rs = pre ? rsqrtf(sh * inv_d + p.eps) : 1.0f;
-          st_relaxed_u64(ll_g + (size_t)(g + 8) * (dff / 2) + (f_lo + rl) / 2,
-                         pack_bf2(gelu_erf_f(acc[2] * rs), gelu_erf_f(acc[3] * rs)), seq);
+          const float rs = pre ? rsqrtf(o.ssq_hi * inv_d + p.eps) : 1.0f;
+          *reinterpret_cast<unsigned*>(g_pk + (size_t)(g + 8) * dff + f_lo + rl) =
+              pack_bf2(gelu_erf_f(o.acc[2] * rs), gelu_erf_f(o.acc[3] * rs));
         }
       }
     }
+    phase_done(2);
+    // every CTA's slice of g must be complete before anyone multiplies by W_down
+    bar_target += (unsigned)G;
+    if (!mma_grid_barrier(sh, bar_target)) return;
+    if (timing) wait_ns = globaltimer_ns() - t_ph;
     // ---------------- W_down: z_t = h + alpha W_down g ----------------
     for (int t0n = 0; t0n < nt_d; t0n += kNT) {
-      NTile tl[kNT];
-      make_tiles(tl, s_wdn, L.stride_f, nd, t0n);
-      const int ntl = nt_d - t0n < kNT ? nt_d - t0n : kNT;
+      set_tiles(s_wdn, L.stride_f, nd, t0n);
+      ds.act = g_pk; ds.K = dff; ds.stride = L.stride_f; ds.gain = nullptr; ds.want_ssq = 0;
+      ds.n_tiles = nt_d - t0n < kNT ? nt_d - t0n : kNT;
       const int rl = (t0n + warp) * 8 + 2 * c;
-      if (!mma_phase<MB>(ll_g, dff, L.stride_f, seq, B, tl, ntl, nullptr, false, red, ssq_red, s_abort, p.sync, acc, sl, sh))
-        return;
-      if (warp < ntl && rl < nd) {
+      const PhaseOut o = mma_phase_packed<MB>(ds, sh);
+      if (!o.ok) return;
+      if (warp < ds.n_tiles && rl < nd) {
         if (has0) {
-          const float z0 = hown[g * L.max_nd + rl] + p.alpha * acc[0], z1 = hown[g * L.max_nd + rl + 1] + p.alpha * acc[1];
+          const float z0 = hown[g * L.max_nd + rl] + p.alpha * o.acc[0], z1 = hown[g * L.max_nd + rl + 1] + p.alpha * o.acc[1];
           const unsigned zw = pack_bf2(z0, z1);
           *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
           st_relaxed_u64(ll_z + (size_t)g * (d / 2) + (d_lo + rl) / 2, zw, seq);
         }
         if (has1) {
-          const float z0 = hown[(g + 8) * L.max_nd + rl] + p.alpha * acc[2];
-          const float z1 = hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * acc[3];
+          const float z0 = hown[(g + 8) * L.max_nd + rl] + p.alpha * o.acc[2];
+          const float z1 = hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * o.acc[3];
           const unsigned zw = pack_bf2(z0, z1);
           *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
           st_relaxed_u64(ll_z + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, zw, seq);
         }
       }
     }
+    phase_done(3);
     // ---------------- W_k, W_v: raw k_t and v_t from RMS(z_t) (Eqs. 1-2; qkRMS is applied by the attention warp) ----
     for (int t0n = 0; t0n < 2 * nt_d; t0n += kNT) {
-      NTile tl[kNT];
 #pragma unroll
       for (int i = 0; i < kNT; ++i) {
         const int ti = t0n + i;
         const bool is_v = ti >= nt_d;
         const int r0 = (is_v ? ti - nt_d : ti) * 8;
-        tl[i].w = (is_v ? s_wv : s_wk) + (size_t)(r0 < nd ? r0 : 0) * L.stride_d;
-        tl[i].valid = nd - r0 < 8 ? (nd - r0 > 0 ? nd - r0 : 1) : 8;
+        ds.w[i] = (is_v ? s_wv : s_wk) + (size_t)(r0 < nd ? r0 : 0) * L.stride_d;
+        ds.valid[i] = nd - r0 < 8 ? (nd - r0 > 0 ? nd - r0 : 1) : 8;
       }
-      const int ntl = 2 * nt_d - t0n < kNT ? 2 * nt_d - t0n : kNT;
-      if (!mma_phase<MB>(ll_z, d, L.stride_d, seq, B, tl, ntl, kv_norm ? g_kv : nullptr, kv_norm, red, ssq_red, s_abort,
-                         p.sync, acc, sl, sh))
-        return;
+      ds.act = ll_z; ds.K = d; ds.stride = L.stride_d;
+      ds.gain = kv_norm ? reinterpret_cast<const __nv_bfloat16*>(p.g_kv) : nullptr; ds.want_ssq = kv_norm ? 1 : 0;
+      ds.n_tiles = 2 * nt_d - t0n < kNT ? 2 * nt_d - t0n : kNT;
+      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
+      if (!o.ok) return;
       const int ti = t0n + warp;
       const bool is_v = ti >= nt_d;
       const int rl = (is_v ? ti - nt_d : ti) * 8 + 2 * c;
-      if (warp < ntl && rl < nd) {
+      if (warp < ds.n_tiles && rl < nd) {
         const size_t col = (size_t)(is_v ? d : 0) + d_lo + rl;
         if (has0) {
-          const float rs = kv_norm ? rsqrtf(sl * inv_d + p.eps) : 1.0f;
-          st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(acc[0] * rs), seq, __float_as_uint(acc[1] * rs), seq);
+          const float rs = kv_norm ? rsqrtf(o.ssq_lo * inv_d + p.eps) : 1.0f;
+          st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(o.acc[0] * rs), seq, __float_as_uint(o.acc[1] * rs), seq);
         }
         if (has1) {
-          const float rs = kv_norm ? rsqrtf(sh * inv_d + p.eps) : 1.0f;
-          st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(acc[2] * rs), seq,
-                        __float_as_uint(acc[3] * rs), seq);
+          const float rs = kv_norm ? rsqrtf(o.ssq_hi * inv_d + p.eps) : 1.0f;
+          st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(o.acc[2] * rs), seq,
+                        __float_as_uint(o.acc[3] * rs), seq);
         }
       }
     }
+    phase_done(4);
+  }
+  if (timing) {
+#pragma unroll
+    for (int i = 2; i < 10; ++i) atomicAdd(&p.sync->phase_ns[i], ph_ns[i]);
   }
 }
 
