@@ -118,6 +118,30 @@ rt_status rt_layer_decode_step(const rt_config *cfg, const rt_layer_weights *w,
                                void *z, void *k_cache, void *v_cache, int32_t N_max,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The single-layer decode step for callers that cannot allocate device memory (the paper has
+ * no counterpart: this is a packaging variant of rt_layer_decode_step, same arithmetic).
+ * Meant for hosts that are handed their input and output buffers and nothing else, that run
+ * where cudaMalloc is forbidden (it synchronises the device), or whose memory is fully
+ * committed to K/V caches.  Instead of a caller-owned workspace it uses a scratch array of
+ * RT_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the library
+ * holds those bytes until the process exits.
+ *  - x, z, k_cache, v_cache, N_max, pos: exactly as for rt_layer_decode_step.
+ *  - Shapes whose rt_workspace_bytes(cfg, B, 1, 1) exceeds RT_STATIC_SCRATCH_BYTES are rejected
+ *    with RT_ERR_WORKSPACE before anything is enqueued.
+ *  - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - The first call on a device looks up the scratch array's device address (with that device
+ *    current); make that first call before any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's contents; the
+ *    words that must start from zero are cleared on the stream at the start of each call.  Two
+ *    calls that overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ *  - The device status word of such a call lives in the built-in scratch and cannot be read
+ *    back through rt_get_status; use the workspace variant where that matters. */
+#define RT_STATIC_SCRATCH_BYTES (8u << 20)
+rt_status rt_layer_decode_step_static(const rt_config *cfg, const rt_layer_weights *w,
+                                      const void *x, int32_t B, int32_t pos,
+                                      void *z, void *k_cache, void *v_cache, int32_t N_max,
+                                      void *cuda_stream);
+
 /* After the caller synchronised the stream: copies the device status word of `workspace`
  * back (a blocking 4-byte copy) and returns it (RT_OK or RT_ERR_TIMEOUT). */
 rt_status rt_get_status(const void *workspace);

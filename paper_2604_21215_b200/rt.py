@@ -25,7 +25,8 @@ RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
-           "rt_profile_enable", "rt_profile_read")
+           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static")
+RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class RtConfig(C.Structure):
@@ -66,6 +67,8 @@ def _load():
     lib.rt_layer_prefill.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P, Z, P]
     lib.rt_layer_decode_step.restype = C.c_int
     lib.rt_layer_decode_step.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P, Z, P]
+    lib.rt_layer_decode_step_static.restype = C.c_int
+    lib.rt_layer_decode_step_static.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P]
     lib.rt_stack_prefill.restype = C.c_int
     lib.rt_stack_prefill.argtypes = [C.POINTER(RtConfig), I, C.POINTER(RtLayerWeights), P, P, I, P, I, I, P, P,
                                      C.POINTER(P), C.POINTER(P), I, P, Z, P]
@@ -119,6 +122,12 @@ def rt_layer_prefill(cfg, w, x, B, N, z, k_cache, v_cache, N_max, workspace, wor
 def rt_layer_decode_step(cfg, w, x, B, pos, z, k_cache, v_cache, N_max, workspace, workspace_bytes, stream) -> int:
     return _lib.rt_layer_decode_step(C.byref(cfg), C.byref(w), x, B, pos, z, k_cache, v_cache, N_max, workspace,
                                      workspace_bytes, stream)
+
+
+def rt_layer_decode_step_static(cfg, w, x, B, pos, z, k_cache, v_cache, N_max, stream) -> int:
+    """Decode step for callers that cannot allocate: no workspace argument, the scratch is a fixed
+    array inside the library (see include/rt.h).  Calls on one device must not overlap."""
+    return _lib.rt_layer_decode_step_static(C.byref(cfg), C.byref(w), x, B, pos, z, k_cache, v_cache, N_max, stream)
 
 
 def rt_stack_prefill(cfg, n_layers, layers, emb, g_final, vocab, ids, B, N, hidden, logits_last, k_caches, v_caches,
