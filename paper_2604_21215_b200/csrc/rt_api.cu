@@ -116,7 +116,7 @@ struct CallCtx { cudaStream_t s; unsigned bar_base = 0; unsigned seq_base = 0; }
 // One layer on position-major scratch; x / z given with explicit strides.
 rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x, long long x_bs, long long x_ts,
                     void* z, long long z_bs, long long z_ts, int B, int n_rows, int pos0, void* k_cache,
-                    void* v_cache, unsigned char* ws, const WsLayout& L, CallCtx& ctx) {
+                    void* v_cache, int n_max, unsigned char* ws, const WsLayout& L, CallCtx& ctx) {
   // n_rows positions starting at cache position pos0 (prefill: pos0 = 0; decode: n_rows = 1)
   cudaStream_t s = ctx.s;
   const float scale_log2 = c->softmax_scale * kLog2e;
@@ -191,6 +191,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2;
   tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
   tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
+  tp.rows_q = n_rows; tp.rows_kv = n_max; tp.sync = lp.sync;
   const int Lf = use_mma ? ml.leaf : leaf_size(c), N = n_rows;
   for (int s0 = 0; s0 < N; s0 += Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
@@ -236,7 +237,7 @@ rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, cons
   if (cudaMemsetAsync(ws + L.ll, 0, L.ll_bytes, s) != cudaSuccess) return RT_ERR_CUDA;
   const long long d = cfg->d_model;
   CallCtx ctx{s};
-  return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, ws, L, ctx);
+  return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, N_max, ws, L, ctx);
 }
 
 rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t pos,
@@ -255,7 +256,7 @@ rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, 
   rt_config c = *cfg;
   c.sched = RT_SCHED_NAIVE;
   CallCtx ctx{s};
-  return run_layer(&c, w, x, d, d, z, d, d, B, 1, pos, k_cache, v_cache, ws, L, ctx);
+  return run_layer(&c, w, x, d, d, z, d, d, B, 1, pos, k_cache, v_cache, N_max, ws, L, ctx);
 }
 
 rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_layer_weights* layers, const void* emb,
@@ -287,7 +288,7 @@ rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_laye
   for (int l = 0; l < n_layers; ++l) {
     void* out = (l == n_layers - 1 && hidden) ? hidden : bufs[(l + 1) & 1];
     st = run_layer(cfg, &layers[l], cur, (long long)N * d, d, out, (long long)N * d, d, B, N, 0, k_caches[l],
-                   v_caches[l], ws, L, ctx);
+                   v_caches[l], N_max, ws, L, ctx);
     if (st != RT_OK) return st;
     cur = out;
   }
@@ -329,7 +330,7 @@ rt_status rt_decode_step(const rt_config* cfg, int32_t n_layers, const rt_layer_
   const void* cur = bufs[0];
   for (int l = 0; l < n_layers; ++l) {
     void* out = bufs[(l + 1) & 1];
-    st = run_layer(&c, &layers[l], cur, d, d, out, d, d, B, 1, pos, k_caches[l], v_caches[l], ws, L, ctx);
+    st = run_layer(&c, &layers[l], cur, d, d, out, d, d, B, 1, pos, k_caches[l], v_caches[l], N_max, ws, L, ctx);
     if (st != RT_OK) return st;
     cur = out;
   }

@@ -69,8 +69,12 @@ struct TileParams {
   const void *k_cache, *v_cache;                 // [N_max, B, d]
   float *st_o, *st_m, *st_l;
   int q0, q1, k0, k1;
+  int rows_q, rows_kv;                           // rows held by the query buffer / the caches (tensor-map bounds)
+  SyncArea* sync;
 };
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s);
+// tensor-core version (bf16, key count a multiple of 64)
+cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s);
 
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,

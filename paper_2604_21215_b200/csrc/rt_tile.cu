@@ -93,6 +93,10 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
 }
 
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  // Whole 64-key blocks only on the tensor-core path: a partial block would bring cache rows that
+  // are not revealed yet (arbitrary bits) into the P.V product.
+  if (dtype == RT_BF16 && (p.k1 - p.k0) % 64 == 0 && p.d % kHeadDim == 0)
+    return tile_tc_launch(p, p.rows_q, p.rows_kv, p.sync, s);
   return tile_simt_launch(dtype, p, s);
 }
 
