@@ -44,7 +44,7 @@ inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsign
 
 // bf16 / tiled-schedule leaf kernel (tensor-core mat-vecs, flag-carrying exchange words).
 struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
-struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [B,d/2] x3, [B,dff/2], [B,2d] words
+struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [16,d/2] words x3, packed bf16 [B,dff], [B,2d] words
 bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out);
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s);
 

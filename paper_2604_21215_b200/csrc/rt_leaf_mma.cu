@@ -109,18 +109,13 @@ __device__ __forceinline__ bool wait_expired(SyncArea* s, unsigned long long& t_
 }
 
 // What one mat-vec phase works on.  Tiles are groups of 8 weight rows in shared memory.
-struct PhaseDesc {
-  const void* act;                 // LL mode: [B][K/2] flag-carrying words; packed mode: [B][K] bf16
-  int K, stride;                   // reduction length, shared-memory row stride of the weights (elements)
-  unsigned seq;                    // flag value of this step (LL mode)
-  int B, n_tiles;
-  const __nv_bfloat16* w[kNT];     // first row of each tile
-  int valid[kNT];                  // rows that exist in each tile (1..8); the rest repeat the last one
-  const __nv_bfloat16* gain;       // optional per-k gain
-  int want_ssq;
-};
-struct PhaseOut { float acc[4]; float ssq_lo, ssq_hi; int ok; };
-struct PhaseShared { float4* red; float* ssq_red; volatile int* s_abort; SyncArea* sync; };
+// Exchange words of a [B, K] bf16 vector are stored in the order the MMA fragments are read:
+// [k-step of 16][16 sequence slots][4 groups of 4 k][2 words of 2 k], so that one warp-wide
+// 16-byte load (8 sequences x 4 groups) covers 512 contiguous bytes.  Index of the word that
+// holds elements k, k+1 (k even) of sequence b:
+__device__ __forceinline__ size_t ll_word(int b, int k) {
+  return ((size_t)((k >> 4) * 16 + b) * 4 + ((k & 15) >> 2)) * 2 + ((k & 3) >> 1);
+}
 
 // Sum of squares (of the raw values) and optional gain for one k-step of fragments; gp points
 // at this thread's 4 gains of the k-step (or is null).
@@ -140,206 +135,21 @@ __device__ __forceinline__ void frag_ssq_gain(unsigned (&a)[4], const __nv_bfloa
   }
 }
 
-// Per-thread shared-memory address of its 8 bytes of weight row g (clamped) of each tile at k = 4c.
-__device__ __forceinline__ void weight_ptrs(const PhaseDesc& ds, int g, int c, const unsigned char* (&wp)[kNT]) {
-#pragma unroll
-  for (int nt = 0; nt < kNT; ++nt) {
-    const int v = ds.valid[nt];
-    const int r = g < v ? g : v - 1;
-    wp[nt] = reinterpret_cast<const unsigned char*>(ds.w[nt < ds.n_tiles ? nt : 0] + (size_t)r * ds.stride + 4 * c);
-  }
-}
-
-// Tail shared by both input modes: reduce the K split over the 8 MMA warps.  Afterwards warp nt
-// (< n_tiles) holds the sums of n-tile nt: acc[0], acc[1] = weight rows 2c, 2c+1 for sequence g,
-// acc[2], acc[3] = the same rows for sequence g+8; ssq_lo / ssq_hi = sum_k act[g or g+8, k]^2.
-__device__ __noinline__ PhaseOut mma_reduce(const float (&acc)[kNT][4], float sq0, float sq1, int n_tiles, int want_ssq,
-                                            const PhaseShared sh) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, c = lane & 3;
-#pragma unroll
-  for (int nt = 0; nt < kNT; ++nt)
-    if (nt < n_tiles) sh.red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
-  if (want_ssq) {
-    sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
-    sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
-    if (c == 0) { sh.ssq_red[warp * 16 + g] = sq0; sh.ssq_red[warp * 16 + 8 + g] = sq1; }
-  }
-  mma_warps_sync();
-  PhaseOut o;
-  o.ok = (*sh.s_abort == 0);
-  o.acc[0] = o.acc[1] = o.acc[2] = o.acc[3] = 0.f;
-  o.ssq_lo = o.ssq_hi = 0.f;
-  if (warp < n_tiles) {
-#pragma unroll
-    for (int w = 0; w < kMmaWarps; ++w) {
-      const float4 v = sh.red[(w * kNT + warp) * 32 + lane];
-      o.acc[0] += v.x; o.acc[1] += v.y; o.acc[2] += v.z; o.acc[3] += v.w;
-    }
-    if (want_ssq) {
-#pragma unroll
-      for (int w = 0; w < kMmaWarps; ++w) { o.ssq_lo += sh.ssq_red[w * 16 + g]; o.ssq_hi += sh.ssq_red[w * 16 + 8 + g]; }
-    }
-  }
-  mma_warps_sync();       // red / ssq_red may be overwritten by the next phase from here on
-  return o;
-}
-
-// One mat-vec phase, activations polled from flag-carrying words: y[b, row] = sum_k W[row, k] act[b, k].
-// MB = 1: B <= 8, MB = 2: B <= 16.  Kept out of line so that the four phases of a token step share
-// one copy of the code (the step runs once per token: straight-line copies thrash the instruction cache).
-template <int MB>
-__device__ __noinline__ PhaseOut mma_phase_ll(const PhaseDesc& ds, const PhaseShared sh, unsigned long long* wait_ns) {
-  constexpr int KC = 8;                                       // k-steps per chunk
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, c = lane & 3;
-  const int K = ds.K, B = ds.B;
-  const unsigned seq = ds.seq;
-  const int n_ks = K / 16;
-  const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
-  const int ks0 = warp * ks_per_warp;
-  const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
-  float acc[kNT][4];
-#pragma unroll
-  for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-  float sq0 = 0.f, sq1 = 0.f;
-  const bool row0 = g < B, row1 = (MB == 2) && (g + 8 < B);
-  const unsigned long long* ll = reinterpret_cast<const unsigned long long*>(ds.act);
-  const unsigned long long* base0 = ll + (size_t)g * (K / 2) + 2 * c;
-  const unsigned long long* base1 = ll + (size_t)(g + 8) * (K / 2) + 2 * c;
-  bool alive = true;
-  const unsigned char* wp[kNT];
-  weight_ptrs(ds, g, c, wp);
-  const __nv_bfloat16* gp = ds.gain ? ds.gain + 4 * c : nullptr;
-  const int n_tiles = ds.n_tiles, want_ssq = ds.want_ssq;
-
-  for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
-    unsigned a[KC][4];
-#pragma unroll
-    for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
-    // a k-step is 8 words per sequence; this thread takes the 2 adjacent ones at 4c
-    unsigned need0 = 0, need1 = 0;
-#pragma unroll
-    for (int i = 0; i < KC; ++i) {
-      if (kc0 + i < ks1) { if (row0) need0 |= 1u << i; if (row1) need1 |= 1u << i; }
-    }
-    unsigned spins = 0;
-    unsigned long long t_start = 0;
-    const unsigned long long t_poll = wait_ns ? globaltimer_ns() : 0ull;
-    while (alive) {
-#pragma unroll
-      for (int i = 0; i < KC; ++i) {
-        if (need0 & (1u << i)) {
-          const uint4 w = ld_relaxed_v4(base0 + (size_t)(kc0 + i) * 8);
-          if (w.y == seq && w.w == seq) { a[i][0] = w.x; a[i][2] = w.z; need0 &= ~(1u << i); }
-        }
-      }
-      if (MB == 2) {
-#pragma unroll
-        for (int i = 0; i < KC; ++i) {
-          if (need1 & (1u << i)) {
-            const uint4 w = ld_relaxed_v4(base1 + (size_t)(kc0 + i) * 8);
-            if (w.y == seq && w.w == seq) { a[i][1] = w.x; a[i][3] = w.z; need1 &= ~(1u << i); }
-          }
-        }
-      }
-      if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
-      if ((++spins & 63u) == 0u) {
-        int bad = 0;
-        if (lane == 0) bad = wait_expired(sh.sync, t_start) ? 1 : 0;
-        if (__shfl_sync(0xffffffffu, bad, 0)) { *sh.s_abort = 1; alive = false; }
-      }
-    }
-    if (wait_ns) *wait_ns += globaltimer_ns() - t_poll;
-    const unsigned char* wc[kNT];
-#pragma unroll
-    for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
-    const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
-#pragma unroll
-    for (int i = 0; i < KC; ++i) {
-      if (kc0 + i < ks1) {
-        if (want_ssq || gp) frag_ssq_gain<MB>(a[i], gc ? gc + i * 16 : nullptr, sq0, sq1);
-#pragma unroll
-        for (int nt = 0; nt < kNT; ++nt) {
-          if (nt < n_tiles) {
-            const uint2 b = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
-            mma_bf16(acc[nt], a[i], b.x, b.y);
-          }
-        }
-      }
-    }
-  }
-  return mma_reduce(acc, sq0, sq1, n_tiles, want_ssq, sh);
-}
-
-// The same product with the activations read as plain packed bf16 ([B][K]) after a grid barrier:
-// used for the wide vector (K = d_ff), where doubling the bytes with flags costs more than it saves.
-// No norm or gain on this input (it is the GELU output).
-// All loads of a round are issued before the first product.
-template <int MB>
-__device__ __noinline__ PhaseOut mma_phase_packed(const PhaseDesc& ds, const PhaseShared sh) {
-  constexpr int KC = 32 / MB;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int g = lane >> 2, c = lane & 3;
-  const int K = ds.K, B = ds.B;
-  const int n_ks = K / 16;
-  const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
-  const int ks0 = warp * ks_per_warp;
-  const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
-  float acc[kNT][4];
-#pragma unroll
-  for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-  const bool row0 = g < B, row1 = (MB == 2) && (g + 8 < B);
-  const __nv_bfloat16* act = reinterpret_cast<const __nv_bfloat16*>(ds.act);
-  const __nv_bfloat16* base0 = act + (size_t)g * K + 4 * c;
-  const __nv_bfloat16* base1 = act + (size_t)(g + 8) * K + 4 * c;
-  const unsigned char* wp[kNT];
-  weight_ptrs(ds, g, c, wp);
-  const int n_tiles = ds.n_tiles;
-  for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
-    unsigned a[KC][4];
-#pragma unroll
-    for (int i = 0; i < KC; ++i) {
-      a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u;
-      if (kc0 + i < ks1) {
-        if (row0) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(base0 + (size_t)(kc0 + i) * 16)); a[i][0] = w.x; a[i][2] = w.y; }
-        if (row1) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(base1 + (size_t)(kc0 + i) * 16)); a[i][1] = w.x; a[i][3] = w.y; }
-      }
-    }
-    const unsigned char* wc[kNT];
-#pragma unroll
-    for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
-#pragma unroll
-    for (int i = 0; i < KC; ++i) {
-      if (kc0 + i < ks1) {
-#pragma unroll
-        for (int nt = 0; nt < kNT; ++nt) {
-          if (nt < n_tiles) {
-            const uint2 b = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
-            mma_bf16(acc[nt], a[i], b.x, b.y);
-          }
-        }
-      }
-    }
-  }
-  return mma_reduce(acc, 0.f, 0.f, n_tiles, 0, sh);
-}
-
 // Barrier over all CTAs, run by the MMA warps only (the attention warps never wait on it).
-__device__ __noinline__ bool mma_grid_barrier(const PhaseShared sh, unsigned target) {
+__device__ __forceinline__ bool mma_grid_barrier(SyncArea* sync, volatile int* s_abort, unsigned target) {
   mma_warps_sync();
   if (threadIdx.x == 0) {
     __threadfence();
-    red_release_add_u32(&sh.sync->bar_count, 1u);
+    red_release_add_u32(&sync->bar_count, 1u);
     unsigned spins = 0;
     unsigned long long t_start = 0;
-    while (ld_acquire_u32(&sh.sync->bar_count) < target) {
-      if ((++spins & 255u) == 0u && wait_expired(sh.sync, t_start)) { *sh.s_abort = 1; break; }
+    while (ld_acquire_u32(&sync->bar_count) < target) {
+      if ((++spins & 255u) == 0u && wait_expired(sync, t_start)) { *s_abort = 1; break; }
     }
     __threadfence();
   }
   mma_warps_sync();
-  return *sh.s_abort == 0;
+  return *s_abort == 0;
 }
 
 // ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
@@ -377,7 +187,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   __syncwarp();
   const float gk0 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane) : 1.0f;
   const float gk1 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane + 1) : 1.0f;
-  unsigned long long* c_word = ll_c + (size_t)b * (d / 2) + h * (kHeadDim / 2) + lane;
+  unsigned long long* c_word = ll_c + ll_word(b, h * kHeadDim + 2 * lane);
   // c of the first position: nothing of this leaf to fold in
   {
     const float il = 1.0f / ls[0];
@@ -507,6 +317,11 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   }
 
   // ------------------------------ MMA warps ------------------------------
+  // The four mat-vec phases of a token step run through ONE inlined copy of the code below (a loop
+  // over the phase index): the step executes once per token, so four straight-line copies would
+  // only thrash the instruction cache, and calls through a real function would put the fragments
+  // and accumulators on the stack, where every access is an L2 round trip.
+  constexpr int KC = 8;                                          // k-steps per round of loads
   const int g = lane >> 2, c = lane & 3;
   const bool pre = (p.norm_flags & RT_NORM_PRE) != 0;
   const bool kv_norm = pre && !(p.norm_flags & RT_NORM_SKIP_Z);
@@ -516,152 +331,241 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   const float inv_d = 1.0f / (float)d;
   const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
   const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
-  const PhaseShared sh{red, ssq_red, s_abort, p.sync};
   unsigned bar_target = p.bar_base;
-
-  PhaseDesc ds;
-  ds.B = B;
-  auto set_tiles = [&](const __nv_bfloat16* w, int stride, int nrows, int first_tile) {
-#pragma unroll
-    for (int i = 0; i < kNT; ++i) {
-      const int r0 = (first_tile + i) * 8;
-      ds.w[i] = w + (size_t)(r0 < nrows ? r0 : 0) * stride;
-      ds.valid[i] = nrows - r0 < 8 ? (nrows - r0 > 0 ? nrows - r0 : 1) : 8;
-    }
-  };
   const bool timing = (cta == 0 && tid == 0);
-  unsigned long long ph_ns[10], wait_ns = 0;
-#pragma unroll
-  for (int i = 0; i < 10; ++i) ph_ns[i] = 0ull;
   unsigned long long t_ph = timing ? globaltimer_ns() : 0ull;
-  auto phase_done = [&](int i) {
-    if (timing) {
-      const unsigned long long now = globaltimer_ns();
-      ph_ns[2 * i] += now - t_ph - wait_ns; ph_ns[2 * i + 1] += wait_ns;
-      t_ph = now; wait_ns = 0;
-    }
-  };
 
   for (int t = p.t0; t < p.t1; ++t) {
-    ds.seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
-    const unsigned seq = ds.seq;
+    const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
+#pragma unroll 1
+    for (int ph = 0; ph < 4; ++ph) {                              // 0: W_o   1: W_up   2: W_down   3: W_k | W_v
+      // ---- what this phase multiplies ----
+      const int K = (ph == 2) ? dff : d;
+      const int stride = (ph == 2) ? L.stride_f : L.stride_d;
+      const int nrows = (ph == 1) ? nf : nd;                       // rows per matrix of this phase
+      const int nt_one = (ph == 1) ? nt_f : nt_d;
+      const int nt_all = (ph == 3) ? 2 * nt_d : nt_one;
+      const unsigned long long* act_ll = (ph == 0) ? ll_c : ((ph == 1) ? ll_h : ll_z);
+      const __nv_bfloat16* gain = nullptr;
+      bool want_ssq = false;
+      if (ph == 1 && pre) { gain = reinterpret_cast<const __nv_bfloat16*>(p.g_mlp); want_ssq = true; }
+      if (ph == 3 && kv_norm) { gain = reinterpret_cast<const __nv_bfloat16*>(p.g_kv); want_ssq = true; }
+      const __nv_bfloat16* gp = gain ? gain + 4 * c : nullptr;
+      unsigned long long wait_ns = 0;
+      if (ph == 2) {
+        // every CTA's slice of g (packed bf16) must be complete before anyone multiplies by W_down
+        bar_target += (unsigned)G;
+        const unsigned long long tb = timing ? globaltimer_ns() : 0ull;
+        if (!mma_grid_barrier(p.sync, s_abort, bar_target)) return;
+        if (timing) wait_ns += globaltimer_ns() - tb;
+      }
+      const int n_ks = K / 16;
+      const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
+      const int ks0 = warp * ks_per_warp;
+      const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
 
-    // ---------------- W_o: a = W_o c_t, h = x_t + alpha a ----------------
-    for (int t0n = 0; t0n < nt_d; t0n += kNT) {
-      set_tiles(s_wo, L.stride_d, nd, t0n);
-      ds.act = ll_c; ds.K = d; ds.stride = L.stride_d; ds.gain = nullptr; ds.want_ssq = 0;
-      ds.n_tiles = nt_d - t0n < kNT ? nt_d - t0n : kNT;
-      const int rl = (t0n + warp) * 8 + 2 * c;                 // local row pair this thread finishes
-      unsigned xw0 = 0, xw1 = 0;
-      const bool mine = warp < ds.n_tiles && rl < nd;
-      if (mine) {
-        if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
-        if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
-      }
-      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
-      if (!o.ok) return;
-      if (mine) {
-        if (has0) {
-          const float h0 = bf_lo(xw0) + p.alpha * o.acc[0], h1 = bf_hi(xw0) + p.alpha * o.acc[1];
-          hown[g * L.max_nd + rl] = h0; hown[g * L.max_nd + rl + 1] = h1;
-          st_relaxed_u64(ll_h + (size_t)g * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
-        }
-        if (has1) {
-          const float h0 = bf_lo(xw1) + p.alpha * o.acc[2], h1 = bf_hi(xw1) + p.alpha * o.acc[3];
-          hown[(g + 8) * L.max_nd + rl] = h0; hown[(g + 8) * L.max_nd + rl + 1] = h1;
-          st_relaxed_u64(ll_h + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, pack_bf2(h0, h1), seq);
-        }
-      }
-    }
-    phase_done(1);
-    // ---------------- W_up: g = GELU(W_up RMS(h)), published as packed bf16 ----------------
-    for (int t0n = 0; t0n < nt_f; t0n += kNT) {
-      set_tiles(s_wup, L.stride_d, nf, t0n);
-      ds.act = ll_h; ds.K = d; ds.stride = L.stride_d;
-      ds.gain = pre ? reinterpret_cast<const __nv_bfloat16*>(p.g_mlp) : nullptr; ds.want_ssq = pre ? 1 : 0;
-      ds.n_tiles = nt_f - t0n < kNT ? nt_f - t0n : kNT;
-      const int rl = (t0n + warp) * 8 + 2 * c;
-      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
-      if (!o.ok) return;
-      if (warp < ds.n_tiles && rl < nf) {
-        if (has0) {
-          const float rs = pre ? rsqrtf(o.ssq_lo * inv_d + p.eps) : 1.0f;
-          *reinterpret_cast<unsigned*>(g_pk + (size_t)g * dff + f_lo + rl) =
-              pack_bf2(gelu_erf_f(o.acc[0] * rs), gelu_erf_f(o.acc[1] * rs));
-        }
-        if (has1) {
-          const float rs = pre ? rsqrtf(o.ssq_hi * inv_d + p.eps) : 1.0f;
-          *reinterpret_cast<unsigned*>(g_pk + (size_t)(g + 8) * dff + f_lo + rl) =
-              pack_bf2(gelu_erf_f(o.acc[2] * rs), gelu_erf_f(o.acc[3] * rs));
-        }
-      }
-    }
-    phase_done(2);
-    // every CTA's slice of g must be complete before anyone multiplies by W_down
-    bar_target += (unsigned)G;
-    if (!mma_grid_barrier(sh, bar_target)) return;
-    if (timing) wait_ns = globaltimer_ns() - t_ph;
-    // ---------------- W_down: z_t = h + alpha W_down g ----------------
-    for (int t0n = 0; t0n < nt_d; t0n += kNT) {
-      set_tiles(s_wdn, L.stride_f, nd, t0n);
-      ds.act = g_pk; ds.K = dff; ds.stride = L.stride_f; ds.gain = nullptr; ds.want_ssq = 0;
-      ds.n_tiles = nt_d - t0n < kNT ? nt_d - t0n : kNT;
-      const int rl = (t0n + warp) * 8 + 2 * c;
-      const PhaseOut o = mma_phase_packed<MB>(ds, sh);
-      if (!o.ok) return;
-      if (warp < ds.n_tiles && rl < nd) {
-        if (has0) {
-          const float z0 = hown[g * L.max_nd + rl] + p.alpha * o.acc[0], z1 = hown[g * L.max_nd + rl + 1] + p.alpha * o.acc[1];
-          const unsigned zw = pack_bf2(z0, z1);
-          *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
-          st_relaxed_u64(ll_z + (size_t)g * (d / 2) + (d_lo + rl) / 2, zw, seq);
-        }
-        if (has1) {
-          const float z0 = hown[(g + 8) * L.max_nd + rl] + p.alpha * o.acc[2];
-          const float z1 = hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * o.acc[3];
-          const unsigned zw = pack_bf2(z0, z1);
-          *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
-          st_relaxed_u64(ll_z + (size_t)(g + 8) * (d / 2) + (d_lo + rl) / 2, zw, seq);
-        }
-      }
-    }
-    phase_done(3);
-    // ---------------- W_k, W_v: raw k_t and v_t from RMS(z_t) (Eqs. 1-2; qkRMS is applied by the attention warp) ----
-    for (int t0n = 0; t0n < 2 * nt_d; t0n += kNT) {
+      const int tile_step = (ph == 2) ? 1 : kNT;                   // W_down: one tile per pass (see below)
+      for (int t0n = 0; t0n < nt_all; t0n += tile_step) {
+        const int n_tiles = nt_all - t0n < tile_step ? nt_all - t0n : tile_step;
+        // this thread's 8 bytes of weight row g (clamped to the rows that exist) of each tile, at k = 4c
+        const unsigned char* wp[kNT];
 #pragma unroll
-      for (int i = 0; i < kNT; ++i) {
-        const int ti = t0n + i;
-        const bool is_v = ti >= nt_d;
-        const int r0 = (is_v ? ti - nt_d : ti) * 8;
-        ds.w[i] = (is_v ? s_wv : s_wk) + (size_t)(r0 < nd ? r0 : 0) * L.stride_d;
-        ds.valid[i] = nd - r0 < 8 ? (nd - r0 > 0 ? nd - r0 : 1) : 8;
+        for (int i = 0; i < kNT; ++i) {
+          const int ti = t0n + i < nt_all ? t0n + i : t0n;
+          const bool second = (ph == 3) && ti >= nt_d;             // W_v tiles follow the W_k tiles
+          const int r0 = (second ? ti - nt_d : ti) * 8;
+          const int valid = nrows - r0 < 8 ? nrows - r0 : 8;
+          const int r = r0 + (g < valid ? g : valid - 1);
+          const __nv_bfloat16* wbase = (ph == 0) ? s_wo : (ph == 1) ? s_wup : (ph == 2) ? s_wdn : (second ? s_wv : s_wk);
+          wp[i] = reinterpret_cast<const unsigned char*>(wbase + (size_t)r * stride + 4 * c);
+        }
+        // rows this thread finishes after the reduction (warp w finishes tile t0n + w)
+        const int ti_e = t0n + warp;
+        const bool second_e = (ph == 3) && ti_e >= nt_d;
+        const int rl = (second_e ? ti_e - nt_d : ti_e) * 8 + 2 * c;
+        const bool mine = warp < n_tiles && rl < nrows;
+        unsigned xw0 = 0, xw1 = 0;
+        if (ph == 0 && mine) {                                     // x_t for the residual, fetched before the wait
+          if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+          if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+        }
+
+        float acc[kNT][4];
+#pragma unroll
+        for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+        float sq0 = 0.f, sq1 = 0.f;
+        bool alive = true;
+        if (ph == 2) {
+          // W_down reads g as packed bf16 after the barrier: plain loads, and ALL of this warp's
+          // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
+          // pass keeps this at 32 products; the two accumulators halve the dependent chain.
+          constexpr int KD = 32 / MB;
+          const __nv_bfloat16* b0p = g_pk + (size_t)g * K + 4 * c;
+          const __nv_bfloat16* b1p = g_pk + (size_t)(g + 8) * K + 4 * c;
+          for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
+            unsigned ad[KD][4];
+#pragma unroll
+            for (int i = 0; i < KD; ++i) {
+              ad[i][0] = ad[i][1] = ad[i][2] = ad[i][3] = 0u;
+              if (kc0 + i < ks1) {
+                if (has0) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(b0p + (size_t)(kc0 + i) * 16)); ad[i][0] = w.x; ad[i][2] = w.y; }
+                if (has1) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(b1p + (size_t)(kc0 + i) * 16)); ad[i][1] = w.x; ad[i][3] = w.y; }
+              }
+            }
+            const unsigned char* wd = wp[0] + (size_t)kc0 * 32;
+#pragma unroll
+            for (int i = 0; i < KD; ++i) {
+              if (kc0 + i < ks1) {
+                const uint2 bw = *reinterpret_cast<const uint2*>(wd + i * 32);
+                mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
+              }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { acc[0][j] += acc[1][j]; acc[1][j] = 0.f; }
+        } else
+        for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
+          unsigned a[KC][4];
+#pragma unroll
+          for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
+          {
+            // flag-carrying words: a k-step is 8 words per sequence, this thread takes the 2 adjacent ones at 4c
+            const unsigned long long* base0 = act_ll + ll_word(g, 4 * c);          // + 128 words per k-step
+            const unsigned long long* base1 = act_ll + ll_word(g + 8, 4 * c);
+            unsigned need0 = 0, need1 = 0;
+#pragma unroll
+            for (int i = 0; i < KC; ++i) {
+              if (kc0 + i < ks1) { if (has0) need0 |= 1u << i; if (has1) need1 |= 1u << i; }
+            }
+            unsigned spins = 0;
+            unsigned long long t_start = 0;
+            const unsigned long long t_poll = timing ? globaltimer_ns() : 0ull;
+            while (alive) {
+              // issue every outstanding load before looking at any flag, so that the loads of a round overlap
+              uint4 w0[KC];
+#pragma unroll
+              for (int i = 0; i < KC; ++i)
+                if (need0 & (1u << i)) w0[i] = ld_relaxed_v4(base0 + (size_t)(kc0 + i) * 128);
+              unsigned got0 = 0;
+#pragma unroll
+              for (int i = 0; i < KC; ++i)
+                if ((need0 & (1u << i)) && w0[i].y == seq && w0[i].w == seq) { a[i][0] = w0[i].x; a[i][2] = w0[i].z; got0 |= 1u << i; }
+              need0 &= ~got0;
+              if (MB == 2) {
+                uint4 w1[KC];
+#pragma unroll
+                for (int i = 0; i < KC; ++i)
+                  if (need1 & (1u << i)) w1[i] = ld_relaxed_v4(base1 + (size_t)(kc0 + i) * 128);
+                unsigned got1 = 0;
+#pragma unroll
+                for (int i = 0; i < KC; ++i)
+                  if ((need1 & (1u << i)) && w1[i].y == seq && w1[i].w == seq) { a[i][1] = w1[i].x; a[i][3] = w1[i].z; got1 |= 1u << i; }
+                need1 &= ~got1;
+              }
+              if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
+              if ((++spins & 63u) == 0u) {
+                int bad = 0;
+                if (lane == 0) bad = wait_expired(p.sync, t_start) ? 1 : 0;
+                if (__shfl_sync(0xffffffffu, bad, 0)) { *s_abort = 1; alive = false; }
+              }
+            }
+            if (timing) wait_ns += globaltimer_ns() - t_poll;
+          }
+          const unsigned char* wc[kNT];
+#pragma unroll
+          for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
+          const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
+#pragma unroll
+          for (int i = 0; i < KC; ++i) {
+            if (kc0 + i < ks1) {
+              if (want_ssq) frag_ssq_gain<MB>(a[i], gc ? gc + i * 16 : nullptr, sq0, sq1);
+#pragma unroll
+              for (int nt = 0; nt < kNT; ++nt) {
+                if (nt < n_tiles) {
+                  const uint2 bw = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
+                  mma_bf16(acc[nt], a[i], bw.x, bw.y);
+                }
+              }
+            }
+          }
+        }
+        // ---- reduce the K split over the 8 warps; warp w then holds the sums of tile t0n + w ----
+#pragma unroll
+        for (int nt = 0; nt < kNT; ++nt)
+          if (nt < n_tiles) red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+        if (want_ssq) {
+          sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
+          sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
+          if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
+        }
+        mma_warps_sync();
+        if (*s_abort) return;
+        float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f, ssq_lo = 0.f, ssq_hi = 0.f;
+        if (warp < n_tiles) {
+#pragma unroll
+          for (int w = 0; w < kMmaWarps; ++w) {
+            const float4 v = red[(w * kNT + warp) * 32 + lane];
+            y0 += v.x; y1 += v.y; y2 += v.z; y3 += v.w;
+          }
+          if (want_ssq) {
+#pragma unroll
+            for (int w = 0; w < kMmaWarps; ++w) { ssq_lo += ssq_red[w * 16 + g]; ssq_hi += ssq_red[w * 16 + 8 + g]; }
+          }
+        }
+        mma_warps_sync();       // red / ssq_red may be overwritten from here on
+        // ---- epilogue: y0, y1 = rows rl, rl+1 for sequence g; y2, y3 = the same rows for sequence g+8 ----
+        if (mine) {
+          if (ph == 0) {                                            // h = x_t + alpha W_o c_t
+            if (has0) {
+              const float h0 = bf_lo(xw0) + p.alpha * y0, h1 = bf_hi(xw0) + p.alpha * y1;
+              hown[g * L.max_nd + rl] = h0; hown[g * L.max_nd + rl + 1] = h1;
+              st_relaxed_u64(ll_h + ll_word(g, d_lo + rl), pack_bf2(h0, h1), seq);
+            }
+            if (has1) {
+              const float h0 = bf_lo(xw1) + p.alpha * y2, h1 = bf_hi(xw1) + p.alpha * y3;
+              hown[(g + 8) * L.max_nd + rl] = h0; hown[(g + 8) * L.max_nd + rl + 1] = h1;
+              st_relaxed_u64(ll_h + ll_word(g + 8, d_lo + rl), pack_bf2(h0, h1), seq);
+            }
+          } else if (ph == 1) {                                     // g = GELU(W_up RMS(h)), packed bf16
+            if (has0) {
+              const float rs = pre ? rsqrtf(ssq_lo * inv_d + p.eps) : 1.0f;
+              *reinterpret_cast<unsigned*>(g_pk + (size_t)g * dff + f_lo + rl) = pack_bf2(gelu_erf_f(y0 * rs), gelu_erf_f(y1 * rs));
+            }
+            if (has1) {
+              const float rs = pre ? rsqrtf(ssq_hi * inv_d + p.eps) : 1.0f;
+              *reinterpret_cast<unsigned*>(g_pk + (size_t)(g + 8) * dff + f_lo + rl) = pack_bf2(gelu_erf_f(y2 * rs), gelu_erf_f(y3 * rs));
+            }
+          } else if (ph == 2) {                                     // z_t = h + alpha W_down g   (layer output)
+            if (has0) {
+              const unsigned zw = pack_bf2(hown[g * L.max_nd + rl] + p.alpha * y0, hown[g * L.max_nd + rl + 1] + p.alpha * y1);
+              *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              st_relaxed_u64(ll_z + ll_word(g, d_lo + rl), zw, seq);
+            }
+            if (has1) {
+              const unsigned zw = pack_bf2(hown[(g + 8) * L.max_nd + rl] + p.alpha * y2, hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * y3);
+              *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              st_relaxed_u64(ll_z + ll_word(g + 8, d_lo + rl), zw, seq);
+            }
+          } else {                                                  // raw k_t, v_t from RMS(z_t): Eqs. (1)-(2) before qkRMS
+            const size_t col = (size_t)(second_e ? d : 0) + d_lo + rl;
+            if (has0) {
+              const float rs = kv_norm ? rsqrtf(ssq_lo * inv_d + p.eps) : 1.0f;
+              st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(y0 * rs), seq, __float_as_uint(y1 * rs), seq);
+            }
+            if (has1) {
+              const float rs = kv_norm ? rsqrtf(ssq_hi * inv_d + p.eps) : 1.0f;
+              st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(y2 * rs), seq, __float_as_uint(y3 * rs), seq);
+            }
+          }
+        }
       }
-      ds.act = ll_z; ds.K = d; ds.stride = L.stride_d;
-      ds.gain = kv_norm ? reinterpret_cast<const __nv_bfloat16*>(p.g_kv) : nullptr; ds.want_ssq = kv_norm ? 1 : 0;
-      ds.n_tiles = 2 * nt_d - t0n < kNT ? 2 * nt_d - t0n : kNT;
-      const PhaseOut o = mma_phase_ll<MB>(ds, sh, timing ? &wait_ns : nullptr);
-      if (!o.ok) return;
-      const int ti = t0n + warp;
-      const bool is_v = ti >= nt_d;
-      const int rl = (is_v ? ti - nt_d : ti) * 8 + 2 * c;
-      if (warp < ds.n_tiles && rl < nd) {
-        const size_t col = (size_t)(is_v ? d : 0) + d_lo + rl;
-        if (has0) {
-          const float rs = kv_norm ? rsqrtf(o.ssq_lo * inv_d + p.eps) : 1.0f;
-          st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(o.acc[0] * rs), seq, __float_as_uint(o.acc[1] * rs), seq);
-        }
-        if (has1) {
-          const float rs = kv_norm ? rsqrtf(o.ssq_hi * inv_d + p.eps) : 1.0f;
-          st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(o.acc[2] * rs), seq,
-                        __float_as_uint(o.acc[3] * rs), seq);
-        }
+      if (timing) {
+        const unsigned long long now = globaltimer_ns();
+        atomicAdd(&p.sync->phase_ns[2 + 2 * ph], now - t_ph - wait_ns);        // fire-and-forget, no stack array
+        atomicAdd(&p.sync->phase_ns[3 + 2 * ph], wait_ns);
+        t_ph = now;
       }
     }
-    phase_done(4);
-  }
-  if (timing) {
-#pragma unroll
-    for (int i = 2; i < 10; ++i) atomicAdd(&p.sync->phase_ns[i], ph_ns[i]);
   }
 }
 
