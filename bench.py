@@ -38,8 +38,9 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "source": "fallback"}
 
 
-# DRAM bytes (read + write) per leaf launch from the ncu captures summarised under profiles/.
-NCU_LEAF_TRAFFIC = {}
+# DRAM bytes (read + write) of one leaf launch (64 token steps) from the ncu capture summarised in
+# profiles/leaf_mma_kernel_c2.txt: the launch stages its weight rows once, everything else stays in L2.
+NCU_LEAF_TRAFFIC = {"c2": 14701568 + 36864}
 
 
 class ClockSampler:
