@@ -130,6 +130,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   pp.g_attn = w->g_attn; pp.g_q = w->g_q; pp.g_k = w->g_k;
   pp.n = ws + L.n; pp.q = ws + L.q; pp.kt = ws + L.kt; pp.vt = ws + L.vt;
   pp.st_o = (float*)(ws + L.st_o); pp.st_m = (float*)(ws + L.st_m); pp.st_l = (float*)(ws + L.st_l);
+  pp.sync = (SyncArea*)(ws + L.sync);
   {
     ProfScope ps(s, kProfPrepass);
     if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;

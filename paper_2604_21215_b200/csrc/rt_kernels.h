@@ -58,8 +58,12 @@ struct PrepassParams {
   void* n;                                       // [N*B, d] normalised input (scratch)
   void *q, *kt, *vt;                             // [N, B, d]
   float *st_o, *st_m, *st_l;
+  SyncArea* sync;
 };
 cudaError_t prepass_launch(int dtype, const PrepassParams& p, cudaStream_t s);
+// tensor-core projection (bf16, d a multiple of 128)
+bool qkv_gemm_tc_supported(const PrepassParams& p);
+cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStream_t s);
 
 // Cross-block tile (Algorithm 2 on a [q0,q1) x [k0,k1) block for every sequence and head).
 struct TileParams {

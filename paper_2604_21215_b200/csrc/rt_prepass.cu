@@ -6,7 +6,8 @@
 //   (m,l,o) = state after UpdateTile(q_t, k~_t, v~_t) on (-inf, 0, 0): m = s<q,k~>, l = 1, o = v~
 // Folding the temporary pair in here (Algorithm 1 does it as the first step of iteration t) is
 // exact: the online-softmax merge does not depend on the order of the contributions.
-// This file holds the SIMT projection used in fp32 mode and as the generic path.
+// This file holds the SIMT projection used in fp32 mode and as the generic path; bf16 with d a
+// multiple of 128 takes the tensor-core projection in rt_prepass_tc.cu.
 #include "rt_kernels.h"
 
 namespace rt {
@@ -135,8 +136,13 @@ template <typename T>
 static cudaError_t prepass_typed(const PrepassParams& p, cudaStream_t s) {
   const int M = p.N * p.B;
   rms_rows_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(p);
-  dim3 grid(ceil_div(M, kGM), 3 * (p.d / kHeadDim));
-  qkv_gemm_simt_kernel<T><<<grid, 256, 0, s>>>(p);
+  if (sizeof(T) == 2 && qkv_gemm_tc_supported(p)) {
+    const cudaError_t e = qkv_gemm_tc_launch(p, p.sync, s);
+    if (e != cudaSuccess) return e;
+  } else {
+    dim3 grid(ceil_div(M, kGM), 3 * (p.d / kHeadDim));
+    qkv_gemm_simt_kernel<T><<<grid, 256, 0, s>>>(p);
+  }
   const long long units = (long long)M * p.H;
   state_init_kernel<T><<<(unsigned)((units + 7) / 8), 256, 0, s>>>(p);
   return cudaGetLastError();

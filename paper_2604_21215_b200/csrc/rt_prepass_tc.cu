@@ -1,0 +1,196 @@
+// Pre-pass projection on the 5th-generation tensor cores (bf16 storage):
+//   [q | k~ | v~][m, :] = n[m, :] . [W_q | W_k | W_v]^T   with qkRMS per head on q and k~
+// (first display of Sec. 2.2; Algorithm 1 line 1 and the temporary pair of line 7, for all
+// positions at once).  A dense contraction: M = B*N rows, K = d, N = 3d columns.
+//
+// One CTA = a 128 x 128 output tile (two heads of one of the three matrices).  Warp 4 lane 0
+// streams 64-wide K blocks of n and W through a 3-stage TMA ring (128-byte swizzle), warp 5
+// lane 0 issues tcgen05.mma (M=128, N=128, K=16, both operands K-major) into a 128-column TMEM
+// accumulator, warps 0-3 own one output row per thread: tcgen05.ld, sum of squares per head,
+// gain, bf16, 16-byte stores.  Two CTAs per SM, so one tile's epilogue overlaps the other's
+// main loop.  All waits are bounded (see rt_tc.cuh).
+#include "rt_kernels.h"
+#include "rt_tc.cuh"
+
+namespace rt {
+
+constexpr int kGemmBN = 128;
+constexpr int kGemmBK = 64;
+constexpr int kGemmStages = 3;
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kGemmABytes = kBM * kGemmBK * 2;        // 16 KB
+constexpr uint32_t kGemmBBytes = kGemmBN * kGemmBK * 2;    // 16 KB
+
+struct GemmSmem {
+  static constexpr uint32_t a = 0;
+  static constexpr uint32_t b = a + kGemmStages * kGemmABytes;
+  static constexpr uint32_t bars = b + kGemmStages * kGemmBBytes;      // full[3], empty[3], acc_ready
+  static constexpr uint32_t tmem_ptr = bars + 64;
+  static constexpr uint32_t abort_flag = tmem_ptr + 8;
+  static constexpr uint32_t total = abort_flag + 8;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 2)
+qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_constant__ CUtensorMap map_wq,
+                   const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv,
+                   const PrepassParams p, SyncArea* sync) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int M = p.N * p.B, d = p.d;
+  const int tiles_per_mat = d / kGemmBN;
+  const int which = blockIdx.y / tiles_per_mat;             // 0: q, 1: k~, 2: v~
+  const int col0 = (blockIdx.y % tiles_per_mat) * kGemmBN;  // first output column within the matrix
+  const int m0 = blockIdx.x * kBM;
+  const int n_kb = d / kGemmBK;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + GemmSmem::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + GemmSmem::tmem_ptr);
+  auto full = [&](int s) { return sbase + GemmSmem::bars + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return sbase + GemmSmem::bars + 8u * (uint32_t)(kGemmStages + s); };
+  const uint32_t acc_ready = sbase + GemmSmem::bars + 8u * (2 * kGemmStages);
+
+  if (tid == 0) {
+    *s_abort = 0;
+    for (int s = 0; s < kGemmStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    mbar_init(acc_ready, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + GemmSmem::tmem_ptr), "n"(kGemmBN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      const CUtensorMap* mw = which == 0 ? &map_wq : (which == 1 ? &map_wk : &map_wv);
+      int issued = 0;
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kGemmStages;
+        if (kb >= kGemmStages) ok = mbar_wait(empty(s), ((kb / kGemmStages) - 1) & 1, s_abort, sync);
+        if (!ok) break;
+        mbar_expect_tx(full(s), kGemmABytes + kGemmBBytes);
+        tma_load_2d(sbase + GemmSmem::a + s * kGemmABytes, &map_n, full(s), kb * kGemmBK, m0);
+        tma_load_2d(sbase + GemmSmem::b + s * kGemmBBytes, mw, full(s), kb * kGemmBK, col0);
+        ++issued;
+      }
+      if (!ok) {
+        // gave up: let the copies already started land before the shared memory goes away (bounded)
+        for (int i = issued > kGemmStages ? issued - kGemmStages : 0; i < issued; ++i) {
+          unsigned spins = 0;
+          while (!mbar_try_wait(full(i % kGemmStages), (i / kGemmStages) & 1) && ++spins < (1u << 20)) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kGemmBN, false);
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kGemmStages;
+        ok = mbar_wait(full(s), (kb / kGemmStages) & 1, s_abort, sync);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t a0 = make_desc(sbase + GemmSmem::a + s * kGemmABytes, 16, 1024);
+        const uint64_t b0 = make_desc(sbase + GemmSmem::b + s * kGemmBBytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < kGemmBK / 16; ++ks)
+          tc_mma(tmem, a0 + 2u * ks, b0 + 2u * ks, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(empty(s));                       // the stage may be refilled once these products have read it
+      }
+      if (ok) tc_commit(acc_ready);
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue: one output row per thread ----------------
+    const int row = warp * 32 + lane;
+    const int m = m0 + row;
+    const bool qkn = (p.norm_flags & RT_NORM_QK) != 0 && which < 2;
+    const __nv_bfloat16* gain = reinterpret_cast<const __nv_bfloat16*>(which == 0 ? p.g_q : p.g_k);
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.q : (which == 1 ? p.kt : p.vt));
+    if (mbar_wait(acc_ready, 0, s_abort, sync)) {
+      tc_fence_after();
+      const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+      for (int hh = 0; hh < kGemmBN / kHeadDim; ++hh) {        // one head (64 columns) at a time
+        uint32_t v0[32], v1[32];
+        tc_ld32(t_row + (uint32_t)(hh * kHeadDim), v0);
+        tc_ld32(t_row + (uint32_t)(hh * kHeadDim + 32), v1);
+        tc_wait_ld();
+        float rs = 1.0f;
+        if (qkn) {
+          float ss = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float a = __uint_as_float(v0[i]), b = __uint_as_float(v1[i]);
+            ss += a * a + b * b;
+          }
+          rs = rsqrtf(ss * (1.0f / kHeadDim) + p.eps);
+        }
+        if (m < M) {
+          const int c_head = col0 + hh * kHeadDim;
+          uint4* dst = reinterpret_cast<uint4*>(out + (size_t)m * d + c_head);
+#pragma unroll
+          for (int c8 = 0; c8 < 8; ++c8) {                     // 8 columns = 16 bytes per store
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int e = c8 * 8 + 2 * j;
+              float x0 = __uint_as_float(e < 32 ? v0[e & 31] : v1[e & 31]) * rs;
+              float x1 = __uint_as_float(e + 1 < 32 ? v0[(e + 1) & 31] : v1[(e + 1) & 31]) * rs;
+              if (qkn && gain) { x0 *= __bfloat162float(gain[c_head + e]); x1 *= __bfloat162float(gain[c_head + e + 1]); }
+              const __nv_bfloat162 pk = __floats2bfloat162_rn(x0, x1);
+              w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+            }
+            dst[c8] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kGemmBN) : "memory");
+  }
+}
+
+// row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
+static bool make_map_2d(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool qkv_gemm_tc_supported(const PrepassParams& p) { return p.d % kGemmBN == 0 && p.d >= kGemmBN; }
+
+cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStream_t s) {
+  const int M = p.N * p.B;
+  CUtensorMap mn, mq, mk, mv;
+  if (!make_map_2d(&mn, p.n, M, p.d, kBM) || !make_map_2d(&mq, p.w_q, p.d, p.d, kGemmBN) ||
+      !make_map_2d(&mk, p.w_k, p.d, p.d, kGemmBN) || !make_map_2d(&mv, p.w_v, p.d, p.d, kGemmBN))
+    return cudaErrorInvalidValue;
+  const size_t smem = GemmSmem::total + 1024;
+  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(ceil_div(M, kBM), 3 * (p.d / kGemmBN));
+  qkv_gemm_tc_kernel<<<grid, kGemmThreads, smem, s>>>(mn, mq, mk, mv, p, sync);
+  return cudaGetLastError();
+}
+
+}  // namespace rt
