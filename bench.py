@@ -91,11 +91,11 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def get_workload(name):
+def get_workload(name, batch=0):
+    import dataclasses
     from paper_2604_21215_b200 import inputs
-    if name.startswith("c5_N"):
-        return inputs.sweep(int(name[4:]))
-    return inputs.WORKLOADS[name]
+    wl = inputs.sweep(int(name[4:])) if name.startswith("c5_N") else inputs.WORKLOADS[name]
+    return dataclasses.replace(wl, B=batch) if batch else wl
 
 
 def config_dict(wl, sched, extra=None):
@@ -144,7 +144,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     from paper_2604_21215_b200 import inputs
-    wl = get_workload(args.workload)
+    wl = get_workload(args.workload, args.batch)
     data = inputs.make_inputs(wl)
     n_pos = sample_positions(wl)
     for _ in range(min(args.warmup, 1)):
@@ -183,7 +183,7 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = get_workload(args.workload)
+    wl = get_workload(args.workload, args.batch)
     data = inputs.make_inputs(wl)
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     leaf_kw = {"leaf": args.leaf} if args.leaf else {}
@@ -239,6 +239,15 @@ def run_cuda(args):
         call(dev_in2)
         host_out.copy_(result, non_blocking=True)
 
+    if args.profile_one_call:
+        # profiling mode (for ncu byte counters): exactly one call, no warm-up, no bench line
+        call(dev_in)
+        torch.cuda.synchronize(dev)
+        c = rt.rt_plan_counters(model.cfg, wl.B, wl.N, wl.n_layers, wl.vocab)
+        print(json.dumps({"profile_one_call": wl.name, "sched": args.sched, "status": int(model.status()),
+                          "model_bytes": c["model_bytes_read"] + c["model_bytes_written"],
+                          "model_kv_bytes_read": c["kv_bytes_read"], "leaf_kv_bytes_l2": c["leaf_kv_bytes_l2"]}))
+        return 0
     for _ in range(max(args.warmup, 3)):
         call(dev_in)
     torch.cuda.synchronize(dev)
@@ -340,6 +349,9 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--sched", default="tiled", choices=["tiled", "naive"])
     ap.add_argument("--leaf", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
+    ap.add_argument("--profile-one-call", action="store_true",
+                    help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
