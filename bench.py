@@ -340,6 +340,57 @@ def run_cuda(args):
     return 0
 
 
+def run_tile_bench(args):
+    """Times Algorithm 2 alone (rt_update_tile) per tile size, in the shape the workload's prefill uses it:
+    queries [P, 2P) against the pairs [0, P) for all B*H (sequence, head) pairs; prints one JSON object."""
+    import torch
+    from paper_2604_21215_b200 import rt
+    wl = get_workload(args.workload, args.batch)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(
+        os.path.join(ROOT, "MEASURED_PEAKS.json")) else {"bf16_tflops": 1590.0}
+    cfg = rt.make_config(wl.d_model, wl.n_heads, wl.d_ff, dtype=wl.dtype)
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    out = []
+    g = torch.Generator(device=dev); g.manual_seed(BASE_TILE_SEED)
+    for P in (64, 128, 256, 512, 1024, 2048, 4096):
+        if P > wl.N // 2 and not args.tile_bench_all:
+            break
+        rows = 2 * P
+        q = torch.randn((rows, wl.B, wl.d_model), generator=g, device=dev).to(tdt)
+        k = torch.randn((rows, wl.B, wl.d_model), generator=g, device=dev).to(tdt)
+        v = torch.randn((rows, wl.B, wl.d_model), generator=g, device=dev).to(tdt)
+        o = torch.zeros((rows, wl.B, wl.d_model), dtype=torch.float32, device=dev)
+        m = torch.zeros((rows, wl.B, wl.n_heads), dtype=torch.float32, device=dev)
+        l = torch.ones((rows, wl.B, wl.n_heads), dtype=torch.float32, device=dev)
+        call = lambda: rt.rt_update_tile(cfg, q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), m.data_ptr(),
+                                         l.data_ptr(), wl.B, rows, rows, P, 2 * P, 0, P, ws.data_ptr(), stream.cuda_stream)
+        for _ in range(3):
+            assert call() == rt.RT_OK
+        evs = []
+        for _ in range(args.steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); call(); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        assert rt.rt_get_status(ws.data_ptr()) == rt.RT_OK
+        ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+        flops = 4.0 * P * P * 64 * wl.B * wl.n_heads
+        tf = flops / (ms * 1e-3) / 1e12
+        out.append({"P": P, "ms": ms, "tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"]})
+    print(json.dumps({"tile_bench": wl.name, "B": wl.B, "H": wl.n_heads, "dtype": wl.dtype,
+                      "peak_tflops": peaks["bf16_tflops"], "tiles": out}))
+    return 0
+
+
+BASE_TILE_SEED = 20260421
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -352,7 +403,11 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
     ap.add_argument("--profile-one-call", action="store_true",
                     help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
+    ap.add_argument("--tile-bench", action="store_true", help="time Algorithm 2 alone per tile size and exit")
+    ap.add_argument("--tile-bench-all", action="store_true", help="with --tile-bench: also sizes beyond N/2")
     args = ap.parse_args()
+    if args.tile_bench:
+        return run_tile_bench(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_cuda(args)

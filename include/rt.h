@@ -163,6 +163,19 @@ typedef struct {
 rt_status rt_plan_counters(const rt_config *cfg, int32_t B, int32_t N, int32_t n_layers, int32_t vocab,
                            rt_counters *out);
 
+/* Algorithm 2 (UpdateTile, App. C) on its own: queries [q0,q1) of `q` attend to the pairs [k0,k1) of
+ * the caches, for every sequence and head, and their running stats are updated in place:
+ *   m_new = max(m, max_j a_ij),  o = o*e^(m-m_new) + sum_j v_j e^(a_ij-m_new),  l likewise,  m = m_new,
+ * with a_ij = softmax_scale <q_i, k_j>.  The library keeps m in log2 units: st_m holds log2(e)*m.
+ * q [rows_q, B, d] and the caches [rows_kv, B, d] are position-major, storage type; st_o [rows_q, B, d],
+ * st_m, st_l [rows_q, B, n_heads] are fp32.  `workspace` needs 256 bytes (device status word, read with
+ * rt_get_status).  This is the cross-block step of rt_layer_prefill, exposed for tests and benchmarks. */
+rt_status rt_update_tile(const rt_config *cfg, const void *q, const void *k_cache, const void *v_cache,
+                         float *st_o, float *st_m, float *st_l,
+                         int32_t B, int32_t rows_q, int32_t rows_kv,
+                         int32_t q0, int32_t q1, int32_t k0, int32_t k1,
+                         void *workspace, void *cuda_stream);
+
 /* Per-kernel-class timing for benchmarks.  While enabled (a process-wide switch, off by
  * default, and the one piece of global state in the library) every call brackets its launches
  * with CUDA events on the caller's stream: class 0 = pre-pass, 1 = leaf recurrence launches,

@@ -348,6 +348,29 @@ rt_status rt_get_status(const void* workspace) {
   return (rt_status)st;
 }
 
+rt_status rt_update_tile(const rt_config* cfg, const void* q, const void* k_cache, const void* v_cache, float* st_o,
+                         float* st_m, float* st_l, int32_t B, int32_t rows_q, int32_t rows_kv, int32_t q0, int32_t q1,
+                         int32_t k0, int32_t k1, void* workspace, void* cuda_stream) {
+  if (!config_ok(cfg) || B <= 0 || !q || !k_cache || !v_cache || !st_o || !st_m || !st_l || !workspace)
+    return RT_ERR_INVALID_ARG;
+  if (q0 < 0 || q1 < q0 || q1 > rows_q || k0 < 0 || k1 < k0 || k1 > rows_kv) return RT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(st_o) || !aligned16(workspace))
+    return RT_ERR_INVALID_ARG;
+  const rt_status sup = config_supported(cfg, B);
+  if (sup != RT_OK) return sup;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (cudaMemsetAsync(workspace, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  TileParams tp;
+  memset(&tp, 0, sizeof(tp));
+  tp.B = B; tp.d = cfg->d_model; tp.H = cfg->n_heads; tp.scale_log2 = cfg->softmax_scale * kLog2e;
+  tp.q = q; tp.k_cache = k_cache; tp.v_cache = v_cache;
+  tp.st_o = st_o; tp.st_m = st_m; tp.st_l = st_l;
+  tp.q0 = q0; tp.q1 = q1; tp.k0 = k0; tp.k1 = k1;
+  tp.rows_q = rows_q; tp.rows_kv = rows_kv; tp.sync = (SyncArea*)workspace;
+  ProfScope ps(s, kProfTile);
+  return tile_launch(cfg->dtype, tp, s) == cudaSuccess ? RT_OK : RT_ERR_CUDA;
+}
+
 rt_status rt_profile_enable(int32_t on) {
   std::lock_guard<std::mutex> g(g_prof_mu);
   g_prof_on = on != 0;

@@ -3,45 +3,46 @@
 // running stats (m, l, o) carried in fp32 in the workspace.
 //
 // One CTA = 128 query rows of one (sequence, head) pair, looping over 64-key blocks:
-//   TMA     Q tile once, K and V blocks double-buffered, straight out of the position-major
-//           cache / query buffer (a 4-D tensor map picks the head's 64 columns of each row),
-//           128-byte swizzle = the tensor cores' canonical shared-memory layout
-//   S       tcgen05.mma  S[128x64] = Q[128x64] . K^T        (A, B K-major; accumulator in TMEM)
-//   softmax 4 warps, one thread per query row: tcgen05.ld of the row, running max in log2 units,
-//           p = 2^(s - m), row sum, P written to shared memory as bf16 in the swizzled layout
-//   PV      tcgen05.mma  PV[128x64] = P[128x64] . V[64x64]  (B is MN-major: V rows are keys)
-//   merge   o = o * 2^(m_old - m_new) + PV in registers (fp32), l likewise
-// A fifth warp owns TMEM allocation, issues the TMA copies and (one elected lane) the MMAs.
-// Three CTAs fit on an SM (64 KB shared memory, 128 TMEM columns each), so the softmax of one CTA
-// overlaps the MMAs of the others.  Every mbarrier wait is bounded: on expiry the CTA records
-// RT_ERR_TIMEOUT, stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and
-// returns.
+//   TMA     (warp 5) Q tile once, K and V blocks through a 3-stage ring, straight out of the
+//           position-major cache / query buffer (a 4-D tensor map picks the head's 64 columns of
+//           each row), 128-byte swizzle = the tensor cores' canonical shared-memory layout
+//   S       (warp 4) tcgen05.mma  S[128x64] = Q[128x64] . K^T   (A, B K-major; accumulator in TMEM)
+//   softmax (warps 0-3, one thread per query row) tcgen05.ld of the row, running max in log2
+//           units, p = 2^(s - m), row sum, P written to shared memory as bf16 in the swizzled layout
+//   PV      (warp 4) tcgen05.mma  PV[128x64] = P[128x64] . V[64x64]  (B is MN-major: V rows are keys)
+//   merge   o = (o + PV_prev) * 2^(m_old - m_new) in registers (fp32), one block late
+// S and PV are double-buffered in TMEM (256 columns) and the product P.V of block kb is folded
+// into o during block kb+1, so the softmax warps never wait for the tensor cores in steady state:
+// S(kb+1) is issued while softmax(kb) runs and PV(kb) runs under softmax(kb+1).  Two CTAs per SM.
+// Every mbarrier wait is bounded: on expiry the CTA records RT_ERR_TIMEOUT, stops issuing work,
+// waits (bounded) for its copies in flight, frees its TMEM and returns.
 #include "rt_kernels.h"
 #include "rt_tc.cuh"
 
 namespace rt {
 
 constexpr int kBK = 64;                // keys per block
-constexpr int kTcThreads = 160;        // 4 softmax warps + 1 control warp
-constexpr int kTmemCols = 128;         // S: columns [0,64), PV: columns [64,128)
+constexpr int kKvStages = 3;
+constexpr int kTcThreads = 192;        // 4 softmax warps + MMA warp + TMA warp
+constexpr int kTmemCols = 256;         // S0 [0,64) S1 [64,128) PV0 [128,192) PV1 [192,256)
 constexpr uint32_t kQBytes = kBM * kHeadDim * 2;     // 16 KB
 constexpr uint32_t kKVBytes = kBK * kHeadDim * 2;    // 8 KB
 constexpr uint32_t kPBytes = kBM * kBK * 2;          // 16 KB
 
 struct TcSmem {                        // offsets from a 1024-byte aligned base
   static constexpr uint32_t q = 0;
-  static constexpr uint32_t k = q + kQBytes;                 // 2 stages
-  static constexpr uint32_t v = k + 2 * kKVBytes;            // 2 stages
-  static constexpr uint32_t p = v + 2 * kKVBytes;
-  static constexpr uint32_t bars = p + kPBytes;              // 10 mbarriers
+  static constexpr uint32_t k = q + kQBytes;
+  static constexpr uint32_t v = k + kKvStages * kKVBytes;
+  static constexpr uint32_t p = v + kKvStages * kKVBytes;
+  static constexpr uint32_t bars = p + kPBytes;              // 16 mbarriers
   static constexpr uint32_t tmem_ptr = bars + 128;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
-enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 3, BAR_S_READY = 5, BAR_S_FREE = 6, BAR_P_READY = 7,
-       BAR_PV_READY = 8, BAR_PV_FREE = 9 };
+enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 4, BAR_S_READY = 7, BAR_S_FREE = 9, BAR_P_READY = 11,
+       BAR_PV_READY = 12, BAR_PV_FREE = 14 };
 
-__global__ void __launch_bounds__(kTcThreads, 3)
+__global__ void __launch_bounds__(kTcThreads, 2)
 tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const TileParams p, SyncArea* sync) {
   extern __shared__ unsigned char smem_raw[];
@@ -50,8 +51,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
   const int qb = p.q0 + blockIdx.x * kBM;                 // first query row of this CTA
-  const int nk = p.k1 - p.k0;
-  const int n_blocks = (nk + kBK - 1) / kBK;
+  const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + TcSmem::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + TcSmem::tmem_ptr);
   auto bar = [&](int i) { return sbase + TcSmem::bars + 8u * (uint32_t)i; };
@@ -59,13 +59,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (tid == 0) {
     *s_abort = 0;
     mbar_init(bar(BAR_Q), 1);
-    mbar_init(bar(BAR_KV_FULL), 1); mbar_init(bar(BAR_KV_FULL + 1), 1);
-    mbar_init(bar(BAR_KV_EMPTY), 1); mbar_init(bar(BAR_KV_EMPTY + 1), 1);
-    mbar_init(bar(BAR_S_READY), 1);
-    mbar_init(bar(BAR_S_FREE), 4);
+    for (int i = 0; i < kKvStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_S_READY + i), 1); mbar_init(bar(BAR_S_FREE + i), 4);
+      mbar_init(bar(BAR_PV_READY + i), 1); mbar_init(bar(BAR_PV_FREE + i), 4);
+    }
     mbar_init(bar(BAR_P_READY), 4);
-    mbar_init(bar(BAR_PV_READY), 1);
-    mbar_init(bar(BAR_PV_FREE), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {
@@ -77,63 +76,67 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  if (warp == 4) {
-    // ------------------------------ control warp: TMA + MMA issue ------------------------------
+  if (warp == 5) {
+    // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(kBK, false);
-      constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true);
       mbar_expect_tx(bar(BAR_Q), kQBytes);
       tma_load_4d(sbase + TcSmem::q, &map_q, bar(BAR_Q), 0, h, b, qb);
-      mbar_expect_tx(bar(BAR_KV_FULL), 2 * kKVBytes);
-      tma_load_4d(sbase + TcSmem::k, &map_k, bar(BAR_KV_FULL), 0, h, b, p.k0);
-      tma_load_4d(sbase + TcSmem::v, &map_v, bar(BAR_KV_FULL), 0, h, b, p.k0);
-      int loads_issued = 1;                                   // K/V blocks whose copies were started
-      bool ok = mbar_wait(bar(BAR_Q), 0, s_abort, sync);
+      int issued = 0;
+      bool ok = true;
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
-        const int st = kb & 1;
-        ok = mbar_wait(bar(BAR_KV_FULL + st), (kb >> 1) & 1, s_abort, sync);
-        if (ok && kb > 0) ok = mbar_wait(bar(BAR_S_FREE), (kb - 1) & 1, s_abort, sync);
+        const int st = kb % kKvStages;
+        if (kb >= kKvStages) ok = mbar_wait(bar(BAR_KV_EMPTY + st), ((kb / kKvStages) - 1) & 1, s_abort, sync);
         if (!ok) break;
-        tc_fence_after();
-        {
-          const uint64_t a0 = make_desc(sbase + TcSmem::q, 16, 1024);
-          const uint64_t b0 = make_desc(sbase + TcSmem::k + st * kKVBytes, 16, 1024);
-#pragma unroll
-          for (int ks = 0; ks < kHeadDim / 16; ++ks)          // 32 bytes along K per step
-            tc_mma(tmem, a0 + 2u * ks, b0 + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-          tc_commit(bar(BAR_S_READY));
-        }
-        // next block's copies: its stage was last read by the PV product of block kb-1
-        if (kb + 1 < n_blocks) {
-          const int sn = (kb + 1) & 1;
-          if (kb >= 1) ok = mbar_wait(bar(BAR_KV_EMPTY + sn), ((kb - 1) >> 1) & 1, s_abort, sync);
-          if (!ok) break;
-          mbar_expect_tx(bar(BAR_KV_FULL + sn), 2 * kKVBytes);
-          tma_load_4d(sbase + TcSmem::k + sn * kKVBytes, &map_k, bar(BAR_KV_FULL + sn), 0, h, b, p.k0 + (kb + 1) * kBK);
-          tma_load_4d(sbase + TcSmem::v + sn * kKVBytes, &map_v, bar(BAR_KV_FULL + sn), 0, h, b, p.k0 + (kb + 1) * kBK);
-          ++loads_issued;
-        }
-        ok = mbar_wait(bar(BAR_P_READY), kb & 1, s_abort, sync);
-        if (ok && kb > 0) ok = mbar_wait(bar(BAR_PV_FREE), (kb - 1) & 1, s_abort, sync);
-        if (!ok) break;
-        tc_fence_after();
-        {
-          const uint64_t a0 = make_desc(sbase + TcSmem::p, 16, 1024);
-          const uint64_t b0 = make_desc(sbase + TcSmem::v + st * kKVBytes, 16, 1024);
-#pragma unroll
-          for (int ks = 0; ks < kBK / 16; ++ks)               // A: 32 bytes along K; B (MN-major): 16 key rows = 2048 bytes
-            tc_mma(tmem + 64u, a0 + 2u * ks, b0 + 128u * ks, idesc_pv, ks > 0 ? 1u : 0u);
-          tc_commit(bar(BAR_PV_READY));
-          tc_commit(bar(BAR_KV_EMPTY + st));
-        }
+        mbar_expect_tx(bar(BAR_KV_FULL + st), 2 * kKVBytes);
+        tma_load_4d(sbase + TcSmem::k + st * kKVBytes, &map_k, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
+        tma_load_4d(sbase + TcSmem::v + st * kKVBytes, &map_v, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
+        ++issued;
       }
       if (!ok) {
         // gave up: let the copies already started land before the shared memory goes away (bounded)
-        for (int i = 0; i < loads_issued && i < 2; ++i) {
-          const int blk = loads_issued - 1 - i;
-          unsigned spins = 0;
-          while (!mbar_try_wait(bar(BAR_KV_FULL + (blk & 1)), (blk >> 1) & 1) && ++spins < (1u << 20)) {}
+        unsigned spins = 0;
+        while (!mbar_try_wait(bar(BAR_Q), 0) && ++spins < (1u << 20)) {}
+        for (int i = issued > kKvStages ? issued - kKvStages : 0; i < issued; ++i) {
+          spins = 0;
+          while (!mbar_try_wait(bar(BAR_KV_FULL + i % kKvStages), (i / kKvStages) & 1) && ++spins < (1u << 20)) {}
         }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 4) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(kBK, false);
+      constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true);
+      const uint64_t q_desc = make_desc(sbase + TcSmem::q, 16, 1024);
+      const uint64_t p_desc = make_desc(sbase + TcSmem::p, 16, 1024);
+      auto issue_s = [&](int kb) -> bool {
+        const int st = kb % kKvStages, sb = kb & 1;
+        if (!mbar_wait(bar(BAR_KV_FULL + st), (kb / kKvStages) & 1, s_abort, sync)) return false;
+        if (kb >= 2 && !mbar_wait(bar(BAR_S_FREE + sb), ((kb >> 1) - 1) & 1, s_abort, sync)) return false;
+        tc_fence_after();
+        const uint64_t k_desc = make_desc(sbase + TcSmem::k + st * kKVBytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // 32 bytes along K per step
+          tc_mma(tmem + (uint32_t)(sb * kBK), q_desc + 2u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
+        tc_commit(bar(BAR_S_READY + sb));
+        return true;
+      };
+      bool ok = mbar_wait(bar(BAR_Q), 0, s_abort, sync);
+      if (ok) ok = issue_s(0);
+      for (int kb = 0; kb < n_blocks && ok; ++kb) {
+        if (kb + 1 < n_blocks) { ok = issue_s(kb + 1); if (!ok) break; }   // runs under softmax(kb)
+        const int st = kb % kKvStages, pb = kb & 1;
+        ok = mbar_wait(bar(BAR_P_READY), kb & 1, s_abort, sync);
+        if (ok && kb >= 2) ok = mbar_wait(bar(BAR_PV_FREE + pb), ((kb >> 1) - 1) & 1, s_abort, sync);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t v_desc = make_desc(sbase + TcSmem::v + st * kKVBytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < kBK / 16; ++ks)                 // A: 32 bytes along K; B (MN-major): 16 key rows = 2048 bytes
+          tc_mma(tmem + (uint32_t)(2 * kBK + pb * kHeadDim), p_desc + 2u * ks, v_desc + 128u * ks, idesc_pv, ks > 0 ? 1u : 0u);
+        tc_commit(bar(BAR_PV_READY + pb));
+        tc_commit(bar(BAR_KV_EMPTY + st));
       }
     }
     __syncwarp();
@@ -156,27 +159,30 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     unsigned char* p_row = smem + TcSmem::p + (row >> 3) * 1024 + (row & 7) * 128;
+    const int sw = row & 7;
     bool ok = true;
     for (int kb = 0; kb < n_blocks; ++kb) {
-      const int n_valid = nk - kb * kBK < kBK ? nk - kb * kBK : kBK;
-      ok = mbar_wait(bar(BAR_S_READY), kb & 1, s_abort, sync);
+      const int sb = kb & 1;
+      ok = mbar_wait(bar(BAR_S_READY + sb), (kb >> 1) & 1, s_abort, sync);
       if (!ok) break;
       tc_fence_after();
       uint32_t s0[32], s1[32];
-      tc_ld32(t_row, s0);
-      tc_ld32(t_row + 32u, s1);
+      tc_ld32(t_row + (uint32_t)(sb * kBK), s0);
+      tc_ld32(t_row + (uint32_t)(sb * kBK + 32), s1);
       tc_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_S_FREE));           // S may be overwritten by the next block's product
-      float mx = -INFINITY;
+      if (lane == 0) mbar_arrive(bar(BAR_S_FREE + sb));      // this S buffer may take block kb+2
+      float mx = __uint_as_float(s0[0]);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        if (i < n_valid) mx = fmaxf(mx, __uint_as_float(s0[i]));
-        if (32 + i < n_valid) mx = fmaxf(mx, __uint_as_float(s1[i]));
-      }
+      for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float corr = ex2(m_run - m_new);
+      // P(kb-1) must have been consumed before this block's P overwrites it (and PV(kb-1) is read below)
+      if (kb >= 1) {
+        ok = mbar_wait(bar(BAR_PV_READY + ((kb - 1) & 1)), ((kb - 1) >> 1) & 1, s_abort, sync);
+        if (!ok) break;
+      }
       float sum = 0.f;
       // p = 2^(s*scale - m_new), packed to bf16 and stored in the swizzled K-major layout
 #pragma unroll
@@ -187,33 +193,51 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const int e0 = c16 * 8 + 2 * j;
           const float x0 = __uint_as_float(e0 < 32 ? s0[e0 & 31] : s1[e0 & 31]);
           const float x1 = __uint_as_float(e0 + 1 < 32 ? s0[(e0 + 1) & 31] : s1[(e0 + 1) & 31]);
-          const float p0 = e0 < n_valid ? ex2(fmaf(x0, p.scale_log2, -m_new)) : 0.f;
-          const float p1 = e0 + 1 < n_valid ? ex2(fmaf(x1, p.scale_log2, -m_new)) : 0.f;
+          const float p0 = ex2(fmaf(x0, p.scale_log2, -m_new));
+          const float p1 = ex2(fmaf(x1, p.scale_log2, -m_new));
+          sum += p0 + p1;
           const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-          // the row sum uses the rounded values the tensor core will see
-          sum += __low2float(pk) + __high2float(pk);
           w[j] = *reinterpret_cast<const uint32_t*>(&pk);
         }
-        *reinterpret_cast<uint4*>(p_row + ((c16 ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(p_row + ((c16 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_P_READY));
       l_run = l_run * corr + sum;
       m_run = m_new;
-      ok = mbar_wait(bar(BAR_PV_READY), kb & 1, s_abort, sync);
-      if (!ok) break;
-      tc_fence_after();
-      tc_ld32(t_row + 64u, s0);
-      tc_ld32(t_row + 96u, s1);
-      tc_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PV_FREE));
+      if (kb >= 1) {
+        // fold the previous block's product in, one block late: o <- (o + PV(kb-1)) * corr(kb)
+        const int pb = (kb - 1) & 1;
+        tc_fence_after();
+        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim), s0);
+        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim + 32), s1);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_PV_FREE + pb));
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        o[i] = fmaf(o[i], corr, __uint_as_float(s0[i]));
-        o[32 + i] = fmaf(o[32 + i], corr, __uint_as_float(s1[i]));
+        for (int i = 0; i < 32; ++i) {
+          o[i] = (o[i] + __uint_as_float(s0[i])) * corr;
+          o[32 + i] = (o[32 + i] + __uint_as_float(s1[i])) * corr;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kHeadDim; ++i) o[i] *= corr;
+      }
+    }
+    if (ok) {
+      const int pb = (n_blocks - 1) & 1;
+      ok = mbar_wait(bar(BAR_PV_READY + pb), ((n_blocks - 1) >> 1) & 1, s_abort, sync);
+      if (ok) {
+        uint32_t s0[32], s1[32];
+        tc_fence_after();
+        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim), s0);
+        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim + 32), s1);
+        tc_wait_ld();
+        tc_fence_before();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) { o[i] += __uint_as_float(s0[i]); o[32 + i] += __uint_as_float(s1[i]); }
       }
     }
     if (ok && row_ok) {

@@ -25,7 +25,7 @@ RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
-           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static")
+           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile")
 RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -69,6 +69,8 @@ def _load():
     lib.rt_layer_decode_step.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P, Z, P]
     lib.rt_layer_decode_step_static.restype = C.c_int
     lib.rt_layer_decode_step_static.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P]
+    lib.rt_update_tile.restype = C.c_int
+    lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P]
     lib.rt_stack_prefill.restype = C.c_int
     lib.rt_stack_prefill.argtypes = [C.POINTER(RtConfig), I, C.POINTER(RtLayerWeights), P, P, I, P, I, I, P, P,
                                      C.POINTER(P), C.POINTER(P), I, P, Z, P]
@@ -140,6 +142,11 @@ def rt_decode_step(cfg, n_layers, layers, emb, g_final, vocab, ids, B, pos, logi
                    workspace, workspace_bytes, stream) -> int:
     return _lib.rt_decode_step(C.byref(cfg), n_layers, layers, emb, g_final, vocab, ids, B, pos, logits, k_caches,
                                v_caches, N_max, workspace, workspace_bytes, stream)
+
+
+def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1, workspace, stream) -> int:
+    return _lib.rt_update_tile(C.byref(cfg), q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1,
+                               workspace, stream)
 
 
 def rt_get_status(workspace) -> int:

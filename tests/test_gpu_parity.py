@@ -181,3 +181,53 @@ def test_c3_full_size_bf16_prefix_and_fixed_point():
     zmax = np.abs(got[0][sel]).max()
     assert np.abs(z2[:, rows] - got[0][sel][:, rows]).max() / zmax <= TOL["bf16"]
     assert rel_err(got[1][sel], k2) <= TOL["bf16"] and rel_err(got[2][sel], v2) <= TOL["bf16"]
+
+
+# ---------------------------------------------------------------- Algorithm 2 on its own (tensor-core and SIMT tile kernels)
+
+@pytest.mark.parametrize("dtype,nq,nk", [("bf16", 200, 128), ("bf16", 128, 320), ("bf16", 77, 96), ("f32", 40, 50)])
+def test_update_tile_matches_algorithm_2(dtype, nq, nk):
+    import torch
+    from oracle import update_tile
+    from paper_2604_21215_b200 import inputs, rt
+    B, H, dh = 2, 3, 64
+    d = H * dh
+    rng = np.random.default_rng(600 + nq + nk)
+    scale = 0.125
+    rows_q, rows_kv = nq + 8, nk + 24
+    q = inputs.round_to(rng.standard_normal((rows_q, B, d)), dtype)
+    k = inputs.round_to(rng.standard_normal((rows_kv, B, d)), dtype)
+    v = inputs.round_to(rng.standard_normal((rows_kv, B, d)), dtype)
+    q0, q1, k0, k1 = 8, 8 + nq, 16, 16 + nk
+    # running stats that already saw 16 earlier pairs (so the carry-in path is exercised)
+    m0 = np.zeros((rows_q, B, H)); l0 = np.zeros((rows_q, B, H)); o0 = np.zeros((rows_q, B, d))
+    m_ref = np.zeros_like(m0); l_ref = np.zeros_like(l0); o_ref = np.zeros_like(o0)
+    for b in range(B):
+        for h in range(H):
+            sl = slice(h * dh, (h + 1) * dh)
+            m_, l_, o_ = update_tile(q[:, b, sl], k[:16, b, sl], v[:16, b, sl], np.full(rows_q, -np.inf),
+                                     np.zeros(rows_q), np.zeros((rows_q, dh)), scale)
+            m0[:, b, h], l0[:, b, h], o0[:, b, sl] = m_, l_, o_
+            m2, l2, o2 = update_tile(q[q0:q1, b, sl], k[k0:k1, b, sl], v[k0:k1, b, sl], m_[q0:q1], l_[q0:q1], o_[q0:q1], scale)
+            m_ref[:, b, h], l_ref[:, b, h], o_ref[:, b, sl] = m_, l_, o_
+            m_ref[q0:q1, b, h], l_ref[q0:q1, b, h], o_ref[q0:q1, b, sl] = m2, l2, o2
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    dev = lambda a, t=tdt: torch.from_numpy(np.ascontiguousarray(a)).to(t).cuda()
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    LOG2E = 1.4426950408889634
+    od, md, ld = dev(o0, torch.float32), dev(m0 * LOG2E, torch.float32), dev(l0, torch.float32)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    cfg = rt.make_config(d, H, 4 * d, dtype=dtype, softmax_scale=scale)
+    st = rt.rt_update_tile(cfg, qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), od.data_ptr(), md.data_ptr(), ld.data_ptr(),
+                           B, rows_q, rows_kv, q0, q1, k0, k1, ws.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert st == rt.RT_OK
+    torch.cuda.synchronize()
+    assert rt.rt_get_status(ws.data_ptr()) == rt.RT_OK
+    tol = TOL[dtype]
+    # the quantity that is unique is the attention value o/l and the maximum; rows outside [q0,q1) are untouched
+    a_gpu = od.double().cpu().numpy().reshape(rows_q, B, H, dh) / ld.double().cpu().numpy()[..., None]
+    a_ref = o_ref.reshape(rows_q, B, H, dh) / l_ref[..., None]
+    assert rel_err(a_gpu, a_ref) <= tol
+    assert np.abs(md.double().cpu().numpy() / LOG2E - m_ref).max() <= tol * max(1.0, np.abs(m_ref).max())
+    lg = ld.double().cpu().numpy() * np.exp(md.double().cpu().numpy() / LOG2E - m_ref)
+    assert rel_err(lg, l_ref) <= tol
