@@ -21,6 +21,8 @@
 //     the mat-vecs of step j+1.  These warps also apply qkRMS to k_j and write the caches.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "rt_kernels.h"
 
 namespace rt {
@@ -390,35 +392,42 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
         }
 
+        // The loops below are written without branches around the loads and the products (indices
+        // are clamped, missing sequences and k-steps contribute zeros): a branch per product costs
+        // more here than the product.
         float acc[kNT][4];
 #pragma unroll
         for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
         float sq0 = 0.f, sq1 = 0.f;
         bool alive = true;
+        const int g0 = has0 ? g : 0, g1 = has1 ? g + 8 : 0;        // rows read by lanes without a sequence (masked below)
+        const unsigned keep0 = has0 ? 0xffffffffu : 0u, keep1 = has1 ? 0xffffffffu : 0u;
         if (ph == 2) {
           // W_down reads g as packed bf16 after the barrier: plain loads, and ALL of this warp's
           // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
           // pass keeps this at 32 products; the two accumulators halve the dependent chain.
           constexpr int KD = 32 / MB;
-          const __nv_bfloat16* b0p = g_pk + (size_t)g * K + 4 * c;
-          const __nv_bfloat16* b1p = g_pk + (size_t)(g + 8) * K + 4 * c;
+          const __nv_bfloat16* b0p = g_pk + (size_t)g0 * K + 4 * c;
+          const __nv_bfloat16* b1p = g_pk + (size_t)g1 * K + 4 * c;
           for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
             unsigned ad[KD][4];
+            const int n_here = ks1 - kc0;
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
-              ad[i][0] = ad[i][1] = ad[i][2] = ad[i][3] = 0u;
-              if (kc0 + i < ks1) {
-                if (has0) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(b0p + (size_t)(kc0 + i) * 16)); ad[i][0] = w.x; ad[i][2] = w.y; }
-                if (has1) { const uint2 w = __ldcg(reinterpret_cast<const uint2*>(b1p + (size_t)(kc0 + i) * 16)); ad[i][1] = w.x; ad[i][3] = w.y; }
-              }
+              const int ks = kc0 + (i < n_here ? i : 0);
+              const unsigned live = i < n_here ? 0xffffffffu : 0u;
+              const uint2 w0 = __ldcg(reinterpret_cast<const uint2*>(b0p + (size_t)ks * 16));
+              ad[i][0] = w0.x & keep0 & live; ad[i][2] = w0.y & keep0 & live;
+              if (MB == 2) {
+                const uint2 w1 = __ldcg(reinterpret_cast<const uint2*>(b1p + (size_t)ks * 16));
+                ad[i][1] = w1.x & keep1 & live; ad[i][3] = w1.y & keep1 & live;
+              } else { ad[i][1] = 0u; ad[i][3] = 0u; }
             }
             const unsigned char* wd = wp[0] + (size_t)kc0 * 32;
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
-              if (kc0 + i < ks1) {
-                const uint2 bw = *reinterpret_cast<const uint2*>(wd + i * 32);
-                mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
-              }
+              const uint2 bw = *reinterpret_cast<const uint2*>(wd + (i < n_here ? i : 0) * 32);
+              mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
             }
           }
 #pragma unroll
@@ -428,39 +437,43 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           unsigned a[KC][4];
 #pragma unroll
           for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
+          const int n_here = ks1 - kc0;                             // k-steps of this round (the rest stay zero)
           {
             // flag-carrying words: a k-step is 8 words per sequence, this thread takes the 2 adjacent ones at 4c
-            const unsigned long long* base0 = act_ll + ll_word(g, 4 * c);          // + 128 words per k-step
-            const unsigned long long* base1 = act_ll + ll_word(g + 8, 4 * c);
+            const unsigned long long* base0 = act_ll + ll_word(g0, 4 * c) + (size_t)kc0 * 128;   // + 128 words per k-step
+            const unsigned long long* base1 = act_ll + ll_word(g1, 4 * c) + (size_t)kc0 * 128;
             unsigned need0 = 0, need1 = 0;
 #pragma unroll
             for (int i = 0; i < KC; ++i) {
-              if (kc0 + i < ks1) { if (has0) need0 |= 1u << i; if (has1) need1 |= 1u << i; }
+              if (i < n_here) { need0 |= (1u << i) & keep0; need1 |= (1u << i) & keep1; }
             }
             unsigned spins = 0;
             unsigned long long t_start = 0;
             const unsigned long long t_poll = timing ? globaltimer_ns() : 0ull;
             while (alive) {
-              // issue every outstanding load before looking at any flag, so that the loads of a round overlap
+              // every word of the round is loaded before any flag is looked at, so the loads overlap;
+              // words that were already valid are simply read again
               uint4 w0[KC];
 #pragma unroll
-              for (int i = 0; i < KC; ++i)
-                if (need0 & (1u << i)) w0[i] = ld_relaxed_v4(base0 + (size_t)(kc0 + i) * 128);
-              unsigned got0 = 0;
+              for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4(base0 + (size_t)(i < n_here ? i : 0) * 128);
 #pragma unroll
-              for (int i = 0; i < KC; ++i)
-                if ((need0 & (1u << i)) && w0[i].y == seq && w0[i].w == seq) { a[i][0] = w0[i].x; a[i][2] = w0[i].z; got0 |= 1u << i; }
-              need0 &= ~got0;
+              for (int i = 0; i < KC; ++i) {
+                const bool okw = (w0[i].y == seq) & (w0[i].w == seq) & ((need0 >> i) & 1u);
+                a[i][0] = okw ? w0[i].x : a[i][0];
+                a[i][2] = okw ? w0[i].z : a[i][2];
+                need0 &= okw ? ~(1u << i) : 0xffffffffu;
+              }
               if (MB == 2) {
                 uint4 w1[KC];
 #pragma unroll
-                for (int i = 0; i < KC; ++i)
-                  if (need1 & (1u << i)) w1[i] = ld_relaxed_v4(base1 + (size_t)(kc0 + i) * 128);
-                unsigned got1 = 0;
+                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4(base1 + (size_t)(i < n_here ? i : 0) * 128);
 #pragma unroll
-                for (int i = 0; i < KC; ++i)
-                  if ((need1 & (1u << i)) && w1[i].y == seq && w1[i].w == seq) { a[i][1] = w1[i].x; a[i][3] = w1[i].z; got1 |= 1u << i; }
-                need1 &= ~got1;
+                for (int i = 0; i < KC; ++i) {
+                  const bool okw = (w1[i].y == seq) & (w1[i].w == seq) & ((need1 >> i) & 1u);
+                  a[i][1] = okw ? w1[i].x : a[i][1];
+                  a[i][3] = okw ? w1[i].z : a[i][3];
+                  need1 &= okw ? ~(1u << i) : 0xffffffffu;
+                }
               }
               if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
               if ((++spins & 63u) == 0u) {
@@ -471,22 +484,29 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
             }
             if (timing) wait_ns += globaltimer_ns() - t_poll;
           }
-          const unsigned char* wc[kNT];
-#pragma unroll
-          for (int nt = 0; nt < kNT; ++nt) wc[nt] = wp[nt] + (size_t)kc0 * 32;
           const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
+          if (want_ssq) {
 #pragma unroll
-          for (int i = 0; i < KC; ++i) {
-            if (kc0 + i < ks1) {
-              if (want_ssq) frag_ssq_gain<MB>(a[i], gc ? gc + i * 16 : nullptr, sq0, sq1);
+            for (int i = 0; i < KC; ++i) frag_ssq_gain<MB>(a[i], gc ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0, sq1);
+          }
+          // products, specialised on the number of tiles so that none sits behind a branch
+          auto products = [&](auto ntc) {
+            constexpr int NTC = decltype(ntc)::value;
 #pragma unroll
-              for (int nt = 0; nt < kNT; ++nt) {
-                if (nt < n_tiles) {
-                  const uint2 bw = *reinterpret_cast<const uint2*>(wc[nt] + i * 32);
-                  mma_bf16(acc[nt], a[i], bw.x, bw.y);
-                }
+            for (int i = 0; i < KC; ++i) {
+              const int off = ((i < n_here ? i : 0) + kc0) * 32;
+#pragma unroll
+              for (int nt = 0; nt < NTC; ++nt) {
+                const uint2 bw = *reinterpret_cast<const uint2*>(wp[nt] + off);
+                mma_bf16(acc[nt], a[i], bw.x, bw.y);
               }
             }
+          };
+          switch (n_tiles) {
+            case 1: products(std::integral_constant<int, 1>{}); break;
+            case 2: products(std::integral_constant<int, 2>{}); break;
+            case 3: products(std::integral_constant<int, 3>{}); break;
+            default: products(std::integral_constant<int, 4>{}); break;
           }
         }
         // ---- reduce the K split over the 8 warps; warp w then holds the sums of tile t0n + w ----

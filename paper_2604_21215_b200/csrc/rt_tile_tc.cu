@@ -173,9 +173,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_S_FREE + sb));      // this S buffer may take block kb+2
-      float mx = __uint_as_float(s0[0]);
+      float mx4[4];                                            // four independent chains, not one of 64
 #pragma unroll
-      for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+      for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
+#pragma unroll
+      for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float corr = ex2(m_run - m_new);
       // P(kb-1) must have been consumed before this block's P overwrites it (and PV(kb-1) is read below)
@@ -183,7 +186,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ok = mbar_wait(bar(BAR_PV_READY + ((kb - 1) & 1)), ((kb - 1) >> 1) & 1, s_abort, sync);
         if (!ok) break;
       }
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      const float neg_m = -m_new;
       // p = 2^(s*scale - m_new), packed to bf16 and stored in the swizzled K-major layout
 #pragma unroll
       for (int c16 = 0; c16 < 8; ++c16) {                     // 16-byte chunk = 8 keys
@@ -193,9 +197,9 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const int e0 = c16 * 8 + 2 * j;
           const float x0 = __uint_as_float(e0 < 32 ? s0[e0 & 31] : s1[e0 & 31]);
           const float x1 = __uint_as_float(e0 + 1 < 32 ? s0[(e0 + 1) & 31] : s1[(e0 + 1) & 31]);
-          const float p0 = ex2(fmaf(x0, p.scale_log2, -m_new));
-          const float p1 = ex2(fmaf(x1, p.scale_log2, -m_new));
-          sum += p0 + p1;
+          const float p0 = ex2(fmaf(x0, p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(x1, p.scale_log2, neg_m));
+          sum4[j] += p0 + p1;
           const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
           w[j] = *reinterpret_cast<const uint32_t*>(&pk);
         }
@@ -204,7 +208,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_P_READY));
-      l_run = l_run * corr + sum;
+      l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       m_run = m_new;
       if (kb >= 1) {
         // fold the previous block's product in, one block late: o <- (o + PV(kb-1)) * corr(kb)
