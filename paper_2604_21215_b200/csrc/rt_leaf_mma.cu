@@ -80,6 +80,14 @@ __device__ __forceinline__ uint4 ld_relaxed_v4(const void* p) {
   asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
   return make_uint4((unsigned)w0, (unsigned)(w0 >> 32), (unsigned)w1, (unsigned)(w1 >> 32));
 }
+// The same load under a predicate (no branch): when `on` is zero nothing is read and the result is
+// two zero words (flag 0 never matches a step number).
+__device__ __forceinline__ uint4 ld_relaxed_v4_if(const void* p, unsigned on) {
+  unsigned long long w0 = 0ull, w1 = 0ull;
+  asm volatile("{\n .reg .pred q;\n setp.ne.u32 q, %3, 0;\n @q ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];\n}"
+               : "+l"(w0), "+l"(w1) : "l"(p), "r"(on) : "memory");
+  return make_uint4((unsigned)w0, (unsigned)(w0 >> 32), (unsigned)w1, (unsigned)(w1 >> 32));
+}
 __device__ __forceinline__ void st_relaxed_u64(void* p, unsigned lo, unsigned hi) {
   const unsigned long long w = ((unsigned long long)hi << 32) | lo;
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
@@ -451,11 +459,11 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
             unsigned long long t_start = 0;
             const unsigned long long t_poll = timing ? globaltimer_ns() : 0ull;
             while (alive) {
-              // every word of the round is loaded before any flag is looked at, so the loads overlap;
-              // words that were already valid are simply read again
+              // every outstanding word of the round is loaded (under a predicate, not a branch) before
+              // any flag is looked at, so the loads overlap
               uint4 w0[KC];
 #pragma unroll
-              for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4(base0 + (size_t)(i < n_here ? i : 0) * 128);
+              for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4_if(base0 + (size_t)(i < n_here ? i : 0) * 128, (need0 >> i) & 1u);
 #pragma unroll
               for (int i = 0; i < KC; ++i) {
                 const bool okw = (w0[i].y == seq) & (w0[i].w == seq) & ((need0 >> i) & 1u);
@@ -466,7 +474,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
               if (MB == 2) {
                 uint4 w1[KC];
 #pragma unroll
-                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4(base1 + (size_t)(i < n_here ? i : 0) * 128);
+                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4_if(base1 + (size_t)(i < n_here ? i : 0) * 128, (need1 >> i) & 1u);
 #pragma unroll
                 for (int i = 0; i < KC; ++i) {
                   const bool okw = (w1[i].y == seq) & (w1[i].w == seq) & ((need1 >> i) & 1u);
