@@ -40,7 +40,7 @@ def measured_peaks():
 
 # DRAM bytes (read + write) of one leaf launch (64 token steps) from the ncu capture summarised in
 # profiles/leaf_mma_kernel_c2.txt: the launch stages its weight rows once, everything else stays in L2.
-NCU_LEAF_TRAFFIC = {"c2": 14701568 + 36864}
+NCU_LEAF_TRAFFIC = {"c2": 14704384 + 24064}
 
 
 class ClockSampler:
@@ -296,14 +296,15 @@ def run_cuda(args):
         leaf_ms = prof["leaf"]["ms"] / n_leaf
         alg_bytes = (chain_w + act) * tok_steps_per_launch
         achieved = alg_bytes / (leaf_ms * 1e-3) / 1e9 if leaf_ms > 0 else 0.0
-        roofline = {"kernel": "leaf_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        roofline = {"kernel": "leaf_mma_kernel" if (wl.dtype == "bf16" and args.sched == "tiled") else "leaf_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                     "traffic": NCU_LEAF_TRAFFIC.get(wl.name),
                     "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": leaf_ms,
                     "us_per_token_step": 1e3 * leaf_ms / max(tok_steps_per_launch, 1),
-                    "note": "weights stay in shared memory for a whole launch, so the kernel is bound by "
-                            "grid-barrier latency and shared-memory reads, not by HBM; the fraction is the "
-                            "effective weight+activation stream against the HBM copy peak"}
+                    "note": "weights stay in shared memory for a whole launch, so the kernel is bound by the "
+                            "latency of its five all-to-all exchanges per token step (L2 round trips), not by HBM; "
+                            "the fraction is the effective weight+activation stream against the HBM copy peak and "
+                            "traffic is the DRAM bytes ncu counted for one launch"}
         tile_ms = prof["tile"]["ms"]
         tile_tflops = (counters["flops_tile"] * args.steps / (tile_ms * 1e-3) / 1e12) if tile_ms > 0 else None
         n_pos = sample_positions(wl)
