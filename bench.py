@@ -171,11 +171,9 @@ def run_reference(args):
 def run_cuda(args):
     import torch
     import torch.distributed as dist
-    from paper_2604_21215_b200 import inputs, rt
+    from paper_2604_21215_b200 import inputs, replicas, rt
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.world_info(os.environ)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -217,8 +215,7 @@ def run_cuda(args):
     tokens = wl.B * wl.N
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize(dev)
 
     def timed(fn, steps):
@@ -277,10 +274,7 @@ def run_cuda(args):
     if model.status() != rt.RT_OK:
         raise SystemExit("device status after the timed region: " + rt.rt_status_string(model.status()))
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total = float(t[0]), float(t[1])
+    total_ms, e2e_total = replicas.max_over_ranks([total_ms, e2e_total], device=dev)
 
     if rank == 0:
         counters = rt.rt_plan_counters(model.cfg, wl.B, wl.N, wl.n_layers, wl.vocab)
@@ -316,14 +310,14 @@ def run_cuda(args):
         gpu_launches = int(launches + 2 * prof["prepass"]["launches"])
         h2d = host_in.numel() * host_in.element_size()
         d2h = host_out.numel() * host_out.element_size()
-        line = {"metric": METRIC, "value": world * tokens * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        line = {"metric": METRIC, "value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, total_ms), "unit": UNIT,
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16/f32-accumulate" if wl.dtype == "bf16" else "f32",
                 "data": "synthetic", "config": config_dict(wl, args.sched, {"leaf": int(model.cfg.leaf) or 64,
                                                                             "parallelism": f"replicas x{world}"}),
                 "clocks": clocks,
-                "e2e": {"value": world * tokens * args.steps / (e2e_total * 1e-3), "unit": UNIT,
+                "e2e": {"value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, e2e_total), "unit": UNIT,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
                 "gpu_launches": gpu_launches,
                 "roofline": roofline, "cpu_baseline": cpu,

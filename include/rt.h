@@ -176,6 +176,12 @@ rt_status rt_update_tile(const rt_config *cfg, const void *q, const void *k_cach
                          int32_t q0, int32_t q1, int32_t k0, int32_t k1,
                          void *workspace, void *cuda_stream);
 
+/* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues a two-CTA kernel
+ * whose grid barrier expects an arrival that never comes.  The wait gives up after its limit (2 s),
+ * the kernel returns normally, and rt_get_status(workspace) then reports RT_ERR_TIMEOUT; the CUDA
+ * context stays usable.  `workspace` needs 256 bytes. */
+rt_status rt_selftest_wait_expiry(void *workspace, void *cuda_stream);
+
 /* Per-kernel-class timing for benchmarks.  While enabled (a process-wide switch, off by
  * default, and the one piece of global state in the library) every call brackets its launches
  * with CUDA events on the caller's stream: class 0 = pre-pass, 1 = leaf recurrence launches,

@@ -3,4 +3,4 @@
 `inputs` draws the seeded synthetic workloads; `rt` is the thin binding over the C-ABI
 library (importing it loads the CUDA library and fails loudly when it is missing).
 """
-__all__ = ["inputs", "rt"]
+__all__ = ["inputs", "replicas", "rt"]

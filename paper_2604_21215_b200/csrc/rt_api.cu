@@ -371,6 +371,13 @@ rt_status rt_update_tile(const rt_config* cfg, const void* q, const void* k_cach
   return tile_launch(cfg->dtype, tp, s) == cudaSuccess ? RT_OK : RT_ERR_CUDA;
 }
 
+rt_status rt_selftest_wait_expiry(void* workspace, void* cuda_stream) {
+  if (!workspace || !aligned16(workspace)) return RT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (cudaMemsetAsync(workspace, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  return wait_expiry_selftest_launch((SyncArea*)workspace, s) == cudaSuccess ? RT_OK : RT_ERR_CUDA;
+}
+
 rt_status rt_profile_enable(int32_t on) {
   std::lock_guard<std::mutex> g(g_prof_mu);
   g_prof_on = on != 0;

@@ -42,6 +42,9 @@ cudaError_t leaf_launch(int dtype, const LeafParams& p, const LeafLaunch& l, cud
 // Barrier arrivals one launch over [t0,t1) adds to bar_count.
 inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsigned)(t1 - t0) * 5u * (unsigned)grid; }
 
+// launches a 2-CTA kernel whose barrier cannot complete (tests the bounded-wait path)
+cudaError_t wait_expiry_selftest_launch(SyncArea* sync, cudaStream_t s);
+
 // bf16 / tiled-schedule leaf kernel (tensor-core mat-vecs, flag-carrying exchange words).
 struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
 struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [16,d/2] words x3, packed bf16 [B,dff], [B,2d] words

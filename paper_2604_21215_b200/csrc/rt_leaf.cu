@@ -419,6 +419,19 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   }
 }
 
+// Self-test of the bounded wait: the barrier below expects one more arrival than there are CTAs,
+// so it can only end through the time limit.
+__global__ void wait_expiry_selftest_kernel(SyncArea* sync) {
+  __shared__ int s_flag;
+  unsigned target = 0;
+  grid_barrier(sync, target, gridDim.x + 1, &s_flag);
+}
+
+cudaError_t wait_expiry_selftest_launch(SyncArea* sync, cudaStream_t s) {
+  void* args[] = {(void*)&sync};
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&wait_expiry_selftest_kernel), dim3(2), dim3(32), args, 0, s);
+}
+
 // ------------------------------------------------------------------------------------ host
 
 static inline int pick_nb(int B) { return B > 4 ? 8 : (B > 2 ? 4 : (B > 1 ? 2 : 1)); }

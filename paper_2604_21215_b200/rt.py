@@ -25,7 +25,7 @@ RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
-           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile")
+           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile", "rt_selftest_wait_expiry")
 RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -69,6 +69,8 @@ def _load():
     lib.rt_layer_decode_step.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P, Z, P]
     lib.rt_layer_decode_step_static.restype = C.c_int
     lib.rt_layer_decode_step_static.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P]
+    lib.rt_selftest_wait_expiry.restype = C.c_int
+    lib.rt_selftest_wait_expiry.argtypes = [P, P]
     lib.rt_update_tile.restype = C.c_int
     lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P]
     lib.rt_stack_prefill.restype = C.c_int
@@ -147,6 +149,10 @@ def rt_decode_step(cfg, n_layers, layers, emb, g_final, vocab, ids, B, pos, logi
 def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1, workspace, stream) -> int:
     return _lib.rt_update_tile(C.byref(cfg), q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1,
                                workspace, stream)
+
+
+def rt_selftest_wait_expiry(workspace, stream) -> int:
+    return _lib.rt_selftest_wait_expiry(workspace, stream)
 
 
 def rt_get_status(workspace) -> int:

@@ -231,3 +231,22 @@ def test_update_tile_matches_algorithm_2(dtype, nq, nk):
     assert np.abs(md.double().cpu().numpy() / LOG2E - m_ref).max() <= tol * max(1.0, np.abs(m_ref).max())
     lg = ld.double().cpu().numpy() * np.exp(md.double().cpu().numpy() / LOG2E - m_ref)
     assert rel_err(lg, l_ref) <= tol
+
+
+# ---------------------------------------------------------------- a wait that runs out is reported, nothing hangs or traps
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    import time
+    import torch
+    from paper_2604_21215_b200 import rt
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    t0 = time.time()
+    assert rt.rt_selftest_wait_expiry(ws.data_ptr(), torch.cuda.current_stream().cuda_stream) == rt.RT_OK
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 30.0                       # the limit is 2 s; the kernel returned by itself
+    assert rt.rt_get_status(ws.data_ptr()) == rt.RT_ERR_TIMEOUT
+    # the context is intact: a normal call right after still matches the oracle
+    x, lw = make_case(128, 2, 256, 1, 20, "f32", seed=77)
+    ref = oracle_layer(x, lw, 128, 2, 256)
+    _, got = run_layer(x, lw, 128, 2, 256, "f32", leaf=16)
+    check(got, ref, TOL["f32"], "after timeout self-test")
