@@ -3,48 +3,50 @@
 // running stats (m, l, o) carried in fp32 in the workspace.
 //
 // One CTA = 128 query rows of one (sequence, head) pair, looping over 64-key blocks:
-//   TMA     (warp 5) Q tile once, K and V blocks through a 3-stage ring, straight out of the
-//           position-major cache / query buffer (a 4-D tensor map picks the head's 64 columns of
-//           each row), 128-byte swizzle = the tensor cores' canonical shared-memory layout
-//   S       (warp 4) tcgen05.mma  S[128x64] = Q[128x64] . K^T   (A, B K-major; accumulator in TMEM)
+//   Q       each softmax thread loads its query row and parks it in TMEM (32 columns of packed bf16)
+//   TMA     (warp 5) K and V blocks through a 4-stage ring, straight out of the position-major
+//           cache (a 4-D tensor map picks the head's 64 columns of each row), 128-byte swizzle =
+//           the tensor cores' canonical shared-memory layout
+//   S       (warp 4) tcgen05.mma  S[128x64] = Q . K^T   (A from TMEM, B K-major from shared memory)
 //   softmax (warps 0-3, one thread per query row) tcgen05.ld of the row, running max in log2
-//           units, p = 2^(s - m), row sum, P written to shared memory as bf16 in the swizzled layout
-//   PV      (warp 4) tcgen05.mma  PV[128x64] = P[128x64] . V[64x64]  (B is MN-major: V rows are keys)
-//   merge   o = (o + PV_prev) * 2^(m_old - m_new) in registers (fp32), one block late
-// S and PV are double-buffered in TMEM (256 columns) and the product P.V of block kb is folded
-// into o during block kb+1, so the softmax warps never wait for the tensor cores in steady state:
-// S(kb+1) is issued while softmax(kb) runs and PV(kb) runs under softmax(kb+1).  Two CTAs per SM.
-// Every mbarrier wait is bounded: on expiry the CTA records RT_ERR_TIMEOUT, stops issuing work,
-// waits (bounded) for its copies in flight, frees its TMEM and returns.
+//           units, p = 2^(s - m), row sum; P goes back into TMEM as packed bf16 over the first
+//           half of the S buffer it came from (tcgen05.st)
+//   PV      (warp 4) tcgen05.mma  PV[128x64] = P . V  (A from TMEM, B = V MN-major: V rows are keys)
+//   merge   o = o * 2^(m_old - m_new) + PV in registers (fp32), one block late
+// Both products take their 128-row operand from TMEM: with N = 64 the shared-memory fetch of a
+// 128x16 A slice per instruction (4 KB for 131 k MACs) was what bounded the tensor pipe, not its
+// math rate.  S is double-buffered (S(kb+1) is issued while softmax(kb) runs) and the product P.V
+// of block kb is folded into o during block kb+1.  TMEM: S0 [0,64) S1 [64,128) PV [128,192)
+// Q [192,224); two CTAs per SM.  Every mbarrier wait is bounded: on expiry the CTA records
+// RT_ERR_TIMEOUT, stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and
+// returns.
 #include "rt_kernels.h"
 #include "rt_tc.cuh"
 
 namespace rt {
 
 constexpr int kBK = 64;                // keys per block
-constexpr int kKvStages = 3;
+constexpr int kKvStages = 4;
 constexpr int kTcThreads = 192;        // 4 softmax warps + MMA warp + TMA warp
-constexpr int kTmemCols = 256;         // S0 [0,64) S1 [64,128) PV0 [128,192) PV1 [192,256)
-constexpr uint32_t kQBytes = kBM * kHeadDim * 2;     // 16 KB
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColPV = 128, kColQ = 192;
 constexpr uint32_t kKVBytes = kBK * kHeadDim * 2;    // 8 KB
-constexpr uint32_t kPBytes = kBM * kBK * 2;          // 16 KB
 
 struct TcSmem {                        // offsets from a 1024-byte aligned base
-  static constexpr uint32_t q = 0;
-  static constexpr uint32_t k = q + kQBytes;
+  static constexpr uint32_t k = 0;
   static constexpr uint32_t v = k + kKvStages * kKVBytes;
-  static constexpr uint32_t p = v + kKvStages * kKVBytes;
-  static constexpr uint32_t bars = p + kPBytes;              // 16 mbarriers
+  static constexpr uint32_t bars = v + kKvStages * kKVBytes;
   static constexpr uint32_t tmem_ptr = bars + 128;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
-enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 4, BAR_S_READY = 7, BAR_S_FREE = 9, BAR_P_READY = 11,
-       BAR_PV_READY = 12, BAR_PV_FREE = 14 };
+// P_READY has one barrier per S/P buffer: a softmax warp may run one block ahead of another, and its
+// arrival for block kb+1 must not count towards block kb.
+enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = 4, BAR_Q_READY = 8, BAR_S_READY = 9, BAR_P_READY = 11, BAR_PV_READY = 13, BAR_PV_FREE = 14 };
 
 __global__ void __launch_bounds__(kTcThreads, 2)
-tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-               const __grid_constant__ CUtensorMap map_v, const TileParams p, SyncArea* sync) {
+tile_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const TileParams p,
+               SyncArea* sync) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -58,13 +60,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   if (tid == 0) {
     *s_abort = 0;
-    mbar_init(bar(BAR_Q), 1);
     for (int i = 0; i < kKvStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(BAR_S_READY + i), 1); mbar_init(bar(BAR_S_FREE + i), 4);
-      mbar_init(bar(BAR_PV_READY + i), 1); mbar_init(bar(BAR_PV_FREE + i), 4);
-    }
-    mbar_init(bar(BAR_P_READY), 4);
+    mbar_init(bar(BAR_Q_READY), 4);
+    mbar_init(bar(BAR_S_READY), 1); mbar_init(bar(BAR_S_READY + 1), 1);
+    mbar_init(bar(BAR_P_READY), 4); mbar_init(bar(BAR_P_READY + 1), 4);
+    mbar_init(bar(BAR_PV_READY), 1);
+    mbar_init(bar(BAR_PV_FREE), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {
@@ -79,8 +80,6 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (warp == 5) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      mbar_expect_tx(bar(BAR_Q), kQBytes);
-      tma_load_4d(sbase + TcSmem::q, &map_q, bar(BAR_Q), 0, h, b, qb);
       int issued = 0;
       bool ok = true;
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
@@ -94,10 +93,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       if (!ok) {
         // gave up: let the copies already started land before the shared memory goes away (bounded)
-        unsigned spins = 0;
-        while (!mbar_try_wait(bar(BAR_Q), 0) && ++spins < (1u << 20)) {}
         for (int i = issued > kKvStages ? issued - kKvStages : 0; i < issued; ++i) {
-          spins = 0;
+          unsigned spins = 0;
           while (!mbar_try_wait(bar(BAR_KV_FULL + i % kKvStages), (i / kKvStages) & 1) && ++spins < (1u << 20)) {}
         }
       }
@@ -108,34 +105,33 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(kBK, false);
       constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true);
-      const uint64_t q_desc = make_desc(sbase + TcSmem::q, 16, 1024);
-      const uint64_t p_desc = make_desc(sbase + TcSmem::p, 16, 1024);
       auto issue_s = [&](int kb) -> bool {
         const int st = kb % kKvStages, sb = kb & 1;
         if (!mbar_wait(bar(BAR_KV_FULL + st), (kb / kKvStages) & 1, s_abort, sync)) return false;
-        if (kb >= 2 && !mbar_wait(bar(BAR_S_FREE + sb), ((kb >> 1) - 1) & 1, s_abort, sync)) return false;
+        // the S buffer also carried P(kb-2): it is free once the product P.V of block kb-2 has run
+        if (kb >= 2 && !mbar_wait(bar(BAR_PV_READY), (kb - 2) & 1, s_abort, sync)) return false;
         tc_fence_after();
         const uint64_t k_desc = make_desc(sbase + TcSmem::k + st * kKVBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // 32 bytes along K per step
-          tc_mma(tmem + (uint32_t)(sb * kBK), q_desc + 2u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // A: 8 TMEM columns (16 bf16) per step; B: 32 bytes along K
+          tc_mma_ts(tmem + (uint32_t)(sb * kBK), tmem + kColQ + 8u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
         tc_commit(bar(BAR_S_READY + sb));
         return true;
       };
-      bool ok = mbar_wait(bar(BAR_Q), 0, s_abort, sync);
+      bool ok = mbar_wait(bar(BAR_Q_READY), 0, s_abort, sync);
       if (ok) ok = issue_s(0);
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
         if (kb + 1 < n_blocks) { ok = issue_s(kb + 1); if (!ok) break; }   // runs under softmax(kb)
-        const int st = kb % kKvStages, pb = kb & 1;
-        ok = mbar_wait(bar(BAR_P_READY), kb & 1, s_abort, sync);
-        if (ok && kb >= 2) ok = mbar_wait(bar(BAR_PV_FREE + pb), ((kb >> 1) - 1) & 1, s_abort, sync);
+        const int st = kb % kKvStages, sb = kb & 1;
+        ok = mbar_wait(bar(BAR_P_READY + sb), (kb >> 1) & 1, s_abort, sync);
+        if (ok && kb >= 1) ok = mbar_wait(bar(BAR_PV_FREE), (kb - 1) & 1, s_abort, sync);   // PV(kb-1) has been read out
         if (!ok) break;
         tc_fence_after();
         const uint64_t v_desc = make_desc(sbase + TcSmem::v + st * kKVBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < kBK / 16; ++ks)                 // A: 32 bytes along K; B (MN-major): 16 key rows = 2048 bytes
-          tc_mma(tmem + (uint32_t)(2 * kBK + pb * kHeadDim), p_desc + 2u * ks, v_desc + 128u * ks, idesc_pv, ks > 0 ? 1u : 0u);
-        tc_commit(bar(BAR_PV_READY + pb));
+        for (int ks = 0; ks < kBK / 16; ++ks)                 // A: P in TMEM, 8 columns per step; B (MN-major): 16 key rows = 2048 bytes
+          tc_mma_ts(tmem + kColPV, tmem + (uint32_t)(sb * kBK) + 8u * ks, v_desc + 128u * ks, idesc_pv, ks > 0 ? 1u : 0u);
+        tc_commit(bar(BAR_PV_READY));
         tc_commit(bar(BAR_KV_EMPTY + st));
       }
     }
@@ -147,6 +143,23 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const bool row_ok = qi < p.q1;
     const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
+    {
+      // this row of Q: 64 bf16 = 32 packed words, parked in TMEM for the S products
+      const uint4* qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + sidx * p.d + h * kHeadDim);
+      uint32_t qa[16], qc[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 a = qsrc[i], c = qsrc[4 + i];
+        qa[4 * i] = a.x; qa[4 * i + 1] = a.y; qa[4 * i + 2] = a.z; qa[4 * i + 3] = a.w;
+        qc[4 * i] = c.x; qc[4 * i + 1] = c.y; qc[4 * i + 2] = c.z; qc[4 * i + 3] = c.w;
+      }
+      tc_st16(t_row + kColQ, qa);
+      tc_st16(t_row + kColQ + 16u, qc);
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_Q_READY));
+    }
     float m_run = p.st_m[sidx * p.H + h];
     float l_run = p.st_l[sidx * p.H + h];
     float o[kHeadDim];
@@ -158,8 +171,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         o[4 * i] = v.x; o[4 * i + 1] = v.y; o[4 * i + 2] = v.z; o[4 * i + 3] = v.w;
       }
     }
-    unsigned char* p_row = smem + TcSmem::p + (row >> 3) * 1024 + (row & 7) * 128;
-    const int sw = row & 7;
+    float corr_prev = 1.0f;
     bool ok = true;
     for (int kb = 0; kb < n_blocks; ++kb) {
       const int sb = kb & 1;
@@ -170,10 +182,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_ld32(t_row + (uint32_t)(sb * kBK), s0);
       tc_ld32(t_row + (uint32_t)(sb * kBK + 32), s1);
       tc_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_S_FREE + sb));      // this S buffer may take block kb+2
-      float mx4[4];                                            // four independent chains, not one of 64
+      float mx4[4];                                            // four independent chains
 #pragma unroll
       for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
 #pragma unroll
@@ -181,67 +190,67 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float corr = ex2(m_run - m_new);
-      // P(kb-1) must have been consumed before this block's P overwrites it (and PV(kb-1) is read below)
-      if (kb >= 1) {
-        ok = mbar_wait(bar(BAR_PV_READY + ((kb - 1) & 1)), ((kb - 1) >> 1) & 1, s_abort, sync);
-        if (!ok) break;
-      }
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       const float neg_m = -m_new;
-      // p = 2^(s*scale - m_new), packed to bf16 and stored in the swizzled K-major layout
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      // p = 2^(s*scale - m_new) as packed bf16, written over the first 32 columns of this S buffer
+      uint32_t w[16];
 #pragma unroll
-      for (int c16 = 0; c16 < 8; ++c16) {                     // 16-byte chunk = 8 keys
-        uint32_t w[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int e0 = c16 * 8 + 2 * j;
-          const float x0 = __uint_as_float(e0 < 32 ? s0[e0 & 31] : s1[e0 & 31]);
-          const float x1 = __uint_as_float(e0 + 1 < 32 ? s0[(e0 + 1) & 31] : s1[(e0 + 1) & 31]);
-          const float p0 = ex2(fmaf(x0, p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(x1, p.scale_log2, neg_m));
-          sum4[j] += p0 + p1;
-          const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-          w[j] = *reinterpret_cast<const uint32_t*>(&pk);
-        }
-        *reinterpret_cast<uint4*>(p_row + ((c16 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int j = 0; j < 16; ++j) {
+        const float p0 = ex2(fmaf(__uint_as_float(s0[2 * j]), p.scale_log2, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(s0[2 * j + 1]), p.scale_log2, neg_m));
+        sum4[j & 3] += p0 + p1;
+        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+        w[j] = *reinterpret_cast<const uint32_t*>(&pk);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_st16(t_row + (uint32_t)(sb * kBK), w);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float p0 = ex2(fmaf(__uint_as_float(s1[2 * j]), p.scale_log2, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(s1[2 * j + 1]), p.scale_log2, neg_m));
+        sum4[j & 3] += p0 + p1;
+        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+        w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+      }
+      tc_st16(t_row + (uint32_t)(sb * kBK + 16), w);
+      tc_wait_st();
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_P_READY));
+      if (lane == 0) mbar_arrive(bar(BAR_P_READY + sb));
       l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       m_run = m_new;
       if (kb >= 1) {
-        // fold the previous block's product in, one block late: o <- (o + PV(kb-1)) * corr(kb)
-        const int pb = (kb - 1) & 1;
+        // fold the previous block's product in, one block late: o <- o * corr(kb-1) + PV(kb-1)
+        ok = mbar_wait(bar(BAR_PV_READY), (kb - 1) & 1, s_abort, sync);
+        if (!ok) break;
         tc_fence_after();
-        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim), s0);
-        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim + 32), s1);
+        tc_ld32(t_row + kColPV, s0);
+        tc_ld32(t_row + kColPV + 32u, s1);
         tc_wait_ld();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_PV_FREE + pb));
+        if (lane == 0) mbar_arrive(bar(BAR_PV_FREE));
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          o[i] = (o[i] + __uint_as_float(s0[i])) * corr;
-          o[32 + i] = (o[32 + i] + __uint_as_float(s1[i])) * corr;
+          o[i] = fmaf(o[i], corr_prev, __uint_as_float(s0[i]));
+          o[32 + i] = fmaf(o[32 + i], corr_prev, __uint_as_float(s1[i]));
         }
-      } else {
-#pragma unroll
-        for (int i = 0; i < kHeadDim; ++i) o[i] *= corr;
       }
+      corr_prev = corr;
     }
     if (ok) {
-      const int pb = (n_blocks - 1) & 1;
-      ok = mbar_wait(bar(BAR_PV_READY + pb), ((n_blocks - 1) >> 1) & 1, s_abort, sync);
+      ok = mbar_wait(bar(BAR_PV_READY), (n_blocks - 1) & 1, s_abort, sync);
       if (ok) {
         uint32_t s0[32], s1[32];
         tc_fence_after();
-        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim), s0);
-        tc_ld32(t_row + (uint32_t)(2 * kBK + pb * kHeadDim + 32), s1);
+        tc_ld32(t_row + kColPV, s0);
+        tc_ld32(t_row + kColPV + 32u, s1);
         tc_wait_ld();
         tc_fence_before();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) { o[i] += __uint_as_float(s0[i]); o[32 + i] += __uint_as_float(s1[i]); }
+        for (int i = 0; i < 32; ++i) {
+          o[i] = fmaf(o[i], corr_prev, __uint_as_float(s0[i]));
+          o[32 + i] = fmaf(o[32 + i], corr_prev, __uint_as_float(s1[i]));
+        }
       }
     }
     if (ok && row_ok) {
@@ -279,15 +288,15 @@ static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H,
 cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s) {
   const int nq = p.q1 - p.q0;
   if (nq <= 0 || p.k1 <= p.k0) return cudaSuccess;
-  CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, p.q, rows_q, p.B, p.H, kBM) || !make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) ||
-      !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
+  (void)rows_q;
+  CUtensorMap mk, mv;
+  if (!make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) || !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
     return cudaErrorInvalidValue;
   const size_t smem = TcSmem::total + 1024;
   cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(ceil_div(nq, kBM), p.B * p.H);
-  tile_tc_kernel<<<grid, kTcThreads, smem, s>>>(mq, mk, mv, p, sync);
+  tile_tc_kernel<<<grid, kTcThreads, smem, s>>>(mk, mv, p, sync);
   return cudaGetLastError();
 }
 
