@@ -2,74 +2,83 @@
 // for queries [q0,q1) against the revealed pairs [k0,k1), every sequence and head, with the
 // running stats (m, l, o) carried in fp32 in the workspace.
 //
-// One CTA = 128 query rows of one (sequence, head) pair, looping over 64-key blocks:
-//   Q       each softmax thread loads its query row and parks it in TMEM (32 columns of packed bf16)
-//   TMA     (warp 5) K and V blocks through a 4-stage ring, straight out of the position-major
-//           cache (a 4-D tensor map picks the head's 64 columns of each row), 128-byte swizzle =
-//           the tensor cores' canonical shared-memory layout
-//   S       (warp 4) tcgen05.mma  S[128x64] = Q . K^T   (A from TMEM, B K-major from shared memory)
-//   softmax (warps 0-3, one thread per query row) tcgen05.ld of the row, running max in log2
-//           units, p = 2^(s - m), row sum; P goes back into TMEM as packed bf16 over the first
-//           half of the S buffer it came from (tcgen05.st)
-//   PV      (warp 4) tcgen05.mma  PV[128x64] = P . V  (A from TMEM, B = V MN-major: V rows are keys)
-//   merge   o = o * 2^(m_old - m_new) + PV in registers (fp32), one block late
-// Both products take their 128-row operand from TMEM: with N = 64 the shared-memory fetch of a
-// 128x16 A slice per instruction (4 KB for 131 k MACs) was what bounded the tensor pipe, not its
-// math rate.  S is double-buffered (S(kb+1) is issued while softmax(kb) runs) and the product P.V
-// of block kb is folded into o during block kb+1.  TMEM: S0 [0,64) S1 [64,128) PV [128,192)
-// Q [192,224); two CTAs per SM.  Every mbarrier wait is bounded: on expiry the CTA records
-// RT_ERR_TIMEOUT, stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and
-// returns.
+// One CTA = NT (1 or 2) query tiles of 128 rows of one (sequence, head) pair, looping over 64-key
+// blocks that both tiles share:
+//   TMA     (last warp) the Q tiles once, then K and V blocks through a ring, straight out of the
+//           position-major buffers (a 4-D tensor map picks the head's 64 columns of each row),
+//           128-byte swizzle = the tensor cores' canonical shared-memory layout
+//   S       (MMA warp) tcgen05.mma  S[128x64] = Q . K^T  into the tile's S columns of TMEM
+//   softmax (4 warps per tile, one thread per query row) tcgen05.ld of the row, block max,
+//           p = 2^(s - m), row sum; P goes back into TMEM as packed bf16 over the first half of
+//           the S columns it came from (tcgen05.st)
+//   PV      (MMA warp) tcgen05.mma  O[128x64] += P . V  (A from TMEM, B = V MN-major: V rows are
+//           keys), ACCUMULATING in the tile's O columns of TMEM
+// The running output never visits registers inside the loop: O is seeded from the carried state
+// before the first block and read back once after the last.  The reference maximum m is raised
+// only when a block's maximum exceeds it by more than 2^8 (the merge of Algorithm 2 is exact for
+// any reference value; the bound keeps p <= 256), and then the row's O and l are rescaled in place.
+// The state is renormalised to the true running maximum when it is written back, so the stored
+// triple is the one Algorithm 2 defines.
+// The two tiles of a CTA alternate on the tensor pipe: while one tile's threads do the softmax of
+// block kb, the pipe runs the other tile's P.V(kb) and S(kb+1).  TMEM per tile: S [0,64) O [64,128).
+// Every mbarrier wait is bounded: on expiry the CTA records RT_ERR_TIMEOUT, stops issuing work,
+// waits (bounded) for its copies in flight, frees its TMEM and returns.
 #include "rt_kernels.h"
 #include "rt_tc.cuh"
 
 namespace rt {
 
 constexpr int kBK = 64;                // keys per block
-constexpr int kKvStages = 4;
-constexpr int kTcThreads = 192;        // 4 softmax warps + MMA warp + TMA warp
-constexpr int kTmemCols = 256;
-constexpr uint32_t kColPV = 128, kColQ = 192;
 constexpr uint32_t kKVBytes = kBK * kHeadDim * 2;    // 8 KB
+constexpr uint32_t kQBytes = kBM * kHeadDim * 2;     // 16 KB
+constexpr float kLazyLog2 = 8.0f;      // the reference maximum may lag the true one by this much (log2 units)
+constexpr int kMaxStages = 6;
 
-struct TcSmem {                        // offsets from a 1024-byte aligned base
-  static constexpr uint32_t k = 0;
-  static constexpr uint32_t v = k + kKvStages * kKVBytes;
-  static constexpr uint32_t bars = v + kKvStages * kKVBytes;
-  static constexpr uint32_t tmem_ptr = bars + 128;
+template <int NT>
+struct TcCfg {
+  static constexpr int stages = NT == 2 ? 4 : 3;
+  static constexpr int ctas_per_sm = NT == 2 ? 2 : 3;
+  static constexpr int threads = (4 * NT + 2) * 32;
+  static constexpr int tmem_cols = 128 * NT;
+  // offsets from a 1024-byte aligned base
+  static constexpr uint32_t q = 0;
+  static constexpr uint32_t k = q + NT * kQBytes;
+  static constexpr uint32_t v = k + stages * kKVBytes;
+  static constexpr uint32_t bars = v + stages * kKVBytes;
+  static constexpr uint32_t tmem_ptr = bars + 8 * 24;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
-// P_READY has one barrier per S/P buffer: a softmax warp may run one block ahead of another, and its
-// arrival for block kb+1 must not count towards block kb.
-enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = 4, BAR_Q_READY = 8, BAR_S_READY = 9, BAR_P_READY = 11, BAR_PV_READY = 13, BAR_PV_FREE = 14 };
+enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kMaxStages, BAR_Q_FULL = 2 * kMaxStages, BAR_S_READY = 2 * kMaxStages + 1, BAR_P_READY = 2 * kMaxStages + 3 };
 
-__global__ void __launch_bounds__(kTcThreads, 2)
-tile_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const TileParams p,
-               SyncArea* sync) {
+template <int NT>
+__global__ void __launch_bounds__(TcCfg<NT>::threads, TcCfg<NT>::ctas_per_sm)
+tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const TileParams p, SyncArea* sync) {
+  using C = TcCfg<NT>;
+  constexpr int kStages = C::stages;
+  constexpr int kMmaWarp = 4 * NT, kTmaWarp = 4 * NT + 1;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
-  const int qb = p.q0 + blockIdx.x * kBM;                 // first query row of this CTA
+  const int qb = p.q0 + blockIdx.x * (kBM * NT);          // first query row of this CTA
+  const int n_tiles = (NT == 2 && p.q1 - qb > kBM) ? 2 : 1;
   const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + TcSmem::abort_flag);
-  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + TcSmem::tmem_ptr);
-  auto bar = [&](int i) { return sbase + TcSmem::bars + 8u * (uint32_t)i; };
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + C::tmem_ptr);
+  auto bar = [&](int i) { return sbase + C::bars + 8u * (uint32_t)i; };
 
   if (tid == 0) {
     *s_abort = 0;
-    for (int i = 0; i < kKvStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
-    mbar_init(bar(BAR_Q_READY), 4);
-    mbar_init(bar(BAR_S_READY), 1); mbar_init(bar(BAR_S_READY + 1), 1);
-    mbar_init(bar(BAR_P_READY), 4); mbar_init(bar(BAR_P_READY + 1), 4);
-    mbar_init(bar(BAR_PV_READY), 1);
-    mbar_init(bar(BAR_PV_FREE), 4);
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
+    mbar_init(bar(BAR_Q_FULL), 1);
+    for (int t = 0; t < NT; ++t) { mbar_init(bar(BAR_S_READY + t), 1); mbar_init(bar(BAR_P_READY + t), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + TcSmem::tmem_ptr), "n"(kTmemCols) : "memory");
+  if (warp == kMmaWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + C::tmem_ptr), "n"(C::tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -77,122 +86,118 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  if (warp == 5) {
+  if (warp == kTmaWarp) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
+      mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)n_tiles * kQBytes);
+      for (int t = 0; t < n_tiles; ++t) tma_load_4d(sbase + C::q + t * kQBytes, &map_q, bar(BAR_Q_FULL), 0, h, b, qb + t * kBM);
       int issued = 0;
       bool ok = true;
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
-        const int st = kb % kKvStages;
-        if (kb >= kKvStages) ok = mbar_wait(bar(BAR_KV_EMPTY + st), ((kb / kKvStages) - 1) & 1, s_abort, sync);
+        const int st = kb % kStages;
+        if (kb >= kStages) ok = mbar_wait(bar(BAR_KV_EMPTY + st), ((kb / kStages) - 1) & 1, s_abort, sync);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_KV_FULL + st), 2 * kKVBytes);
-        tma_load_4d(sbase + TcSmem::k + st * kKVBytes, &map_k, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
-        tma_load_4d(sbase + TcSmem::v + st * kKVBytes, &map_v, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
+        tma_load_4d(sbase + C::k + st * kKVBytes, &map_k, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
+        tma_load_4d(sbase + C::v + st * kKVBytes, &map_v, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
         ++issued;
       }
       if (!ok) {
         // gave up: let the copies already started land before the shared memory goes away (bounded)
-        for (int i = issued > kKvStages ? issued - kKvStages : 0; i < issued; ++i) {
-          unsigned spins = 0;
-          while (!mbar_try_wait(bar(BAR_KV_FULL + i % kKvStages), (i / kKvStages) & 1) && ++spins < (1u << 20)) {}
+        unsigned spins = 0;
+        while (!mbar_try_wait(bar(BAR_Q_FULL), 0) && ++spins < (1u << 20)) {}
+        for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
+          spins = 0;
+          while (!mbar_try_wait(bar(BAR_KV_FULL + i % kStages), (i / kStages) & 1) && ++spins < (1u << 20)) {}
         }
       }
     }
     __syncwarp();
-  } else if (warp == 4) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(kBK, false);
       constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true);
-      auto issue_s = [&](int kb) -> bool {
-        const int st = kb % kKvStages, sb = kb & 1;
-        if (!mbar_wait(bar(BAR_KV_FULL + st), (kb / kKvStages) & 1, s_abort, sync)) return false;
-        // the S buffer also carried P(kb-2): it is free once the product P.V of block kb-2 has run
-        if (kb >= 2 && !mbar_wait(bar(BAR_PV_READY), (kb - 2) & 1, s_abort, sync)) return false;
-        tc_fence_after();
-        const uint64_t k_desc = make_desc(sbase + TcSmem::k + st * kKVBytes, 16, 1024);
+      // S_t(kb) = Q_t . K(kb)^T over the tile's S columns; the commit also covers every product issued before it
+      auto issue_s = [&](int t, int kb) {
+        const int st = kb % kStages;
+        const uint64_t q_desc = make_desc(sbase + C::q + t * kQBytes, 16, 1024);
+        const uint64_t k_desc = make_desc(sbase + C::k + st * kKVBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // A: 8 TMEM columns (16 bf16) per step; B: 32 bytes along K
-          tc_mma_ts(tmem + (uint32_t)(sb * kBK), tmem + kColQ + 8u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
-        tc_commit(bar(BAR_S_READY + sb));
-        return true;
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // both operands K-major: 32 bytes along K per step
+          tc_mma(tmem + (uint32_t)(t * 128), q_desc + 2u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
       };
-      bool ok = mbar_wait(bar(BAR_Q_READY), 0, s_abort, sync);
-      if (ok) ok = issue_s(0);
-      for (int kb = 0; kb < n_blocks && ok; ++kb) {
-        if (kb + 1 < n_blocks) { ok = issue_s(kb + 1); if (!ok) break; }   // runs under softmax(kb)
-        const int st = kb % kKvStages, sb = kb & 1;
-        ok = mbar_wait(bar(BAR_P_READY + sb), (kb >> 1) & 1, s_abort, sync);
-        if (ok && kb >= 1) ok = mbar_wait(bar(BAR_PV_FREE), (kb - 1) & 1, s_abort, sync);   // PV(kb-1) has been read out
-        if (!ok) break;
+      bool ok = mbar_wait(bar(BAR_Q_FULL), 0, s_abort, sync);
+      if (ok) ok = mbar_wait(bar(BAR_KV_FULL), 0, s_abort, sync);
+      if (ok) {
         tc_fence_after();
-        const uint64_t v_desc = make_desc(sbase + TcSmem::v + st * kKVBytes, 16, 1024);
+        for (int t = 0; t < n_tiles; ++t) { issue_s(t, 0); tc_commit(bar(BAR_S_READY + t)); }
+      }
+      for (int kb = 0; kb < n_blocks && ok; ++kb) {
+        const int st = kb % kStages;
+        const bool more = kb + 1 < n_blocks;
+        if (more) ok = mbar_wait(bar(BAR_KV_FULL + (kb + 1) % kStages), ((kb + 1) / kStages) & 1, s_abort, sync);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          ok = mbar_wait(bar(BAR_P_READY + t), kb & 1, s_abort, sync);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t v_desc = make_desc(sbase + C::v + st * kKVBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < kBK / 16; ++ks)                 // A: P in TMEM, 8 columns per step; B (MN-major): 16 key rows = 2048 bytes
-          tc_mma_ts(tmem + kColPV, tmem + (uint32_t)(sb * kBK) + 8u * ks, v_desc + 128u * ks, idesc_pv, ks > 0 ? 1u : 0u);
-        tc_commit(bar(BAR_PV_READY));
-        tc_commit(bar(BAR_KV_EMPTY + st));
+          for (int ks = 0; ks < kBK / 16; ++ks)               // A: P in TMEM, 8 columns per step; B (MN-major): 16 key rows = 2048 bytes
+            tc_mma_ts(tmem + (uint32_t)(t * 128 + 64), tmem + (uint32_t)(t * 128) + 8u * ks, v_desc + 128u * ks, idesc_pv, 1u);
+          if (t == n_tiles - 1) tc_commit(bar(BAR_KV_EMPTY + st));   // both tiles have used K(kb) and V(kb)
+          if (more) issue_s(t, kb + 1);
+          tc_commit(bar(BAR_S_READY + t));                    // S(kb+1) ready, and O holds blocks 0..kb
+        }
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 4 * n_tiles) {
     // ------------------------------ softmax warps: one thread per query row ------------------------------
-    const int row = warp * 32 + lane;
-    const int qi = qb + row;
+    const int t = warp >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const int qi = qb + t * kBM + row;
     const bool row_ok = qi < p.q1;
-    const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(t * 128);
+    const uint32_t t_o = t_s + 64u;
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
-    {
-      // this row of Q: 64 bf16 = 32 packed words, parked in TMEM for the S products
-      const uint4* qsrc = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.q) + sidx * p.d + h * kHeadDim);
-      uint32_t qa[16], qc[16];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 a = qsrc[i], c = qsrc[4 + i];
-        qa[4 * i] = a.x; qa[4 * i + 1] = a.y; qa[4 * i + 2] = a.z; qa[4 * i + 3] = a.w;
-        qc[4 * i] = c.x; qc[4 * i + 1] = c.y; qc[4 * i + 2] = c.z; qc[4 * i + 3] = c.w;
-      }
-      tc_st16(t_row + kColQ, qa);
-      tc_st16(t_row + kColQ + 16u, qc);
-      tc_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_Q_READY));
-    }
-    float m_run = p.st_m[sidx * p.H + h];
+    float m_used = p.st_m[sidx * p.H + h];                   // reference maximum of l and O (log2 units)
+    float m_true = m_used;                                   // running maximum
     float l_run = p.st_l[sidx * p.H + h];
-    float o[kHeadDim];
+    uint32_t s0[32], s1[32];
     {
-      const float4* src = reinterpret_cast<const float4*>(p.st_o + sidx * p.d + h * kHeadDim);
+      // seed O with the carried output
+      const uint4* src = reinterpret_cast<const uint4*>(p.st_o + sidx * p.d + h * kHeadDim);
 #pragma unroll
-      for (int i = 0; i < kHeadDim / 4; ++i) {
-        const float4 v = src[i];
-        o[4 * i] = v.x; o[4 * i + 1] = v.y; o[4 * i + 2] = v.z; o[4 * i + 3] = v.w;
+      for (int i = 0; i < 8; ++i) {
+        const uint4 a = src[i], c = src[8 + i];
+        s0[4 * i] = a.x; s0[4 * i + 1] = a.y; s0[4 * i + 2] = a.z; s0[4 * i + 3] = a.w;
+        s1[4 * i] = c.x; s1[4 * i + 1] = c.y; s1[4 * i + 2] = c.z; s1[4 * i + 3] = c.w;
       }
+      tc_st32(t_o, s0);
+      tc_st32(t_o + 32u, s1);
     }
-    float corr_prev = 1.0f;
     bool ok = true;
     for (int kb = 0; kb < n_blocks; ++kb) {
-      const int sb = kb & 1;
-      ok = mbar_wait(bar(BAR_S_READY + sb), (kb >> 1) & 1, s_abort, sync);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY + t), kb & 1, s_abort, sync));
       if (!ok) break;
       tc_fence_after();
-      uint32_t s0[32], s1[32];
-      tc_ld32(t_row + (uint32_t)(sb * kBK), s0);
-      tc_ld32(t_row + (uint32_t)(sb * kBK + 32), s1);
+      tc_ld32(t_s, s0);
+      tc_ld32(t_s + 32u, s1);
       tc_wait_ld();
       float mx4[4];                                            // four independent chains
 #pragma unroll
       for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
 #pragma unroll
       for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float corr = ex2(m_run - m_new);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      m_true = fmaxf(m_true, mx);
+      const bool raise = mx > m_used + kLazyLog2;
+      const float m_new = raise ? m_true : m_used;
+      const float corr = ex2(m_used - m_new);                  // 1 when the reference stays
       const float neg_m = -m_new;
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      // p = 2^(s*scale - m_new) as packed bf16, written over the first 32 columns of this S buffer
+      // p = 2^(s*scale - m) as packed bf16, written over the first 32 columns of the S buffer
       uint32_t w[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
@@ -202,7 +207,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
         w[j] = *reinterpret_cast<const uint32_t*>(&pk);
       }
-      tc_st16(t_row + (uint32_t)(sb * kBK), w);
+      tc_st16(t_s, w);
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         const float p0 = ex2(fmaf(__uint_as_float(s1[2 * j]), p.scale_log2, neg_m));
@@ -211,61 +216,52 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
         w[j] = *reinterpret_cast<const uint32_t*>(&pk);
       }
-      tc_st16(t_row + (uint32_t)(sb * kBK + 16), w);
+      tc_st16(t_s + 16u, w);
+      l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      m_used = m_new;
+      if (__any_sync(0xffffffffu, raise)) {
+        // rare: rescale this warp's rows of O in place (O is quiescent: S_READY(kb) covers P.V(kb-1))
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          tc_ld32(t_o + 32u * half, s0);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) s0[i] = __float_as_uint(__uint_as_float(s0[i]) * corr);
+          tc_st32(t_o + 32u * half, s0);
+        }
+      }
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_P_READY + sb));
-      l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-      m_run = m_new;
-      if (kb >= 1) {
-        // fold the previous block's product in, one block late: o <- o * corr(kb-1) + PV(kb-1)
-        ok = mbar_wait(bar(BAR_PV_READY), (kb - 1) & 1, s_abort, sync);
-        if (!ok) break;
-        tc_fence_after();
-        tc_ld32(t_row + kColPV, s0);
-        tc_ld32(t_row + kColPV + 32u, s1);
-        tc_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_PV_FREE));
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          o[i] = fmaf(o[i], corr_prev, __uint_as_float(s0[i]));
-          o[32 + i] = fmaf(o[32 + i], corr_prev, __uint_as_float(s1[i]));
-        }
-      }
-      corr_prev = corr;
+      if (lane == 0) mbar_arrive(bar(BAR_P_READY + t));
     }
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY + t), n_blocks & 1, s_abort, sync));
     if (ok) {
-      ok = mbar_wait(bar(BAR_PV_READY), (n_blocks - 1) & 1, s_abort, sync);
-      if (ok) {
-        uint32_t s0[32], s1[32];
-        tc_fence_after();
-        tc_ld32(t_row + kColPV, s0);
-        tc_ld32(t_row + kColPV + 32u, s1);
-        tc_wait_ld();
-        tc_fence_before();
+      tc_fence_after();
+      tc_ld32(t_o, s0);
+      tc_ld32(t_o + 32u, s1);
+      tc_wait_ld();
+      tc_fence_before();
+      if (row_ok) {
+        const float c = ex2(m_used - m_true);                  // back to the true maximum
+        p.st_m[sidx * p.H + h] = m_true;
+        p.st_l[sidx * p.H + h] = l_run * c;
+        float4* dst = reinterpret_cast<float4*>(p.st_o + sidx * p.d + h * kHeadDim);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          o[i] = fmaf(o[i], corr_prev, __uint_as_float(s0[i]));
-          o[32 + i] = fmaf(o[32 + i], corr_prev, __uint_as_float(s1[i]));
+        for (int i = 0; i < 8; ++i) {
+          dst[i] = make_float4(__uint_as_float(s0[4 * i]) * c, __uint_as_float(s0[4 * i + 1]) * c,
+                               __uint_as_float(s0[4 * i + 2]) * c, __uint_as_float(s0[4 * i + 3]) * c);
+          dst[8 + i] = make_float4(__uint_as_float(s1[4 * i]) * c, __uint_as_float(s1[4 * i + 1]) * c,
+                                   __uint_as_float(s1[4 * i + 2]) * c, __uint_as_float(s1[4 * i + 3]) * c);
         }
       }
-    }
-    if (ok && row_ok) {
-      p.st_m[sidx * p.H + h] = m_run;
-      p.st_l[sidx * p.H + h] = l_run;
-      float4* dst = reinterpret_cast<float4*>(p.st_o + sidx * p.d + h * kHeadDim);
-#pragma unroll
-      for (int i = 0; i < kHeadDim / 4; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(C::tmem_cols) : "memory");
   }
 }
 
@@ -284,20 +280,32 @@ static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int NT>
+static cudaError_t launch_nt(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TileParams& p,
+                             SyncArea* sync, cudaStream_t s) {
+  using C = TcCfg<NT>;
+  const size_t smem = C::total + 1024;
+  cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(ceil_div(p.q1 - p.q0, kBM * NT), p.B * p.H);
+  tile_tc_kernel<NT><<<grid, C::threads, smem, s>>>(mq, mk, mv, p, sync);
+  return cudaGetLastError();
+}
+
 // rows_q / rows_kv: number of rows the query buffer / caches hold (bounds for the tensor maps).
 cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s) {
   const int nq = p.q1 - p.q0;
   if (nq <= 0 || p.k1 <= p.k0) return cudaSuccess;
-  (void)rows_q;
-  CUtensorMap mk, mv;
-  if (!make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) || !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
+  CUtensorMap mq, mk, mv;
+  if (!make_map(&mq, p.q, rows_q, p.B, p.H, kBM) || !make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) ||
+      !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
     return cudaErrorInvalidValue;
-  const size_t smem = TcSmem::total + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  dim3 grid(ceil_div(nq, kBM), p.B * p.H);
-  tile_tc_kernel<<<grid, kTcThreads, smem, s>>>(mk, mv, p, sync);
-  return cudaGetLastError();
+  // two query tiles per CTA share the K/V stream once there are enough CTAs to fill the GPU that way
+  int sms = 148;
+  { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+  const long long ctas2 = (long long)ceil_div(nq, 2 * kBM) * p.B * p.H;
+  if (nq >= 2 * kBM && ctas2 >= 2LL * sms) return launch_nt<2>(mq, mk, mv, p, sync, s);
+  return launch_nt<1>(mq, mk, mv, p, sync, s);
 }
 
 }  // namespace rt
