@@ -36,8 +36,8 @@ constexpr int kMaxStages = 6;
 
 template <int NT>
 struct TcCfg {
-  static constexpr int stages = NT == 2 ? 4 : 3;
-  static constexpr int ctas_per_sm = NT == 2 ? 2 : 3;
+  static constexpr int stages = NT == 2 ? 4 : 2;
+  static constexpr int ctas_per_sm = NT == 2 ? 2 : 4;     // four query tiles per SM either way
   static constexpr int threads = (4 * NT + 2) * 32;
   static constexpr int tmem_cols = 128 * NT;
   // offsets from a 1024-byte aligned base
@@ -300,11 +300,13 @@ cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncAre
   if (!make_map(&mq, p.q, rows_q, p.B, p.H, kBM) || !make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) ||
       !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
     return cudaErrorInvalidValue;
-  // two query tiles per CTA share the K/V stream once there are enough CTAs to fill the GPU that way
+  // Four query tiles are resident per SM either way.  Single-tile CTAs (own K/V ring, own issuing
+  // thread) start and drain faster; two tiles per CTA halve the K/V traffic from L2, which pays
+  // once the launch is many waves long.
   int sms = 148;
   { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
   const long long ctas2 = (long long)ceil_div(nq, 2 * kBM) * p.B * p.H;
-  if (nq >= 2 * kBM && ctas2 >= 2LL * sms) return launch_nt<2>(mq, mk, mv, p, sync, s);
+  if (nq >= 2 * kBM && ctas2 >= 8LL * sms) return launch_nt<2>(mq, mk, mv, p, sync, s);
   return launch_nt<1>(mq, mk, mv, p, sync, s);
 }
 
