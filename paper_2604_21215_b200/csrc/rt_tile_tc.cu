@@ -2,25 +2,24 @@
 // for queries [q0,q1) against the revealed pairs [k0,k1), every sequence and head, with the
 // running stats (m, l, o) carried in fp32 in the workspace.
 //
-// One CTA = NT (1 or 2) query tiles of 128 rows of one (sequence, head) pair, looping over 64-key
-// blocks that both tiles share:
-//   TMA     (last warp) the Q tiles once, then K and V blocks through a ring, straight out of the
-//           position-major buffers (a 4-D tensor map picks the head's 64 columns of each row),
+// One CTA = one query tile of 128 rows of one (sequence, head) pair, looping over 64-key blocks:
+//   TMA     (warp 5) the Q tile once, then K and V blocks through a 2-stage ring, straight out of
+//           the position-major buffers (a 4-D tensor map picks the head's 64 columns of each row),
 //           128-byte swizzle = the tensor cores' canonical shared-memory layout
-//   S       (MMA warp) tcgen05.mma  S[128x64] = Q . K^T  into the tile's S columns of TMEM
-//   softmax (4 warps per tile, one thread per query row) tcgen05.ld of the row, block max,
+//   S       (warp 4) tcgen05.mma  S[128x64] = Q . K^T  into the S columns of TMEM
+//   softmax (warps 0-3, one thread per query row) tcgen05.ld of the row, block max,
 //           p = 2^(s - m), row sum; P goes back into TMEM as packed bf16 over the first half of
 //           the S columns it came from (tcgen05.st)
-//   PV      (MMA warp) tcgen05.mma  O[128x64] += P . V  (A from TMEM, B = V MN-major: V rows are
-//           keys), ACCUMULATING in the tile's O columns of TMEM
+//   PV      (warp 4) tcgen05.mma  O[128x64] += P . V  (A from TMEM, B = V MN-major: V rows are
+//           keys), ACCUMULATING in the O columns of TMEM
 // The running output never visits registers inside the loop: O is seeded from the carried state
 // before the first block and read back once after the last.  The reference maximum m is raised
 // only when a block's maximum exceeds it by more than 2^8 (the merge of Algorithm 2 is exact for
 // any reference value; the bound keeps p <= 256), and then the row's O and l are rescaled in place.
 // The state is renormalised to the true running maximum when it is written back, so the stored
 // triple is the one Algorithm 2 defines.
-// The two tiles of a CTA alternate on the tensor pipe: while one tile's threads do the softmax of
-// block kb, the pipe runs the other tile's P.V(kb) and S(kb+1).  TMEM per tile: S [0,64) O [64,128).
+// TMEM: S [0,64) O [64,128); 48 KB of shared memory and 80 registers per thread, so four CTAs share
+// an SM and their chains (softmax -> P.V -> S -> softmax) interleave on the tensor pipe.
 // Every mbarrier wait is bounded: on expiry the CTA records RT_ERR_TIMEOUT, stops issuing work,
 // waits (bounded) for its copies in flight, frees its TMEM and returns.
 #include "rt_kernels.h"
@@ -32,39 +31,35 @@ constexpr int kBK = 64;                // keys per block
 constexpr uint32_t kKVBytes = kBK * kHeadDim * 2;    // 8 KB
 constexpr uint32_t kQBytes = kBM * kHeadDim * 2;     // 16 KB
 constexpr float kLazyLog2 = 8.0f;      // the reference maximum may lag the true one by this much (log2 units)
-constexpr int kMaxStages = 6;
 
-template <int NT>
 struct TcCfg {
-  static constexpr int stages = NT == 2 ? 4 : 2;
-  static constexpr int ctas_per_sm = NT == 2 ? 2 : 4;     // four query tiles per SM either way
-  static constexpr int threads = (4 * NT + 2) * 32;
-  static constexpr int tmem_cols = 128 * NT;
+  static constexpr int stages = 2;
+  static constexpr int ctas_per_sm = 4;
+  static constexpr int threads = 6 * 32;                 // 4 softmax warps + MMA warp + TMA warp
+  static constexpr int tmem_cols = 128;
   // offsets from a 1024-byte aligned base
   static constexpr uint32_t q = 0;
-  static constexpr uint32_t k = q + NT * kQBytes;
+  static constexpr uint32_t k = q + kQBytes;
   static constexpr uint32_t v = k + stages * kKVBytes;
   static constexpr uint32_t bars = v + stages * kKVBytes;
   static constexpr uint32_t tmem_ptr = bars + 8 * 24;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
-enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kMaxStages, BAR_Q_FULL = 2 * kMaxStages, BAR_S_READY = 2 * kMaxStages + 1, BAR_P_READY = 2 * kMaxStages + 3 };
+enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = 2, BAR_Q_FULL = 4, BAR_S_READY = 5, BAR_P_READY = 6 };
 
-template <int NT>
-__global__ void __launch_bounds__(TcCfg<NT>::threads, TcCfg<NT>::ctas_per_sm)
+__global__ void __launch_bounds__(TcCfg::threads, TcCfg::ctas_per_sm)
 tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const TileParams p, SyncArea* sync) {
-  using C = TcCfg<NT>;
+  using C = TcCfg;
   constexpr int kStages = C::stages;
-  constexpr int kMmaWarp = 4 * NT, kTmaWarp = 4 * NT + 1;
+  constexpr int kMmaWarp = 4, kTmaWarp = 5;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
-  const int qb = p.q0 + blockIdx.x * (kBM * NT);          // first query row of this CTA
-  const int n_tiles = (NT == 2 && p.q1 - qb > kBM) ? 2 : 1;
+  const int qb = p.q0 + blockIdx.x * kBM;                 // first query row of this CTA
   const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + C::tmem_ptr);
@@ -74,7 +69,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     *s_abort = 0;
     for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
     mbar_init(bar(BAR_Q_FULL), 1);
-    for (int t = 0; t < NT; ++t) { mbar_init(bar(BAR_S_READY + t), 1); mbar_init(bar(BAR_P_READY + t), 4); }
+    mbar_init(bar(BAR_S_READY), 1);
+    mbar_init(bar(BAR_P_READY), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -89,8 +85,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (warp == kTmaWarp) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)n_tiles * kQBytes);
-      for (int t = 0; t < n_tiles; ++t) tma_load_4d(sbase + C::q + t * kQBytes, &map_q, bar(BAR_Q_FULL), 0, h, b, qb + t * kBM);
+      mbar_expect_tx(bar(BAR_Q_FULL), kQBytes);
+      tma_load_4d(sbase + C::q, &map_q, bar(BAR_Q_FULL), 0, h, b, qb);
       int issued = 0;
       bool ok = true;
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
@@ -118,47 +114,45 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(kBK, false);
       constexpr uint32_t idesc_pv = make_idesc(kHeadDim, true);
-      // S_t(kb) = Q_t . K(kb)^T over the tile's S columns; the commit also covers every product issued before it
-      auto issue_s = [&](int t, int kb) {
+      // S(kb) = Q . K(kb)^T over the S columns (both operands K-major: 32 bytes along K per step)
+      auto issue_s = [&](int kb) {
         const int st = kb % kStages;
-        const uint64_t q_desc = make_desc(sbase + C::q + t * kQBytes, 16, 1024);
+        const uint64_t q_desc = make_desc(sbase + C::q, 16, 1024);
         const uint64_t k_desc = make_desc(sbase + C::k + st * kKVBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks)            // both operands K-major: 32 bytes along K per step
-          tc_mma(tmem + (uint32_t)(t * 128), q_desc + 2u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)
+          tc_mma(tmem, q_desc + 2u * ks, k_desc + 2u * ks, idesc_s, ks > 0 ? 1u : 0u);
       };
       bool ok = mbar_wait(bar(BAR_Q_FULL), 0, s_abort, sync);
       if (ok) ok = mbar_wait(bar(BAR_KV_FULL), 0, s_abort, sync);
       if (ok) {
         tc_fence_after();
-        for (int t = 0; t < n_tiles; ++t) { issue_s(t, 0); tc_commit(bar(BAR_S_READY + t)); }
+        issue_s(0);
+        tc_commit(bar(BAR_S_READY));
       }
       for (int kb = 0; kb < n_blocks && ok; ++kb) {
         const int st = kb % kStages;
         const bool more = kb + 1 < n_blocks;
         if (more) ok = mbar_wait(bar(BAR_KV_FULL + (kb + 1) % kStages), ((kb + 1) / kStages) & 1, s_abort, sync);
-        for (int t = 0; t < n_tiles && ok; ++t) {
-          ok = mbar_wait(bar(BAR_P_READY + t), kb & 1, s_abort, sync);
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t v_desc = make_desc(sbase + C::v + st * kKVBytes, 16, 1024);
+        if (ok) ok = mbar_wait(bar(BAR_P_READY), kb & 1, s_abort, sync);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t v_desc = make_desc(sbase + C::v + st * kKVBytes, 16, 1024);
 #pragma unroll
-          for (int ks = 0; ks < kBK / 16; ++ks)               // A: P in TMEM, 8 columns per step; B (MN-major): 16 key rows = 2048 bytes
-            tc_mma_ts(tmem + (uint32_t)(t * 128 + 64), tmem + (uint32_t)(t * 128) + 8u * ks, v_desc + 128u * ks, idesc_pv, 1u);
-          if (t == n_tiles - 1) tc_commit(bar(BAR_KV_EMPTY + st));   // both tiles have used K(kb) and V(kb)
-          if (more) issue_s(t, kb + 1);
-          tc_commit(bar(BAR_S_READY + t));                    // S(kb+1) ready, and O holds blocks 0..kb
-        }
+        for (int ks = 0; ks < kBK / 16; ++ks)                 // A: P in TMEM, 8 columns per step; B (MN-major): 16 key rows = 2048 bytes
+          tc_mma_ts(tmem + 64u, tmem + 8u * ks, v_desc + 128u * ks, idesc_pv, 1u);
+        tc_commit(bar(BAR_KV_EMPTY + st));                    // K(kb) and V(kb) have been used
+        if (more) issue_s(kb + 1);                            // P(kb) has been read by then: the pipe runs in issue order
+        tc_commit(bar(BAR_S_READY));                          // S(kb+1) ready, and O holds blocks 0..kb
       }
     }
     __syncwarp();
-  } else if (warp < 4 * n_tiles) {
+  } else {
     // ------------------------------ softmax warps: one thread per query row ------------------------------
-    const int t = warp >> 2;
-    const int row = (warp & 3) * 32 + lane;
-    const int qi = qb + t * kBM + row;
+    const int row = warp * 32 + lane;
+    const int qi = qb + row;
     const bool row_ok = qi < p.q1;
-    const uint32_t t_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(t * 128);
+    const uint32_t t_s = tmem + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_o = t_s + 64u;
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
     float m_used = p.st_m[sidx * p.H + h];                   // reference maximum of l and O (log2 units)
@@ -179,7 +173,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     bool ok = true;
     for (int kb = 0; kb < n_blocks; ++kb) {
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY + t), kb & 1, s_abort, sync));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY), kb & 1, s_abort, sync));
       if (!ok) break;
       tc_fence_after();
       tc_ld32(t_s, s0);
@@ -233,9 +227,9 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_P_READY + t));
+      if (lane == 0) mbar_arrive(bar(BAR_P_READY));
     }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY + t), n_blocks & 1, s_abort, sync));
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY), n_blocks & 1, s_abort, sync));
     if (ok) {
       tc_fence_after();
       tc_ld32(t_o, s0);
@@ -280,18 +274,6 @@ static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NT>
-static cudaError_t launch_nt(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TileParams& p,
-                             SyncArea* sync, cudaStream_t s) {
-  using C = TcCfg<NT>;
-  const size_t smem = C::total + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  dim3 grid(ceil_div(p.q1 - p.q0, kBM * NT), p.B * p.H);
-  tile_tc_kernel<NT><<<grid, C::threads, smem, s>>>(mq, mk, mv, p, sync);
-  return cudaGetLastError();
-}
-
 // rows_q / rows_kv: number of rows the query buffer / caches hold (bounds for the tensor maps).
 cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s) {
   const int nq = p.q1 - p.q0;
@@ -300,14 +282,12 @@ cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncAre
   if (!make_map(&mq, p.q, rows_q, p.B, p.H, kBM) || !make_map(&mk, p.k_cache, rows_kv, p.B, p.H, kBK) ||
       !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
     return cudaErrorInvalidValue;
-  // Four query tiles are resident per SM either way.  Single-tile CTAs (own K/V ring, own issuing
-  // thread) start and drain faster; two tiles per CTA halve the K/V traffic from L2, which pays
-  // once the launch is many waves long.
-  int sms = 148;
-  { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
-  const long long ctas2 = (long long)ceil_div(nq, 2 * kBM) * p.B * p.H;
-  if (nq >= 2 * kBM && ctas2 >= 8LL * sms) return launch_nt<2>(mq, mk, mv, p, sync, s);
-  return launch_nt<1>(mq, mk, mv, p, sync, s);
+  const size_t smem = TcCfg::total + 1024;
+  cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(ceil_div(nq, kBM), p.B * p.H);
+  tile_tc_kernel<<<grid, TcCfg::threads, smem, s>>>(mq, mk, mv, p, sync);
+  return cudaGetLastError();
 }
 
 }  // namespace rt

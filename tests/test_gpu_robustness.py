@@ -1,0 +1,156 @@
+"""GPU checks beyond element-wise parity: run-to-run determinism, writes confined to the result
+buffers, and the two large configurations (the 8-layer stack at full size, a long sequence) via
+properties the oracle can evaluate on sampled positions."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def rel_err(got, ref):
+    return float(np.abs(got - ref).max() / np.abs(ref).max())
+
+
+def _layer(d, H, dff, dtype, lw, **kw):
+    from paper_2604_21215_b200 import rt
+    layer = rt.Layer(d, H, dff, dtype=dtype, **kw)
+    layer.set_weights(lw)
+    return layer
+
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N", [("bf16", 768, 12, 3072, 4, 600), ("f32", 128, 2, 512, 3, 150)])
+def test_repeat_runs_are_bit_identical(dtype, d, H, dff, B, N):
+    # Every reduction has a fixed order (no floating-point atomics), so two runs must agree to the bit;
+    # a race in an exchange or a merge would show up as a difference.
+    import torch
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("rep", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=910)
+    layer = _layer(d, H, dff, dtype, data["layers"][0])
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    xd = torch.from_numpy(data["x"]).to(tdt).cuda()
+    outs = []
+    for _ in range(3):
+        layer.reserve(B, N)
+        layer.k_cache.zero_(); layer.v_cache.zero_()
+        zd = torch.empty_like(xd)
+        layer.prefill_device(xd, zd)
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        outs.append((zd.clone(), layer.k_cache.clone(), layer.v_cache.clone()))
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N", [("bf16", 256, 4, 1024, 3, 333), ("f32", 128, 2, 512, 2, 77)])
+def test_nothing_outside_the_result_buffers_is_written(dtype, d, H, dff, B, N):
+    # z, the caches and the workspace sit inside larger allocations filled with a pattern; after the
+    # call the guard bands on both sides (and the cache rows beyond N) must be unchanged.
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    wl = inputs.Workload("guard", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=911)
+    layer = _layer(d, H, dff, dtype, data["layers"][0])
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    esz = 2 if dtype == "bf16" else 4
+    guard = 4096                                   # bytes on each side
+    N_max = N + 5
+
+    def banded(nbytes):
+        buf = torch.full((guard + nbytes + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+        return buf, buf[guard:guard + nbytes]
+
+    xd = torch.from_numpy(data["x"]).to(tdt).cuda().contiguous()
+    zbuf, zin = banded(B * N * d * esz)
+    kbuf, kin = banded(N_max * B * d * esz)
+    vbuf, vin = banded(N_max * B * d * esz)
+    need = rt.rt_workspace_bytes(layer.cfg, B, N, 1)
+    wbuf, win = banded(need)
+    win.zero_()
+    s = torch.cuda.current_stream().cuda_stream
+    st = rt.rt_layer_prefill(layer.cfg, layer.w, xd.data_ptr(), B, N, zin.data_ptr(), kin.data_ptr(), vin.data_ptr(), N_max,
+                             win.data_ptr(), need, s)
+    torch.cuda.synchronize()
+    assert st == rt.RT_OK and rt.rt_get_status(win.data_ptr()) == rt.RT_OK
+    for buf in (zbuf, kbuf, vbuf, wbuf):
+        assert bool((buf[:guard] == 0xA5).all()) and bool((buf[-guard:] == 0xA5).all())
+    tail = N * B * d * esz                          # cache rows N .. N_max are not part of the result
+    assert bool((kin[tail:] == 0xA5).all()) and bool((vin[tail:] == 0xA5).all())
+    # and the result itself is the usual one
+    z = zin.view(tdt).view(B, N, d).to(torch.float64).cpu().numpy()
+    from oracle import RTConfig, RTWeights, layer_seq
+    ref = layer_seq(RTConfig(d, H, 64, dff), RTWeights(**data["layers"][0]), data["x"])
+    assert rel_err(z, ref[0]) <= TOL[dtype]
+
+
+def test_long_sequence_fixed_point_on_sampled_positions():
+    # One point of the sequence-length sweep (B=1, d=1024, N=8192: cross tiles up to 4096 x 4096).
+    # The oracle rebuilds all pairs from the GPU's z and recomputes sampled positions independently.
+    from oracle import RTConfig, RTWeights, layer_fixed_point
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.sweep(8192)
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    layer = _layer(wl.d_model, wl.n_heads, wl.d_ff, "bf16", lw)
+    z, k, v = layer.prefill(data["x"])
+    assert np.isfinite(z).all()
+    rows = np.r_[0:16, 4088:4104, 6140:6150, 8176:8192]
+    cfg = RTConfig(wl.d_model, wl.n_heads, 64, wl.d_ff)
+    z2, k2, v2 = layer_fixed_point(cfg, RTWeights(**lw), data["x"], z, rows=rows)
+    assert np.abs(z2[:, rows] - z[:, rows]).max() / np.abs(z).max() <= TOL["bf16"]
+    assert rel_err(k, k2) <= TOL["bf16"] and rel_err(v, v2) <= TOL["bf16"]
+
+
+def test_stack_full_size_is_consistent_with_its_layers():
+    # Configuration 4 at full size (8 layers, B=16, N=2048, vocabulary 32000).  The oracle cannot replay
+    # it, so: (1) the stack call equals chaining the single-layer call over a gathered embedding, bit for
+    # bit (same kernels, same order); (2) the last layer passes the fixed-point check on sampled positions
+    # of one sequence; (3) the logits equal the tied head applied in fp64 to the returned hidden state.
+    import torch
+    from oracle import RTConfig, RTWeights, layer_fixed_point, rms
+    from paper_2604_21215_b200 import inputs, rt
+    wl = inputs.WORKLOADS["c4"]
+    data = inputs.make_inputs(wl)
+    L, d, H, dff, V, B, N = wl.n_layers, wl.d_model, wl.n_heads, wl.d_ff, wl.vocab, wl.B, wl.N
+    st = rt.Stack(L, d, H, dff, V, dtype="bf16", residual_scale=wl.residual_scale)
+    st.set_weights(data["layers"], data["emb"])
+    ids = torch.as_tensor(np.asarray(data["ids"]), dtype=torch.int32, device="cuda").contiguous()
+    st.reserve(B, N)
+    hid = torch.empty((B, N, d), dtype=torch.bfloat16, device="cuda")
+    logits = torch.empty((B, V), dtype=torch.float32, device="cuda")
+    st.prefill_device(ids, hid, logits)
+    torch.cuda.synchronize()
+    assert st.status() == 0
+    # (1) chain of single-layer calls
+    x = st.emb[ids.long()].contiguous()
+    x_last = None
+    for li in range(L):
+        layer = rt.Layer(d, H, dff, dtype="bf16", residual_scale=wl.residual_scale)
+        layer.set_weights(data["layers"][li])
+        layer.reserve(B, N)
+        z = torch.empty_like(x)
+        layer.prefill_device(x, z)
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        assert torch.equal(layer.k_cache, st.k_caches[li]) and torch.equal(layer.v_cache, st.v_caches[li])
+        x_last, x = x, z
+        del layer
+    assert torch.equal(x, hid)
+    # (2) fixed point of the last layer on one sequence
+    cfg = RTConfig(d, H, 64, dff, residual_scale=wl.residual_scale)
+    sel = slice(11, 12)
+    rows = np.r_[0:8, 1020:1030, 2040:2048]
+    xin = x_last[sel].to(torch.float64).cpu().numpy()
+    zc = hid[sel].to(torch.float64).cpu().numpy()
+    z2, k2, v2 = layer_fixed_point(cfg, RTWeights(**data["layers"][L - 1]), xin, zc, rows=rows)
+    assert np.abs(z2[:, rows] - zc[:, rows]).max() / np.abs(zc).max() <= TOL["bf16"]
+    kg = st.k_caches[L - 1][:, 11].to(torch.float64).cpu().numpy()[None]
+    vg = st.v_caches[L - 1][:, 11].to(torch.float64).cpu().numpy()[None]
+    assert rel_err(kg, k2) <= TOL["bf16"] and rel_err(vg, v2) <= TOL["bf16"]
+    # (3) tied head on the last position
+    h_last = hid[:, -1].to(torch.float64).cpu().numpy()
+    ref_logits = rms(h_last, np.ones(d), cfg.rms_eps) @ np.asarray(data["emb"], dtype=np.float64).T
+    assert rel_err(logits.to(torch.float64).cpu().numpy(), ref_logits) <= TOL["bf16"]
