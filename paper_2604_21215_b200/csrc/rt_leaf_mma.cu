@@ -88,6 +88,15 @@ __device__ __forceinline__ uint4 ld_relaxed_v4_if(const void* p, unsigned on) {
                : "+l"(w0), "+l"(w1) : "l"(p), "r"(on) : "memory");
   return make_uint4((unsigned)w0, (unsigned)(w0 >> 32), (unsigned)w1, (unsigned)(w1 >> 32));
 }
+// 8 bytes through L2 under a predicate (zeros when `on` is zero).  An asm statement, so that a run
+// of these stays a run of loads: written as plain loads the compiler placed each one's first use
+// right behind it and the round trips added up.
+__device__ __forceinline__ uint2 ld_cg_v2_if(const void* p, unsigned on) {
+  uint2 w = make_uint2(0u, 0u);
+  asm volatile("{\n .reg .pred q;\n setp.ne.u32 q, %3, 0;\n @q ld.global.cg.v2.u32 {%0,%1}, [%2];\n}"
+               : "+r"(w.x), "+r"(w.y) : "l"(p), "r"(on) : "memory");
+  return w;
+}
 __device__ __forceinline__ void st_relaxed_u64(void* p, unsigned lo, unsigned hi) {
   const unsigned long long w = ((unsigned long long)hi << 32) | lo;
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
@@ -101,6 +110,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const unsigned (&a)[4], 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+#ifdef RT_TIMELINE
+__device__ unsigned long long g_dbg[3 * 8 * 4 * 8];      // [cta slot][warp][phase][point]
+#define TL(pt) if (tl_on) g_dbg[((tl_slot * 8 + warp) * 4 + ph) * 8 + (pt)] = globaltimer_ns()
+#else
+#define TL(pt)
+#endif
 __device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory"); }
 
 // A wait that ran out: record it for the host and tell every other waiter to leave.
@@ -149,14 +164,13 @@ __device__ __forceinline__ void frag_ssq_gain(unsigned (&a)[4], const __nv_bfloa
 __device__ __forceinline__ bool mma_grid_barrier(SyncArea* sync, volatile int* s_abort, unsigned target) {
   mma_warps_sync();
   if (threadIdx.x == 0) {
-    __threadfence();
+    // the release is cumulative over what the CTA barrier above ordered before it: no separate fence
     red_release_add_u32(&sync->bar_count, 1u);
     unsigned spins = 0;
     unsigned long long t_start = 0;
     while (ld_acquire_u32(&sync->bar_count) < target) {
       if ((++spins & 255u) == 0u && wait_expired(sync, t_start)) { *s_abort = 1; break; }
     }
-    __threadfence();
   }
   mma_warps_sync();
   return *s_abort == 0;
@@ -347,8 +361,13 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
 
   for (int t = p.t0; t < p.t1; ++t) {
     const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
+#ifdef RT_TIMELINE
+    const int tl_slot = cta == 0 ? 0 : (cta == 77 ? 1 : 2);
+    const bool tl_on = (cta == 0 || cta == 77 || cta == 147) && lane == 0 && t == p.t0 + 20 && p.t0 == 1024;
+#endif
 #pragma unroll 1
     for (int ph = 0; ph < 4; ++ph) {                              // 0: W_o   1: W_up   2: W_down   3: W_k | W_v
+      TL(0);
       // ---- what this phase multiplies ----
       const int K = (ph == 2) ? dff : d;
       const int stride = (ph == 2) ? L.stride_f : L.stride_d;
@@ -369,6 +388,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
         if (!mma_grid_barrier(p.sync, s_abort, bar_target)) return;
         if (timing) wait_ns += globaltimer_ns() - tb;
       }
+      TL(1);
       const int n_ks = K / 16;
       const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
       const int ks0 = warp * ks_per_warp;
@@ -420,22 +440,27 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
             unsigned ad[KD][4];
             const int n_here = ks1 - kc0;
+            uint2 w0[KD], w1[MB == 2 ? KD : 1];
+#pragma unroll
+            for (int i = 0; i < KD; ++i) w0[i] = ld_cg_v2_if(b0p + (size_t)(kc0 + (i < n_here ? i : 0)) * 16, (i < n_here ? 1u : 0u) & keep0);
+            if (MB == 2) {
+#pragma unroll
+              for (int i = 0; i < KD; ++i) w1[i] = ld_cg_v2_if(b1p + (size_t)(kc0 + (i < n_here ? i : 0)) * 16, (i < n_here ? 1u : 0u) & keep1);
+            }
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
-              const int ks = kc0 + (i < n_here ? i : 0);
-              const unsigned live = i < n_here ? 0xffffffffu : 0u;
-              const uint2 w0 = __ldcg(reinterpret_cast<const uint2*>(b0p + (size_t)ks * 16));
-              ad[i][0] = w0.x & keep0 & live; ad[i][2] = w0.y & keep0 & live;
-              if (MB == 2) {
-                const uint2 w1 = __ldcg(reinterpret_cast<const uint2*>(b1p + (size_t)ks * 16));
-                ad[i][1] = w1.x & keep1 & live; ad[i][3] = w1.y & keep1 & live;
-              } else { ad[i][1] = 0u; ad[i][3] = 0u; }
+              ad[i][0] = w0[i].x; ad[i][2] = w0[i].y;
+              if (MB == 2) { ad[i][1] = w1[i].x; ad[i][3] = w1[i].y; } else { ad[i][1] = 0u; ad[i][3] = 0u; }
             }
+            TL(2);
             const unsigned char* wd = wp[0] + (size_t)kc0 * 32;
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
               const uint2 bw = *reinterpret_cast<const uint2*>(wd + (i < n_here ? i : 0) * 32);
               mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
+#ifdef RT_TIMELINE
+              if (i == 1 && tl_on && acc[0][0] != 123.f) TL(7);
+#endif
             }
           }
 #pragma unroll
@@ -491,6 +516,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
               }
             }
             if (timing) wait_ns += globaltimer_ns() - t_poll;
+            TL(2);
           }
           const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
           if (want_ssq) {
@@ -517,6 +543,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
             default: products(std::integral_constant<int, 4>{}); break;
           }
         }
+        TL(3);
         // ---- reduce the K split over the 8 warps; warp w then holds the sums of tile t0n + w ----
 #pragma unroll
         for (int nt = 0; nt < kNT; ++nt)
@@ -527,6 +554,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
         }
         mma_warps_sync();
+        TL(4);
         if (*s_abort) return;
         float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f, ssq_lo = 0.f, ssq_hi = 0.f;
         if (warp < n_tiles) {
@@ -541,6 +569,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           }
         }
         mma_warps_sync();       // red / ssq_red may be overwritten from here on
+        TL(5);
         // ---- epilogue: y0, y1 = rows rl, rl+1 for sequence g; y2, y3 = the same rows for sequence g+8 ----
         if (mine) {
           if (ph == 0) {                                            // h = x_t + alpha W_o c_t
@@ -587,6 +616,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           }
         }
       }
+      TL(6);
       if (timing) {
         const unsigned long long now = globaltimer_ns();
         atomicAdd(&p.sync->phase_ns[2 + 2 * ph], now - t_ph - wait_ns);        // fire-and-forget, no stack array
@@ -598,6 +628,13 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
 }
 
 // ------------------------------------------------------------------------------------ host
+#ifdef RT_TIMELINE
+}  // namespace rt
+extern "C" int rt_debug_read(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, rt::g_dbg, sizeof(rt::g_dbg));
+}
+namespace rt {
+#endif
 
 // Picks the leaf capacity and the launch shape; returns false when this kernel does not take
 // the shape (the generic leaf kernel does).
