@@ -486,9 +486,13 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
             while (alive) {
               // every outstanding word of the round is loaded (under a predicate, not a branch) before
               // any flag is looked at, so the loads overlap
-              uint4 w0[KC];
+              uint4 w0[KC], w1[MB == 2 ? KC : 1];
 #pragma unroll
               for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4_if(base0 + (size_t)(i < n_here ? i : 0) * 128, (need0 >> i) & 1u);
+              if (MB == 2) {
+#pragma unroll
+                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4_if(base1 + (size_t)(i < n_here ? i : 0) * 128, (need1 >> i) & 1u);
+              }
 #pragma unroll
               for (int i = 0; i < KC; ++i) {
                 const bool okw = (w0[i].y == seq) & (w0[i].w == seq) & ((need0 >> i) & 1u);
@@ -497,9 +501,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
                 need0 &= okw ? ~(1u << i) : 0xffffffffu;
               }
               if (MB == 2) {
-                uint4 w1[KC];
-#pragma unroll
-                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4_if(base1 + (size_t)(i < n_here ? i : 0) * 128, (need1 >> i) & 1u);
 #pragma unroll
                 for (int i = 0; i < KC; ++i) {
                   const bool okw = (w1[i].y == seq) & (w1[i].w == seq) & ((need1 >> i) & 1u);
