@@ -63,7 +63,9 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
   // flag-carrying exchange words of the bf16 leaf kernel: c, h, z [B,d/2], g [B,dff/2], raw k|v [B,2d]
   // (c, h, z are laid out for 16 sequence slots whatever B is)
-  L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)B * (f / 2 + 2 * d)) * 8;
+  // exchange buffers of the tensor-core leaf kernel: c, h, z as flag-carrying words (16 sequence slots each),
+  // g as packed bf16 in fragment order (16 sequence slots), raw k|v as flag-carrying fp32 words
+  L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)16 * (f / 4) + (size_t)B * 2 * d) * 8;
   L.ll = take(L.ll_bytes);
   L.hid0 = take(tok * d * e);
   L.hid1 = take(tok * d * e);
@@ -173,7 +175,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     unsigned long long* w = (unsigned long long*)(ws + L.ll);
     const size_t bd2 = (size_t)16 * (c->d_model / 2);
     mb.ll_c = w; mb.ll_h = w + bd2; mb.ll_z = w + 2 * bd2; mb.ll_g = w + 3 * bd2;
-    mb.ll_kv = mb.ll_g + (size_t)B * (c->d_ff / 2);
+    mb.ll_kv = mb.ll_g + (size_t)16 * (c->d_ff / 4);
   }
   auto leaf_mma = [&](int t0, int t1) -> bool {
     lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;

@@ -351,7 +351,10 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   const bool kv_norm = pre && !(p.norm_flags & RT_NORM_SKIP_Z);
   const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(p.x);
   __nv_bfloat16* z = reinterpret_cast<__nv_bfloat16*>(p.z);
-  __nv_bfloat16* g_pk = reinterpret_cast<__nv_bfloat16*>(ll_g);      // packed bf16 [B][dff]
+  // g as packed bf16 in the order the fragments are read: [k-step of 16][16 sequence slots][16 k], so the
+  // 8 sequences x 32 bytes one warp-wide load touches are 256 contiguous bytes (2 lines instead of 8)
+  __nv_bfloat16* g_pk = reinterpret_cast<__nv_bfloat16*>(ll_g);
+  auto g_index = [](int b, int k) -> size_t { return ((size_t)((k >> 4) * 16 + b) << 4) + (size_t)(k & 15); };
   const float inv_d = 1.0f / (float)d;
   const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
   const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
@@ -435,17 +438,17 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
           // pass keeps this at 32 products; the two accumulators halve the dependent chain.
           constexpr int KD = 32 / MB;
-          const __nv_bfloat16* b0p = g_pk + (size_t)g0 * K + 4 * c;
-          const __nv_bfloat16* b1p = g_pk + (size_t)g1 * K + 4 * c;
+          const __nv_bfloat16* b0p = g_pk + g_index(g0, 4 * c);          // + 256 elements per k-step
+          const __nv_bfloat16* b1p = g_pk + g_index(g1, 4 * c);
           for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
             unsigned ad[KD][4];
             const int n_here = ks1 - kc0;
             uint2 w0[KD], w1[MB == 2 ? KD : 1];
 #pragma unroll
-            for (int i = 0; i < KD; ++i) w0[i] = ld_cg_v2_if(b0p + (size_t)(kc0 + (i < n_here ? i : 0)) * 16, (i < n_here ? 1u : 0u) & keep0);
+            for (int i = 0; i < KD; ++i) w0[i] = ld_cg_v2_if(b0p + (size_t)(kc0 + (i < n_here ? i : 0)) * 256, (i < n_here ? 1u : 0u) & keep0);
             if (MB == 2) {
 #pragma unroll
-              for (int i = 0; i < KD; ++i) w1[i] = ld_cg_v2_if(b1p + (size_t)(kc0 + (i < n_here ? i : 0)) * 16, (i < n_here ? 1u : 0u) & keep1);
+              for (int i = 0; i < KD; ++i) w1[i] = ld_cg_v2_if(b1p + (size_t)(kc0 + (i < n_here ? i : 0)) * 256, (i < n_here ? 1u : 0u) & keep1);
             }
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
@@ -587,11 +590,11 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           } else if (ph == 1) {                                     // g = GELU(W_up RMS(h)), packed bf16
             if (has0) {
               const float rs = pre ? rsqrtf(ssq_lo * inv_d + p.eps) : 1.0f;
-              *reinterpret_cast<unsigned*>(g_pk + (size_t)g * dff + f_lo + rl) = pack_bf2(gelu_erf_f(y0 * rs), gelu_erf_f(y1 * rs));
+              *reinterpret_cast<unsigned*>(g_pk + g_index(g, f_lo + rl)) = pack_bf2(gelu_erf_f(y0 * rs), gelu_erf_f(y1 * rs));
             }
             if (has1) {
               const float rs = pre ? rsqrtf(ssq_hi * inv_d + p.eps) : 1.0f;
-              *reinterpret_cast<unsigned*>(g_pk + (size_t)(g + 8) * dff + f_lo + rl) = pack_bf2(gelu_erf_f(y2 * rs), gelu_erf_f(y3 * rs));
+              *reinterpret_cast<unsigned*>(g_pk + g_index(g + 8, f_lo + rl)) = pack_bf2(gelu_erf_f(y2 * rs), gelu_erf_f(y3 * rs));
             }
           } else if (ph == 2) {                                     // z_t = h + alpha W_down g   (layer output)
             if (has0) {
