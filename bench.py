@@ -383,6 +383,63 @@ def run_tile_bench(args):
     return 0
 
 
+def run_decode_bench(args):
+    """Times rt_decode_step (one new token per sequence through every layer, attention over the whole cache) at a
+    given cache length, in the stack shape of the workload; prints one JSON object.  The caches are filled with
+    seeded random values (the step's cost does not depend on them)."""
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    wl = get_workload(args.workload, args.batch)
+    if not wl.vocab:
+        raise SystemExit("--decode-bench needs a stack workload (c4)")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    data = inputs.make_inputs(wl, N=8)
+    st = rt.Stack(wl.n_layers, wl.d_model, wl.n_heads, wl.d_ff, wl.vocab, dtype=wl.dtype, residual_scale=wl.residual_scale)
+    st.set_weights(data["layers"], data["emb"])
+    out = []
+    g = torch.Generator(device=dev); g.manual_seed(BASE_TILE_SEED + 1)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    esz = 2 if wl.dtype == "bf16" else 4
+    for pos in (1024, 4096, 16384):
+        n_max = pos + args.steps + 4
+        st.k_caches = []
+        st.reserve(wl.B, 1, n_max)
+        for t in st.k_caches + st.v_caches:
+            t.copy_(torch.randn(t.shape, generator=g, device=dev).to(t.dtype))
+        need = rt.rt_workspace_bytes(st.cfg, wl.B, 1, wl.n_layers)
+        if st.ws is None or st.ws.numel() < need:
+            st.ws = torch.zeros(need, dtype=torch.uint8, device=dev)
+        ids = torch.randint(0, wl.vocab, (wl.B,), generator=g, device=dev, dtype=torch.int32)
+        logits = torch.empty((wl.B, wl.vocab), dtype=torch.float32, device=dev)
+
+        def step(p):
+            rt._check(rt.rt_decode_step(st.cfg, wl.n_layers, st.layers, st.emb.data_ptr(), None, wl.vocab, ids.data_ptr(),
+                                        wl.B, p, logits.data_ptr(), st._kp, st._vp, st.N_max, st.ws.data_ptr(),
+                                        st.ws.numel(), stream.cuda_stream), "rt_decode_step")
+        for i in range(3):
+            step(pos + i)
+        evs = []
+        for i in range(args.steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); step(pos + 3 + i); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        assert st.status() == rt.RT_OK
+        ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+        cache_bytes = 2.0 * pos * wl.B * wl.d_model * esz * wl.n_layers
+        weight_bytes = (4 * wl.d_model ** 2 + 2 * wl.d_model * wl.d_ff) * esz * wl.n_layers + wl.vocab * wl.d_model * esz
+        gbs = (cache_bytes + weight_bytes) / (ms * 1e-3) / 1e9
+        out.append({"pos": pos, "ms_per_step": ms, "tokens_per_s": wl.B / (ms * 1e-3), "cache_bytes": cache_bytes,
+                    "weight_bytes": weight_bytes, "achieved_gbs": gbs, "frac_of_measured_hbm_peak": gbs / peaks["hbm_gbs"]})
+    print(json.dumps({"decode_bench": wl.name, "B": wl.B, "n_layers": wl.n_layers, "dtype": wl.dtype,
+                      "peak_gbs": peaks["hbm_gbs"], "points": out}))
+    return 0
+
+
 BASE_TILE_SEED = 20260421
 
 
@@ -400,9 +457,12 @@ def main():
                     help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
     ap.add_argument("--tile-bench", action="store_true", help="time Algorithm 2 alone per tile size and exit")
     ap.add_argument("--tile-bench-all", action="store_true", help="with --tile-bench: also sizes beyond N/2")
+    ap.add_argument("--decode-bench", action="store_true", help="time rt_decode_step at several cache lengths and exit")
     args = ap.parse_args()
     if args.tile_bench:
         return run_tile_bench(args)
+    if args.decode_bench:
+        return run_decode_bench(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_cuda(args)

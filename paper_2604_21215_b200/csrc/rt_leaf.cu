@@ -149,7 +149,6 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   float* red = reinterpret_cast<float*>(smem + L.off_red);
   float* ssq_red = reinterpret_cast<float*>(smem + L.off_ssq);
   float* hown = reinterpret_cast<float*>(smem + L.off_hown);
-  float* sq = reinterpret_cast<float*>(smem + L.off_q);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -231,65 +230,59 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
       per = ((nkeys + nch - 1) / nch + 31) & ~31;
       nch = (nkeys + per - 1) / per;
       const int units = B * H * nch;
-      float* my_q = sq + warp * kHeadDim;
       for (int u = cta + G * warp; u < units; u += G * kLeafWarps) {
         const int c = u % nch, bh = u / nch, b = bh / H, h = bh % H;
         const int j0 = p.attn_begin + c * per;
         const int j1 = (j0 + per < t) ? j0 + per : t;
         const T* qrow = xq + ((size_t)row * B + b) * d + h * kHeadDim;
-        __syncwarp();
-        my_q[2 * lane] = to_f(qrow[2 * lane]);
-        my_q[2 * lane + 1] = to_f(qrow[2 * lane + 1]);
-        __syncwarp();
+        const float q0 = to_f(qrow[2 * lane]), q1 = to_f(qrow[2 * lane + 1]);      // this lane's two dimensions
+        // The pair revealed by the previous step of this launch is still un-normalised in ex_k: the warp
+        // applies qkRMS (Eq. 1), writes the cache row and keeps the rounded values for its own product.
+        const bool fresh = (t - 1 >= p.t0) && (t - 1 >= j0) && (t - 1 < j1);
+        float kn0 = 0.f, kn1 = 0.f;
+        if (fresh) {
+          const float2 r2 = __ldcg(reinterpret_cast<const float2*>(p.ex_k + (size_t)b * d + h * kHeadDim + 2 * lane));
+          const float ss = warp_sum(r2.x * r2.x + r2.y * r2.y);
+          const float rs = qkn ? rsqrtf(ss * (1.0f / kHeadDim) + p.eps) : 1.0f;
+          const float g0 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane) : 1.0f;
+          const float g1 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane + 1) : 1.0f;
+          T* kdst = kc + ((size_t)(t - 1) * B + b) * d + h * kHeadDim + 2 * lane;
+          const T ka = from_f<T>(r2.x * rs * g0), kb = from_f<T>(r2.y * rs * g1);
+          kdst[0] = ka; kdst[1] = kb;
+          kn0 = to_f(ka); kn1 = to_f(kb);
+        }
         float m_run = -INFINITY, l_run = 0.f, o0 = 0.f, o1 = 0.f;
         for (int jb = j0; jb < j1; jb += 32) {
-          const int j = jb + lane;
-          const bool valid = j < j1;
-          float s = 0.f;
-          if (valid) {
-            if (j == t - 1 && j >= p.t0) {
-              // revealed by the previous step of this launch: still un-normalised in ex_k
-              const float* raw = p.ex_k + (size_t)b * d + h * kHeadDim;
-              float ss = 0.f;
-#pragma unroll 4
-              for (int e = 0; e < kHeadDim; e += 4) {
-                const float4 r4 = ldcg_f4(raw + e);
-                ss += r4.x * r4.x + r4.y * r4.y + r4.z * r4.z + r4.w * r4.w;
-              }
-              const float rs = qkn ? rsqrtf(ss * (1.0f / kHeadDim) + p.eps) : 1.0f;
-              T* kdst = kc + ((size_t)j * B + b) * d + h * kHeadDim;
-#pragma unroll 4
-              for (int e = 0; e < kHeadDim; e += 4) {
-                const float4 r4 = ldcg_f4(raw + e);
-                const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+          const int cnt = (j1 - jb < 32) ? (j1 - jb) : 32;
+          // K: one coalesced row load per key (lanes over the head's dimensions), all 32 in flight, then a
+          // transposed reduction leaves the score of key jb + lane in this lane
+          float prod[32];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float gk = qkn ? gain_at(g_k, h * kHeadDim + e + i) : 1.0f;
-                  const T kq = from_f<T>(rr[i] * rs * gk);
-                  kdst[e + i] = kq;
-                  s += my_q[e + i] * to_f(kq);
-                }
-              }
-            } else {
-              const T* krow = kc + ((size_t)j * B + b) * d + h * kHeadDim;
-#pragma unroll 4
-              for (int e = 0; e < kHeadDim; e += 2) {
-                const float2 k2 = ldcg_T2(krow + e);
-                s += my_q[e] * k2.x + my_q[e + 1] * k2.y;
-              }
-            }
+          for (int jj = 0; jj < 32; ++jj) {
+            const int j = jb + (jj < cnt ? jj : 0);
+            float2 k2 = ldcg_T2(kc + ((size_t)j * B + b) * d + h * kHeadDim + 2 * lane);
+            if (fresh && j == t - 1) k2 = make_float2(kn0, kn1);
+            prod[jj] = q0 * k2.x + q1 * k2.y;
           }
-          const float s2 = valid ? s * p.scale_log2 : -INFINITY;
+          // V rows of the batch, requested before the scores are needed
+          float2 vv[32];
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            const int j = jb + (jj < cnt ? jj : 0);
+            vv[jj] = ldcg_T2(vc + ((size_t)j * B + b) * d + h * kHeadDim + 2 * lane);
+          }
+          warp_transpose_sum32(prod, lane);
+          const bool valid = lane < cnt;
+          const float s2 = valid ? prod[0] * p.scale_log2 : -INFINITY;
           const float m_new = fmaxf(m_run, warp_max(s2));
           const float pj = valid ? exp2f(s2 - m_new) : 0.f;
           const float corr = exp2f(m_run - m_new);
           l_run = l_run * corr + warp_sum(pj);
           o0 *= corr; o1 *= corr;
-          const int cnt = (j1 - jb < 32) ? (j1 - jb) : 32;
-          for (int jj = 0; jj < cnt; ++jj) {
-            const float pw = __shfl_sync(0xffffffffu, pj, jj);
-            const float2 v2 = ldcg_T2(vc + ((size_t)(jb + jj) * B + b) * d + h * kHeadDim + 2 * lane);
-            o0 += pw * v2.x; o1 += pw * v2.y;
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            const float pw = __shfl_sync(0xffffffffu, pj, jj);       // 0 for the keys beyond cnt
+            o0 += pw * vv[jj].x; o1 += pw * vv[jj].y;
           }
           m_run = m_new;
         }
