@@ -154,3 +154,43 @@ def test_stack_full_size_is_consistent_with_its_layers():
     h_last = hid[:, -1].to(torch.float64).cpu().numpy()
     ref_logits = rms(h_last, np.ones(d), cfg.rms_eps) @ np.asarray(data["emb"], dtype=np.float64).T
     assert rel_err(logits.to(torch.float64).cpu().numpy(), ref_logits) <= TOL["bf16"]
+
+
+def _random_cases():
+    rng = np.random.default_rng(20260421)
+    cases = []
+    for i in range(14):
+        H = int(rng.choice([1, 2, 3, 4, 5, 8]))
+        d = 64 * H
+        dff = int(rng.choice([128, 208, 384, 1024, 1536]))
+        B = int(rng.integers(1, 17))
+        N = int(rng.integers(1, 420))
+        leaf = int(rng.choice([0, 16, 32, 64]))
+        dtype = "bf16" if i % 3 else "f32"
+        flags = int(rng.choice([3, 3, 3, 1, 2, 0, 3 | 8]))
+        gains = bool(rng.integers(0, 2))
+        alpha = float(rng.choice([1.0, 0.5, 1 / np.sqrt(8)]))
+        cases.append((dtype, d, H, dff, B, N, leaf, flags, gains, alpha))
+    return cases
+
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N,leaf,flags,gains,alpha", _random_cases())
+def test_random_shapes_match_oracle(dtype, d, H, dff, B, N, leaf, flags, gains, alpha):
+    # Shapes off the beaten path: head counts that are not powers of two, MLP widths that are not
+    # multiples of 64, every batch size up to 16, lengths with ragged last leaves, every leaf size,
+    # norm flags, gains and residual scales; tiled schedule, both storage types.
+    from oracle import RTConfig, RTWeights, layer_seq
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("rnd", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=7000 + d + dff + B + N)
+    lw = data["layers"][0]
+    if gains:
+        rng = np.random.default_rng(N)
+        for g in ("g_attn", "g_mlp", "g_kv", "g_q", "g_k"):
+            lw[g] = inputs.round_to(1.0 + 0.2 * rng.standard_normal(d), dtype)
+    ref = layer_seq(RTConfig(d, H, 64, dff, norm_flags=flags, residual_scale=alpha), RTWeights(**lw), data["x"])
+    layer = _layer(d, H, dff, dtype, lw, leaf=leaf, norm_flags=flags, residual_scale=alpha)
+    got = layer.prefill(data["x"])
+    for name, g_, r_ in zip(("z", "k", "v"), got, ref):
+        assert np.isfinite(g_).all(), name
+        assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
