@@ -22,7 +22,7 @@ independent (the paper states everything per sequence).
 from __future__ import annotations
 
 from dataclasses import dataclass
-from typing import List, Optional, Tuple
+from typing import Sequence, List, Optional, Tuple
 
 import numpy as np
 
@@ -51,11 +51,19 @@ class RTConfig:
     rms_eps: float = 1e-6
     softmax_scale: Optional[float] = None   # None -> 1/sqrt(head_dim); 1.0 = Sec. 2's literal Attn
     residual_scale: float = 1.0             # alpha = 1/sqrt(L)  (Sec. 2, pre-LN parameterisation)
+    alibi_slopes: Optional[Sequence[float]] = None   # [H]; logit of query i on the persistent pair j gets
+                                                     # -slope_h (i - j) (App. D: ALiBi); None = no bias
 
     def __post_init__(self):
         assert self.n_heads * self.head_dim == self.d_model
         if self.softmax_scale is None:
             self.softmax_scale = 1.0 / np.sqrt(self.head_dim)
+        if self.alibi_slopes is not None:
+            self.alibi_slopes = np.asarray(self.alibi_slopes, dtype=np.float64)
+            assert self.alibi_slopes.shape == (self.n_heads,)
+
+    def slope(self, h: int) -> float:
+        return 0.0 if self.alibi_slopes is None else float(self.alibi_slopes[h])
 
 
 @dataclass
@@ -112,10 +120,13 @@ def gelu(a: np.ndarray) -> np.ndarray:
     return 0.5 * a * (1.0 + _erf(a / np.sqrt(2.0)))
 
 
-def attn(keys: np.ndarray, values: np.ndarray, q: np.ndarray, scale: float) -> np.ndarray:
+def attn(keys: np.ndarray, values: np.ndarray, q: np.ndarray, scale: float, bias=None) -> np.ndarray:
     """The Attn operator of Sec. 2 for one head and one query:
-    sum_i v_i exp(s<k_i,q>) / sum_j exp(s<k_j,q>);  keys, values [l, dh], q [dh]."""
+    sum_i v_i exp(s<k_i,q>) / sum_j exp(s<k_j,q>);  keys, values [l, dh], q [dh].
+    bias [l] (optional) is added to the logits (the ALiBi distances of App. D)."""
     logits = scale * (keys @ q)
+    if bias is not None:
+        logits = logits + bias
     p = np.exp(logits - logits.max())
     p /= p.sum()
     return p @ values
@@ -166,6 +177,8 @@ def layer_seq(cfg: RTConfig, w: RTWeights, x: np.ndarray):
         qh = q.reshape(B, H, dh)
         # logits against the i persistent pairs of earlier positions, then the temporary pair
         lp = s * np.einsum("bjhe,bhe->bhj", k[:, :i].reshape(B, i, H, dh), qh)
+        if cfg.alibi_slopes is not None:             # distance i - j to the persistent pair j; 0 to the temporary pair
+            lp = lp - cfg.alibi_slopes[None, :, None] * (i - np.arange(i))[None, None, :]
         lt = s * np.sum(qh * kt.reshape(B, H, dh), axis=-1, keepdims=True)
         logits = np.concatenate([lp, lt], axis=-1)                     # [B, H, i+1]
         p = np.exp(logits - logits.max(axis=-1, keepdims=True))
@@ -179,10 +192,13 @@ def layer_seq(cfg: RTConfig, w: RTWeights, x: np.ndarray):
 
 # ----------------------------------------------------------------------------- Alg. 2 and Alg. 1
 
-def update_tile(qs, ks, vs, m, l, o, scale):
+def update_tile(qs, ks, vs, m, l, o, scale, bias=None):
     """Algorithm 2 (UpdateTile) for one head: queries qs [nq, dh], tile ks, vs [nk, dh],
-    running stats m [nq], l [nq], o [nq, dh]; returns the updated (m, l, o)."""
+    running stats m [nq], l [nq], o [nq, dh]; returns the updated (m, l, o).
+    bias [nq, nk] (optional) is added to the tile logits."""
     al = scale * (qs @ ks.T)                      # tile logits
+    if bias is not None:
+        al = al + bias
     m_tile = al.max(axis=1)
     m_new = np.maximum(m, m_tile)
     resc = np.exp(m - m_new)                      # exp(-inf - finite) = 0 on first use
@@ -231,11 +247,15 @@ def layer_blk(cfg: RTConfig, w: RTWeights, x: np.ndarray, leaf: int = 1,
             q[i], kt[i], vt[i] = _temp_qkv(x[b, i], w, cfg)
         m = np.full((H, N), -np.inf); l = np.zeros((H, N)); o = np.zeros((H, N, dh))
 
-        def upd(qlo, qhi, K, V):                        # 0-based half-open query range
-            for h in range(H):
+        def upd(qlo, qhi, K, V, klo=None):              # 0-based half-open query range; klo = position of K[0]
+            for h in range(H):                          # (None: the temporary pair, at distance 0)
                 sl = slice(h * dh, (h + 1) * dh)
+                bias = None
+                if cfg.alibi_slopes is not None and klo is not None:
+                    dist = np.arange(qlo, qhi)[:, None] - (klo + np.arange(K.shape[0]))[None, :]
+                    bias = -cfg.slope(h) * dist
                 m[h, qlo:qhi], l[h, qlo:qhi], o[h, qlo:qhi] = update_tile(
-                    q[qlo:qhi, sl], K[:, sl], V[:, sl], m[h, qlo:qhi], l[h, qlo:qhi], o[h, qlo:qhi], s)
+                    q[qlo:qhi, sl], K[:, sl], V[:, sl], m[h, qlo:qhi], l[h, qlo:qhi], o[h, qlo:qhi], s, bias)
 
         for t in range(1, N + 1):                       # 1-based as in the algorithm
             i = t - 1
@@ -243,7 +263,7 @@ def layer_blk(cfg: RTConfig, w: RTWeights, x: np.ndarray, leaf: int = 1,
             if self_first:
                 upd(i, i + 1, kt[i:i + 1], vt[i:i + 1])
             if not eager_leaf and i > start:
-                upd(i, i + 1, k[b, start:i], v[b, start:i])
+                upd(i, i + 1, k[b, start:i], v[b, start:i], start)
             if not self_first:
                 upd(i, i + 1, kt[i:i + 1], vt[i:i + 1])
             c = np.concatenate([o[h, i] / l[h, i] for h in range(H)])        # a_t = o_t / l_t per head
@@ -252,10 +272,10 @@ def layer_blk(cfg: RTConfig, w: RTWeights, x: np.ndarray, leaf: int = 1,
             if eager_leaf:
                 hi = min(start + leaf, N)
                 if i + 1 < hi:
-                    upd(i + 1, hi, k[b, i:i + 1], v[b, i:i + 1])
+                    upd(i + 1, hi, k[b, i:i + 1], v[b, i:i + 1], i)
             if t in tiles:
                 u, vv, s0, e0 = tiles[t]
-                upd(u - 1, vv, k[b, s0 - 1:e0], v[b, s0 - 1:e0])
+                upd(u - 1, vv, k[b, s0 - 1:e0], v[b, s0 - 1:e0], s0 - 1)
     return z, k, v
 
 
@@ -283,7 +303,8 @@ def layer_fixed_point(cfg: RTConfig, w: RTWeights, x: np.ndarray, z_claim: np.nd
                 sl = slice(h * dh, (h + 1) * dh)
                 keys = np.concatenate([k[b, :i, sl], kt[b, i:i + 1, sl]])
                 vals = np.concatenate([v[b, :i, sl], vt[b, i:i + 1, sl]])
-                c[sl] = attn(keys, vals, q[b, i, sl], s)
+                bias = None if cfg.alibi_slopes is None else -cfg.slope(h) * (i - np.arange(i + 1))
+                c[sl] = attn(keys, vals, q[b, i, sl], s, bias)
             a = c @ w.w_o.T
             hres = x[b, i] + cfg.residual_scale * a
             z2[b, i] = hres + cfg.residual_scale * _mlp(hres, w, cfg)
@@ -307,7 +328,8 @@ def layer_decode(cfg: RTConfig, w: RTWeights, x_new: np.ndarray, k_cache: np.nda
             sl = slice(h * dh, (h + 1) * dh)
             keys = np.concatenate([k_cache[b, :pos, sl], kt[None, sl]])
             vals = np.concatenate([v_cache[b, :pos, sl], vt[None, sl]])
-            c[sl] = attn(keys, vals, q[sl], s)
+            bias = None if cfg.alibi_slopes is None else -cfg.slope(h) * (pos - np.arange(pos + 1))
+            c[sl] = attn(keys, vals, q[sl], s, bias)
         z[b], k_cache[b, pos], v_cache[b, pos] = _output_and_persistent(x_new[b], c @ w.w_o.T, w, cfg)
     return z
 

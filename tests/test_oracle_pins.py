@@ -345,3 +345,102 @@ def test_stack_prefill_then_decode_and_tied_head():
     assert np.allclose(lg, logits, rtol=1e-10, atol=1e-11)
     for (k, v), (kk, vv) in zip(caches, caches5):
         assert np.allclose(k, kk, rtol=1e-10, atol=1e-11) and np.allclose(v, vv, rtol=1e-10, atol=1e-11)
+
+
+# ------------------------------------------------------------------ ALiBi distances (App. D: "alibi positional embeddings")
+
+def geometric_slopes(H, max_bias=8.0):
+    # head h (1-based) gets 2^(-max_bias h / H): the geometric sequence of the ALiBi paper for H a power of two
+    return np.array([2.0 ** (-max_bias * (h + 1) / H) for h in range(H)])
+
+
+def test_alibi_zero_query_gives_geometric_weights():
+    # W_q = 0: every content logit is 0, so position i weighs the persistent pair j by r^(i-j),
+    # r = exp(-slope_h), and its own temporary pair by 1 (distance 0): a geometric moving average.
+    rng = np.random.default_rng(40)
+    H = 2
+    cfg, w = rand_layer(rng, 16, H, 24, alpha=0.7)
+    cfg.alibi_slopes = np.array([0.3, 1.1])
+    w.w_q = np.zeros_like(w.w_q)
+    w.w_down = np.zeros_like(w.w_down)            # z_i = x_i + alpha W_o c_i exposes c_i
+    x = rng.standard_normal((2, 10, 16))
+    z, k, v = layer_seq(cfg, w, x)
+    n = x / np.sqrt((x ** 2).mean(-1, keepdims=True) + cfg.rms_eps)
+    vt = n @ w.w_v.T
+    for i in range(10):
+        c = np.zeros((2, 16))
+        for h in range(H):
+            sl = slice(8 * h, 8 * h + 8)
+            r = math.exp(-cfg.alibi_slopes[h])
+            num = vt[:, i, sl].copy()
+            den = 1.0
+            for j in range(i):
+                num += r ** (i - j) * v[:, j, sl]
+                den += r ** (i - j)
+            c[:, sl] = num / den
+        assert np.allclose((z[:, i] - x[:, i]) / 0.7, c @ w.w_o.T, rtol=1e-11, atol=1e-12)
+
+
+def test_alibi_two_block_construction_equals_textbook_alibi_attention():
+    # The construction under which the layer is plain causal attention (App. A), with distances:
+    # dense softmax(s Q K^T - slope_h |i - j|) V with the diagonal at distance 0.
+    e, N, B, H = 4, 9, 2, 2
+    dh, d = 2 * e, 2 * e * H
+    rng = np.random.default_rng(41)
+    carry = np.array([h * dh + j for h in range(H) for j in range(e)])
+    scratch = carry + e
+    QT, KT, VT = (rng.standard_normal((H * e, H * e)) for _ in range(3))
+    Wq = np.zeros((d, d)); Wk = np.zeros((d, d)); Wv = np.zeros((d, d))
+    Wq[np.ix_(carry, carry)] = QT
+    Wk[np.ix_(carry, carry)] = KT
+    Wv[np.ix_(scratch, carry)] = VT
+    slopes = geometric_slopes(H)
+    cfg = RTConfig(d, H, dh, 5, norm_flags=0, softmax_scale=0.41, alibi_slopes=slopes)
+    w = RTWeights(Wq, Wk, Wv, np.eye(d), rng.standard_normal((5, d)), np.zeros((d, 5)))
+    c = rng.standard_normal((B, N, H * e))
+    x = np.zeros((B, N, d)); x[..., carry] = c
+    z, _, _ = layer_seq(cfg, w, x)
+    Q = c @ QT.T; K = c @ KT.T; Vv = c @ VT.T
+    dist = np.arange(N)[:, None] - np.arange(N)[None, :]
+    for b in range(B):
+        for h in range(H):
+            sl = slice(h * e, (h + 1) * e)
+            S = 0.41 * Q[b, :, sl] @ K[b, :, sl].T - slopes[h] * dist
+            S[np.triu_indices(N, 1)] = -np.inf
+            P = np.exp(S - S.max(axis=1, keepdims=True))
+            P /= P.sum(axis=1, keepdims=True)
+            assert np.allclose(z[b][:, scratch[sl]], P @ Vv[b, :, sl], rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("leaf,self_first,eager", [(1, True, False), (4, False, False), (8, True, True), (16, True, False)])
+def test_alibi_blocked_fixed_point_and_decode_agree_with_sequential(leaf, self_first, eager):
+    rng = np.random.default_rng(42)
+    H = 4
+    cfg, w = rand_layer(rng, 32, H, 40, alpha=0.6, gains=True)
+    cfg.alibi_slopes = geometric_slopes(H)
+    x = rng.standard_normal((2, 21, 32))
+    z, k, v = layer_seq(cfg, w, x)
+    z2, k2, v2 = layer_blk(cfg, w, x, leaf=leaf, self_first=self_first, eager_leaf=eager)
+    assert np.allclose(z2, z, rtol=1e-10, atol=1e-11) and np.allclose(k2, k, rtol=1e-10, atol=1e-11)
+    z3, k3, v3 = layer_fixed_point(cfg, w, x, z)
+    assert np.allclose(z3, z, rtol=1e-10, atol=1e-11)
+    kc = np.zeros((2, 21, 32)); vc = np.zeros((2, 21, 32))
+    kc[:, :20], vc[:, :20] = k[:, :20], v[:, :20]
+    zn = layer_decode(cfg, w, x[:, 20], kc, vc, 20)
+    assert np.allclose(zn, z[:, 20], rtol=1e-10, atol=1e-11)
+
+
+def test_alibi_limits():
+    # slope 0 is no bias at all; a very large slope leaves only the temporary pair (distance 0)
+    rng = np.random.default_rng(43)
+    cfg, w = rand_layer(rng, 16, 2, 24)
+    x = rng.standard_normal((1, 8, 16))
+    z0, _, _ = layer_seq(cfg, w, x)
+    cfg.alibi_slopes = np.zeros(2)
+    z1, _, _ = layer_seq(cfg, w, x)
+    assert np.array_equal(z0, z1)
+    cfg.alibi_slopes = np.full(2, 1e4)
+    w.w_down = np.zeros_like(w.w_down)
+    z2, _, _ = layer_seq(cfg, w, x)
+    n = x / np.sqrt((x ** 2).mean(-1, keepdims=True) + cfg.rms_eps)
+    assert np.allclose(z2 - x, (n @ w.w_v.T) @ w.w_o.T, rtol=1e-12, atol=1e-13)
