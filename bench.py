@@ -91,6 +91,11 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def alibi_slopes(n_heads, max_bias=8.0):
+    """Geometric slopes 2^(-max_bias h / H), h = 1..H (the paper's experiments: maximum bias 8)."""
+    return [2.0 ** (-max_bias * (h + 1) / n_heads) for h in range(n_heads)]
+
+
 def get_workload(name, batch=0):
     import dataclasses
     from paper_2604_21215_b200 import inputs
@@ -112,8 +117,9 @@ def config_dict(wl, sched, extra=None):
 def oracle_sample(wl, data, n_pos):
     """Runs the oracle, as it stands, on the first n_pos positions of the workload; returns seconds."""
     from oracle import RTConfig, RTWeights, layer_seq, stack_prefill
-    cfg = RTConfig(wl.d_model, wl.n_heads, wl.head_dim, wl.d_ff, residual_scale=wl.residual_scale)
-    layers = [RTWeights(**lw) for lw in data["layers"]]
+    cfg = RTConfig(wl.d_model, wl.n_heads, wl.head_dim, wl.d_ff, residual_scale=wl.residual_scale,
+                   alibi_slopes=data["layers"][0].get("alibi_slopes"))
+    layers = [RTWeights(**{k: v for k, v in lw.items() if k != "alibi_slopes"}) for lw in data["layers"]]
     t0 = time.perf_counter()
     if wl.vocab:
         stack_prefill(cfg, layers, data["emb"], None, data["ids"][:, :n_pos])
@@ -187,6 +193,9 @@ def run_cuda(args):
     leaf_kw = {"leaf": args.leaf} if args.leaf else {}
     stream = torch.cuda.current_stream(dev)
 
+    if args.alibi:                                     # the same slopes for every layer
+        for lw in data["layers"]:
+            lw["alibi_slopes"] = alibi_slopes(wl.n_heads)
     if wl.vocab:
         model = rt.Stack(wl.n_layers, wl.d_model, wl.n_heads, wl.d_ff, wl.vocab, dtype=wl.dtype, device=str(dev),
                          sched=args.sched, residual_scale=wl.residual_scale, **leaf_kw)
@@ -314,7 +323,7 @@ def run_cuda(args):
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16/f32-accumulate" if wl.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": config_dict(wl, args.sched, {"leaf": int(model.cfg.leaf) or 64,
+                "data": "synthetic", "config": config_dict(wl, args.sched, {"alibi": bool(args.alibi), "leaf": int(model.cfg.leaf) or 64,
                                                                             "parallelism": f"replicas x{world}"}),
                 "clocks": clocks,
                 "e2e": {"value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, e2e_total), "unit": UNIT,
@@ -352,6 +361,8 @@ def run_tile_bench(args):
     stream = torch.cuda.current_stream(dev)
     out = []
     g = torch.Generator(device=dev); g.manual_seed(BASE_TILE_SEED)
+    slopes = torch.tensor(alibi_slopes(wl.n_heads), dtype=torch.float32, device=dev) if args.alibi else None
+    alibi_ptr = slopes.data_ptr() if args.alibi else None
     for P in (64, 128, 256, 512, 1024, 2048, 4096):
         if P > wl.N // 2 and not args.tile_bench_all:
             break
@@ -363,7 +374,7 @@ def run_tile_bench(args):
         m = torch.zeros((rows, wl.B, wl.n_heads), dtype=torch.float32, device=dev)
         l = torch.ones((rows, wl.B, wl.n_heads), dtype=torch.float32, device=dev)
         call = lambda: rt.rt_update_tile(cfg, q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), m.data_ptr(),
-                                         l.data_ptr(), wl.B, rows, rows, P, 2 * P, 0, P, ws.data_ptr(), stream.cuda_stream)
+                                         l.data_ptr(), wl.B, rows, rows, P, 2 * P, 0, P, alibi_ptr, ws.data_ptr(), stream.cuda_stream)
         for _ in range(3):
             assert call() == rt.RT_OK
         evs = []
@@ -378,7 +389,7 @@ def run_tile_bench(args):
         flops = 4.0 * P * P * 64 * wl.B * wl.n_heads
         tf = flops / (ms * 1e-3) / 1e12
         out.append({"P": P, "ms": ms, "tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"]})
-    print(json.dumps({"tile_bench": wl.name, "B": wl.B, "H": wl.n_heads, "dtype": wl.dtype,
+    print(json.dumps({"tile_bench": wl.name, "B": wl.B, "H": wl.n_heads, "dtype": wl.dtype, "alibi": bool(args.alibi),
                       "peak_tflops": peaks["bf16_tflops"], "tiles": out}))
     return 0
 
@@ -457,6 +468,8 @@ def main():
                     help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
     ap.add_argument("--tile-bench", action="store_true", help="time Algorithm 2 alone per tile size and exit")
     ap.add_argument("--tile-bench-all", action="store_true", help="with --tile-bench: also sizes beyond N/2")
+    ap.add_argument("--alibi", action="store_true",
+                    help="add ALiBi distances (slopes 2^(-8 h / H), h = 1..H) to the attention logits")
     ap.add_argument("--decode-bench", action="store_true", help="time rt_decode_step at several cache lengths and exit")
     args = ap.parse_args()
     if args.tile_bench:

@@ -78,6 +78,9 @@ typedef struct {            /* device pointers; read-only */
   const void *w_down;                  /* [d_model, d_ff]   MLP(u) = w_down GELU(w_up u), exact (erf) GELU, no biases */
   const void *g_attn, *g_mlp, *g_kv;   /* [d_model] RMS gains of RMS(x), the MLP pre-norm and RMS(z); NULL = ones; g_kv NULL = g_attn */
   const void *g_q, *g_k;               /* [d_model] qkRMS gains; NULL = ones */
+  const float *alibi_slopes;           /* [n_heads] fp32, or NULL for none.  ALiBi distances (App. D: the paper's experiments
+                                          use them, maximum bias 8): the logit of query i on the persistent pair of position j
+                                          gets -alibi_slopes[h] * (i - j); the temporary pair of position i sits at distance 0 */
 } rt_layer_weights;
 
 /* Bytes of workspace a call with these shapes needs (N = positions per call: the prefill
@@ -166,7 +169,9 @@ rt_status rt_plan_counters(const rt_config *cfg, int32_t B, int32_t N, int32_t n
 /* Algorithm 2 (UpdateTile, App. C) on its own: queries [q0,q1) of `q` attend to the pairs [k0,k1) of
  * the caches, for every sequence and head, and their running stats are updated in place:
  *   m_new = max(m, max_j a_ij),  o = o*e^(m-m_new) + sum_j v_j e^(a_ij-m_new),  l likewise,  m = m_new,
- * with a_ij = softmax_scale <q_i, k_j>.  The library keeps m in log2 units: st_m holds log2(e)*m.
+ * with a_ij = softmax_scale <q_i, k_j> - alibi_slopes[h] * (i - j)  (rows of q and of the caches are positions;
+ * alibi_slopes [n_heads] fp32 on the device, or NULL for no distance term).  The library keeps m in log2 units:
+ * st_m holds log2(e)*m.
  * q [rows_q, B, d] and the caches [rows_kv, B, d] are position-major, storage type; st_o [rows_q, B, d],
  * st_m, st_l [rows_q, B, n_heads] are fp32.  `workspace` needs 256 bytes (device status word, read with
  * rt_get_status).  This is the cross-block step of rt_layer_prefill, exposed for tests and benchmarks. */
@@ -174,7 +179,7 @@ rt_status rt_update_tile(const rt_config *cfg, const void *q, const void *k_cach
                          float *st_o, float *st_m, float *st_l,
                          int32_t B, int32_t rows_q, int32_t rows_kv,
                          int32_t q0, int32_t q1, int32_t k0, int32_t k1,
-                         void *workspace, void *cuda_stream);
+                         const float *alibi_slopes, void *workspace, void *cuda_stream);
 
 /* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues a two-CTA kernel
  * whose grid barrier expects an arrival that never comes.  The wait gives up after its limit (2 s),

@@ -145,7 +145,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   lp.B = B; lp.d = c->d_model; lp.H = c->n_heads; lp.dff = c->d_ff;
   lp.norm_flags = c->norm_flags; lp.eps = c->rms_eps; lp.scale_log2 = scale_log2; lp.alpha = c->residual_scale;
   lp.w_o = w->w_o; lp.w_up = w->w_up; lp.w_down = w->w_down; lp.w_k = w->w_k; lp.w_v = w->w_v;
-  lp.g_mlp = w->g_mlp; lp.g_kv = w->g_kv ? w->g_kv : w->g_attn; lp.g_k = w->g_k;
+  lp.g_mlp = w->g_mlp; lp.g_kv = w->g_kv ? w->g_kv : w->g_attn; lp.g_k = w->g_k; lp.alibi = w->alibi_slopes;
   lp.x = x; lp.x_bs = x_bs; lp.x_ts = x_ts;
   lp.z = z; lp.z_bs = z_bs; lp.z_ts = z_ts;
   lp.k_cache = k_cache; lp.v_cache = v_cache;
@@ -192,7 +192,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   }
   TileParams tp;
   memset(&tp, 0, sizeof(tp));
-  tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2;
+  tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2; tp.alibi = w->alibi_slopes;
   tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
   tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
   tp.rows_q = n_rows; tp.rows_kv = n_max; tp.sync = lp.sync;
@@ -352,7 +352,7 @@ rt_status rt_get_status(const void* workspace) {
 
 rt_status rt_update_tile(const rt_config* cfg, const void* q, const void* k_cache, const void* v_cache, float* st_o,
                          float* st_m, float* st_l, int32_t B, int32_t rows_q, int32_t rows_kv, int32_t q0, int32_t q1,
-                         int32_t k0, int32_t k1, void* workspace, void* cuda_stream) {
+                         int32_t k0, int32_t k1, const float* alibi_slopes, void* workspace, void* cuda_stream) {
   if (!config_ok(cfg) || B <= 0 || !q || !k_cache || !v_cache || !st_o || !st_m || !st_l || !workspace)
     return RT_ERR_INVALID_ARG;
   if (q0 < 0 || q1 < q0 || q1 > rows_q || k0 < 0 || k1 < k0 || k1 > rows_kv) return RT_ERR_INVALID_ARG;
@@ -364,7 +364,7 @@ rt_status rt_update_tile(const rt_config* cfg, const void* q, const void* k_cach
   if (cudaMemsetAsync(workspace, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
   TileParams tp;
   memset(&tp, 0, sizeof(tp));
-  tp.B = B; tp.d = cfg->d_model; tp.H = cfg->n_heads; tp.scale_log2 = cfg->softmax_scale * kLog2e;
+  tp.B = B; tp.d = cfg->d_model; tp.H = cfg->n_heads; tp.scale_log2 = cfg->softmax_scale * kLog2e; tp.alibi = alibi_slopes;
   tp.q = q; tp.k_cache = k_cache; tp.v_cache = v_cache;
   tp.st_o = st_o; tp.st_m = st_m; tp.st_l = st_l;
   tp.q0 = q0; tp.q1 = q1; tp.k0 = k0; tp.k1 = k1;

@@ -16,6 +16,7 @@ struct LeafParams {
   float eps, scale_log2, alpha;
   const void *w_o, *w_up, *w_down, *w_k, *w_v;   // storage type
   const void *g_mlp, *g_kv, *g_k;                // storage type or NULL
+  const float* alibi;                            // [H] slopes of the ALiBi distances (natural-log units) or NULL
   const void* x;  long long x_bs, x_ts;          // x[b, t, :] = x + b*x_bs + (t-row_off)*x_ts   (elements)
   void* z;        long long z_bs, z_ts;
   void *k_cache, *v_cache;                       // [N_max, B, d] storage type
@@ -72,6 +73,7 @@ cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStrea
 struct TileParams {
   int B, d, H;
   float scale_log2;
+  const float* alibi;                            // [H] slopes of the ALiBi distances (natural-log units) or NULL
   const void* q;                                 // [N, B, d]
   const void *k_cache, *v_cache;                 // [N_max, B, d]
   float *st_o, *st_m, *st_l;

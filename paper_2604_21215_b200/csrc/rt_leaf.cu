@@ -236,6 +236,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
         const int j1 = (j0 + per < t) ? j0 + per : t;
         const T* qrow = xq + ((size_t)row * B + b) * d + h * kHeadDim;
         const float q0 = to_f(qrow[2 * lane]), q1 = to_f(qrow[2 * lane + 1]);      // this lane's two dimensions
+        const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;                 // ALiBi distances, log2 units
         // The pair revealed by the previous step of this launch is still un-normalised in ex_k: the warp
         // applies qkRMS (Eq. 1), writes the cache row and keeps the rounded values for its own product.
         const bool fresh = (t - 1 >= p.t0) && (t - 1 >= j0) && (t - 1 < j1);
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
           }
           warp_transpose_sum32(prod, lane);
           const bool valid = lane < cnt;
-          const float s2 = valid ? prod[0] * p.scale_log2 : -INFINITY;
+          const float s2 = valid ? prod[0] * p.scale_log2 - slope_l2 * (float)(t - (jb + lane)) : -INFINITY;
           const float m_new = fmaxf(m_run, warp_max(s2));
           const float pj = valid ? exp2f(s2 - m_new) : 0.f;
           const float corr = exp2f(m_run - m_new);

@@ -194,6 +194,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(p.k_cache);
   __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(p.v_cache);
   const bool qkn = (p.norm_flags & RT_NORM_QK) != 0;
+  const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;     // ALiBi distances, in log2 units
 
   // queries and carried stats of the leaf (written by earlier kernels of this call)
   for (int i = 0; i < n; ++i) {
@@ -254,7 +255,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
       // critical path: finish query j+1 and publish c_{j+1}
       const int i = j + 1;
       const unsigned qw = *reinterpret_cast<const unsigned*>(qs + i * kQStride + 2 * lane);
-      const float s = warp_sum(bf_lo(qw) * kf0 + bf_hi(qw) * kf1) * p.scale_log2;
+      const float s = warp_sum(bf_lo(qw) * kf0 + bf_hi(qw) * kf1) * p.scale_log2 - slope_l2;      // distance (j+1) - j = 1
       const float m_old = ms[i], l_old = ls[i];
       const float m_new = fmaxf(m_old, s);
       const float corr = exp2f(m_old - m_new), pj = exp2f(s - m_new);
@@ -275,7 +276,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
         const unsigned qw = *reinterpret_cast<const unsigned*>(qi + e);
         s += bf_lo(qw) * kbuf[e] + bf_hi(qw) * kbuf[e + 1];
       }
-      s *= p.scale_log2;
+      s = s * p.scale_log2 - slope_l2 * (float)(i - j);
       const float m_old = ms[i];
       const float m_new = fmaxf(m_old, s);
       const float corr = exp2f(m_old - m_new), pj = exp2f(s - m_new);

@@ -2,6 +2,7 @@
 // pairs [k0,k1), for every sequence and head, with the running stats (m, l, o) carried in
 // fp32 between tiles.  This file holds the SIMT version (fp32 mode, and any shape the
 // tensor-core version does not take).  m is kept in log2 units: p = 2^(s*log2e*<q,k> - m).
+// With ALiBi distances the logit of query i on pair j also gets -slope_h (i - j) (times log2e).
 #include "rt_kernels.h"
 
 namespace rt {
@@ -22,6 +23,7 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
   const T* Vc = reinterpret_cast<const T*>(p.v_cache);
   const size_t col0 = (size_t)b * p.d + h * kHeadDim;
   const size_t rstride = (size_t)p.B * p.d;
+  const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
 
   for (int i = tid; i < kTQ * kHeadDim; i += 128) {
     const int r = i / kHeadDim, e = i % kHeadDim;
@@ -56,7 +58,7 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
       float s = 0.f;
 #pragma unroll 16
       for (int e = 0; e < kHeadDim; ++e) s += Qs[qr][e] * Ks[lane][e];
-      const float s2 = valid ? s * p.scale_log2 : -INFINITY;
+      const float s2 = valid ? s * p.scale_log2 - slope_l2 * (float)(qb + qr - (kb + lane)) : -INFINITY;
       const float m_new = fmaxf(m[i], warp_max(s2));
       const float pj = valid ? exp2f(s2 - m_new) : 0.f;
       const float corr = exp2f(m[i] - m_new);

@@ -156,6 +156,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const uint32_t t_o = t_s + 64u;
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
     float m_used = p.st_m[sidx * p.H + h];                   // reference maximum of l and O (log2 units)
+    const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
+    const float step_raw = slope_l2 / p.scale_log2;          // slope per column, in units of the raw product
     float m_true = m_used;                                   // running maximum
     float l_run = p.st_l[sidx * p.H + h];
     uint32_t s0[32], s1[32];
@@ -179,17 +181,28 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_ld32(t_s, s0);
       tc_ld32(t_s + 32u, s1);
       tc_wait_ld();
+      // ALiBi distances: the logit of this row's query (position qi) on key j gets -slope (qi - j)
+      // = base + slope * column: the column part goes into the raw products (divided by the scale that is
+      // applied below), the row constant into the maximum and the exponent offset
+      const float base_l2 = -slope_l2 * (float)(qi - (p.k0 + kb * kBK));
+      if (slope_l2 != 0.f) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          s0[i] = __float_as_uint(fmaf(step_raw, (float)i, __uint_as_float(s0[i])));
+          s1[i] = __float_as_uint(fmaf(step_raw, (float)(i + 32), __uint_as_float(s1[i])));
+        }
+      }
       float mx4[4];                                            // four independent chains
 #pragma unroll
       for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
 #pragma unroll
       for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      const float mx = fmaf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), p.scale_log2, base_l2);
       m_true = fmaxf(m_true, mx);
       const bool raise = mx > m_used + kLazyLog2;
       const float m_new = raise ? m_true : m_used;
       const float corr = ex2(m_used - m_new);                  // 1 when the reference stays
-      const float neg_m = -m_new;
+      const float neg_m = base_l2 - m_new;
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       // p = 2^(s*scale - m) as packed bf16, written over the first 32 columns of the S buffer
       uint32_t w[16];

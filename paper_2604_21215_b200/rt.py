@@ -37,7 +37,7 @@ class RtConfig(C.Structure):
 
 class RtLayerWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_q", "w_k", "w_v", "w_o", "w_up", "w_down",
-                                           "g_attn", "g_mlp", "g_kv", "g_q", "g_k")]
+                                           "g_attn", "g_mlp", "g_kv", "g_q", "g_k", "alibi_slopes")]
 
 
 class RtCounters(C.Structure):
@@ -72,7 +72,7 @@ def _load():
     lib.rt_selftest_wait_expiry.restype = C.c_int
     lib.rt_selftest_wait_expiry.argtypes = [P, P]
     lib.rt_update_tile.restype = C.c_int
-    lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P]
+    lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P, P]
     lib.rt_stack_prefill.restype = C.c_int
     lib.rt_stack_prefill.argtypes = [C.POINTER(RtConfig), I, C.POINTER(RtLayerWeights), P, P, I, P, I, I, P, P,
                                      C.POINTER(P), C.POINTER(P), I, P, Z, P]
@@ -146,9 +146,10 @@ def rt_decode_step(cfg, n_layers, layers, emb, g_final, vocab, ids, B, pos, logi
                                v_caches, N_max, workspace, workspace_bytes, stream)
 
 
-def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1, workspace, stream) -> int:
+def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1, alibi_slopes,
+                   workspace, stream) -> int:
     return _lib.rt_update_tile(C.byref(cfg), q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1,
-                               workspace, stream)
+                               alibi_slopes, workspace, stream)
 
 
 def rt_selftest_wait_expiry(workspace, stream) -> int:
@@ -225,6 +226,10 @@ def _pack_weights(wd: dict, dtype: str, device):
             t = _to_dev(wd[n], dtype, device)
             keep.append(t)
             setattr(st, n, t.data_ptr())
+    if wd.get("alibi_slopes") is not None:           # [n_heads], always fp32
+        t = _to_dev(np.asarray(wd["alibi_slopes"], dtype=np.float64), "f32", device)
+        keep.append(t)
+        st.alibi_slopes = t.data_ptr()
     return st, keep
 
 

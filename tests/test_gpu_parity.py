@@ -219,7 +219,7 @@ def test_update_tile_matches_algorithm_2(dtype, nq, nk):
     ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
     cfg = rt.make_config(d, H, 4 * d, dtype=dtype, softmax_scale=scale)
     st = rt.rt_update_tile(cfg, qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), od.data_ptr(), md.data_ptr(), ld.data_ptr(),
-                           B, rows_q, rows_kv, q0, q1, k0, k1, ws.data_ptr(), torch.cuda.current_stream().cuda_stream)
+                           B, rows_q, rows_kv, q0, q1, k0, k1, None, ws.data_ptr(), torch.cuda.current_stream().cuda_stream)
     assert st == rt.RT_OK
     torch.cuda.synchronize()
     assert rt.rt_get_status(ws.data_ptr()) == rt.RT_OK

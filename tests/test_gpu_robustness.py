@@ -194,3 +194,95 @@ def test_random_shapes_match_oracle(dtype, d, H, dff, B, N, leaf, flags, gains, 
     for name, g_, r_ in zip(("z", "k", "v"), got, ref):
         assert np.isfinite(g_).all(), name
         assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
+
+
+# ---------------------------------------------------------------- ALiBi distances (optional slopes per head)
+
+def _slopes(H, max_bias=8.0):
+    return np.array([2.0 ** (-max_bias * (h + 1) / H) for h in range(H)])
+
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N,leaf,sched", [
+    ("f32", 128, 2, 512, 2, 150, 16, "tiled"), ("f32", 128, 2, 512, 3, 70, 0, "naive"),
+    ("bf16", 256, 4, 1024, 5, 300, 32, "tiled"), ("bf16", 768, 12, 3072, 4, 520, 0, "tiled"),
+    ("bf16", 512, 8, 2048, 16, 200, 0, "tiled"), ("bf16", 256, 4, 512, 3, 260, 64, "naive")])
+def test_alibi_prefill_matches_oracle(dtype, d, H, dff, B, N, leaf, sched):
+    from oracle import RTConfig, RTWeights, layer_seq
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("alibi", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=8100 + N)
+    lw = data["layers"][0]
+    ref = layer_seq(RTConfig(d, H, 64, dff, alibi_slopes=_slopes(H)), RTWeights(**lw), data["x"])
+    base = layer_seq(RTConfig(d, H, 64, dff), RTWeights(**lw), data["x"])
+    assert rel_err(base[0], ref[0]) > 10 * TOL[dtype]          # the distances do change the result
+    lw = dict(lw, alibi_slopes=_slopes(H))
+    layer = _layer(d, H, dff, dtype, lw, leaf=leaf, sched=sched)
+    got = layer.prefill(data["x"])
+    for name, g_, r_ in zip(("z", "k", "v"), got, ref):
+        assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_alibi_prefill_then_decode_matches_oracle(dtype):
+    from oracle import RTConfig, RTWeights, layer_seq
+    from paper_2604_21215_b200 import inputs
+    d, H, dff, B, N = 128, 2, 256, 3, 45
+    wl = inputs.Workload("alibi_dec", 1, B, N + 2, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=8200)
+    lw = data["layers"][0]
+    ref = layer_seq(RTConfig(d, H, 64, dff, alibi_slopes=_slopes(H)), RTWeights(**lw), data["x"])
+    layer = _layer(d, H, dff, dtype, dict(lw, alibi_slopes=_slopes(H)), leaf=16)
+    got = layer.prefill(data["x"][:, :N], N_max=N + 2)
+    assert rel_err(got[0], ref[0][:, :N]) <= TOL[dtype]
+    for step in range(2):
+        zn = layer.decode(data["x"][:, N + step], N + step)
+        assert rel_err(zn, ref[0][:, N + step]) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,nq,nk", [("bf16", 200, 128), ("bf16", 130, 320), ("f32", 40, 50)])
+def test_alibi_update_tile_matches_algorithm_2(dtype, nq, nk):
+    # Algorithm 2 alone with distances: tensor-core kernel (bf16, key counts that are multiples of 64) and SIMT kernel
+    import torch
+    from oracle import update_tile
+    from paper_2604_21215_b200 import inputs, rt
+    B, H, d = 2, 3, 192
+    rng = np.random.default_rng(8300 + nq)
+    rows = 16 + nk + nq
+    k0, k1, q0, q1 = 16, 16 + nk, 16 + nk, 16 + nk + nq
+    q = inputs.round_to(rng.standard_normal((rows, B, d)), dtype)
+    k = inputs.round_to(rng.standard_normal((rows, B, d)), dtype)
+    v = inputs.round_to(rng.standard_normal((rows, B, d)), dtype)
+    scale = 0.125
+    slopes = _slopes(H)
+    m0 = rng.standard_normal((rows, B, H)); l0 = 1.0 + rng.random((rows, B, H)); o0 = rng.standard_normal((rows, B, d))
+    m_ref, l_ref, o_ref = m0.copy(), l0.copy(), o0.copy()
+    dist = np.arange(q0, q1)[:, None] - np.arange(k0, k1)[None, :]
+    for b in range(B):
+        for h in range(H):
+            sl = slice(64 * h, 64 * h + 64)
+            m2, l2, o2 = update_tile(q[q0:q1, b, sl], k[k0:k1, b, sl], v[k0:k1, b, sl], m0[q0:q1, b, h], l0[q0:q1, b, h],
+                                     o0[q0:q1, b, sl], scale, -slopes[h] * dist)
+            m_ref[q0:q1, b, h], l_ref[q0:q1, b, h], o_ref[q0:q1, b, sl] = m2, l2, o2
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = lambda a, t=tdt: torch.from_numpy(np.ascontiguousarray(a)).to(t).cuda()
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    LOG2E = 1.4426950408889634
+    od, md, ld = dev(o0, torch.float32), dev(m0 * LOG2E, torch.float32), dev(l0, torch.float32)
+    sd = dev(slopes, torch.float32)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    cfg = rt.make_config(d, H, 4 * d, dtype=dtype, softmax_scale=scale)
+    st = rt.rt_update_tile(cfg, qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), od.data_ptr(), md.data_ptr(), ld.data_ptr(),
+                           B, rows, rows, q0, q1, k0, k1, sd.data_ptr(), ws.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert st == rt.RT_OK and rt.rt_get_status(ws.data_ptr()) == rt.RT_OK
+    # compare what is unique: the normalised output o/l and the log-sum m + log2(l)
+    og, mg, lg = (t.to(torch.float64).cpu().numpy() for t in (od, md, ld))
+    tol = TOL[dtype]
+    for h in range(H):
+        sl = slice(64 * h, 64 * h + 64)
+        a_g = og[..., sl] / lg[..., h:h + 1]
+        a_r = o_ref[..., sl] / l_ref[..., h:h + 1]
+        assert np.abs(a_g - a_r).max() / np.abs(a_r).max() <= tol
+    lse_g = mg / LOG2E + np.log(lg)
+    lse_r = m_ref + np.log(l_ref)
+    assert np.abs(lse_g - lse_r).max() <= tol * max(1.0, np.abs(lse_r).max())
