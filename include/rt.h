@@ -181,6 +181,21 @@ rt_status rt_update_tile(const rt_config *cfg, const void *q, const void *k_cach
                          int32_t q0, int32_t q1, int32_t k0, int32_t k1,
                          const float *alibi_slopes, void *workspace, void *cuda_stream);
 
+/* One parallel sweep over all positions (Sec. 6, "activation checkpointing": with the layer outputs known, the
+ * persistent pairs of all positions can be rebuilt at once and every position recomputed independently).
+ * Given the layer input x [B,N,d] and claimed outputs z_claim [B,N,d]:
+ *   k_j = qkRMS[W_k RMS(z_claim_j)], v_j = W_v RMS(z_claim_j)            -> k_cache, v_cache rows [0,N)  (Eqs. 1-2)
+ *   a_i = attention of q_i over the pairs j < i and its temporary pair;  z'_i = x_i + alpha (a_i + MLP[RMS(x_i + alpha a_i)])
+ *                                                                         -> z_out [B,N,d]
+ * Because z_i depends only on z_j, j < i, the true outputs are the unique fixed point: z_out equals z_claim (up to
+ * rounding) exactly when z_claim is what rt_layer_prefill returns.  All products run over the B*N rows at once
+ * (tensor cores for bf16 storage), the attention as one causal pass inside 64-blocks plus one launch per level of
+ * Algorithm 1.  x, z_claim, z_out are distinct buffers; the workspace needs rt_recompute_workspace_bytes. */
+size_t    rt_recompute_workspace_bytes(const rt_config *cfg, int32_t B, int32_t N);
+rt_status rt_layer_recompute(const rt_config *cfg, const rt_layer_weights *w, const void *x, const void *z_claim,
+                             int32_t B, int32_t N, void *z_out, void *k_cache, void *v_cache, int32_t N_max,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues a two-CTA kernel
  * whose grid barrier expects an arrival that never comes.  The wait gives up after its limit (2 s),
  * the kernel returns normally, and rt_get_status(workspace) then reports RT_ERR_TIMEOUT; the CUDA

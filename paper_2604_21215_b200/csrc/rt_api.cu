@@ -244,6 +244,102 @@ rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, cons
   return run_layer(cfg, w, x, (long long)N * d, d, z, (long long)N * d, d, B, N, 0, k_cache, v_cache, N_max, ws, L, ctx);
 }
 
+size_t rt_recompute_workspace_bytes(const rt_config* cfg, int32_t B, int32_t N) {
+  if (!config_ok(cfg) || B <= 0 || N <= 0) return 0;
+  return ws_layout(cfg, B, N).total + align_up((size_t)B * N * cfg->d_ff * esize_of(cfg->dtype), 256);
+}
+
+rt_status rt_layer_recompute(const rt_config* cfg, const rt_layer_weights* w, const void* x, const void* z_claim,
+                             int32_t B, int32_t N, void* z_out, void* k_cache, void* v_cache, int32_t N_max,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!config_ok(cfg) || B <= 0 || N <= 0 || !workspace || !aligned16(workspace)) return RT_ERR_INVALID_ARG;
+  rt_status st = config_supported(cfg, 1);
+  if (st != RT_OK) return st;
+  if (workspace_bytes < rt_recompute_workspace_bytes(cfg, B, N)) return RT_ERR_WORKSPACE;
+  if (!weights_ok(w) || !x || !z_claim || !z_out || !k_cache || !v_cache || z_out == x || z_out == z_claim || N_max < N)
+    return RT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(z_claim) || !aligned16(z_out) || !aligned16(k_cache) || !aligned16(v_cache))
+    return RT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)workspace;
+  const WsLayout L = ws_layout(cfg, B, N);
+  if (cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;
+  const long long d = cfg->d_model, f = cfg->d_ff;
+  const long long tok = (long long)B * N;
+  const float scale_log2 = cfg->softmax_scale * kLog2e;
+  SyncArea* sync = (SyncArea*)(ws + L.sync);
+  const bool pre = (cfg->norm_flags & RT_NORM_PRE) != 0;
+
+  // 1. every persistent pair from the claimed outputs (Eqs. 1-2): k = qkRMS[W_k RMS(z)], v = W_v RMS(z)
+  PrepassParams pz;
+  memset(&pz, 0, sizeof(pz));
+  pz.B = B; pz.N = N; pz.d = cfg->d_model; pz.H = cfg->n_heads;
+  pz.norm_flags = (cfg->norm_flags & RT_NORM_SKIP_Z) ? (cfg->norm_flags & ~RT_NORM_PRE) : cfg->norm_flags;
+  pz.eps = cfg->rms_eps; pz.scale_log2 = scale_log2;
+  pz.x = z_claim; pz.x_bs = (long long)N * d; pz.x_ts = d;
+  pz.w_q = w->w_q; pz.w_k = w->w_k; pz.w_v = w->w_v;
+  pz.g_attn = w->g_kv ? w->g_kv : w->g_attn; pz.g_q = w->g_q; pz.g_k = w->g_k;
+  pz.n = ws + L.n; pz.q = ws + L.q; pz.kt = k_cache; pz.vt = v_cache;
+  pz.st_o = (float*)(ws + L.st_o); pz.st_m = (float*)(ws + L.st_m); pz.st_l = (float*)(ws + L.st_l);
+  pz.mats = 6; pz.no_seed = 1; pz.sync = sync;
+  {
+    ProfScope ps(s, kProfPrepass);
+    if (prepass_launch(cfg->dtype, pz, s) != cudaSuccess) return RT_ERR_CUDA;
+  }
+  // 2. queries, temporary pairs and the seeded running stats from the layer input, as in the prefill
+  PrepassParams px = pz;
+  px.norm_flags = cfg->norm_flags;
+  px.x = x; px.g_attn = w->g_attn;
+  px.kt = ws + L.kt; px.vt = ws + L.vt;
+  px.mats = 0; px.no_seed = 0;
+  {
+    ProfScope ps(s, kProfPrepass);
+    if (prepass_launch(cfg->dtype, px, s) != cudaSuccess) return RT_ERR_CUDA;
+  }
+  // 3. attention of every query over all earlier persistent pairs: the pairs inside a 64-block under a causal
+  //    mask, then Algorithm 1's cross tiles, one launch per level (all pairs are known, so the tiles of a level are
+  //    independent; each query row meets exactly one tile per level)
+  TileParams tp;
+  memset(&tp, 0, sizeof(tp));
+  tp.B = B; tp.d = cfg->d_model; tp.H = cfg->n_heads; tp.scale_log2 = scale_log2; tp.alibi = w->alibi_slopes;
+  tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
+  tp.st_o = px.st_o; tp.st_m = px.st_m; tp.st_l = px.st_l;
+  tp.rows_q = N; tp.rows_kv = N_max; tp.sync = sync; tp.q_limit = N;
+  {
+    ProfScope ps(s, kProfTile);
+    tp.q0 = 0; tp.q1 = kAutoLeaf; tp.k0 = 0; tp.k1 = kAutoLeaf;
+    tp.batch = (N + kAutoLeaf - 1) / kAutoLeaf; tp.batch_stride = kAutoLeaf; tp.causal = 1;
+    if (tile_simt_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    tp.causal = 0;
+    for (long long P = kAutoLeaf; P < N; P *= 2) {
+      tp.q0 = (int)P; tp.q1 = (int)(2 * P); tp.k0 = 0; tp.k1 = (int)P;
+      tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
+      if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    }
+  }
+  // 4. position-wise chain over all rows at once
+  ProfScope ps(s, kProfOther);
+  void* cbuf = ws + L.kt;                                       // the temporary pairs are folded into the stats by now
+  void* ubuf = ws + L.vt;
+  float* hbuf = (float*)(ws + L.st_o);                          // free once c = o / l is taken
+  void* gbuf = ws + L.total;
+  if (attn_value_launch(cfg->dtype, px.st_o, px.st_l, cbuf, tok, (int)d, cfg->n_heads, s) != cudaSuccess) return RT_ERR_CUDA;
+  DenseParams dp;
+  memset(&dp, 0, sizeof(dp));
+  dp.M = (int)tok; dp.B = B; dp.alpha = cfg->residual_scale; dp.h = hbuf;
+  dp.N = (int)d; dp.K = (int)d; dp.A = cbuf; dp.W = w->w_o; dp.epi = DENSE_RES_X;
+  dp.x = x; dp.x_bs = (long long)N * d; dp.x_ts = d;
+  if (dense_launch(cfg->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+  if (rms_rows_f32_launch(cfg->dtype, hbuf, w->g_mlp, ubuf, (int)tok, (int)d, cfg->rms_eps, pre ? 1 : 0, s) != cudaSuccess)
+    return RT_ERR_CUDA;
+  dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;
+  if (dense_launch(cfg->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+  dp.N = (int)d; dp.K = (int)f; dp.A = gbuf; dp.W = w->w_down; dp.epi = DENSE_RES_H;
+  dp.out = z_out; dp.o_bs = (long long)N * d; dp.o_ts = d;
+  if (dense_launch(cfg->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+  return RT_OK;
+}
+
 rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t pos,
                                void* z, void* k_cache, void* v_cache, int32_t N_max, void* workspace,
                                size_t workspace_bytes, void* cuda_stream) {

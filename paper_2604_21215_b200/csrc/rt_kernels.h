@@ -62,6 +62,8 @@ struct PrepassParams {
   void* n;                                       // [N*B, d] normalised input (scratch)
   void *q, *kt, *vt;                             // [N, B, d]
   float *st_o, *st_m, *st_l;
+  int mats;                                      // which projections to compute: bit 0 q, bit 1 k, bit 2 v (0 = all three)
+  int no_seed;                                   // 1: leave the running stats alone (projection only)
   SyncArea* sync;
 };
 cudaError_t prepass_launch(int dtype, const PrepassParams& p, cudaStream_t s);
@@ -78,17 +80,37 @@ struct TileParams {
   const void *k_cache, *v_cache;                 // [N_max, B, d]
   float *st_o, *st_m, *st_l;
   int q0, q1, k0, k1;
+  int batch, batch_stride, q_limit;              // batch > 1: blockIdx.z-th copy of the tile, shifted by z * batch_stride rows
+                                                 // (one level of Algorithm 1 in one launch); q_limit > 0 clips the queries
+  int causal;                                    // 1: only pairs with key position < query position (SIMT kernel only)
   int rows_q, rows_kv;                           // rows held by the query buffer / the caches (tensor-map bounds)
   SyncArea* sync;
 };
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s);
 // tensor-core version (bf16, key count a multiple of 64)
 cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s);
+cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s);
 
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,
                          void* x, cudaStream_t s);
 cudaError_t head_launch(int dtype, const void* emb, const void* g_final, const void* hidden, long long h_bs,
                         int B, int d, int vocab, int norm_flags, float eps, float* logits, cudaStream_t s);
+
+// Position-wise part of the parallel sweep (Sec. 6, activation checkpointing): dense products over all rows.
+enum { DENSE_RES_X = 0, DENSE_GELU = 1, DENSE_RES_H = 2 };
+struct DenseParams {
+  int M, N, K, B;                                // C[M,N] = A[M,K] W[N,K]^T; rows m = position * B + sequence
+  const void *A, *W;                             // storage type, K contiguous
+  int epi;                                       // DENSE_RES_X: h = x + alpha C (fp32);  DENSE_GELU: out = GELU(C);
+                                                 // DENSE_RES_H: out = h + alpha C (storage type, caller's strides)
+  float alpha;
+  const void* x; long long x_bs, x_ts;           // x[b, r, :] (DENSE_RES_X)
+  float* h;                                      // [M, N] fp32 (written by DENSE_RES_X, read by DENSE_RES_H)
+  void* out; long long o_bs, o_ts;               // DENSE_GELU: [M, N];  DENSE_RES_H: out[b, r, :]
+};
+cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s);
+cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s);
+cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s);
 
 }  // namespace rt

@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(256) qkv_gemm_simt_kernel(const PrepassParams 
   const int M = p.N * p.B, d = p.d;
   const int heads = d / kHeadDim;
   const int which = blockIdx.y / heads;        // 0: q, 1: k~, 2: v~
+  if (p.mats && !((p.mats >> which) & 1)) return;
   const int head = blockIdx.y % heads;
   const int m0 = blockIdx.x * kGM;
   const T* W = reinterpret_cast<const T*>(which == 0 ? p.w_q : (which == 1 ? p.w_k : p.w_v)) + (size_t)head * kHeadDim * d;
@@ -143,8 +144,10 @@ static cudaError_t prepass_typed(const PrepassParams& p, cudaStream_t s) {
     dim3 grid(ceil_div(M, kGM), 3 * (p.d / kHeadDim));
     qkv_gemm_simt_kernel<T><<<grid, 256, 0, s>>>(p);
   }
-  const long long units = (long long)M * p.H;
-  state_init_kernel<T><<<(unsigned)((units + 7) / 8), 256, 0, s>>>(p);
+  if (!p.no_seed) {
+    const long long units = (long long)M * p.H;
+    state_init_kernel<T><<<(unsigned)((units + 7) / 8), 256, 0, s>>>(p);
+  }
   return cudaGetLastError();
 }
 

@@ -44,6 +44,7 @@ qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_const
   const int col0 = (blockIdx.y % tiles_per_mat) * kGemmBN;  // first output column within the matrix
   const int m0 = blockIdx.x * kBM;
   const int n_kb = d / kGemmBK;
+  if (p.mats && !((p.mats >> which) & 1)) return;          // projection not asked for (uniform per CTA)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + GemmSmem::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + GemmSmem::tmem_ptr);
   auto full = [&](int s) { return sbase + GemmSmem::bars + 8u * (uint32_t)s; };

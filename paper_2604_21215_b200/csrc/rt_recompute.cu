@@ -1,0 +1,317 @@
+// Parallel sweep over all positions at once (Sec. 6, activation checkpointing): with the layer
+// outputs z known, every persistent pair can be rebuilt at once (Eqs. 1-2) and every a_i, z_i
+// recomputed independently of the others.  The position-wise part of that sweep is a chain of dense
+// products over all B*N rows, which is what this file holds:
+//   c   = o / l                                 (attention value per head from the running stats)
+//   h   = x + alpha W_o c                       (first display of Sec. 2.2)
+//   u   = RMS_{g_mlp}(h)
+//   g   = GELU(W_up u)
+//   z'  = h + alpha W_down g
+// Rows are position-major (m = position * B + sequence) as everywhere in the workspace.
+// bf16 storage with column counts that are multiples of 128 takes the tcgen05 kernel (same main loop
+// as the pre-pass projection: TMA ring of 64-wide K blocks, 128 x 128 accumulator in TMEM, one output
+// row per epilogue thread); everything else takes a plain SIMT product.
+#include "rt_kernels.h"
+#include "rt_tc.cuh"
+
+namespace rt {
+
+__device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+
+// ---- c = o / l ------------------------------------------------------------------------------
+template <typename T>
+__global__ void attn_value_kernel(const float* st_o, const float* st_l, T* c, long long rows, int d, int H) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;       // one thread = 4 columns
+  const long long total = rows * (d / 4);
+  if (i >= total) return;
+  const long long m = i / (d / 4);
+  const int col = (int)(i % (d / 4)) * 4;
+  const float il = 1.0f / st_l[m * H + col / kHeadDim];
+  const float4 o = *reinterpret_cast<const float4*>(st_o + m * d + col);
+  T* dst = c + m * d + col;
+  dst[0] = from_f<T>(o.x * il); dst[1] = from_f<T>(o.y * il); dst[2] = from_f<T>(o.z * il); dst[3] = from_f<T>(o.w * il);
+}
+
+// ---- u = RMS_g(h) for fp32 rows -------------------------------------------------------------------
+template <typename T>
+__global__ void rms_rows_f32_kernel(const float* h, const T* g, T* u, int rows, int d, float eps, int pre) {
+  const int lane = threadIdx.x & 31;
+  const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (m >= rows) return;
+  const float* hr = h + (size_t)m * d;
+  float ss = 0.f;
+  for (int k = lane; k < d; k += 32) ss += hr[k] * hr[k];
+  ss = warp_sum(ss);
+  const float rs = pre ? rsqrtf(ss / (float)d + eps) : 1.0f;
+  for (int k = lane; k < d; k += 32) u[(size_t)m * d + k] = from_f<T>(hr[k] * rs * (pre ? gain_at(g, k) : 1.0f));
+}
+
+// ---- epilogues of the dense products ------------------------------------------------------------
+// value(m, n, acc) -> stored where the epilogue says; m = r * B + b
+template <typename T>
+__device__ __forceinline__ void epi_store(const DenseParams& p, int m, int n, float acc) {
+  if (p.epi == DENSE_RES_X) {                                  // h = x + alpha acc  (fp32, position-major)
+    const int b = m % p.B, r = m / p.B;
+    const float xv = to_f(reinterpret_cast<const T*>(p.x)[(size_t)b * p.x_bs + (size_t)r * p.x_ts + n]);
+    p.h[(size_t)m * p.N + n] = xv + p.alpha * acc;
+  } else if (p.epi == DENSE_GELU) {                            // g = GELU(acc)  (storage type)
+    reinterpret_cast<T*>(p.out)[(size_t)m * p.N + n] = from_f<T>(gelu_exact(acc));
+  } else {                                                     // z' = h + alpha acc  (storage type, caller's strides)
+    const int b = m % p.B, r = m / p.B;
+    reinterpret_cast<T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n] = from_f<T>(p.h[(size_t)m * p.N + n] + p.alpha * acc);
+  }
+}
+
+// ---- SIMT product: C[m, n] = sum_k A[m,k] W[n,k] ----------------------------------------------------
+constexpr int kDM = 64, kDN = 64, kDK = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(256) dense_simt_kernel(const DenseParams p) {
+  __shared__ float As[kDK][kDM + 4];
+  __shared__ float Bs[kDK][kDN + 4];
+  const T* A = reinterpret_cast<const T*>(p.A);
+  const T* W = reinterpret_cast<const T*>(p.W);
+  const int m0 = blockIdx.x * kDM, n0 = blockIdx.y * kDN;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  const int lr = tid >> 2, lk = (tid & 3) * 4;
+  for (int k0 = 0; k0 < p.K; k0 += kDK) {
+    float f[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f};
+    if (m0 + lr < p.M) reinterpret_cast<const Vec4<T>*>(A + (size_t)(m0 + lr) * p.K + k0 + lk)->to_float(f);
+    if (n0 + lr < p.N) reinterpret_cast<const Vec4<T>*>(W + (size_t)(n0 + lr) * p.K + k0 + lk)->to_float(g);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { As[lk + i][lr] = f[i]; Bs[lk + i][lr] = g[i]; }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kDK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += a[i] * b[j];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= p.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n < p.N) epi_store<T>(p, m, n, acc[i][j]);
+    }
+  }
+}
+
+// ---- tcgen05 product (bf16; N a multiple of 128, K a multiple of 64) ------------------------------------
+constexpr int kTBN = 128, kTBK = 64, kTStages = 3, kTThreads = 192;
+constexpr uint32_t kTABytes = kBM * kTBK * 2, kTBBytes = kTBN * kTBK * 2;
+
+struct DenseSmem {
+  static constexpr uint32_t a = 0;
+  static constexpr uint32_t b = a + kTStages * kTABytes;
+  static constexpr uint32_t bars = b + kTStages * kTBBytes;      // full[3], empty[3], acc_ready
+  static constexpr uint32_t tmem_ptr = bars + 64;
+  static constexpr uint32_t abort_flag = tmem_ptr + 8;
+  static constexpr uint32_t total = abort_flag + 8;
+};
+
+__global__ void __launch_bounds__(kTThreads, 2)
+dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
+                SyncArea* sync) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kTBN;
+  const int n_kb = p.K / kTBK;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + DenseSmem::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + DenseSmem::tmem_ptr);
+  auto full = [&](int s) { return sbase + DenseSmem::bars + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return sbase + DenseSmem::bars + 8u * (uint32_t)(kTStages + s); };
+  const uint32_t acc_ready = sbase + DenseSmem::bars + 8u * (2 * kTStages);
+
+  if (tid == 0) {
+    *s_abort = 0;
+    for (int s = 0; s < kTStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    mbar_init(acc_ready, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + DenseSmem::tmem_ptr), "n"(kTBN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kTStages;
+        if (kb >= kTStages) ok = mbar_wait(empty(s), ((kb / kTStages) - 1) & 1, s_abort, sync);
+        if (!ok) break;
+        mbar_expect_tx(full(s), kTABytes + kTBBytes);
+        tma_load_2d(sbase + DenseSmem::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
+        tma_load_2d(sbase + DenseSmem::b + s * kTBBytes, &map_w, full(s), kb * kTBK, n0);
+        ++issued;
+      }
+      if (!ok) {
+        // gave up: let the copies already started land before the shared memory goes away (bounded)
+        for (int i = issued > kTStages ? issued - kTStages : 0; i < issued; ++i) {
+          unsigned spins = 0;
+          while (!mbar_try_wait(full(i % kTStages), (i / kTStages) & 1) && ++spins < (1u << 20)) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kTBN, false);
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kTStages;
+        ok = mbar_wait(full(s), (kb / kTStages) & 1, s_abort, sync);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t a0 = make_desc(sbase + DenseSmem::a + s * kTABytes, 16, 1024);
+        const uint64_t b0 = make_desc(sbase + DenseSmem::b + s * kTBBytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < kTBK / 16; ++ks)
+          tc_mma(tmem, a0 + 2u * ks, b0 + 2u * ks, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(empty(s));
+      }
+      if (ok) tc_commit(acc_ready);
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue: one output row per thread, 32 columns at a time ----------------
+    const int m = m0 + warp * 32 + lane;
+    if (mbar_wait(acc_ready, 0, s_abort, sync)) {
+      tc_fence_after();
+      const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+      const int b = m % p.B, r = m / p.B;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kTBN; c0 += 32) {
+        uint32_t v[32];
+        tc_ld32(t_row + (uint32_t)c0, v);
+        tc_wait_ld();
+        if (m >= p.M) continue;
+        const int n = n0 + c0;
+        if (p.epi == DENSE_RES_X) {
+          const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n);
+          float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {                           // 8 columns per 16-byte load of x
+            const uint4 xw = xs[q];
+            const unsigned w4[4] = {xw.x, xw.y, xw.z, xw.w};
+            float o[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              o[2 * j] = __uint_as_float(w4[j] << 16) + p.alpha * __uint_as_float(v[8 * q + 2 * j]);
+              o[2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u) + p.alpha * __uint_as_float(v[8 * q + 2 * j + 1]);
+            }
+            dst[2 * q] = make_float4(o[0], o[1], o[2], o[3]);
+            dst[2 * q + 1] = make_float4(o[4], o[5], o[6], o[7]);
+          }
+        } else {
+          float o[32];
+          if (p.epi == DENSE_GELU) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = gelu_exact(__uint_as_float(v[j]));
+          } else {
+            const float4* hs = reinterpret_cast<const float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 hv = hs[q];
+              o[4 * q] = hv.x + p.alpha * __uint_as_float(v[4 * q]);
+              o[4 * q + 1] = hv.y + p.alpha * __uint_as_float(v[4 * q + 1]);
+              o[4 * q + 2] = hv.z + p.alpha * __uint_as_float(v[4 * q + 2]);
+              o[4 * q + 3] = hv.w + p.alpha * __uint_as_float(v[4 * q + 3]);
+            }
+          }
+          __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                              (p.epi == DENSE_GELU ? (size_t)m * p.N + n : (size_t)b * p.o_bs + (size_t)r * p.o_ts + n);
+          uint4* dst = reinterpret_cast<uint4*>(ob);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const __nv_bfloat162 pk = __floats2bfloat162_rn(o[8 * q + 2 * j], o[8 * q + 2 * j + 1]);
+              w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+            }
+            dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTBN) : "memory");
+  }
+}
+
+// row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
+static bool make_map_rows(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kTBK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s) {
+  if (p.M <= 0) return cudaSuccess;
+  const bool strides_ok = p.epi == DENSE_GELU || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
+                                                  ((p.epi == DENSE_RES_X ? p.x_ts : p.o_ts) % 8 == 0));
+  if (dtype == RT_BF16 && p.N % kTBN == 0 && p.K % kTBK == 0 && strides_ok) {
+    CUtensorMap ma, mw;
+    if (!make_map_rows(&ma, p.A, p.M, p.K, kBM) || !make_map_rows(&mw, p.W, p.N, p.K, kTBN)) return cudaErrorInvalidValue;
+    const size_t smem = DenseSmem::total + 1024;
+    cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(ceil_div(p.M, kBM), p.N / kTBN);
+    dense_tc_kernel<<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+    return cudaGetLastError();
+  }
+  dim3 grid(ceil_div(p.M, kDM), ceil_div(p.N, kDN));
+  if (dtype == RT_BF16) dense_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(p);
+  else dense_simt_kernel<float><<<grid, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s) {
+  const long long total = rows * (d / 4);
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (dtype == RT_BF16) attn_value_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(st_o, st_l, (__nv_bfloat16*)c, rows, d, H);
+  else attn_value_kernel<float><<<blocks, 256, 0, s>>>(st_o, st_l, (float*)c, rows, d, H);
+  return cudaGetLastError();
+}
+
+cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s) {
+  if (dtype == RT_BF16) rms_rows_f32_kernel<__nv_bfloat16><<<ceil_div(rows, 8), 256, 0, s>>>(h, (const __nv_bfloat16*)g, (__nv_bfloat16*)u, rows, d, eps, pre);
+  else rms_rows_f32_kernel<float><<<ceil_div(rows, 8), 256, 0, s>>>(h, (const float*)g, (float*)u, rows, d, eps, pre);
+  return cudaGetLastError();
+}
+
+}  // namespace rt

@@ -17,7 +17,13 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
   __shared__ float Vs[kTK][kHeadDim];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
-  const int qb = p.q0 + blockIdx.x * kTQ;
+  const int shift = (int)blockIdx.z * p.batch_stride;                   // copy z of the tile (one level in one launch)
+  const int q0 = p.q0 + shift, k0 = p.k0 + shift;
+  int q1 = p.q1 + shift, k1 = p.k1 + shift;
+  if (p.q_limit > 0 && q1 > p.q_limit) q1 = p.q_limit;
+  if (p.q_limit > 0 && k1 > p.q_limit) k1 = p.q_limit;         // (a causal block's keys end where its queries do)
+  const int qb = q0 + blockIdx.x * kTQ;
+  if (qb >= q1) return;
   const T* Q = reinterpret_cast<const T*>(p.q);
   const T* Kc = reinterpret_cast<const T*>(p.k_cache);
   const T* Vc = reinterpret_cast<const T*>(p.v_cache);
@@ -27,14 +33,14 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
 
   for (int i = tid; i < kTQ * kHeadDim; i += 128) {
     const int r = i / kHeadDim, e = i % kHeadDim;
-    Qs[r][e] = (qb + r < p.q1) ? to_f(Q[(size_t)(qb + r) * rstride + col0 + e]) : 0.f;
+    Qs[r][e] = (qb + r < q1) ? to_f(Q[(size_t)(qb + r) * rstride + col0 + e]) : 0.f;
   }
   // each warp owns 4 query rows; lane holds dims lane and lane+32 of o
   float m[4], l[4], oa[4], ob[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int qi = qb + warp * 4 + i;
-    if (qi < p.q1) {
+    if (qi < q1) {
       const size_t sidx = (size_t)qi * p.B + b;
       m[i] = p.st_m[sidx * p.H + h];
       l[i] = p.st_l[sidx * p.H + h];
@@ -42,19 +48,21 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
       ob[i] = p.st_o[sidx * p.d + h * kHeadDim + lane + 32];
     } else { m[i] = 0.f; l[i] = 0.f; oa[i] = 0.f; ob[i] = 0.f; }
   }
-  for (int kb = p.k0; kb < p.k1; kb += kTK) {
+  for (int kb = k0; kb < k1; kb += kTK) {
     __syncthreads();
     for (int i = tid; i < kTK * kHeadDim; i += 128) {
       const int r = i / kHeadDim, e = i % kHeadDim;
-      const bool ok = kb + r < p.k1;
+      const bool ok = kb + r < k1;
       Ks[r][e] = ok ? to_f(Kc[(size_t)(kb + r) * rstride + col0 + e]) : 0.f;
       Vs[r][e] = ok ? to_f(Vc[(size_t)(kb + r) * rstride + col0 + e]) : 0.f;
     }
     __syncthreads();
-    const bool valid = kb + lane < p.k1;
+    const bool in_range = kb + lane < k1;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int qr = warp * 4 + i;
+      const bool valid = in_range && (!p.causal || kb + lane < qb + qr);   // causal: only earlier positions
+      if (p.causal && kb >= qb + qr) continue;                            // whole chunk masked for this row (warp-uniform)
       float s = 0.f;
 #pragma unroll 16
       for (int e = 0; e < kHeadDim; ++e) s += Qs[qr][e] * Ks[lane][e];
@@ -76,7 +84,7 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int qi = qb + warp * 4 + i;
-    if (qi < p.q1) {
+    if (qi < q1) {
       const size_t sidx = (size_t)qi * p.B + b;
       if (lane == 0) { p.st_m[sidx * p.H + h] = m[i]; p.st_l[sidx * p.H + h] = l[i]; }
       p.st_o[sidx * p.d + h * kHeadDim + lane] = oa[i];
@@ -88,7 +96,7 @@ __global__ void __launch_bounds__(128) tile_simt_kernel(const TileParams p) {
 cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
   const int nq = p.q1 - p.q0;
   if (nq <= 0 || p.k1 <= p.k0) return cudaSuccess;
-  dim3 grid(ceil_div(nq, kTQ), p.B * p.H);
+  dim3 grid(ceil_div(nq, kTQ), p.B * p.H, p.batch > 1 ? p.batch : 1);
   if (dtype == RT_BF16) tile_simt_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(p);
   else tile_simt_kernel<float><<<grid, 128, 0, s>>>(p);
   return cudaGetLastError();

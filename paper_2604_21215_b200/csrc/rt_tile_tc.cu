@@ -59,7 +59,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
-  const int qb = p.q0 + blockIdx.x * kBM;                 // first query row of this CTA
+  const int shift = (int)blockIdx.z * p.batch_stride;     // copy z of the tile (one level of Algorithm 1 in one launch)
+  const int k0 = p.k0 + shift;
+  int q1 = p.q1 + shift;
+  if (p.q_limit > 0 && q1 > p.q_limit) q1 = p.q_limit;
+  const int qb = p.q0 + shift + blockIdx.x * kBM;         // first query row of this CTA
+  if (qb >= q1) return;                                   // nothing left of this copy (uniform per CTA)
   const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + C::tmem_ptr);
@@ -94,8 +99,8 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (kb >= kStages) ok = mbar_wait(bar(BAR_KV_EMPTY + st), ((kb / kStages) - 1) & 1, s_abort, sync);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_KV_FULL + st), 2 * kKVBytes);
-        tma_load_4d(sbase + C::k + st * kKVBytes, &map_k, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
-        tma_load_4d(sbase + C::v + st * kKVBytes, &map_v, bar(BAR_KV_FULL + st), 0, h, b, p.k0 + kb * kBK);
+        tma_load_4d(sbase + C::k + st * kKVBytes, &map_k, bar(BAR_KV_FULL + st), 0, h, b, k0 + kb * kBK);
+        tma_load_4d(sbase + C::v + st * kKVBytes, &map_v, bar(BAR_KV_FULL + st), 0, h, b, k0 + kb * kBK);
         ++issued;
       }
       if (!ok) {
@@ -151,7 +156,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ------------------------------ softmax warps: one thread per query row ------------------------------
     const int row = warp * 32 + lane;
     const int qi = qb + row;
-    const bool row_ok = qi < p.q1;
+    const bool row_ok = qi < q1;
     const uint32_t t_s = tmem + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_o = t_s + 64u;
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
@@ -184,7 +189,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // ALiBi distances: the logit of this row's query (position qi) on key j gets -slope (qi - j)
       // = base + slope * column: the column part goes into the raw products (divided by the scale that is
       // applied below), the row constant into the maximum and the exponent offset
-      const float base_l2 = -slope_l2 * (float)(qi - (p.k0 + kb * kBK));
+      const float base_l2 = -slope_l2 * (float)(qi - (k0 + kb * kBK));
       if (slope_l2 != 0.f) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -298,7 +303,7 @@ cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncAre
   const size_t smem = TcCfg::total + 1024;
   cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(ceil_div(nq, kBM), p.B * p.H);
+  dim3 grid(ceil_div(nq, kBM), p.B * p.H, p.batch > 1 ? p.batch : 1);
   tile_tc_kernel<<<grid, TcCfg::threads, smem, s>>>(mq, mk, mv, p, sync);
   return cudaGetLastError();
 }

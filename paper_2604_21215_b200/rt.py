@@ -25,7 +25,8 @@ RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
-           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile", "rt_selftest_wait_expiry")
+           "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile", "rt_selftest_wait_expiry",
+           "rt_recompute_workspace_bytes", "rt_layer_recompute")
 RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -71,6 +72,10 @@ def _load():
     lib.rt_layer_decode_step_static.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P]
     lib.rt_selftest_wait_expiry.restype = C.c_int
     lib.rt_selftest_wait_expiry.argtypes = [P, P]
+    lib.rt_recompute_workspace_bytes.restype = Z
+    lib.rt_recompute_workspace_bytes.argtypes = [C.POINTER(RtConfig), I, I]
+    lib.rt_layer_recompute.restype = C.c_int
+    lib.rt_layer_recompute.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, P, I, I, P, P, P, I, P, Z, P]
     lib.rt_update_tile.restype = C.c_int
     lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P, P]
     lib.rt_stack_prefill.restype = C.c_int
@@ -150,6 +155,15 @@ def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_k
                    workspace, stream) -> int:
     return _lib.rt_update_tile(C.byref(cfg), q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_kv, q0, q1, k0, k1,
                                alibi_slopes, workspace, stream)
+
+
+def rt_recompute_workspace_bytes(cfg: RtConfig, B: int, N: int) -> int:
+    return int(_lib.rt_recompute_workspace_bytes(C.byref(cfg), B, N))
+
+
+def rt_layer_recompute(cfg, w, x, z_claim, B, N, z_out, k_cache, v_cache, N_max, workspace, workspace_bytes, stream) -> int:
+    return _lib.rt_layer_recompute(C.byref(cfg), C.byref(w), x, z_claim, B, N, z_out, k_cache, v_cache, N_max, workspace,
+                                   workspace_bytes, stream)
 
 
 def rt_selftest_wait_expiry(workspace, stream) -> int:
@@ -286,6 +300,25 @@ class Layer:
         _check(self.status(), "rt_layer_prefill (device)")
         to_np = lambda t: t.to(torch.float64).cpu().numpy()
         return (to_np(zd), to_np(self.k_cache[:N].permute(1, 0, 2)), to_np(self.v_cache[:N].permute(1, 0, 2)))
+
+    def recompute(self, x, z_claim):
+        """One parallel sweep: x, z_claim [B,N,d] -> z', k, v (fp64 numpy, each [B,N,d]); the caches are rebuilt from z_claim."""
+        torch = _torch()
+        xd = _to_dev(x, self.dtype, self.device)
+        zc = _to_dev(z_claim, self.dtype, self.device)
+        B, N, _ = xd.shape
+        self.reserve(B, N)
+        need = rt_recompute_workspace_bytes(self.cfg, B, N)
+        if self.ws.numel() < need:
+            self.ws = torch.zeros(need, dtype=torch.uint8, device=self.device)
+        zo = torch.empty_like(xd)
+        s = torch.cuda.current_stream(self.device).cuda_stream
+        _check(rt_layer_recompute(self.cfg, self.w, xd.data_ptr(), zc.data_ptr(), B, N, zo.data_ptr(), self.k_cache.data_ptr(),
+                                  self.v_cache.data_ptr(), self.N_max, self.ws.data_ptr(), self.ws.numel(), s), "rt_layer_recompute")
+        torch.cuda.synchronize(self.device)
+        _check(self.status(), "rt_layer_recompute (device)")
+        to_np = lambda t: t.to(torch.float64).cpu().numpy()
+        return (to_np(zo), to_np(self.k_cache[:N].permute(1, 0, 2)), to_np(self.v_cache[:N].permute(1, 0, 2)))
 
     def decode(self, x_new, pos: int):
         """x_new [B,d] at position pos (caches must hold pos rows) -> z_new [B,d] fp64 numpy."""
