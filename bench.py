@@ -451,6 +451,71 @@ def run_decode_bench(args):
     return 0
 
 
+def run_recompute_bench(args):
+    """Times rt_layer_recompute (the parallel sweep of Sec. 6: all positions at once, given the outputs) on the
+    workload's single-layer shape; prints one JSON object with the per-class kernel times and the tensor rate."""
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    wl = get_workload(args.workload, args.batch)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(
+        os.path.join(ROOT, "MEASURED_PEAKS.json")) else {"bf16_tflops": 1590.0}
+    import dataclasses
+    if wl.vocab:
+        wl = dataclasses.replace(wl, vocab=0, n_layers=1)
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    if args.alibi:
+        lw["alibi_slopes"] = alibi_slopes(wl.n_heads)
+    layer = rt.Layer(wl.d_model, wl.n_heads, wl.d_ff, dtype=wl.dtype, residual_scale=wl.residual_scale)
+    layer.set_weights(lw)
+    layer.reserve(wl.B, wl.N)
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    x = torch.from_numpy(data["x"]).to(tdt).to(dev)
+    g = torch.Generator(device=dev); g.manual_seed(BASE_TILE_SEED + 2)
+    zc = (x.float() + 0.5 * torch.randn(x.shape, generator=g, device=dev)).to(tdt)
+    zo = torch.empty_like(x)
+    need = rt.rt_recompute_workspace_bytes(layer.cfg, wl.B, wl.N)
+    ws = torch.zeros(need, dtype=torch.uint8, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def call():
+        rt._check(rt.rt_layer_recompute(layer.cfg, layer.w, x.data_ptr(), zc.data_ptr(), wl.B, wl.N, zo.data_ptr(),
+                                        layer.k_cache.data_ptr(), layer.v_cache.data_ptr(), layer.N_max, ws.data_ptr(),
+                                        ws.numel(), stream.cuda_stream), "rt_layer_recompute")
+    for _ in range(max(3, args.warmup)):
+        call()
+    torch.cuda.synchronize(dev)
+    rt.rt_profile_enable(True)
+    rt.rt_profile_read()
+    evs = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); call(); b.record(stream)
+        evs.append((a, b))
+    torch.cuda.synchronize(dev)
+    prof = rt.rt_profile_read()
+    rt.rt_profile_enable(False)
+    assert rt.rt_get_status(ws.data_ptr()) == rt.RT_OK
+    ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+    tok, d, f = wl.B * wl.N, wl.d_model, wl.d_ff
+    flops_proj = 10.0 * tok * d * d
+    flops_chain = 2.0 * tok * d * d + 4.0 * tok * d * f
+    flops_attn = 2.0 * wl.B * d * wl.N * (wl.N - 1)
+    tf = (flops_proj + flops_chain + flops_attn) / (ms * 1e-3) / 1e12
+    per = {k: v["ms"] / args.steps for k, v in prof.items()}
+    print(json.dumps({"recompute_bench": wl.name, "B": wl.B, "N": wl.N, "d_model": d, "d_ff": f, "dtype": wl.dtype,
+                      "alibi": bool(args.alibi), "ms_per_call": ms, "tokens_per_s": tok / (ms * 1e-3), "tflops": tf,
+                      "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "peak_tflops": peaks["bf16_tflops"],
+                      "gflop": {"projections": flops_proj / 1e9, "chain": flops_chain / 1e9, "attention": flops_attn / 1e9},
+                      "ms_by_class": {"projections": per.get("prepass"), "attention": per.get("tile"),
+                                      "chain": per.get("other")}}))
+    return 0
+
+
 BASE_TILE_SEED = 20260421
 
 
@@ -470,12 +535,16 @@ def main():
     ap.add_argument("--tile-bench-all", action="store_true", help="with --tile-bench: also sizes beyond N/2")
     ap.add_argument("--alibi", action="store_true",
                     help="add ALiBi distances (slopes 2^(-8 h / H), h = 1..H) to the attention logits")
+    ap.add_argument("--recompute-bench", action="store_true",
+                    help="time rt_layer_recompute (parallel sweep given the outputs) and exit")
     ap.add_argument("--decode-bench", action="store_true", help="time rt_decode_step at several cache lengths and exit")
     args = ap.parse_args()
     if args.tile_bench:
         return run_tile_bench(args)
     if args.decode_bench:
         return run_decode_bench(args)
+    if args.recompute_bench:
+        return run_recompute_bench(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_cuda(args)

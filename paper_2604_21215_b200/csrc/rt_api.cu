@@ -307,11 +307,21 @@ rt_status rt_layer_recompute(const rt_config* cfg, const rt_layer_weights* w, co
   tp.rows_q = N; tp.rows_kv = N_max; tp.sync = sync; tp.q_limit = N;
   {
     ProfScope ps(s, kProfTile);
-    tp.q0 = 0; tp.q1 = kAutoLeaf; tp.k0 = 0; tp.k1 = kAutoLeaf;
-    tp.batch = (N + kAutoLeaf - 1) / kAutoLeaf; tp.batch_stride = kAutoLeaf; tp.causal = 1;
-    if (tile_simt_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    // diagonal blocks under the causal mask: whole blocks in one batched launch (tensor cores for bf16), the
+    // ragged last block on its own; then the levels of Algorithm 1 from the block size upwards
+    const int Lb = cfg->dtype == RT_BF16 ? 2 * kAutoLeaf : kAutoLeaf;
+    const int full = N / Lb;
+    tp.causal = 1;
+    if (full > 0) {
+      tp.q0 = 0; tp.q1 = Lb; tp.k0 = 0; tp.k1 = Lb; tp.batch = full; tp.batch_stride = Lb;
+      if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    }
+    if (full * Lb < N) {
+      tp.q0 = full * Lb; tp.q1 = N; tp.k0 = full * Lb; tp.k1 = N; tp.batch = 1; tp.batch_stride = 0;
+      if (tile_simt_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+    }
     tp.causal = 0;
-    for (long long P = kAutoLeaf; P < N; P *= 2) {
+    for (long long P = Lb; P < N; P *= 2) {
       tp.q0 = (int)P; tp.q1 = (int)(2 * P); tp.k0 = 0; tp.k1 = (int)P;
       tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
       if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;

@@ -82,7 +82,7 @@ struct TileParams {
   int q0, q1, k0, k1;
   int batch, batch_stride, q_limit;              // batch > 1: blockIdx.z-th copy of the tile, shifted by z * batch_stride rows
                                                  // (one level of Algorithm 1 in one launch); q_limit > 0 clips the queries
-  int causal;                                    // 1: only pairs with key position < query position (SIMT kernel only)
+  int causal;                                    // 1: only pairs with key position < query position
   int rows_q, rows_kv;                           // rows held by the query buffer / the caches (tensor-map bounds)
   SyncArea* sync;
 };

@@ -197,6 +197,15 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           s1[i] = __float_as_uint(fmaf(step_raw, (float)(i + 32), __uint_as_float(s1[i])));
         }
       }
+      if (p.causal) {
+        // only pairs at earlier positions than this row's query: the rest of the block gets -inf (p = 0)
+        const int n_valid = qi - (k0 + kb * kBK);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i >= n_valid) s0[i] = 0xff800000u;
+          if (i + 32 >= n_valid) s1[i] = 0xff800000u;
+        }
+      }
       float mx4[4];                                            // four independent chains
 #pragma unroll
       for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
