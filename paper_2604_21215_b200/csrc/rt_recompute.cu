@@ -111,18 +111,24 @@ __global__ void __launch_bounds__(256) dense_simt_kernel(const DenseParams p) {
 }
 
 // ---- tcgen05 product (bf16; N a multiple of 128, K a multiple of 64) ------------------------------------
-constexpr int kTBN = 128, kTBK = 64, kTStages = 3, kTThreads = 192;
-constexpr uint32_t kTABytes = kBM * kTBK * 2, kTBBytes = kTBN * kTBK * 2;
+// Output tile 128 x BN.  BN = 256 halves the bytes fetched from L2 per product (the 128 x 128 tile is bound by the
+// L2 -> SM stream: 32 KB per 2 MFLOP); its two 48 KB stages still leave room for two CTAs per SM.
+constexpr int kTBK = 64, kTThreads = 192;
+constexpr uint32_t kTABytes = kBM * kTBK * 2;
 
+template <int BN>
 struct DenseSmem {
+  static constexpr int stages = BN == 256 ? 2 : 3;
+  static constexpr uint32_t b_bytes = BN * kTBK * 2;
   static constexpr uint32_t a = 0;
-  static constexpr uint32_t b = a + kTStages * kTABytes;
-  static constexpr uint32_t bars = b + kTStages * kTBBytes;      // full[3], empty[3], acc_ready
+  static constexpr uint32_t b = a + stages * kTABytes;
+  static constexpr uint32_t bars = b + stages * b_bytes;         // full[], empty[], acc_ready
   static constexpr uint32_t tmem_ptr = bars + 64;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
 
+template <int BN>
 __global__ void __launch_bounds__(kTThreads, 2)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
                 SyncArea* sync) {
@@ -130,13 +136,17 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  using DS = DenseSmem<BN>;
+  constexpr int kTStages = DS::stages;
+  constexpr int kTBN = BN;
+  constexpr uint32_t kTBBytes = DS::b_bytes;
   const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kTBN;
   const int n_kb = p.K / kTBK;
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + DenseSmem::abort_flag);
-  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + DenseSmem::tmem_ptr);
-  auto full = [&](int s) { return sbase + DenseSmem::bars + 8u * (uint32_t)s; };
-  auto empty = [&](int s) { return sbase + DenseSmem::bars + 8u * (uint32_t)(kTStages + s); };
-  const uint32_t acc_ready = sbase + DenseSmem::bars + 8u * (2 * kTStages);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + DS::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + DS::tmem_ptr);
+  auto full = [&](int s) { return sbase + DS::bars + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return sbase + DS::bars + 8u * (uint32_t)(kTStages + s); };
+  const uint32_t acc_ready = sbase + DS::bars + 8u * (2 * kTStages);
 
   if (tid == 0) {
     *s_abort = 0;
@@ -145,7 +155,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + DenseSmem::tmem_ptr), "n"(kTBN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + DS::tmem_ptr), "n"(kTBN) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -163,8 +173,8 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (kb >= kTStages) ok = mbar_wait(empty(s), ((kb / kTStages) - 1) & 1, s_abort, sync);
         if (!ok) break;
         mbar_expect_tx(full(s), kTABytes + kTBBytes);
-        tma_load_2d(sbase + DenseSmem::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
-        tma_load_2d(sbase + DenseSmem::b + s * kTBBytes, &map_w, full(s), kb * kTBK, n0);
+        tma_load_2d(sbase + DS::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
+        tma_load_2d(sbase + DS::b + s * kTBBytes, &map_w, full(s), kb * kTBK, n0);
         ++issued;
       }
       if (!ok) {
@@ -186,8 +196,8 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         ok = mbar_wait(full(s), (kb / kTStages) & 1, s_abort, sync);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t a0 = make_desc(sbase + DenseSmem::a + s * kTABytes, 16, 1024);
-        const uint64_t b0 = make_desc(sbase + DenseSmem::b + s * kTBBytes, 16, 1024);
+        const uint64_t a0 = make_desc(sbase + DS::a + s * kTABytes, 16, 1024);
+        const uint64_t b0 = make_desc(sbase + DS::b + s * kTBBytes, 16, 1024);
 #pragma unroll
         for (int ks = 0; ks < kTBK / 16; ++ks)
           tc_mma(tmem, a0 + 2u * ks, b0 + 2u * ks, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
@@ -284,14 +294,22 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
   if (p.M <= 0) return cudaSuccess;
   const bool strides_ok = p.epi == DENSE_GELU || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
                                                   ((p.epi == DENSE_RES_X ? p.x_ts : p.o_ts) % 8 == 0));
-  if (dtype == RT_BF16 && p.N % kTBN == 0 && p.K % kTBK == 0 && strides_ok) {
+  if (dtype == RT_BF16 && p.N % 128 == 0 && p.K % kTBK == 0 && strides_ok) {
+    const int bn = p.N % 256 == 0 ? 256 : 128;
     CUtensorMap ma, mw;
-    if (!make_map_rows(&ma, p.A, p.M, p.K, kBM) || !make_map_rows(&mw, p.W, p.N, p.K, kTBN)) return cudaErrorInvalidValue;
-    const size_t smem = DenseSmem::total + 1024;
-    cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    dim3 grid(ceil_div(p.M, kBM), p.N / kTBN);
-    dense_tc_kernel<<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+    if (!make_map_rows(&ma, p.A, p.M, p.K, kBM) || !make_map_rows(&mw, p.W, p.N, p.K, bn)) return cudaErrorInvalidValue;
+    dim3 grid(ceil_div(p.M, kBM), p.N / bn);
+    if (bn == 256) {
+      const size_t smem = DenseSmem<256>::total + 1024;
+      cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      dense_tc_kernel<256><<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+    } else {
+      const size_t smem = DenseSmem<128>::total + 1024;
+      cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      dense_tc_kernel<128><<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+    }
     return cudaGetLastError();
   }
   dim3 grid(ceil_div(p.M, kDM), ceil_div(p.N, kDN));
