@@ -61,8 +61,6 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_z = take((size_t)B * d * 4);
   L.ex_k = take((size_t)B * d * 4);
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
-  // flag-carrying exchange words of the bf16 leaf kernel: c, h, z [B,d/2], g [B,dff/2], raw k|v [B,2d]
-  // (c, h, z are laid out for 16 sequence slots whatever B is)
   // exchange buffers of the tensor-core leaf kernel: c, h, z as flag-carrying words (16 sequence slots each),
   // g as packed bf16 in fragment order (16 sequence slots), raw k|v as flag-carrying fp32 words
   L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)16 * (f / 4) + (size_t)B * 2 * d) * 8;

@@ -48,6 +48,9 @@ struct TcCfg {
 };
 enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = 2, BAR_Q_FULL = 4, BAR_S_READY = 5, BAR_P_READY = 6 };
 
+// ALIBI / CAUSAL are compile-time so that the plain kernel carries none of their registers or instructions
+// (it runs at 80 registers per thread, four CTAs per SM, and loses a fifth of its rate to a few spills).
+template <bool ALIBI, bool CAUSAL>
 __global__ void __launch_bounds__(TcCfg::threads, TcCfg::ctas_per_sm)
 tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const TileParams p, SyncArea* sync) {
@@ -59,12 +62,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
-  const int shift = (int)blockIdx.z * p.batch_stride;     // copy z of the tile (one level of Algorithm 1 in one launch)
-  const int k0 = p.k0 + shift;
-  int q1 = p.q1 + shift;
-  if (p.q_limit > 0 && q1 > p.q_limit) q1 = p.q_limit;
-  const int qb = p.q0 + shift + blockIdx.x * kBM;         // first query row of this CTA
-  if (qb >= q1) return;                                   // nothing left of this copy (uniform per CTA)
+  // copy blockIdx.z of the tile (one level of Algorithm 1 in one launch); the few values derived from it are
+  // recomputed where they are used rather than kept in registers across the roles
+  auto shift = [&]() { return (int)blockIdx.z * p.batch_stride; };
+  auto q_end = [&]() { const int q1 = p.q1 + shift(); return (p.q_limit > 0 && q1 > p.q_limit) ? p.q_limit : q1; };
+  const int qb = p.q0 + shift() + blockIdx.x * kBM;       // first query row of this CTA
+  if (qb >= q_end()) return;                              // nothing left of this copy (uniform per CTA)
   const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + C::tmem_ptr);
@@ -90,6 +93,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (warp == kTmaWarp) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
+      const int k0 = p.k0 + shift();
       mbar_expect_tx(bar(BAR_Q_FULL), kQBytes);
       tma_load_4d(sbase + C::q, &map_q, bar(BAR_Q_FULL), 0, h, b, qb);
       int issued = 0;
@@ -156,12 +160,12 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ------------------------------ softmax warps: one thread per query row ------------------------------
     const int row = warp * 32 + lane;
     const int qi = qb + row;
-    const bool row_ok = qi < q1;
+    const bool row_ok = qi < q_end();
     const uint32_t t_s = tmem + ((uint32_t)(warp * 32) << 16);
     const uint32_t t_o = t_s + 64u;
     const size_t sidx = (size_t)(row_ok ? qi : p.q0) * p.B + b;
     float m_used = p.st_m[sidx * p.H + h];                   // reference maximum of l and O (log2 units)
-    const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
+    const float slope_l2 = ALIBI ? p.alibi[h] * kLog2e : 0.f;
     const float step_raw = slope_l2 / p.scale_log2;          // slope per column, in units of the raw product
     float m_true = m_used;                                   // running maximum
     float l_run = p.st_l[sidx * p.H + h];
@@ -189,17 +193,18 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // ALiBi distances: the logit of this row's query (position qi) on key j gets -slope (qi - j)
       // = base + slope * column: the column part goes into the raw products (divided by the scale that is
       // applied below), the row constant into the maximum and the exponent offset
-      const float base_l2 = -slope_l2 * (float)(qi - (k0 + kb * kBK));
-      if (slope_l2 != 0.f) {
+      float base_l2 = 0.f;
+      if (ALIBI) {
+        base_l2 = -slope_l2 * (float)(qi - (p.k0 + shift() + kb * kBK));
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           s0[i] = __float_as_uint(fmaf(step_raw, (float)i, __uint_as_float(s0[i])));
           s1[i] = __float_as_uint(fmaf(step_raw, (float)(i + 32), __uint_as_float(s1[i])));
         }
       }
-      if (p.causal) {
+      if (CAUSAL) {
         // only pairs at earlier positions than this row's query: the rest of the block gets -inf (p = 0)
-        const int n_valid = qi - (k0 + kb * kBK);
+        const int n_valid = qi - (p.k0 + shift() + kb * kBK);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           if (i >= n_valid) s0[i] = 0xff800000u;
@@ -211,12 +216,14 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
 #pragma unroll
       for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
-      const float mx = fmaf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), p.scale_log2, base_l2);
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      if (ALIBI) mx += base_l2;
       m_true = fmaxf(m_true, mx);
       const bool raise = mx > m_used + kLazyLog2;
       const float m_new = raise ? m_true : m_used;
       const float corr = ex2(m_used - m_new);                  // 1 when the reference stays
-      const float neg_m = base_l2 - m_new;
+      float neg_m = -m_new;
+      if (ALIBI) neg_m += base_l2;
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       // p = 2^(s*scale - m) as packed bf16, written over the first 32 columns of the S buffer
       uint32_t w[16];
@@ -310,11 +317,18 @@ cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncAre
       !make_map(&mv, p.v_cache, rows_kv, p.B, p.H, kBK))
     return cudaErrorInvalidValue;
   const size_t smem = TcCfg::total + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tile_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   dim3 grid(ceil_div(nq, kBM), p.B * p.H, p.batch > 1 ? p.batch : 1);
-  tile_tc_kernel<<<grid, TcCfg::threads, smem, s>>>(mq, mk, mv, p, sync);
-  return cudaGetLastError();
+  auto go = [&](auto kernel) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, TcCfg::threads, smem, s>>>(mq, mk, mv, p, sync);
+    return cudaGetLastError();
+  };
+  const bool alibi = p.alibi != nullptr, causal = p.causal != 0;
+  if (alibi && causal) return go(tile_tc_kernel<true, true>);
+  if (alibi) return go(tile_tc_kernel<true, false>);
+  if (causal) return go(tile_tc_kernel<false, true>);
+  return go(tile_tc_kernel<false, false>);
 }
 
 }  // namespace rt
