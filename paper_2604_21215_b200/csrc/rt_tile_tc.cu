@@ -187,35 +187,40 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_READY), kb & 1, s_abort, sync));
       if (!ok) break;
       tc_fence_after();
-      tc_ld32(t_s, s0);
-      tc_ld32(t_s + 32u, s1);
-      tc_wait_ld();
       // ALiBi distances: the logit of this row's query (position qi) on key j gets -slope (qi - j)
       // = base + slope * column: the column part goes into the raw products (divided by the scale that is
-      // applied below), the row constant into the maximum and the exponent offset
+      // applied below), the row constant into the maximum and the exponent offset.  Causal launches turn the
+      // pairs at or beyond the row's position into -inf (p = 0).
       float base_l2 = 0.f;
-      if (ALIBI) {
-        base_l2 = -slope_l2 * (float)(qi - (p.k0 + shift() + kb * kBK));
+      if (ALIBI) base_l2 = -slope_l2 * (float)(qi - (p.k0 + shift() + kb * kBK));
+      auto adjust = [&](uint32_t (&v)[32], int col0) {
+        if (ALIBI) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          s0[i] = __float_as_uint(fmaf(step_raw, (float)i, __uint_as_float(s0[i])));
-          s1[i] = __float_as_uint(fmaf(step_raw, (float)(i + 32), __uint_as_float(s1[i])));
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaf(step_raw, (float)(i + col0), __uint_as_float(v[i])));
         }
-      }
-      if (CAUSAL) {
-        // only pairs at earlier positions than this row's query: the rest of the block gets -inf (p = 0)
-        const int n_valid = qi - (p.k0 + shift() + kb * kBK);
+        if (CAUSAL) {
+          const int n_valid = qi - (p.k0 + shift() + kb * kBK);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (i >= n_valid) s0[i] = 0xff800000u;
-          if (i + 32 >= n_valid) s1[i] = 0xff800000u;
+          for (int i = 0; i < 32; ++i)
+            if (i + col0 >= n_valid) v[i] = 0xff800000u;
         }
-      }
+      };
+      // The row lives in registers half at a time (32 of its 64 values): the second half is read for the
+      // maximum, dropped, and read again for the exponentials.  A TMEM load costs little; holding all 64
+      // values next to the packed P words would not fit the 80 registers four resident CTAs leave a thread.
       float mx4[4];                                            // four independent chains
+      tc_ld32(t_s + 32u, s1);
+      tc_wait_ld();
+      adjust(s1, 32);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j]));
+      for (int j = 0; j < 4; ++j) mx4[j] = __uint_as_float(s1[j]);
 #pragma unroll
-      for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+      for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(s1[i]));
+      tc_ld32(t_s, s0);
+      tc_wait_ld();
+      adjust(s0, 0);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(s0[i]));
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
       if (ALIBI) mx += base_l2;
       m_true = fmaxf(m_true, mx);
@@ -235,7 +240,10 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
         w[j] = *reinterpret_cast<const uint32_t*>(&pk);
       }
+      tc_ld32(t_s + 32u, s1);                                  // columns 32..63 are still the raw products
       tc_st16(t_s, w);
+      tc_wait_ld();
+      adjust(s1, 32);
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         const float p0 = ex2(fmaf(__uint_as_float(s1[2 * j]), p.scale_log2, neg_m));
