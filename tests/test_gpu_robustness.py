@@ -286,3 +286,25 @@ def test_alibi_update_tile_matches_algorithm_2(dtype, nq, nk):
     lse_g = mg / LOG2E + np.log(lg)
     lse_r = m_ref + np.log(l_ref)
     assert np.abs(lse_g - lse_r).max() <= tol * max(1.0, np.abs(lse_r).max())
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_alibi_stack_prefill_and_decode_match_oracle(dtype):
+    from oracle import RTConfig, RTWeights, stack_prefill, stack_decode
+    from paper_2604_21215_b200 import inputs, rt
+    L, d, H, dff, V, B, N = 3, 128, 2, 256, 300, 2, 70
+    wl = inputs.Workload("alibi_stack", L, B, N + 1, d, H, dff, dtype, vocab=V, residual_scale=1 / np.sqrt(L))
+    data = inputs.make_inputs(wl, seed=8400)
+    slopes = _slopes(H)
+    ocfg = RTConfig(d, H, 64, dff, residual_scale=wl.residual_scale, alibi_slopes=slopes)
+    ow = [RTWeights(**lw) for lw in data["layers"]]
+    hid_ref, logits_ref, caches_ref = stack_prefill(ocfg, ow, data["emb"], None, data["ids"])
+    st = rt.Stack(L, d, H, dff, V, dtype=dtype, leaf=16, residual_scale=wl.residual_scale)
+    st.set_weights([dict(lw, alibi_slopes=slopes) for lw in data["layers"]], data["emb"])
+    hid, logits = st.prefill(data["ids"])
+    tol = TOL[dtype]
+    assert rel_err(hid, hid_ref) <= tol and rel_err(logits, logits_ref) <= tol
+    hid2, _ = st.prefill(data["ids"][:, :N], N_max=N + 1)
+    assert rel_err(hid2, hid_ref[:, :N]) <= tol
+    lg = st.decode(data["ids"][:, N], N)
+    assert rel_err(lg, logits_ref) <= tol
