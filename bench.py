@@ -142,6 +142,8 @@ def sample_positions(wl):
     n = 1024 if wl.d_model <= 768 else 512
     if wl.n_layers > 1:
         n = max(32, n // wl.n_layers)
+    if wl.B > 64:                                      # wide batches: keep the sample near 16 k tokens
+        n = max(8, 16384 // wl.B)
     return min(wl.N, n)
 
 
@@ -308,6 +310,20 @@ def run_cuda(args):
                             "latency of its five all-to-all exchanges per token step (L2 round trips), not by HBM; "
                             "the fraction is the effective weight+activation stream against the HBM copy peak and "
                             "traffic is the DRAM bytes ncu counted for one launch"}
+        if wl.B > 64:
+            # wide batches: the token step is a chain of dense products over the B rows (tcgen05), one position at
+            # a time; the leaf class of the profile holds them together with the small in-leaf attention kernels
+            tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))).get("bf16_tflops_sustained", 1403.5)) \
+                if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else 1400.0
+            flops = 2.0 * B * (5 * d * d + 2 * d * f) * wl.N * wl.n_layers * args.steps      # W_o, W_up, W_down, W_k, W_v per step
+            ms_all = prof["leaf"]["ms"]
+            achieved = flops / (ms_all * 1e-3) / 1e12 if ms_all > 0 else 0.0
+            roofline = {"kernel": "dense_tc_kernel (wide-batch token steps, with their small kernels)", "bound": "tensor",
+                        "achieved": achieved, "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak,
+                        "peak_source": "measured (sustained)", "traffic": None,
+                        "us_per_token_step": 1e3 * ms_all / max(wl.N * wl.n_layers * args.steps, 1),
+                        "note": "M = B rows per product: each token step is ten short dependent launches, so launch latency "
+                                "and the L2 stream of the weights, not the tensor pipe, set the time"}
         tile_ms = prof["tile"]["ms"]
         tile_tflops = (counters["flops_tile"] * args.steps / (tile_ms * 1e-3) / 1e12) if tile_ms > 0 else None
         n_pos = sample_positions(wl)
@@ -317,13 +333,21 @@ def run_cuda(args):
         launches = sum(v["launches"] for v in prof.values())
         # the pre-pass group is three kernels, every other group one
         gpu_launches = int(launches + 2 * prof["prepass"]["launches"])
+        if wl.B > 64:
+            # wide batches: per position one in-leaf attention launch (not for the first of a leaf), c = o/l, three dense
+            # products (W_o and W_down split at this shape: + a reduction each), RMS(h), and RMS(z) + the K/V projection;
+            # per call the pre-pass (3) and one cross tile per leaf boundary
+            lf = int(model.cfg.leaf) or 32
+            n_leaves = (wl.N + lf - 1) // lf
+            per_call = (wl.N - n_leaves) + wl.N + 3 * wl.N + 2 * wl.N + wl.N + 2 * wl.N + 3 + (n_leaves - 1)
+            gpu_launches = int(per_call * wl.n_layers * args.steps)
         h2d = host_in.numel() * host_in.element_size()
         d2h = host_out.numel() * host_out.element_size()
         line = {"metric": METRIC, "value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, total_ms), "unit": UNIT,
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16/f32-accumulate" if wl.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": config_dict(wl, args.sched, {"alibi": bool(args.alibi), "leaf": int(model.cfg.leaf) or 64,
+                "data": "synthetic", "config": config_dict(wl, args.sched, {"alibi": bool(args.alibi), "leaf": int(model.cfg.leaf) or (32 if wl.B > 64 else 64),
                                                                             "parallelism": f"replicas x{world}"}),
                 "clocks": clocks,
                 "e2e": {"value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, e2e_total), "unit": UNIT,

@@ -34,11 +34,13 @@ bool config_ok(const rt_config* c) {
   return true;
 }
 
-rt_status config_supported(const rt_config* c, int B) {
+constexpr int kSmallBatchMax = 64;      // above this the per-token chain runs as dense products (tiled prefill only)
+
+rt_status config_supported(const rt_config* c, int B, bool wide_ok = false) {
   if (c->head_dim != kHeadDim) return RT_ERR_UNSUPPORTED;
   if (c->norm_flags & RT_NORM_QK_FULL) return RT_ERR_UNSUPPORTED;
   if (c->d_ff % 4) return RT_ERR_UNSUPPORTED;
-  if (B > 64) return RT_ERR_UNSUPPORTED;                 // the per-token chain is written for small batches
+  if (B > kSmallBatchMax && !(wide_ok && c->sched == RT_SCHED_TILED)) return RT_ERR_UNSUPPORTED;
   return RT_OK;
 }
 
@@ -136,6 +138,73 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
   }
 
+  if (B > kSmallBatchMax) {
+    // Wide batches (the regime of the paper's own experiments, Sec. 6: B in the hundreds): a token step is a chain
+    // of dense products with M = B rows, so it runs on the tensor cores through the same kernels as the parallel
+    // sweep, one position at a time; the schedule (leaf, then the cross tile of Algorithm 1) is unchanged.
+    if (c->sched != RT_SCHED_TILED || pos0 != 0) return RT_ERR_UNSUPPORTED;
+    const long long d = c->d_model, f = c->d_ff;
+    const size_t e = esize_of(c->dtype);
+    SyncArea* sync = (SyncArea*)(ws + L.sync);
+    float* hbuf = (float*)(ws + L.ex_h);                        // [B, d] fp32
+    void* gbuf = ws + L.ex_g;                                   // [B, d_ff] storage type
+    void* ubuf = ws + L.ex_z;                                   // [B, d] storage type
+    void* cbuf = ws + L.ex_k;                                   // [B, d] storage type
+    const bool pre = (c->norm_flags & RT_NORM_PRE) != 0;
+    TileParams tp;
+    memset(&tp, 0, sizeof(tp));
+    tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2; tp.alibi = w->alibi_slopes;
+    tp.q = ws + L.q; tp.k_cache = k_cache; tp.v_cache = v_cache;
+    tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
+    tp.rows_q = n_rows; tp.rows_kv = n_max; tp.sync = sync;
+    PrepassParams pk = pp;                                      // persistent pair of one position from its output
+    pk.N = 1; pk.x_bs = z_bs; pk.x_ts = z_ts;
+    pk.norm_flags = (c->norm_flags & RT_NORM_SKIP_Z) ? (c->norm_flags & ~RT_NORM_PRE) : c->norm_flags;
+    pk.g_attn = w->g_kv ? w->g_kv : w->g_attn;
+    pk.mats = 6; pk.no_seed = 1;
+    DenseParams dp;
+    memset(&dp, 0, sizeof(dp));
+    dp.M = B; dp.B = B; dp.alpha = c->residual_scale; dp.h = hbuf;
+    dp.partial = (float*)(ws + L.ex_part); dp.partial_bytes = (size_t)B * c->n_heads * kMaxChunks * 68 * 4;
+    // in-leaf attention re-reads the leaf's pairs for every position (leaf^2 * B * d bytes per leaf), so wide
+    // batches default to a shorter leaf
+    const int Lf = c->leaf ? c->leaf : 32, N = n_rows;
+    for (int s0 = 0; s0 < N; s0 += Lf) {
+      const int e0 = s0 + Lf < N ? s0 + Lf : N;
+      {
+        ProfScope ps(s, kProfLeaf);
+        for (int t = s0; t < e0; ++t) {
+          if (t > s0) {                                         // pairs of this leaf revealed so far
+            tp.q0 = t; tp.q1 = t + 1; tp.k0 = s0; tp.k1 = t;
+            if (row_attn_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          }
+          const size_t row = (size_t)t * B;
+          if (attn_value_launch(c->dtype, pp.st_o + row * d, pp.st_l + row * c->n_heads, cbuf, B, (int)d, c->n_heads, s) != cudaSuccess)
+            return RT_ERR_CUDA;
+          dp.N = (int)d; dp.K = (int)d; dp.A = cbuf; dp.W = w->w_o; dp.epi = DENSE_RES_X;
+          dp.x = (const unsigned char*)x + (size_t)t * x_ts * e; dp.x_bs = x_bs; dp.x_ts = 0;
+          if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+          if (rms_rows_f32_launch(c->dtype, hbuf, w->g_mlp, ubuf, B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess) return RT_ERR_CUDA;
+          dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;
+          if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+          dp.N = (int)d; dp.K = (int)f; dp.A = gbuf; dp.W = w->w_down; dp.epi = DENSE_RES_H;
+          dp.out = (unsigned char*)z + (size_t)t * z_ts * e; dp.o_bs = z_bs; dp.o_ts = 0;
+          if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+          pk.x = (const unsigned char*)z + (size_t)t * z_ts * e;
+          pk.kt = (unsigned char*)k_cache + row * d * e; pk.vt = (unsigned char*)v_cache + row * d * e;
+          if (prepass_launch(c->dtype, pk, s) != cudaSuccess) return RT_ERR_CUDA;
+        }
+      }
+      if (e0 < N) {
+        const int P = e0 & -e0;
+        tp.q0 = e0; tp.q1 = e0 + P < N ? e0 + P : N; tp.k0 = e0 - P; tp.k1 = e0;
+        ProfScope ps(s, kProfTile);
+        if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+      }
+    }
+    return RT_OK;
+  }
+
   LeafLaunch ll;
   if (leaf_plan(c->dtype, B, c->d_model, c->d_ff, &ll) != cudaSuccess) return RT_ERR_CUDA;
   LeafParams lp;
@@ -208,9 +277,9 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   return RT_OK;
 }
 
-rt_status common_checks(const rt_config* c, int B, int N, int n_layers, void* ws, size_t ws_bytes) {
+rt_status common_checks(const rt_config* c, int B, int N, int n_layers, void* ws, size_t ws_bytes, bool wide_ok = false) {
   if (!config_ok(c) || B <= 0 || N <= 0 || n_layers <= 0 || !ws || !aligned16(ws)) return RT_ERR_INVALID_ARG;
-  const rt_status st = config_supported(c, B);
+  const rt_status st = config_supported(c, B, wide_ok);
   if (st != RT_OK) return st;
   if (ws_bytes < ws_layout(c, B, N).total) return RT_ERR_WORKSPACE;
   return RT_OK;
@@ -228,7 +297,7 @@ size_t rt_workspace_bytes(const rt_config* cfg, int32_t B, int32_t N, int32_t n_
 rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, const void* x, int32_t B, int32_t N,
                            void* z, void* k_cache, void* v_cache, int32_t N_max, void* workspace,
                            size_t workspace_bytes, void* cuda_stream) {
-  rt_status st = common_checks(cfg, B, N, 1, workspace, workspace_bytes);
+  rt_status st = common_checks(cfg, B, N, 1, workspace, workspace_bytes, true);
   if (st != RT_OK) return st;
   if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || x == z || N_max < N) return RT_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(z) || !aligned16(k_cache) || !aligned16(v_cache)) return RT_ERR_INVALID_ARG;
@@ -371,7 +440,7 @@ rt_status rt_stack_prefill(const rt_config* cfg, int32_t n_layers, const rt_laye
                            const void* g_final, int32_t vocab, const int32_t* ids, int32_t B, int32_t N, void* hidden,
                            float* logits_last, void* const* k_caches, void* const* v_caches, int32_t N_max,
                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  rt_status st = common_checks(cfg, B, N, n_layers, workspace, workspace_bytes);
+  rt_status st = common_checks(cfg, B, N, n_layers, workspace, workspace_bytes, true);
   if (st != RT_OK) return st;
   if (!layers || !emb || !ids || !k_caches || !v_caches || vocab <= 0 || N_max < N) return RT_ERR_INVALID_ARG;
   if (!aligned16(emb) || (hidden && !aligned16(hidden)) || (g_final && !aligned16(g_final))) return RT_ERR_INVALID_ARG;

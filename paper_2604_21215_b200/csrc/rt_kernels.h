@@ -90,6 +90,8 @@ cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s);
 // tensor-core version (bf16, key count a multiple of 64)
 cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncArea* sync, cudaStream_t s);
 cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s);
+// one query row (position q0) per (sequence, head) against the pairs [k0, k1): the in-leaf step of wide batches
+cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s);
 
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,
@@ -108,6 +110,8 @@ struct DenseParams {
   const void* x; long long x_bs, x_ts;           // x[b, r, :] (DENSE_RES_X)
   float* h;                                      // [M, N] fp32 (written by DENSE_RES_X, read by DENSE_RES_H)
   void* out; long long o_bs, o_ts;               // DENSE_GELU: [M, N];  DENSE_RES_H: out[b, r, :]
+  float* partial; size_t partial_bytes;          // optional scratch for a split contraction (few rows): [splits, M, N] fp32
+  int splits;                                    // set by the launcher
 };
 cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s);
 cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s);

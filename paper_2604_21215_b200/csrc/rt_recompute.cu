@@ -141,7 +141,11 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   constexpr int kTBN = BN;
   constexpr uint32_t kTBBytes = DS::b_bytes;
   const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kTBN;
-  const int n_kb = p.K / kTBK;
+  // split z of the contraction: k blocks [kb0, kb0 + n_kb)
+  const int splits = p.splits > 1 ? p.splits : 1;
+  const int kb_all = p.K / kTBK;
+  const int kb0 = (int)((long long)kb_all * blockIdx.z / splits);
+  const int n_kb = (int)((long long)kb_all * (blockIdx.z + 1) / splits) - kb0;
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + DS::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + DS::tmem_ptr);
   auto full = [&](int s) { return sbase + DS::bars + 8u * (uint32_t)s; };
@@ -173,8 +177,8 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (kb >= kTStages) ok = mbar_wait(empty(s), ((kb / kTStages) - 1) & 1, s_abort, sync);
         if (!ok) break;
         mbar_expect_tx(full(s), kTABytes + kTBBytes);
-        tma_load_2d(sbase + DS::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
-        tma_load_2d(sbase + DS::b + s * kTBBytes, &map_w, full(s), kb * kTBK, n0);
+        tma_load_2d(sbase + DS::a + s * kTABytes, &map_a, full(s), (kb0 + kb) * kTBK, m0);
+        tma_load_2d(sbase + DS::b + s * kTBBytes, &map_w, full(s), (kb0 + kb) * kTBK, n0);
         ++issued;
       }
       if (!ok) {
@@ -220,6 +224,13 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         tc_wait_ld();
         if (m >= p.M) continue;
         const int n = n0 + c0;
+        if (splits > 1) {                                          // raw partial sums; dense_reduce_kernel finishes
+          float4* dst = reinterpret_cast<float4*>(p.partial + ((size_t)blockIdx.z * p.M + m) * p.N + n);
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          continue;
+        }
         if (p.epi == DENSE_RES_X) {
           const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n);
           float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
@@ -277,6 +288,17 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   }
 }
 
+// Sums the partial products of a split contraction in a fixed order and applies the epilogue.
+template <typename T>
+__global__ void dense_reduce_kernel(const DenseParams p) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)p.M * p.N) return;
+  const int m = (int)(i / p.N), n = (int)(i % p.N);
+  float acc = 0.f;
+  for (int z = 0; z < p.splits; ++z) acc += p.partial[((size_t)z * p.M + m) * p.N + n];
+  epi_store<T>(p, m, n, acc);
+}
+
 // row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
 static bool make_map_rows(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows) {
   EncodeTiledFn fn = encode_fn();
@@ -295,20 +317,39 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
   const bool strides_ok = p.epi == DENSE_GELU || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
                                                   ((p.epi == DENSE_RES_X ? p.x_ts : p.o_ts) % 8 == 0));
   if (dtype == RT_BF16 && p.N % 128 == 0 && p.K % kTBK == 0 && strides_ok) {
-    const int bn = p.N % 256 == 0 ? 256 : 128;
+    // Few rows (the wide-batch token step: M = B): narrow tiles and a split contraction so that the launch still
+    // fills the GPU; the partial sums are combined in a fixed order by a second small kernel.
+    int sms = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+    const int m_tiles = ceil_div(p.M, kBM);
+    int bn = p.N % 256 == 0 ? 256 : 128;
+    if (bn == 256 && m_tiles * (p.N / 256) < sms) bn = 128;
+    DenseParams q = p;
+    q.splits = 1;
+    const int ctas = m_tiles * (p.N / bn), kb_all = p.K / kTBK;
+    if (p.partial && ctas < sms / 2 && kb_all >= 8) {
+      int want = (sms + ctas - 1) / ctas;                         // about one wave
+      if (want > 8) want = 8;
+      while (want > 1 && kb_all / want < 4) --want;               // at least 4 k blocks per split
+      if ((size_t)want * p.M * p.N * sizeof(float) <= p.partial_bytes) q.splits = want;
+    }
     CUtensorMap ma, mw;
     if (!make_map_rows(&ma, p.A, p.M, p.K, kBM) || !make_map_rows(&mw, p.W, p.N, p.K, bn)) return cudaErrorInvalidValue;
-    dim3 grid(ceil_div(p.M, kBM), p.N / bn);
+    dim3 grid(m_tiles, p.N / bn, q.splits);
     if (bn == 256) {
       const size_t smem = DenseSmem<256>::total + 1024;
       cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      dense_tc_kernel<256><<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+      dense_tc_kernel<256><<<grid, kTThreads, smem, s>>>(ma, mw, q, sync);
     } else {
       const size_t smem = DenseSmem<128>::total + 1024;
       cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      dense_tc_kernel<128><<<grid, kTThreads, smem, s>>>(ma, mw, p, sync);
+      dense_tc_kernel<128><<<grid, kTThreads, smem, s>>>(ma, mw, q, sync);
+    }
+    if (q.splits > 1) {
+      const long long total = (long long)p.M * p.N;
+      dense_reduce_kernel<__nv_bfloat16><<<(unsigned)((total + 255) / 256), 256, 0, s>>>(q);
     }
     return cudaGetLastError();
   }

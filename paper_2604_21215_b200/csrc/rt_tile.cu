@@ -102,6 +102,65 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+// ---- one query row per (sequence, head) against a short run of pairs -----------------------------------
+// Used by the wide-batch token step: position t attends to the pairs of its own leaf revealed so far,
+// [k0, k1) with k1 = t.  One warp per (sequence, head): each K and V row is one coalesced load (lanes over
+// the head's dimensions), the 32 per-lane partial products become per-key scores by a transposed reduction.
+template <typename T>
+__global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
+  const int lane = threadIdx.x & 31;
+  const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (u >= p.B * p.H) return;
+  const int b = u / p.H, h = u % p.H;
+  const int t = p.q0;
+  const T* Kc = reinterpret_cast<const T*>(p.k_cache);
+  const T* Vc = reinterpret_cast<const T*>(p.v_cache);
+  const size_t col = (size_t)b * p.d + h * kHeadDim + 2 * lane;
+  const size_t rstride = (size_t)p.B * p.d;
+  const T* qrow = reinterpret_cast<const T*>(p.q) + (size_t)t * rstride + col;
+  const float q0 = to_f(qrow[0]), q1 = to_f(qrow[1]);
+  const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
+  const size_t sidx = (size_t)t * p.B + b;
+  float m_run = p.st_m[sidx * p.H + h], l_run = p.st_l[sidx * p.H + h];
+  float2 o = *reinterpret_cast<const float2*>(p.st_o + sidx * p.d + h * kHeadDim + 2 * lane);
+  for (int jb = p.k0; jb < p.k1; jb += 32) {
+    const int cnt = (p.k1 - jb < 32) ? (p.k1 - jb) : 32;
+    float prod[32];
+    float2 vv[32];
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj) {
+      const int j = jb + (jj < cnt ? jj : 0);
+      const float2 k2 = ldcg_T2(Kc + (size_t)j * rstride + col);
+      vv[jj] = ldcg_T2(Vc + (size_t)j * rstride + col);
+      prod[jj] = q0 * k2.x + q1 * k2.y;
+    }
+    warp_transpose_sum32(prod, lane);
+    const bool valid = lane < cnt;
+    const float s2 = valid ? prod[0] * p.scale_log2 - slope_l2 * (float)(t - (jb + lane)) : -INFINITY;
+    const float m_new = fmaxf(m_run, warp_max(s2));
+    const float pj = valid ? exp2f(s2 - m_new) : 0.f;
+    const float corr = exp2f(m_run - m_new);
+    l_run = l_run * corr + warp_sum(pj);
+    o.x *= corr; o.y *= corr;
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj) {
+      const float pw = __shfl_sync(0xffffffffu, pj, jj);
+      o.x += pw * vv[jj].x; o.y += pw * vv[jj].y;
+    }
+    m_run = m_new;
+  }
+  if (lane == 0) { p.st_m[sidx * p.H + h] = m_run; p.st_l[sidx * p.H + h] = l_run; }
+  *reinterpret_cast<float2*>(p.st_o + sidx * p.d + h * kHeadDim + 2 * lane) = o;
+}
+
+cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  if (p.k1 <= p.k0) return cudaSuccess;
+  const int blocks = ceil_div(p.B * p.H, 8);
+  if (dtype == RT_BF16) row_attn_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(p);
+  else row_attn_kernel<float><<<blocks, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
   // Whole 64-key blocks only on the tensor-core path: a partial block would bring cache rows that
   // are not revealed yet (arbitrary bits) into the P.V product.

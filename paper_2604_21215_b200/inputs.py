@@ -40,8 +40,11 @@ WORKLOADS: Dict[str, Workload] = {
     "c3": Workload("c3", 1, 8, 4096, 1024, 16, 4096, "bf16"),
     "c4": Workload("c4", 8, 16, 2048, 1024, 16, 4096, "bf16", vocab=32000,
                    residual_scale=1.0 / np.sqrt(8.0)),
+    # not one of the five: the shape of the paper's own latency table (Sec. 6: one layer, N = 512, d = 1024,
+    # 16 heads, batch 512), where a token step is a dense product over the batch
+    "p512": Workload("p512", 1, 512, 512, 1024, 16, 4096, "bf16"),
 }
-CONFIG_INDEX = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+CONFIG_INDEX = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "p512": 40}
 
 
 def sweep(N: int) -> Workload:

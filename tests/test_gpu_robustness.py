@@ -308,3 +308,35 @@ def test_alibi_stack_prefill_and_decode_match_oracle(dtype):
     assert rel_err(hid2, hid_ref[:, :N]) <= tol
     lg = st.decode(data["ids"][:, N], N)
     assert rel_err(lg, logits_ref) <= tol
+
+
+# ---------------------------------------------------------------- wide batches: the token step as dense products
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N,leaf,alibi", [
+    ("f32", 128, 2, 256, 70, 40, 16, False), ("bf16", 256, 4, 1024, 130, 75, 32, True),
+    ("bf16", 128, 2, 512, 96, 33, 16, False)])
+def test_wide_batch_prefill_matches_oracle(dtype, d, H, dff, B, N, leaf, alibi):
+    # B > 64: every token step runs as dense products over the B rows (tensor cores for bf16)
+    from oracle import RTConfig, RTWeights, layer_seq
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("wide", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=8500 + B)
+    lw = data["layers"][0]
+    slopes = _slopes(H) if alibi else None
+    ref = layer_seq(RTConfig(d, H, 64, dff, alibi_slopes=slopes, residual_scale=0.7), RTWeights(**lw), data["x"])
+    layer = _layer(d, H, dff, dtype, dict(lw, alibi_slopes=slopes) if alibi else lw, leaf=leaf, residual_scale=0.7)
+    got = layer.prefill(data["x"])
+    for name, g_, r_ in zip(("z", "k", "v"), got, ref):
+        assert np.isfinite(g_).all(), name
+        assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
+
+
+def test_wide_batch_unsupported_paths_say_so():
+    from paper_2604_21215_b200 import inputs, rt
+    d, H, dff, B, N = 128, 2, 256, 70, 8
+    wl = inputs.Workload("wide", 1, B, N, d, H, dff, "f32")
+    data = inputs.make_inputs(wl, seed=1)
+    layer = _layer(d, H, dff, "f32", data["layers"][0], sched="naive")
+    with pytest.raises(rt.RtError) as ei:
+        layer.prefill(data["x"])
+    assert ei.value.status == rt.RT_ERR_UNSUPPORTED
