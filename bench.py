@@ -334,12 +334,12 @@ def run_cuda(args):
         # the pre-pass group is three kernels, every other group one
         gpu_launches = int(launches + 2 * prof["prepass"]["launches"])
         if wl.B > 64:
-            # wide batches: per position one in-leaf attention launch (not for the first of a leaf), c = o/l, three dense
-            # products (W_o and W_down split at this shape: + a reduction each), RMS(h), and RMS(z) + the K/V projection;
-            # per call the pre-pass (3) and one cross tile per leaf boundary
+            # wide batches: per position one in-leaf attention launch (which also leaves c = o/l), three dense products
+            # (W_o and W_down split at this shape: + a reduction each, which also leaves the row norms) and the K/V
+            # projection; per call the pre-pass (3) and one cross tile per leaf boundary
             lf = int(model.cfg.leaf) or 32
             n_leaves = (wl.N + lf - 1) // lf
-            per_call = (wl.N - n_leaves) + wl.N + 3 * wl.N + 2 * wl.N + wl.N + 2 * wl.N + 3 + (n_leaves - 1)
+            per_call = wl.N + 3 * wl.N + 2 * wl.N + wl.N + 3 + (n_leaves - 1)
             gpu_launches = int(per_call * wl.n_layers * args.steps)
         h2d = host_in.numel() * host_in.element_size()
         d2h = host_out.numel() * host_out.element_size()

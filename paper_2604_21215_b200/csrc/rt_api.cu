@@ -174,22 +174,27 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
       {
         ProfScope ps(s, kProfLeaf);
         for (int t = s0; t < e0; ++t) {
-          if (t > s0) {                                         // pairs of this leaf revealed so far
-            tp.q0 = t; tp.q1 = t + 1; tp.k0 = s0; tp.k1 = t;
-            if (row_attn_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
-          }
+          // pairs of this leaf revealed so far (none for its first position), then c = o / l of the finished row
+          tp.q0 = t; tp.q1 = t + 1; tp.k0 = s0; tp.k1 = t; tp.c_out = cbuf;
+          if (row_attn_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          tp.c_out = nullptr;
           const size_t row = (size_t)t * B;
-          if (attn_value_launch(c->dtype, pp.st_o + row * d, pp.st_l + row * c->n_heads, cbuf, B, (int)d, c->n_heads, s) != cudaSuccess)
-            return RT_ERR_CUDA;
+          bool normed = false;
           dp.N = (int)d; dp.K = (int)d; dp.A = cbuf; dp.W = w->w_o; dp.epi = DENSE_RES_X;
           dp.x = (const unsigned char*)x + (size_t)t * x_ts * e; dp.x_bs = x_bs; dp.x_ts = 0;
-          if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
-          if (rms_rows_f32_launch(c->dtype, hbuf, w->g_mlp, ubuf, B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess) return RT_ERR_CUDA;
+          dp.norm_out = ubuf; dp.norm_gain = w->g_mlp; dp.norm_eps = c->rms_eps; dp.norm_pre = pre ? 1 : 0;   // u = RMS(h)
+          if (dense_launch(c->dtype, dp, sync, s, &normed) != cudaSuccess) return RT_ERR_CUDA;
+          if (!normed && rms_rows_f32_launch(c->dtype, hbuf, w->g_mlp, ubuf, B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess)
+            return RT_ERR_CUDA;
+          dp.norm_out = nullptr;
           dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;
           if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
           dp.N = (int)d; dp.K = (int)f; dp.A = gbuf; dp.W = w->w_down; dp.epi = DENSE_RES_H;
           dp.out = (unsigned char*)z + (size_t)t * z_ts * e; dp.o_bs = z_bs; dp.o_ts = 0;
-          if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+          dp.norm_out = pk.n; dp.norm_gain = pk.g_attn; dp.norm_pre = (pk.norm_flags & RT_NORM_PRE) ? 1 : 0;          // RMS(z)
+          if (dense_launch(c->dtype, dp, sync, s, &normed) != cudaSuccess) return RT_ERR_CUDA;
+          dp.norm_out = nullptr;
+          pk.skip_rms = normed ? 1 : 0;
           pk.x = (const unsigned char*)z + (size_t)t * z_ts * e;
           pk.kt = (unsigned char*)k_cache + row * d * e; pk.vt = (unsigned char*)v_cache + row * d * e;
           if (prepass_launch(c->dtype, pk, s) != cudaSuccess) return RT_ERR_CUDA;

@@ -136,7 +136,7 @@ __global__ void state_init_kernel(const PrepassParams p) {
 template <typename T>
 static cudaError_t prepass_typed(const PrepassParams& p, cudaStream_t s) {
   const int M = p.N * p.B;
-  rms_rows_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(p);
+  if (!p.skip_rms) rms_rows_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(p);
   if (sizeof(T) == 2 && qkv_gemm_tc_supported(p)) {
     const cudaError_t e = qkv_gemm_tc_launch(p, p.sync, s);
     if (e != cudaSuccess) return e;

@@ -288,15 +288,47 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   }
 }
 
-// Sums the partial products of a split contraction in a fixed order and applies the epilogue.
+// Sums the partial products of a split contraction in a fixed order and applies the epilogue; one CTA per
+// output row, so it can also leave RMS_g(row) of the result for the product that follows.
 template <typename T>
-__global__ void dense_reduce_kernel(const DenseParams p) {
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (long long)p.M * p.N) return;
-  const int m = (int)(i / p.N), n = (int)(i % p.N);
-  float acc = 0.f;
-  for (int z = 0; z < p.splits; ++z) acc += p.partial[((size_t)z * p.M + m) * p.N + n];
-  epi_store<T>(p, m, n, acc);
+__global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) {
+  __shared__ float red[8];
+  const int m = blockIdx.x, tid = threadIdx.x;
+  const int b = m % p.B, r = m / p.B;
+  float ss = 0.f;
+  for (int n = tid; n < p.N; n += 256) {
+    float acc = 0.f;
+    for (int z = 0; z < p.splits; ++z) acc += p.partial[((size_t)z * p.M + m) * p.N + n];
+    float v;
+    if (p.epi == DENSE_RES_X) {
+      v = to_f(reinterpret_cast<const T*>(p.x)[(size_t)b * p.x_bs + (size_t)r * p.x_ts + n]) + p.alpha * acc;
+      p.h[(size_t)m * p.N + n] = v;
+    } else if (p.epi == DENSE_GELU) {
+      v = gelu_exact(acc);
+      reinterpret_cast<T*>(p.out)[(size_t)m * p.N + n] = from_f<T>(v);
+    } else {
+      const T zr = from_f<T>(p.h[(size_t)m * p.N + n] + p.alpha * acc);
+      reinterpret_cast<T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n] = zr;
+      v = to_f(zr);                                              // the next product sees the stored (rounded) z
+    }
+    ss += v * v;
+  }
+  if (!p.norm_out) return;
+  ss = warp_sum(ss);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float rs = p.norm_pre ? rsqrtf(tot / (float)p.N + p.norm_eps) : 1.0f;
+  const T* g = reinterpret_cast<const T*>(p.norm_gain);
+  for (int n = tid; n < p.N; n += 256) {
+    float v;
+    if (p.epi == DENSE_RES_X) v = p.h[(size_t)m * p.N + n];
+    else if (p.epi == DENSE_GELU) v = to_f(reinterpret_cast<const T*>(p.out)[(size_t)m * p.N + n]);
+    else v = to_f(reinterpret_cast<const T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n]);
+    reinterpret_cast<T*>(p.norm_out)[(size_t)m * p.N + n] = from_f<T>(v * rs * (p.norm_pre ? gain_at(g, n) : 1.0f));
+  }
 }
 
 // row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
@@ -312,7 +344,8 @@ static bool make_map_rows(CUtensorMap* map, const void* base, long long rows, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s) {
+cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s, bool* normed) {
+  if (normed) *normed = false;
   if (p.M <= 0) return cudaSuccess;
   const bool strides_ok = p.epi == DENSE_GELU || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
                                                   ((p.epi == DENSE_RES_X ? p.x_ts : p.o_ts) % 8 == 0));
@@ -348,8 +381,8 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       dense_tc_kernel<128><<<grid, kTThreads, smem, s>>>(ma, mw, q, sync);
     }
     if (q.splits > 1) {
-      const long long total = (long long)p.M * p.N;
-      dense_reduce_kernel<__nv_bfloat16><<<(unsigned)((total + 255) / 256), 256, 0, s>>>(q);
+      dense_reduce_kernel<__nv_bfloat16><<<p.M, 256, 0, s>>>(q);
+      if (normed && p.norm_out) *normed = true;
     }
     return cudaGetLastError();
   }

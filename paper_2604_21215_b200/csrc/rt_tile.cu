@@ -151,10 +151,15 @@ __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
   }
   if (lane == 0) { p.st_m[sidx * p.H + h] = m_run; p.st_l[sidx * p.H + h] = l_run; }
   *reinterpret_cast<float2*>(p.st_o + sidx * p.d + h * kHeadDim + 2 * lane) = o;
+  if (p.c_out) {                                               // the row is complete: c = o / l for the output projection
+    const float il = 1.0f / l_run;
+    T* c = reinterpret_cast<T*>(p.c_out) + col;
+    c[0] = from_f<T>(o.x * il); c[1] = from_f<T>(o.y * il);
+  }
 }
 
 cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s) {
-  if (p.k1 <= p.k0) return cudaSuccess;
+  if (p.k1 <= p.k0 && !p.c_out) return cudaSuccess;
   const int blocks = ceil_div(p.B * p.H, 8);
   if (dtype == RT_BF16) row_attn_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(p);
   else row_attn_kernel<float><<<blocks, 256, 0, s>>>(p);
