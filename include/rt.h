@@ -210,8 +210,10 @@ rt_status rt_selftest_wait_expiry(void *workspace, void *cuda_stream);
  * with CUDA events on the caller's stream: class 0 = pre-pass, 1 = leaf recurrence launches,
  * 2 = cross-block tiles, 3 = embedding / head.  rt_profile_read waits for the recorded events
  * (so call it after the work was enqueued), returns the summed milliseconds and the number of
- * bracketed launch groups per class since the last read, and forgets them.  The paper has no
- * counterpart; its latency protocol (Sec. 6, "The setup") times whole layers only. */
+ * bracketed launch groups per class since the last read, and forgets them.  on = 2 additionally makes
+ * CTA 0 of the leaf kernels accumulate per-phase nanoseconds in the workspace's sync area (a diagnostic:
+ * it slows the token step by a few per cent, because every phase waits for the slowest CTA).  The paper
+ * has no counterpart; its latency protocol (Sec. 6, "The setup") times whole layers only. */
 typedef struct { double ms[4]; uint64_t launches[4]; } rt_profile;
 rt_status rt_profile_enable(int32_t on);
 rt_status rt_profile_read(rt_profile *out);

@@ -91,6 +91,7 @@ enum ProfClass { kProfPrepass = 0, kProfLeaf = 1, kProfTile = 2, kProfOther = 3,
 struct ProfSpan { cudaEvent_t a, b; int cls; };
 std::mutex g_prof_mu;
 bool g_prof_on = false;
+bool g_prof_timers = false;      // rt_profile_enable(2): also the in-kernel phase timers of the leaf kernels
 std::vector<ProfSpan> g_prof_spans;
 constexpr size_t kProfMaxSpans = 1u << 20;
 
@@ -228,6 +229,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   lp.ex_z = (float*)(ws + L.ex_z); lp.ex_k = (float*)(ws + L.ex_k);
   lp.ex_part = (float*)(ws + L.ex_part);
   lp.max_chunks = kMaxChunks;
+  lp.timers = g_prof_timers ? 1 : 0;
   lp.sync = (SyncArea*)(ws + L.sync);
 
   auto leaf = [&](int t0, int t1, int attn_begin) -> bool {
@@ -561,6 +563,7 @@ rt_status rt_selftest_wait_expiry(void* workspace, void* cuda_stream) {
 rt_status rt_profile_enable(int32_t on) {
   std::lock_guard<std::mutex> g(g_prof_mu);
   g_prof_on = on != 0;
+  g_prof_timers = on >= 2;
   return RT_OK;
 }
 

@@ -32,6 +32,7 @@ struct LeafParams {
   unsigned bar_base;                             // arrivals counted by earlier launches of the same call (bar_count is
                                                  // zeroed once per API call and only ever grows)
   unsigned seq_base;                             // token steps enqueued before this launch in the same call (flag values)
+  int timers;                                    // 1: CTA 0 accumulates per-phase times in the sync area (costs a few per cent)
   SyncArea* sync;
 };
 

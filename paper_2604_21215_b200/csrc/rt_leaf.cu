@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(kLeafThreads, 1) leaf_kernel(const LeafParams 
   const int n_bg = (B + NB - 1) / NB;
 
   // phase timing by one thread of CTA 0 (two timer reads per phase)
-  const bool timing = (cta == 0 && tid == 0);
+  const bool timing = p.timers && (cta == 0 && tid == 0);
   unsigned long long t_prev = timing ? globaltimer_ns() : 0ull, acc_ns[10];
 #pragma unroll
   for (int i = 0; i < 10; ++i) acc_ns[i] = 0ull;

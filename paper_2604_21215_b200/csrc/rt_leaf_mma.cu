@@ -177,6 +177,7 @@ __device__ __forceinline__ bool mma_grid_barrier(SyncArea* sync, volatile int* s
 }
 
 // ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
+template <bool TIMERS>
 __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsigned char* smem_slot, int pair,
                                const unsigned long long* ll_kv, unsigned long long* ll_c) {
   const int lane = threadIdx.x & 31;
@@ -220,7 +221,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   }
   const unsigned long long* k_words = ll_kv + (size_t)b * (2 * d) + h * kHeadDim + 2 * lane;
   const unsigned long long* v_words = k_words + d;
-  const bool timing = (pair == 0 && lane == 0);
+  const bool timing = TIMERS && (pair == 0 && lane == 0);
   unsigned long long a_work = 0, a_wait = 0, t_mark = timing ? globaltimer_ns() : 0ull;
   for (int j = 0; j < n; ++j) {
     const unsigned seq = p.seq_base + (unsigned)j + 1u;      // step that reveals position t0 + j
@@ -291,7 +292,8 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   if (timing) { atomicAdd(&p.sync->phase_ns[0], a_work); atomicAdd(&p.sync->phase_ns[1], a_wait); }
 }
 
-template <int MB>
+// TIMERS is compile-time: with the per-phase timers compiled in, the kernel is a few per cent slower even when they are off.
+template <int MB, bool TIMERS>
 __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
                                                                       unsigned long long* ll_c, unsigned long long* ll_h,
                                                                       unsigned long long* ll_g, unsigned long long* ll_z,
@@ -337,7 +339,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   if (warp >= kMmaWarps) {
     const int slot = warp - kMmaWarps;
     const int pair = cta + slot * G;
-    if (pair < B * H) attention_role(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
+    if (pair < B * H) attention_role<TIMERS>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
     return;
   }
 
@@ -360,7 +362,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
   const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
   unsigned bar_target = p.bar_base;
-  const bool timing = (cta == 0 && tid == 0);
+  const bool timing = TIMERS && (cta == 0 && tid == 0);
   unsigned long long t_ph = timing ? globaltimer_ns() : 0ull;
 
   for (int t = p.t0; t < p.t1; ++t) {
@@ -663,8 +665,10 @@ bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* o
 
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {
   LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid));
-  const void* fn = p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2>)
-                           : reinterpret_cast<const void*>(&leaf_mma_kernel<1>);
+  const void* fn = p.timers ? (p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2, true>)
+                                       : reinterpret_cast<const void*>(&leaf_mma_kernel<1, true>))
+                            : (p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2, false>)
+                                       : reinterpret_cast<const void*>(&leaf_mma_kernel<1, false>));
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
   if (e != cudaSuccess) return e;
   LeafParams pp = p;

@@ -187,8 +187,9 @@ def rt_plan_tiles(N: int, leaf: int) -> List[tuple]:
     return [tuple(buf[4 * i:4 * i + 4]) for i in range(n)]
 
 
-def rt_profile_enable(on: bool) -> None:
-    _check(_lib.rt_profile_enable(1 if on else 0), "rt_profile_enable")
+def rt_profile_enable(on) -> None:
+    """False/0: off; True/1: event spans per kernel class; 2: also the leaf kernels' in-kernel phase timers."""
+    _check(_lib.rt_profile_enable(int(on)), "rt_profile_enable")
 
 
 def rt_profile_read() -> Dict[str, Dict[str, float]]:
