@@ -292,8 +292,9 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   if (timing) { atomicAdd(&p.sync->phase_ns[0], a_work); atomicAdd(&p.sync->phase_ns[1], a_wait); }
 }
 
-// TIMERS is compile-time: with the per-phase timers compiled in, the kernel is a few per cent slower even when they are off.
-template <int MB, bool TIMERS>
+// TIMERS and GAINS are compile-time: the token step is a latency chain of code that runs once per token, and every
+// instruction and live register that is compiled in costs time even when its branch is not taken.
+template <int MB, bool TIMERS, bool GAINS>
 __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
                                                                       unsigned long long* ll_c, unsigned long long* ll_h,
                                                                       unsigned long long* ll_g, unsigned long long* ll_z,
@@ -383,9 +384,9 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
       const unsigned long long* act_ll = (ph == 0) ? ll_c : ((ph == 1) ? ll_h : ll_z);
       const __nv_bfloat16* gain = nullptr;
       bool want_ssq = false;
-      if (ph == 1 && pre) { gain = reinterpret_cast<const __nv_bfloat16*>(p.g_mlp); want_ssq = true; }
-      if (ph == 3 && kv_norm) { gain = reinterpret_cast<const __nv_bfloat16*>(p.g_kv); want_ssq = true; }
-      const __nv_bfloat16* gp = gain ? gain + 4 * c : nullptr;
+      if (ph == 1 && pre) { if (GAINS) gain = reinterpret_cast<const __nv_bfloat16*>(p.g_mlp); want_ssq = true; }
+      if (ph == 3 && kv_norm) { if (GAINS) gain = reinterpret_cast<const __nv_bfloat16*>(p.g_kv); want_ssq = true; }
+      const __nv_bfloat16* gp = (GAINS && gain) ? gain + 4 * c : nullptr;
       unsigned long long wait_ns = 0;
       if (ph == 2) {
         // every CTA's slice of g (packed bf16) must be complete before anyone multiplies by W_down
@@ -525,10 +526,10 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
             if (timing) wait_ns += globaltimer_ns() - t_poll;
             TL(2);
           }
-          const __nv_bfloat16* gc = gp ? gp + (size_t)kc0 * 16 : nullptr;
+          const __nv_bfloat16* gc = (GAINS && gp) ? gp + (size_t)kc0 * 16 : nullptr;
           if (want_ssq) {
 #pragma unroll
-            for (int i = 0; i < KC; ++i) frag_ssq_gain<MB>(a[i], gc ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0, sq1);
+            for (int i = 0; i < KC; ++i) frag_ssq_gain<MB>(a[i], (GAINS && gc) ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0, sq1);
           }
           // products, specialised on the number of tiles so that none sits behind a branch
           auto products = [&](auto ntc) {
@@ -665,10 +666,16 @@ bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* o
 
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {
   LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid));
-  const void* fn = p.timers ? (p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2, true>)
-                                       : reinterpret_cast<const void*>(&leaf_mma_kernel<1, true>))
-                            : (p.B > 8 ? reinterpret_cast<const void*>(&leaf_mma_kernel<2, false>)
-                                       : reinterpret_cast<const void*>(&leaf_mma_kernel<1, false>));
+  // compile-time variants: row blocks (B > 8), per-phase timers, RMS gains present
+  const bool gains = p.g_mlp != nullptr || p.g_kv != nullptr;
+  auto pick = [&](auto mb) -> const void* {
+    constexpr int MB = decltype(mb)::value;
+    if (p.timers) return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, true>)
+                               : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, false>);
+    return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, true>)
+                 : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, false>);
+  };
+  const void* fn = p.B > 8 ? pick(std::integral_constant<int, 2>{}) : pick(std::integral_constant<int, 1>{});
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
   if (e != cudaSuccess) return e;
   LeafParams pp = p;
