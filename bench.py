@@ -40,7 +40,7 @@ def measured_peaks():
 
 # DRAM bytes (read + write) of one leaf launch (64 token steps) from the ncu capture summarised in
 # profiles/leaf_mma_kernel_c2.txt: the launch stages its weight rows once, everything else stays in L2.
-NCU_LEAF_TRAFFIC = {"c2": 14702848 + 48384}
+NCU_LEAF_TRAFFIC = {"c2": 14701056 + 28416}
 
 
 class ClockSampler:
