@@ -340,3 +340,37 @@ def test_wide_batch_unsupported_paths_say_so():
     with pytest.raises(rt.RtError) as ei:
         layer.prefill(data["x"])
     assert ei.value.status == rt.RT_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("gains", [False, True])
+def test_phase_timer_variants_compute_the_same(gains):
+    # rt_profile_enable(2) selects the leaf-kernel variants with the per-phase timers compiled in; they must
+    # give the same output bit for bit and leave non-zero phase times in the workspace's sync area.
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    d, H, dff, B, N = 256, 4, 1024, 3, 150
+    wl = inputs.Workload("timers", 1, B, N, d, H, dff, "bf16")
+    data = inputs.make_inputs(wl, seed=8600)
+    lw = data["layers"][0]
+    if gains:
+        rng = np.random.default_rng(5)
+        for g in ("g_attn", "g_mlp", "g_kv", "g_q", "g_k"):
+            lw[g] = inputs.round_to(1.0 + 0.2 * rng.standard_normal(d), "bf16")
+    layer = _layer(d, H, dff, "bf16", lw)
+    xd = torch.from_numpy(data["x"]).to(torch.bfloat16).cuda()
+    layer.reserve(B, N)
+    outs = []
+    try:
+        for mode in (0, 2):
+            rt.rt_profile_enable(mode)
+            zd = torch.empty_like(xd)
+            layer.prefill_device(xd, zd)
+            torch.cuda.synchronize()
+            assert layer.status() == 0
+            phase_ns = layer.ws[:256].cpu().numpy().view(np.uint64)[2:12]
+            outs.append((zd.clone(), layer.k_cache.clone(), int(phase_ns.sum())))
+    finally:
+        rt.rt_profile_enable(0)
+        rt.rt_profile_read()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert outs[0][2] == 0 and outs[1][2] > 0
