@@ -314,7 +314,8 @@ def test_alibi_stack_prefill_and_decode_match_oracle(dtype):
 
 @pytest.mark.parametrize("dtype,d,H,dff,B,N,leaf,alibi", [
     ("f32", 128, 2, 256, 70, 40, 16, False), ("bf16", 256, 4, 1024, 130, 75, 32, True),
-    ("bf16", 128, 2, 512, 96, 33, 16, False), ("bf16", 256, 4, 768, 40, 50, 0, False)])
+    ("bf16", 128, 2, 512, 96, 33, 16, False), ("bf16", 256, 4, 768, 40, 50, 0, False),
+    ("bf16", 192, 3, 208, 30, 40, 16, True)])
 def test_wide_batch_prefill_matches_oracle(dtype, d, H, dff, B, N, leaf, alibi):
     # B > 64 (bf16: B >= 24): every token step runs as dense products over the B rows (tensor cores for bf16)
     from oracle import RTConfig, RTWeights, layer_seq
