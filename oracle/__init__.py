@@ -6,6 +6,6 @@ It shares no code with the CUDA path.
 """
 from .rt_oracle import (  # noqa: F401
     RTConfig, RTWeights, rms, qk_rms, gelu, attn,
-    layer_seq, layer_blk, layer_fixed_point, layer_decode,
+    layer_seq, layer_blk, layer_fixed_point, layer_decode, layer_blockrec,
     stack_prefill, stack_decode, alg1_tiles, update_tile,
 )

@@ -311,6 +311,35 @@ def layer_fixed_point(cfg: RTConfig, w: RTWeights, x: np.ndarray, z_claim: np.nd
     return z2, k, v
 
 
+
+# ----------------------------------------------------------------------------- blocked recurrence
+
+def layer_blockrec(cfg: RTConfig, w: RTWeights, x: np.ndarray, S: int):
+    """Recurrence executed over blocks of S positions (Sec. 9 names this extension in one sentence and does not
+    define it; the reading taken here): positions are grouped in consecutive blocks of S.  Position i attends
+    to the PERSISTENT pairs (Eqs. 1-2, from the outputs z_j) of every position j in an earlier block and to the
+    TEMPORARY pairs (from the inputs x_j, first display of Sec. 2.2) of the positions j <= i of its own block, so
+    all positions of a block can be computed at once; the block's persistent pairs follow from its outputs.
+    S = 1 is the layer of Sec. 2.2; S >= N is an ordinary pre-LN Transformer layer.  With ALiBi slopes the
+    distance i - j applies to both kinds of pair.  Returns z, k, v like layer_seq."""
+    x = np.asarray(x, dtype=np.float64)
+    B, N, d = x.shape
+    H, dh, s = cfg.n_heads, cfg.head_dim, cfg.softmax_scale
+    z = np.zeros_like(x); k = np.zeros_like(x); v = np.zeros_like(x)
+    q, kt, vt = _temp_qkv(x, w, cfg)
+    for b in range(B):
+        for i in range(N):
+            blk = (i // S) * S                                   # first position of i's block
+            c = np.zeros(d)
+            for h in range(H):
+                sl = slice(h * dh, (h + 1) * dh)
+                keys = np.concatenate([k[b, :blk, sl], kt[b, blk:i + 1, sl]])
+                vals = np.concatenate([v[b, :blk, sl], vt[b, blk:i + 1, sl]])
+                bias = None if cfg.alibi_slopes is None else -cfg.slope(h) * (i - np.arange(i + 1))
+                c[sl] = attn(keys, vals, q[b, i, sl], s, bias)
+            z[b, i], k[b, i], v[b, i] = _output_and_persistent(x[b, i], c @ w.w_o.T, w, cfg)
+    return z, k, v
+
 # ----------------------------------------------------------------------------- O-dec
 
 def layer_decode(cfg: RTConfig, w: RTWeights, x_new: np.ndarray, k_cache: np.ndarray,
