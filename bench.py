@@ -114,15 +114,17 @@ def config_dict(wl, sched, extra=None):
 
 # ------------------------------------------------------------------------------------ oracle arm
 
-def oracle_sample(wl, data, n_pos):
+def oracle_sample(wl, data, n_pos, recur_block=0):
     """Runs the oracle, as it stands, on the first n_pos positions of the workload; returns seconds."""
-    from oracle import RTConfig, RTWeights, layer_seq, stack_prefill
+    from oracle import RTConfig, RTWeights, layer_blockrec, layer_seq, stack_prefill
     cfg = RTConfig(wl.d_model, wl.n_heads, wl.head_dim, wl.d_ff, residual_scale=wl.residual_scale,
                    alibi_slopes=data["layers"][0].get("alibi_slopes"))
     layers = [RTWeights(**{k: v for k, v in lw.items() if k != "alibi_slopes"}) for lw in data["layers"]]
     t0 = time.perf_counter()
     if wl.vocab:
         stack_prefill(cfg, layers, data["emb"], None, data["ids"][:, :n_pos])
+    elif recur_block > 1:
+        layer_blockrec(cfg, layers[0], data["x"][:, :n_pos], recur_block)
     else:
         layer_seq(cfg, layers[0], data["x"][:, :n_pos])
     return time.perf_counter() - t0
@@ -193,6 +195,8 @@ def run_cuda(args):
     data = inputs.make_inputs(wl)
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     leaf_kw = {"leaf": args.leaf} if args.leaf else {}
+    if args.recur_block > 1:
+        leaf_kw["recur_block"] = args.recur_block
     stream = torch.cuda.current_stream(dev)
 
     if args.alibi:                                     # the same slopes for every layer
@@ -324,10 +328,23 @@ def run_cuda(args):
                         "us_per_token_step": 1e3 * ms_all / max(wl.N * wl.n_layers * args.steps, 1),
                         "note": "M = B rows per product: each token step is ten short dependent launches, so launch latency "
                                 "and the L2 stream of the weights, not the tensor pipe, set the time"}
+        if args.recur_block > 1:
+            # recurrence over blocks: every block is a parallel sweep of dense products and attention tiles
+            tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))).get("bf16_tflops_sustained", 1403.5)) \
+                if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else 1400.0
+            tok_all = B * wl.N * wl.n_layers * args.steps
+            flops = 2.0 * tok_all * (5 * d * d + 2 * d * f) + 6.0 * tok_all * d * d + 2.0 * B * d * wl.N * (wl.N - 1) * wl.n_layers * args.steps
+            ms_all = prof["leaf"]["ms"] + prof["tile"]["ms"] + prof["prepass"]["ms"]
+            achieved = flops / (ms_all * 1e-3) / 1e12 if ms_all > 0 else 0.0
+            roofline = {"kernel": "dense_tc_kernel + tile_tc_kernel (recurrence over blocks)", "bound": "tensor",
+                        "achieved": achieved, "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak,
+                        "peak_source": "measured (sustained)", "traffic": None,
+                        "us_per_token_step": 1e3 * ms_all / max(wl.N * wl.n_layers * args.steps, 1),
+                        "note": "all products of a call (projections, chain, attention) over the summed kernel time"}
         tile_ms = prof["tile"]["ms"]
         tile_tflops = (counters["flops_tile"] * args.steps / (tile_ms * 1e-3) / 1e12) if tile_ms > 0 else None
         n_pos = sample_positions(wl)
-        t_cpu = oracle_sample(wl, data, n_pos)
+        t_cpu = oracle_sample(wl, data, n_pos, args.recur_block)
         cpu = {"value": wl.B * n_pos / t_cpu, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle",
                "sample": f"first {n_pos} of {wl.N} positions, all {wl.B} sequences, one run ({t_cpu:.1f} s)"}
         launches = sum(v["launches"] for v in prof.values())
@@ -347,7 +364,7 @@ def run_cuda(args):
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16/f32-accumulate" if wl.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": config_dict(wl, args.sched, {"alibi": bool(args.alibi), "leaf": int(model.cfg.leaf) or (32 if wl.B > 64 else 64),
+                "data": "synthetic", "config": config_dict(wl, args.sched, {"alibi": bool(args.alibi), "recur_block": int(args.recur_block), "leaf": int(model.cfg.leaf) or (32 if wl.B > 64 else 64),
                                                                             "parallelism": f"replicas x{world}"}),
                 "clocks": clocks,
                 "e2e": {"value": replicas.aggregate_tokens_per_s(tokens, args.steps, world, e2e_total), "unit": UNIT,
@@ -557,6 +574,8 @@ def main():
                     help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
     ap.add_argument("--tile-bench", action="store_true", help="time Algorithm 2 alone per tile size and exit")
     ap.add_argument("--tile-bench-all", action="store_true", help="with --tile-bench: also sizes beyond N/2")
+    ap.add_argument("--recur-block", type=int, default=0,
+                    help="recurrence over blocks of this many positions (config.recur_block); 0 = the layer as defined")
     ap.add_argument("--alibi", action="store_true",
                     help="add ALiBi distances (slopes 2^(-8 h / H), h = 1..H) to the attention logits")
     ap.add_argument("--recompute-bench", action="store_true",

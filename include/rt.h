@@ -70,6 +70,11 @@ typedef struct {
   float rms_eps;            /* added to the mean square inside the root (the paper gives none; 1e-6) */
   float softmax_scale;      /* logits = scale * <q, k>.  Sec. 2's Attn has scale 1; 1/sqrt(head_dim) is customary */
   float residual_scale;     /* alpha = 1/sqrt(L) of Sec. 2; 1 for a single layer */
+  int32_t recur_block;      /* 0 or 1: the layer of Sec. 2.2.  S > 1: recurrence over blocks of S positions (Sec. 9 names this
+                               extension without defining it; the reading taken: position i attends to the persistent pairs
+                               of all positions in earlier blocks and to the temporary pairs of the positions j <= i of its own
+                               block, so a block is computed in one parallel sweep; S >= N is an ordinary pre-LN Transformer
+                               layer).  Prefill entry points only, tiled schedule; decode returns RT_ERR_UNSUPPORTED */
 } rt_config;
 
 typedef struct {            /* device pointers; read-only */

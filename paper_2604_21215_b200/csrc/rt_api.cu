@@ -17,7 +17,8 @@ constexpr int kMaxChunks = 32;
 constexpr int kAutoLeaf = 64;
 
 struct WsLayout {
-  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, ll, ll_bytes, hid0, hid1, total;
+  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, ll, ll_bytes, hid0, hid1,
+      blk_h, blk_u, blk_c, blk_g, total;
 };
 
 size_t esize_of(int dtype) { return dtype == RT_BF16 ? 2 : 4; }
@@ -31,6 +32,7 @@ bool config_ok(const rt_config* c) {
   if (c->leaf != 0 && (c->leaf < 16 || c->leaf > 256 || (c->leaf & (c->leaf - 1)))) return false;
   if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
   if (c->norm_flags & ~15) return false;
+  if (c->recur_block < 0) return false;
   return true;
 }
 
@@ -69,6 +71,15 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ll = take(L.ll_bytes);
   L.hid0 = take(tok * d * e);
   L.hid1 = take(tok * d * e);
+  // recurrence over blocks: the position-wise chain of one block (rows = block length x B)
+  L.blk_h = L.blk_u = L.blk_c = L.blk_g = 0;
+  if (c->recur_block > 1) {
+    const size_t rows = (size_t)B * (c->recur_block < N ? c->recur_block : N);
+    L.blk_h = take(rows * d * 4);
+    L.blk_u = take(rows * d * e);
+    L.blk_c = take(rows * d * e);
+    L.blk_g = take(rows * f * e);
+  }
   L.total = o;
   return L;
 }
@@ -137,6 +148,90 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   {
     ProfScope ps(s, kProfPrepass);
     if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
+  }
+
+  if (c->recur_block > 1) {
+    // Recurrence over blocks of S positions: a block is one parallel sweep (in-block causal attention over the
+    // TEMPORARY pairs, the position-wise chain as dense products over the block's rows, then its persistent pairs),
+    // and blocks follow each other with Algorithm 1's cross tiles at block granularity.
+    if (c->sched != RT_SCHED_TILED || pos0 != 0) return RT_ERR_UNSUPPORTED;
+    const int S = c->recur_block, N = n_rows;
+    const long long d = c->d_model, f = c->d_ff;
+    const size_t e = esize_of(c->dtype);
+    SyncArea* sync = (SyncArea*)(ws + L.sync);
+    const bool pre = (c->norm_flags & RT_NORM_PRE) != 0;
+    TileParams tp;
+    memset(&tp, 0, sizeof(tp));
+    tp.B = B; tp.d = c->d_model; tp.H = c->n_heads; tp.scale_log2 = scale_log2; tp.alibi = w->alibi_slopes;
+    tp.q = ws + L.q; tp.st_o = pp.st_o; tp.st_m = pp.st_m; tp.st_l = pp.st_l;
+    tp.rows_q = n_rows; tp.sync = sync;
+    PrepassParams pk = pp;                                      // persistent pairs of a block from its outputs
+    pk.x_bs = z_bs; pk.x_ts = z_ts;
+    pk.norm_flags = (c->norm_flags & RT_NORM_SKIP_Z) ? (c->norm_flags & ~RT_NORM_PRE) : c->norm_flags;
+    pk.g_attn = w->g_kv ? w->g_kv : w->g_attn;
+    pk.mats = 6; pk.no_seed = 1;
+    DenseParams dp;
+    memset(&dp, 0, sizeof(dp));
+    dp.B = B; dp.alpha = c->residual_scale; dp.h = (float*)(ws + L.blk_h);
+    const int Lb = c->dtype == RT_BF16 ? 2 * kAutoLeaf : kAutoLeaf;
+    for (int s0 = 0; s0 < N; s0 += S) {
+      const int e0 = s0 + S < N ? s0 + S : N, rows = e0 - s0;
+      {
+        // 1. in-block attention over the temporary pairs of strictly earlier positions (the pair of the position
+        //    itself is in the seeded state): causal diagonal blocks, then the levels inside the block
+        ProfScope ps(s, kProfTile);
+        tp.k_cache = ws + L.kt; tp.v_cache = ws + L.vt; tp.rows_kv = n_rows; tp.q_limit = e0;
+        const int full = rows / Lb;
+        tp.causal = 1;
+        if (full > 0) {
+          tp.q0 = s0; tp.q1 = s0 + Lb; tp.k0 = s0; tp.k1 = s0 + Lb; tp.batch = full; tp.batch_stride = Lb;
+          if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+        }
+        if (full * Lb < rows) {
+          tp.q0 = s0 + full * Lb; tp.q1 = e0; tp.k0 = tp.q0; tp.k1 = e0; tp.batch = 1; tp.batch_stride = 0;
+          if (tile_simt_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+        }
+        tp.causal = 0;
+        for (long long P = Lb; P < rows; P *= 2) {
+          tp.q0 = s0 + (int)P; tp.q1 = s0 + (int)(2 * P); tp.k0 = s0; tp.k1 = s0 + (int)P;
+          tp.batch = (int)((rows - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
+          if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+        }
+        tp.batch = 0; tp.batch_stride = 0; tp.q_limit = 0;
+      }
+      {
+        // 2. position-wise chain over the block's rows, 3. its persistent pairs
+        ProfScope ps(s, kProfLeaf);
+        const size_t row = (size_t)s0 * B;
+        void* cbuf = ws + L.blk_c; void* ubuf = ws + L.blk_u; void* gbuf = ws + L.blk_g;
+        if (attn_value_launch(c->dtype, pp.st_o + row * d, pp.st_l + row * c->n_heads, cbuf, (long long)rows * B, (int)d, c->n_heads, s) != cudaSuccess)
+          return RT_ERR_CUDA;
+        dp.M = rows * B;
+        dp.N = (int)d; dp.K = (int)d; dp.A = cbuf; dp.W = w->w_o; dp.epi = DENSE_RES_X;
+        dp.x = (const unsigned char*)x + (size_t)s0 * x_ts * e; dp.x_bs = x_bs; dp.x_ts = x_ts;
+        if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+        if (rms_rows_f32_launch(c->dtype, dp.h, w->g_mlp, ubuf, rows * B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess) return RT_ERR_CUDA;
+        dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;
+        if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+        dp.N = (int)d; dp.K = (int)f; dp.A = gbuf; dp.W = w->w_down; dp.epi = DENSE_RES_H;
+        dp.out = (unsigned char*)z + (size_t)s0 * z_ts * e; dp.o_bs = z_bs; dp.o_ts = z_ts;
+        if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
+        pk.N = rows;
+        pk.x = (const unsigned char*)z + (size_t)s0 * z_ts * e;
+        pk.kt = (unsigned char*)k_cache + row * d * e; pk.vt = (unsigned char*)v_cache + row * d * e;
+        if (prepass_launch(c->dtype, pk, s) != cudaSuccess) return RT_ERR_CUDA;
+      }
+      if (e0 < N) {
+        // 4. Algorithm 1 at block granularity: the next P positions attend to the last P persistent pairs
+        const int u = e0 / S;
+        const long long P = (long long)S * (u & -u);
+        tp.k_cache = k_cache; tp.v_cache = v_cache; tp.rows_kv = n_max;
+        tp.q0 = e0; tp.q1 = e0 + P < N ? (int)(e0 + P) : N; tp.k0 = (int)(e0 - P); tp.k1 = e0;
+        ProfScope ps(s, kProfTile);
+        if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+      }
+    }
+    return RT_OK;
   }
 
   // bf16 batches the persistent tensor-core leaf kernel does not take (B > 16) are faster as dense products from
@@ -334,6 +429,7 @@ rt_status rt_layer_recompute(const rt_config* cfg, const rt_layer_weights* w, co
   if (!config_ok(cfg) || B <= 0 || N <= 0 || !workspace || !aligned16(workspace)) return RT_ERR_INVALID_ARG;
   rt_status st = config_supported(cfg, 1);
   if (st != RT_OK) return st;
+  if (cfg->recur_block > 1) return RT_ERR_UNSUPPORTED;          // the sweep is the fixed-point map of the layer of Sec. 2.2
   if (workspace_bytes < rt_recompute_workspace_bytes(cfg, B, N)) return RT_ERR_WORKSPACE;
   if (!weights_ok(w) || !x || !z_claim || !z_out || !k_cache || !v_cache || z_out == x || z_out == z_claim || N_max < N)
     return RT_ERR_INVALID_ARG;

@@ -375,3 +375,42 @@ def test_phase_timer_variants_compute_the_same(gains):
         rt.rt_profile_read()
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
     assert outs[0][2] == 0 and outs[1][2] > 0
+
+
+# ---------------------------------------------------------------- recurrence over blocks of positions (config.recur_block)
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N,S,alibi", [
+    ("f32", 128, 2, 256, 2, 70, 16, False), ("f32", 128, 2, 256, 3, 50, 7, True), ("f32", 128, 2, 512, 2, 40, 64, False),
+    ("bf16", 256, 4, 1024, 3, 300, 64, False), ("bf16", 256, 4, 1024, 2, 520, 256, True), ("bf16", 768, 12, 3072, 2, 200, 32, False),
+    ("bf16", 128, 2, 512, 70, 48, 16, False)])
+def test_blocked_recurrence_matches_oracle(dtype, d, H, dff, B, N, S, alibi):
+    from oracle import RTConfig, RTWeights, layer_blockrec, layer_seq
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("blockrec", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=8700 + N + S)
+    lw = data["layers"][0]
+    slopes = _slopes(H) if alibi else None
+    cfg = RTConfig(d, H, 64, dff, alibi_slopes=slopes, residual_scale=0.8)
+    ref = layer_blockrec(cfg, RTWeights(**lw), data["x"], S)
+    if S < N:
+        assert rel_err(layer_seq(cfg, RTWeights(**lw), data["x"])[0], ref[0]) > 10 * TOL[dtype]    # a different model
+    layer = _layer(d, H, dff, dtype, dict(lw, alibi_slopes=slopes) if alibi else lw, residual_scale=0.8, recur_block=S)
+    got = layer.prefill(data["x"])
+    for name, g_, r_ in zip(("z", "k", "v"), got, ref):
+        assert np.isfinite(g_).all(), name
+        assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
+
+
+def test_blocked_recurrence_unsupported_paths_say_so():
+    from paper_2604_21215_b200 import inputs, rt
+    d, H, dff, B, N = 128, 2, 256, 2, 20
+    wl = inputs.Workload("blockrec", 1, B, N, d, H, dff, "f32")
+    data = inputs.make_inputs(wl, seed=2)
+    layer = _layer(d, H, dff, "f32", data["layers"][0], recur_block=8)
+    layer.prefill(data["x"][:, :16], N_max=N)
+    with pytest.raises(rt.RtError) as ei:
+        layer.decode(data["x"][:, 16], 16)
+    assert ei.value.status == rt.RT_ERR_UNSUPPORTED
+    with pytest.raises(rt.RtError) as ei:
+        layer.recompute(data["x"], data["x"])
+    assert ei.value.status == rt.RT_ERR_UNSUPPORTED
