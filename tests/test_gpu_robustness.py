@@ -414,3 +414,21 @@ def test_blocked_recurrence_unsupported_paths_say_so():
     with pytest.raises(rt.RtError) as ei:
         layer.recompute(data["x"], data["x"])
     assert ei.value.status == rt.RT_ERR_UNSUPPORTED
+
+
+def test_blocked_recurrence_stack_matches_oracle():
+    # the stack entry point with recur_block: embedding, L blocked layers, final norm and tied head
+    from oracle import RTConfig, RTWeights, layer_blockrec, rms
+    from paper_2604_21215_b200 import inputs, rt
+    L, d, H, dff, V, B, N, S = 2, 128, 2, 256, 200, 2, 60, 16
+    wl = inputs.Workload("blockrec_stack", L, B, N, d, H, dff, "f32", vocab=V, residual_scale=1 / np.sqrt(L))
+    data = inputs.make_inputs(wl, seed=8800)
+    cfg = RTConfig(d, H, 64, dff, residual_scale=wl.residual_scale)
+    x = np.asarray(data["emb"], dtype=np.float64)[np.asarray(data["ids"])]
+    for lw in data["layers"]:
+        x, _, _ = layer_blockrec(cfg, RTWeights(**lw), x, S)
+    logits_ref = rms(x[:, -1], np.ones(d), cfg.rms_eps) @ np.asarray(data["emb"], dtype=np.float64).T
+    st = rt.Stack(L, d, H, dff, V, dtype="f32", residual_scale=wl.residual_scale, recur_block=S)
+    st.set_weights(data["layers"], data["emb"])
+    hid, logits = st.prefill(data["ids"])
+    assert rel_err(hid, x) <= TOL["f32"] and rel_err(logits, logits_ref) <= TOL["f32"]
