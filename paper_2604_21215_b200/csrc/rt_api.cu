@@ -169,9 +169,10 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     pk.x_bs = z_bs; pk.x_ts = z_ts;
     pk.norm_flags = (c->norm_flags & RT_NORM_SKIP_Z) ? (c->norm_flags & ~RT_NORM_PRE) : c->norm_flags;
     pk.g_attn = w->g_kv ? w->g_kv : w->g_attn;
-    pk.mats = 6; pk.no_seed = 1;
+    pk.mats = 6; pk.no_seed = 1; pk.chained = 1;              // the chain of a block: programmatic dependent launches
     DenseParams dp;
     memset(&dp, 0, sizeof(dp));
+    dp.chained = 1;
     dp.B = B; dp.alpha = c->residual_scale; dp.h = (float*)(ws + L.blk_h);
     const int Lb = c->dtype == RT_BF16 ? 2 * kAutoLeaf : kAutoLeaf;
     for (int s0 = 0; s0 < N; s0 += S) {
@@ -204,13 +205,13 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
         ProfScope ps(s, kProfLeaf);
         const size_t row = (size_t)s0 * B;
         void* cbuf = ws + L.blk_c; void* ubuf = ws + L.blk_u; void* gbuf = ws + L.blk_g;
-        if (attn_value_launch(c->dtype, pp.st_o + row * d, pp.st_l + row * c->n_heads, cbuf, (long long)rows * B, (int)d, c->n_heads, s) != cudaSuccess)
+        if (attn_value_launch(c->dtype, pp.st_o + row * d, pp.st_l + row * c->n_heads, cbuf, (long long)rows * B, (int)d, c->n_heads, s, true) != cudaSuccess)
           return RT_ERR_CUDA;
         dp.M = rows * B;
         dp.N = (int)d; dp.K = (int)d; dp.A = cbuf; dp.W = w->w_o; dp.epi = DENSE_RES_X;
         dp.x = (const unsigned char*)x + (size_t)s0 * x_ts * e; dp.x_bs = x_bs; dp.x_ts = x_ts;
         if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
-        if (rms_rows_f32_launch(c->dtype, dp.h, w->g_mlp, ubuf, rows * B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess) return RT_ERR_CUDA;
+        if (rms_rows_f32_launch(c->dtype, dp.h, w->g_mlp, ubuf, rows * B, (int)d, c->rms_eps, pre ? 1 : 0, s, true) != cudaSuccess) return RT_ERR_CUDA;
         dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;
         if (dense_launch(c->dtype, dp, sync, s) != cudaSuccess) return RT_ERR_CUDA;
         dp.N = (int)d; dp.K = (int)f; dp.A = gbuf; dp.W = w->w_down; dp.epi = DENSE_RES_H;
@@ -263,8 +264,12 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     pk.norm_flags = (c->norm_flags & RT_NORM_SKIP_Z) ? (c->norm_flags & ~RT_NORM_PRE) : c->norm_flags;
     pk.g_attn = w->g_kv ? w->g_kv : w->g_attn;
     pk.mats = 6; pk.no_seed = 1;
+    // the seven launches of a token step are short and strictly dependent: chained (programmatic dependent
+    // launches), each is scheduled while its predecessor drains
+    pk.chained = 1; tp.chained = 1;
     DenseParams dp;
     memset(&dp, 0, sizeof(dp));
+    dp.chained = 1;
     dp.M = B; dp.B = B; dp.alpha = c->residual_scale; dp.h = hbuf;
     dp.partial = (float*)(ws + L.ex_part); dp.partial_bytes = (size_t)B * c->n_heads * kMaxChunks * 68 * 4;
     // in-leaf attention re-reads the leaf's pairs for every position (leaf^2 * B * d bytes per leaf), so wide
@@ -285,7 +290,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
           dp.x = (const unsigned char*)x + (size_t)t * x_ts * e; dp.x_bs = x_bs; dp.x_ts = 0;
           dp.norm_out = ubuf; dp.norm_gain = w->g_mlp; dp.norm_eps = c->rms_eps; dp.norm_pre = pre ? 1 : 0;   // u = RMS(h)
           if (dense_launch(c->dtype, dp, sync, s, &normed) != cudaSuccess) return RT_ERR_CUDA;
-          if (!normed && rms_rows_f32_launch(c->dtype, hbuf, w->g_mlp, ubuf, B, (int)d, c->rms_eps, pre ? 1 : 0, s) != cudaSuccess)
+          if (!normed && rms_rows_f32_launch(c->dtype, hbuf, w->g_mlp, ubuf, B, (int)d, c->rms_eps, pre ? 1 : 0, s, true) != cudaSuccess)
             return RT_ERR_CUDA;
           dp.norm_out = nullptr;
           dp.N = (int)f; dp.K = (int)d; dp.A = ubuf; dp.W = w->w_up; dp.epi = DENSE_GELU; dp.out = gbuf;

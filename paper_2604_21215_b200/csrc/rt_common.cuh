@@ -1,5 +1,6 @@
 // Shared device helpers of the RT prefill kernels (sm_100a).
 #pragma once
+#include <utility>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -140,5 +141,27 @@ __device__ __forceinline__ bool grid_barrier(SyncArea* s, unsigned& target, unsi
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// A kernel launched with launch_chained(..., true) may be scheduled while its predecessor in the stream is still
+// running; it must call grid_dep_sync() before it reads or writes anything the predecessor touches, in every CTA and
+// before any early return (a grid whose CTAs left without waiting would count as finished too early for ITS
+// successor).  Launched the ordinary way, both calls do nothing.
+__device__ __forceinline__ void grid_dep_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // let the successor be scheduled behind us
+  asm volatile("griddepcontrol.wait;" ::: "memory");                   // until the predecessor's writes are visible
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool chained,
+                                  Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = chained ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 }  // namespace rt

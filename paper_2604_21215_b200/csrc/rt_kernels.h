@@ -66,6 +66,7 @@ struct PrepassParams {
   int mats;                                      // which projections to compute: bit 0 q, bit 1 k, bit 2 v (0 = all three)
   int no_seed;                                   // 1: leave the running stats alone (projection only)
   int skip_rms;                                  // 1: `n` already holds the normalised rows
+  int chained;                                   // 1: launch the projection as a programmatic dependent launch
   SyncArea* sync;
 };
 cudaError_t prepass_launch(int dtype, const PrepassParams& p, cudaStream_t s);
@@ -85,6 +86,7 @@ struct TileParams {
   int batch, batch_stride, q_limit;              // batch > 1: blockIdx.z-th copy of the tile, shifted by z * batch_stride rows
                                                  // (one level of Algorithm 1 in one launch); q_limit > 0 clips the queries
   int causal;                                    // 1: only pairs with key position < query position
+  int chained;                                   // row_attn only: launch as a programmatic dependent launch
   void* c_out;                                   // row_attn only: also write the attention value o/l of the row, [B, d] storage type
   int rows_q, rows_kv;                           // rows held by the query buffer / the caches (tensor-map bounds)
   SyncArea* sync;
@@ -115,12 +117,15 @@ struct DenseParams {
   void* out; long long o_bs, o_ts;               // DENSE_GELU: [M, N];  DENSE_RES_H: out[b, r, :]
   float* partial; size_t partial_bytes;          // optional scratch for a split contraction (few rows): [splits, M, N] fp32
   int splits;                                    // set by the launcher
+  int chained;                                   // 1: launch the product (and its reduction) as programmatic dependent launches
   // optional: also write RMS_g(row) of the epilogue's result (h or z) for the next product.  Only a split
   // contraction does this (its reduction kernel owns whole rows); `normed` tells the caller whether it happened.
   void* norm_out; const void* norm_gain; float norm_eps; int norm_pre;
 };
 cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s, bool* normed = nullptr);
-cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s);
-cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s);
+cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s,
+                              bool chained = false);
+cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s,
+                                bool chained = false);
 
 }  // namespace rt

@@ -15,6 +15,7 @@ namespace rt {
 // ---- n = RMS(x) (or a copy when pre-norm is off), position-major rows m = r*B + b ----------
 template <typename T>
 __global__ void rms_rows_kernel(const PrepassParams p) {
+  grid_dep_sync();
   const int lane = threadIdx.x & 31;
   const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (m >= p.N * p.B) return;
@@ -136,7 +137,10 @@ __global__ void state_init_kernel(const PrepassParams p) {
 template <typename T>
 static cudaError_t prepass_typed(const PrepassParams& p, cudaStream_t s) {
   const int M = p.N * p.B;
-  if (!p.skip_rms) rms_rows_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(p);
+  if (!p.skip_rms) {
+    const cudaError_t e = launch_chained(rms_rows_kernel<T>, dim3(ceil_div(M, 8)), dim3(256), 0, s, p.chained != 0, p);
+    if (e != cudaSuccess) return e;
+  }
   if (sizeof(T) == 2 && qkv_gemm_tc_supported(p)) {
     const cudaError_t e = qkv_gemm_tc_launch(p, p.sync, s);
     if (e != cudaSuccess) return e;

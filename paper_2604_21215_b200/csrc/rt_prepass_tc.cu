@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(kGemmThreads, 2)
 qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_constant__ CUtensorMap map_wq,
                    const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv,
                    const PrepassParams p, SyncArea* sync) {
+  grid_dep_sync();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -190,8 +191,7 @@ cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStrea
   cudaError_t e = cudaFuncSetAttribute(qkv_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(ceil_div(M, kBM), 3 * (p.d / kGemmBN));
-  qkv_gemm_tc_kernel<<<grid, kGemmThreads, smem, s>>>(mn, mq, mk, mv, p, sync);
-  return cudaGetLastError();
+  return launch_chained(qkv_gemm_tc_kernel, grid, dim3(kGemmThreads), smem, s, p.chained != 0, mn, mq, mk, mv, p, sync);
 }
 
 }  // namespace rt

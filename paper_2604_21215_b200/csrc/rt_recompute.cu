@@ -21,6 +21,7 @@ __device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.0f +
 // ---- c = o / l ------------------------------------------------------------------------------
 template <typename T>
 __global__ void attn_value_kernel(const float* st_o, const float* st_l, T* c, long long rows, int d, int H) {
+  grid_dep_sync();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;       // one thread = 4 columns
   const long long total = rows * (d / 4);
   if (i >= total) return;
@@ -35,6 +36,7 @@ __global__ void attn_value_kernel(const float* st_o, const float* st_l, T* c, lo
 // ---- u = RMS_g(h) for fp32 rows -------------------------------------------------------------------
 template <typename T>
 __global__ void rms_rows_f32_kernel(const float* h, const T* g, T* u, int rows, int d, float eps, int pre) {
+  grid_dep_sync();
   const int lane = threadIdx.x & 31;
   const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (m >= rows) return;
@@ -132,6 +134,7 @@ template <int BN>
 __global__ void __launch_bounds__(kTThreads, 2)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
                 SyncArea* sync) {
+  grid_dep_sync();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -292,6 +295,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // output row, so it can also leave RMS_g(row) of the result for the product that follows.
 template <typename T>
 __global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) {
+  grid_dep_sync();
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
   const int b = m % p.B, r = m / p.B;
@@ -373,15 +377,18 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       const size_t smem = DenseSmem<256>::total + 1024;
       cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      dense_tc_kernel<256><<<grid, kTThreads, smem, s>>>(ma, mw, q, sync);
+      e = launch_chained(dense_tc_kernel<256>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
+      if (e != cudaSuccess) return e;
     } else {
       const size_t smem = DenseSmem<128>::total + 1024;
       cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      dense_tc_kernel<128><<<grid, kTThreads, smem, s>>>(ma, mw, q, sync);
+      e = launch_chained(dense_tc_kernel<128>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
+      if (e != cudaSuccess) return e;
     }
     if (q.splits > 1) {
-      dense_reduce_kernel<__nv_bfloat16><<<p.M, 256, 0, s>>>(q);
+      cudaError_t er = launch_chained(dense_reduce_kernel<__nv_bfloat16>, dim3(p.M), dim3(256), 0, s, p.chained != 0, q);
+      if (er != cudaSuccess) return er;
       if (normed && p.norm_out) *normed = true;
     }
     return cudaGetLastError();
@@ -392,18 +399,19 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
   return cudaGetLastError();
 }
 
-cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s) {
+cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s,
+                              bool chained) {
   const long long total = rows * (d / 4);
-  const unsigned blocks = (unsigned)((total + 255) / 256);
-  if (dtype == RT_BF16) attn_value_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(st_o, st_l, (__nv_bfloat16*)c, rows, d, H);
-  else attn_value_kernel<float><<<blocks, 256, 0, s>>>(st_o, st_l, (float*)c, rows, d, H);
-  return cudaGetLastError();
+  const dim3 blocks((unsigned)((total + 255) / 256));
+  if (dtype == RT_BF16) return launch_chained(attn_value_kernel<__nv_bfloat16>, blocks, dim3(256), 0, s, chained, st_o, st_l, (__nv_bfloat16*)c, rows, d, H);
+  return launch_chained(attn_value_kernel<float>, blocks, dim3(256), 0, s, chained, st_o, st_l, (float*)c, rows, d, H);
 }
 
-cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s) {
-  if (dtype == RT_BF16) rms_rows_f32_kernel<__nv_bfloat16><<<ceil_div(rows, 8), 256, 0, s>>>(h, (const __nv_bfloat16*)g, (__nv_bfloat16*)u, rows, d, eps, pre);
-  else rms_rows_f32_kernel<float><<<ceil_div(rows, 8), 256, 0, s>>>(h, (const float*)g, (float*)u, rows, d, eps, pre);
-  return cudaGetLastError();
+cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s,
+                                bool chained) {
+  const dim3 blocks(ceil_div(rows, 8));
+  if (dtype == RT_BF16) return launch_chained(rms_rows_f32_kernel<__nv_bfloat16>, blocks, dim3(256), 0, s, chained, h, (const __nv_bfloat16*)g, (__nv_bfloat16*)u, rows, d, eps, pre);
+  return launch_chained(rms_rows_f32_kernel<float>, blocks, dim3(256), 0, s, chained, h, (const float*)g, (float*)u, rows, d, eps, pre);
 }
 
 }  // namespace rt

@@ -108,6 +108,7 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
 // the head's dimensions), the 32 per-lane partial products become per-key scores by a transposed reduction.
 template <typename T>
 __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
+  grid_dep_sync();
   const int lane = threadIdx.x & 31;
   const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (u >= p.B * p.H) return;
@@ -161,9 +162,8 @@ __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
 cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s) {
   if (p.k1 <= p.k0 && !p.c_out) return cudaSuccess;
   const int blocks = ceil_div(p.B * p.H, 8);
-  if (dtype == RT_BF16) row_attn_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(p);
-  else row_attn_kernel<float><<<blocks, 256, 0, s>>>(p);
-  return cudaGetLastError();
+  if (dtype == RT_BF16) return launch_chained(row_attn_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, s, p.chained != 0, p);
+  return launch_chained(row_attn_kernel<float>, dim3(blocks), dim3(256), 0, s, p.chained != 0, p);
 }
 
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
