@@ -9,3 +9,4 @@ from .rt_oracle import (  # noqa: F401
     layer_seq, layer_blk, layer_fixed_point, layer_decode, layer_blockrec,
     stack_prefill, stack_decode, alg1_tiles, update_tile,
 )
+from .rt_oracle_grad import layer_grad, layer_seq_torch  # noqa: F401,E402
