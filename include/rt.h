@@ -205,6 +205,27 @@ rt_status rt_layer_recompute(const rt_config *cfg, const rt_layer_weights *w, co
                              int32_t B, int32_t N, void *z_out, void *k_cache, void *v_cache, int32_t N_max,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Backward pass of one layer (Sec. 6, "The backward pass" and "activation checkpointing").
+ * Inputs: the layer input x [B,N,d] and its outputs z [B,N,d] as rt_layer_prefill returned them (storage type; z is the
+ * next layer's input, so a training loop keeps it anyway), and dz = dL/dz [B,N,d] fp32.
+ * Outputs: dx = dL/dx [B,N,d] fp32 and the parameter gradients in `grads` (fp32, device, shapes of the parameters,
+ * OVERWRITTEN; a NULL entry is skipped; the entry of a gain the layer does not have (NULL in `w`) is set to zero).
+ * When w->g_kv is NULL the gain of RMS(z) IS g_attn, and grads->g_attn carries both uses.
+ * The call first rebuilds every intermediate from x and z in one parallel sweep, then walks the positions in reverse
+ * accumulating only d(k_j, v_j) -- position i needs dL/dz_i, which needs d(k_i, v_i) complete; pairs in other leaves
+ * of 64 positions receive their share from Algorithm 1's tiles run backwards -- and finally forms dq, the temporary
+ * pairs, dx and every parameter gradient as products over all B*N rows at once.
+ * fp32 arithmetic on CUDA cores throughout (both storage types); recur_block > 1 returns RT_ERR_UNSUPPORTED.
+ * The workspace needs rt_backward_workspace_bytes (about 30 fp32 arrays of B*N*d plus 3 of B*N*d_ff). */
+typedef struct {
+  float *w_q, *w_k, *w_v, *w_o, *w_up, *w_down;   /* shapes of rt_layer_weights */
+  float *g_attn, *g_mlp, *g_kv, *g_q, *g_k;       /* [d_model] */
+} rt_layer_grads;
+size_t    rt_backward_workspace_bytes(const rt_config *cfg, int32_t B, int32_t N);
+rt_status rt_layer_backward(const rt_config *cfg, const rt_layer_weights *w, const void *x, const void *z, const float *dz,
+                            int32_t B, int32_t N, float *dx, const rt_layer_grads *grads,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Self-test of the bounded device-side wait (no counterpart in the paper): enqueues a two-CTA kernel
  * whose grid barrier expects an arrival that never comes.  The wait gives up after its limit (2 s),
  * the kernel returns normally, and rt_get_status(workspace) then reports RT_ERR_TIMEOUT; the CUDA

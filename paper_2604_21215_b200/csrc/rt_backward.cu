@@ -1,0 +1,700 @@
+// Backward pass of one RT layer (Sec. 6, "The backward pass"; activation checkpointing as in Sec. 6).
+//
+// Given the layer input x, its outputs z (kept anyway: they are the next layer's input) and dL/dz, the call
+//   1. rebuilds every intermediate in one parallel sweep (persistent pairs from z, queries and temporary pairs from x,
+//      attention values and their log-sum-exp, the chain h, u, W_up u),
+//   2. walks the positions in reverse and accumulates ONLY d(k_j, v_j): position i needs the final dL/dz_i, which
+//      needs d(k_i, v_i) complete; pairs of other leaves get their share from the tiles of Algorithm 1 run backwards
+//      (the same tiles, visited in reverse order, each as one launch over all its keys),
+//   3. computes everything else -- dq, the temporary pairs, dx and all parameter gradients -- as large products over
+//      all rows at once.
+// All arithmetic here is fp32 on CUDA cores (first version: correctness and the schedule; no tensor cores yet).
+#include <math.h>
+#include <string.h>
+
+#include "rt_common.cuh"
+
+namespace rt {
+namespace {
+
+// ------------------------------------------------------------------------------------------------ generic product
+// C[m, n] = alpha * sum_k A(m, k) Bm(k, n)  (+ C when accumulate), A(m,k) = A[m*a_rs + k*a_cs], Bm(k,n) = Bm[k*b_rs + n*b_cs].
+template <typename TA, typename TB>
+__global__ void __launch_bounds__(256) gemm_kernel(int M, int N, int K, const TA* __restrict__ A, long long a_rs, long long a_cs,
+                                                   const TB* __restrict__ Bm, long long b_rs, long long b_cs,
+                                                   float* __restrict__ C, long long ldc, float alpha, int accumulate) {
+  __shared__ float As[16][68];
+  __shared__ float Bs[16][68];
+  const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < K; k0 += 16) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      int m, k;
+      if (a_cs == 1) { k = t & 15; m = (t >> 4) + 16 * it; } else { m = t & 63; k = (t >> 6) + 4 * it; }
+      float v = 0.f;
+      if (m0 + m < M && k0 + k < K) v = to_f(A[(long long)(m0 + m) * a_rs + (long long)(k0 + k) * a_cs]);
+      As[k][m] = v;
+      int n;
+      if (b_cs == 1) { n = t & 63; k = (t >> 6) + 4 * it; } else { k = t & 15; n = (t >> 4) + 16 * it; }
+      v = 0.f;
+      if (n0 + n < N && k0 + k < K) v = to_f(Bm[(long long)(k0 + k) * b_rs + (long long)(n0 + n) * b_cs]);
+      Bs[k][n] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      if (m < M && n < N) {
+        float* c = C + (long long)m * ldc + n;
+        *c = (accumulate ? *c : 0.f) + alpha * acc[i][j];
+      }
+    }
+}
+
+template <typename TA, typename TB>
+cudaError_t gemm(int M, int N, int K, const TA* A, long long a_rs, long long a_cs, const TB* Bm, long long b_rs, long long b_cs,
+                 float* C, long long ldc, float alpha, bool accumulate, cudaStream_t s) {
+  gemm_kernel<TA, TB><<<dim3(ceil_div(N, 64), ceil_div(M, 64)), 256, 0, s>>>(M, N, K, A, a_rs, a_cs, Bm, b_rs, b_cs, C, ldc, alpha,
+                                                                              accumulate ? 1 : 0);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------ RMS forward / backward
+// Row r = i*B + b of a [B, N, *] array sits at b*bs + i*ts; position-major fp32 buffers use bs = width, ts = B*width.
+__device__ __forceinline__ long long row_at(long long r, int B, long long bs, long long ts) { return (r % B) * bs + (r / B) * ts; }
+
+// y = g u / sqrt(mean_G(u^2) + eps) over groups of G entries (G = d: RMS of Sec. 2; G = 64: qkRMS per head); copy when !enable.
+template <typename TI, typename TG>
+__global__ void norm_fwd_kernel(const TI* __restrict__ in, long long bs, long long ts, int B, const TG* __restrict__ g,
+                                float* __restrict__ out, long long rows, int d, int G, float eps, int enable) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31, groups = d / G;
+  if (wid >= rows * groups) return;
+  const long long r = wid / groups;
+  const int c0 = (int)(wid % groups) * G;
+  const TI* src = in + row_at(r, B, bs, ts) + c0;
+  float* dst = out + r * d + c0;
+  float ss = 0.f;
+  for (int e = lane; e < G; e += 32) { const float v = to_f(src[e]); ss = fmaf(v, v, ss); }
+  ss = warp_sum(ss);
+  const float inv = rsqrtf(ss / G + eps);
+  for (int e = lane; e < G; e += 32) dst[e] = enable ? to_f(src[e]) * inv * gain_at(g, c0 + e) : to_f(src[e]);
+}
+
+// With y = g u inv, inv = (mean(u^2)+eps)^(-1/2), t = g dy and uh = u inv:  du = inv (t - uh mean(t uh)),  dg += dy uh.
+// out = (add ? add : 0) + du;  gprod (=|+=) dy uh.  out and gprod may each be NULL.  !enable: du = dy.
+template <typename TU, typename TG>
+__global__ void norm_bwd_kernel(const float* dy, const TU* __restrict__ u, long long u_bs, long long u_ts, int B,
+                                const TG* __restrict__ g, const float* add, float* out, long long o_bs, long long o_ts,
+                                float* gprod, int gprod_acc, long long rows, int d, int G, float eps, int enable) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31, groups = d / G;
+  if (wid >= rows * groups) return;
+  const long long r = wid / groups;
+  const int c0 = (int)(wid % groups) * G;
+  const float* dyr = dy + r * d + c0;
+  const TU* ur = u + row_at(r, B, u_bs, u_ts) + c0;
+  float ss = 0.f, tu = 0.f;
+  if (enable) {
+    for (int e = lane; e < G; e += 32) {
+      const float v = to_f(ur[e]);
+      ss = fmaf(v, v, ss);
+      tu = fmaf(dyr[e] * gain_at(g, c0 + e), v, tu);
+    }
+    ss = warp_sum(ss); tu = warp_sum(tu);
+  }
+  const float inv = rsqrtf(ss / G + eps);
+  const float mean = tu * inv / G;
+  for (int e = lane; e < G; e += 32) {
+    float du = dyr[e], gp = 0.f;
+    if (enable) {
+      const float uh = to_f(ur[e]) * inv;
+      du = inv * (dyr[e] * gain_at(g, c0 + e) - uh * mean);
+      gp = dyr[e] * uh;
+    }
+    if (out) out[row_at(r, B, o_bs, o_ts) + c0 + e] = (add ? add[r * d + c0 + e] : 0.f) + du;
+    if (gprod) gprod[r * d + c0 + e] = (gprod_acc ? gprod[r * d + c0 + e] : 0.f) + gp;
+  }
+}
+
+// column sums of a [rows, d] array in two fixed-order steps
+__global__ void col_partial_kernel(const float* __restrict__ a, long long rows, int d, float* __restrict__ part, int P) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d) return;
+  const long long chunk = (rows + P - 1) / P, r0 = blockIdx.y * chunk, r1 = r0 + chunk < rows ? r0 + chunk : rows;
+  float s = 0.f;
+  for (long long r = r0; r < r1; ++r) s += a[r * d + c];
+  part[(long long)blockIdx.y * d + c] = s;
+}
+__global__ void col_final_kernel(const float* __restrict__ part, int P, int d, float* out, int accumulate) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d) return;
+  float s = 0.f;
+  for (int p = 0; p < P; ++p) s += part[(long long)p * d + c];
+  out[c] = (accumulate ? out[c] : 0.f) + s;
+}
+
+// h = x + alpha a  (x [B,N,d] storage type, a and h position-major fp32)
+template <typename T>
+__global__ void residual_kernel(const T* __restrict__ x, long long bs, long long ts, int B, const float* __restrict__ a, float alpha,
+                                float* __restrict__ h, long long rows, int d) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * d) return;
+  const long long r = idx / d;
+  const int c = (int)(idx % d);
+  h[idx] = to_f(x[row_at(r, B, bs, ts) + c]) + alpha * a[idx];
+}
+
+__device__ __forceinline__ float gelu_f(float a) { return 0.5f * a * (1.f + erff(a * 0.70710678118654752f)); }
+// d/da [a Phi(a)] = Phi(a) + a phi(a)
+__device__ __forceinline__ float gelu_grad_f(float a) {
+  return 0.5f * (1.f + erff(a * 0.70710678118654752f)) + a * 0.3989422804014327f * __expf(-0.5f * a * a);
+}
+__global__ void gelu_kernel(const float* __restrict__ a, float* __restrict__ out, long long n) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < n) out[idx] = gelu_f(a[idx]);
+}
+
+// ------------------------------------------------------------------------------------------------ attention
+struct AttnBufs {
+  const float *q, *k, *v, *kt, *vt;        // position-major [rows, d]
+  float *lse, *D;                          // [rows, H]: log2-sum-exp of the logits (log2 units), <dc, c> per head
+  float *c;                                // [rows, d] attention value
+  const float* dc;                         // [rows, d] gradient of the attention value
+  float *dK, *dV, *dkt, *dvt, *dq;
+  const float* alibi;                      // [H] or NULL
+  float scale, scale_log2;
+  int B, H, d, N;
+};
+
+// One warp per (position i, sequence, head): the softmax of Sec. 2.2 over the pairs j < i and the temporary pair;
+// keeps c = attention value and the log2-sum-exp of the logits.
+__global__ void attn_stats_kernel(AttnBufs a) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)a.N * a.B * a.H) return;
+  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
+  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long ri = ((long long)i * a.B + b) * a.d + col;
+  const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  float m = -INFINITY, l = 0.f, o0 = 0.f, o1 = 0.f;
+  auto step = [&](float s, float2 vv) {
+    const float mn = fmaxf(m, s);
+    const float corr = exp2f(m - mn), p = exp2f(s - mn);
+    l = l * corr + p; o0 = o0 * corr + p * vv.x; o1 = o1 * corr + p * vv.y;
+    m = mn;
+  };
+  int j = 0;
+  for (; j + 4 <= i; j += 4) {
+    float s[4]; float2 vv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long rj = ((long long)(j + u) * a.B + b) * a.d + col;
+      const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+      vv[u] = *reinterpret_cast<const float2*>(a.v + rj);
+      s[u] = q.x * kk.x + q.y * kk.y;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) s[u] = warp_sum(s[u]) * a.scale_log2 - slope * (float)(i - j - u);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) step(s[u], vv[u]);
+  }
+  for (; j < i; ++j) {
+    const long long rj = ((long long)j * a.B + b) * a.d + col;
+    const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+    step(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - slope * (float)(i - j), *reinterpret_cast<const float2*>(a.v + rj));
+  }
+  {
+    const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
+    step(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2, *reinterpret_cast<const float2*>(a.vt + ri));
+  }
+  const float inv = 1.f / l;
+  *reinterpret_cast<float2*>(a.c + ri) = make_float2(o0 * inv, o1 * inv);
+  if (lane == 0) a.lse[((long long)i * a.B + b) * a.H + h] = m + log2f(l);
+}
+
+// Gradient of the pairs: one warp per (key j, sequence, head) holds k_j, v_j and sums over the queries [q0, q1):
+//   p = exp2(logit - lse_i), ds = p (<dc_i, v_j> - D_i), dk_j += scale ds q_i, dv_j += p dc_i.
+// self = 1 (the in-leaf step of position i = q0): keys [k0, i]; every warp computes D_i = <dc_i, c_i> itself, and the warp
+// of j = i stores it and handles the temporary pair of position i instead of a persistent one.
+__global__ void attn_bwd_kv_kernel(AttnBufs a, int q0, int q1, int k0, int k1, int self) {
+  grid_dep_sync();
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)(k1 - k0) * a.B * a.H) return;
+  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
+  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long rj = ((long long)j * a.B + b) * a.d + col;
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  if (self) {
+    const int i = q0;
+    const long long ri = ((long long)i * a.B + b) * a.d + col;
+    const long long si = ((long long)i * a.B + b) * a.H + h;
+    const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
+    const float2 cc = *reinterpret_cast<const float2*>(a.c + ri);
+    const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+    const float D = warp_sum(dc.x * cc.x + dc.y * cc.y);
+    const float lse = a.lse[si];
+    if (j == i) {
+      if (lane == 0) a.D[si] = D;
+      const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
+      const float2 vv = *reinterpret_cast<const float2*>(a.vt + ri);
+      const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - lse);
+      const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
+      *reinterpret_cast<float2*>(a.dkt + ri) = make_float2(ds * q.x, ds * q.y);
+      *reinterpret_cast<float2*>(a.dvt + ri) = make_float2(p * dc.x, p * dc.y);
+    } else {
+      const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+      const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
+      const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - slope * (float)(i - j) - lse);
+      const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
+      float2* dk = reinterpret_cast<float2*>(a.dK + rj);
+      float2* dv = reinterpret_cast<float2*>(a.dV + rj);
+      float2 t = *dk; t.x += ds * q.x; t.y += ds * q.y; *dk = t;
+      t = *dv; t.x += p * dc.x; t.y += p * dc.y; *dv = t;
+    }
+    return;
+  }
+  const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+  const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
+  float dk0 = 0.f, dk1 = 0.f, dv0 = 0.f, dv1 = 0.f;
+  const long long rstride = (long long)a.B * a.d;
+  long long ri = ((long long)q0 * a.B + b) * a.d + col;
+  long long si = ((long long)q0 * a.B + b) * a.H + h;
+#pragma unroll 2
+  for (int i = q0; i < q1; ++i, ri += rstride, si += (long long)a.B * a.H) {
+    const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+    const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
+    const float lse = a.lse[si], D = a.D[si];
+    float s = q.x * kk.x + q.y * kk.y, dp = dc.x * vv.x + dc.y * vv.y;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dp += __shfl_xor_sync(0xffffffffu, dp, o); }
+    const float p = exp2f(s * a.scale_log2 - slope * (float)(i - j) - lse);
+    const float ds = p * (dp - D) * a.scale;
+    dk0 = fmaf(ds, q.x, dk0); dk1 = fmaf(ds, q.y, dk1);
+    dv0 = fmaf(p, dc.x, dv0); dv1 = fmaf(p, dc.y, dv1);
+  }
+  float2* dk = reinterpret_cast<float2*>(a.dK + rj);
+  float2* dv = reinterpret_cast<float2*>(a.dV + rj);
+  float2 t = *dk; t.x += dk0; t.y += dk1; *dk = t;
+  t = *dv; t.x += dv0; t.y += dv1; *dv = t;
+}
+
+// Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).
+__global__ void attn_bwd_q_kernel(AttnBufs a) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)a.N * a.B * a.H) return;
+  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
+  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long ri = ((long long)i * a.B + b) * a.d + col;
+  const long long si = ((long long)i * a.B + b) * a.H + h;
+  const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+  const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
+  const float lse = a.lse[si], D = a.D[si];
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  float g0 = 0.f, g1 = 0.f;
+  long long rj = (long long)b * a.d + col;
+  const long long rstride = (long long)a.B * a.d;
+#pragma unroll 2
+  for (int j = 0; j < i; ++j, rj += rstride) {
+    const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+    const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
+    float s = q.x * kk.x + q.y * kk.y, dp = dc.x * vv.x + dc.y * vv.y;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dp += __shfl_xor_sync(0xffffffffu, dp, o); }
+    const float ds = exp2f(s * a.scale_log2 - slope * (float)(i - j) - lse) * (dp - D);
+    g0 = fmaf(ds, kk.x, g0); g1 = fmaf(ds, kk.y, g1);
+  }
+  {
+    const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
+    const float2 vv = *reinterpret_cast<const float2*>(a.vt + ri);
+    const float s = warp_sum(q.x * kk.x + q.y * kk.y), dp = warp_sum(dc.x * vv.x + dc.y * vv.y);
+    const float ds = exp2f(s * a.scale_log2 - lse) * (dp - D);
+    g0 = fmaf(ds, kk.x, g0); g1 = fmaf(ds, kk.y, g1);
+  }
+  *reinterpret_cast<float2*>(a.dq + ri) = make_float2(g0 * a.scale, g1 * a.scale);
+}
+
+// ------------------------------------------------------------------------------------------------ the reverse loop's products
+// One position i, the B rows of the batch: out[b, n] = alpha * (sum_k in1[b,k] W1[k,n] + sum_k in2[b,k] W2[k,n]) where the
+// rows in1 (in2) are built by a prologue from the state of the reverse loop (mode), W = a weight matrix as stored
+// ([its outputs, its inputs] = [K, Ncols]: the transposed product of the forward pass, read row by row).
+enum { RM_PAIR = 1, RM_DOWN = 2, RM_UP = 3, RM_OUT = 4 };
+constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmCols = 32;
+struct RowmatParams {
+  int mode, B, d, dff, i, K, Ncols;
+  int norm_on, qk_on;                     // whether the prologue's RMS / qkRMS is active
+  float eps, alpha;
+  const void *W1, *W2, *gain;             // storage type
+  const void* z; long long z_bs, z_ts;    // layer output [B,N,d], storage type (RM_DOWN)
+  const float* dz; long long dz_bs, dz_ts;
+  const float *dK, *dV, *kraw, *h, *act;
+  float *dkraw, *dr, *Gz, *dpre, *du, *dh, *dc;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p) {
+  grid_dep_sync();
+  extern __shared__ __align__(16) float smem[];
+  float* in1 = smem;                                        // [K][4]
+  float* in2 = in1 + (size_t)p.K * kRowsPerCta;             // [K][4] (RM_PAIR only)
+  float* red = in2 + (p.mode == RM_PAIR ? (size_t)p.K * kRowsPerCta : 0);   // [16][32][4]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b0 = blockIdx.y * kRowsPerCta;
+  const bool writer = blockIdx.x == 0;
+  const int d = p.d;
+  const T* gain = reinterpret_cast<const T*>(p.gain);
+
+  // ---- prologue: the input rows of this CTA's sequences, transposed into shared memory
+  if (p.mode == RM_PAIR) {
+    // in1 = qkRMS backward of dK_i through k_i = qkRMS(kraw_i) per head; in2 = dV_i
+    const int H = d / kHeadDim;
+    for (int task = warp; task < kRowsPerCta * H; task += kRmThreads / 32) {
+      const int r = task / H, h = task % H, b = b0 + r;
+      const int c0 = h * kHeadDim;
+      float o0 = 0.f, o1 = 0.f, v0 = 0.f, v1 = 0.f;
+      if (b < p.B) {
+        const long long at = ((long long)p.i * p.B + b) * d + c0;
+        const float dy0 = p.dK[at + lane], dy1 = p.dK[at + lane + 32];
+        v0 = p.dV[at + lane]; v1 = p.dV[at + lane + 32];
+        if (p.qk_on) {
+          const float u0 = p.kraw[at + lane], u1 = p.kraw[at + lane + 32];
+          const float g0 = gain_at(gain, c0 + lane), g1 = gain_at(gain, c0 + lane + 32);
+          const float ss = warp_sum(u0 * u0 + u1 * u1), tu = warp_sum(dy0 * g0 * u0 + dy1 * g1 * u1);
+          const float inv = rsqrtf(ss / kHeadDim + p.eps), mean = tu * inv / kHeadDim;
+          o0 = inv * (dy0 * g0 - u0 * inv * mean); o1 = inv * (dy1 * g1 - u1 * inv * mean);
+        } else { o0 = dy0; o1 = dy1; }
+        if (writer) { p.dkraw[at + lane] = o0; p.dkraw[at + lane + 32] = o1; }
+      }
+      in1[(c0 + lane) * kRowsPerCta + r] = o0; in1[(c0 + lane + 32) * kRowsPerCta + r] = o1;
+      in2[(c0 + lane) * kRowsPerCta + r] = v0; in2[(c0 + lane + 32) * kRowsPerCta + r] = v1;
+    }
+  } else if (p.mode == RM_UP) {
+    for (int idx = threadIdx.x; idx < kRowsPerCta * p.K; idx += kRmThreads) {
+      const int r = idx / p.K, k = idx % p.K, b = b0 + r;
+      in1[k * kRowsPerCta + r] = b < p.B ? p.dpre[((long long)p.i * p.B + b) * p.K + k] : 0.f;
+    }
+  } else {
+    // RM_DOWN: Gz = dz_i + RMS backward of dr_i through RMS(z_i);  RM_OUT: dh = Gz_i + RMS backward of du_i through RMS(h_i)
+    const T* zT = reinterpret_cast<const T*>(p.z);
+    for (int r = warp; r < kRowsPerCta; r += kRmThreads / 32) {
+      const int b = b0 + r;
+      if (b >= p.B) {
+        for (int e = lane; e < d; e += 32) in1[e * kRowsPerCta + r] = 0.f;
+        continue;
+      }
+      const long long at = ((long long)p.i * p.B + b) * d;
+      const float* dy = (p.mode == RM_DOWN ? p.dr : p.du) + at;
+      const float* addv = p.mode == RM_DOWN ? p.dz + (long long)b * p.dz_bs + (long long)p.i * p.dz_ts : p.Gz + at;
+      const T* zr = zT + (long long)b * p.z_bs + (long long)p.i * p.z_ts;
+      float* keep = (p.mode == RM_DOWN ? p.Gz : p.dh) + at;
+      float ss = 0.f, tu = 0.f;
+      if (p.norm_on) {
+        for (int e = lane; e < d; e += 32) {
+          const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
+          ss = fmaf(u, u, ss);
+          tu = fmaf(dy[e] * gain_at(gain, e), u, tu);
+        }
+        ss = warp_sum(ss); tu = warp_sum(tu);
+      }
+      const float inv = rsqrtf(ss / d + p.eps), mean = tu * inv / d;
+      for (int e = lane; e < d; e += 32) {
+        float du = dy[e];
+        if (p.norm_on) {
+          const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
+          du = inv * (dy[e] * gain_at(gain, e) - u * inv * mean);
+        }
+        const float val = addv[e] + du;
+        in1[e * kRowsPerCta + r] = val;
+        if (writer) keep[e] = val;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- product: this CTA's 32 columns; a warp's lanes = 4 rows of W x 8 groups of 4 columns
+  const int kq = lane >> 3, cq = lane & 7;
+  const int n0 = blockIdx.x * kRmCols + 4 * cq;
+  float acc[kRowsPerCta][4] = {};
+  auto run = [&](const T* W, const float* in) {
+#pragma unroll 4
+    for (int k = warp * 4 + kq; k < p.K; k += (kRmThreads / 32) * 4) {
+      Vec4<T> wv;
+      wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols + n0);
+      float wf[4];
+      wv.to_float(wf);
+      const float4 a4 = *reinterpret_cast<const float4*>(in + (size_t)k * kRowsPerCta);
+      const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+      for (int r = 0; r < kRowsPerCta; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
+    }
+  };
+  run(reinterpret_cast<const T*>(p.W1), in1);
+  if (p.mode == RM_PAIR) run(reinterpret_cast<const T*>(p.W2), in2);
+#pragma unroll
+  for (int r = 0; r < kRowsPerCta; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float v = acc[r][c];
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      if (kq == 0) red[(warp * kRmCols + 4 * cq + c) * kRowsPerCta + r] = v;
+    }
+  __syncthreads();
+  if (threadIdx.x < kRmCols * kRowsPerCta) {
+    const int col = threadIdx.x >> 2, r = threadIdx.x & 3, b = b0 + r;
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kRmThreads / 32; ++w) s += red[(w * kRmCols + col) * kRowsPerCta + r];
+    if (b < p.B) {
+      const int n = blockIdx.x * kRmCols + col;
+      const long long at = ((long long)p.i * p.B + b) * p.Ncols + n;
+      s *= p.alpha;
+      if (p.mode == RM_PAIR) p.dr[at] = s;
+      else if (p.mode == RM_DOWN) p.dpre[at] = s * gelu_grad_f(p.act[at]);
+      else if (p.mode == RM_UP) p.du[at] = s;
+      else p.dc[at] = s;
+    }
+  }
+}
+
+size_t rowmat_smem(int mode, int K) {
+  return ((size_t)K * kRowsPerCta * (mode == RM_PAIR ? 2 : 1) + (kRmThreads / 32) * kRmCols * kRowsPerCta) * sizeof(float);
+}
+
+// ------------------------------------------------------------------------------------------------ workspace
+struct BwdLayout {
+  size_t sync, n, qraw, ktraw, vt, q, kt, r, kraw, k, v, c, h, u, act, gl, lse, D;
+  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part;
+  size_t zero_begin, zero_end, total;
+};
+constexpr int kColParts = 128;
+
+BwdLayout bwd_layout(const rt_config* c, int B, int N) {
+  BwdLayout L;
+  const size_t d = c->d_model, f = c->d_ff, H = c->n_heads, rows = (size_t)B * N;
+  size_t o = 0;
+  auto take = [&](size_t floats) { size_t at = o; o += align_up(floats * 4, 256); return at; };
+  L.sync = take(sizeof(SyncArea) / 4);
+  L.n = take(rows * d); L.qraw = take(rows * d); L.ktraw = take(rows * d); L.vt = take(rows * d);
+  L.q = take(rows * d); L.kt = take(rows * d); L.r = take(rows * d); L.kraw = take(rows * d);
+  L.k = take(rows * d); L.v = take(rows * d); L.c = take(rows * d); L.h = take(rows * d); L.u = take(rows * d);
+  L.act = take(rows * f); L.gl = take(rows * f); L.lse = take(rows * H); L.D = take(rows * H);
+  L.zero_begin = o;
+  L.dK = take(rows * d); L.dV = take(rows * d);
+  L.zero_end = o;
+  L.dkraw = take(rows * d); L.dr = take(rows * d); L.Gz = take(rows * d); L.dpre = take(rows * f);
+  L.du = take(rows * d); L.dh = take(rows * d); L.dc = take(rows * d); L.dq = take(rows * d);
+  L.dkt = take(rows * d); L.dvt = take(rows * d); L.dn = take(rows * d); L.gprod = take(rows * d);
+  L.part = take((size_t)kColParts * (d > f ? d : f));
+  L.total = o;
+  return L;
+}
+
+bool bwd_config_ok(const rt_config* c) {
+  if (!c) return false;
+  if (c->d_model <= 0 || c->n_heads <= 0 || c->d_ff <= 0 || (long long)c->n_heads * c->head_dim != c->d_model) return false;
+  if (c->dtype != RT_F32 && c->dtype != RT_BF16) return false;
+  if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
+  if (c->norm_flags & ~15) return false;
+  return true;
+}
+
+#define RT_TRY(...) do { if ((__VA_ARGS__) != cudaSuccess) return RT_ERR_CUDA; } while (0)
+
+template <typename T>
+rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* x, const T* z, const float* dz, int B, int N,
+                        float* dx, const rt_layer_grads* gr, unsigned char* ws, cudaStream_t s) {
+  const BwdLayout L = bwd_layout(c, B, N);
+  const int d = c->d_model, f = c->d_ff, H = c->n_heads;
+  const long long rows = (long long)B * N;
+  const long long xbs = (long long)N * d, xts = d;             // [B, N, d]
+  const long long pbs = d, pts = (long long)B * d;             // position-major fp32 [rows, d] seen as (b, i)
+  const bool pre = (c->norm_flags & RT_NORM_PRE) != 0, qk = (c->norm_flags & RT_NORM_QK) != 0;
+  const bool z_norm = pre && !(c->norm_flags & RT_NORM_SKIP_Z);
+  const float eps = c->rms_eps, alpha = c->residual_scale;
+  auto F = [&](size_t off) { return reinterpret_cast<float*>(ws + off); };
+  const T *Wq = (const T*)w->w_q, *Wk = (const T*)w->w_k, *Wv = (const T*)w->w_v, *Wo = (const T*)w->w_o;
+  const T *Wup = (const T*)w->w_up, *Wdn = (const T*)w->w_down;
+  const T *g_attn = (const T*)w->g_attn, *g_mlp = (const T*)w->g_mlp, *g_q = (const T*)w->g_q, *g_k = (const T*)w->g_k;
+  const T* g_kv = (const T*)(w->g_kv ? w->g_kv : w->g_attn);
+  const int tpb = 256;
+  auto warps_grid = [&](long long warps) { return (unsigned)((warps * 32 + tpb - 1) / tpb); };
+  auto elems_grid = [&](long long n) { return (unsigned)((n + tpb - 1) / tpb); };
+
+  RT_TRY(cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s));
+  RT_TRY(cudaMemsetAsync(ws + L.zero_begin, 0, L.zero_end - L.zero_begin, s));
+
+  // ---- 1. the parallel sweep: every intermediate of the forward pass from x and z
+  norm_fwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(x, xbs, xts, B, g_attn, F(L.n), rows, d, d, eps, pre ? 1 : 0);
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wq, 1, d, F(L.qraw), d, 1.f, false, s));
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wk, 1, d, F(L.ktraw), d, 1.f, false, s));
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wv, 1, d, F(L.vt), d, 1.f, false, s));
+  norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.qraw), pbs, pts, B, g_q, F(L.q), rows, d, kHeadDim, eps, qk);
+  norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.ktraw), pbs, pts, B, g_k, F(L.kt), rows, d, kHeadDim, eps, qk);
+  norm_fwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(z, xbs, xts, B, g_kv, F(L.r), rows, d, d, eps, z_norm ? 1 : 0);
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wk, 1, d, F(L.kraw), d, 1.f, false, s));
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wv, 1, d, F(L.v), d, 1.f, false, s));
+  norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.kraw), pbs, pts, B, g_k, F(L.k), rows, d, kHeadDim, eps, qk);
+  AttnBufs ab;
+  memset(&ab, 0, sizeof(ab));
+  ab.q = F(L.q); ab.k = F(L.k); ab.v = F(L.v); ab.kt = F(L.kt); ab.vt = F(L.vt); ab.lse = F(L.lse); ab.D = F(L.D);
+  ab.c = F(L.c); ab.dc = F(L.dc); ab.dK = F(L.dK); ab.dV = F(L.dV); ab.dkt = F(L.dkt); ab.dvt = F(L.dvt); ab.dq = F(L.dq);
+  ab.alibi = w->alibi_slopes; ab.scale = c->softmax_scale; ab.scale_log2 = c->softmax_scale * kLog2e;
+  ab.B = B; ab.H = H; ab.d = d; ab.N = N;
+  attn_stats_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.c), d, 1, Wo, 1, d, F(L.dn), d, 1.f, false, s));          // a = W_o c (dn as scratch)
+  residual_kernel<T><<<elems_grid(rows * d), tpb, 0, s>>>(x, xbs, xts, B, F(L.dn), alpha, F(L.h), rows, d);
+  norm_fwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.h), pbs, pts, B, g_mlp, F(L.u), rows, d, d, eps, pre ? 1 : 0);
+  RT_TRY(gemm<float, T>((int)rows, f, d, F(L.u), d, 1, Wup, 1, d, F(L.act), f, 1.f, false, s));
+  gelu_kernel<<<elems_grid(rows * f), tpb, 0, s>>>(F(L.act), F(L.gl), rows * f);
+  RT_TRY(cudaGetLastError());
+
+  // ---- 2. the reverse loop: only d(k_j, v_j) accumulate here
+  RowmatParams rp;
+  memset(&rp, 0, sizeof(rp));
+  rp.B = B; rp.d = d; rp.dff = f; rp.eps = eps;
+  rp.z = z; rp.z_bs = xbs; rp.z_ts = xts; rp.dz = dz; rp.dz_bs = xbs; rp.dz_ts = xts;
+  rp.dK = F(L.dK); rp.dV = F(L.dV); rp.kraw = F(L.kraw); rp.h = F(L.h); rp.act = F(L.act);
+  rp.dkraw = F(L.dkraw); rp.dr = F(L.dr); rp.Gz = F(L.Gz); rp.dpre = F(L.dpre); rp.du = F(L.du); rp.dh = F(L.dh); rp.dc = F(L.dc);
+  const size_t smem_max = rowmat_smem(RM_PAIR, d) > rowmat_smem(RM_UP, f) ? rowmat_smem(RM_PAIR, d) : rowmat_smem(RM_UP, f);
+  if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
+  RT_TRY(cudaFuncSetAttribute(rowmat_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  const unsigned row_ctas = (unsigned)ceil_div(B, kRowsPerCta);
+  auto rowmat = [&](int mode, int i, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al) {
+    rp.mode = mode; rp.i = i; rp.K = K; rp.Ncols = Ncols; rp.W1 = W1; rp.W2 = W2; rp.gain = gain;
+    rp.norm_on = norm_on; rp.qk_on = qk ? 1 : 0; rp.alpha = al;
+    return launch_chained(rowmat_kernel<T>, dim3(Ncols / kRmCols, row_ctas), dim3(kRmThreads), rowmat_smem(mode, K), s, true, rp);
+  };
+  const int Lf = 64;                                             // leaf of the reverse schedule
+  for (int s0 = ((N - 1) / Lf) * Lf; s0 >= 0; s0 -= Lf) {
+    const int e0 = s0 + Lf < N ? s0 + Lf : N;
+    if (e0 < N) {                                                // Algorithm 1's tile at block end e0, backwards
+      const int P = e0 & -e0;
+      const int q1 = e0 + P < N ? e0 + P : N;
+      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, true, ab, e0, q1, e0 - P, e0, 0));
+    }
+    for (int i = e0 - 1; i >= s0; --i) {
+      RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f));
+      RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha));
+      RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f));
+      RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha));
+      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)(i - s0 + 1) * B * H)), dim3(tpb), 0, s, true, ab, i, i + 1,
+                            s0, i + 1, 1));
+    }
+  }
+
+  // ---- 3. everything else over all rows at once
+  attn_bwd_q_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
+  float* gprod = F(L.gprod);
+  float* part = F(L.part);
+  auto col_sum = [&](const float* a, int width, float* out, bool acc) {
+    col_partial_kernel<<<dim3(ceil_div(width, 128), kColParts), 128, 0, s>>>(a, rows, width, part, kColParts);
+    col_final_kernel<<<ceil_div(width, 128), 128, 0, s>>>(part, kColParts, width, out, acc ? 1 : 0);
+  };
+  // qkRMS backward of dq and of the temporary keys (in place), and their gain products
+  const bool want_gq = gr->g_q && w->g_q && qk, want_gk = gr->g_k && w->g_k && qk;
+  norm_bwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.dq), F(L.qraw), pbs, pts, B, g_q, nullptr, F(L.dq), pbs, pts,
+                                                                 want_gq ? gprod : nullptr, 0, rows, d, kHeadDim, eps, qk);
+  if (want_gq) col_sum(gprod, d, gr->g_q, false);
+  else if (gr->g_q) RT_TRY(cudaMemsetAsync(gr->g_q, 0, (size_t)d * 4, s));
+  norm_bwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.dkt), F(L.ktraw), pbs, pts, B, g_k, nullptr, F(L.dkt), pbs, pts,
+                                                                 want_gk ? gprod : nullptr, 0, rows, d, kHeadDim, eps, qk);
+  if (want_gk) {
+    norm_bwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.dK), F(L.kraw), pbs, pts, B, g_k, nullptr, nullptr, pbs, pts,
+                                                                   gprod, 1, rows, d, kHeadDim, eps, qk);
+    col_sum(gprod, d, gr->g_k, false);
+  } else if (gr->g_k) RT_TRY(cudaMemsetAsync(gr->g_k, 0, (size_t)d * 4, s));
+  // dn = dqraw W_q + dktraw W_k + dvt W_v;  dx = dh + RMS backward of dn through RMS(x)
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dq), d, 1, Wq, d, 1, F(L.dn), d, 1.f, false, s));
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dkt), d, 1, Wk, d, 1, F(L.dn), d, 1.f, true, s));
+  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dvt), d, 1, Wv, d, 1, F(L.dn), d, 1.f, true, s));
+  const bool want_ga = gr->g_attn && w->g_attn && pre;
+  norm_bwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.dn), x, xbs, xts, B, g_attn, F(L.dh), dx, xbs, xts,
+                                                         want_ga ? gprod : nullptr, 0, rows, d, d, eps, pre ? 1 : 0);
+  // gains of RMS(x) and RMS(z): one array when g_kv is not given (then RMS(z) uses g_attn)
+  const bool kv_alias = w->g_kv == nullptr;
+  if (want_ga) {
+    if (kv_alias && z_norm)
+      norm_bwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.dr), z, xbs, xts, B, g_kv, nullptr, nullptr, pbs, pts, gprod, 1, rows, d,
+                                                             d, eps, 1);
+    col_sum(gprod, d, gr->g_attn, false);
+  } else if (gr->g_attn) RT_TRY(cudaMemsetAsync(gr->g_attn, 0, (size_t)d * 4, s));
+  if (gr->g_kv) {
+    if (!kv_alias && z_norm) {
+      norm_bwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.dr), z, xbs, xts, B, g_kv, nullptr, nullptr, pbs, pts, gprod, 0, rows, d,
+                                                             d, eps, 1);
+      col_sum(gprod, d, gr->g_kv, false);
+    } else RT_TRY(cudaMemsetAsync(gr->g_kv, 0, (size_t)d * 4, s));
+  }
+  if (gr->g_mlp) {
+    if (w->g_mlp && pre) {
+      norm_bwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.du), F(L.h), pbs, pts, B, g_mlp, nullptr, nullptr, pbs, pts, gprod, 0,
+                                                                 rows, d, d, eps, 1);
+      col_sum(gprod, d, gr->g_mlp, false);
+    } else RT_TRY(cudaMemsetAsync(gr->g_mlp, 0, (size_t)d * 4, s));
+  }
+  // parameter matrices: dW[o, i] = sum_rows dY[row, o] X[row, i]
+  auto wgrad = [&](float* out, const float* dY, int n_out, const float* X, int n_in, float al, bool acc) {
+    return gemm<float, float>(n_out, n_in, (int)rows, dY, 1, n_out, X, n_in, 1, out, n_in, al, acc, s);
+  };
+  if (gr->w_q) RT_TRY(wgrad(gr->w_q, F(L.dq), d, F(L.n), d, 1.f, false));
+  if (gr->w_k) { RT_TRY(wgrad(gr->w_k, F(L.dkraw), d, F(L.r), d, 1.f, false)); RT_TRY(wgrad(gr->w_k, F(L.dkt), d, F(L.n), d, 1.f, true)); }
+  if (gr->w_v) { RT_TRY(wgrad(gr->w_v, F(L.dV), d, F(L.r), d, 1.f, false)); RT_TRY(wgrad(gr->w_v, F(L.dvt), d, F(L.n), d, 1.f, true)); }
+  if (gr->w_o) RT_TRY(wgrad(gr->w_o, F(L.dh), d, F(L.c), d, alpha, false));
+  if (gr->w_up) RT_TRY(wgrad(gr->w_up, F(L.dpre), f, F(L.u), d, 1.f, false));
+  if (gr->w_down) RT_TRY(wgrad(gr->w_down, F(L.Gz), d, F(L.gl), f, alpha, false));
+  RT_TRY(cudaGetLastError());
+  return RT_OK;
+}
+
+}  // namespace
+}  // namespace rt
+
+extern "C" {
+
+size_t rt_backward_workspace_bytes(const rt_config* cfg, int32_t B, int32_t N) {
+  if (!rt::bwd_config_ok(cfg) || B <= 0 || N <= 0) return 0;
+  return rt::bwd_layout(cfg, B, N).total;
+}
+
+rt_status rt_layer_backward(const rt_config* cfg, const rt_layer_weights* w, const void* x, const void* z, const float* dz,
+                            int32_t B, int32_t N, float* dx, const rt_layer_grads* grads, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+  using namespace rt;
+  if (!bwd_config_ok(cfg) || B <= 0 || N <= 0 || !workspace || ((uintptr_t)workspace & 15)) return RT_ERR_INVALID_ARG;
+  if (cfg->head_dim != kHeadDim || (cfg->norm_flags & RT_NORM_QK_FULL) || cfg->d_ff % 32 || cfg->recur_block > 1)
+    return RT_ERR_UNSUPPORTED;
+  if (!w || !w->w_q || !w->w_k || !w->w_v || !w->w_o || !w->w_up || !w->w_down || !x || !z || !dz || !dx || !grads)
+    return RT_ERR_INVALID_ARG;
+  if (((uintptr_t)x | (uintptr_t)z | (uintptr_t)dz | (uintptr_t)dx) & 15) return RT_ERR_INVALID_ARG;
+  if (workspace_bytes < bwd_layout(cfg, B, N).total) return RT_ERR_WORKSPACE;
+  if ((long long)B * N > 0x7fffffffLL / 2) return RT_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (cfg->dtype == RT_BF16)
+    return backward_impl<__nv_bfloat16>(cfg, w, (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, dz, B, N, dx, grads,
+                                        (unsigned char*)workspace, s);
+  return backward_impl<float>(cfg, w, (const float*)x, (const float*)z, dz, B, N, dx, grads, (unsigned char*)workspace, s);
+}
+
+}  // extern "C"

@@ -26,7 +26,7 @@ RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
            "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile", "rt_selftest_wait_expiry",
-           "rt_recompute_workspace_bytes", "rt_layer_recompute")
+           "rt_recompute_workspace_bytes", "rt_layer_recompute", "rt_backward_workspace_bytes", "rt_layer_backward")
 RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -40,6 +40,11 @@ class RtConfig(C.Structure):
 class RtLayerWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_q", "w_k", "w_v", "w_o", "w_up", "w_down",
                                            "g_attn", "g_mlp", "g_kv", "g_q", "g_k", "alibi_slopes")]
+
+
+class RtLayerGrads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_q", "w_k", "w_v", "w_o", "w_up", "w_down",
+                                           "g_attn", "g_mlp", "g_kv", "g_q", "g_k")]
 
 
 class RtCounters(C.Structure):
@@ -76,6 +81,10 @@ def _load():
     lib.rt_recompute_workspace_bytes.restype = Z
     lib.rt_recompute_workspace_bytes.argtypes = [C.POINTER(RtConfig), I, I]
     lib.rt_layer_recompute.restype = C.c_int
+    lib.rt_backward_workspace_bytes.restype = Z
+    lib.rt_backward_workspace_bytes.argtypes = [C.POINTER(RtConfig), I, I]
+    lib.rt_layer_backward.restype = C.c_int
+    lib.rt_layer_backward.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, P, P, I, I, P, C.POINTER(RtLayerGrads), P, Z, P]
     lib.rt_layer_recompute.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, P, I, I, P, P, P, I, P, Z, P]
     lib.rt_update_tile.restype = C.c_int
     lib.rt_update_tile.argtypes = [C.POINTER(RtConfig), P, P, P, P, P, P, I, I, I, I, I, I, I, P, P, P]
@@ -160,6 +169,14 @@ def rt_update_tile(cfg, q, k_cache, v_cache, st_o, st_m, st_l, B, rows_q, rows_k
 
 def rt_recompute_workspace_bytes(cfg: RtConfig, B: int, N: int) -> int:
     return int(_lib.rt_recompute_workspace_bytes(C.byref(cfg), B, N))
+
+
+def rt_backward_workspace_bytes(cfg: RtConfig, B: int, N: int) -> int:
+    return int(_lib.rt_backward_workspace_bytes(C.byref(cfg), B, N))
+
+
+def rt_layer_backward(cfg, w, x, z, dz, B, N, dx, grads, workspace, workspace_bytes, stream) -> int:
+    return _lib.rt_layer_backward(C.byref(cfg), C.byref(w), x, z, dz, B, N, dx, C.byref(grads), workspace, workspace_bytes, stream)
 
 
 def rt_layer_recompute(cfg, w, x, z_claim, B, N, z_out, k_cache, v_cache, N_max, workspace, workspace_bytes, stream) -> int:
@@ -322,6 +339,40 @@ class Layer:
         _check(self.status(), "rt_layer_recompute (device)")
         to_np = lambda t: t.to(torch.float64).cpu().numpy()
         return (to_np(zo), to_np(self.k_cache[:N].permute(1, 0, 2)), to_np(self.v_cache[:N].permute(1, 0, 2)))
+
+    def backward_device(self, x_dev, z_dev, dz_dev, dx_dev, grads: "RtLayerGrads", ws, stream=None) -> None:
+        """x_dev, z_dev [B,N,d] storage type, dz_dev, dx_dev [B,N,d] fp32, ws a uint8 workspace tensor (enqueue only)."""
+        torch = _torch()
+        B, N, _ = x_dev.shape
+        s = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
+        _check(rt_layer_backward(self.cfg, self.w, x_dev.data_ptr(), z_dev.data_ptr(), dz_dev.data_ptr(), B, N, dx_dev.data_ptr(),
+                                 grads, ws.data_ptr(), ws.numel(), s), "rt_layer_backward")
+
+    def backward(self, x, z, dz):
+        """x, z [B,N,d] (z = this layer's outputs), dz = dL/dz [B,N,d] -> dx [B,N,d] and a dict of parameter gradients
+        (fp64 numpy; one entry per parameter the layer has)."""
+        torch = _torch()
+        xd = _to_dev(x, self.dtype, self.device)
+        zd = _to_dev(z, self.dtype, self.device)
+        dzd = _to_dev(dz, "f32", self.device)
+        B, N, d = xd.shape
+        need = rt_backward_workspace_bytes(self.cfg, B, N)
+        if need == 0:
+            raise RtError(RT_ERR_INVALID_ARG, "rt_backward_workspace_bytes")
+        ws = torch.zeros(need, dtype=torch.uint8, device=self.device)
+        dxd = torch.empty((B, N, d), dtype=torch.float32, device=self.device)
+        grads, out = RtLayerGrads(), {}
+        shapes = {"w_up": (self.cfg.d_ff, d), "w_down": (d, self.cfg.d_ff)}
+        for n in _W_NAMES + _G_NAMES:
+            if n in _G_NAMES and not getattr(self.w, n):
+                continue
+            out[n] = torch.empty(shapes.get(n, (d, d) if n in _W_NAMES else (d,)), dtype=torch.float32, device=self.device)
+            setattr(grads, n, out[n].data_ptr())
+        self.backward_device(xd, zd, dzd, dxd, grads, ws)
+        torch.cuda.synchronize(self.device)
+        _check(rt_get_status(ws.data_ptr()), "rt_layer_backward (device)")
+        to_np = lambda t: t.to(torch.float64).cpu().numpy()
+        return to_np(dxd), {n: to_np(t) for n, t in out.items()}
 
     def decode(self, x_new, pos: int):
         """x_new [B,d] at position pos (caches must hold pos rows) -> z_new [B,d] fp64 numpy."""

@@ -1,0 +1,95 @@
+"""GPU parity of the layer's backward pass (rt_layer_backward; Sec. 6, "The backward pass") against the gradient
+oracle (reverse-mode differentiation of the plain definition, fp64) on identical seeded inputs."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+G_NAMES = ("g_attn", "g_mlp", "g_kv", "g_q", "g_k")
+
+
+def rel_err(got, ref):
+    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))
+
+
+def _case(dtype, d, H, dff, B, N, seed, gains, alibi):
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("bwd", 1, B, N, d, H, dff, dtype)
+    data = inputs.make_inputs(wl, seed=seed)
+    lw = data["layers"][0]
+    rng = np.random.default_rng(seed + 1)
+    for g in gains:
+        lw[g] = inputs.round_to(1.0 + 0.2 * rng.standard_normal(d), dtype)
+    slopes = np.array([2.0 ** (-8.0 * (h + 1) / H) for h in range(H)]) if alibi else None
+    dz = rng.standard_normal(data["x"].shape).astype(np.float32).astype(np.float64)
+    return data["x"], lw, slopes, dz
+
+
+@pytest.mark.parametrize("dtype,d,H,dff,B,N,flags,gains,alibi,alpha", [
+    ("f32", 128, 2, 256, 2, 150, 3, (), False, 1.0),                         # three leaves, ragged last one
+    ("f32", 192, 3, 224, 3, 77, 3 | 8, G_NAMES, True, 0.5),                 # every gain, ALiBi, persistent pair from z itself
+    ("f32", 128, 2, 256, 1, 64, 0, (), False, 1.0),                          # no norms, one full leaf
+    ("f32", 128, 2, 128, 6, 70, 1, ("g_attn", "g_mlp"), False, 0.7),         # no qkRMS; RMS(z) shares g_attn; ragged row chunk
+    ("f32", 64, 1, 96, 5, 1, 3, G_NAMES, False, 1.0),                        # a single position
+    ("f32", 128, 2, 256, 2, 300, 3, ("g_k", "g_kv"), True, 1.0),             # cross tiles of 64, 128 and 256 keys
+    ("bf16", 256, 4, 512, 3, 200, 3, G_NAMES, False, 1.0),
+    ("bf16", 128, 2, 384, 9, 130, 3, (), True, 0.6)])
+def test_backward_matches_gradient_oracle(dtype, d, H, dff, B, N, flags, gains, alibi, alpha):
+    from oracle import RTConfig, RTWeights, layer_grad
+    from paper_2604_21215_b200 import inputs, rt
+    x, lw, slopes, dz = _case(dtype, d, H, dff, B, N, 7700 + N, gains, alibi)
+    cfg = RTConfig(d, H, 64, dff, norm_flags=flags, residual_scale=alpha, alibi_slopes=slopes)
+    z_ref, dx_ref, g_ref = layer_grad(cfg, RTWeights(**lw), x, dz)
+    layer = rt.Layer(d, H, dff, dtype=dtype, norm_flags=flags, residual_scale=alpha)
+    layer.set_weights(dict(lw, alibi_slopes=slopes) if alibi else lw)
+    dx, g = layer.backward(x, inputs.round_to(z_ref, dtype), dz)
+    tol = TOL[dtype]
+    assert np.isfinite(dx).all()
+    assert rel_err(dx, dx_ref) <= tol, ("dx", rel_err(dx, dx_ref))
+    want = {"w_q", "w_k", "w_v", "w_o", "w_up", "w_down"} | set(gains)
+    assert set(g) == want
+    for name in sorted(want):
+        if np.abs(g_ref[name]).max() == 0.0:                                  # e.g. g_q without qkRMS
+            assert np.abs(g[name]).max() == 0.0, name
+            continue
+        assert rel_err(g[name], g_ref[name]) <= tol, (name, rel_err(g[name], g_ref[name]))
+
+
+def test_backward_from_the_prefill_outputs_and_determinism():
+    # z as the GPU's own prefill returned it (what a training step has at hand); two runs agree bit for bit
+    from oracle import RTConfig, RTWeights, layer_grad
+    from paper_2604_21215_b200 import rt
+    d, H, dff, B, N = 128, 2, 256, 4, 200
+    x, lw, _, dz = _case("f32", d, H, dff, B, N, 31, ("g_attn", "g_kv"), False)
+    layer = rt.Layer(d, H, dff, dtype="f32")
+    layer.set_weights(lw)
+    z, _, _ = layer.prefill(x)
+    dx1, g1 = layer.backward(x, z, dz)
+    dx2, g2 = layer.backward(x, z, dz)
+    assert np.array_equal(dx1, dx2) and all(np.array_equal(g1[n], g2[n]) for n in g1)
+    _, dx_ref, g_ref = layer_grad(RTConfig(d, H, 64, dff), RTWeights(**lw), x, dz)
+    assert rel_err(dx1, dx_ref) <= TOL["f32"]
+    for n in g1:
+        assert rel_err(g1[n], g_ref[n]) <= TOL["f32"], n
+
+
+def test_backward_argument_errors():
+    import torch
+    from paper_2604_21215_b200 import rt
+    x, lw, _, dz = _case("f32", 128, 2, 256, 1, 8, 1, (), False)
+    layer = rt.Layer(128, 2, 256, dtype="f32")
+    layer.set_weights(lw)
+    xd = torch.zeros((1, 8, 128), device="cuda"); zd = torch.zeros_like(xd); dzd = torch.zeros_like(xd); dxd = torch.zeros_like(xd)
+    need = rt.rt_backward_workspace_bytes(layer.cfg, 1, 8)
+    assert need > 0
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    gr = rt.RtLayerGrads()
+    call = lambda x_, nbytes, cfg=layer.cfg: rt.rt_layer_backward(cfg, layer.w, x_, zd.data_ptr(), dzd.data_ptr(), 1, 8, dxd.data_ptr(),
+                                                                  gr, ws.data_ptr(), nbytes, 0)
+    assert call(xd.data_ptr(), need) == rt.RT_OK                               # no parameter gradient requested: dx only
+    assert call(None, need) == rt.RT_ERR_INVALID_ARG
+    assert call(xd.data_ptr(), need - 1) == rt.RT_ERR_WORKSPACE
+    blocked = rt.make_config(128, 2, 256, dtype="f32", recur_block=4)
+    assert call(xd.data_ptr(), need, blocked) == rt.RT_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
