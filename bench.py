@@ -575,6 +575,77 @@ def run_recompute_bench(args):
     return 0
 
 
+def run_backward_bench(args):
+    """Times rt_layer_backward (Sec. 6, the backward pass: parallel sweep of the intermediates, reverse loop over the
+    positions, batched products) next to the forward pass on the workload's single-layer shape; one JSON object."""
+    import dataclasses
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    wl = get_workload(args.workload, args.batch)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    if wl.vocab:
+        wl = dataclasses.replace(wl, vocab=0, n_layers=1)
+    data = inputs.make_inputs(wl)
+    lw = data["layers"][0]
+    if args.alibi:
+        lw["alibi_slopes"] = alibi_slopes(wl.n_heads)
+    layer = rt.Layer(wl.d_model, wl.n_heads, wl.d_ff, dtype=wl.dtype, residual_scale=wl.residual_scale)
+    layer.set_weights(lw)
+    layer.reserve(wl.B, wl.N)
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    d, f = wl.d_model, wl.d_ff
+    x = torch.from_numpy(data["x"]).to(tdt).to(dev)
+    z = torch.empty_like(x)
+    g = torch.Generator(device=dev); g.manual_seed(BASE_TILE_SEED + 3)
+    dz = torch.randn(x.shape, generator=g, device=dev, dtype=torch.float32)
+    dx = torch.empty_like(dz)
+    ws = torch.zeros(rt.rt_backward_workspace_bytes(layer.cfg, wl.B, wl.N), dtype=torch.uint8, device=dev)
+    grads, keep = rt.RtLayerGrads(), []
+    for n, shape in (("w_q", (d, d)), ("w_k", (d, d)), ("w_v", (d, d)), ("w_o", (d, d)), ("w_up", (f, d)), ("w_down", (d, f))):
+        keep.append(torch.empty(shape, dtype=torch.float32, device=dev))
+        setattr(grads, n, keep[-1].data_ptr())
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def timed(fn):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize(dev)
+        evs = []
+        for _ in range(args.steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        return sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+
+    fwd_ms = timed(lambda: layer.prefill_device(x, z))
+    assert layer.status() == rt.RT_OK
+    bwd = lambda: layer.backward_device(x, z, dz, dx, grads, ws)
+    bwd_ms = timed(bwd)
+    rt.rt_profile_enable(True)
+    rt.rt_profile_read()
+    bwd(); torch.cuda.synchronize(dev)
+    prof = rt.rt_profile_read()
+    rt.rt_profile_enable(False)
+    assert rt.rt_get_status(ws.data_ptr()) == rt.RT_OK and bool(torch.isfinite(dx).all())
+    tok = wl.B * wl.N
+    # products of the backward pass proper (twice the forward's) plus the recomputed forward products
+    flops_fwd = 12.0 * tok * d * d + 4.0 * tok * d * f + 2.0 * wl.B * d * wl.N * (wl.N + 1)
+    print(json.dumps({"backward_bench": wl.name, "B": wl.B, "N": wl.N, "d_model": d, "d_ff": f, "dtype": wl.dtype,
+                      "alibi": bool(args.alibi), "forward_ms": fwd_ms, "backward_ms": bwd_ms,
+                      "backward_tokens_per_s": tok / (bwd_ms * 1e-3), "backward_over_forward": bwd_ms / fwd_ms,
+                      "us_per_position_reverse_loop": prof["leaf"]["ms"] * 1e3 / wl.N,
+                      "gflop": 3.0 * flops_fwd / 1e9, "tflops": 3.0 * flops_fwd / (bwd_ms * 1e-3) / 1e12,
+                      "arithmetic": "fp32 on CUDA cores",
+                      "ms_by_phase": {"sweep_of_intermediates": prof["prepass"]["ms"], "reverse_loop_steps": prof["leaf"]["ms"],
+                                      "reverse_loop_tiles": prof["tile"]["ms"], "products_over_all_rows": prof["other"]["ms"]},
+                      "workspace_gb": ws.numel() / 1e9}))
+    return 0
+
+
 BASE_TILE_SEED = 20260421
 
 
@@ -599,6 +670,7 @@ def main():
     ap.add_argument("--recompute-bench", action="store_true",
                     help="time rt_layer_recompute (parallel sweep given the outputs) and exit")
     ap.add_argument("--decode-bench", action="store_true", help="time rt_decode_step at several cache lengths and exit")
+    ap.add_argument("--backward-bench", action="store_true", help="time rt_layer_backward next to the forward pass and exit")
     args = ap.parse_args()
     if args.tile_bench:
         return run_tile_bench(args)
@@ -606,6 +678,8 @@ def main():
         return run_decode_bench(args)
     if args.recompute_bench:
         return run_recompute_bench(args)
+    if args.backward_bench:
+        return run_backward_bench(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_cuda(args)

@@ -399,6 +399,11 @@ rt_status common_checks(const rt_config* c, int B, int N, int n_layers, void* ws
 
 }  // namespace
 
+namespace rt {
+ProfSpanScope::ProfSpanScope(cudaStream_t s, int cls) { impl = new ProfScope(s, cls); }
+ProfSpanScope::~ProfSpanScope() { delete static_cast<ProfScope*>(impl); }
+}  // namespace rt
+
 extern "C" {
 
 size_t rt_workspace_bytes(const rt_config* cfg, int32_t B, int32_t N, int32_t n_layers) {

@@ -13,6 +13,7 @@
 #include <string.h>
 
 #include "rt_common.cuh"
+#include "rt_kernels.h"
 
 namespace rt {
 namespace {
@@ -546,6 +547,9 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   RT_TRY(cudaMemsetAsync(ws + L.zero_begin, 0, L.zero_end - L.zero_begin, s));
 
   // ---- 1. the parallel sweep: every intermediate of the forward pass from x and z
+  AttnBufs ab;
+  {
+  ProfSpanScope span(s, 0);
   norm_fwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(x, xbs, xts, B, g_attn, F(L.n), rows, d, d, eps, pre ? 1 : 0);
   RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wq, 1, d, F(L.qraw), d, 1.f, false, s));
   RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wk, 1, d, F(L.ktraw), d, 1.f, false, s));
@@ -556,7 +560,6 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wk, 1, d, F(L.kraw), d, 1.f, false, s));
   RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wv, 1, d, F(L.v), d, 1.f, false, s));
   norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.kraw), pbs, pts, B, g_k, F(L.k), rows, d, kHeadDim, eps, qk);
-  AttnBufs ab;
   memset(&ab, 0, sizeof(ab));
   ab.q = F(L.q); ab.k = F(L.k); ab.v = F(L.v); ab.kt = F(L.kt); ab.vt = F(L.vt); ab.lse = F(L.lse); ab.D = F(L.D);
   ab.c = F(L.c); ab.dc = F(L.dc); ab.dK = F(L.dK); ab.dV = F(L.dV); ab.dkt = F(L.dkt); ab.dvt = F(L.dvt); ab.dq = F(L.dq);
@@ -569,6 +572,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   RT_TRY(gemm<float, T>((int)rows, f, d, F(L.u), d, 1, Wup, 1, d, F(L.act), f, 1.f, false, s));
   gelu_kernel<<<elems_grid(rows * f), tpb, 0, s>>>(F(L.act), F(L.gl), rows * f);
   RT_TRY(cudaGetLastError());
+  }
 
   // ---- 2. the reverse loop: only d(k_j, v_j) accumulate here
   RowmatParams rp;
@@ -592,8 +596,10 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     if (e0 < N) {                                                // Algorithm 1's tile at block end e0, backwards
       const int P = e0 & -e0;
       const int q1 = e0 + P < N ? e0 + P : N;
+      ProfSpanScope span(s, 2);
       RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, true, ab, e0, q1, e0 - P, e0, 0));
     }
+    ProfSpanScope span(s, 1);
     for (int i = e0 - 1; i >= s0; --i) {
       RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f));
       RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha));
@@ -605,6 +611,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   }
 
   // ---- 3. everything else over all rows at once
+  ProfSpanScope span(s, 3);
   attn_bwd_q_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
   float* gprod = F(L.gprod);
   float* part = F(L.part);

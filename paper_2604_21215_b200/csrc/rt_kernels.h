@@ -128,4 +128,14 @@ cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, v
 cudaError_t rms_rows_f32_launch(int dtype, const float* h, const void* g, void* u, int rows, int d, float eps, int pre, cudaStream_t s,
                                 bool chained = false);
 
+// Event-pair span for rt_profile_enable / rt_profile_read from other translation units (classes: 0 sweeps / pre-pass,
+// 1 per-position steps, 2 attention tiles, 3 everything else).  Does nothing while profiling is off.
+struct ProfSpanScope {
+  void* impl = nullptr;
+  ProfSpanScope(cudaStream_t s, int cls);
+  ~ProfSpanScope();
+  ProfSpanScope(const ProfSpanScope&) = delete;
+  ProfSpanScope& operator=(const ProfSpanScope&) = delete;
+};
+
 }  // namespace rt
