@@ -231,6 +231,43 @@ __global__ void attn_stats_kernel(AttnBufs a) {
   if (lane == 0) a.lse[((long long)i * a.B + b) * a.H + h] = m + log2f(l);
 }
 
+// State of the reverse loop written earlier in the SAME (cooperative) kernel by other CTAs must not come from L1.
+template <bool COOP> __device__ __forceinline__ float ld_state(const float* p) { return COOP ? __ldcg(p) : *p; }
+template <bool COOP> __device__ __forceinline__ float2 ld_state2(const float* p) {
+  return COOP ? __ldcg(reinterpret_cast<const float2*>(p)) : *reinterpret_cast<const float2*>(p);
+}
+
+// In-leaf step of position i for one (key j in [s0, i], sequence, head), one warp: see attn_bwd_kv_kernel (self = 1).
+template <bool COOP>
+__device__ __forceinline__ void attn_self_task(const AttnBufs& a, int i, int j, int b, int h, int lane) {
+  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long rj = ((long long)j * a.B + b) * a.d + col;
+  const long long ri = ((long long)i * a.B + b) * a.d + col;
+  const long long si = ((long long)i * a.B + b) * a.H + h;
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  const float2 dc = ld_state2<COOP>(a.dc + ri);
+  const float2 cc = *reinterpret_cast<const float2*>(a.c + ri);
+  const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+  const float D = warp_sum(dc.x * cc.x + dc.y * cc.y);
+  const float lse = a.lse[si];
+  if (j == i) {
+    if (lane == 0) a.D[si] = D;
+    const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
+    const float2 vv = *reinterpret_cast<const float2*>(a.vt + ri);
+    const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - lse);
+    const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
+    *reinterpret_cast<float2*>(a.dkt + ri) = make_float2(ds * q.x, ds * q.y);
+    *reinterpret_cast<float2*>(a.dvt + ri) = make_float2(p * dc.x, p * dc.y);
+  } else {
+    const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
+    const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
+    const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - slope * (float)(i - j) - lse);
+    const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
+    float2 t = ld_state2<COOP>(a.dK + rj); t.x += ds * q.x; t.y += ds * q.y; *reinterpret_cast<float2*>(a.dK + rj) = t;
+    t = ld_state2<COOP>(a.dV + rj); t.x += p * dc.x; t.y += p * dc.y; *reinterpret_cast<float2*>(a.dV + rj) = t;
+  }
+}
+
 // Gradient of the pairs: one warp per (key j, sequence, head) holds k_j, v_j and sums over the queries [q0, q1):
 //   p = exp2(logit - lse_i), ds = p (<dc_i, v_j> - D_i), dk_j += scale ds q_i, dv_j += p dc_i.
 // self = 1 (the in-leaf step of position i = q0): keys [k0, i]; every warp computes D_i = <dc_i, c_i> itself, and the warp
@@ -245,32 +282,7 @@ __global__ void attn_bwd_kv_kernel(AttnBufs a, int q0, int q1, int k0, int k1, i
   const long long rj = ((long long)j * a.B + b) * a.d + col;
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
   if (self) {
-    const int i = q0;
-    const long long ri = ((long long)i * a.B + b) * a.d + col;
-    const long long si = ((long long)i * a.B + b) * a.H + h;
-    const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
-    const float2 cc = *reinterpret_cast<const float2*>(a.c + ri);
-    const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
-    const float D = warp_sum(dc.x * cc.x + dc.y * cc.y);
-    const float lse = a.lse[si];
-    if (j == i) {
-      if (lane == 0) a.D[si] = D;
-      const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
-      const float2 vv = *reinterpret_cast<const float2*>(a.vt + ri);
-      const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - lse);
-      const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
-      *reinterpret_cast<float2*>(a.dkt + ri) = make_float2(ds * q.x, ds * q.y);
-      *reinterpret_cast<float2*>(a.dvt + ri) = make_float2(p * dc.x, p * dc.y);
-    } else {
-      const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
-      const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
-      const float p = exp2f(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - slope * (float)(i - j) - lse);
-      const float ds = p * (warp_sum(dc.x * vv.x + dc.y * vv.y) - D) * a.scale;
-      float2* dk = reinterpret_cast<float2*>(a.dK + rj);
-      float2* dv = reinterpret_cast<float2*>(a.dV + rj);
-      float2 t = *dk; t.x += ds * q.x; t.y += ds * q.y; *dk = t;
-      t = *dv; t.x += p * dc.x; t.y += p * dc.y; *dv = t;
-    }
+    attn_self_task<false>(a, q0, j, b, h, lane);
     return;
   }
   const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
@@ -339,7 +351,7 @@ __global__ void attn_bwd_q_kernel(AttnBufs a) {
 // rows in1 (in2) are built by a prologue from the state of the reverse loop (mode), W = a weight matrix as stored
 // ([its outputs, its inputs] = [K, Ncols]: the transposed product of the forward pass, read row by row).
 enum { RM_PAIR = 1, RM_DOWN = 2, RM_UP = 3, RM_OUT = 4 };
-constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmCols = 32;
+constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmWarps = kRmThreads / 32, kRmCols = 16;
 struct RowmatParams {
   int mode, B, d, dff, i, K, Ncols;
   int norm_on, qk_on;                     // whether the prologue's RMS / qkRMS is active
@@ -351,31 +363,31 @@ struct RowmatParams {
   float *dkraw, *dr, *Gz, *dpre, *du, *dh, *dc;
 };
 
-template <typename T>
-__global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p) {
-  grid_dep_sync();
-  extern __shared__ __align__(16) float smem[];
+// One task: the columns [cx*16, cx*16+16) of the product for the sequences [cy*4, cy*4+4).  All threads of the CTA.
+template <typename T, bool COOP>
+__device__ void rowmat_body(const RowmatParams& p, int cx, int cy, float* smem) {
   float* in1 = smem;                                        // [K][4]
   float* in2 = in1 + (size_t)p.K * kRowsPerCta;             // [K][4] (RM_PAIR only)
-  float* red = in2 + (p.mode == RM_PAIR ? (size_t)p.K * kRowsPerCta : 0);   // [16][32][4]
+  float* red = in2 + (p.mode == RM_PAIR ? (size_t)p.K * kRowsPerCta : 0);   // [16 warps][16 cols][4]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b0 = blockIdx.y * kRowsPerCta;
-  const bool writer = blockIdx.x == 0;
+  const int b0 = cy * kRowsPerCta;
+  const bool writer = cx == 0;
   const int d = p.d;
   const T* gain = reinterpret_cast<const T*>(p.gain);
+  __syncthreads();                                          // shared memory of the previous task is free
 
-  // ---- prologue: the input rows of this CTA's sequences, transposed into shared memory
+  // ---- prologue: the input rows of this task's sequences, transposed into shared memory
   if (p.mode == RM_PAIR) {
     // in1 = qkRMS backward of dK_i through k_i = qkRMS(kraw_i) per head; in2 = dV_i
     const int H = d / kHeadDim;
-    for (int task = warp; task < kRowsPerCta * H; task += kRmThreads / 32) {
+    for (int task = warp; task < kRowsPerCta * H; task += kRmWarps) {
       const int r = task / H, h = task % H, b = b0 + r;
       const int c0 = h * kHeadDim;
       float o0 = 0.f, o1 = 0.f, v0 = 0.f, v1 = 0.f;
       if (b < p.B) {
         const long long at = ((long long)p.i * p.B + b) * d + c0;
-        const float dy0 = p.dK[at + lane], dy1 = p.dK[at + lane + 32];
-        v0 = p.dV[at + lane]; v1 = p.dV[at + lane + 32];
+        const float dy0 = ld_state<COOP>(p.dK + at + lane), dy1 = ld_state<COOP>(p.dK + at + lane + 32);
+        v0 = ld_state<COOP>(p.dV + at + lane); v1 = ld_state<COOP>(p.dV + at + lane + 32);
         if (p.qk_on) {
           const float u0 = p.kraw[at + lane], u1 = p.kraw[at + lane + 32];
           const float g0 = gain_at(gain, c0 + lane), g1 = gain_at(gain, c0 + lane + 32);
@@ -389,55 +401,61 @@ __global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p
       in2[(c0 + lane) * kRowsPerCta + r] = v0; in2[(c0 + lane + 32) * kRowsPerCta + r] = v1;
     }
   } else if (p.mode == RM_UP) {
+#pragma unroll 4
     for (int idx = threadIdx.x; idx < kRowsPerCta * p.K; idx += kRmThreads) {
       const int r = idx / p.K, k = idx % p.K, b = b0 + r;
-      in1[k * kRowsPerCta + r] = b < p.B ? p.dpre[((long long)p.i * p.B + b) * p.K + k] : 0.f;
+      in1[k * kRowsPerCta + r] = b < p.B ? ld_state<COOP>(p.dpre + ((long long)p.i * p.B + b) * p.K + k) : 0.f;
     }
   } else {
     // RM_DOWN: Gz = dz_i + RMS backward of dr_i through RMS(z_i);  RM_OUT: dh = Gz_i + RMS backward of du_i through RMS(h_i)
+    // four warps per row: each takes a quarter of the row, the two sums meet in shared memory
     const T* zT = reinterpret_cast<const T*>(p.z);
-    for (int r = warp; r < kRowsPerCta; r += kRmThreads / 32) {
-      const int b = b0 + r;
-      if (b >= p.B) {
-        for (int e = lane; e < d; e += 32) in1[e * kRowsPerCta + r] = 0.f;
-        continue;
+    const int r = warp >> 2, part = warp & 3, b = b0 + r;
+    const int e_lo = part * (d / 4), e_hi = e_lo + d / 4;
+    const long long at = ((long long)p.i * p.B + (b < p.B ? b : 0)) * d;
+    const float* dy = (p.mode == RM_DOWN ? p.dr : p.du) + at;
+    const T* zr = zT + (long long)(b < p.B ? b : 0) * p.z_bs + (long long)p.i * p.z_ts;
+    float ss = 0.f, tu = 0.f;
+    if (p.norm_on && b < p.B) {
+#pragma unroll 4
+      for (int e = e_lo + lane; e < e_hi; e += 32) {
+        const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
+        ss = fmaf(u, u, ss);
+        tu = fmaf(ld_state<COOP>(dy + e) * gain_at(gain, e), u, tu);
       }
-      const long long at = ((long long)p.i * p.B + b) * d;
-      const float* dy = (p.mode == RM_DOWN ? p.dr : p.du) + at;
-      const float* addv = p.mode == RM_DOWN ? p.dz + (long long)b * p.dz_bs + (long long)p.i * p.dz_ts : p.Gz + at;
-      const T* zr = zT + (long long)b * p.z_bs + (long long)p.i * p.z_ts;
-      float* keep = (p.mode == RM_DOWN ? p.Gz : p.dh) + at;
-      float ss = 0.f, tu = 0.f;
-      if (p.norm_on) {
-        for (int e = lane; e < d; e += 32) {
-          const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
-          ss = fmaf(u, u, ss);
-          tu = fmaf(dy[e] * gain_at(gain, e), u, tu);
-        }
-        ss = warp_sum(ss); tu = warp_sum(tu);
-      }
-      const float inv = rsqrtf(ss / d + p.eps), mean = tu * inv / d;
-      for (int e = lane; e < d; e += 32) {
-        float du = dy[e];
+      ss = warp_sum(ss); tu = warp_sum(tu);
+    }
+    if (lane == 0) { red[warp * 2] = ss; red[warp * 2 + 1] = tu; }
+    __syncthreads();
+    ss = red[(r * 4) * 2] + red[(r * 4 + 1) * 2] + red[(r * 4 + 2) * 2] + red[(r * 4 + 3) * 2];
+    tu = red[(r * 4) * 2 + 1] + red[(r * 4 + 1) * 2 + 1] + red[(r * 4 + 2) * 2 + 1] + red[(r * 4 + 3) * 2 + 1];
+    const float inv = rsqrtf(ss / d + p.eps), mean = tu * inv / d;
+    const float* addv = p.mode == RM_DOWN ? p.dz + (long long)(b < p.B ? b : 0) * p.dz_bs + (long long)p.i * p.dz_ts : p.Gz + at;
+    float* keep = (p.mode == RM_DOWN ? p.Gz : p.dh) + at;
+#pragma unroll 4
+    for (int e = e_lo + lane; e < e_hi; e += 32) {
+      float val = 0.f;
+      if (b < p.B) {
+        float du = ld_state<COOP>(dy + e);
         if (p.norm_on) {
           const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
-          du = inv * (dy[e] * gain_at(gain, e) - u * inv * mean);
+          du = inv * (du * gain_at(gain, e) - u * inv * mean);
         }
-        const float val = addv[e] + du;
-        in1[e * kRowsPerCta + r] = val;
+        val = (p.mode == RM_DOWN ? addv[e] : ld_state<COOP>(addv + e)) + du;
         if (writer) keep[e] = val;
       }
+      in1[e * kRowsPerCta + r] = val;
     }
   }
   __syncthreads();
 
-  // ---- product: this CTA's 32 columns; a warp's lanes = 4 rows of W x 8 groups of 4 columns
-  const int kq = lane >> 3, cq = lane & 7;
-  const int n0 = blockIdx.x * kRmCols + 4 * cq;
+  // ---- product: 16 columns per task; a warp's lanes = 8 rows of W x 4 groups of 4 columns
+  const int kq = lane >> 2, cq = lane & 3;
+  const int n0 = cx * kRmCols + 4 * cq;
   float acc[kRowsPerCta][4] = {};
   auto run = [&](const T* W, const float* in) {
-#pragma unroll 4
-    for (int k = warp * 4 + kq; k < p.K; k += (kRmThreads / 32) * 4) {
+#pragma unroll 8
+    for (int k = warp * 8 + kq; k < p.K; k += kRmWarps * 8) {
       Vec4<T> wv;
       wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols + n0);
       float wf[4];
@@ -457,6 +475,7 @@ __global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float v = acc[r][c];
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 16);
       if (kq == 0) red[(warp * kRmCols + 4 * cq + c) * kRowsPerCta + r] = v;
@@ -464,23 +483,72 @@ __global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p
   __syncthreads();
   if (threadIdx.x < kRmCols * kRowsPerCta) {
     const int col = threadIdx.x >> 2, r = threadIdx.x & 3, b = b0 + r;
-    float s = 0.f;
+    float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRmThreads / 32; ++w) s += red[(w * kRmCols + col) * kRowsPerCta + r];
+    for (int w = 0; w < kRmWarps; ++w) sum += red[(w * kRmCols + col) * kRowsPerCta + r];
     if (b < p.B) {
-      const int n = blockIdx.x * kRmCols + col;
+      const int n = cx * kRmCols + col;
       const long long at = ((long long)p.i * p.B + b) * p.Ncols + n;
-      s *= p.alpha;
-      if (p.mode == RM_PAIR) p.dr[at] = s;
-      else if (p.mode == RM_DOWN) p.dpre[at] = s * gelu_grad_f(p.act[at]);
-      else if (p.mode == RM_UP) p.du[at] = s;
-      else p.dc[at] = s;
+      sum *= p.alpha;
+      if (p.mode == RM_PAIR) p.dr[at] = sum;
+      else if (p.mode == RM_DOWN) p.dpre[at] = sum * gelu_grad_f(p.act[at]);
+      else if (p.mode == RM_UP) p.du[at] = sum;
+      else p.dc[at] = sum;
     }
   }
 }
 
+template <typename T>
+__global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p) {
+  grid_dep_sync();
+  extern __shared__ __align__(16) float smem[];
+  rowmat_body<T, false>(p, blockIdx.x, blockIdx.y, smem);
+}
+
 size_t rowmat_smem(int mode, int K) {
-  return ((size_t)K * kRowsPerCta * (mode == RM_PAIR ? 2 : 1) + (kRmThreads / 32) * kRmCols * kRowsPerCta) * sizeof(float);
+  return ((size_t)K * kRowsPerCta * (mode == RM_PAIR ? 2 : 1) + kRmWarps * kRmCols * kRowsPerCta) * sizeof(float);
+}
+
+// The reverse loop over one leaf [s0, e0) as ONE cooperative kernel: the five steps of a position separated by grid
+// barriers instead of kernel boundaries.  Every wait is bounded (grid_barrier); when one runs out the kernel returns.
+struct LoopParams {
+  const void *Wk, *Wv, *Wdn, *Wup, *Wo, *g_k, *g_kv, *g_mlp;
+  int z_norm, pre, qk;
+  float alpha;
+  int s0, e0;
+  unsigned bar_base;
+  SyncArea* sync;
+};
+constexpr int kLoopBarriersPerPosition = 5;
+
+template <typename T>
+__global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p, const LoopParams lp, const AttnBufs a) {
+  extern __shared__ __align__(16) float smem[];
+  __shared__ int s_flag;
+  unsigned target = lp.bar_base;
+  const int chunks = (p.B + kRowsPerCta - 1) / kRowsPerCta;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  p.qk_on = lp.qk;
+  auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al) {
+    p.mode = mode; p.K = K; p.Ncols = Ncols; p.W1 = W1; p.W2 = W2; p.gain = gain; p.norm_on = norm_on; p.alpha = al;
+    const int nx = Ncols / kRmCols;
+    for (int t = blockIdx.x; t < nx * chunks; t += gridDim.x) rowmat_body<T, true>(p, t % nx, t / nx, smem);
+  };
+  for (int i = lp.e0 - 1; i >= lp.s0; --i) {
+    p.i = i;
+    phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f);
+    if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    phase(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.g_kv, lp.z_norm, lp.alpha);
+    if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f);
+    if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha);
+    if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    const int tasks = (i - lp.s0 + 1) * a.B * a.H;
+    for (int t = blockIdx.x * kRmWarps + warp; t < tasks; t += gridDim.x * kRmWarps)
+      attn_self_task<true>(a, i, lp.s0 + t / (a.B * a.H), (t / a.H) % a.B, t % a.H, lane);
+    if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ workspace
@@ -590,6 +658,20 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     rp.norm_on = norm_on; rp.qk_on = qk ? 1 : 0; rp.alpha = al;
     return launch_chained(rowmat_kernel<T>, dim3(Ncols / kRmCols, row_ctas), dim3(kRmThreads), rowmat_smem(mode, K), s, true, rp);
   };
+  // one cooperative launch per leaf when a CTA per SM can be resident; else one launch per step
+  int dev = 0, sms = 0, per_sm = 0, coop = 0;
+  RT_TRY(cudaGetDevice(&dev));
+  RT_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  RT_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+  RT_TRY(cudaFuncSetAttribute(bwd_loop_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
+  RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_loop_kernel<T>, kRmThreads, smem_max));
+  const bool use_coop = coop && per_sm >= 1;
+  LoopParams lp;
+  memset(&lp, 0, sizeof(lp));
+  lp.Wk = Wk; lp.Wv = Wv; lp.Wdn = Wdn; lp.Wup = Wup; lp.Wo = Wo; lp.g_k = g_k; lp.g_kv = g_kv; lp.g_mlp = g_mlp;
+  lp.z_norm = z_norm ? 1 : 0; lp.pre = pre ? 1 : 0; lp.qk = qk ? 1 : 0; lp.alpha = alpha;
+  lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
+  unsigned bar_base = 0;
   const int Lf = 64;                                             // leaf of the reverse schedule
   for (int s0 = ((N - 1) / Lf) * Lf; s0 >= 0; s0 -= Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
@@ -597,9 +679,17 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
       const int P = e0 & -e0;
       const int q1 = e0 + P < N ? e0 + P : N;
       ProfSpanScope span(s, 2);
-      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, true, ab, e0, q1, e0 - P, e0, 0));
+      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop, ab, e0, q1, e0 - P,
+                            e0, 0));
     }
     ProfSpanScope span(s, 1);
+    if (use_coop) {
+      lp.s0 = s0; lp.e0 = e0; lp.bar_base = bar_base;
+      void* args[] = {(void*)&rp, (void*)&lp, (void*)&ab};
+      RT_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&bwd_loop_kernel<T>), dim3(sms), dim3(kRmThreads), args, smem_max, s));
+      bar_base += (unsigned)(e0 - s0) * kLoopBarriersPerPosition * (unsigned)sms;
+      continue;
+    }
     for (int i = e0 - 1; i >= s0; --i) {
       RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f));
       RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha));
