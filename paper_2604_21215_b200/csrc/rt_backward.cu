@@ -351,149 +351,207 @@ __global__ void attn_bwd_q_kernel(AttnBufs a) {
 // rows in1 (in2) are built by a prologue from the state of the reverse loop (mode), W = a weight matrix as stored
 // ([its outputs, its inputs] = [K, Ncols]: the transposed product of the forward pass, read row by row).
 enum { RM_PAIR = 1, RM_DOWN = 2, RM_UP = 3, RM_OUT = 4 };
-constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmWarps = kRmThreads / 32, kRmCols = 16;
+constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmWarps = kRmThreads / 32;
 struct RowmatParams {
   int mode, B, d, dff, i, K, Ncols;
+  int cols;                               // columns per task: 16 or 32
+  int nsplit;                             // RM_PAIR: 2 (task 0 = W_k with dk, task 1 = W_v with dv); RM_UP: parts of the contraction
   int norm_on, qk_on;                     // whether the prologue's RMS / qkRMS is active
+  int n_in;                               // partial sums the prologue adds up (RM_DOWN: 2, RM_OUT: RM_UP's nsplit)
   float eps, alpha;
   const void *W1, *W2, *gain;             // storage type
   const void* z; long long z_bs, z_ts;    // layer output [B,N,d], storage type (RM_DOWN)
   const float* dz; long long dz_bs, dz_ts;
   const float *dK, *dV, *kraw, *h, *act;
+  float* part;                            // [4][B][d] partial sums of the split products (RM_PAIR, RM_UP), summed by the next step
   float *dkraw, *dr, *Gz, *dpre, *du, *dh, *dc;
 };
+inline int rowmat_tasks(const RowmatParams& p) { return (p.Ncols / p.cols) * ((p.B + kRowsPerCta - 1) / kRowsPerCta) * p.nsplit; }
 
-// One task: the columns [cx*16, cx*16+16) of the product for the sequences [cy*4, cy*4+4).  All threads of the CTA.
+// One task: `cols` columns of the product for four sequences and one part of a split contraction.  All threads of the CTA.
+// Task index t = ((cy * nx) + cx) * nsplit + sp.
 template <typename T, bool COOP>
-__device__ void rowmat_body(const RowmatParams& p, int cx, int cy, float* smem) {
-  float* in1 = smem;                                        // [K][4]
-  float* in2 = in1 + (size_t)p.K * kRowsPerCta;             // [K][4] (RM_PAIR only)
-  float* red = in2 + (p.mode == RM_PAIR ? (size_t)p.K * kRowsPerCta : 0);   // [16 warps][16 cols][4]
+__device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
+  const int nx = p.Ncols / p.cols;
+  const int sp = t % p.nsplit, cx = (t / p.nsplit) % nx, cy = t / (p.nsplit * nx);
+  const int d = p.d;
+  const int Kin = p.mode == RM_UP ? p.K / p.nsplit : p.K;   // input entries per row this task needs
+  const int k_base = p.mode == RM_UP ? sp * Kin : 0;
+  float* in = smem;                                         // [Kin][4] the product's input rows, transposed
+  float* st1 = in + (size_t)Kin * kRowsPerCta;              // [Kin][4] staging (u of the RMS backward)
+  float* st2 = st1 + (size_t)Kin * kRowsPerCta;             // [Kin][4] staging (the term added)
+  float* red = st2 + (size_t)Kin * kRowsPerCta;             // [16 warps][cols][4]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b0 = cy * kRowsPerCta;
-  const bool writer = cx == 0;
-  const int d = p.d;
+  const bool writer = cx == 0 && sp == 0;
   const T* gain = reinterpret_cast<const T*>(p.gain);
+  const long long part_stride = (long long)p.B * d;
   __syncthreads();                                          // shared memory of the previous task is free
 
   // ---- prologue: the input rows of this task's sequences, transposed into shared memory
   if (p.mode == RM_PAIR) {
-    // in1 = qkRMS backward of dK_i through k_i = qkRMS(kraw_i) per head; in2 = dV_i
-    const int H = d / kHeadDim;
-    for (int task = warp; task < kRowsPerCta * H; task += kRmWarps) {
-      const int r = task / H, h = task % H, b = b0 + r;
-      const int c0 = h * kHeadDim;
-      float o0 = 0.f, o1 = 0.f, v0 = 0.f, v1 = 0.f;
-      if (b < p.B) {
-        const long long at = ((long long)p.i * p.B + b) * d + c0;
-        const float dy0 = ld_state<COOP>(p.dK + at + lane), dy1 = ld_state<COOP>(p.dK + at + lane + 32);
-        v0 = ld_state<COOP>(p.dV + at + lane); v1 = ld_state<COOP>(p.dV + at + lane + 32);
-        if (p.qk_on) {
-          const float u0 = p.kraw[at + lane], u1 = p.kraw[at + lane + 32];
-          const float g0 = gain_at(gain, c0 + lane), g1 = gain_at(gain, c0 + lane + 32);
-          const float ss = warp_sum(u0 * u0 + u1 * u1), tu = warp_sum(dy0 * g0 * u0 + dy1 * g1 * u1);
-          const float inv = rsqrtf(ss / kHeadDim + p.eps), mean = tu * inv / kHeadDim;
-          o0 = inv * (dy0 * g0 - u0 * inv * mean); o1 = inv * (dy1 * g1 - u1 * inv * mean);
-        } else { o0 = dy0; o1 = dy1; }
-        if (writer) { p.dkraw[at + lane] = o0; p.dkraw[at + lane + 32] = o1; }
+    // task 0: qkRMS backward of dK_i through k_i = qkRMS(kraw_i) per head;  task 1: dV_i as it is
+    // (loads of a batch first, stores after: the round trips to L2 overlap instead of queueing behind the stores)
+    const float* src = sp ? p.dV : p.dK;
+    const bool need_u = !sp && p.qk_on;
+    for (int base = threadIdx.x; base < kRowsPerCta * d; base += kRmThreads * 8) {
+      float v[8], u[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int idx = base + j * kRmThreads, r = idx / d, e = idx - r * d, b = b0 + r;
+        v[j] = 0.f; u[j] = 0.f;
+        if (idx < kRowsPerCta * d && b < p.B) {
+          const long long at = ((long long)p.i * p.B + b) * d + e;
+          v[j] = ld_state<COOP>(src + at);
+          if (need_u) u[j] = p.kraw[at];
+        }
       }
-      in1[(c0 + lane) * kRowsPerCta + r] = o0; in1[(c0 + lane + 32) * kRowsPerCta + r] = o1;
-      in2[(c0 + lane) * kRowsPerCta + r] = v0; in2[(c0 + lane + 32) * kRowsPerCta + r] = v1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int idx = base + j * kRmThreads, r = idx / d, e = idx - r * d;
+        if (idx < kRowsPerCta * d) { in[e * kRowsPerCta + r] = v[j]; st1[e * kRowsPerCta + r] = u[j]; }
+      }
+    }
+    if (!sp && p.qk_on) {
+      __syncthreads();
+      const int H = d / kHeadDim;
+      for (int task = warp; task < kRowsPerCta * H; task += kRmWarps) {
+        const int r = task / H, c0 = (task % H) * kHeadDim, b = b0 + r;
+        const int e0 = c0 + lane, e1 = e0 + 32;
+        const float dy0 = in[e0 * kRowsPerCta + r], dy1 = in[e1 * kRowsPerCta + r];
+        const float u0 = st1[e0 * kRowsPerCta + r], u1 = st1[e1 * kRowsPerCta + r];
+        const float g0 = gain_at(gain, e0), g1 = gain_at(gain, e1);
+        const float ss = warp_sum(u0 * u0 + u1 * u1), tu = warp_sum(dy0 * g0 * u0 + dy1 * g1 * u1);
+        const float inv = rsqrtf(ss / kHeadDim + p.eps), mean = tu * inv / kHeadDim;
+        const float o0 = inv * (dy0 * g0 - u0 * inv * mean), o1 = inv * (dy1 * g1 - u1 * inv * mean);
+        in[e0 * kRowsPerCta + r] = o0; in[e1 * kRowsPerCta + r] = o1;
+        if (writer && b < p.B) {
+          const long long at = ((long long)p.i * p.B + b) * d;
+          p.dkraw[at + e0] = o0; p.dkraw[at + e1] = o1;
+        }
+      }
+    } else if (writer) {                                    // no qkRMS: dk_raw = dk
+      for (int idx = threadIdx.x; idx < kRowsPerCta * d; idx += kRmThreads) {
+        const int r = idx / d, e = idx % d, b = b0 + r;
+        if (b < p.B) p.dkraw[((long long)p.i * p.B + b) * d + e] = in[e * kRowsPerCta + r];
+      }
     }
   } else if (p.mode == RM_UP) {
-#pragma unroll 4
-    for (int idx = threadIdx.x; idx < kRowsPerCta * p.K; idx += kRmThreads) {
-      const int r = idx / p.K, k = idx % p.K, b = b0 + r;
-      in1[k * kRowsPerCta + r] = b < p.B ? ld_state<COOP>(p.dpre + ((long long)p.i * p.B + b) * p.K + k) : 0.f;
+    for (int base = threadIdx.x; base < kRowsPerCta * Kin; base += kRmThreads * 8) {
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int idx = base + j * kRmThreads, r = idx / Kin, k = idx - r * Kin, b = b0 + r;
+        v[j] = (idx < kRowsPerCta * Kin && b < p.B) ? ld_state<COOP>(p.dpre + ((long long)p.i * p.B + b) * p.K + k_base + k) : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int idx = base + j * kRmThreads, r = idx / Kin, k = idx - r * Kin;
+        if (idx < kRowsPerCta * Kin) in[k * kRowsPerCta + r] = v[j];
+      }
     }
   } else {
-    // RM_DOWN: Gz = dz_i + RMS backward of dr_i through RMS(z_i);  RM_OUT: dh = Gz_i + RMS backward of du_i through RMS(h_i)
-    // four warps per row: each takes a quarter of the row, the two sums meet in shared memory
+    // RM_DOWN: Gz = dz_i + RMS backward of dr_i through RMS(z_i);  RM_OUT: dh = Gz_i + RMS backward of du_i through RMS(h_i),
+    // dr_i (du_i) being the sum of the previous step's partial products.  Four warps per row, a quarter of the row each.
     const T* zT = reinterpret_cast<const T*>(p.z);
-    const int r = warp >> 2, part = warp & 3, b = b0 + r;
-    const int e_lo = part * (d / 4), e_hi = e_lo + d / 4;
-    const long long at = ((long long)p.i * p.B + (b < p.B ? b : 0)) * d;
-    const float* dy = (p.mode == RM_DOWN ? p.dr : p.du) + at;
-    const T* zr = zT + (long long)(b < p.B ? b : 0) * p.z_bs + (long long)p.i * p.z_ts;
+    const int r = warp >> 2, quarter = warp & 3, b = b0 + r;
+    const bool live = b < p.B;
+    const int e_lo = quarter * (d / 4), e_hi = e_lo + d / 4;
+    const long long at = ((long long)p.i * p.B + (live ? b : 0)) * d;
+    const float* pin = p.part + (long long)(live ? b : 0) * d;
+    const T* zr = zT + (long long)(live ? b : 0) * p.z_bs + (long long)p.i * p.z_ts;
+    const float* dzr = p.dz + (long long)(live ? b : 0) * p.dz_bs + (long long)p.i * p.dz_ts;
+    float* total = (p.mode == RM_DOWN ? p.dr : p.du) + at;   // the summed partials, kept for the gain gradients
     float ss = 0.f, tu = 0.f;
-    if (p.norm_on && b < p.B) {
-#pragma unroll 4
-      for (int e = e_lo + lane; e < e_hi; e += 32) {
-        const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
-        ss = fmaf(u, u, ss);
-        tu = fmaf(ld_state<COOP>(dy + e) * gain_at(gain, e), u, tu);
+    for (int base = e_lo; base < e_hi; base += 256) {
+      float dyv[8], uv[8], av[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + lane + 32 * u;
+        dyv[u] = 0.f; uv[u] = 0.f; av[u] = 0.f;
+        float pv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (e < e_hi && live) {
+#pragma unroll
+          for (int m = 0; m < 4; ++m)
+            if (m < p.n_in) pv[m] = ld_state<COOP>(pin + m * part_stride + e);
+          if (p.norm_on) uv[u] = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
+          av[u] = p.mode == RM_DOWN ? dzr[e] : ld_state<COOP>(p.Gz + at + e);
+        }
+        dyv[u] = ((pv[0] + pv[1]) + pv[2]) + pv[3];
       }
-      ss = warp_sum(ss); tu = warp_sum(tu);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = base + lane + 32 * u;
+        if (e < e_hi) {
+          if (writer && live) total[e] = dyv[u];
+          const float tg = p.norm_on ? dyv[u] * gain_at(gain, e) : dyv[u];
+          ss = fmaf(uv[u], uv[u], ss);
+          tu = fmaf(tg, uv[u], tu);
+          in[e * kRowsPerCta + r] = tg; st1[e * kRowsPerCta + r] = uv[u]; st2[e * kRowsPerCta + r] = av[u];
+        }
+      }
     }
+    ss = warp_sum(ss); tu = warp_sum(tu);
     if (lane == 0) { red[warp * 2] = ss; red[warp * 2 + 1] = tu; }
     __syncthreads();
     ss = red[(r * 4) * 2] + red[(r * 4 + 1) * 2] + red[(r * 4 + 2) * 2] + red[(r * 4 + 3) * 2];
     tu = red[(r * 4) * 2 + 1] + red[(r * 4 + 1) * 2 + 1] + red[(r * 4 + 2) * 2 + 1] + red[(r * 4 + 3) * 2 + 1];
     const float inv = rsqrtf(ss / d + p.eps), mean = tu * inv / d;
-    const float* addv = p.mode == RM_DOWN ? p.dz + (long long)(b < p.B ? b : 0) * p.dz_bs + (long long)p.i * p.dz_ts : p.Gz + at;
     float* keep = (p.mode == RM_DOWN ? p.Gz : p.dh) + at;
-#pragma unroll 4
     for (int e = e_lo + lane; e < e_hi; e += 32) {
-      float val = 0.f;
-      if (b < p.B) {
-        float du = ld_state<COOP>(dy + e);
-        if (p.norm_on) {
-          const float u = p.mode == RM_DOWN ? to_f(zr[e]) : p.h[at + e];
-          du = inv * (du * gain_at(gain, e) - u * inv * mean);
-        }
-        val = (p.mode == RM_DOWN ? addv[e] : ld_state<COOP>(addv + e)) + du;
-        if (writer) keep[e] = val;
-      }
-      in1[e * kRowsPerCta + r] = val;
+      const float tg = in[e * kRowsPerCta + r];
+      const float du = p.norm_on ? inv * (tg - st1[e * kRowsPerCta + r] * inv * mean) : tg;
+      const float val = live ? st2[e * kRowsPerCta + r] + du : 0.f;
+      in[e * kRowsPerCta + r] = val;
+      if (writer && live) keep[e] = val;
     }
   }
   __syncthreads();
 
-  // ---- product: 16 columns per task; a warp's lanes = 8 rows of W x 4 groups of 4 columns
-  const int kq = lane >> 2, cq = lane & 3;
-  const int n0 = cx * kRmCols + 4 * cq;
+  // ---- product: a warp's lanes = (32 / ncq) rows of W x ncq groups of 4 columns
+  const int ncq = p.cols / 4;
+  const int kq = lane / ncq, cq = lane % ncq, krows = 32 / ncq;
+  const int n0 = cx * p.cols + 4 * cq;
+  const T* W = reinterpret_cast<const T*>(p.mode == RM_PAIR && sp ? p.W2 : p.W1) + (long long)k_base * p.Ncols + n0;
   float acc[kRowsPerCta][4] = {};
-  auto run = [&](const T* W, const float* in) {
 #pragma unroll 8
-    for (int k = warp * 8 + kq; k < p.K; k += kRmWarps * 8) {
-      Vec4<T> wv;
-      wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols + n0);
-      float wf[4];
-      wv.to_float(wf);
-      const float4 a4 = *reinterpret_cast<const float4*>(in + (size_t)k * kRowsPerCta);
-      const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+  for (int k = warp * krows + kq; k < Kin; k += kRmWarps * krows) {
+    Vec4<T> wv;
+    wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols);
+    float wf[4];
+    wv.to_float(wf);
+    const float4 a4 = *reinterpret_cast<const float4*>(in + (size_t)k * kRowsPerCta);
+    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
 #pragma unroll
-      for (int r = 0; r < kRowsPerCta; ++r)
+    for (int r = 0; r < kRowsPerCta; ++r)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
-    }
-  };
-  run(reinterpret_cast<const T*>(p.W1), in1);
-  if (p.mode == RM_PAIR) run(reinterpret_cast<const T*>(p.W2), in2);
+      for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
+  }
 #pragma unroll
   for (int r = 0; r < kRowsPerCta; ++r)
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float v = acc[r][c];
-      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      if (ncq <= 4) v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 16);
-      if (kq == 0) red[(warp * kRmCols + 4 * cq + c) * kRowsPerCta + r] = v;
+      if (kq == 0) red[(warp * p.cols + 4 * cq + c) * kRowsPerCta + r] = v;
     }
   __syncthreads();
-  if (threadIdx.x < kRmCols * kRowsPerCta) {
+  if (threadIdx.x < p.cols * kRowsPerCta) {
     const int col = threadIdx.x >> 2, r = threadIdx.x & 3, b = b0 + r;
     float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRmWarps; ++w) sum += red[(w * kRmCols + col) * kRowsPerCta + r];
+    for (int w = 0; w < kRmWarps; ++w) sum += red[(w * p.cols + col) * kRowsPerCta + r];
     if (b < p.B) {
-      const int n = cx * kRmCols + col;
-      const long long at = ((long long)p.i * p.B + b) * p.Ncols + n;
+      const int n = cx * p.cols + col;
       sum *= p.alpha;
-      if (p.mode == RM_PAIR) p.dr[at] = sum;
-      else if (p.mode == RM_DOWN) p.dpre[at] = sum * gelu_grad_f(p.act[at]);
-      else if (p.mode == RM_UP) p.du[at] = sum;
-      else p.dc[at] = sum;
+      if (p.mode == RM_PAIR || p.mode == RM_UP) p.part[sp * part_stride + (long long)b * d + n] = sum;
+      else {
+        const long long at = ((long long)p.i * p.B + b) * p.Ncols + n;
+        if (p.mode == RM_DOWN) p.dpre[at] = sum * gelu_grad_f(p.act[at]);
+        else p.dc[at] = sum;
+      }
     }
   }
 }
@@ -502,18 +560,18 @@ template <typename T>
 __global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p) {
   grid_dep_sync();
   extern __shared__ __align__(16) float smem[];
-  rowmat_body<T, false>(p, blockIdx.x, blockIdx.y, smem);
+  rowmat_body<T, false>(p, blockIdx.x, smem);
 }
 
-size_t rowmat_smem(int mode, int K) {
-  return ((size_t)K * kRowsPerCta * (mode == RM_PAIR ? 2 : 1) + kRmWarps * kRmCols * kRowsPerCta) * sizeof(float);
-}
+// shared memory of a task: three [K][4] arrays and the reduction area
+size_t rowmat_smem(int K, int cols) { return ((size_t)K * kRowsPerCta * 3 + kRmWarps * cols * kRowsPerCta) * sizeof(float); }
 
 // The reverse loop over one leaf [s0, e0) as ONE cooperative kernel: the five steps of a position separated by grid
 // barriers instead of kernel boundaries.  Every wait is bounded (grid_barrier); when one runs out the kernel returns.
 struct LoopParams {
   const void *Wk, *Wv, *Wdn, *Wup, *Wo, *g_k, *g_kv, *g_mlp;
   int z_norm, pre, qk;
+  int cols_down, up_split;                // task shapes: columns per task of the W_down step, parts of the W_up contraction
   float alpha;
   int s0, e0;
   unsigned bar_base;
@@ -529,32 +587,55 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
   const int chunks = (p.B + kRowsPerCta - 1) / kRowsPerCta;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   p.qk_on = lp.qk;
-  auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al) {
+  auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
+                   int nsplit, int n_in) {
     p.mode = mode; p.K = K; p.Ncols = Ncols; p.W1 = W1; p.W2 = W2; p.gain = gain; p.norm_on = norm_on; p.alpha = al;
-    const int nx = Ncols / kRmCols;
-    for (int t = blockIdx.x; t < nx * chunks; t += gridDim.x) rowmat_body<T, true>(p, t % nx, t / nx, smem);
+    p.cols = cols; p.nsplit = nsplit; p.n_in = n_in;
+    const int tasks = (Ncols / cols) * chunks * nsplit;
+    for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true>(p, t, smem);
   };
+#ifdef RT_BWD_TIMERS
+  unsigned long long t_mark = globaltimer_ns();
+  auto mark = [&](int slot) {
+    if (blockIdx.x == 0) {
+      __syncthreads();
+      if (threadIdx.x == 0) { const unsigned long long now = globaltimer_ns(); lp.sync->phase_ns[slot] += now - t_mark; t_mark = now; }
+    }
+  };
+#else
+  auto mark = [](int) {};
+#endif
   for (int i = lp.e0 - 1; i >= lp.s0; --i) {
     p.i = i;
-    phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f);
+    phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f, 16, 2, 0);
+    mark(0);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    phase(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.g_kv, lp.z_norm, lp.alpha);
+    mark(1);
+    phase(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.g_kv, lp.z_norm, lp.alpha, lp.cols_down, 1, 2);
+    mark(2);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f);
+    mark(3);
+    phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f, 16, lp.up_split, 0);
+    mark(4);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha);
+    mark(5);
+    phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha, 16, 1, lp.up_split);
+    mark(6);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    mark(7);
     const int tasks = (i - lp.s0 + 1) * a.B * a.H;
     for (int t = blockIdx.x * kRmWarps + warp; t < tasks; t += gridDim.x * kRmWarps)
       attn_self_task<true>(a, i, lp.s0 + t / (a.B * a.H), (t / a.H) % a.B, t % a.H, lane);
+    mark(8);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
+    mark(9);
   }
 }
 
 // ------------------------------------------------------------------------------------------------ workspace
 struct BwdLayout {
   size_t sync, n, qraw, ktraw, vt, q, kt, r, kraw, k, v, c, h, u, act, gl, lse, D;
-  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part;
+  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2;
   size_t zero_begin, zero_end, total;
 };
 constexpr int kColParts = 128;
@@ -576,6 +657,7 @@ BwdLayout bwd_layout(const rt_config* c, int B, int N) {
   L.du = take(rows * d); L.dh = take(rows * d); L.dc = take(rows * d); L.dq = take(rows * d);
   L.dkt = take(rows * d); L.dvt = take(rows * d); L.dn = take(rows * d); L.gprod = take(rows * d);
   L.part = take((size_t)kColParts * (d > f ? d : f));
+  L.part2 = take((size_t)4 * B * d);
   L.total = o;
   return L;
 }
@@ -649,20 +731,29 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   rp.z = z; rp.z_bs = xbs; rp.z_ts = xts; rp.dz = dz; rp.dz_bs = xbs; rp.dz_ts = xts;
   rp.dK = F(L.dK); rp.dV = F(L.dV); rp.kraw = F(L.kraw); rp.h = F(L.h); rp.act = F(L.act);
   rp.dkraw = F(L.dkraw); rp.dr = F(L.dr); rp.Gz = F(L.Gz); rp.dpre = F(L.dpre); rp.du = F(L.du); rp.dh = F(L.dh); rp.dc = F(L.dc);
-  const size_t smem_max = rowmat_smem(RM_PAIR, d) > rowmat_smem(RM_UP, f) ? rowmat_smem(RM_PAIR, d) : rowmat_smem(RM_UP, f);
-  if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
-  RT_TRY(cudaFuncSetAttribute(rowmat_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-  const unsigned row_ctas = (unsigned)ceil_div(B, kRowsPerCta);
-  auto rowmat = [&](int mode, int i, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al) {
-    rp.mode = mode; rp.i = i; rp.K = K; rp.Ncols = Ncols; rp.W1 = W1; rp.W2 = W2; rp.gain = gain;
-    rp.norm_on = norm_on; rp.qk_on = qk ? 1 : 0; rp.alpha = al;
-    return launch_chained(rowmat_kernel<T>, dim3(Ncols / kRmCols, row_ctas), dim3(kRmThreads), rowmat_smem(mode, K), s, true, rp);
-  };
-  // one cooperative launch per leaf when a CTA per SM can be resident; else one launch per step
   int dev = 0, sms = 0, per_sm = 0, coop = 0;
   RT_TRY(cudaGetDevice(&dev));
   RT_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   RT_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+  const int chunks = ceil_div(B, kRowsPerCta);
+  // task shapes: the W_up contraction in as many parts (of whole 128-row strides) as keep the grid busy once; the
+  // W_down step with 32 columns per task when 16 would need more than one round of the grid
+  int up_split = 1;
+  for (int c = 4; c >= 2; --c)
+    if (f % (c * 128) == 0 && (d / 16) * chunks * c <= sms) { up_split = c; break; }
+  const int cols_down = (f / 16) * chunks > sms ? 32 : 16;
+  rp.part = F(L.part2);
+  const int k_max = d > f / up_split ? d : f / up_split;
+  const size_t smem_max = rowmat_smem(k_max, 32);
+  if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
+  RT_TRY(cudaFuncSetAttribute(rowmat_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
+  auto rowmat = [&](int mode, int i, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
+                    int nsplit, int n_in) {
+    rp.mode = mode; rp.i = i; rp.K = K; rp.Ncols = Ncols; rp.W1 = W1; rp.W2 = W2; rp.gain = gain;
+    rp.norm_on = norm_on; rp.qk_on = qk ? 1 : 0; rp.alpha = al; rp.cols = cols; rp.nsplit = nsplit; rp.n_in = n_in;
+    return launch_chained(rowmat_kernel<T>, dim3(rowmat_tasks(rp)), dim3(kRmThreads), smem_max, s, true, rp);
+  };
+  // one cooperative launch per leaf when a CTA per SM can be resident; else one launch per step
   RT_TRY(cudaFuncSetAttribute(bwd_loop_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
   RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_loop_kernel<T>, kRmThreads, smem_max));
   const bool use_coop = coop && per_sm >= 1;
@@ -670,6 +761,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   memset(&lp, 0, sizeof(lp));
   lp.Wk = Wk; lp.Wv = Wv; lp.Wdn = Wdn; lp.Wup = Wup; lp.Wo = Wo; lp.g_k = g_k; lp.g_kv = g_kv; lp.g_mlp = g_mlp;
   lp.z_norm = z_norm ? 1 : 0; lp.pre = pre ? 1 : 0; lp.qk = qk ? 1 : 0; lp.alpha = alpha;
+  lp.cols_down = cols_down; lp.up_split = up_split;
   lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   unsigned bar_base = 0;
   const int Lf = 64;                                             // leaf of the reverse schedule
@@ -691,10 +783,10 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
       continue;
     }
     for (int i = e0 - 1; i >= s0; --i) {
-      RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f));
-      RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha));
-      RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f));
-      RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha));
+      RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f, 16, 2, 0));
+      RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha, cols_down, 1, 2));
+      RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f, 16, up_split, 0));
+      RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha, 16, 1, up_split));
       RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)(i - s0 + 1) * B * H)), dim3(tpb), 0, s, true, ab, i, i + 1,
                             s0, i + 1, 1));
     }
