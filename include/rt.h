@@ -209,13 +209,14 @@ rt_status rt_layer_recompute(const rt_config *cfg, const rt_layer_weights *w, co
  * Inputs: the layer input x [B,N,d] and its outputs z [B,N,d] as rt_layer_prefill returned them (storage type; z is the
  * next layer's input, so a training loop keeps it anyway), and dz = dL/dz [B,N,d] fp32.
  * Outputs: dx = dL/dx [B,N,d] fp32 and the parameter gradients in `grads` (fp32, device, shapes of the parameters,
- * OVERWRITTEN; a NULL entry is skipped; the entry of a gain the layer does not have (NULL in `w`) is set to zero).
+ * OVERWRITTEN; 16-byte aligned; a NULL entry is skipped; the entry of a gain the layer does not have (NULL in `w`) is set to zero).
  * When w->g_kv is NULL the gain of RMS(z) IS g_attn, and grads->g_attn carries both uses.
  * The call first rebuilds every intermediate from x and z in one parallel sweep, then walks the positions in reverse
  * accumulating only d(k_j, v_j) -- position i needs dL/dz_i, which needs d(k_i, v_i) complete; pairs in other leaves
  * of 64 positions receive their share from Algorithm 1's tiles run backwards -- and finally forms dq, the temporary
  * pairs, dx and every parameter gradient as products over all B*N rows at once.
- * fp32 arithmetic on CUDA cores throughout (both storage types); recur_block > 1 returns RT_ERR_UNSUPPORTED.
+ * The reverse loop and the attention terms are fp32 on CUDA cores; with bf16 storage the products over all rows run
+ * on the tensor cores (operands rounded to bf16, fp32 accumulation).  recur_block > 1 returns RT_ERR_UNSUPPORTED.
  * The workspace needs rt_backward_workspace_bytes (about 30 fp32 arrays of B*N*d plus 3 of B*N*d_ff). */
 typedef struct {
   float *w_q, *w_k, *w_v, *w_o, *w_up, *w_down;   /* shapes of rt_layer_weights */

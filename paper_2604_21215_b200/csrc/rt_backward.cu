@@ -8,7 +8,8 @@
 //      (the same tiles, visited in reverse order, each as one launch over all its keys),
 //   3. computes everything else -- dq, the temporary pairs, dx and all parameter gradients -- as large products over
 //      all rows at once.
-// All arithmetic here is fp32 on CUDA cores (first version: correctness and the schedule; no tensor cores yet).
+// The reverse loop and the attention terms are fp32 on CUDA cores; the products over all rows of stages 1 and 3 run on
+// the tensor cores (bf16 copies of the operands, fp32 accumulation) when the storage type is bf16.
 #include <math.h>
 #include <string.h>
 
@@ -74,6 +75,36 @@ cudaError_t gemm(int M, int N, int K, const TA* A, long long a_rs, long long a_c
   gemm_kernel<TA, TB><<<dim3(ceil_div(N, 64), ceil_div(M, 64)), 256, 0, s>>>(M, N, K, A, a_rs, a_cs, Bm, b_rs, b_cs, C, ldc, alpha,
                                                                               accumulate ? 1 : 0);
   return cudaGetLastError();
+}
+
+// bf16 operands of the tensor-core products (bf16 storage only): a copy, or a transposed copy, of an fp32 / bf16 array
+__global__ void to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, long long n) {
+  const long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (idx + 3 < n) {
+    const float4 v = *reinterpret_cast<const float4*>(in + idx);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(out + idx) = make_uint2(*reinterpret_cast<unsigned*>(&a), *reinterpret_cast<unsigned*>(&b));
+  } else {
+    for (long long j = idx; j < n; ++j) out[j] = __float2bfloat16_rn(in[j]);
+  }
+}
+// out[c * R + r] = in[r * C + c]
+template <typename TI>
+__global__ void transpose_bf16_kernel(const TI* __restrict__ in, long long R, int C, __nv_bfloat16* __restrict__ out) {
+  __shared__ float tile[32][33];
+  const long long r0 = (long long)blockIdx.y * 32;
+  const int c0 = blockIdx.x * 32;
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const long long r = r0 + j;
+    const int c = c0 + threadIdx.x;
+    tile[j][threadIdx.x] = (r < R && c < C) ? to_f(in[r * C + c]) : 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const int c = c0 + j;
+    const long long r = r0 + threadIdx.x;
+    if (r < R && c < C) out[(long long)c * R + r] = __float2bfloat16_rn(tile[threadIdx.x][j]);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ RMS forward / backward
@@ -635,7 +666,7 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
 // ------------------------------------------------------------------------------------------------ workspace
 struct BwdLayout {
   size_t sync, n, qraw, ktraw, vt, q, kt, r, kraw, k, v, c, h, u, act, gl, lse, D;
-  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2;
+  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2, sa, sb, wt;
   size_t zero_begin, zero_end, total;
 };
 constexpr int kColParts = 128;
@@ -658,6 +689,8 @@ BwdLayout bwd_layout(const rt_config* c, int B, int N) {
   L.dkt = take(rows * d); L.dvt = take(rows * d); L.dn = take(rows * d); L.gprod = take(rows * d);
   L.part = take((size_t)kColParts * (d > f ? d : f));
   L.part2 = take((size_t)4 * B * d);
+  // bf16 operands of the tensor-core products (bf16 storage): two [rows, max(d, d_ff)] arrays and one [d, d]
+  L.sa = take(rows * (d > f ? d : f) / 2 + 64); L.sb = take(rows * (d > f ? d : f) / 2 + 64); L.wt = take(d * d / 2 + 64);
   L.total = o;
   return L;
 }
@@ -693,6 +726,42 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   auto warps_grid = [&](long long warps) { return (unsigned)((warps * 32 + tpb - 1) / tpb); };
   auto elems_grid = [&](long long n) { return (unsigned)((n + tpb - 1) / tpb); };
 
+  // Products over all rows.  bf16 storage with tile-friendly widths: tensor cores (dense_tc_kernel) on bf16 copies of
+  // the operands, fp32 accumulation and fp32 results; otherwise the fp32 product above.
+  constexpr bool kBf16 = sizeof(T) == 2;
+  const bool tc = kBf16 && d % 128 == 0 && f % 128 == 0;
+  const bool tc_w = tc && rows % 64 == 0;                       // dW = dY^T X contracts over the rows
+  SyncArea* sync = reinterpret_cast<SyncArea*>(ws + L.sync);
+  __nv_bfloat16* SA = reinterpret_cast<__nv_bfloat16*>(ws + L.sa);
+  __nv_bfloat16* SB = reinterpret_cast<__nv_bfloat16*>(ws + L.sb);
+  __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(ws + L.wt);
+  auto tc_product = [&](int M, int Nn, int K, const void* A, const void* W, float* out, float al, bool acc) {
+    DenseParams dp;
+    memset(&dp, 0, sizeof(dp));
+    dp.M = M; dp.N = Nn; dp.K = K; dp.B = 1; dp.A = A; dp.W = W; dp.epi = DENSE_F32; dp.alpha = al; dp.accumulate = acc ? 1 : 0;
+    dp.h = out;
+    return dense_launch(RT_BF16, dp, sync, s);
+  };
+  auto to_bf16 = [&](const float* in, __nv_bfloat16* out, long long n) {
+    to_bf16_kernel<<<elems_grid((n + 3) / 4), tpb, 0, s>>>(in, out, n);
+  };
+  auto transpose_f = [&](const float* in, long long R, int C, __nv_bfloat16* out) {
+    transpose_bf16_kernel<float><<<dim3(ceil_div(C, 32), (unsigned)((R + 31) / 32)), dim3(32, 8), 0, s>>>(in, R, C, out);
+  };
+  const float* sa_holds = nullptr;                               // which array SA currently holds as a plain bf16 copy
+  // out[rows, n_out] = A[rows, k] W[n_out, k]^T  (a product of the forward pass)
+  auto fwd_product = [&](const float* A, int k, const T* W, int n_out, float* out) -> cudaError_t {
+    if (!tc) return gemm<float, T>((int)rows, n_out, k, A, k, 1, W, 1, k, out, n_out, 1.f, false, s);
+    if (sa_holds != A) { to_bf16(A, SA, rows * k); sa_holds = A; }
+    return tc_product((int)rows, n_out, k, SA, W, out, 1.f, false);
+  };
+  // out[rows, n_in] (+)= dY[rows, n_out] W[n_out, n_in]  (gradient of a product's input)
+  auto dgrad_product = [&](const float* dY, int n_out, const T* W, int n_in, float* out, bool acc) -> cudaError_t {
+    if (!tc) return gemm<float, T>((int)rows, n_in, n_out, dY, n_out, 1, W, n_in, 1, out, n_in, 1.f, acc, s);
+    to_bf16(dY, SA, rows * n_out); sa_holds = nullptr;
+    transpose_bf16_kernel<T><<<dim3(ceil_div(n_in, 32), ceil_div(n_out, 32)), dim3(32, 8), 0, s>>>(W, n_out, n_in, WT);
+    return tc_product((int)rows, n_in, n_out, SA, WT, out, 1.f, acc);
+  };
   RT_TRY(cudaMemsetAsync(ws + L.sync, 0, sizeof(SyncArea), s));
   RT_TRY(cudaMemsetAsync(ws + L.zero_begin, 0, L.zero_end - L.zero_begin, s));
 
@@ -701,14 +770,14 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   {
   ProfSpanScope span(s, 0);
   norm_fwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(x, xbs, xts, B, g_attn, F(L.n), rows, d, d, eps, pre ? 1 : 0);
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wq, 1, d, F(L.qraw), d, 1.f, false, s));
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wk, 1, d, F(L.ktraw), d, 1.f, false, s));
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.n), d, 1, Wv, 1, d, F(L.vt), d, 1.f, false, s));
+  RT_TRY(fwd_product(F(L.n), d, Wq, d, F(L.qraw)));
+  RT_TRY(fwd_product(F(L.n), d, Wk, d, F(L.ktraw)));
+  RT_TRY(fwd_product(F(L.n), d, Wv, d, F(L.vt)));
   norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.qraw), pbs, pts, B, g_q, F(L.q), rows, d, kHeadDim, eps, qk);
   norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.ktraw), pbs, pts, B, g_k, F(L.kt), rows, d, kHeadDim, eps, qk);
   norm_fwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(z, xbs, xts, B, g_kv, F(L.r), rows, d, d, eps, z_norm ? 1 : 0);
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wk, 1, d, F(L.kraw), d, 1.f, false, s));
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.r), d, 1, Wv, 1, d, F(L.v), d, 1.f, false, s));
+  RT_TRY(fwd_product(F(L.r), d, Wk, d, F(L.kraw)));
+  RT_TRY(fwd_product(F(L.r), d, Wv, d, F(L.v)));
   norm_fwd_kernel<float, T><<<warps_grid(rows * H), tpb, 0, s>>>(F(L.kraw), pbs, pts, B, g_k, F(L.k), rows, d, kHeadDim, eps, qk);
   memset(&ab, 0, sizeof(ab));
   ab.q = F(L.q); ab.k = F(L.k); ab.v = F(L.v); ab.kt = F(L.kt); ab.vt = F(L.vt); ab.lse = F(L.lse); ab.D = F(L.D);
@@ -716,10 +785,10 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   ab.alibi = w->alibi_slopes; ab.scale = c->softmax_scale; ab.scale_log2 = c->softmax_scale * kLog2e;
   ab.B = B; ab.H = H; ab.d = d; ab.N = N;
   attn_stats_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.c), d, 1, Wo, 1, d, F(L.dn), d, 1.f, false, s));          // a = W_o c (dn as scratch)
+  RT_TRY(fwd_product(F(L.c), d, Wo, d, F(L.dn)));                     // a = W_o c (dn as scratch)
   residual_kernel<T><<<elems_grid(rows * d), tpb, 0, s>>>(x, xbs, xts, B, F(L.dn), alpha, F(L.h), rows, d);
   norm_fwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.h), pbs, pts, B, g_mlp, F(L.u), rows, d, d, eps, pre ? 1 : 0);
-  RT_TRY(gemm<float, T>((int)rows, f, d, F(L.u), d, 1, Wup, 1, d, F(L.act), f, 1.f, false, s));
+  RT_TRY(fwd_product(F(L.u), d, Wup, f, F(L.act)));
   gelu_kernel<<<elems_grid(rows * f), tpb, 0, s>>>(F(L.act), F(L.gl), rows * f);
   RT_TRY(cudaGetLastError());
   }
@@ -815,9 +884,9 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     col_sum(gprod, d, gr->g_k, false);
   } else if (gr->g_k) RT_TRY(cudaMemsetAsync(gr->g_k, 0, (size_t)d * 4, s));
   // dn = dqraw W_q + dktraw W_k + dvt W_v;  dx = dh + RMS backward of dn through RMS(x)
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dq), d, 1, Wq, d, 1, F(L.dn), d, 1.f, false, s));
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dkt), d, 1, Wk, d, 1, F(L.dn), d, 1.f, true, s));
-  RT_TRY(gemm<float, T>((int)rows, d, d, F(L.dvt), d, 1, Wv, d, 1, F(L.dn), d, 1.f, true, s));
+  RT_TRY(dgrad_product(F(L.dq), d, Wq, d, F(L.dn), false));
+  RT_TRY(dgrad_product(F(L.dkt), d, Wk, d, F(L.dn), true));
+  RT_TRY(dgrad_product(F(L.dvt), d, Wv, d, F(L.dn), true));
   const bool want_ga = gr->g_attn && w->g_attn && pre;
   norm_bwd_kernel<T, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.dn), x, xbs, xts, B, g_attn, F(L.dh), dx, xbs, xts,
                                                          want_ga ? gprod : nullptr, 0, rows, d, d, eps, pre ? 1 : 0);
@@ -844,12 +913,18 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     } else RT_TRY(cudaMemsetAsync(gr->g_mlp, 0, (size_t)d * 4, s));
   }
   // parameter matrices: dW[o, i] = sum_rows dY[row, o] X[row, i]
-  auto wgrad = [&](float* out, const float* dY, int n_out, const float* X, int n_in, float al, bool acc) {
-    return gemm<float, float>(n_out, n_in, (int)rows, dY, 1, n_out, X, n_in, 1, out, n_in, al, acc, s);
+  const float* sb_holds = nullptr;                               // which array SB currently holds transposed
+  auto wgrad = [&](float* out, const float* dY, int n_out, const float* X, int n_in, float al, bool acc) -> cudaError_t {
+    if (!tc_w) return gemm<float, float>(n_out, n_in, (int)rows, dY, 1, n_out, X, n_in, 1, out, n_in, al, acc, s);
+    transpose_f(dY, rows, n_out, SA); sa_holds = nullptr;
+    if (sb_holds != X) { transpose_f(X, rows, n_in, SB); sb_holds = X; }
+    return tc_product(n_out, n_in, (int)rows, SA, SB, out, al, acc);
   };
+  if (gr->w_k) RT_TRY(wgrad(gr->w_k, F(L.dkraw), d, F(L.r), d, 1.f, false));
+  if (gr->w_v) RT_TRY(wgrad(gr->w_v, F(L.dV), d, F(L.r), d, 1.f, false));
+  if (gr->w_k) RT_TRY(wgrad(gr->w_k, F(L.dkt), d, F(L.n), d, 1.f, true));
+  if (gr->w_v) RT_TRY(wgrad(gr->w_v, F(L.dvt), d, F(L.n), d, 1.f, true));
   if (gr->w_q) RT_TRY(wgrad(gr->w_q, F(L.dq), d, F(L.n), d, 1.f, false));
-  if (gr->w_k) { RT_TRY(wgrad(gr->w_k, F(L.dkraw), d, F(L.r), d, 1.f, false)); RT_TRY(wgrad(gr->w_k, F(L.dkt), d, F(L.n), d, 1.f, true)); }
-  if (gr->w_v) { RT_TRY(wgrad(gr->w_v, F(L.dV), d, F(L.r), d, 1.f, false)); RT_TRY(wgrad(gr->w_v, F(L.dvt), d, F(L.n), d, 1.f, true)); }
   if (gr->w_o) RT_TRY(wgrad(gr->w_o, F(L.dh), d, F(L.c), d, alpha, false));
   if (gr->w_up) RT_TRY(wgrad(gr->w_up, F(L.dpre), f, F(L.u), d, 1.f, false));
   if (gr->w_down) RT_TRY(wgrad(gr->w_down, F(L.Gz), d, F(L.gl), f, alpha, false));
@@ -877,6 +952,12 @@ rt_status rt_layer_backward(const rt_config* cfg, const rt_layer_weights* w, con
   if (!w || !w->w_q || !w->w_k || !w->w_v || !w->w_o || !w->w_up || !w->w_down || !x || !z || !dz || !dx || !grads)
     return RT_ERR_INVALID_ARG;
   if (((uintptr_t)x | (uintptr_t)z | (uintptr_t)dz | (uintptr_t)dx) & 15) return RT_ERR_INVALID_ARG;
+  {
+    const float* gp[] = {grads->w_q, grads->w_k, grads->w_v, grads->w_o, grads->w_up, grads->w_down,
+                         grads->g_attn, grads->g_mlp, grads->g_kv, grads->g_q, grads->g_k};
+    for (const float* ptr : gp)
+      if ((uintptr_t)ptr & 15) return RT_ERR_INVALID_ARG;
+  }
   if (workspace_bytes < bwd_layout(cfg, B, N).total) return RT_ERR_WORKSPACE;
   if ((long long)B * N > 0x7fffffffLL / 2) return RT_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)cuda_stream;

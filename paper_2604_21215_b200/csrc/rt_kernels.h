@@ -105,13 +105,15 @@ cudaError_t head_launch(int dtype, const void* emb, const void* g_final, const v
                         int B, int d, int vocab, int norm_flags, float eps, float* logits, cudaStream_t s);
 
 // Position-wise part of the parallel sweep (Sec. 6, activation checkpointing): dense products over all rows.
-enum { DENSE_RES_X = 0, DENSE_GELU = 1, DENSE_RES_H = 2 };
+enum { DENSE_RES_X = 0, DENSE_GELU = 1, DENSE_RES_H = 2, DENSE_F32 = 3 };
 struct DenseParams {
   int M, N, K, B;                                // C[M,N] = A[M,K] W[N,K]^T; rows m = position * B + sequence
   const void *A, *W;                             // storage type, K contiguous
   int epi;                                       // DENSE_RES_X: h = x + alpha C (fp32);  DENSE_GELU: out = GELU(C);
                                                  // DENSE_RES_H: out = h + alpha C (storage type, caller's strides)
+                                                 // DENSE_F32: h = alpha C, or h += alpha C with `accumulate` (fp32 [M, N])
   float alpha;
+  int accumulate;                                // DENSE_F32 only
   const void* x; long long x_bs, x_ts;           // x[b, r, :] (DENSE_RES_X)
   float* h;                                      // [M, N] fp32 (written by DENSE_RES_X, read by DENSE_RES_H)
   void* out; long long o_bs, o_ts;               // DENSE_GELU: [M, N];  DENSE_RES_H: out[b, r, :]

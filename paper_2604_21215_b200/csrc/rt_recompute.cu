@@ -58,6 +58,9 @@ __device__ __forceinline__ void epi_store(const DenseParams& p, int m, int n, fl
     p.h[(size_t)m * p.N + n] = xv + p.alpha * acc;
   } else if (p.epi == DENSE_GELU) {                            // g = GELU(acc)  (storage type)
     reinterpret_cast<T*>(p.out)[(size_t)m * p.N + n] = from_f<T>(gelu_exact(acc));
+  } else if (p.epi == DENSE_F32) {                             // C itself (fp32 [M, N]), optionally added to what is there
+    float* dst = p.h + (size_t)m * p.N + n;
+    *dst = (p.accumulate ? *dst : 0.f) + p.alpha * acc;
   } else {                                                     // z' = h + alpha acc  (storage type, caller's strides)
     const int b = m % p.B, r = m / p.B;
     reinterpret_cast<T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n] = from_f<T>(p.h[(size_t)m * p.N + n] + p.alpha * acc);
@@ -234,6 +237,17 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
           continue;
         }
+        if (p.epi == DENSE_F32) {
+          float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 o = make_float4(p.alpha * __uint_as_float(v[4 * q]), p.alpha * __uint_as_float(v[4 * q + 1]),
+                                   p.alpha * __uint_as_float(v[4 * q + 2]), p.alpha * __uint_as_float(v[4 * q + 3]));
+            if (p.accumulate) { const float4 old = dst[q]; o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+            dst[q] = o;
+          }
+          continue;
+        }
         if (p.epi == DENSE_RES_X) {
           const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n);
           float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
@@ -351,7 +365,7 @@ static bool make_map_rows(CUtensorMap* map, const void* base, long long rows, in
 cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s, bool* normed) {
   if (normed) *normed = false;
   if (p.M <= 0) return cudaSuccess;
-  const bool strides_ok = p.epi == DENSE_GELU || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
+  const bool strides_ok = p.epi == DENSE_GELU || p.epi == DENSE_F32 || (((p.epi == DENSE_RES_X ? p.x_bs : p.o_bs) % 8 == 0) &&
                                                   ((p.epi == DENSE_RES_X ? p.x_ts : p.o_ts) % 8 == 0));
   if (dtype == RT_BF16 && p.N % 128 == 0 && p.K % kTBK == 0 && strides_ok) {
     // Few rows (the wide-batch token step: M = B): narrow tiles and a split contraction so that the launch still
