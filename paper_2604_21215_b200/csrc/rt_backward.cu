@@ -11,6 +11,7 @@
 // The reverse loop and the attention terms are fp32 on CUDA cores; the products over all rows of stages 1 and 3 run on
 // the tensor cores (bf16 copies of the operands, fp32 accumulation) when the storage type is bf16.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "rt_common.cuh"
@@ -382,7 +383,7 @@ __global__ void attn_bwd_q_kernel(AttnBufs a) {
 // rows in1 (in2) are built by a prologue from the state of the reverse loop (mode), W = a weight matrix as stored
 // ([its outputs, its inputs] = [K, Ncols]: the transposed product of the forward pass, read row by row).
 enum { RM_PAIR = 1, RM_DOWN = 2, RM_UP = 3, RM_OUT = 4 };
-constexpr int kRowsPerCta = 4, kRmThreads = 512, kRmWarps = kRmThreads / 32;
+constexpr int kRmThreads = 512, kRmWarps = kRmThreads / 32;   // rows (sequences) per task: RB = 4 or 8, a template parameter
 struct RowmatParams {
   int mode, B, d, dff, i, K, Ncols;
   int cols;                               // columns per task: 16 or 32
@@ -397,11 +398,11 @@ struct RowmatParams {
   float* part;                            // [4][B][d] partial sums of the split products (RM_PAIR, RM_UP), summed by the next step
   float *dkraw, *dr, *Gz, *dpre, *du, *dh, *dc;
 };
-inline int rowmat_tasks(const RowmatParams& p) { return (p.Ncols / p.cols) * ((p.B + kRowsPerCta - 1) / kRowsPerCta) * p.nsplit; }
+inline int rowmat_tasks(const RowmatParams& p, int rb) { return (p.Ncols / p.cols) * ((p.B + rb - 1) / rb) * p.nsplit; }
 
 // One task: `cols` columns of the product for four sequences and one part of a split contraction.  All threads of the CTA.
 // Task index t = ((cy * nx) + cx) * nsplit + sp.
-template <typename T, bool COOP>
+template <typename T, bool COOP, int RB>
 __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   const int nx = p.Ncols / p.cols;
   const int sp = t % p.nsplit, cx = (t / p.nsplit) % nx, cy = t / (p.nsplit * nx);
@@ -409,11 +410,11 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   const int Kin = p.mode == RM_UP ? p.K / p.nsplit : p.K;   // input entries per row this task needs
   const int k_base = p.mode == RM_UP ? sp * Kin : 0;
   float* in = smem;                                         // [Kin][4] the product's input rows, transposed
-  float* st1 = in + (size_t)Kin * kRowsPerCta;              // [Kin][4] staging (u of the RMS backward)
-  float* st2 = st1 + (size_t)Kin * kRowsPerCta;             // [Kin][4] staging (the term added)
-  float* red = st2 + (size_t)Kin * kRowsPerCta;             // [16 warps][cols][4]
+  float* st1 = in + (size_t)Kin * RB;              // [Kin][4] staging (u of the RMS backward)
+  float* st2 = st1 + (size_t)Kin * RB;             // [Kin][4] staging (the term added)
+  float* red = p.mode == RM_UP ? st1 : st2 + (size_t)Kin * RB;   // [16 warps][cols][RB] (the W_up step stages nothing)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b0 = cy * kRowsPerCta;
+  const int b0 = cy * RB;
   const bool writer = cx == 0 && sp == 0;
   const T* gain = reinterpret_cast<const T*>(p.gain);
   const long long part_stride = (long long)p.B * d;
@@ -425,13 +426,13 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
     // (loads of a batch first, stores after: the round trips to L2 overlap instead of queueing behind the stores)
     const float* src = sp ? p.dV : p.dK;
     const bool need_u = !sp && p.qk_on;
-    for (int base = threadIdx.x; base < kRowsPerCta * d; base += kRmThreads * 8) {
+    for (int base = threadIdx.x; base < RB * d; base += kRmThreads * 8) {
       float v[8], u[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int idx = base + j * kRmThreads, r = idx / d, e = idx - r * d, b = b0 + r;
         v[j] = 0.f; u[j] = 0.f;
-        if (idx < kRowsPerCta * d && b < p.B) {
+        if (idx < RB * d && b < p.B) {
           const long long at = ((long long)p.i * p.B + b) * d + e;
           v[j] = ld_state<COOP>(src + at);
           if (need_u) u[j] = p.kraw[at];
@@ -440,54 +441,55 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int idx = base + j * kRmThreads, r = idx / d, e = idx - r * d;
-        if (idx < kRowsPerCta * d) { in[e * kRowsPerCta + r] = v[j]; st1[e * kRowsPerCta + r] = u[j]; }
+        if (idx < RB * d) { in[e * RB + r] = v[j]; st1[e * RB + r] = u[j]; }
       }
     }
     if (!sp && p.qk_on) {
       __syncthreads();
       const int H = d / kHeadDim;
-      for (int task = warp; task < kRowsPerCta * H; task += kRmWarps) {
+      for (int task = warp; task < RB * H; task += kRmWarps) {
         const int r = task / H, c0 = (task % H) * kHeadDim, b = b0 + r;
         const int e0 = c0 + lane, e1 = e0 + 32;
-        const float dy0 = in[e0 * kRowsPerCta + r], dy1 = in[e1 * kRowsPerCta + r];
-        const float u0 = st1[e0 * kRowsPerCta + r], u1 = st1[e1 * kRowsPerCta + r];
+        const float dy0 = in[e0 * RB + r], dy1 = in[e1 * RB + r];
+        const float u0 = st1[e0 * RB + r], u1 = st1[e1 * RB + r];
         const float g0 = gain_at(gain, e0), g1 = gain_at(gain, e1);
         const float ss = warp_sum(u0 * u0 + u1 * u1), tu = warp_sum(dy0 * g0 * u0 + dy1 * g1 * u1);
         const float inv = rsqrtf(ss / kHeadDim + p.eps), mean = tu * inv / kHeadDim;
         const float o0 = inv * (dy0 * g0 - u0 * inv * mean), o1 = inv * (dy1 * g1 - u1 * inv * mean);
-        in[e0 * kRowsPerCta + r] = o0; in[e1 * kRowsPerCta + r] = o1;
+        in[e0 * RB + r] = o0; in[e1 * RB + r] = o1;
         if (writer && b < p.B) {
           const long long at = ((long long)p.i * p.B + b) * d;
           p.dkraw[at + e0] = o0; p.dkraw[at + e1] = o1;
         }
       }
     } else if (writer) {                                    // no qkRMS: dk_raw = dk
-      for (int idx = threadIdx.x; idx < kRowsPerCta * d; idx += kRmThreads) {
+      for (int idx = threadIdx.x; idx < RB * d; idx += kRmThreads) {
         const int r = idx / d, e = idx % d, b = b0 + r;
-        if (b < p.B) p.dkraw[((long long)p.i * p.B + b) * d + e] = in[e * kRowsPerCta + r];
+        if (b < p.B) p.dkraw[((long long)p.i * p.B + b) * d + e] = in[e * RB + r];
       }
     }
   } else if (p.mode == RM_UP) {
-    for (int base = threadIdx.x; base < kRowsPerCta * Kin; base += kRmThreads * 8) {
+    for (int base = threadIdx.x; base < RB * Kin; base += kRmThreads * 8) {
       float v[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int idx = base + j * kRmThreads, r = idx / Kin, k = idx - r * Kin, b = b0 + r;
-        v[j] = (idx < kRowsPerCta * Kin && b < p.B) ? ld_state<COOP>(p.dpre + ((long long)p.i * p.B + b) * p.K + k_base + k) : 0.f;
+        v[j] = (idx < RB * Kin && b < p.B) ? ld_state<COOP>(p.dpre + ((long long)p.i * p.B + b) * p.K + k_base + k) : 0.f;
       }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int idx = base + j * kRmThreads, r = idx / Kin, k = idx - r * Kin;
-        if (idx < kRowsPerCta * Kin) in[k * kRowsPerCta + r] = v[j];
+        if (idx < RB * Kin) in[k * RB + r] = v[j];
       }
     }
   } else {
     // RM_DOWN: Gz = dz_i + RMS backward of dr_i through RMS(z_i);  RM_OUT: dh = Gz_i + RMS backward of du_i through RMS(h_i),
     // dr_i (du_i) being the sum of the previous step's partial products.  Four warps per row, a quarter of the row each.
     const T* zT = reinterpret_cast<const T*>(p.z);
-    const int r = warp >> 2, quarter = warp & 3, b = b0 + r;
+    constexpr int WPR = kRmWarps / RB;                       // warps per row
+    const int r = warp / WPR, quarter = warp % WPR, b = b0 + r;
     const bool live = b < p.B;
-    const int e_lo = quarter * (d / 4), e_hi = e_lo + d / 4;
+    const int e_lo = quarter * (d / WPR), e_hi = e_lo + d / WPR;
     const long long at = ((long long)p.i * p.B + (live ? b : 0)) * d;
     const float* pin = p.part + (long long)(live ? b : 0) * d;
     const T* zr = zT + (long long)(live ? b : 0) * p.z_bs + (long long)p.i * p.z_ts;
@@ -518,22 +520,23 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
           const float tg = p.norm_on ? dyv[u] * gain_at(gain, e) : dyv[u];
           ss = fmaf(uv[u], uv[u], ss);
           tu = fmaf(tg, uv[u], tu);
-          in[e * kRowsPerCta + r] = tg; st1[e * kRowsPerCta + r] = uv[u]; st2[e * kRowsPerCta + r] = av[u];
+          in[e * RB + r] = tg; st1[e * RB + r] = uv[u]; st2[e * RB + r] = av[u];
         }
       }
     }
     ss = warp_sum(ss); tu = warp_sum(tu);
     if (lane == 0) { red[warp * 2] = ss; red[warp * 2 + 1] = tu; }
     __syncthreads();
-    ss = red[(r * 4) * 2] + red[(r * 4 + 1) * 2] + red[(r * 4 + 2) * 2] + red[(r * 4 + 3) * 2];
-    tu = red[(r * 4) * 2 + 1] + red[(r * 4 + 1) * 2 + 1] + red[(r * 4 + 2) * 2 + 1] + red[(r * 4 + 3) * 2 + 1];
+    ss = 0.f; tu = 0.f;
+#pragma unroll
+    for (int w = 0; w < WPR; ++w) { ss += red[(r * WPR + w) * 2]; tu += red[(r * WPR + w) * 2 + 1]; }
     const float inv = rsqrtf(ss / d + p.eps), mean = tu * inv / d;
     float* keep = (p.mode == RM_DOWN ? p.Gz : p.dh) + at;
     for (int e = e_lo + lane; e < e_hi; e += 32) {
-      const float tg = in[e * kRowsPerCta + r];
-      const float du = p.norm_on ? inv * (tg - st1[e * kRowsPerCta + r] * inv * mean) : tg;
-      const float val = live ? st2[e * kRowsPerCta + r] + du : 0.f;
-      in[e * kRowsPerCta + r] = val;
+      const float tg = in[e * RB + r];
+      const float du = p.norm_on ? inv * (tg - st1[e * RB + r] * inv * mean) : tg;
+      const float val = live ? st2[e * RB + r] + du : 0.f;
+      in[e * RB + r] = val;
       if (writer && live) keep[e] = val;
     }
   }
@@ -544,36 +547,40 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   const int kq = lane / ncq, cq = lane % ncq, krows = 32 / ncq;
   const int n0 = cx * p.cols + 4 * cq;
   const T* W = reinterpret_cast<const T*>(p.mode == RM_PAIR && sp ? p.W2 : p.W1) + (long long)k_base * p.Ncols + n0;
-  float acc[kRowsPerCta][4] = {};
+  float acc[RB][4] = {};
 #pragma unroll 8
   for (int k = warp * krows + kq; k < Kin; k += kRmWarps * krows) {
     Vec4<T> wv;
     wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols);
     float wf[4];
     wv.to_float(wf);
-    const float4 a4 = *reinterpret_cast<const float4*>(in + (size_t)k * kRowsPerCta);
-    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+    float av[RB];
 #pragma unroll
-    for (int r = 0; r < kRowsPerCta; ++r)
+    for (int r4 = 0; r4 < RB / 4; ++r4) {
+      const float4 a4 = *reinterpret_cast<const float4*>(in + (size_t)k * RB + 4 * r4);
+      av[4 * r4] = a4.x; av[4 * r4 + 1] = a4.y; av[4 * r4 + 2] = a4.z; av[4 * r4 + 3] = a4.w;
+    }
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
   }
 #pragma unroll
-  for (int r = 0; r < kRowsPerCta; ++r)
+  for (int r = 0; r < RB; ++r)
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float v = acc[r][c];
       if (ncq <= 4) v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 16);
-      if (kq == 0) red[(warp * p.cols + 4 * cq + c) * kRowsPerCta + r] = v;
+      if (kq == 0) red[(warp * p.cols + 4 * cq + c) * RB + r] = v;
     }
   __syncthreads();
-  if (threadIdx.x < p.cols * kRowsPerCta) {
-    const int col = threadIdx.x >> 2, r = threadIdx.x & 3, b = b0 + r;
+  if (threadIdx.x < p.cols * RB) {
+    const int col = threadIdx.x / RB, r = threadIdx.x % RB, b = b0 + r;
     float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRmWarps; ++w) sum += red[(w * p.cols + col) * kRowsPerCta + r];
+    for (int w = 0; w < kRmWarps; ++w) sum += red[(w * p.cols + col) * RB + r];
     if (b < p.B) {
       const int n = cx * p.cols + col;
       sum *= p.alpha;
@@ -587,15 +594,18 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   }
 }
 
-template <typename T>
+template <typename T, int RB>
 __global__ void __launch_bounds__(kRmThreads) rowmat_kernel(const RowmatParams p) {
   grid_dep_sync();
   extern __shared__ __align__(16) float smem[];
-  rowmat_body<T, false>(p, blockIdx.x, smem);
+  rowmat_body<T, false, RB>(p, blockIdx.x, smem);
 }
 
 // shared memory of a task: three [K][4] arrays and the reduction area
-size_t rowmat_smem(int K, int cols) { return ((size_t)K * kRowsPerCta * 3 + kRmWarps * cols * kRowsPerCta) * sizeof(float); }
+size_t rowmat_smem(int d, int k_up, int cols, int rb) {
+  const size_t in = (size_t)(3 * d > k_up ? 3 * d : k_up) * rb;
+  return (in + (size_t)kRmWarps * cols * rb) * sizeof(float);
+}
 
 // The reverse loop over one leaf [s0, e0) as ONE cooperative kernel: the five steps of a position separated by grid
 // barriers instead of kernel boundaries.  Every wait is bounded (grid_barrier); when one runs out the kernel returns.
@@ -610,12 +620,12 @@ struct LoopParams {
 };
 constexpr int kLoopBarriersPerPosition = 5;
 
-template <typename T>
+template <typename T, int RB>
 __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p, const LoopParams lp, const AttnBufs a) {
   extern __shared__ __align__(16) float smem[];
   __shared__ int s_flag;
   unsigned target = lp.bar_base;
-  const int chunks = (p.B + kRowsPerCta - 1) / kRowsPerCta;
+  const int chunks = (p.B + RB - 1) / RB;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   p.qk_on = lp.qk;
   auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
@@ -623,7 +633,7 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
     p.mode = mode; p.K = K; p.Ncols = Ncols; p.W1 = W1; p.W2 = W2; p.gain = gain; p.norm_on = norm_on; p.alpha = al;
     p.cols = cols; p.nsplit = nsplit; p.n_in = n_in;
     const int tasks = (Ncols / cols) * chunks * nsplit;
-    for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true>(p, t, smem);
+    for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true, RB>(p, t, smem);
   };
 #ifdef RT_BWD_TIMERS
   unsigned long long t_mark = globaltimer_ns();
@@ -804,7 +814,8 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   RT_TRY(cudaGetDevice(&dev));
   RT_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   RT_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
-  const int chunks = ceil_div(B, kRowsPerCta);
+  const int rb = 4;                                              // sequences per task (8 per task measured slower: B = 8, d = 1024: 69 vs 59 us per position)
+  const int chunks = ceil_div(B, rb);
   // task shapes: the W_up contraction in as many parts (of whole 128-row strides) as keep the grid busy once; the
   // W_down step with 32 columns per task when 16 would need more than one round of the grid
   int up_split = 1;
@@ -812,20 +823,24 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     if (f % (c * 128) == 0 && (d / 16) * chunks * c <= sms) { up_split = c; break; }
   const int cols_down = (f / 16) * chunks > sms ? 32 : 16;
   rp.part = F(L.part2);
-  const int k_max = d > f / up_split ? d : f / up_split;
-  const size_t smem_max = rowmat_smem(k_max, 32);
+  const size_t smem_max = rowmat_smem(d, f / up_split, 32, rb);
   if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
-  RT_TRY(cudaFuncSetAttribute(rowmat_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
+  const void* step_fn = reinterpret_cast<const void*>(&rowmat_kernel<T, 4>);
+  const void* loop_fn = reinterpret_cast<const void*>(&bwd_loop_kernel<T, 4>);
+  RT_TRY(cudaFuncSetAttribute(step_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
   auto rowmat = [&](int mode, int i, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
                     int nsplit, int n_in) {
     rp.mode = mode; rp.i = i; rp.K = K; rp.Ncols = Ncols; rp.W1 = W1; rp.W2 = W2; rp.gain = gain;
     rp.norm_on = norm_on; rp.qk_on = qk ? 1 : 0; rp.alpha = al; rp.cols = cols; rp.nsplit = nsplit; rp.n_in = n_in;
-    return launch_chained(rowmat_kernel<T>, dim3(rowmat_tasks(rp)), dim3(kRmThreads), smem_max, s, true, rp);
+    const dim3 grid(rowmat_tasks(rp, rb)), block(kRmThreads);
+    return launch_chained(rowmat_kernel<T, 4>, grid, block, smem_max, s, true, rp);
   };
-  // one cooperative launch per leaf when a CTA per SM can be resident; else one launch per step
-  RT_TRY(cudaFuncSetAttribute(bwd_loop_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
-  RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_loop_kernel<T>, kRmThreads, smem_max));
-  const bool use_coop = coop && per_sm >= 1;
+  RT_TRY(cudaFuncSetAttribute(loop_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
+  RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_loop_kernel<T, 4>, kRmThreads, smem_max));
+  // RT_BACKWARD_STEP_LAUNCHES=1 in the environment forces the one-launch-per-step form (kept for devices without
+  // cooperative launch; the tests run both forms)
+  const char* force_steps = getenv("RT_BACKWARD_STEP_LAUNCHES");
+  const bool use_coop = coop && per_sm >= 1 && !(force_steps && force_steps[0] == '1');
   LoopParams lp;
   memset(&lp, 0, sizeof(lp));
   lp.Wk = Wk; lp.Wv = Wv; lp.Wdn = Wdn; lp.Wup = Wup; lp.Wo = Wo; lp.g_k = g_k; lp.g_kv = g_kv; lp.g_mlp = g_mlp;
@@ -847,7 +862,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     if (use_coop) {
       lp.s0 = s0; lp.e0 = e0; lp.bar_base = bar_base;
       void* args[] = {(void*)&rp, (void*)&lp, (void*)&ab};
-      RT_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&bwd_loop_kernel<T>), dim3(sms), dim3(kRmThreads), args, smem_max, s));
+      RT_TRY(cudaLaunchCooperativeKernel(loop_fn, dim3(sms), dim3(kRmThreads), args, smem_max, s));
       bar_base += (unsigned)(e0 - s0) * kLoopBarriersPerPosition * (unsigned)sms;
       continue;
     }
