@@ -216,51 +216,83 @@ struct AttnBufs {
   int B, H, d, N;
 };
 
+// ---- eight lanes per (query, key) pair -------------------------------------------------------------------------------
+// The three all-pairs kernels below split a warp into four groups of eight lanes; a group works on one pair at a time,
+// each lane holding eight consecutive entries of the 64-wide head, so a dot product costs three shuffles for four pairs.
+struct F8 { float v[8]; };
+__device__ __forceinline__ F8 ld8(const float* p) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  return F8{{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w}};
+}
+__device__ __forceinline__ void st8(float* p, const F8& x) {
+  *reinterpret_cast<float4*>(p) = make_float4(x.v[0], x.v[1], x.v[2], x.v[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(x.v[4], x.v[5], x.v[6], x.v[7]);
+}
+__device__ __forceinline__ float dot8(const F8& a, const F8& b) {
+  float s = 0.f;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) s = fmaf(a.v[e], b.v[e], s);
+  return s;
+}
+__device__ __forceinline__ float group_sum(float v) {          // over the eight lanes of a group
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  v += __shfl_xor_sync(0xffffffffu, v, 4);
+  return v;
+}
+__device__ __forceinline__ float across_groups_sum(float v) {   // over the four groups, lane by lane
+  v += __shfl_xor_sync(0xffffffffu, v, 8);
+  v += __shfl_xor_sync(0xffffffffu, v, 16);
+  return v;
+}
+
 // One warp per (position i, sequence, head): the softmax of Sec. 2.2 over the pairs j < i and the temporary pair;
-// keeps c = attention value and the log2-sum-exp of the logits.
+// keeps c = attention value and the log2-sum-exp of the logits.  Group g takes the pairs j = g, g+4, ... with its own
+// running (m, l, o); the four partial softmaxes are merged at the end.
 __global__ void attn_stats_kernel(AttnBufs a) {
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, g = lane >> 3, t = lane & 7;
   if (wid >= (long long)a.N * a.B * a.H) return;
   const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
-  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long col = (long long)h * kHeadDim + 8 * t;
   const long long ri = ((long long)i * a.B + b) * a.d + col;
-  const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
+  const long long rstride = (long long)a.B * a.d;
+  const F8 q = ld8(a.q + ri);
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
-  float m = -INFINITY, l = 0.f, o0 = 0.f, o1 = 0.f;
-  auto step = [&](float s, float2 vv) {
-    const float mn = fmaxf(m, s);
-    const float corr = exp2f(m - mn), p = exp2f(s - mn);
-    l = l * corr + p; o0 = o0 * corr + p * vv.x; o1 = o1 * corr + p * vv.y;
-    m = mn;
-  };
-  int j = 0;
-  for (; j + 4 <= i; j += 4) {
-    float s[4]; float2 vv[4];
+  float m = -INFINITY, l = 0.f;
+  F8 o = {};
+  for (int j0 = 0; j0 < i; j0 += 4) {                        // uniform trip count: the shuffles need every lane
+    const int j = j0 + g;
+    const bool valid = j < i;
+    const long long rj = (long long)(valid ? j : 0) * rstride + (long long)b * a.d + col;
+    const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
+    const float sd = group_sum(dot8(q, kk));
+    if (valid) {
+      const float sc = sd * a.scale_log2 - slope * (float)(i - j);
+      const float mn = fmaxf(m, sc);
+      const float corr = exp2f(m - mn), p = exp2f(sc - mn);
+      l = l * corr + p;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const long long rj = ((long long)(j + u) * a.B + b) * a.d + col;
-      const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
-      vv[u] = *reinterpret_cast<const float2*>(a.v + rj);
-      s[u] = q.x * kk.x + q.y * kk.y;
+      for (int e = 0; e < 8; ++e) o.v[e] = fmaf(p, vv.v[e], o.v[e] * corr);
+      m = mn;
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) s[u] = warp_sum(s[u]) * a.scale_log2 - slope * (float)(i - j - u);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) step(s[u], vv[u]);
   }
-  for (; j < i; ++j) {
-    const long long rj = ((long long)j * a.B + b) * a.d + col;
-    const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
-    step(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2 - slope * (float)(i - j), *reinterpret_cast<const float2*>(a.v + rj));
-  }
-  {
-    const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
-    step(warp_sum(q.x * kk.x + q.y * kk.y) * a.scale_log2, *reinterpret_cast<const float2*>(a.vt + ri));
-  }
+  // merge the four groups, then the temporary pair of the position itself
+  float m_all = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
+  m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, 16));
+  const F8 kt = ld8(a.kt + ri), vt = ld8(a.vt + ri);
+  const float st = group_sum(dot8(q, kt)) * a.scale_log2;
+  const float mf = fmaxf(m_all, st);
+  const float w = m == -INFINITY ? 0.f : exp2f(m - mf);       // this group's weight in the merged sums
+  l = across_groups_sum(l * w);
+  const float pt = exp2f(st - mf);
+  l += pt;
   const float inv = 1.f / l;
-  *reinterpret_cast<float2*>(a.c + ri) = make_float2(o0 * inv, o1 * inv);
-  if (lane == 0) a.lse[((long long)i * a.B + b) * a.H + h] = m + log2f(l);
+  F8 c;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) c.v[e] = (across_groups_sum(o.v[e] * w) + pt * vt.v[e]) * inv;
+  if (g == 0) st8(a.c + ri, c);
+  if (lane == 0) a.lse[((long long)i * a.B + b) * a.H + h] = mf + log2f(l);
 }
 
 // State of the reverse loop written earlier in the SAME (cooperative) kernel by other CTAs must not come from L1.
@@ -310,72 +342,82 @@ __global__ void attn_bwd_kv_kernel(AttnBufs a, int q0, int q1, int k0, int k1, i
   const int lane = threadIdx.x & 31;
   if (wid >= (long long)(k1 - k0) * a.B * a.H) return;
   const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
-  const long long col = (long long)h * kHeadDim + 2 * lane;
-  const long long rj = ((long long)j * a.B + b) * a.d + col;
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
   if (self) {
     attn_self_task<false>(a, q0, j, b, h, lane);
     return;
   }
-  const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
-  const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
-  float dk0 = 0.f, dk1 = 0.f, dv0 = 0.f, dv1 = 0.f;
-  const long long rstride = (long long)a.B * a.d;
-  long long ri = ((long long)q0 * a.B + b) * a.d + col;
-  long long si = ((long long)q0 * a.B + b) * a.H + h;
-#pragma unroll 2
-  for (int i = q0; i < q1; ++i, ri += rstride, si += (long long)a.B * a.H) {
-    const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
-    const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
+  // a tile of Algorithm 1 backwards: group g takes the queries q0 + g, q0 + g + 4, ...
+  const int g = lane >> 3, t = lane & 7;
+  const long long col8 = (long long)h * kHeadDim + 8 * t;
+  const long long rj8 = ((long long)j * a.B + b) * a.d + col8;
+  const long long rstride = (long long)a.B * a.d, sstride = (long long)a.B * a.H;
+  const F8 kk = ld8(a.k + rj8), vv = ld8(a.v + rj8);
+  F8 dk = {}, dv = {};
+  for (int i0 = q0; i0 < q1; i0 += 4) {
+    const int i = i0 + g;
+    const bool valid = i < q1;
+    const int ic = valid ? i : q0;
+    const long long ri = (long long)ic * rstride + (long long)b * a.d + col8;
+    const long long si = (long long)ic * sstride + (long long)b * a.H + h;
+    const F8 q = ld8(a.q + ri), dc = ld8(a.dc + ri);
     const float lse = a.lse[si], D = a.D[si];
-    float s = q.x * kk.x + q.y * kk.y, dp = dc.x * vv.x + dc.y * vv.y;
+    const float sd = group_sum(dot8(q, kk)), dp = group_sum(dot8(dc, vv));
+    if (valid) {
+      const float p = exp2f(sd * a.scale_log2 - slope * (float)(i - j) - lse);
+      const float ds = p * (dp - D) * a.scale;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dp += __shfl_xor_sync(0xffffffffu, dp, o); }
-    const float p = exp2f(s * a.scale_log2 - slope * (float)(i - j) - lse);
-    const float ds = p * (dp - D) * a.scale;
-    dk0 = fmaf(ds, q.x, dk0); dk1 = fmaf(ds, q.y, dk1);
-    dv0 = fmaf(p, dc.x, dv0); dv1 = fmaf(p, dc.y, dv1);
+      for (int e = 0; e < 8; ++e) { dk.v[e] = fmaf(ds, q.v[e], dk.v[e]); dv.v[e] = fmaf(p, dc.v[e], dv.v[e]); }
+    }
   }
-  float2* dk = reinterpret_cast<float2*>(a.dK + rj);
-  float2* dv = reinterpret_cast<float2*>(a.dV + rj);
-  float2 t = *dk; t.x += dk0; t.y += dk1; *dk = t;
-  t = *dv; t.x += dv0; t.y += dv1; *dv = t;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { dk.v[e] = across_groups_sum(dk.v[e]); dv.v[e] = across_groups_sum(dv.v[e]); }
+  if (g == 0) {
+    F8 cur = ld8(a.dK + rj8);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) cur.v[e] += dk.v[e];
+    st8(a.dK + rj8, cur);
+    cur = ld8(a.dV + rj8);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) cur.v[e] += dv.v[e];
+    st8(a.dV + rj8, cur);
+  }
 }
 
-// Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).
+// Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).  One warp per
+// (position, sequence, head); group g takes the pairs j = g, g+4, ...
 __global__ void attn_bwd_q_kernel(AttnBufs a) {
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, g = lane >> 3, t = lane & 7;
   if (wid >= (long long)a.N * a.B * a.H) return;
   const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
-  const long long col = (long long)h * kHeadDim + 2 * lane;
+  const long long col = (long long)h * kHeadDim + 8 * t;
   const long long ri = ((long long)i * a.B + b) * a.d + col;
   const long long si = ((long long)i * a.B + b) * a.H + h;
-  const float2 q = *reinterpret_cast<const float2*>(a.q + ri);
-  const float2 dc = *reinterpret_cast<const float2*>(a.dc + ri);
+  const long long rstride = (long long)a.B * a.d;
+  const F8 q = ld8(a.q + ri), dc = ld8(a.dc + ri);
   const float lse = a.lse[si], D = a.D[si];
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
-  float g0 = 0.f, g1 = 0.f;
-  long long rj = (long long)b * a.d + col;
-  const long long rstride = (long long)a.B * a.d;
-#pragma unroll 2
-  for (int j = 0; j < i; ++j, rj += rstride) {
-    const float2 kk = *reinterpret_cast<const float2*>(a.k + rj);
-    const float2 vv = *reinterpret_cast<const float2*>(a.v + rj);
-    float s = q.x * kk.x + q.y * kk.y, dp = dc.x * vv.x + dc.y * vv.y;
+  F8 acc = {};
+  for (int j0 = 0; j0 < i; j0 += 4) {
+    const int j = j0 + g;
+    const bool valid = j < i;
+    const long long rj = (long long)(valid ? j : 0) * rstride + (long long)b * a.d + col;
+    const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
+    const float sd = group_sum(dot8(q, kk)), dp = group_sum(dot8(dc, vv));
+    if (valid) {
+      const float ds = exp2f(sd * a.scale_log2 - slope * (float)(i - j) - lse) * (dp - D);
 #pragma unroll
-    for (int o = 16; o; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); dp += __shfl_xor_sync(0xffffffffu, dp, o); }
-    const float ds = exp2f(s * a.scale_log2 - slope * (float)(i - j) - lse) * (dp - D);
-    g0 = fmaf(ds, kk.x, g0); g1 = fmaf(ds, kk.y, g1);
+      for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(ds, kk.v[e], acc.v[e]);
+    }
   }
-  {
-    const float2 kk = *reinterpret_cast<const float2*>(a.kt + ri);
-    const float2 vv = *reinterpret_cast<const float2*>(a.vt + ri);
-    const float s = warp_sum(q.x * kk.x + q.y * kk.y), dp = warp_sum(dc.x * vv.x + dc.y * vv.y);
-    const float ds = exp2f(s * a.scale_log2 - lse) * (dp - D);
-    g0 = fmaf(ds, kk.x, g0); g1 = fmaf(ds, kk.y, g1);
-  }
-  *reinterpret_cast<float2*>(a.dq + ri) = make_float2(g0 * a.scale, g1 * a.scale);
+  const F8 kt = ld8(a.kt + ri), vt = ld8(a.vt + ri);
+  const float st = group_sum(dot8(q, kt)), dpt = group_sum(dot8(dc, vt));
+  const float dst = exp2f(st * a.scale_log2 - lse) * (dpt - D);
+  F8 out;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) out.v[e] = (across_groups_sum(acc.v[e]) + dst * kt.v[e]) * a.scale;
+  if (g == 0) st8(a.dq + ri, out);
 }
 
 // ------------------------------------------------------------------------------------------------ the reverse loop's products

@@ -50,8 +50,8 @@ def test_backward_matches_gradient_oracle(dtype, d, H, dff, B, N, flags, gains, 
     want = {"w_q", "w_k", "w_v", "w_o", "w_up", "w_down"} | set(gains)
     assert set(g) == want
     for name in sorted(want):
-        if np.abs(g_ref[name]).max() == 0.0:                                  # e.g. g_q without qkRMS
-            assert np.abs(g[name]).max() == 0.0, name
+        if np.abs(g_ref[name]).max() == 0.0:                                  # e.g. a gain no norm uses; q, k at N = 1
+            assert np.abs(g[name]).max() <= tol * np.abs(dx_ref).max(), name   # zero up to the rounding of the other terms
             continue
         assert rel_err(g[name], g_ref[name]) <= tol, (name, rel_err(g[name], g_ref[name]))
 
