@@ -621,9 +621,16 @@ def run_backward_bench(args):
         torch.cuda.synchronize(dev)
         return sum(a.elapsed_time(b) for a, b in evs) / len(evs)
 
+    bwd = lambda: layer.backward_device(x, z, dz, dx, grads, ws)
+    if args.profile_one_call:
+        # profiling mode (launch list under ncu): the forward pass once for z, ONE backward call, no bench line
+        layer.prefill_device(x, z)
+        bwd()
+        torch.cuda.synchronize(dev)
+        print(json.dumps({"profile_one_call": "backward " + wl.name, "status": int(rt.rt_get_status(ws.data_ptr()))}))
+        return 0
     fwd_ms = timed(lambda: layer.prefill_device(x, z))
     assert layer.status() == rt.RT_OK
-    bwd = lambda: layer.backward_device(x, z, dz, dx, grads, ws)
     bwd_ms = timed(bwd)
     rt.rt_profile_enable(True)
     rt.rt_profile_read()
