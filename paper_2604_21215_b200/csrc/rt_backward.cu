@@ -439,6 +439,7 @@ struct RowmatParams {
   const float *dK, *dV, *kraw, *h, *act;
   float* part;                            // [4][B][d] partial sums of the split products (RM_PAIR, RM_UP), summed by the next step
   float *dkraw, *dr, *Gz, *dpre, *du, *dh, *dc;
+  SyncArea* sync;                         // step timers of instrumented builds
 };
 inline int rowmat_tasks(const RowmatParams& p, int rb) { return (p.Ncols / p.cols) * ((p.B + rb - 1) / rb) * p.nsplit; }
 
@@ -461,6 +462,17 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   const T* gain = reinterpret_cast<const T*>(p.gain);
   const long long part_stride = (long long)p.B * d;
   __syncthreads();                                          // shared memory of the previous task is free
+#ifdef RT_BWD_TIMERS2
+  unsigned long long tb = globaltimer_ns();
+  auto bmark = [&](int slot) {
+    if (COOP && blockIdx.x == 0 && p.mode == RT_BWD_TIMERS2) {
+      __syncthreads();
+      if (threadIdx.x == 0) { const unsigned long long now = globaltimer_ns(); p.sync->phase_ns[slot] += now - tb; tb = now; }
+    }
+  };
+#else
+  auto bmark = [](int) {};
+#endif
 
   // ---- prologue: the input rows of this task's sequences, transposed into shared memory
   if (p.mode == RM_PAIR) {
@@ -582,6 +594,7 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
       if (writer && live) keep[e] = val;
     }
   }
+  bmark(0);
   __syncthreads();
 
   // ---- product: a warp's lanes = (32 / ncq) rows of W x ncq groups of 4 columns
@@ -607,6 +620,7 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
   }
+  bmark(1);
 #pragma unroll
   for (int r = 0; r < RB; ++r)
 #pragma unroll
@@ -634,6 +648,7 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
       }
     }
   }
+  bmark(2);
 }
 
 template <typename T, int RB>
@@ -864,7 +879,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   for (int c = 4; c >= 2; --c)
     if (f % (c * 128) == 0 && (d / 16) * chunks * c <= sms) { up_split = c; break; }
   const int cols_down = (f / 16) * chunks > sms ? 32 : 16;
-  rp.part = F(L.part2);
+  rp.part = F(L.part2); rp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   const size_t smem_max = rowmat_smem(d, f / up_split, 32, rb);
   if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
   const void* step_fn = reinterpret_cast<const void*>(&rowmat_kernel<T, 4>);

@@ -93,6 +93,47 @@ def test_backward_one_launch_per_step_form_agrees(monkeypatch):
         assert rel_err(dx2, dx1) <= tol and all(rel_err(g2[n], g1[n]) <= tol for n in g1)
 
 
+def test_backward_directional_derivative_at_c2_shape():
+    # Full c2 shape (B = 4, N = 2048, d = 768: 32 leaves, tiles backwards up to 1024 keys), fp32 storage, where the
+    # gradient oracle would take far too long: the property that holds at any size is
+    #   (L(x + e v) - L(x - e v)) / (2 e) = <dL/dx, v>,  L = sum(z * dz),
+    # with L evaluated by the GPU's own forward pass (itself checked against the oracle elsewhere), and likewise along a
+    # direction in W_v (which enters both the temporary and the persistent pairs) and in W_down.
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    wl = inputs.WORKLOADS["c2"]
+    d, H, dff, B, N = wl.d_model, wl.n_heads, wl.d_ff, wl.B, wl.N
+    x, lw, _, dz = _case("f32", d, H, dff, B, N, 4242, ("g_attn", "g_kv", "g_k"), False)
+    rng = np.random.default_rng(99)
+    layer = rt.Layer(d, H, dff, dtype="f32")
+
+    def loss(xx, ww):
+        layer.set_weights(ww)
+        z, _, _ = layer.prefill(xx)
+        return z, float(np.sum(z * dz))
+
+    z0, _ = loss(x, lw)
+    dx, g = layer.backward(x, z0, dz)
+    assert np.isfinite(dx).all()
+    eps = 2e-3
+
+    def f32(a):
+        return a.astype(np.float32).astype(np.float64)
+
+    v = rng.standard_normal(x.shape)
+    xp, xm = f32(x + eps * v), f32(x - eps * v)
+    fd = (loss(xp, lw)[1] - loss(xm, lw)[1])
+    an = float(np.sum(dx * (xp - xm)))                      # the step actually taken after rounding to fp32
+    assert abs(fd - an) <= 1e-2 * abs(fd), ("x", fd, an)
+    for name in ("w_v", "w_down"):
+        dirn = rng.standard_normal(lw[name].shape) / np.sqrt(lw[name].shape[1])
+        wp, wm = dict(lw), dict(lw)
+        wp[name], wm[name] = f32(lw[name] + eps * dirn), f32(lw[name] - eps * dirn)
+        fd = loss(x, wp)[1] - loss(x, wm)[1]
+        an = float(np.sum(g[name] * (wp[name] - wm[name])))
+        assert abs(fd - an) <= 1e-2 * abs(fd), (name, fd, an)
+
+
 def test_backward_argument_errors():
     import torch
     from paper_2604_21215_b200 import rt
