@@ -246,28 +246,29 @@ __device__ __forceinline__ float across_groups_sum(float v) {   // over the four
   return v;
 }
 
-// One warp per (position i, sequence, head): the softmax of Sec. 2.2 over the pairs j < i and the temporary pair;
-// keeps c = attention value and the log2-sum-exp of the logits.  Group g takes the pairs j = g, g+4, ... with its own
-// running (m, l, o); the four partial softmaxes are merged at the end.
+// The softmax of Sec. 2.2 for every (position, sequence, head): attention value c and log2-sum-exp of the logits over
+// the pairs j < i and the temporary pair.  One warp per FOUR consecutive positions of one (sequence, head): group g is
+// position 4 iq + g, all four groups read the same pair j in the same instruction (one fetch, broadcast), and the warps
+// of a CTA are consecutive position quads of the same (sequence, head), so the pair rows stay in L1.
 __global__ void attn_stats_kernel(AttnBufs a) {
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31, g = lane >> 3, t = lane & 7;
-  if (wid >= (long long)a.N * a.B * a.H) return;
-  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
+  const int NQ = (a.N + 3) / 4;
+  if (wid >= (long long)NQ * a.B * a.H) return;
+  const int iq = (int)(wid % NQ), h = (int)((wid / NQ) % a.H), b = (int)(wid / ((long long)NQ * a.H));
+  const int i = 4 * iq + g;
+  const bool live = i < a.N;
   const long long col = (long long)h * kHeadDim + 8 * t;
-  const long long ri = ((long long)i * a.B + b) * a.d + col;
+  const long long ri = ((long long)(live ? i : a.N - 1) * a.B + b) * a.d + col;
   const long long rstride = (long long)a.B * a.d;
   const F8 q = ld8(a.q + ri);
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
   float m = -INFINITY, l = 0.f;
   F8 o = {};
-  for (int j0 = 0; j0 < i; j0 += 4) {                        // uniform trip count: the shuffles need every lane
-    const int j = j0 + g;
-    const bool valid = j < i;
-    const long long rj = (long long)(valid ? j : 0) * rstride + (long long)b * a.d + col;
-    const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
-    const float sd = group_sum(dot8(q, kk));
-    if (valid) {
+  const int jend = 4 * iq + 3 < a.N - 1 ? 4 * iq + 3 : a.N - 1;   // pairs needed by the last position of the quad
+  long long rj = (long long)b * a.d + col;
+  auto update = [&](int j, float sd, const F8& vv) {
+    if (j < i) {
       const float sc = sd * a.scale_log2 - slope * (float)(i - j);
       const float mn = fmaxf(m, sc);
       const float corr = exp2f(m - mn), p = exp2f(sc - mn);
@@ -276,23 +277,39 @@ __global__ void attn_stats_kernel(AttnBufs a) {
       for (int e = 0; e < 8; ++e) o.v[e] = fmaf(p, vv.v[e], o.v[e] * corr);
       m = mn;
     }
+  };
+  int j = 0;
+  for (; j + 4 <= jend; j += 4, rj += 4 * rstride) {          // four pairs in flight
+    F8 vv[4];
+    float sd[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const F8 kk = ld8(a.k + rj + u * rstride);
+      vv[u] = ld8(a.v + rj + u * rstride);
+      sd[u] = dot8(q, kk);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) sd[u] = group_sum(sd[u]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) update(j + u, sd[u], vv[u]);
   }
-  // merge the four groups, then the temporary pair of the position itself
-  float m_all = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
-  m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, 16));
-  const F8 kt = ld8(a.kt + ri), vt = ld8(a.vt + ri);
+  for (; j < jend; ++j, rj += rstride) {
+    const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
+    update(j, group_sum(dot8(q, kk)), vv);
+  }
+  const F8 kt = ld8(a.kt + ri), vt = ld8(a.vt + ri);           // the temporary pair of the position itself
   const float st = group_sum(dot8(q, kt)) * a.scale_log2;
-  const float mf = fmaxf(m_all, st);
-  const float w = m == -INFINITY ? 0.f : exp2f(m - mf);       // this group's weight in the merged sums
-  l = across_groups_sum(l * w);
-  const float pt = exp2f(st - mf);
-  l += pt;
+  const float mf = fmaxf(m, st);
+  const float w = m == -INFINITY ? 0.f : exp2f(m - mf), pt = exp2f(st - mf);
+  l = l * w + pt;
   const float inv = 1.f / l;
   F8 c;
 #pragma unroll
-  for (int e = 0; e < 8; ++e) c.v[e] = (across_groups_sum(o.v[e] * w) + pt * vt.v[e]) * inv;
-  if (g == 0) st8(a.c + ri, c);
-  if (lane == 0) a.lse[((long long)i * a.B + b) * a.H + h] = mf + log2f(l);
+  for (int e = 0; e < 8; ++e) c.v[e] = (o.v[e] * w + pt * vt.v[e]) * inv;
+  if (live) {
+    st8(a.c + ri, c);
+    if (t == 0) a.lse[((long long)i * a.B + b) * a.H + h] = mf + log2f(l);
+  }
 }
 
 // State of the reverse loop written earlier in the SAME (cooperative) kernel by other CTAs must not come from L1.
@@ -332,21 +349,28 @@ __device__ __forceinline__ void attn_self_task(const AttnBufs& a, int i, int j, 
   }
 }
 
-// Gradient of the pairs: one warp per (key j, sequence, head) holds k_j, v_j and sums over the queries [q0, q1):
+// In-leaf step of position i as a launch of its own (the one-launch-per-step form of the reverse loop): one warp per
+// (key j in [k0, i], sequence, head), see attn_self_task.
+__global__ void attn_bwd_kv_kernel(AttnBufs a, int i, int k0) {
+  grid_dep_sync();
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)(i + 1 - k0) * a.B * a.H) return;
+  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
+  attn_self_task<false>(a, i, j, b, h, lane);
+}
+
+// A tile of Algorithm 1 backwards: the pairs [k0, k1) receive the share of the queries [q0, q1) (all later positions):
 //   p = exp2(logit - lse_i), ds = p (<dc_i, v_j> - D_i), dk_j += scale ds q_i, dv_j += p dc_i.
-// self = 1 (the in-leaf step of position i = q0): keys [k0, i]; every warp computes D_i = <dc_i, c_i> itself, and the warp
-// of j = i stores it and handles the temporary pair of position i instead of a persistent one.
-__global__ void attn_bwd_kv_kernel(AttnBufs a, int q0, int q1, int k0, int k1, int self) {
+// One warp per (key j, sequence, head) holds k_j, v_j; its four groups take the queries q0 + g, q0 + g + 4, ... and the
+// four partial sums are added in a fixed order at the end (no atomics).
+__global__ void attn_bwd_kv_tile_kernel(AttnBufs a, int q0, int q1, int k0, int k1) {
   grid_dep_sync();
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (wid >= (long long)(k1 - k0) * a.B * a.H) return;
   const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
-  if (self) {
-    attn_self_task<false>(a, q0, j, b, h, lane);
-    return;
-  }
   // a tile of Algorithm 1 backwards: group g takes the queries q0 + g, q0 + g + 4, ...
   const int g = lane >> 3, t = lane & 7;
   const long long col8 = (long long)h * kHeadDim + 8 * t;
@@ -384,28 +408,51 @@ __global__ void attn_bwd_kv_kernel(AttnBufs a, int q0, int q1, int k0, int k1, i
   }
 }
 
-// Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).  One warp per
-// (position, sequence, head); group g takes the pairs j = g, g+4, ...
+// Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).  Same layout as
+// attn_stats_kernel: one warp per four consecutive positions of one (sequence, head), group g = position 4 iq + g.
 __global__ void attn_bwd_q_kernel(AttnBufs a) {
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31, g = lane >> 3, t = lane & 7;
-  if (wid >= (long long)a.N * a.B * a.H) return;
-  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), i = (int)(wid / ((long long)a.H * a.B));
+  const int NQ = (a.N + 3) / 4;
+  if (wid >= (long long)NQ * a.B * a.H) return;
+  const int iq = (int)(wid % NQ), h = (int)((wid / NQ) % a.H), b = (int)(wid / ((long long)NQ * a.H));
+  const int i = 4 * iq + g;
+  const bool live = i < a.N;
+  const int ic = live ? i : a.N - 1;
   const long long col = (long long)h * kHeadDim + 8 * t;
-  const long long ri = ((long long)i * a.B + b) * a.d + col;
-  const long long si = ((long long)i * a.B + b) * a.H + h;
+  const long long ri = ((long long)ic * a.B + b) * a.d + col;
+  const long long si = ((long long)ic * a.B + b) * a.H + h;
   const long long rstride = (long long)a.B * a.d;
   const F8 q = ld8(a.q + ri), dc = ld8(a.dc + ri);
   const float lse = a.lse[si], D = a.D[si];
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
   F8 acc = {};
-  for (int j0 = 0; j0 < i; j0 += 4) {
-    const int j = j0 + g;
-    const bool valid = j < i;
-    const long long rj = (long long)(valid ? j : 0) * rstride + (long long)b * a.d + col;
+  const int jend = 4 * iq + 3 < a.N - 1 ? 4 * iq + 3 : a.N - 1;
+  long long rj = (long long)b * a.d + col;
+  int j = 0;
+  for (; j + 4 <= jend; j += 4, rj += 4 * rstride) {          // four pairs in flight
+    F8 kk[4];
+    float sd[4], dp[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      kk[u] = ld8(a.k + rj + u * rstride);
+      const F8 vv = ld8(a.v + rj + u * rstride);
+      sd[u] = dot8(q, kk[u]); dp[u] = dot8(dc, vv);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { sd[u] = group_sum(sd[u]); dp[u] = group_sum(dp[u]); }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (j + u < i) {
+        const float ds = exp2f(sd[u] * a.scale_log2 - slope * (float)(i - j - u) - lse) * (dp[u] - D);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(ds, kk[u].v[e], acc.v[e]);
+      }
+  }
+  for (; j < jend; ++j, rj += rstride) {
     const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
     const float sd = group_sum(dot8(q, kk)), dp = group_sum(dot8(dc, vv));
-    if (valid) {
+    if (j < i) {
       const float ds = exp2f(sd * a.scale_log2 - slope * (float)(i - j) - lse) * (dp - D);
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(ds, kk.v[e], acc.v[e]);
@@ -416,8 +463,8 @@ __global__ void attn_bwd_q_kernel(AttnBufs a) {
   const float dst = exp2f(st * a.scale_log2 - lse) * (dpt - D);
   F8 out;
 #pragma unroll
-  for (int e = 0; e < 8; ++e) out.v[e] = (across_groups_sum(acc.v[e]) + dst * kt.v[e]) * a.scale;
-  if (g == 0) st8(a.dq + ri, out);
+  for (int e = 0; e < 8; ++e) out.v[e] = (acc.v[e] + dst * kt.v[e]) * a.scale;
+  if (live) st8(a.dq + ri, out);
 }
 
 // ------------------------------------------------------------------------------------------------ the reverse loop's products
@@ -851,7 +898,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   ab.c = F(L.c); ab.dc = F(L.dc); ab.dK = F(L.dK); ab.dV = F(L.dV); ab.dkt = F(L.dkt); ab.dvt = F(L.dvt); ab.dq = F(L.dq);
   ab.alibi = w->alibi_slopes; ab.scale = c->softmax_scale; ab.scale_log2 = c->softmax_scale * kLog2e;
   ab.B = B; ab.H = H; ab.d = d; ab.N = N;
-  attn_stats_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
+  attn_stats_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
   RT_TRY(fwd_product(F(L.c), d, Wo, d, F(L.dn)));                     // a = W_o c (dn as scratch)
   residual_kernel<T><<<elems_grid(rows * d), tpb, 0, s>>>(x, xbs, xts, B, F(L.dn), alpha, F(L.h), rows, d);
   norm_fwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.h), pbs, pts, B, g_mlp, F(L.u), rows, d, d, eps, pre ? 1 : 0);
@@ -912,8 +959,8 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
       const int P = e0 & -e0;
       const int q1 = e0 + P < N ? e0 + P : N;
       ProfSpanScope span(s, 2);
-      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop, ab, e0, q1, e0 - P,
-                            e0, 0));
+      RT_TRY(launch_chained(attn_bwd_kv_tile_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop, ab,
+                            e0, q1, e0 - P, e0));
     }
     ProfSpanScope span(s, 1);
     if (use_coop) {
@@ -928,14 +975,13 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
       RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha, cols_down, 1, 2));
       RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f, 16, up_split, 0));
       RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha, 16, 1, up_split));
-      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)(i - s0 + 1) * B * H)), dim3(tpb), 0, s, true, ab, i, i + 1,
-                            s0, i + 1, 1));
+      RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)(i - s0 + 1) * B * H)), dim3(tpb), 0, s, true, ab, i, s0));
     }
   }
 
   // ---- 3. everything else over all rows at once
   ProfSpanScope span(s, 3);
-  attn_bwd_q_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab);
+  attn_bwd_q_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
   float* gprod = F(L.gprod);
   float* part = F(L.part);
   auto col_sum = [&](const float* a, int width, float* out, bool acc) {
