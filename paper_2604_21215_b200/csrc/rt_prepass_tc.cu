@@ -166,29 +166,18 @@ qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_const
   }
 }
 
-// row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
-static bool make_map_2d(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kGemmBK, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
+static_assert(kGemmBK == 64, "tensor_map_rows_bf16 encodes 64-column boxes");
 
 bool qkv_gemm_tc_supported(const PrepassParams& p) { return p.d % kGemmBN == 0 && p.d >= kGemmBN; }
 
 cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStream_t s) {
   const int M = p.N * p.B;
   CUtensorMap mn, mq, mk, mv;
-  if (!make_map_2d(&mn, p.n, M, p.d, kBM) || !make_map_2d(&mq, p.w_q, p.d, p.d, kGemmBN) ||
-      !make_map_2d(&mk, p.w_k, p.d, p.d, kGemmBN) || !make_map_2d(&mv, p.w_v, p.d, p.d, kGemmBN))
+  if (!tensor_map_rows_bf16(&mn, p.n, M, p.d, kBM) || !tensor_map_rows_bf16(&mq, p.w_q, p.d, p.d, kGemmBN) ||
+      !tensor_map_rows_bf16(&mk, p.w_k, p.d, p.d, kGemmBN) || !tensor_map_rows_bf16(&mv, p.w_v, p.d, p.d, kGemmBN))
     return cudaErrorInvalidValue;
   const size_t smem = GemmSmem::total + 1024;
-  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&qkv_gemm_tc_kernel), (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(ceil_div(M, kBM), 3 * (p.d / kGemmBN));
   return launch_chained(qkv_gemm_tc_kernel, grid, dim3(kGemmThreads), smem, s, p.chained != 0, mn, mq, mk, mv, p, sync);

@@ -349,18 +349,7 @@ __global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) 
   }
 }
 
-// row-major [rows, cols] bf16, box = 64 columns x box_rows rows, 128-byte swizzle
-static bool make_map_rows(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kTBK, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
+static_assert(kTBK == 64, "tensor_map_rows_bf16 encodes 64-column boxes");
 
 cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s, bool* normed) {
   if (normed) *normed = false;
@@ -370,8 +359,7 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
   if (dtype == RT_BF16 && p.N % 128 == 0 && p.K % kTBK == 0 && strides_ok) {
     // Few rows (the wide-batch token step: M = B): narrow tiles and a split contraction so that the launch still
     // fills the GPU; the partial sums are combined in a fixed order by a second small kernel.
-    int sms = 148;
-    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+    const int sms = sm_count();
     const int m_tiles = ceil_div(p.M, kBM);
     int bn = p.N % 256 == 0 ? 256 : 128;
     if (bn == 256 && m_tiles * (p.N / 256) < sms) bn = 128;
@@ -385,17 +373,17 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       if ((size_t)want * p.M * p.N * sizeof(float) <= p.partial_bytes) q.splits = want;
     }
     CUtensorMap ma, mw;
-    if (!make_map_rows(&ma, p.A, p.M, p.K, kBM) || !make_map_rows(&mw, p.W, p.N, p.K, bn)) return cudaErrorInvalidValue;
+    if (!tensor_map_rows_bf16(&ma, p.A, p.M, p.K, kBM) || !tensor_map_rows_bf16(&mw, p.W, p.N, p.K, bn)) return cudaErrorInvalidValue;
     dim3 grid(m_tiles, p.N / bn, q.splits);
     if (bn == 256) {
       const size_t smem = DenseSmem<256>::total + 1024;
-      cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_tc_kernel<256>), (int)smem);
       if (e != cudaSuccess) return e;
       e = launch_chained(dense_tc_kernel<256>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
       if (e != cudaSuccess) return e;
     } else {
       const size_t smem = DenseSmem<128>::total + 1024;
-      cudaError_t e = cudaFuncSetAttribute(dense_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_tc_kernel<128>), (int)smem);
       if (e != cudaSuccess) return e;
       e = launch_chained(dense_tc_kernel<128>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
       if (e != cudaSuccess) return e;

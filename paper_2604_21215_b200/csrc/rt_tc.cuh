@@ -133,5 +133,56 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Row-major [rows, cols] bf16 array, box = 64 columns x box_rows rows, 128-byte swizzle.  An encoded map is a pure
+// function of these arguments, so each thread remembers the ones it made: a token step of a wide batch needs ten maps
+// and they are the same at every position.
+inline bool tensor_map_rows_bf16(CUtensorMap* out, const void* base, long long rows, int cols, int box_rows) {
+  struct Entry { const void* base; long long rows; int cols, box_rows; CUtensorMap map; };
+  constexpr int kEntries = 64;
+  thread_local Entry tab[kEntries];
+  thread_local int used = 0, next = 0;
+  for (int i = 0; i < used; ++i)
+    if (tab[i].base == base && tab[i].rows == rows && tab[i].cols == cols && tab[i].box_rows == box_rows) { *out = tab[i].map; return true; }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  if (fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  const int slot = used < kEntries ? used++ : (next++ % kEntries);
+  tab[slot].base = base; tab[slot].rows = rows; tab[slot].cols = cols; tab[slot].box_rows = box_rows; tab[slot].map = *out;
+  return true;
+}
+
+// cudaFuncSetAttribute(max dynamic shared memory) once per (kernel, device) instead of before every launch.
+inline cudaError_t ensure_dynamic_smem(const void* fn, int bytes) {
+  struct Entry { const void* fn; int dev, bytes; };
+  constexpr int kEntries = 32;
+  thread_local Entry tab[kEntries];
+  thread_local int used = 0;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  for (int i = 0; i < used; ++i)
+    if (tab[i].fn == fn && tab[i].dev == dev && tab[i].bytes >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && used < kEntries) { tab[used].fn = fn; tab[used].dev = dev; tab[used].bytes = bytes; ++used; }
+  return e;
+}
+
+// multiprocessor count of the current device, remembered per thread and device
+inline int sm_count() {
+  thread_local int cached_dev = -1, cached = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cached;
+  if (dev != cached_dev) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) { cached = n; cached_dev = dev; }
+  }
+  return cached;
+}
 
 }  // namespace rt
