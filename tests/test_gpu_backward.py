@@ -34,7 +34,9 @@ def _case(dtype, d, H, dff, B, N, seed, gains, alibi):
     ("f32", 64, 1, 96, 5, 1, 3, G_NAMES, False, 1.0),                        # a single position
     ("f32", 128, 2, 256, 2, 300, 3, ("g_k", "g_kv"), True, 1.0),             # cross tiles of 64, 128 and 256 keys
     ("bf16", 256, 4, 512, 3, 200, 3, G_NAMES, False, 1.0),
-    ("bf16", 128, 2, 384, 9, 130, 3, (), True, 0.6)])
+    ("bf16", 128, 2, 384, 9, 130, 3, (), True, 0.6),
+    ("bf16", 192, 3, 224, 2, 96, 3, ("g_mlp", "g_q"), False, 1.0),            # widths off the tensor-core products
+    ("bf16", 128, 2, 384, 3, 77, 3, G_NAMES, False, 0.8)])                   # row count off the tensor-core dW products
 def test_backward_matches_gradient_oracle(dtype, d, H, dff, B, N, flags, gains, alibi, alpha):
     from oracle import RTConfig, RTWeights, layer_grad
     from paper_2604_21215_b200 import inputs, rt
