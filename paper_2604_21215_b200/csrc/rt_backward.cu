@@ -492,8 +492,10 @@ inline int rowmat_tasks(const RowmatParams& p, int rb) { return (p.Ncols / p.col
 
 // One task: `cols` columns of the product for four sequences and one part of a split contraction.  All threads of the CTA.
 // Task index t = ((cy * nx) + cx) * nsplit + sp.
+// `wslice` (optional): this task's part of the weight matrix already in shared memory, [Kin][cols] -- the cooperative
+// kernel keeps it there for all positions of a leaf.
 template <typename T, bool COOP, int RB>
-__device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
+__device__ void rowmat_body(const RowmatParams& p, int t, float* smem, const T* wslice = nullptr) {
   const int nx = p.Ncols / p.cols;
   const int sp = t % p.nsplit, cx = (t / p.nsplit) % nx, cy = t / (p.nsplit * nx);
   const int d = p.d;
@@ -648,12 +650,14 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem) {
   const int ncq = p.cols / 4;
   const int kq = lane / ncq, cq = lane % ncq, krows = 32 / ncq;
   const int n0 = cx * p.cols + 4 * cq;
-  const T* W = reinterpret_cast<const T*>(p.mode == RM_PAIR && sp ? p.W2 : p.W1) + (long long)k_base * p.Ncols + n0;
+  const T* W = wslice ? wslice + 4 * cq
+                      : reinterpret_cast<const T*>(p.mode == RM_PAIR && sp ? p.W2 : p.W1) + (long long)k_base * p.Ncols + n0;
+  const long long wstride = wslice ? p.cols : p.Ncols;
   float acc[RB][4] = {};
 #pragma unroll 8
   for (int k = warp * krows + kq; k < Kin; k += kRmWarps * krows) {
     Vec4<T> wv;
-    wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * p.Ncols);
+    wv.v = *reinterpret_cast<const decltype(wv.v)*>(W + (long long)k * wstride);
     float wf[4];
     wv.to_float(wf);
     float av[RB];
@@ -717,6 +721,8 @@ struct LoopParams {
   const void *Wk, *Wv, *Wdn, *Wup, *Wo, *g_k, *g_kv, *g_mlp;
   int z_norm, pre, qk;
   int cols_down, up_split;                // task shapes: columns per task of the W_down step, parts of the W_up contraction
+  int resident;                           // 1: every step has at most one task per CTA and its weight slices fit: keep them in shared memory
+  unsigned stage_bytes;                   // shared memory of the staging areas (the slices follow)
   float alpha;
   int s0, e0;
   unsigned bar_base;
@@ -732,12 +738,39 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
   const int chunks = (p.B + RB - 1) / RB;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   p.qk_on = lp.qk;
+  // weight slices of this CTA's four tasks, resident for the whole leaf
+  const T* slice[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (lp.resident) {
+    T* wsm = reinterpret_cast<T*>(reinterpret_cast<unsigned char*>(smem) + lp.stage_bytes);
+    auto stage = [&](int mode, int K, int Ncols, const void* W1, const void* W2, int cols, int nsplit) {
+      const int nx = Ncols / cols, tasks = nx * chunks * nsplit, t = blockIdx.x;
+      const int Kin = mode == RM_UP ? K / nsplit : K;
+      if (t < tasks) {
+        const int sp = t % nsplit, cx = (t / nsplit) % nx;
+        const T* src = reinterpret_cast<const T*>(mode == RM_PAIR && sp ? W2 : W1) + (long long)(mode == RM_UP ? sp * Kin : 0) * Ncols + cx * cols;
+        const int quads = cols / 4;
+        for (int idx = threadIdx.x; idx < Kin * quads; idx += kRmThreads) {
+          const int k = idx / quads, c4 = idx - k * quads;
+          Vec4<T> v;
+          v.v = *reinterpret_cast<const decltype(v.v)*>(src + (long long)k * Ncols + 4 * c4);
+          *reinterpret_cast<decltype(v.v)*>(wsm + (size_t)k * cols + 4 * c4) = v.v;
+        }
+        slice[mode] = wsm;
+      }
+      wsm += (size_t)Kin * cols;                              // every CTA advances alike: the layout is fixed
+    };
+    stage(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, 16, 2);
+    stage(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.cols_down, 1);
+    stage(RM_UP, p.dff, p.d, lp.Wup, nullptr, 16, lp.up_split);
+    stage(RM_OUT, p.d, p.d, lp.Wo, nullptr, 16, 1);
+    __syncthreads();
+  }
   auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
                    int nsplit, int n_in) {
     p.mode = mode; p.K = K; p.Ncols = Ncols; p.W1 = W1; p.W2 = W2; p.gain = gain; p.norm_on = norm_on; p.alpha = al;
     p.cols = cols; p.nsplit = nsplit; p.n_in = n_in;
     const int tasks = (Ncols / cols) * chunks * nsplit;
-    for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true, RB>(p, t, smem);
+    for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true, RB>(p, t, smem, slice[mode]);
   };
 #ifdef RT_BWD_TIMERS
   unsigned long long t_mark = globaltimer_ns();
@@ -944,12 +977,24 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   // RT_BACKWARD_STEP_LAUNCHES=1 in the environment forces the one-launch-per-step form (kept for devices without
   // cooperative launch; the tests run both forms)
   const char* force_steps = getenv("RT_BACKWARD_STEP_LAUNCHES");
-  const bool use_coop = coop && per_sm >= 1 && !(force_steps && force_steps[0] == '1');
+  bool use_coop = coop && per_sm >= 1 && !(force_steps && force_steps[0] == '1');
+  // weight slices resident in shared memory when every step has at most one task per CTA and they fit beside the staging
+  const size_t slice_bytes = ((size_t)d * 16 + (size_t)d * cols_down + (size_t)(f / up_split) * 16 + (size_t)d * 16) * sizeof(T);
+  const bool one_task = (d / 16) * chunks * 2 <= sms && (f / cols_down) * chunks <= sms && (d / 16) * chunks * up_split <= sms;
+  size_t loop_smem = smem_max;
+  bool resident = false;
+  if (use_coop && one_task && smem_max + slice_bytes <= 220 * 1024) {
+    int per_sm_res = 0;
+    RT_TRY(cudaFuncSetAttribute(loop_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem_max + slice_bytes)));
+    RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_res, bwd_loop_kernel<T, 4>, kRmThreads, smem_max + slice_bytes));
+    if (per_sm_res >= 1) { resident = true; loop_smem = smem_max + slice_bytes; }
+  }
   LoopParams lp;
   memset(&lp, 0, sizeof(lp));
   lp.Wk = Wk; lp.Wv = Wv; lp.Wdn = Wdn; lp.Wup = Wup; lp.Wo = Wo; lp.g_k = g_k; lp.g_kv = g_kv; lp.g_mlp = g_mlp;
   lp.z_norm = z_norm ? 1 : 0; lp.pre = pre ? 1 : 0; lp.qk = qk ? 1 : 0; lp.alpha = alpha;
   lp.cols_down = cols_down; lp.up_split = up_split;
+  lp.resident = resident ? 1 : 0; lp.stage_bytes = (unsigned)smem_max;
   lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   unsigned bar_base = 0;
   const int Lf = 64;                                             // leaf of the reverse schedule
@@ -966,7 +1011,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     if (use_coop) {
       lp.s0 = s0; lp.e0 = e0; lp.bar_base = bar_base;
       void* args[] = {(void*)&rp, (void*)&lp, (void*)&ab};
-      RT_TRY(cudaLaunchCooperativeKernel(loop_fn, dim3(sms), dim3(kRmThreads), args, smem_max, s));
+      RT_TRY(cudaLaunchCooperativeKernel(loop_fn, dim3(sms), dim3(kRmThreads), args, loop_smem, s));
       bar_base += (unsigned)(e0 - s0) * kLoopBarriersPerPosition * (unsigned)sms;
       continue;
     }
