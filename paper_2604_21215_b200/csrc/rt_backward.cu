@@ -720,7 +720,7 @@ size_t rowmat_smem(int d, int k_up, int cols, int rb) {
 struct LoopParams {
   const void *Wk, *Wv, *Wdn, *Wup, *Wo, *g_k, *g_kv, *g_mlp;
   int z_norm, pre, qk;
-  int cols_down, up_split;                // task shapes: columns per task of the W_down step, parts of the W_up contraction
+  int cols_pair, cols_down, cols_up, cols_out, up_split;   // task shapes: columns per task of each step, parts of the W_up contraction
   int resident;                           // 1: every step has at most one task per CTA and its weight slices fit: keep them in shared memory
   unsigned stage_bytes;                   // shared memory of the staging areas (the slices follow)
   float alpha;
@@ -759,10 +759,10 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
       }
       wsm += (size_t)Kin * cols;                              // every CTA advances alike: the layout is fixed
     };
-    stage(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, 16, 2);
+    stage(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.cols_pair, 2);
     stage(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.cols_down, 1);
-    stage(RM_UP, p.dff, p.d, lp.Wup, nullptr, 16, lp.up_split);
-    stage(RM_OUT, p.d, p.d, lp.Wo, nullptr, 16, 1);
+    stage(RM_UP, p.dff, p.d, lp.Wup, nullptr, lp.cols_up, lp.up_split);
+    stage(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.cols_out, 1);
     __syncthreads();
   }
   auto phase = [&](int mode, int K, int Ncols, const void* W1, const void* W2, const void* gain, int norm_on, float al, int cols,
@@ -785,7 +785,7 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
 #endif
   for (int i = lp.e0 - 1; i >= lp.s0; --i) {
     p.i = i;
-    phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f, 16, 2, 0);
+    phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f, lp.cols_pair, 2, 0);
     mark(0);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
     mark(1);
@@ -793,11 +793,11 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
     mark(2);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
     mark(3);
-    phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f, 16, lp.up_split, 0);
+    phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f, lp.cols_up, lp.up_split, 0);
     mark(4);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
     mark(5);
-    phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha, 16, 1, lp.up_split);
+    phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha, lp.cols_out, 1, lp.up_split);
     mark(6);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
     mark(7);
@@ -955,10 +955,13 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   const int chunks = ceil_div(B, rb);
   // task shapes: the W_up contraction in as many parts (of whole 128-row strides) as keep the grid busy once; the
   // W_down step with 32 columns per task when 16 would need more than one round of the grid
-  int up_split = 1;
-  for (int c = 4; c >= 2; --c)
-    if (f % (c * 128) == 0 && (d / 16) * chunks * c <= sms) { up_split = c; break; }
+  // 16 columns per task, 32 where 16 would need more than one round of the grid (each task repeats the step's prologue)
+  const int cols_pair = (d / 16) * chunks * 2 > sms ? 32 : 16;
+  const int cols_out = (d / 16) * chunks > sms ? 32 : 16;
   const int cols_down = (f / 16) * chunks > sms ? 32 : 16;
+  int up_split = 1, cols_up = (d / 16) * chunks > sms ? 32 : 16;
+  for (int c = 4; c >= 2; --c)
+    if (f % (c * 128) == 0 && (d / cols_up) * chunks * c <= sms) { up_split = c; break; }
   rp.part = F(L.part2); rp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   const size_t smem_max = rowmat_smem(d, f / up_split, 32, rb);
   if (smem_max > 200 * 1024) return RT_ERR_UNSUPPORTED;
@@ -979,8 +982,9 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   const char* force_steps = getenv("RT_BACKWARD_STEP_LAUNCHES");
   bool use_coop = coop && per_sm >= 1 && !(force_steps && force_steps[0] == '1');
   // weight slices resident in shared memory when every step has at most one task per CTA and they fit beside the staging
-  const size_t slice_bytes = ((size_t)d * 16 + (size_t)d * cols_down + (size_t)(f / up_split) * 16 + (size_t)d * 16) * sizeof(T);
-  const bool one_task = (d / 16) * chunks * 2 <= sms && (f / cols_down) * chunks <= sms && (d / 16) * chunks * up_split <= sms;
+  const size_t slice_bytes = ((size_t)d * cols_pair + (size_t)d * cols_down + (size_t)(f / up_split) * cols_up + (size_t)d * cols_out) * sizeof(T);
+  const bool one_task = (d / cols_pair) * chunks * 2 <= sms && (f / cols_down) * chunks <= sms && (d / cols_up) * chunks * up_split <= sms &&
+                        (d / cols_out) * chunks <= sms;
   size_t loop_smem = smem_max;
   bool resident = false;
   if (use_coop && one_task && smem_max + slice_bytes <= 220 * 1024) {
@@ -993,7 +997,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   memset(&lp, 0, sizeof(lp));
   lp.Wk = Wk; lp.Wv = Wv; lp.Wdn = Wdn; lp.Wup = Wup; lp.Wo = Wo; lp.g_k = g_k; lp.g_kv = g_kv; lp.g_mlp = g_mlp;
   lp.z_norm = z_norm ? 1 : 0; lp.pre = pre ? 1 : 0; lp.qk = qk ? 1 : 0; lp.alpha = alpha;
-  lp.cols_down = cols_down; lp.up_split = up_split;
+  lp.cols_pair = cols_pair; lp.cols_down = cols_down; lp.cols_up = cols_up; lp.cols_out = cols_out; lp.up_split = up_split;
   lp.resident = resident ? 1 : 0; lp.stage_bytes = (unsigned)smem_max;
   lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   unsigned bar_base = 0;
@@ -1016,10 +1020,10 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
       continue;
     }
     for (int i = e0 - 1; i >= s0; --i) {
-      RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f, 16, 2, 0));
+      RT_TRY(rowmat(RM_PAIR, i, d, d, Wk, Wv, g_k, 0, 1.f, cols_pair, 2, 0));
       RT_TRY(rowmat(RM_DOWN, i, d, f, Wdn, nullptr, g_kv, z_norm ? 1 : 0, alpha, cols_down, 1, 2));
-      RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f, 16, up_split, 0));
-      RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha, 16, 1, up_split));
+      RT_TRY(rowmat(RM_UP, i, f, d, Wup, nullptr, nullptr, 0, 1.f, cols_up, up_split, 0));
+      RT_TRY(rowmat(RM_OUT, i, d, d, Wo, nullptr, g_mlp, pre ? 1 : 0, alpha, cols_out, 1, up_split));
       RT_TRY(launch_chained(attn_bwd_kv_kernel, dim3(warps_grid((long long)(i - s0 + 1) * B * H)), dim3(tpb), 0, s, true, ab, i, s0));
     }
   }
