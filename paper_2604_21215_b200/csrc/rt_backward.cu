@@ -368,8 +368,10 @@ __global__ void attn_bwd_kv_tile_kernel(AttnBufs a, int q0, int q1, int k0, int 
   grid_dep_sync();
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  if (wid >= (long long)(k1 - k0) * a.B * a.H) return;
-  const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
+  const int P = k1 - k0;
+  if (wid >= (long long)P * a.B * a.H) return;
+  // consecutive warps = consecutive keys of one (sequence, head): the warps of a CTA walk the same query rows together
+  const int j = k0 + (int)(wid % P), h = (int)((wid / P) % a.H), b = (int)(wid / ((long long)P * a.H));
   const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
   // a tile of Algorithm 1 backwards: group g takes the queries q0 + g, q0 + g + 4, ...
   const int g = lane >> 3, t = lane & 7;
