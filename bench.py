@@ -646,7 +646,8 @@ def run_backward_bench(args):
                       "backward_tokens_per_s": tok / (bwd_ms * 1e-3), "backward_over_forward": bwd_ms / fwd_ms,
                       "us_per_position_reverse_loop": prof["leaf"]["ms"] * 1e3 / wl.N,
                       "gflop": 3.0 * flops_fwd / 1e9, "tflops": 3.0 * flops_fwd / (bwd_ms * 1e-3) / 1e12,
-                      "arithmetic": "fp32 on CUDA cores",
+                      "arithmetic": "reverse loop and attention terms fp32 on CUDA cores; products over all rows on the tensor cores "
+                                    "for bf16 storage",
                       "ms_by_phase": {"sweep_of_intermediates": prof["prepass"]["ms"], "reverse_loop_steps": prof["leaf"]["ms"],
                                       "reverse_loop_tiles": prof["tile"]["ms"], "products_over_all_rows": prof["other"]["ms"]},
                       "workspace_gb": ws.numel() / 1e9}))
