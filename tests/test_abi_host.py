@@ -60,6 +60,28 @@ def test_invalid_arguments_are_rejected_on_the_host():
     assert rt.rt_workspace_bytes(leafbad, 1, 16) == 0
 
 
+def test_backward_host_checks_need_no_gpu():
+    # workspace size and argument checks of the backward pass run on the host, before any CUDA call
+    cfg = rt.make_config(128, 2, 512, dtype="f32")
+    need = rt.rt_backward_workspace_bytes(cfg, 2, 64)
+    assert need > 0 and rt.rt_backward_workspace_bytes(cfg, 4, 64) > need
+    assert rt.rt_backward_workspace_bytes(rt.make_config(128, 3, 512, dtype="f32"), 2, 64) == 0
+    assert rt.rt_backward_workspace_bytes(cfg, 0, 64) == 0
+    w, gr = rt.RtLayerWeights(), rt.RtLayerGrads()
+    assert rt.rt_layer_backward(cfg, w, None, None, None, 2, 64, None, gr, None, 0, None) == rt.RT_ERR_INVALID_ARG
+    buf = (C.c_char * 4096)()
+    addr = (C.addressof(buf) + 255) & ~255
+    for n in ("w_q", "w_k", "w_v", "w_o", "w_up", "w_down"):
+        setattr(w, n, addr)
+    call = lambda c, nbytes, g=gr: rt.rt_layer_backward(c, w, addr, addr, addr, 2, 64, addr, g, addr, nbytes, None)
+    assert call(cfg, need - 1) == rt.RT_ERR_WORKSPACE
+    assert call(rt.make_config(128, 2, 512, dtype="f32", recur_block=8), need) == rt.RT_ERR_UNSUPPORTED
+    assert call(rt.make_config(128, 4, 512, dtype="f32", head_dim=32), need) == rt.RT_ERR_UNSUPPORTED
+    odd = rt.RtLayerGrads()
+    odd.w_q = addr + 4                                        # gradient arrays must be 16-byte aligned
+    assert call(cfg, need, odd) == rt.RT_ERR_INVALID_ARG
+
+
 def test_plan_counters_follow_the_n_log_n_model():
     # K/V rows streamed by the cross tiles: one half of the rows per level above the leaf.
     cfg = rt.make_config(1024, 16, 4096, dtype="bf16", leaf=64)
