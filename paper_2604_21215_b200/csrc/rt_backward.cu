@@ -199,6 +199,10 @@ __device__ __forceinline__ float gelu_f(float a) { return 0.5f * a * (1.f + erff
 __device__ __forceinline__ float gelu_grad_f(float a) {
   return 0.5f * (1.f + erff(a * 0.70710678118654752f)) + a * 0.3989422804014327f * __expf(-0.5f * a * a);
 }
+__global__ void gelu_bwd_kernel(float* __restrict__ dg, const float* __restrict__ a, long long n) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < n) dg[idx] *= gelu_grad_f(a[idx]);
+}
 __global__ void gelu_kernel(const float* __restrict__ a, float* __restrict__ out, long long n) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx < n) out[idx] = gelu_f(a[idx]);
@@ -815,10 +819,11 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
 // ------------------------------------------------------------------------------------------------ workspace
 struct BwdLayout {
   size_t sync, n, qraw, ktraw, vt, q, kt, r, kraw, k, v, c, h, u, act, gl, lse, D;
-  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2, sa, sb, wt;
+  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2, sa, sb, wt, wt5, dzp;
   size_t zero_begin, zero_end, total;
 };
 constexpr int kColParts = 128;
+constexpr int kWideBatchFrom = 32;      // above this many sequences a step of the reverse loop runs as dense products over the batch
 
 BwdLayout bwd_layout(const rt_config* c, int B, int N) {
   BwdLayout L;
@@ -838,6 +843,8 @@ BwdLayout bwd_layout(const rt_config* c, int B, int N) {
   L.dkt = take(rows * d); L.dvt = take(rows * d); L.dn = take(rows * d); L.gprod = take(rows * d);
   L.part = take((size_t)kColParts * (d > f ? d : f));
   L.part2 = take((size_t)4 * B * d);
+  // wide batches: bf16 transposes of the five matrices of the reverse loop, dL/dz in position-major order
+  L.wt5 = take((3 * d * d + 2 * d * f) / 2 + 64); L.dzp = B > kWideBatchFrom ? take(rows * d) : o;
   // bf16 operands of the tensor-core products (bf16 storage): two [rows, max(d, d_ff)] arrays and one [d, d]
   L.sa = take(rows * (d > f ? d : f) / 2 + 64); L.sb = take(rows * (d > f ? d : f) / 2 + 64); L.wt = take(d * d / 2 + 64);
   L.total = o;
@@ -1004,16 +1011,66 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   unsigned bar_base = 0;
   const int Lf = 64;                                             // leaf of the reverse schedule
+  // Wide batches (the paper's own regime, Sec. 6): a step of the reverse loop is a dense product over the B rows of the
+  // position -- tensor cores for bf16 storage -- between small row-wise kernels, instead of tasks of four sequences.
+  const bool wide = B > kWideBatchFrom;
+  const size_t pos_d = (size_t)B * d, pos_f = (size_t)B * f;
+  __nv_bfloat16* WkT = reinterpret_cast<__nv_bfloat16*>(ws + L.wt5);
+  __nv_bfloat16 *WvT = WkT + (size_t)d * d, *WoT = WvT + (size_t)d * d, *WdnT = WoT + (size_t)d * d, *WupT = WdnT + (size_t)d * f;
+  if (wide) {
+    norm_fwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(dz, xbs, xts, B, (const T*)nullptr, F(L.dzp), rows, d, d, eps, 0);
+    if (tc) {
+      auto tr = [&](const T* W, int n_out, int n_in, __nv_bfloat16* out) {
+        transpose_bf16_kernel<T><<<dim3(ceil_div(n_in, 32), ceil_div(n_out, 32)), dim3(32, 8), 0, s>>>(W, n_out, n_in, out);
+      };
+      tr(Wk, d, d, WkT); tr(Wv, d, d, WvT); tr(Wo, d, d, WoT); tr(Wdn, d, f, WdnT); tr(Wup, f, d, WupT);
+    }
+    RT_TRY(cudaGetLastError());
+  }
+  // out[B, n_in] (+)= al * dY[B, n_out] W[n_out, n_in] for the rows of one position
+  auto step_product = [&](const float* dY, int n_out, const T* W, const __nv_bfloat16* Wt, int n_in, float* out, float al, bool acc) -> cudaError_t {
+    if (!tc) return gemm<float, T>(B, n_in, n_out, dY, n_out, 1, W, n_in, 1, out, n_in, al, acc, s);
+    to_bf16(dY, SA, (long long)B * n_out); sa_holds = nullptr;
+    return tc_product(B, n_in, n_out, SA, Wt, out, al, acc);
+  };
+  auto wide_position = [&](int i, int s0) -> rt_status {
+    const size_t od = (size_t)i * pos_d, of = (size_t)i * pos_f;
+    // dk_raw = qkRMS backward of dk_i;  dr = dk_raw W_k + dv_i W_v
+    norm_bwd_kernel<float, T><<<warps_grid((long long)B * H), tpb, 0, s>>>(F(L.dK) + od, F(L.kraw) + od, pbs, pts, B, g_k, nullptr, F(L.dkraw) + od,
+                                                                          pbs, pts, nullptr, 0, B, d, kHeadDim, eps, qk);
+    RT_TRY(step_product(F(L.dkraw) + od, d, Wk, WkT, d, F(L.dr) + od, 1.f, false));
+    RT_TRY(step_product(F(L.dV) + od, d, Wv, WvT, d, F(L.dr) + od, 1.f, true));
+    // Gz = dz_i + RMS backward of dr;  dpre = (alpha Gz W_down) * GELU'
+    norm_bwd_kernel<T, T><<<warps_grid(B), tpb, 0, s>>>(F(L.dr) + od, z + (size_t)i * xts, xbs, xts, B, g_kv, F(L.dzp) + od, F(L.Gz) + od, pbs,
+                                                        pts, nullptr, 0, B, d, d, eps, z_norm ? 1 : 0);
+    RT_TRY(step_product(F(L.Gz) + od, d, Wdn, WdnT, f, F(L.dpre) + of, alpha, false));
+    gelu_bwd_kernel<<<elems_grid((long long)pos_f), tpb, 0, s>>>(F(L.dpre) + of, F(L.act) + of, (long long)pos_f);
+    // du = dpre W_up;  dh = Gz + RMS backward of du;  dc = alpha dh W_o
+    RT_TRY(step_product(F(L.dpre) + of, f, Wup, WupT, d, F(L.du) + od, 1.f, false));
+    norm_bwd_kernel<float, T><<<warps_grid(B), tpb, 0, s>>>(F(L.du) + od, F(L.h) + od, pbs, pts, B, g_mlp, F(L.Gz) + od, F(L.dh) + od, pbs, pts,
+                                                            nullptr, 0, B, d, d, eps, pre ? 1 : 0);
+    RT_TRY(step_product(F(L.dh) + od, d, Wo, WoT, d, F(L.dc) + od, alpha, false));
+    // the query's share of the pairs of its own leaf, its temporary pair and D_i
+    attn_bwd_kv_kernel<<<warps_grid((long long)(i - s0 + 1) * B * H), tpb, 0, s>>>(ab, i, s0);
+    return cudaGetLastError() == cudaSuccess ? RT_OK : RT_ERR_CUDA;
+  };
   for (int s0 = ((N - 1) / Lf) * Lf; s0 >= 0; s0 -= Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
     if (e0 < N) {                                                // Algorithm 1's tile at block end e0, backwards
       const int P = e0 & -e0;
       const int q1 = e0 + P < N ? e0 + P : N;
       ProfSpanScope span(s, 2);
-      RT_TRY(launch_chained(attn_bwd_kv_tile_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop, ab,
+      RT_TRY(launch_chained(attn_bwd_kv_tile_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop && !wide, ab,
                             e0, q1, e0 - P, e0));
     }
     ProfSpanScope span(s, 1);
+    if (wide) {
+      for (int i = e0 - 1; i >= s0; --i) {
+        const rt_status st = wide_position(i, s0);
+        if (st != RT_OK) return st;
+      }
+      continue;
+    }
     if (use_coop) {
       lp.s0 = s0; lp.e0 = e0; lp.bar_base = bar_base;
       void* args[] = {(void*)&rp, (void*)&lp, (void*)&ab};

@@ -36,7 +36,10 @@ def _case(dtype, d, H, dff, B, N, seed, gains, alibi):
     ("bf16", 256, 4, 512, 3, 200, 3, G_NAMES, False, 1.0),
     ("bf16", 128, 2, 384, 9, 130, 3, (), True, 0.6),
     ("bf16", 192, 3, 224, 2, 96, 3, ("g_mlp", "g_q"), False, 1.0),            # widths off the tensor-core products
-    ("bf16", 128, 2, 384, 3, 77, 3, G_NAMES, False, 0.8)])                   # row count off the tensor-core dW products
+    ("bf16", 128, 2, 384, 3, 77, 3, G_NAMES, False, 0.8),                    # row count off the tensor-core dW products
+    ("bf16", 128, 2, 256, 40, 70, 3, G_NAMES, True, 0.7),                    # wide batch: steps as dense products (tensor cores)
+    ("f32", 128, 2, 160, 36, 66, 3 | 8, ("g_attn", "g_k"), False, 1.0),      # wide batch, fp32 products
+    ("bf16", 192, 3, 224, 33, 65, 1, (), False, 1.0)])                       # wide batch, widths off the tensor-core products
 def test_backward_matches_gradient_oracle(dtype, d, H, dff, B, N, flags, gains, alibi, alpha):
     from oracle import RTConfig, RTWeights, layer_grad
     from paper_2604_21215_b200 import inputs, rt
