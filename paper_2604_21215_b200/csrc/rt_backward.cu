@@ -80,6 +80,7 @@ cudaError_t gemm(int M, int N, int K, const TA* A, long long a_rs, long long a_c
 
 // bf16 operands of the tensor-core products (bf16 storage only): a copy, or a transposed copy, of an fp32 / bf16 array
 __global__ void to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, long long n) {
+  grid_dep_sync();
   const long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (idx + 3 < n) {
     const float4 v = *reinterpret_cast<const float4*>(in + idx);
@@ -132,10 +133,13 @@ __global__ void norm_fwd_kernel(const TI* __restrict__ in, long long bs, long lo
 
 // With y = g u inv, inv = (mean(u^2)+eps)^(-1/2), t = g dy and uh = u inv:  du = inv (t - uh mean(t uh)),  dg += dy uh.
 // out = (add ? add : 0) + du;  gprod (=|+=) dy uh.  out and gprod may each be NULL.  !enable: du = dy.
+// out_bf (optional): a bf16 copy of bf_scale * out, [rows, d], the operand of the tensor-core product that follows.
 template <typename TU, typename TG>
 __global__ void norm_bwd_kernel(const float* dy, const TU* __restrict__ u, long long u_bs, long long u_ts, int B,
                                 const TG* __restrict__ g, const float* add, float* out, long long o_bs, long long o_ts,
-                                float* gprod, int gprod_acc, long long rows, int d, int G, float eps, int enable) {
+                                float* gprod, int gprod_acc, long long rows, int d, int G, float eps, int enable,
+                                __nv_bfloat16* out_bf = nullptr, float bf_scale = 1.f) {
+  grid_dep_sync();
   const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31, groups = d / G;
   if (wid >= rows * groups) return;
@@ -161,7 +165,9 @@ __global__ void norm_bwd_kernel(const float* dy, const TU* __restrict__ u, long 
       du = inv * (dyr[e] * gain_at(g, c0 + e) - uh * mean);
       gp = dyr[e] * uh;
     }
-    if (out) out[row_at(r, B, o_bs, o_ts) + c0 + e] = (add ? add[r * d + c0 + e] : 0.f) + du;
+    const float res = (add ? add[r * d + c0 + e] : 0.f) + du;
+    if (out) out[row_at(r, B, o_bs, o_ts) + c0 + e] = res;
+    if (out_bf) out_bf[r * d + c0 + e] = __float2bfloat16_rn(res * bf_scale);   // operand copy for the next product
     if (gprod) gprod[r * d + c0 + e] = (gprod_acc ? gprod[r * d + c0 + e] : 0.f) + gp;
   }
 }
@@ -199,9 +205,14 @@ __device__ __forceinline__ float gelu_f(float a) { return 0.5f * a * (1.f + erff
 __device__ __forceinline__ float gelu_grad_f(float a) {
   return 0.5f * (1.f + erff(a * 0.70710678118654752f)) + a * 0.3989422804014327f * __expf(-0.5f * a * a);
 }
-__global__ void gelu_bwd_kernel(float* __restrict__ dg, const float* __restrict__ a, long long n) {
+__global__ void gelu_bwd_kernel(float* __restrict__ dg, const float* __restrict__ a, long long n, __nv_bfloat16* out_bf) {
+  grid_dep_sync();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx < n) dg[idx] *= gelu_grad_f(a[idx]);
+  if (idx < n) {
+    const float v = dg[idx] * gelu_grad_f(a[idx]);
+    dg[idx] = v;
+    if (out_bf) out_bf[idx] = __float2bfloat16_rn(v);
+  }
 }
 __global__ void gelu_kernel(const float* __restrict__ a, float* __restrict__ out, long long n) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -362,6 +373,48 @@ __global__ void attn_bwd_kv_kernel(AttnBufs a, int i, int k0) {
   if (wid >= (long long)(i + 1 - k0) * a.B * a.H) return;
   const int h = (int)(wid % a.H), b = (int)((wid / a.H) % a.B), j = k0 + (int)(wid / ((long long)a.H * a.B));
   attn_self_task<false>(a, i, j, b, h, lane);
+}
+
+// In-leaf step of position i for wide batches: one warp per (sequence, head) walks the pairs [k0, i) of the leaf, four at
+// a time (a group of eight lanes per pair, which it owns: plain read-modify-write), then the temporary pair and D_i.
+__global__ void attn_self_wide_kernel(AttnBufs a, int i, int k0) {
+  grid_dep_sync();
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31, g = lane >> 3, t = lane & 7;
+  if (wid >= (long long)a.B * a.H) return;
+  const int h = (int)(wid % a.H), b = (int)(wid / a.H);
+  const long long col = (long long)h * kHeadDim + 8 * t;
+  const long long rstride = (long long)a.B * a.d;
+  const long long ri = (long long)i * rstride + (long long)b * a.d + col;
+  const long long si = ((long long)i * a.B + b) * a.H + h;
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  const F8 q = ld8(a.q + ri), dc = ld8(a.dc + ri), cc = ld8(a.c + ri);
+  const float D = group_sum(dot8(dc, cc)), lse = a.lse[si];
+  for (int j0 = k0; j0 < i; j0 += 4) {
+    const int j = j0 + g;
+    const bool valid = j < i;
+    const long long rj = (long long)(valid ? j : k0) * rstride + (long long)b * a.d + col;
+    const F8 kk = ld8(a.k + rj), vv = ld8(a.v + rj);
+    F8 gk = ld8(a.dK + rj), gv = ld8(a.dV + rj);
+    const float sd = group_sum(dot8(q, kk)), dp = group_sum(dot8(dc, vv));
+    if (valid) {
+      const float p = exp2f(sd * a.scale_log2 - slope * (float)(i - j) - lse);
+      const float ds = p * (dp - D) * a.scale;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { gk.v[e] = fmaf(ds, q.v[e], gk.v[e]); gv.v[e] = fmaf(p, dc.v[e], gv.v[e]); }
+      st8(a.dK + rj, gk); st8(a.dV + rj, gv);
+    }
+  }
+  const F8 kt = ld8(a.kt + ri), vt = ld8(a.vt + ri);
+  const float p = exp2f(group_sum(dot8(q, kt)) * a.scale_log2 - lse);
+  const float ds = p * (group_sum(dot8(dc, vt)) - D) * a.scale;
+  if (g == 0) {
+    F8 o1, o2;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { o1.v[e] = ds * q.v[e]; o2.v[e] = p * dc.v[e]; }
+    st8(a.dkt + ri, o1); st8(a.dvt + ri, o2);
+    if (t == 0) a.D[si] = D;
+  }
 }
 
 // A tile of Algorithm 1 backwards: the pairs [k0, k1) receive the share of the queries [q0, q1) (all later positions):
@@ -823,6 +876,7 @@ struct BwdLayout {
   size_t zero_begin, zero_end, total;
 };
 constexpr int kColParts = 128;
+constexpr int kWideLeaf = 16;
 constexpr int kWideBatchFrom = 32;      // above this many sequences a step of the reverse loop runs as dense products over the batch
 
 BwdLayout bwd_layout(const rt_config* c, int B, int N) {
@@ -891,11 +945,12 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   __nv_bfloat16* SA = reinterpret_cast<__nv_bfloat16*>(ws + L.sa);
   __nv_bfloat16* SB = reinterpret_cast<__nv_bfloat16*>(ws + L.sb);
   __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(ws + L.wt);
-  auto tc_product = [&](int M, int Nn, int K, const void* A, const void* W, float* out, float al, bool acc) {
+  auto tc_product = [&](int M, int Nn, int K, const void* A, const void* W, float* out, float al, bool acc, bool chained = false) {
     DenseParams dp;
     memset(&dp, 0, sizeof(dp));
     dp.M = M; dp.N = Nn; dp.K = K; dp.B = 1; dp.A = A; dp.W = W; dp.epi = DENSE_F32; dp.alpha = al; dp.accumulate = acc ? 1 : 0;
-    dp.h = out;
+    dp.h = out; dp.chained = chained ? 1 : 0;
+    if (chained) { dp.partial = F(L.gprod); dp.partial_bytes = (size_t)rows * d * sizeof(float); }   // few rows: split contraction
     return dense_launch(RT_BF16, dp, sync, s);
   };
   auto to_bf16 = [&](const float* in, __nv_bfloat16* out, long long n) {
@@ -1010,7 +1065,9 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   lp.resident = resident ? 1 : 0; lp.stage_bytes = (unsigned)smem_max;
   lp.sync = reinterpret_cast<SyncArea*>(ws + L.sync);
   unsigned bar_base = 0;
-  const int Lf = 64;                                             // leaf of the reverse schedule
+  // leaf of the reverse schedule; wide batches take short leaves (the in-leaf step re-reads and rewrites the fp32
+  // pairs of its leaf at every position, the tiles do not)
+  const int Lf = B > kWideBatchFrom ? kWideLeaf : 64;
   // Wide batches (the paper's own regime, Sec. 6): a step of the reverse loop is a dense product over the B rows of the
   // position -- tensor cores for bf16 storage -- between small row-wise kernels, instead of tasks of four sequences.
   const bool wide = B > kWideBatchFrom;
@@ -1027,32 +1084,42 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     }
     RT_TRY(cudaGetLastError());
   }
-  // out[B, n_in] (+)= al * dY[B, n_out] W[n_out, n_in] for the rows of one position
-  auto step_product = [&](const float* dY, int n_out, const T* W, const __nv_bfloat16* Wt, int n_in, float* out, float al, bool acc) -> cudaError_t {
+  // out[B, n_in] (+)= al * dY[B, n_out] W[n_out, n_in] for the rows of one position; A_bf = bf16 copy of dY (scale folded in)
+  auto step_product = [&](const float* dY, const __nv_bfloat16* A_bf, int n_out, const T* W, const __nv_bfloat16* Wt, int n_in, float* out,
+                          float al, bool acc) -> cudaError_t {
     if (!tc) return gemm<float, T>(B, n_in, n_out, dY, n_out, 1, W, n_in, 1, out, n_in, al, acc, s);
-    to_bf16(dY, SA, (long long)B * n_out); sa_holds = nullptr;
-    return tc_product(B, n_in, n_out, SA, Wt, out, al, acc);
+    return tc_product(B, n_in, n_out, A_bf, Wt, out, 1.f, acc, true);
   };
+  // The launches of a position are chained (programmatic dependent launches); each producer also leaves the bf16 operand
+  // of the product that follows (SA, SB), so a position is eleven launches.
   auto wide_position = [&](int i, int s0) -> rt_status {
     const size_t od = (size_t)i * pos_d, of = (size_t)i * pos_f;
+    sa_holds = nullptr;
+    const dim3 blk(tpb);
     // dk_raw = qkRMS backward of dk_i;  dr = dk_raw W_k + dv_i W_v
-    norm_bwd_kernel<float, T><<<warps_grid((long long)B * H), tpb, 0, s>>>(F(L.dK) + od, F(L.kraw) + od, pbs, pts, B, g_k, nullptr, F(L.dkraw) + od,
-                                                                          pbs, pts, nullptr, 0, B, d, kHeadDim, eps, qk);
-    RT_TRY(step_product(F(L.dkraw) + od, d, Wk, WkT, d, F(L.dr) + od, 1.f, false));
-    RT_TRY(step_product(F(L.dV) + od, d, Wv, WvT, d, F(L.dr) + od, 1.f, true));
+    RT_TRY(launch_chained(norm_bwd_kernel<float, T>, dim3(warps_grid((long long)B * H)), blk, 0, s, true, (const float*)(F(L.dK) + od),
+                          (const float*)(F(L.kraw) + od), pbs, pts, B, g_k, (const float*)nullptr, F(L.dkraw) + od, pbs, pts, (float*)nullptr, 0,
+                          (long long)B, d, (int)kHeadDim, eps, qk ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, 1.f));
+    if (tc) RT_TRY(launch_chained(to_bf16_kernel, dim3(elems_grid((long long)(pos_d + 3) / 4)), blk, 0, s, true, (const float*)(F(L.dV) + od), SB,
+                                  (long long)pos_d));
+    RT_TRY(step_product(F(L.dkraw) + od, SA, d, Wk, WkT, d, F(L.dr) + od, 1.f, false));
+    RT_TRY(step_product(F(L.dV) + od, SB, d, Wv, WvT, d, F(L.dr) + od, 1.f, true));
     // Gz = dz_i + RMS backward of dr;  dpre = (alpha Gz W_down) * GELU'
-    norm_bwd_kernel<T, T><<<warps_grid(B), tpb, 0, s>>>(F(L.dr) + od, z + (size_t)i * xts, xbs, xts, B, g_kv, F(L.dzp) + od, F(L.Gz) + od, pbs,
-                                                        pts, nullptr, 0, B, d, d, eps, z_norm ? 1 : 0);
-    RT_TRY(step_product(F(L.Gz) + od, d, Wdn, WdnT, f, F(L.dpre) + of, alpha, false));
-    gelu_bwd_kernel<<<elems_grid((long long)pos_f), tpb, 0, s>>>(F(L.dpre) + of, F(L.act) + of, (long long)pos_f);
+    RT_TRY(launch_chained(norm_bwd_kernel<T, T>, dim3(warps_grid(B)), blk, 0, s, true, (const float*)(F(L.dr) + od), z + (size_t)i * xts, xbs, xts, B,
+                          g_kv, (const float*)(F(L.dzp) + od), F(L.Gz) + od, pbs, pts, (float*)nullptr, 0, (long long)B, d, d, eps,
+                          z_norm ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
+    RT_TRY(step_product(F(L.Gz) + od, SA, d, Wdn, WdnT, f, F(L.dpre) + of, alpha, false));
+    RT_TRY(launch_chained(gelu_bwd_kernel, dim3(elems_grid((long long)pos_f)), blk, 0, s, true, F(L.dpre) + of, (const float*)(F(L.act) + of),
+                          (long long)pos_f, tc ? SA : (__nv_bfloat16*)nullptr));
     // du = dpre W_up;  dh = Gz + RMS backward of du;  dc = alpha dh W_o
-    RT_TRY(step_product(F(L.dpre) + of, f, Wup, WupT, d, F(L.du) + od, 1.f, false));
-    norm_bwd_kernel<float, T><<<warps_grid(B), tpb, 0, s>>>(F(L.du) + od, F(L.h) + od, pbs, pts, B, g_mlp, F(L.Gz) + od, F(L.dh) + od, pbs, pts,
-                                                            nullptr, 0, B, d, d, eps, pre ? 1 : 0);
-    RT_TRY(step_product(F(L.dh) + od, d, Wo, WoT, d, F(L.dc) + od, alpha, false));
+    RT_TRY(step_product(F(L.dpre) + of, SA, f, Wup, WupT, d, F(L.du) + od, 1.f, false));
+    RT_TRY(launch_chained(norm_bwd_kernel<float, T>, dim3(warps_grid(B)), blk, 0, s, true, (const float*)(F(L.du) + od), (const float*)(F(L.h) + od),
+                          pbs, pts, B, g_mlp, (const float*)(F(L.Gz) + od), F(L.dh) + od, pbs, pts, (float*)nullptr, 0, (long long)B, d, d, eps,
+                          pre ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
+    RT_TRY(step_product(F(L.dh) + od, SA, d, Wo, WoT, d, F(L.dc) + od, alpha, false));
     // the query's share of the pairs of its own leaf, its temporary pair and D_i
-    attn_bwd_kv_kernel<<<warps_grid((long long)(i - s0 + 1) * B * H), tpb, 0, s>>>(ab, i, s0);
-    return cudaGetLastError() == cudaSuccess ? RT_OK : RT_ERR_CUDA;
+    RT_TRY(launch_chained(attn_self_wide_kernel, dim3(warps_grid((long long)B * H)), blk, 0, s, true, ab, i, s0));
+    return RT_OK;
   };
   for (int s0 = ((N - 1) / Lf) * Lf; s0 >= 0; s0 -= Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;

@@ -324,6 +324,10 @@ __global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) 
     } else if (p.epi == DENSE_GELU) {
       v = gelu_exact(acc);
       reinterpret_cast<T*>(p.out)[(size_t)m * p.N + n] = from_f<T>(v);
+    } else if (p.epi == DENSE_F32) {
+      float* dst = p.h + (size_t)m * p.N + n;
+      v = (p.accumulate ? *dst : 0.f) + p.alpha * acc;
+      *dst = v;
     } else {
       const T zr = from_f<T>(p.h[(size_t)m * p.N + n] + p.alpha * acc);
       reinterpret_cast<T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n] = zr;
