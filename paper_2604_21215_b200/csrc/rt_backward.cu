@@ -172,6 +172,42 @@ __global__ void norm_bwd_kernel(const float* dy, const TU* __restrict__ u, long 
   }
 }
 
+// The same backward of a full-width RMS (G = d) with one CTA of 256 threads per row: for the few rows of one position
+// of a wide batch, where a warp per row would leave the GPU idle.
+template <typename TU, typename TG>
+__global__ void __launch_bounds__(256) norm_bwd_row_kernel(const float* dy, const TU* __restrict__ u, long long u_bs, long long u_ts, int B,
+                                                           const TG* __restrict__ g, const float* add, float* out, int d, float eps,
+                                                           int enable, __nv_bfloat16* out_bf, float bf_scale) {
+  grid_dep_sync();
+  __shared__ float red[2][8];
+  const long long r = blockIdx.x;
+  const int tid = threadIdx.x;
+  const float* dyr = dy + r * d;
+  const TU* ur = u + row_at(r, B, u_bs, u_ts);
+  float ss = 0.f, tu = 0.f;
+  if (enable) {
+    for (int e = tid; e < d; e += 256) {
+      const float v = to_f(ur[e]);
+      ss = fmaf(v, v, ss);
+      tu = fmaf(dyr[e] * gain_at(g, e), v, tu);
+    }
+    ss = warp_sum(ss); tu = warp_sum(tu);
+    if ((tid & 31) == 0) { red[0][tid >> 5] = ss; red[1][tid >> 5] = tu; }
+    __syncthreads();
+    ss = 0.f; tu = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { ss += red[0][w]; tu += red[1][w]; }
+  }
+  const float inv = rsqrtf(ss / d + eps), mean = tu * inv / d;
+  for (int e = tid; e < d; e += 256) {
+    float du = dyr[e];
+    if (enable) du = inv * (dyr[e] * gain_at(g, e) - to_f(ur[e]) * inv * mean);
+    const float res = add[r * d + e] + du;
+    out[r * d + e] = res;
+    if (out_bf) out_bf[r * d + e] = __float2bfloat16_rn(res * bf_scale);
+  }
+}
+
 // column sums of a [rows, d] array in two fixed-order steps
 __global__ void col_partial_kernel(const float* __restrict__ a, long long rows, int d, float* __restrict__ part, int P) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1105,17 +1141,16 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     RT_TRY(step_product(F(L.dkraw) + od, SA, d, Wk, WkT, d, F(L.dr) + od, 1.f, false));
     RT_TRY(step_product(F(L.dV) + od, SB, d, Wv, WvT, d, F(L.dr) + od, 1.f, true));
     // Gz = dz_i + RMS backward of dr;  dpre = (alpha Gz W_down) * GELU'
-    RT_TRY(launch_chained(norm_bwd_kernel<T, T>, dim3(warps_grid(B)), blk, 0, s, true, (const float*)(F(L.dr) + od), z + (size_t)i * xts, xbs, xts, B,
-                          g_kv, (const float*)(F(L.dzp) + od), F(L.Gz) + od, pbs, pts, (float*)nullptr, 0, (long long)B, d, d, eps,
-                          z_norm ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
+    RT_TRY(launch_chained(norm_bwd_row_kernel<T, T>, dim3(B), dim3(256), 0, s, true, (const float*)(F(L.dr) + od), z + (size_t)i * xts, xbs, xts, B,
+                          g_kv, (const float*)(F(L.dzp) + od), F(L.Gz) + od, d, eps, z_norm ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
     RT_TRY(step_product(F(L.Gz) + od, SA, d, Wdn, WdnT, f, F(L.dpre) + of, alpha, false));
     RT_TRY(launch_chained(gelu_bwd_kernel, dim3(elems_grid((long long)pos_f)), blk, 0, s, true, F(L.dpre) + of, (const float*)(F(L.act) + of),
                           (long long)pos_f, tc ? SA : (__nv_bfloat16*)nullptr));
     // du = dpre W_up;  dh = Gz + RMS backward of du;  dc = alpha dh W_o
     RT_TRY(step_product(F(L.dpre) + of, SA, f, Wup, WupT, d, F(L.du) + od, 1.f, false));
-    RT_TRY(launch_chained(norm_bwd_kernel<float, T>, dim3(warps_grid(B)), blk, 0, s, true, (const float*)(F(L.du) + od), (const float*)(F(L.h) + od),
-                          pbs, pts, B, g_mlp, (const float*)(F(L.Gz) + od), F(L.dh) + od, pbs, pts, (float*)nullptr, 0, (long long)B, d, d, eps,
-                          pre ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
+    RT_TRY(launch_chained(norm_bwd_row_kernel<float, T>, dim3(B), dim3(256), 0, s, true, (const float*)(F(L.du) + od), (const float*)(F(L.h) + od),
+                          pbs, pts, B, g_mlp, (const float*)(F(L.Gz) + od), F(L.dh) + od, d, eps, pre ? 1 : 0,
+                          tc ? SA : (__nv_bfloat16*)nullptr, alpha));
     RT_TRY(step_product(F(L.dh) + od, SA, d, Wo, WoT, d, F(L.dc) + od, alpha, false));
     // the query's share of the pairs of its own leaf, its temporary pair and D_i
     RT_TRY(launch_chained(attn_self_wide_kernel, dim3(warps_grid((long long)B * H)), blk, 0, s, true, ab, i, s0));
