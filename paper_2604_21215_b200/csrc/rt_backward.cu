@@ -363,6 +363,35 @@ __global__ void attn_stats_kernel(AttnBufs a) {
   }
 }
 
+// Tensor-core route of the attention statistics (bf16 storage): the running softmax state (o, m in log2 units, l) is
+// seeded with the temporary pair here, advanced over all earlier pairs by the forward pass's own tile kernels
+// (Algorithm 2), and turned into c = o / l and the log2-sum-exp afterwards.  One warp per (position, sequence, head).
+__global__ void stats_seed_kernel(AttnBufs a, float* st_o, float* st_m, float* st_l) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)a.N * a.B * a.H) return;
+  const int h = (int)(wid % a.H);
+  const long long row = wid / a.H;
+  const long long at = row * a.d + (long long)h * kHeadDim + 2 * lane;
+  const float2 q = *reinterpret_cast<const float2*>(a.q + at), kt = *reinterpret_cast<const float2*>(a.kt + at);
+  const float s = warp_sum(q.x * kt.x + q.y * kt.y) * a.scale_log2;
+  *reinterpret_cast<float2*>(st_o + at) = *reinterpret_cast<const float2*>(a.vt + at);
+  if (lane == 0) { st_m[row * a.H + h] = s; st_l[row * a.H + h] = 1.f; }
+}
+__global__ void stats_finish_kernel(AttnBufs a, float* st_o, float* st_m, const float* st_l) {
+  const long long wid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (long long)a.N * a.B * a.H) return;
+  const int h = (int)(wid % a.H);
+  const long long row = wid / a.H;
+  const long long at = row * a.d + (long long)h * kHeadDim + 2 * lane;
+  const float l = st_l[row * a.H + h], inv = 1.f / l;
+  float2 o = *reinterpret_cast<const float2*>(st_o + at);
+  o.x *= inv; o.y *= inv;
+  *reinterpret_cast<float2*>(st_o + at) = o;                   // c in place
+  if (lane == 0) st_m[row * a.H + h] += log2f(l);              // log2-sum-exp in place
+}
+
 // State of the reverse loop written earlier in the SAME (cooperative) kernel by other CTAs must not come from L1.
 template <bool COOP> __device__ __forceinline__ float ld_state(const float* p) { return COOP ? __ldcg(p) : *p; }
 template <bool COOP> __device__ __forceinline__ float2 ld_state2(const float* p) {
@@ -908,7 +937,7 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
 // ------------------------------------------------------------------------------------------------ workspace
 struct BwdLayout {
   size_t sync, n, qraw, ktraw, vt, q, kt, r, kraw, k, v, c, h, u, act, gl, lse, D;
-  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2, sa, sb, wt, wt5, dzp;
+  size_t dK, dV, dkraw, dr, Gz, dpre, du, dh, dc, dq, dkt, dvt, dn, gprod, part, part2, sa, sb, wt, wt5, dzp, qkv16;
   size_t zero_begin, zero_end, total;
 };
 constexpr int kColParts = 128;
@@ -934,6 +963,7 @@ BwdLayout bwd_layout(const rt_config* c, int B, int N) {
   L.part = take((size_t)kColParts * (d > f ? d : f));
   L.part2 = take((size_t)4 * B * d);
   // wide batches: bf16 transposes of the five matrices of the reverse loop, dL/dz in position-major order
+  L.qkv16 = take(3 * rows * d / 2 + 64);                       // bf16 copies of q, k, v for the tile kernels
   L.wt5 = take((3 * d * d + 2 * d * f) / 2 + 64); L.dzp = B > kWideBatchFrom ? take(rows * d) : o;
   // bf16 operands of the tensor-core products (bf16 storage): two [rows, max(d, d_ff)] arrays and one [d, d]
   L.sa = take(rows * (d > f ? d : f) / 2 + 64); L.sb = take(rows * (d > f ? d : f) / 2 + 64); L.wt = take(d * d / 2 + 64);
@@ -1031,7 +1061,39 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   ab.c = F(L.c); ab.dc = F(L.dc); ab.dK = F(L.dK); ab.dV = F(L.dV); ab.dkt = F(L.dkt); ab.dvt = F(L.dvt); ab.dq = F(L.dq);
   ab.alibi = w->alibi_slopes; ab.scale = c->softmax_scale; ab.scale_log2 = c->softmax_scale * kLog2e;
   ab.B = B; ab.H = H; ab.d = d; ab.N = N;
-  attn_stats_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
+  if (tc) {
+    // running softmax state in place of (c, lse, D): seed, the forward pass's tile kernels, finish
+    float *st_o = F(L.c), *st_m = F(L.lse), *st_l = F(L.D);
+    __nv_bfloat16* q16 = reinterpret_cast<__nv_bfloat16*>(ws + L.qkv16);
+    __nv_bfloat16 *k16 = q16 + rows * d, *v16 = k16 + rows * d;
+    to_bf16(F(L.q), q16, rows * d); to_bf16(F(L.k), k16, rows * d); to_bf16(F(L.v), v16, rows * d);
+    stats_seed_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab, st_o, st_m, st_l);
+    TileParams tp;
+    memset(&tp, 0, sizeof(tp));
+    tp.B = B; tp.d = d; tp.H = H; tp.scale_log2 = ab.scale_log2; tp.alibi = w->alibi_slopes;
+    tp.q = q16; tp.k_cache = k16; tp.v_cache = v16; tp.st_o = st_o; tp.st_m = st_m; tp.st_l = st_l;
+    tp.rows_q = N; tp.rows_kv = N; tp.sync = sync; tp.q_limit = N;
+    const int Lb = 128;                                         // diagonal blocks under the causal mask, then Algorithm 1's levels
+    const int full = N / Lb;
+    tp.causal = 1;
+    if (full > 0) {
+      tp.q0 = 0; tp.q1 = Lb; tp.k0 = 0; tp.k1 = Lb; tp.batch = full; tp.batch_stride = Lb;
+      RT_TRY(tile_launch(RT_BF16, tp, s));
+    }
+    if (full * Lb < N) {
+      tp.q0 = full * Lb; tp.q1 = N; tp.k0 = full * Lb; tp.k1 = N; tp.batch = 1; tp.batch_stride = 0;
+      RT_TRY(tile_simt_launch(RT_BF16, tp, s));
+    }
+    tp.causal = 0;
+    for (long long P = Lb; P < N; P *= 2) {
+      tp.q0 = (int)P; tp.q1 = (int)(2 * P); tp.k0 = 0; tp.k1 = (int)P;
+      tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
+      RT_TRY(tile_launch(RT_BF16, tp, s));
+    }
+    stats_finish_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab, st_o, st_m, st_l);
+  } else {
+    attn_stats_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
+  }
   RT_TRY(fwd_product(F(L.c), d, Wo, d, F(L.dn)));                     // a = W_o c (dn as scratch)
   residual_kernel<T><<<elems_grid(rows * d), tpb, 0, s>>>(x, xbs, xts, B, F(L.dn), alpha, F(L.h), rows, d);
   norm_fwd_kernel<float, T><<<warps_grid(rows), tpb, 0, s>>>(F(L.h), pbs, pts, B, g_mlp, F(L.u), rows, d, d, eps, pre ? 1 : 0);
