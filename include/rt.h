@@ -215,6 +215,7 @@ rt_status rt_layer_recompute(const rt_config *cfg, const rt_layer_weights *w, co
  * accumulating only d(k_j, v_j) -- position i needs dL/dz_i, which needs d(k_i, v_i) complete; pairs in other leaves
  * of 64 positions receive their share from Algorithm 1's tiles run backwards -- and finally forms dq, the temporary
  * pairs, dx and every parameter gradient as products over all B*N rows at once.
+ * Batches above 32 sequences run each step of the reverse loop as dense products over the batch (Sec. 6's regime).
  * The reverse loop and the attention terms are fp32 on CUDA cores; with bf16 storage the products over all rows run
  * on the tensor cores (operands rounded to bf16, fp32 accumulation).  recur_block > 1 returns RT_ERR_UNSUPPORTED.
  * The workspace needs rt_backward_workspace_bytes (about 30 fp32 arrays of B*N*d plus 3 of B*N*d_ff). */
