@@ -532,6 +532,102 @@ __global__ void attn_bwd_kv_tile_kernel(AttnBufs a, int q0, int q1, int k0, int 
   }
 }
 
+// The same tile with 64 x 64 blocks of (query, key) pairs held in shared memory (key counts that are multiples of 64):
+// one CTA per (64 keys, sequence, head); for each block of 64 queries it forms S = Q K^T and dP = dC V^T as 4 x 4
+// register tiles per thread, P and dS from them, and adds dS^T Q to dk and P^T dC to dv -- every operand row is fetched
+// once per block instead of once per pair.  Queries in order, fixed summation order, no atomics.
+constexpr int kPB = 64, kPBS = kPB + 1;                        // block edge, padded row stride in shared memory
+constexpr size_t kPairBlockSmem = (6 * kPB * kPBS + 2 * kPB) * sizeof(float);
+__global__ void __launch_bounds__(256) attn_bwd_kv_block_kernel(AttnBufs a, int q0, int q1, int k0, int k1) {
+  grid_dep_sync();
+  extern __shared__ __align__(16) float sm[];
+  float *Qs = sm, *Cs = Qs + kPB * kPBS, *Ks = Cs + kPB * kPBS, *Vs = Ks + kPB * kPBS, *Ps = Vs + kPB * kPBS, *Ss = Ps + kPB * kPBS;
+  float *lse_s = Ss + kPB * kPBS, *D_s = lse_s + kPB;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int b = blockIdx.y / a.H, h = blockIdx.y % a.H;
+  const int kb = k0 + kPB * blockIdx.x;
+  const long long col0 = (long long)b * a.d + (long long)h * kHeadDim;
+  const long long rstride = (long long)a.B * a.d;
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  for (int idx = tid; idx < kPB * 16; idx += 256) {             // the 64 keys of this CTA: rows of 64 entries as 16 float4
+    const int j = idx >> 4, e4 = (idx & 15) * 4;
+    const float4 kk = *reinterpret_cast<const float4*>(a.k + (long long)(kb + j) * rstride + col0 + e4);
+    const float4 vv = *reinterpret_cast<const float4*>(a.v + (long long)(kb + j) * rstride + col0 + e4);
+    float* kd = Ks + j * kPBS + e4; kd[0] = kk.x; kd[1] = kk.y; kd[2] = kk.z; kd[3] = kk.w;
+    float* vd = Vs + j * kPBS + e4; vd[0] = vv.x; vd[1] = vv.y; vd[2] = vv.z; vd[3] = vv.w;
+  }
+  float dk[4][4] = {}, dv[4][4] = {};                           // keys ty + 16 jj, entries tx + 16 ee
+  for (int qb = q0; qb < q1; qb += kPB) {
+    const int nq = q1 - qb < kPB ? q1 - qb : kPB;
+    __syncthreads();                                            // the previous block's tiles are no longer read
+    for (int idx = tid; idx < kPB * 16; idx += 256) {
+      const int i = idx >> 4, e4 = (idx & 15) * 4;
+      float4 qq = make_float4(0.f, 0.f, 0.f, 0.f), cc = qq;
+      if (i < nq) {
+        qq = *reinterpret_cast<const float4*>(a.q + (long long)(qb + i) * rstride + col0 + e4);
+        cc = *reinterpret_cast<const float4*>(a.dc + (long long)(qb + i) * rstride + col0 + e4);
+      }
+      float* qd = Qs + i * kPBS + e4; qd[0] = qq.x; qd[1] = qq.y; qd[2] = qq.z; qd[3] = qq.w;
+      float* cd = Cs + i * kPBS + e4; cd[0] = cc.x; cd[1] = cc.y; cd[2] = cc.z; cd[3] = cc.w;
+    }
+    if (tid < kPB) {
+      const long long si = ((long long)(qb + (tid < nq ? tid : 0)) * a.B + b) * a.H + h;
+      lse_s[tid] = a.lse[si]; D_s[tid] = a.D[si];
+    }
+    __syncthreads();
+    // S and dP: queries ty + 16 ii, keys tx + 16 jj
+    float sv[4][4] = {}, dp[4][4] = {};
+#pragma unroll 4
+    for (int e = 0; e < kPB; ++e) {
+      float qv[4], cv[4], kv[4], vv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        qv[u] = Qs[(ty + 16 * u) * kPBS + e]; cv[u] = Cs[(ty + 16 * u) * kPBS + e];
+        kv[u] = Ks[(tx + 16 * u) * kPBS + e]; vv[u] = Vs[(tx + 16 * u) * kPBS + e];
+      }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) { sv[ii][jj] = fmaf(qv[ii], kv[jj], sv[ii][jj]); dp[ii][jj] = fmaf(cv[ii], vv[jj], dp[ii][jj]); }
+    }
+#pragma unroll
+    for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int il = ty + 16 * ii, jl = tx + 16 * jj;
+        float p = 0.f, ds = 0.f;
+        if (il < nq) {
+          p = exp2f(sv[ii][jj] * a.scale_log2 - slope * (float)(qb + il - kb - jl) - lse_s[il]);
+          ds = p * (dp[ii][jj] - D_s[il]) * a.scale;
+        }
+        Ps[il * kPBS + jl] = p; Ss[il * kPBS + jl] = ds;
+      }
+    __syncthreads();
+    // dk += dS^T Q, dv += P^T dC: keys ty + 16 jj, entries tx + 16 ee
+#pragma unroll 4
+    for (int i = 0; i < kPB; ++i) {
+      float sj[4], pj[4], qe[4], ce[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        sj[u] = Ss[i * kPBS + ty + 16 * u]; pj[u] = Ps[i * kPBS + ty + 16 * u];
+        qe[u] = Qs[i * kPBS + tx + 16 * u]; ce[u] = Cs[i * kPBS + tx + 16 * u];
+      }
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+        for (int ee = 0; ee < 4; ++ee) { dk[jj][ee] = fmaf(sj[jj], qe[ee], dk[jj][ee]); dv[jj][ee] = fmaf(pj[jj], ce[ee], dv[jj][ee]); }
+    }
+  }
+#pragma unroll
+  for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+    for (int ee = 0; ee < 4; ++ee) {
+      const long long at = (long long)(kb + ty + 16 * jj) * rstride + col0 + tx + 16 * ee;
+      a.dK[at] += dk[jj][ee];
+      a.dV[at] += dv[jj][ee];
+    }
+}
+
 // Gradient of the queries, all positions at once: dq_i = scale (sum_{j<i} ds_ij k_j + ds_ii~ k~_i).  Same layout as
 // attn_stats_kernel: one warp per four consecutive positions of one (sequence, head), group g = position 4 iq + g.
 __global__ void attn_bwd_q_kernel(AttnBufs a) {
@@ -1218,14 +1314,20 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     RT_TRY(launch_chained(attn_self_wide_kernel, dim3(warps_grid((long long)B * H)), blk, 0, s, true, ab, i, s0));
     return RT_OK;
   };
+  RT_TRY(cudaFuncSetAttribute(attn_bwd_kv_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairBlockSmem));
   for (int s0 = ((N - 1) / Lf) * Lf; s0 >= 0; s0 -= Lf) {
     const int e0 = s0 + Lf < N ? s0 + Lf : N;
     if (e0 < N) {                                                // Algorithm 1's tile at block end e0, backwards
       const int P = e0 & -e0;
       const int q1 = e0 + P < N ? e0 + P : N;
       ProfSpanScope span(s, 2);
-      RT_TRY(launch_chained(attn_bwd_kv_tile_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop && !wide, ab,
-                            e0, q1, e0 - P, e0));
+      if (P % kPB == 0 && (long long)B * H <= 65535) {
+        RT_TRY(launch_chained(attn_bwd_kv_block_kernel, dim3(P / kPB, B * H), dim3(256), kPairBlockSmem, s, !use_coop && !wide, ab, e0, q1,
+                              e0 - P, e0));
+      } else {
+        RT_TRY(launch_chained(attn_bwd_kv_tile_kernel, dim3(warps_grid((long long)P * B * H)), dim3(tpb), 0, s, !use_coop && !wide, ab,
+                              e0, q1, e0 - P, e0));
+      }
     }
     ProfSpanScope span(s, 1);
     if (wide) {
