@@ -687,6 +687,119 @@ __global__ void attn_bwd_q_kernel(AttnBufs a) {
   if (live) st8(a.dq + ri, out);
 }
 
+// dq of all positions with 64 x 64 blocks of pairs in shared memory: one CTA per (64 queries, sequence, head) walks the
+// key blocks up to its own (pairs j < i only), forms S and dP as register tiles, dS from them, and adds dS K to dq;
+// the temporary pair of each position is added at the end.
+constexpr size_t kPairBlockSmemQ = (5 * kPB * kPBS + 2 * kPB) * sizeof(float);
+__global__ void __launch_bounds__(256) attn_bwd_q_block_kernel(AttnBufs a) {
+  extern __shared__ __align__(16) float sm[];
+  float *Qs = sm, *Cs = Qs + kPB * kPBS, *Ks = Cs + kPB * kPBS, *Vs = Ks + kPB * kPBS, *Ss = Vs + kPB * kPBS;
+  float *lse_s = Ss + kPB * kPBS, *D_s = lse_s + kPB;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int b = blockIdx.y / a.H, h = blockIdx.y % a.H;
+  const int qb = kPB * blockIdx.x;
+  const int nq = a.N - qb < kPB ? a.N - qb : kPB;
+  const long long col0 = (long long)b * a.d + (long long)h * kHeadDim;
+  const long long rstride = (long long)a.B * a.d;
+  const float slope = a.alibi ? a.alibi[h] * kLog2e : 0.f;
+  for (int idx = tid; idx < kPB * 16; idx += 256) {
+    const int i = idx >> 4, e4 = (idx & 15) * 4;
+    float4 qq = make_float4(0.f, 0.f, 0.f, 0.f), cc = qq;
+    if (i < nq) {
+      qq = *reinterpret_cast<const float4*>(a.q + (long long)(qb + i) * rstride + col0 + e4);
+      cc = *reinterpret_cast<const float4*>(a.dc + (long long)(qb + i) * rstride + col0 + e4);
+    }
+    float* qd = Qs + i * kPBS + e4; qd[0] = qq.x; qd[1] = qq.y; qd[2] = qq.z; qd[3] = qq.w;
+    float* cd = Cs + i * kPBS + e4; cd[0] = cc.x; cd[1] = cc.y; cd[2] = cc.z; cd[3] = cc.w;
+  }
+  if (tid < kPB) {
+    const long long si = ((long long)(qb + (tid < nq ? tid : 0)) * a.B + b) * a.H + h;
+    lse_s[tid] = a.lse[si]; D_s[tid] = a.D[si];
+  }
+  float dq[4][4] = {};                                          // queries ty + 16 ii, entries tx + 16 ee
+  const int k_end = qb + nq - 1;                                // pairs j < i <= qb + nq - 1
+  for (int kb = 0; kb < k_end; kb += kPB) {
+    const int nk = k_end - kb < kPB ? k_end - kb : kPB;
+    __syncthreads();
+    for (int idx = tid; idx < kPB * 16; idx += 256) {
+      const int j = idx >> 4, e4 = (idx & 15) * 4;
+      float4 kk = make_float4(0.f, 0.f, 0.f, 0.f), vv = kk;
+      if (j < nk) {
+        kk = *reinterpret_cast<const float4*>(a.k + (long long)(kb + j) * rstride + col0 + e4);
+        vv = *reinterpret_cast<const float4*>(a.v + (long long)(kb + j) * rstride + col0 + e4);
+      }
+      float* kd = Ks + j * kPBS + e4; kd[0] = kk.x; kd[1] = kk.y; kd[2] = kk.z; kd[3] = kk.w;
+      float* vd = Vs + j * kPBS + e4; vd[0] = vv.x; vd[1] = vv.y; vd[2] = vv.z; vd[3] = vv.w;
+    }
+    __syncthreads();
+    float sv[4][4] = {}, dp[4][4] = {};
+#pragma unroll 4
+    for (int e = 0; e < kPB; ++e) {
+      float qv[4], cv[4], kv[4], vv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        qv[u] = Qs[(ty + 16 * u) * kPBS + e]; cv[u] = Cs[(ty + 16 * u) * kPBS + e];
+        kv[u] = Ks[(tx + 16 * u) * kPBS + e]; vv[u] = Vs[(tx + 16 * u) * kPBS + e];
+      }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) { sv[ii][jj] = fmaf(qv[ii], kv[jj], sv[ii][jj]); dp[ii][jj] = fmaf(cv[ii], vv[jj], dp[ii][jj]); }
+    }
+#pragma unroll
+    for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int il = ty + 16 * ii, jl = tx + 16 * jj;
+        const int i = qb + il, j = kb + jl;
+        float ds = 0.f;
+        if (il < nq && j < i)
+          ds = exp2f(sv[ii][jj] * a.scale_log2 - slope * (float)(i - j) - lse_s[il]) * (dp[ii][jj] - D_s[il]);
+        Ss[il * kPBS + jl] = ds;
+      }
+    __syncthreads();
+#pragma unroll 4
+    for (int j = 0; j < kPB; ++j) {
+      float si[4], ke[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { si[u] = Ss[(ty + 16 * u) * kPBS + j]; ke[u] = Ks[j * kPBS + tx + 16 * u]; }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii)
+#pragma unroll
+        for (int ee = 0; ee < 4; ++ee) dq[ii][ee] = fmaf(si[ii], ke[ee], dq[ii][ee]);
+    }
+  }
+  // the temporary pair of each position: one warp per eight queries, then the scaled sum goes out
+  __syncthreads();
+  {
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int il = warp; il < kPB; il += 8) {
+      float ds = 0.f;
+      if (il < nq) {
+        const long long at = (long long)(qb + il) * rstride + col0;
+        const float kt0 = a.kt[at + lane], kt1 = a.kt[at + lane + 32], vt0 = a.vt[at + lane], vt1 = a.vt[at + lane + 32];
+        const float st = warp_sum(Qs[il * kPBS + lane] * kt0 + Qs[il * kPBS + lane + 32] * kt1);
+        const float dpt = warp_sum(Cs[il * kPBS + lane] * vt0 + Cs[il * kPBS + lane + 32] * vt1);
+        ds = exp2f(st * a.scale_log2 - lse_s[il]) * (dpt - D_s[il]);
+      }
+      if (lane == 0) Ss[il * kPBS] = ds;                        // column 0 of Ss: ds of the temporary pair
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int ii = 0; ii < 4; ++ii) {
+    const int il = ty + 16 * ii;
+    if (il < nq) {
+      const long long at = (long long)(qb + il) * rstride + col0;
+#pragma unroll
+      for (int ee = 0; ee < 4; ++ee) {
+        const int e = tx + 16 * ee;
+        a.dq[at + e] = (dq[ii][ee] + Ss[il * kPBS] * a.kt[at + e]) * a.scale;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ the reverse loop's products
 // One position i, the B rows of the batch: out[b, n] = alpha * (sum_k in1[b,k] W1[k,n] + sum_k in2[b,k] W2[k,n]) where the
 // rows in1 (in2) are built by a prologue from the state of the reverse loop (mode), W = a weight matrix as stored
@@ -1355,7 +1468,12 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
 
   // ---- 3. everything else over all rows at once
   ProfSpanScope span(s, 3);
-  attn_bwd_q_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
+  if ((long long)B * H <= 65535) {
+    RT_TRY(cudaFuncSetAttribute(attn_bwd_q_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairBlockSmemQ));
+    attn_bwd_q_block_kernel<<<dim3(ceil_div(N, kPB), B * H), 256, kPairBlockSmemQ, s>>>(ab);
+  } else {
+    attn_bwd_q_kernel<<<warps_grid((long long)((N + 3) / 4) * B * H), tpb, 0, s>>>(ab);
+  }
   float* gprod = F(L.gprod);
   float* part = F(L.part);
   auto col_sum = [&](const float* a, int width, float* out, bool acc) {
