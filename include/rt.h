@@ -218,7 +218,7 @@ rt_status rt_layer_recompute(const rt_config *cfg, const rt_layer_weights *w, co
  * Batches above 32 sequences run each step of the reverse loop as dense products over the batch (Sec. 6's regime).
  * The reverse loop and the attention terms are fp32 on CUDA cores; with bf16 storage the products over all rows run
  * on the tensor cores (operands rounded to bf16, fp32 accumulation).  recur_block > 1 returns RT_ERR_UNSUPPORTED.
- * The workspace needs rt_backward_workspace_bytes (about 30 fp32 arrays of B*N*d plus 3 of B*N*d_ff). */
+ * The workspace needs rt_backward_workspace_bytes (about 40 fp32 arrays of B*N*d plus 4 of B*N*d_ff: 1.1 GB at B=4, N=2048, d=768; 48 GB at B=N=512, d=1024). */
 typedef struct {
   float *w_q, *w_k, *w_v, *w_o, *w_up, *w_down;   /* shapes of rt_layer_weights */
   float *g_attn, *g_mlp, *g_kv, *g_q, *g_k;       /* [d_model] */
