@@ -1116,8 +1116,32 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
 #else
   auto mark = [](int) {};
 #endif
+  // The rows of the next position that nobody has touched since the sweep (dz, z, h, k_raw, W_up u) would each cost a trip
+  // to HBM in the middle of a step: the last CTA (never the busiest) asks L2 for them one position ahead.
+  auto warm = [&](int pos) {
+    if (blockIdx.x != gridDim.x - 1 || pos < 0) return;
+    const T* zT = reinterpret_cast<const T*>(p.z);
+    for (int b = 0; b < p.B; ++b) {
+      const long long at = ((long long)pos * p.B + b) * p.d;
+      const int lines_d = p.d / 32, lines_f = p.dff / 32;       // 128-byte lines of fp32 rows
+      for (int l = threadIdx.x; l < 3 * lines_d + lines_f + lines_d / 2 + 1; l += kRmThreads) {
+        const void* ptr;
+        if (l < lines_d) ptr = p.dz + (long long)b * p.dz_bs + (long long)pos * p.dz_ts + 32 * l;
+        else if (l < 2 * lines_d) ptr = p.h + at + 32 * (l - lines_d);
+        else if (l < 3 * lines_d) ptr = p.kraw + at + 32 * (l - 2 * lines_d);
+        else if (l < 3 * lines_d + lines_f) ptr = p.act + ((long long)pos * p.B + b) * p.dff + 32 * (l - 3 * lines_d);
+        else {
+          const int off = 64 * (l - 3 * lines_d - lines_f);     // 128-byte lines of the storage-type row of z (at most d entries)
+          ptr = zT + (long long)b * p.z_bs + (long long)pos * p.z_ts + (off < p.d ? off : 0);
+        }
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+      }
+    }
+  };
+  warm(lp.e0 - 1);
   for (int i = lp.e0 - 1; i >= lp.s0; --i) {
     p.i = i;
+    warm(i - 1);
     phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f, lp.cols_pair, 2, 0);
     mark(0);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
