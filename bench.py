@@ -208,8 +208,6 @@ def run_cuda(args):
     leaf_kw = {"leaf": args.leaf} if args.leaf else {}
     if args.recur_block > 1:
         leaf_kw["recur_block"] = args.recur_block
-    if args.leaf_groups:
-        leaf_kw["leaf_groups"] = args.leaf_groups
     stream = torch.cuda.current_stream(dev)
 
     if args.alibi:                                     # the same slopes for every layer
@@ -669,7 +667,6 @@ def main():
     ap.add_argument("--sched", default="tiled", choices=["tiled", "naive"])
     ap.add_argument("--leaf", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
-    ap.add_argument("--leaf-groups", type=int, default=0, help="rt_config.leaf_groups (0 = auto)")
     ap.add_argument("--profile-one-call", action="store_true",
                     help="run one call and exit (used under ncu to count DRAM / L2 bytes of a whole call)")
     ap.add_argument("--tile-bench", action="store_true", help="time Algorithm 2 alone per tile size and exit")

@@ -75,10 +75,6 @@ typedef struct {
                                of all positions in earlier blocks and to the temporary pairs of the positions j <= i of its own
                                block, so a block is computed in one parallel sweep; S >= N is an ordinary pre-LN Transformer
                                layer).  Prefill entry points only, tiled schedule; decode returns RT_ERR_UNSUPPORTED */
-  int32_t leaf_groups;      /* 0 = auto.  1, 2 or 4: the bf16 leaf kernel (B <= 16) splits the batch into this many groups of
-                               sequences and runs them through the per-token chain side by side, so that one group's products
-                               overlap the other groups' exchanges (sequences are independent, Sec. 2.2).  A tuning knob: the
-                               result does not depend on it.  A count the batch cannot fill is lowered */
 } rt_config;
 
 typedef struct {            /* device pointers; read-only */

@@ -33,7 +33,6 @@ bool config_ok(const rt_config* c) {
   if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
   if (c->norm_flags & ~15) return false;
   if (c->recur_block < 0) return false;
-  if (c->leaf_groups != 0 && c->leaf_groups != 1 && c->leaf_groups != 2 && c->leaf_groups != 4) return false;
   return true;
 }
 
@@ -66,10 +65,9 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_z = take((size_t)B * d * 4);
   L.ex_k = take((size_t)B * d * 4);
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
-  // exchange buffers of the tensor-core leaf kernel, per sequence group: c, h, z as flag-carrying words, g as
-  // packed bf16 in fragment order and its completion counters; raw k|v as flag-carrying fp32 words for the batch
-  L.ll_bytes = ((size_t)kLeafMmaMaxGroups * (3 * leaf_mma_words_d((int)d) + leaf_mma_words_g((int)f)) + (size_t)B * 2 * d) * 8 +
-               (size_t)kLeafMmaMaxGroups * kLeafMmaRanges * 128;
+  // exchange buffers of the tensor-core leaf kernel: c, h, z as flag-carrying words (16 sequence slots each),
+  // g as packed bf16 in fragment order (16 sequence slots), raw k|v as flag-carrying fp32 words
+  L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)16 * (f / 4) + (size_t)B * 2 * d) * 8;
   L.ll = take(L.ll_bytes);
   L.hid0 = take(tok * d * e);
   L.hid1 = take(tok * d * e);
@@ -350,22 +348,20 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   // bf16 tiled prefill takes the tensor-core leaf kernel when the shape fits it
   LeafMmaLaunch ml;
   const bool use_mma = c->dtype == RT_BF16 && c->sched == RT_SCHED_TILED && pos0 == 0 &&
-                       leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, c->leaf_groups, &ml);
+                       leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
   LeafMmaBuffers mb;
   {
     unsigned long long* w = (unsigned long long*)(ws + L.ll);
-    mb.grp_words_d = leaf_mma_words_d(c->d_model);
-    mb.grp_words_g = leaf_mma_words_g(c->d_ff);
-    const size_t all_d = (size_t)kLeafMmaMaxGroups * mb.grp_words_d;
-    mb.ll_c = w; mb.ll_h = w + all_d; mb.ll_z = w + 2 * all_d; mb.ll_g = w + 3 * all_d;
-    mb.ll_kv = mb.ll_g + (size_t)kLeafMmaMaxGroups * mb.grp_words_g;
-    mb.g_cnt = (unsigned*)(mb.ll_kv + (size_t)B * 2 * c->d_model);
+    const size_t bd2 = (size_t)16 * (c->d_model / 2);
+    mb.ll_c = w; mb.ll_h = w + bd2; mb.ll_z = w + 2 * bd2; mb.ll_g = w + 3 * bd2;
+    mb.ll_kv = mb.ll_g + (size_t)16 * (c->d_ff / 4);
   }
   auto leaf_mma = [&](int t0, int t1) -> bool {
     lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
     ProfScope ps(s, kProfLeaf);
     if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return false;
     ctx.seq_base += (unsigned)(t1 - t0);
+    ctx.bar_base += (unsigned)(t1 - t0) * (unsigned)ml.grid;      // one grid barrier per token step
     return true;
   };
 

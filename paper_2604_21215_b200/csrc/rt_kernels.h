@@ -48,21 +48,9 @@ inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsign
 cudaError_t wait_expiry_selftest_launch(SyncArea* sync, cudaStream_t s);
 
 // bf16 / tiled-schedule leaf kernel (tensor-core mat-vecs, flag-carrying exchange words).
-// The batch is split into `groups` independent groups of sequences that run through the chain side by side.
-constexpr int kLeafMmaMaxGroups = 4;
-constexpr int kLeafMmaRanges = 8;              // completion counters per group for the MLP's hidden vector
-struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; int groups, warps_per_group; };
-// Exchange buffers, all zeroed at the start of an API call.  c, h, z: per group `grp_words_d` flag-carrying 64-bit
-// words; g: per group `grp_words_g` words of packed bf16; raw k|v: [B, 2d] flag-carrying fp32 words for the whole
-// batch; g_cnt: per group kLeafMmaRanges counters, one 128-byte line each.
-struct LeafMmaBuffers {
-  unsigned long long *ll_c, *ll_h, *ll_z, *ll_g, *ll_kv;
-  unsigned* g_cnt;
-  size_t grp_words_d, grp_words_g;
-};
-size_t leaf_mma_words_d(int d);
-size_t leaf_mma_words_g(int dff);
-bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, int want_groups, LeafMmaLaunch* out);
+struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
+struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [16,d/2] words x3, packed bf16 [B,dff], [B,2d] words
+bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out);
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s);
 
 // Pre-pass (Algorithm 1, line 1 and the temporary pair of line 7, hoisted out of the loop).

@@ -9,15 +9,10 @@
 //     A consumer polls the payload words themselves: one L2 round trip per exchange, no
 //     separate fence + counter + reload.  Flags are unique per step of an API call and the
 //     buffers are zeroed at the start of the call.
-//   * the mat-vec products run on the tensor cores as m16n8k16 MMAs with the sequences as
-//     the M dimension (rows without a sequence are zero) and 8 weight rows as the N dimension,
-//     K split over the MMA warps of a group and reduced through shared memory.  The fragments
-//     of the activations are exactly the polled words; weight fragments are 8-byte shared loads.
-//   * sequences are independent (Sec. 2.2 states the layer per sequence), and a token step is
-//     bound by the latency of its exchanges, not by throughput.  The batch is therefore split
-//     into NG groups of sequences, each with its own MMA warps, exchange buffers, flags and
-//     counters, all reading the same weights in shared memory: while one group's words are in
-//     flight the other groups' products run.
+//   * the mat-vec products run on the tensor cores as m16n8k16 MMAs with the B sequences as
+//     the M dimension (rows >= B are zero) and 8 weight rows as the N dimension, K split over
+//     the 8 MMA warps of the CTA and reduced through shared memory.  The fragments of the
+//     activations are exactly the polled words; weight fragments are 8-byte shared loads.
 //   * two extra warps per CTA do the in-leaf attention (Algorithm 2 with one key at a time):
 //     each owns one (sequence, head) pair and keeps the running stats (m, l, o) of every query
 //     of the leaf in shared memory.  When the pair (k_j, v_j) arrives it first finishes query
@@ -32,10 +27,11 @@
 
 namespace rt {
 
+constexpr int kMmaWarps = 8;
+constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kAttnSlots = 2;
+constexpr int kLeafMmaThreads = kMmaThreads + 32 * kAttnSlots;
 constexpr int kNT = 4;                  // n-tiles (8 weight rows each) per pass
-constexpr int kSlots = 8;               // sequence slots of a group: the MMA rows that carry data
-constexpr int kRanges = kLeafMmaRanges; // completion counters of a group's g vector (ranges of d_ff)
 constexpr int kQStride = kHeadDim + 2;  // bf16 elements per query row in shared memory
 constexpr int kOStride = kHeadDim + 1;  // floats per o row in shared memory
 
@@ -43,27 +39,20 @@ struct LeafMmaLayout {
   int max_nd, max_nf;          // weight rows per CTA (upper bounds): d-row matrices, W_up
   int stride_d, stride_f;      // shared-memory row strides in elements (K + 16)
   int lf;                      // leaf capacity of the attention state
-  int ng, wg;                  // sequence groups, MMA warps per group
-  size_t off_grp, grp_bytes;   // per-group scratch: abort word, red[2], ssq[2], own rows of h
-  size_t g_red, g_ssq, g_hown; // offsets inside a group's scratch
-  size_t off_wo, off_wup, off_wdn, off_wk, off_wv, off_attn, attn_bytes, total;
+  size_t off_wo, off_wup, off_wdn, off_wk, off_wv, off_red, off_ssq, off_hown, off_attn, attn_bytes, total;
 };
 
-LeafMmaLayout leaf_mma_layout(int d, int dff, int grid, int lf, int slots, int ng, int wg) {
+LeafMmaLayout leaf_mma_layout(int d, int dff, int grid, int lf, int slots) {
   LeafMmaLayout L;
   L.max_nd = 2 * ceil_div(d / 2, grid);
   L.max_nf = 2 * ceil_div(dff / 2, grid);
   L.stride_d = d + 16;
   L.stride_f = dff + 16;
   L.lf = lf;
-  L.ng = ng; L.wg = wg;
-  size_t g = 16;                                              // the group's two abort words (used alternately)
-  L.g_red = g;   g += 2 * sizeof(float2) * wg * kNT * 32;     // two buffers, used alternately
-  L.g_ssq = g;   g += 2 * sizeof(float) * wg * kSlots;
-  L.g_hown = g;  g += align_up(sizeof(float) * kSlots * (size_t)L.max_nd, 16);
-  L.grp_bytes = align_up(g, 16);
-  size_t o = 0;
-  L.off_grp = o;   o += L.grp_bytes * ng;
+  size_t o = 64;                                             // abort flag
+  L.off_red = o;   o += sizeof(float4) * kMmaWarps * kNT * 32;
+  L.off_ssq = o;   o += sizeof(float) * kMmaWarps * 16;
+  L.off_hown = o;  o += align_up(sizeof(float) * 16 * (size_t)L.max_nd, 16);
   L.attn_bytes = align_up((size_t)lf * kQStride * 2 + (size_t)lf * kOStride * 4 + (size_t)lf * 8 + 2 * kHeadDim * 4, 16);
   L.off_attn = o;  o += L.attn_bytes * slots;
   o = align_up(o, 128);
@@ -116,19 +105,18 @@ __device__ __forceinline__ void st_relaxed_v4(void* p, unsigned a, unsigned b, u
   const unsigned long long w0 = ((unsigned long long)b << 32) | a, w1 = ((unsigned long long)d << 32) | c;
   asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1,%2};" ::"l"(p), "l"(w0), "l"(w1) : "memory");
 }
-// m16n8k16 with rows 8..15 of A all zero: the sequences of a group fill rows 0..7 only, so c[2] and c[3]
-// (rows 8..15 of the result) stay zero and only c[0], c[1] are used.
-__device__ __forceinline__ void mma_bf16_top(float (&c)[4], unsigned a0, unsigned a2, unsigned b0, unsigned b1) {
-  const unsigned zero = 0u;
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// Barrier over the MMA warps of one group (named barrier 1 + group).
-template <int WG>
-__device__ __forceinline__ void group_sync(int grp) {
-  asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(WG * 32) : "memory");
-}
+#ifdef RT_TIMELINE
+__device__ unsigned long long g_dbg[3 * 8 * 4 * 8];      // [cta slot][warp][phase][point]
+#define TL(pt) if (tl_on) g_dbg[((tl_slot * 8 + warp) * 4 + ph) * 8 + (pt)] = globaltimer_ns()
+#else
+#define TL(pt)
+#endif
+__device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory"); }
 
 // A wait that ran out: record it for the host and tell every other waiter to leave.
 __device__ __noinline__ void report_timeout(SyncArea* s) {
@@ -145,41 +133,56 @@ __device__ __forceinline__ bool wait_expired(SyncArea* s, unsigned long long& t_
   return false;
 }
 
-// Exchange words of a group's [sequences, K] bf16 vector are stored in the order the MMA fragments
-// are read: [k-step of 16][8 sequence slots][4 groups of 4 k][2 words of 2 k], so that one warp-wide
-// 16-byte load (8 sequences x 4 groups) covers 512 contiguous bytes.  Index of the word that holds
-// elements k, k+1 (k even) of the group's sequence b:
+// What one mat-vec phase works on.  Tiles are groups of 8 weight rows in shared memory.
+// Exchange words of a [B, K] bf16 vector are stored in the order the MMA fragments are read:
+// [k-step of 16][16 sequence slots][4 groups of 4 k][2 words of 2 k], so that one warp-wide
+// 16-byte load (8 sequences x 4 groups) covers 512 contiguous bytes.  Index of the word that
+// holds elements k, k+1 (k even) of sequence b:
 __device__ __forceinline__ size_t ll_word(int b, int k) {
-  return ((size_t)((k >> 4) * kSlots + b) * 4 + ((k & 15) >> 2)) * 2 + ((k & 3) >> 1);
+  return ((size_t)((k >> 4) * 16 + b) * 4 + ((k & 15) >> 2)) * 2 + ((k & 3) >> 1);
 }
-constexpr int kWordsPerKStep = kSlots * 8;      // 64-bit words of one k-step
-// g as packed bf16 in the order the fragments are read: [k-step of 16][8 sequence slots][16 k], so
-// the 8 sequences x 32 bytes one warp-wide load touches are 256 contiguous bytes
-__device__ __forceinline__ size_t g_index(int b, int k) { return ((size_t)((k >> 4) * kSlots + b) << 4) + (size_t)(k & 15); }
-constexpr int kGElemsPerKStep = kSlots * 16;
 
 // Sum of squares (of the raw values) and optional gain for one k-step of fragments; gp points
 // at this thread's 4 gains of the k-step (or is null).
-__device__ __forceinline__ void frag_ssq_gain(unsigned& a0, unsigned& a2, const __nv_bfloat16* gp, float& sq) {
-  const float v0 = bf_lo(a0), v1 = bf_hi(a0), v2 = bf_lo(a2), v3 = bf_hi(a2);
-  sq += v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+template <int MB>
+__device__ __forceinline__ void frag_ssq_gain(unsigned (&a)[4], const __nv_bfloat16* gp, float& sq0, float& sq1) {
+  float gn[4] = {1.f, 1.f, 1.f, 1.f};
   if (gp) {
     const uint2 gw = *reinterpret_cast<const uint2*>(gp);
-    a0 = pack_bf2(v0 * bf_lo(gw.x), v1 * bf_hi(gw.x));
-    a2 = pack_bf2(v2 * bf_lo(gw.y), v3 * bf_hi(gw.y));
+    gn[0] = bf_lo(gw.x); gn[1] = bf_hi(gw.x); gn[2] = bf_lo(gw.y); gn[3] = bf_hi(gw.y);
   }
+#pragma unroll
+  for (int r = 0; r < MB; ++r) {
+    const float v0 = bf_lo(a[r]), v1 = bf_hi(a[r]), v2 = bf_lo(a[2 + r]), v3 = bf_hi(a[2 + r]);
+    const float s = v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+    if (r == 0) sq0 += s; else sq1 += s;
+    if (gp) { a[r] = pack_bf2(v0 * gn[0], v1 * gn[1]); a[2 + r] = pack_bf2(v2 * gn[2], v3 * gn[3]); }
+  }
+}
+
+// Barrier over all CTAs, run by the MMA warps only (the attention warps never wait on it).
+__device__ __forceinline__ bool mma_grid_barrier(SyncArea* sync, volatile int* s_abort, unsigned target) {
+  mma_warps_sync();
+  if (threadIdx.x == 0) {
+    // the release is cumulative over what the CTA barrier above ordered before it: no separate fence
+    red_release_add_u32(&sync->bar_count, 1u);
+    unsigned spins = 0;
+    unsigned long long t_start = 0;
+    while (ld_acquire_u32(&sync->bar_count) < target) {
+      if ((++spins & 255u) == 0u && wait_expired(sync, t_start)) { *s_abort = 1; break; }
+    }
+  }
+  mma_warps_sync();
+  return *s_abort == 0;
 }
 
 // ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
 template <bool TIMERS>
 __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsigned char* smem_slot, int pair,
-                               const unsigned long long* ll_kv, unsigned long long* ll_c_all, size_t grp_words_d) {
+                               const unsigned long long* ll_kv, unsigned long long* ll_c) {
   const int lane = threadIdx.x & 31;
   const int B = p.B, d = p.d, H = p.H;
   const int b = pair / H, h = pair % H;
-  const int Bg = (B + L.ng - 1) / L.ng;
-  const int grp = b / Bg, bl = b - grp * Bg;                    // the sequence's group and its slot there
-  unsigned long long* ll_c = ll_c_all + (size_t)grp * grp_words_d;
   const int n = p.t1 - p.t0;
   __nv_bfloat16* qs = reinterpret_cast<__nv_bfloat16*>(smem_slot);
   float* os = reinterpret_cast<float*>(smem_slot + (size_t)L.lf * kQStride * 2);
@@ -210,7 +213,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   __syncwarp();
   const float gk0 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane) : 1.0f;
   const float gk1 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane + 1) : 1.0f;
-  unsigned long long* c_word = ll_c + ll_word(bl, h * kHeadDim + 2 * lane);
+  unsigned long long* c_word = ll_c + ll_word(b, h * kHeadDim + 2 * lane);
   // c of the first position: nothing of this leaf to fold in
   {
     const float il = 1.0f / ls[0];
@@ -289,20 +292,18 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   if (timing) { atomicAdd(&p.sync->phase_ns[0], a_work); atomicAdd(&p.sync->phase_ns[1], a_wait); }
 }
 
-// NG groups of WG MMA warps.  TIMERS and GAINS are compile-time: the token step is a latency chain of code that runs
-// once per token, and every instruction and live register that is compiled in costs time even when its branch is not
-// taken.
-template <int NG, int WG, bool TIMERS, bool GAINS>
-__global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
-                                                                                  const LeafMmaBuffers buf) {
+// TIMERS and GAINS are compile-time: the token step is a latency chain of code that runs once per token, and every
+// instruction and live register that is compiled in costs time even when its branch is not taken.
+template <int MB, bool TIMERS, bool GAINS>
+__global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
+                                                                      unsigned long long* ll_c, unsigned long long* ll_h,
+                                                                      unsigned long long* ll_g, unsigned long long* ll_z,
+                                                                      unsigned long long* ll_kv) {
   extern __shared__ __align__(128) unsigned char smem[];
-  constexpr int kThreads = (NG * WG + kAttnSlots) * 32;
-  // k-steps per round of polled loads / of loads of g (W_down): as many as the registers of the launch shape
-  // hold (the register file is dealt out per 4 warps: up to 12 warps leave a thread 168 registers, 20 leave 96)
-  constexpr int KC = NG * WG > 8 ? 8 : (WG >= 8 ? 8 : 16);
-  constexpr int KD = NG * WG > 8 ? 16 : 32;
-  constexpr int RPW = kRanges / WG;                              // completion counters a warp waits for
-  static_assert(kRanges % WG == 0 && RPW >= 1, "ranges of g are dealt out evenly to the warps of a group");
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem);
+  float4* red = reinterpret_cast<float4*>(smem + L.off_red);
+  float* ssq_red = reinterpret_cast<float*>(smem + L.off_ssq);
+  float* hown = reinterpret_cast<float*>(smem + L.off_hown);
   __nv_bfloat16* s_wo = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wo);
   __nv_bfloat16* s_wup = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wup);
   __nv_bfloat16* s_wdn = reinterpret_cast<__nv_bfloat16*>(smem + L.off_wdn);
@@ -311,19 +312,19 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int B = p.B, d = p.d, dff = p.dff;
+  const int B = p.B, d = p.d, H = p.H, dff = p.dff;
   if (*reinterpret_cast<volatile unsigned*>(&p.sync->abort_flag)) return;
   // rows are dealt out in pairs so that a published word (two consecutive rows) has one owner
   const int d_lo = 2 * (int)((long long)(d / 2) * cta / G), d_hi = 2 * (int)((long long)(d / 2) * (cta + 1) / G);
   const int f_lo = 2 * (int)((long long)(dff / 2) * cta / G), f_hi = 2 * (int)((long long)(dff / 2) * (cta + 1) / G);
   const int nd = d_hi - d_lo, nf = f_hi - f_lo;
 
-  if (tid < 2 * NG) reinterpret_cast<volatile int*>(smem + L.off_grp + (size_t)(tid >> 1) * L.grp_bytes)[tid & 1] = 0;
+  if (tid == 0) *s_abort = 0;
   {
     auto stage = [&](__nv_bfloat16* dst, int dst_stride, const void* src_base, int row_lo, int nrows, int K) {
       const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(src_base) + (size_t)row_lo * K);
       const int per_row = K / 8;
-      for (int i = tid; i < nrows * per_row; i += kThreads) {
+      for (int i = tid; i < nrows * per_row; i += kLeafMmaThreads) {
         const int r = i / per_row, v = i % per_row;
         *reinterpret_cast<uint4*>(dst + (size_t)r * dst_stride + v * 8) = src[(size_t)r * per_row + v];
       }
@@ -336,11 +337,10 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
   }
   __syncthreads();
 
-  if (warp >= NG * WG) {
-    const int slot = warp - NG * WG;
+  if (warp >= kMmaWarps) {
+    const int slot = warp - kMmaWarps;
     const int pair = cta + slot * G;
-    if (pair < B * p.H)
-      attention_role<TIMERS>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, buf.ll_kv, buf.ll_c, buf.grp_words_d);
+    if (pair < B * H) attention_role<TIMERS>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
     return;
   }
 
@@ -349,61 +349,32 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
   // over the phase index): the step executes once per token, so four straight-line copies would
   // only thrash the instruction cache, and calls through a real function would put the fragments
   // and accumulators on the stack, where every access is an L2 round trip.
-  const int grp = NG > 1 ? warp / WG : 0, lw = NG > 1 ? warp % WG : warp;
-  const int Bg = (B + NG - 1) / NG;
-  const int b_lo = grp * Bg;
-  const int nb = B - b_lo < Bg ? B - b_lo : Bg;                  // sequences of this group
-  if (nb <= 0) return;                                           // (the launcher never makes an empty group)
-  unsigned char* gs = smem + L.off_grp + (size_t)grp * L.grp_bytes;
-  // A warp whose wait ran out sets the abort word of the pass it is in; every warp of the group reads that word
-  // right after the pass's barrier, so all of them leave at the same barrier (two words, alternating like the
-  // reduction buffers: a warp already in the next pass cannot disturb a slower warp's read of this one)
-  volatile int* s_abort = reinterpret_cast<volatile int*>(gs);
-  float2* red = reinterpret_cast<float2*>(gs + L.g_red);
-  float* ssq_red = reinterpret_cast<float*>(gs + L.g_ssq);
-  float* hown = reinterpret_cast<float*>(gs + L.g_hown);
-  unsigned long long* ll_c = buf.ll_c + (size_t)grp * buf.grp_words_d;
-  unsigned long long* ll_h = buf.ll_h + (size_t)grp * buf.grp_words_d;
-  unsigned long long* ll_z = buf.ll_z + (size_t)grp * buf.grp_words_d;
-  __nv_bfloat16* g_pk = reinterpret_cast<__nv_bfloat16*>(buf.ll_g + (size_t)grp * buf.grp_words_g);
-  unsigned* g_cnt = buf.g_cnt + (size_t)grp * kRanges * 32;      // one 128-byte line per counter
-  unsigned long long* ll_kv = buf.ll_kv;
-
+  constexpr int KC = 8;                                          // k-steps per round of loads
   const int g = lane >> 2, c = lane & 3;
   const bool pre = (p.norm_flags & RT_NORM_PRE) != 0;
   const bool kv_norm = pre && !(p.norm_flags & RT_NORM_SKIP_Z);
   const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(p.x);
   __nv_bfloat16* z = reinterpret_cast<__nv_bfloat16*>(p.z);
+  // g as packed bf16 in the order the fragments are read: [k-step of 16][16 sequence slots][16 k], so the
+  // 8 sequences x 32 bytes one warp-wide load touches are 256 contiguous bytes (2 lines instead of 8)
+  __nv_bfloat16* g_pk = reinterpret_cast<__nv_bfloat16*>(ll_g);
+  auto g_index = [](int b, int k) -> size_t { return ((size_t)((k >> 4) * 16 + b) << 4) + (size_t)(k & 15); };
   const float inv_d = 1.0f / (float)d;
   const int nt_d = (nd + 7) / 8, nt_f = (nf + 7) / 8;
-  const bool has0 = g < nb;
-  const int bq = b_lo + (has0 ? g : 0);                          // this lane's sequence in the batch
-  const int g0 = has0 ? g : 0;                                   // slot read by lanes without a sequence (masked)
-  const unsigned keep0 = has0 ? 0xffffffffu : 0u;
+  const bool has0 = g < B, has1 = (MB == 2) && (g + 8 < B);
+  unsigned bar_target = p.bar_base;
   const bool timing = TIMERS && (cta == 0 && tid == 0);
   unsigned long long t_ph = timing ? globaltimer_ns() : 0ull;
 
-  // Completion counters of g: the k-steps of d_ff are cut into kRanges ranges, warp lw multiplies the RPW ranges
-  // [lw * RPW, (lw + 1) * RPW).  A producer CTA bumps the counter of every range its rows of W_up fall in once per
-  // token step, so a consumer warp waits for the few CTAs that write its part of g, not for the whole grid.
-  const int n_ks_f = dff / 16;
-  const int ks_per_range = (n_ks_f + kRanges - 1) / kRanges;
-  const int my_r_lo = nf > 0 ? (f_lo / 16) / ks_per_range : 0;   // ranges this CTA produces for
-  const int my_r_hi = nf > 0 ? ((f_hi - 1) / 16) / ks_per_range : -1;
-  unsigned cnt_per_step = 0;                                     // lane i < RPW: arrivals per step at range lw*RPW + i
-  if (lane < RPW) {
-    const int r = lw * RPW + lane;
-    for (int cc = 0; cc < G; ++cc) {
-      const int lo = 2 * (int)((long long)(dff / 2) * cc / G), hi = 2 * (int)((long long)(dff / 2) * (cc + 1) / G);
-      if (hi > lo && (lo / 16) / ks_per_range <= r && ((hi - 1) / 16) / ks_per_range >= r) ++cnt_per_step;
-    }
-  }
-  unsigned pass = 0;                                             // passes so far: selects the reduction buffer
-
   for (int t = p.t0; t < p.t1; ++t) {
     const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
+#ifdef RT_TIMELINE
+    const int tl_slot = cta == 0 ? 0 : (cta == 77 ? 1 : 2);
+    const bool tl_on = (cta == 0 || cta == 77 || cta == 147) && lane == 0 && t == p.t0 + 20 && p.t0 == 1024;
+#endif
 #pragma unroll 1
     for (int ph = 0; ph < 4; ++ph) {                              // 0: W_o   1: W_up   2: W_down   3: W_k | W_v
+      TL(0);
       // ---- what this phase multiplies ----
       const int K = (ph == 2) ? dff : d;
       const int stride = (ph == 2) ? L.stride_f : L.stride_d;
@@ -417,32 +388,21 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
       if (ph == 3 && kv_norm) { if (GAINS) gain = reinterpret_cast<const __nv_bfloat16*>(p.g_kv); want_ssq = true; }
       const __nv_bfloat16* gp = (GAINS && gain) ? gain + 4 * c : nullptr;
       unsigned long long wait_ns = 0;
-      bool alive = true;
-      const int n_ks = K / 16;
-      const int ks_per_warp = (ph == 2) ? ks_per_range * RPW : (n_ks + WG - 1) / WG;
-      const int ks0 = lw * ks_per_warp < n_ks ? lw * ks_per_warp : n_ks;
-      const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
       if (ph == 2) {
-        // this warp's part of g (packed bf16, written by a few CTAs) must be complete before it multiplies by W_down
+        // every CTA's slice of g (packed bf16) must be complete before anyone multiplies by W_down
+        bar_target += (unsigned)G;
         const unsigned long long tb = timing ? globaltimer_ns() : 0ull;
-        const unsigned target = seq * cnt_per_step;
-        unsigned spins = 0;
-        unsigned long long t_start = 0;
-        while (true) {
-          bool ok = true;
-          if (lane < RPW) ok = ld_acquire_u32(g_cnt + (size_t)(lw * RPW + lane) * 32) >= target;
-          if (__all_sync(0xffffffffu, ok)) break;
-          if ((++spins & 63u) == 0u) {
-            int bad = 0;
-            if (lane == 0) bad = wait_expired(p.sync, t_start) ? 1 : 0;
-            if (__shfl_sync(0xffffffffu, bad, 0)) { s_abort[pass & 1u] = 1; alive = false; break; }
-          }
-        }
+        if (!mma_grid_barrier(p.sync, s_abort, bar_target)) return;
         if (timing) wait_ns += globaltimer_ns() - tb;
       }
+      TL(1);
+      const int n_ks = K / 16;
+      const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
+      const int ks0 = warp * ks_per_warp;
+      const int ks1 = ks0 + ks_per_warp < n_ks ? ks0 + ks_per_warp : n_ks;
 
       const int tile_step = (ph == 2) ? 1 : kNT;                   // W_down: one tile per pass (see below)
-      for (int t0n = 0; t0n < nt_all; t0n += tile_step, ++pass) {
+      for (int t0n = 0; t0n < nt_all; t0n += tile_step) {
         const int n_tiles = nt_all - t0n < tile_step ? nt_all - t0n : tile_step;
         // this thread's 8 bytes of weight row g (clamped to the rows that exist) of each tile, at k = 4c
         const unsigned char* wp[kNT];
@@ -457,13 +417,15 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
           wp[i] = reinterpret_cast<const unsigned char*>(wbase + (size_t)r * stride + 4 * c);
         }
         // rows this thread finishes after the reduction (warp w finishes tile t0n + w)
-        const int ti_e = t0n + lw;
+        const int ti_e = t0n + warp;
         const bool second_e = (ph == 3) && ti_e >= nt_d;
         const int rl = (second_e ? ti_e - nt_d : ti_e) * 8 + 2 * c;
-        const bool mine = lw < n_tiles && rl < nrows && has0;
-        unsigned xw0 = 0;
-        if (ph == 0 && mine)                                       // x_t for the residual, fetched before the wait
-          xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)bq * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+        const bool mine = warp < n_tiles && rl < nrows;
+        unsigned xw0 = 0, xw1 = 0;
+        if (ph == 0 && mine) {                                     // x_t for the residual, fetched before the wait
+          if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+          if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+        }
 
         // The loops below are written without branches around the loads and the products (indices
         // are clamped, missing sequences and k-steps contribute zeros): a branch per product costs
@@ -471,40 +433,59 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
         float acc[kNT][4];
 #pragma unroll
         for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-        float sq0 = 0.f;
+        float sq0 = 0.f, sq1 = 0.f;
+        bool alive = true;
+        const int g0 = has0 ? g : 0, g1 = has1 ? g + 8 : 0;        // rows read by lanes without a sequence (masked below)
+        const unsigned keep0 = has0 ? 0xffffffffu : 0u, keep1 = has1 ? 0xffffffffu : 0u;
         if (ph == 2) {
-          // W_down reads g as packed bf16 behind its completion counters: plain loads, and a whole round of this
-          // warp's k-steps is in flight before the first product.  One tile per pass; the four accumulators cut
-          // the dependent chain of products.
-          const __nv_bfloat16* b0p = g_pk + g_index(g0, 4 * c);          // + kGElemsPerKStep elements per k-step
+          // W_down reads g as packed bf16 after the barrier: plain loads, and ALL of this warp's
+          // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
+          // pass keeps this at 32 products; the two accumulators halve the dependent chain.
+          constexpr int KD = 32 / MB;
+          const __nv_bfloat16* b0p = g_pk + g_index(g0, 4 * c);          // + 256 elements per k-step
+          const __nv_bfloat16* b1p = g_pk + g_index(g1, 4 * c);
           for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
+            unsigned ad[KD][4];
             const int n_here = ks1 - kc0;
-            uint2 w0[KD];
+            uint2 w0[KD], w1[MB == 2 ? KD : 1];
 #pragma unroll
-            for (int i = 0; i < KD; ++i)
-              w0[i] = ld_cg_v2_if(b0p + (size_t)(kc0 + (i < n_here ? i : 0)) * kGElemsPerKStep, (i < n_here ? 1u : 0u) & keep0);
+            for (int i = 0; i < KD; ++i) w0[i] = ld_cg_v2_if(b0p + (size_t)(kc0 + (i < n_here ? i : 0)) * 256, (i < n_here ? 1u : 0u) & keep0);
+            if (MB == 2) {
+#pragma unroll
+              for (int i = 0; i < KD; ++i) w1[i] = ld_cg_v2_if(b1p + (size_t)(kc0 + (i < n_here ? i : 0)) * 256, (i < n_here ? 1u : 0u) & keep1);
+            }
+#pragma unroll
+            for (int i = 0; i < KD; ++i) {
+              ad[i][0] = w0[i].x; ad[i][2] = w0[i].y;
+              if (MB == 2) { ad[i][1] = w1[i].x; ad[i][3] = w1[i].y; } else { ad[i][1] = 0u; ad[i][3] = 0u; }
+            }
+            TL(2);
             const unsigned char* wd = wp[0] + (size_t)kc0 * 32;
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
               const uint2 bw = *reinterpret_cast<const uint2*>(wd + (i < n_here ? i : 0) * 32);
-              mma_bf16_top(acc[i & 3], w0[i].x, w0[i].y, bw.x, bw.y);
+              mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
+#ifdef RT_TIMELINE
+              if (i == 1 && tl_on && acc[0][0] != 123.f) TL(7);
+#endif
             }
           }
-          acc[0][0] += acc[1][0] + acc[2][0] + acc[3][0];
-          acc[0][1] += acc[1][1] + acc[2][1] + acc[3][1];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { acc[0][j] += acc[1][j]; acc[1][j] = 0.f; }
         } else
         for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
-          unsigned a0[KC], a2[KC];
+          unsigned a[KC][4];
 #pragma unroll
-          for (int i = 0; i < KC; ++i) { a0[i] = a2[i] = 0u; }
+          for (int i = 0; i < KC; ++i) { a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0u; }
           const int n_here = ks1 - kc0;                             // k-steps of this round (the rest stay zero)
           {
             // flag-carrying words: a k-step is 8 words per sequence, this thread takes the 2 adjacent ones at 4c
-            const unsigned long long* base0 = act_ll + ll_word(g0, 4 * c) + (size_t)kc0 * kWordsPerKStep;
-            unsigned need0 = 0;
+            const unsigned long long* base0 = act_ll + ll_word(g0, 4 * c) + (size_t)kc0 * 128;   // + 128 words per k-step
+            const unsigned long long* base1 = act_ll + ll_word(g1, 4 * c) + (size_t)kc0 * 128;
+            unsigned need0 = 0, need1 = 0;
 #pragma unroll
             for (int i = 0; i < KC; ++i) {
-              if (i < n_here) need0 |= (1u << i) & keep0;
+              if (i < n_here) { need0 |= (1u << i) & keep0; need1 |= (1u << i) & keep1; }
             }
             unsigned spins = 0;
             unsigned long long t_start = 0;
@@ -512,29 +493,43 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
             while (alive) {
               // every outstanding word of the round is loaded (under a predicate, not a branch) before
               // any flag is looked at, so the loads overlap
-              uint4 w0[KC];
+              uint4 w0[KC], w1[MB == 2 ? KC : 1];
 #pragma unroll
-              for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4_if(base0 + (size_t)(i < n_here ? i : 0) * kWordsPerKStep, (need0 >> i) & 1u);
+              for (int i = 0; i < KC; ++i) w0[i] = ld_relaxed_v4_if(base0 + (size_t)(i < n_here ? i : 0) * 128, (need0 >> i) & 1u);
+              if (MB == 2) {
+#pragma unroll
+                for (int i = 0; i < KC; ++i) w1[i] = ld_relaxed_v4_if(base1 + (size_t)(i < n_here ? i : 0) * 128, (need1 >> i) & 1u);
+              }
 #pragma unroll
               for (int i = 0; i < KC; ++i) {
                 const bool okw = (w0[i].y == seq) & (w0[i].w == seq) & ((need0 >> i) & 1u);
-                a0[i] = okw ? w0[i].x : a0[i];
-                a2[i] = okw ? w0[i].z : a2[i];
+                a[i][0] = okw ? w0[i].x : a[i][0];
+                a[i][2] = okw ? w0[i].z : a[i][2];
                 need0 &= okw ? ~(1u << i) : 0xffffffffu;
               }
-              if (__all_sync(0xffffffffu, need0 == 0u)) break;
+              if (MB == 2) {
+#pragma unroll
+                for (int i = 0; i < KC; ++i) {
+                  const bool okw = (w1[i].y == seq) & (w1[i].w == seq) & ((need1 >> i) & 1u);
+                  a[i][1] = okw ? w1[i].x : a[i][1];
+                  a[i][3] = okw ? w1[i].z : a[i][3];
+                  need1 &= okw ? ~(1u << i) : 0xffffffffu;
+                }
+              }
+              if (__all_sync(0xffffffffu, (need0 | need1) == 0u)) break;
               if ((++spins & 63u) == 0u) {
                 int bad = 0;
                 if (lane == 0) bad = wait_expired(p.sync, t_start) ? 1 : 0;
-                if (__shfl_sync(0xffffffffu, bad, 0)) { s_abort[pass & 1u] = 1; alive = false; }
+                if (__shfl_sync(0xffffffffu, bad, 0)) { *s_abort = 1; alive = false; }
               }
             }
             if (timing) wait_ns += globaltimer_ns() - t_poll;
+            TL(2);
           }
           const __nv_bfloat16* gc = (GAINS && gp) ? gp + (size_t)kc0 * 16 : nullptr;
           if (want_ssq) {
 #pragma unroll
-            for (int i = 0; i < KC; ++i) frag_ssq_gain(a0[i], a2[i], (GAINS && gc) ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0);
+            for (int i = 0; i < KC; ++i) frag_ssq_gain<MB>(a[i], (GAINS && gc) ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0, sq1);
           }
           // products, specialised on the number of tiles so that none sits behind a branch
           auto products = [&](auto ntc) {
@@ -545,7 +540,7 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
 #pragma unroll
               for (int nt = 0; nt < NTC; ++nt) {
                 const uint2 bw = *reinterpret_cast<const uint2*>(wp[nt] + off);
-                mma_bf16_top(acc[nt], a0[i], a2[i], bw.x, bw.y);
+                mma_bf16(acc[nt], a[i], bw.x, bw.y);
               }
             }
           };
@@ -556,59 +551,80 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
             default: products(std::integral_constant<int, 4>{}); break;
           }
         }
-        // ---- reduce the K split over the group's warps; warp w then holds the sums of tile t0n + w.  The buffers
-        // alternate between passes, so one barrier per pass is enough: a warp can only write a buffer again after
-        // it has passed the next pass's barrier, which every warp reaches after its reads of this pass ----
-        if (!alive) s_abort[pass & 1u] = 1;
-        float2* redb = red + (size_t)(pass & 1u) * (WG * kNT * 32);
-        float* ssqb = ssq_red + (size_t)(pass & 1u) * (WG * kSlots);
+        TL(3);
+        // ---- reduce the K split over the 8 warps; warp w then holds the sums of tile t0n + w ----
 #pragma unroll
         for (int nt = 0; nt < kNT; ++nt)
-          if (nt < n_tiles) redb[(lw * kNT + nt) * 32 + lane] = make_float2(acc[nt][0], acc[nt][1]);
+          if (nt < n_tiles) red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
         if (want_ssq) {
           sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
-          if (c == 0) ssqb[lw * kSlots + g] = sq0;
+          sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
+          if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
         }
-        group_sync<WG>(grp);
-        if (s_abort[pass & 1u]) return;
-        // ---- epilogue: y0, y1 = rows rl, rl+1 of the tile this warp finishes, for the sequence of slot g ----
-        if (lw < n_tiles) {
-          float y0 = 0.f, y1 = 0.f, ssq = 0.f;
+        mma_warps_sync();
+        TL(4);
+        if (*s_abort) return;
+        float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f, ssq_lo = 0.f, ssq_hi = 0.f;
+        if (warp < n_tiles) {
 #pragma unroll
-          for (int w = 0; w < WG; ++w) {
-            const float2 v = redb[(w * kNT + lw) * 32 + lane];
-            y0 += v.x; y1 += v.y;
+          for (int w = 0; w < kMmaWarps; ++w) {
+            const float4 v = red[(w * kNT + warp) * 32 + lane];
+            y0 += v.x; y1 += v.y; y2 += v.z; y3 += v.w;
           }
           if (want_ssq) {
 #pragma unroll
-            for (int w = 0; w < WG; ++w) ssq += ssqb[w * kSlots + g];
+            for (int w = 0; w < kMmaWarps; ++w) { ssq_lo += ssq_red[w * 16 + g]; ssq_hi += ssq_red[w * 16 + 8 + g]; }
           }
-          if (mine) {
-            if (ph == 0) {                                            // h = x_t + alpha W_o c_t
+        }
+        mma_warps_sync();       // red / ssq_red may be overwritten from here on
+        TL(5);
+        // ---- epilogue: y0, y1 = rows rl, rl+1 for sequence g; y2, y3 = the same rows for sequence g+8 ----
+        if (mine) {
+          if (ph == 0) {                                            // h = x_t + alpha W_o c_t
+            if (has0) {
               const float h0 = bf_lo(xw0) + p.alpha * y0, h1 = bf_hi(xw0) + p.alpha * y1;
               hown[g * L.max_nd + rl] = h0; hown[g * L.max_nd + rl + 1] = h1;
               st_relaxed_u64(ll_h + ll_word(g, d_lo + rl), pack_bf2(h0, h1), seq);
-            } else if (ph == 1) {                                     // g = GELU(W_up RMS(h)), packed bf16
-              const float rs = pre ? rsqrtf(ssq * inv_d + p.eps) : 1.0f;
+            }
+            if (has1) {
+              const float h0 = bf_lo(xw1) + p.alpha * y2, h1 = bf_hi(xw1) + p.alpha * y3;
+              hown[(g + 8) * L.max_nd + rl] = h0; hown[(g + 8) * L.max_nd + rl + 1] = h1;
+              st_relaxed_u64(ll_h + ll_word(g + 8, d_lo + rl), pack_bf2(h0, h1), seq);
+            }
+          } else if (ph == 1) {                                     // g = GELU(W_up RMS(h)), packed bf16
+            if (has0) {
+              const float rs = pre ? rsqrtf(ssq_lo * inv_d + p.eps) : 1.0f;
               *reinterpret_cast<unsigned*>(g_pk + g_index(g, f_lo + rl)) = pack_bf2(gelu_erf_f(y0 * rs), gelu_erf_f(y1 * rs));
-            } else if (ph == 2) {                                     // z_t = h + alpha W_down g   (layer output)
+            }
+            if (has1) {
+              const float rs = pre ? rsqrtf(ssq_hi * inv_d + p.eps) : 1.0f;
+              *reinterpret_cast<unsigned*>(g_pk + g_index(g + 8, f_lo + rl)) = pack_bf2(gelu_erf_f(y2 * rs), gelu_erf_f(y3 * rs));
+            }
+          } else if (ph == 2) {                                     // z_t = h + alpha W_down g   (layer output)
+            if (has0) {
               const unsigned zw = pack_bf2(hown[g * L.max_nd + rl] + p.alpha * y0, hown[g * L.max_nd + rl + 1] + p.alpha * y1);
-              *reinterpret_cast<unsigned*>(z + (size_t)bq * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
               st_relaxed_u64(ll_z + ll_word(g, d_lo + rl), zw, seq);
-            } else {                                                  // raw k_t, v_t from RMS(z_t): Eqs. (1)-(2) before qkRMS
-              const size_t col = (size_t)(second_e ? d : 0) + d_lo + rl;
-              const float rs = kv_norm ? rsqrtf(ssq * inv_d + p.eps) : 1.0f;
-              st_relaxed_v4(ll_kv + (size_t)bq * (2 * d) + col, __float_as_uint(y0 * rs), seq, __float_as_uint(y1 * rs), seq);
+            }
+            if (has1) {
+              const unsigned zw = pack_bf2(hown[(g + 8) * L.max_nd + rl] + p.alpha * y2, hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * y3);
+              *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              st_relaxed_u64(ll_z + ll_word(g + 8, d_lo + rl), zw, seq);
+            }
+          } else {                                                  // raw k_t, v_t from RMS(z_t): Eqs. (1)-(2) before qkRMS
+            const size_t col = (size_t)(second_e ? d : 0) + d_lo + rl;
+            if (has0) {
+              const float rs = kv_norm ? rsqrtf(ssq_lo * inv_d + p.eps) : 1.0f;
+              st_relaxed_v4(ll_kv + (size_t)g * (2 * d) + col, __float_as_uint(y0 * rs), seq, __float_as_uint(y1 * rs), seq);
+            }
+            if (has1) {
+              const float rs = kv_norm ? rsqrtf(ssq_hi * inv_d + p.eps) : 1.0f;
+              st_relaxed_v4(ll_kv + (size_t)(g + 8) * (2 * d) + col, __float_as_uint(y2 * rs), seq, __float_as_uint(y3 * rs), seq);
             }
           }
         }
       }
-      if (ph == 1) {
-        // all of this CTA's rows of g are written: tell the warps (of every CTA) that multiply those ranges.  The
-        // release is cumulative over what the group barrier ordered before it.
-        group_sync<WG>(grp);
-        if (lw == 0 && lane <= my_r_hi - my_r_lo) red_release_add_u32(g_cnt + (size_t)(my_r_lo + lane) * 32, 1u);
-      }
+      TL(6);
       if (timing) {
         const unsigned long long now = globaltimer_ns();
         atomicAdd(&p.sync->phase_ns[2 + 2 * ph], now - t_ph - wait_ns);        // fire-and-forget, no stack array
@@ -620,33 +636,28 @@ __global__ void __launch_bounds__((NG * WG + kAttnSlots) * 32, 1) leaf_mma_kerne
 }
 
 // ------------------------------------------------------------------------------------ host
+#ifdef RT_TIMELINE
+}  // namespace rt
+extern "C" int rt_debug_read(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, rt::g_dbg, sizeof(rt::g_dbg));
+}
+namespace rt {
+#endif
 
-// Exchange-buffer sizes in 64-bit words (see LeafMmaBuffers): one group's c / h / z vector, one group's g vector.
-size_t leaf_mma_words_d(int d) { return (size_t)(d / 16) * kWordsPerKStep; }
-size_t leaf_mma_words_g(int dff) { return (size_t)(dff / 16) * kGElemsPerKStep / 4; }
-
-// Picks the number of sequence groups, the leaf capacity and the launch shape; returns false when this kernel
-// does not take the shape (the generic leaf kernel does).
-bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, int want_groups, LeafMmaLaunch* out) {
+// Picks the leaf capacity and the launch shape; returns false when this kernel does not take
+// the shape (the generic leaf kernel does).
+bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out) {
   int dev = 0, sms = 0, max_smem = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
   if (B > 16 || (d % 64) || (dff % 16) || B * H > kAttnSlots * sms) return false;
-  // groups: as many as requested (or two), lowered until no group is empty and raised until none has more than 8 sequences
-  int ng = want_groups > 0 ? want_groups : 2;
-  if (ng != 1 && ng != 2 && ng != 4) return false;
-  while (ng > 1 && (ng > B || ceil_div(B, ng) * (ng - 1) >= B)) ng /= 2;
-  while (ng < kLeafMmaMaxGroups && ceil_div(B, ng) > kSlots) ng *= 2;
-  if (ceil_div(B, ng) > kSlots) return false;
-  const int wg = ng == 1 ? 8 : 4;
   const int cands[3] = {64, 32, 16};
   for (int lf : cands) {
     if (want_leaf && lf != want_leaf) continue;
-    const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms), ng, wg);
+    const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms));
     if (L.total <= (size_t)max_smem) {
-      out->grid = sms; out->block = (ng * wg + kAttnSlots) * 32; out->smem = L.total; out->leaf = lf;
-      out->groups = ng; out->warps_per_group = wg;
+      out->grid = sms; out->block = kLeafMmaThreads; out->smem = L.total; out->leaf = lf;
       return true;
     }
   }
@@ -654,26 +665,22 @@ bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, int want_groups,
 }
 
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {
-  LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid), l.groups, l.warps_per_group);
-  // compile-time variants: groups x warps per group, per-phase timers, RMS gains present
+  LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid));
+  // compile-time variants: row blocks (B > 8), per-phase timers, RMS gains present
   const bool gains = p.g_mlp != nullptr || p.g_kv != nullptr;
-  auto pick = [&](auto ng, auto wg) -> const void* {
-    constexpr int NG = decltype(ng)::value, WG = decltype(wg)::value;
-    if (p.timers) return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<NG, WG, true, true>)
-                               : reinterpret_cast<const void*>(&leaf_mma_kernel<NG, WG, true, false>);
-    return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<NG, WG, false, true>)
-                 : reinterpret_cast<const void*>(&leaf_mma_kernel<NG, WG, false, false>);
+  auto pick = [&](auto mb) -> const void* {
+    constexpr int MB = decltype(mb)::value;
+    if (p.timers) return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, true>)
+                               : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, false>);
+    return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, true>)
+                 : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, false>);
   };
-  const void* fn = nullptr;
-  if (l.groups == 1 && l.warps_per_group == 8) fn = pick(std::integral_constant<int, 1>{}, std::integral_constant<int, 8>{});
-  else if (l.groups == 2 && l.warps_per_group == 4) fn = pick(std::integral_constant<int, 2>{}, std::integral_constant<int, 4>{});
-  else if (l.groups == 4 && l.warps_per_group == 4) fn = pick(std::integral_constant<int, 4>{}, std::integral_constant<int, 4>{});
-  if (!fn) return cudaErrorInvalidValue;
+  const void* fn = p.B > 8 ? pick(std::integral_constant<int, 2>{}) : pick(std::integral_constant<int, 1>{});
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);
   if (e != cudaSuccess) return e;
   LeafParams pp = p;
   LeafMmaBuffers b = buf;
-  void* args[] = {(void*)&pp, (void*)&L, (void*)&b};
+  void* args[] = {(void*)&pp, (void*)&L, (void*)&b.ll_c, (void*)&b.ll_h, (void*)&b.ll_g, (void*)&b.ll_z, (void*)&b.ll_kv};
   return cudaLaunchCooperativeKernel(fn, dim3(l.grid), dim3(l.block), args, l.smem, s);
 }
 

@@ -34,7 +34,7 @@ class RtConfig(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32),
                 ("dtype", C.c_int32), ("sched", C.c_int32), ("leaf", C.c_int32), ("norm_flags", C.c_int32),
                 ("rms_eps", C.c_float), ("softmax_scale", C.c_float), ("residual_scale", C.c_float),
-                ("recur_block", C.c_int32), ("leaf_groups", C.c_int32)]
+                ("recur_block", C.c_int32)]
 
 
 class RtLayerWeights(C.Structure):
@@ -219,10 +219,10 @@ def rt_profile_read() -> Dict[str, Dict[str, float]]:
 def make_config(d_model: int, n_heads: int, d_ff: int, dtype: str = "bf16", sched: str = "tiled", leaf: int = 0,
                 norm_flags: int = RT_NORM_PRE | RT_NORM_QK, rms_eps: float = 1e-6,
                 softmax_scale: Optional[float] = None, residual_scale: float = 1.0, head_dim: int = 64,
-                recur_block: int = 0, leaf_groups: int = 0) -> RtConfig:
+                recur_block: int = 0) -> RtConfig:
     return RtConfig(d_model, n_heads, head_dim, d_ff, {"f32": RT_F32, "bf16": RT_BF16}[dtype],
                     {"tiled": RT_SCHED_TILED, "naive": RT_SCHED_NAIVE}[sched], leaf, norm_flags, rms_eps,
-                    (1.0 / math.sqrt(head_dim)) if softmax_scale is None else softmax_scale, residual_scale, recur_block, leaf_groups)
+                    (1.0 / math.sqrt(head_dim)) if softmax_scale is None else softmax_scale, residual_scale, recur_block)
 
 
 # ------------------------------------------------------------------ conveniences on torch tensors
