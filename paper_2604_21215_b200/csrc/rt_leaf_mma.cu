@@ -110,12 +110,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const unsigned (&a)[4], 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-#ifdef RT_TIMELINE
-__device__ unsigned long long g_dbg[3 * 8 * 4 * 8];      // [cta slot][warp][phase][point]
-#define TL(pt) if (tl_on) g_dbg[((tl_slot * 8 + warp) * 4 + ph) * 8 + (pt)] = globaltimer_ns()
-#else
-#define TL(pt)
-#endif
 __device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory"); }
 
 // A wait that ran out: record it for the host and tell every other waiter to leave.
@@ -368,13 +362,8 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
 
   for (int t = p.t0; t < p.t1; ++t) {
     const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
-#ifdef RT_TIMELINE
-    const int tl_slot = cta == 0 ? 0 : (cta == 77 ? 1 : 2);
-    const bool tl_on = (cta == 0 || cta == 77 || cta == 147) && lane == 0 && t == p.t0 + 20 && p.t0 == 1024;
-#endif
 #pragma unroll 1
     for (int ph = 0; ph < 4; ++ph) {                              // 0: W_o   1: W_up   2: W_down   3: W_k | W_v
-      TL(0);
       // ---- what this phase multiplies ----
       const int K = (ph == 2) ? dff : d;
       const int stride = (ph == 2) ? L.stride_f : L.stride_d;
@@ -395,7 +384,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
         if (!mma_grid_barrier(p.sync, s_abort, bar_target)) return;
         if (timing) wait_ns += globaltimer_ns() - tb;
       }
-      TL(1);
       const int n_ks = K / 16;
       const int ks_per_warp = (n_ks + kMmaWarps - 1) / kMmaWarps;
       const int ks0 = warp * ks_per_warp;
@@ -404,18 +392,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
       const int tile_step = (ph == 2) ? 1 : kNT;                   // W_down: one tile per pass (see below)
       for (int t0n = 0; t0n < nt_all; t0n += tile_step) {
         const int n_tiles = nt_all - t0n < tile_step ? nt_all - t0n : tile_step;
-        // this thread's 8 bytes of weight row g (clamped to the rows that exist) of each tile, at k = 4c
-        const unsigned char* wp[kNT];
-#pragma unroll
-        for (int i = 0; i < kNT; ++i) {
-          const int ti = t0n + i < nt_all ? t0n + i : t0n;
-          const bool second = (ph == 3) && ti >= nt_d;             // W_v tiles follow the W_k tiles
-          const int r0 = (second ? ti - nt_d : ti) * 8;
-          const int valid = nrows - r0 < 8 ? nrows - r0 : 8;
-          const int r = r0 + (g < valid ? g : valid - 1);
-          const __nv_bfloat16* wbase = (ph == 0) ? s_wo : (ph == 1) ? s_wup : (ph == 2) ? s_wdn : (second ? s_wv : s_wk);
-          wp[i] = reinterpret_cast<const unsigned char*>(wbase + (size_t)r * stride + 4 * c);
-        }
         // rows this thread finishes after the reduction (warp w finishes tile t0n + w)
         const int ti_e = t0n + warp;
         const bool second_e = (ph == 3) && ti_e >= nt_d;
@@ -430,9 +406,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
         // The loops below are written without branches around the loads and the products (indices
         // are clamped, missing sequences and k-steps contribute zeros): a branch per product costs
         // more here than the product.
-        float acc[kNT][4];
-#pragma unroll
-        for (int nt = 0; nt < kNT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
         float sq0 = 0.f, sq1 = 0.f;
         bool alive = true;
         const int g0 = has0 ? g : 0, g1 = has1 ? g + 8 : 0;        // rows read by lanes without a sequence (masked below)
@@ -442,6 +415,12 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
           // pass keeps this at 32 products; the two accumulators halve the dependent chain.
           constexpr int KD = 32 / MB;
+          float acc[2][4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { acc[0][j] = acc[1][j] = 0.f; }
+          // this thread's 8 bytes of weight row g (clamped to the rows that exist) of the tile, at k = 4c
+          const int valid = nrows - t0n * 8 < 8 ? nrows - t0n * 8 : 8;
+          const unsigned char* wd0 = reinterpret_cast<const unsigned char*>(s_wdn + (size_t)(t0n * 8 + (g < valid ? g : valid - 1)) * stride + 4 * c);
           const __nv_bfloat16* b0p = g_pk + g_index(g0, 4 * c);          // + 256 elements per k-step
           const __nv_bfloat16* b1p = g_pk + g_index(g1, 4 * c);
           for (int kc0 = ks0; kc0 < ks1; kc0 += KD) {
@@ -459,20 +438,18 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
               ad[i][0] = w0[i].x; ad[i][2] = w0[i].y;
               if (MB == 2) { ad[i][1] = w1[i].x; ad[i][3] = w1[i].y; } else { ad[i][1] = 0u; ad[i][3] = 0u; }
             }
-            TL(2);
-            const unsigned char* wd = wp[0] + (size_t)kc0 * 32;
+            const unsigned char* wd = wd0 + (size_t)kc0 * 32;
 #pragma unroll
             for (int i = 0; i < KD; ++i) {
               const uint2 bw = *reinterpret_cast<const uint2*>(wd + (i < n_here ? i : 0) * 32);
               mma_bf16(acc[i & 1], ad[i], bw.x, bw.y);
-#ifdef RT_TIMELINE
-              if (i == 1 && tl_on && acc[0][0] != 123.f) TL(7);
-#endif
             }
           }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) { acc[0][j] += acc[1][j]; acc[1][j] = 0.f; }
-        } else
+          red[(warp * kNT) * 32 + lane] = make_float4(acc[0][0] + acc[1][0], acc[0][1] + acc[1][1], acc[0][2] + acc[1][2], acc[0][3] + acc[1][3]);
+        } else {
+        if (ks0 >= ks1) {                                          // a warp without k-steps (narrow layers) contributes zeros
+          for (int nt = 0; nt < n_tiles; ++nt) red[(warp * kNT + nt) * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         for (int kc0 = ks0; kc0 < ks1; kc0 += KC) {
           unsigned a[KC][4];
 #pragma unroll
@@ -524,45 +501,43 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
               }
             }
             if (timing) wait_ns += globaltimer_ns() - t_poll;
-            TL(2);
           }
           const __nv_bfloat16* gc = (GAINS && gp) ? gp + (size_t)kc0 * 16 : nullptr;
           if (want_ssq) {
 #pragma unroll
             for (int i = 0; i < KC; ++i) frag_ssq_gain<MB>(a[i], (GAINS && gc) ? gc + (i < n_here ? i : 0) * 16 : nullptr, sq0, sq1);
           }
-          // products, specialised on the number of tiles so that none sits behind a branch
-          auto products = [&](auto ntc) {
-            constexpr int NTC = decltype(ntc)::value;
+          // products, one tile of 8 weight rows after the other (a rolled loop: the step runs once per token, so
+          // compact code counts for more than interleaving the tiles' products; two accumulators per tile halve the
+          // dependent chain), each tile's partial sums going straight to the reduction buffer
+#pragma unroll 1
+          for (int nt = 0; nt < n_tiles; ++nt) {
+            float ce[4] = {0.f, 0.f, 0.f, 0.f}, co[4] = {0.f, 0.f, 0.f, 0.f};
+            const int ti = t0n + nt;
+            const bool second = (ph == 3) && ti >= nt_d;
+            const int r0 = (second ? ti - nt_d : ti) * 8;
+            const int valid = nrows - r0 < 8 ? nrows - r0 : 8;
+            const int r = r0 + (g < valid ? g : valid - 1);
+            const __nv_bfloat16* wbase = (ph == 0) ? s_wo : (ph == 1) ? s_wup : (second ? s_wv : s_wk);
+            const unsigned char* w = reinterpret_cast<const unsigned char*>(wbase + (size_t)r * stride + 4 * c) + (size_t)kc0 * 32;
 #pragma unroll
             for (int i = 0; i < KC; ++i) {
-              const int off = ((i < n_here ? i : 0) + kc0) * 32;
-#pragma unroll
-              for (int nt = 0; nt < NTC; ++nt) {
-                const uint2 bw = *reinterpret_cast<const uint2*>(wp[nt] + off);
-                mma_bf16(acc[nt], a[i], bw.x, bw.y);
-              }
+              const uint2 bw = *reinterpret_cast<const uint2*>(w + (i < n_here ? i : 0) * 32);
+              if (i & 1) mma_bf16(co, a[i], bw.x, bw.y); else mma_bf16(ce, a[i], bw.x, bw.y);
             }
-          };
-          switch (n_tiles) {
-            case 1: products(std::integral_constant<int, 1>{}); break;
-            case 2: products(std::integral_constant<int, 2>{}); break;
-            case 3: products(std::integral_constant<int, 3>{}); break;
-            default: products(std::integral_constant<int, 4>{}); break;
+            float4 v = make_float4(ce[0] + co[0], ce[1] + co[1], ce[2] + co[2], ce[3] + co[3]);
+            if (kc0 > ks0) { const float4 o = red[(warp * kNT + nt) * 32 + lane]; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+            red[(warp * kNT + nt) * 32 + lane] = v;
           }
         }
-        TL(3);
+        }
         // ---- reduce the K split over the 8 warps; warp w then holds the sums of tile t0n + w ----
-#pragma unroll
-        for (int nt = 0; nt < kNT; ++nt)
-          if (nt < n_tiles) red[(warp * kNT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
         if (want_ssq) {
           sq0 += __shfl_xor_sync(0xffffffffu, sq0, 1); sq0 += __shfl_xor_sync(0xffffffffu, sq0, 2);
           sq1 += __shfl_xor_sync(0xffffffffu, sq1, 1); sq1 += __shfl_xor_sync(0xffffffffu, sq1, 2);
           if (c == 0) { ssq_red[warp * 16 + g] = sq0; ssq_red[warp * 16 + 8 + g] = sq1; }
         }
         mma_warps_sync();
-        TL(4);
         if (*s_abort) return;
         float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f, ssq_lo = 0.f, ssq_hi = 0.f;
         if (warp < n_tiles) {
@@ -577,7 +552,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           }
         }
         mma_warps_sync();       // red / ssq_red may be overwritten from here on
-        TL(5);
         // ---- epilogue: y0, y1 = rows rl, rl+1 for sequence g; y2, y3 = the same rows for sequence g+8 ----
         if (mine) {
           if (ph == 0) {                                            // h = x_t + alpha W_o c_t
@@ -624,7 +598,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           }
         }
       }
-      TL(6);
       if (timing) {
         const unsigned long long now = globaltimer_ns();
         atomicAdd(&p.sync->phase_ns[2 + 2 * ph], now - t_ph - wait_ns);        // fire-and-forget, no stack array
@@ -636,13 +609,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
 }
 
 // ------------------------------------------------------------------------------------ host
-#ifdef RT_TIMELINE
-}  // namespace rt
-extern "C" int rt_debug_read(unsigned long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, rt::g_dbg, sizeof(rt::g_dbg));
-}
-namespace rt {
-#endif
 
 // Picks the leaf capacity and the launch shape; returns false when this kernel does not take
 // the shape (the generic leaf kernel does).
