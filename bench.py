@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the RT prefill hot path on synthetic data.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5_N<len>] [--sched tiled|naive]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c2|c3|c5_N<len>] [--sched tiled|naive]
     python bench.py --impl reference ...          # times the fp64 CPU oracle instead
 
 A step is one pass of the whole hot path (pre-pass, every leaf launch, every cross tile) over
@@ -38,9 +38,18 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "source": "fallback"}
 
 
-# DRAM bytes (read + write) of one leaf launch (64 token steps) from the ncu capture summarised in
-# profiles/leaf_mma_kernel_c2.txt: the launch stages its weight rows once, everything else stays in L2.
-NCU_LEAF_TRAFFIC = {"c2": 14701056 + 28416}
+def leaf_traffic_table():
+    """DRAM bytes (read + write) of ONE leaf launch per workload, from single-launch ncu captures; the table lives in
+    profiles/leaf_mma_kernel_dram_bytes.md as rows `| workload | bytes |` (a launch stages its weight rows once,
+    everything else stays in L2).  Workloads without a row report null."""
+    out = {}
+    path = os.path.join(ROOT, "profiles", "leaf_mma_kernel_dram_bytes.md")
+    if os.path.exists(path):
+        for ln in open(path):
+            f = [t.strip() for t in ln.strip().strip("|").split("|")]
+            if len(f) >= 2 and f[1].isdigit():
+                out[f[0]] = int(f[1])
+    return out
 
 
 class ClockSampler:
@@ -174,8 +183,9 @@ def run_reference(args):
     tot = sum(times)
     value = wl.B * n_pos * args.steps / tot
     cores = oracle_cores()
-    sample = (f"fp64 oracle (numpy) on the first {n_pos} of {wl.N} positions of all {wl.B} sequences per step; "
-              "later positions cost more (longer prefixes), so the full workload would be slower per token")
+    sample = (f"fp64 oracle (numpy + BLAS) on the first {n_pos} of {wl.N} positions of all {wl.B} sequences per step "
+              "(the positions the CUDA arm's cpu_baseline times); later positions cost more (longer prefixes), so the "
+              "full workload would be slower per token")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -325,7 +335,7 @@ def run_cuda(args):
         achieved = alg_bytes / (leaf_ms * 1e-3) / 1e9 if leaf_ms > 0 else 0.0
         roofline = {"kernel": "leaf_mma_kernel" if (wl.dtype == "bf16" and args.sched == "tiled") else "leaf_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "traffic": NCU_LEAF_TRAFFIC.get(wl.name),
+                    "traffic": leaf_traffic_table().get(wl.name),
                     "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": leaf_ms,
                     "us_per_token_step": 1e3 * leaf_ms / max(tok_steps_per_launch, 1),
                     "note": "weights stay in shared memory for a whole launch, so the kernel is bound by the "
@@ -362,9 +372,11 @@ def run_cuda(args):
         tile_ms = prof["tile"]["ms"]
         tile_tflops = (counters["flops_tile"] * args.steps / (tile_ms * 1e-3) / 1e12) if tile_ms > 0 else None
         n_pos = sample_positions(wl)
+        oracle_sample(wl, data, min(n_pos, 16), args.recur_block)         # untimed: starts the BLAS threads
         t_cpu = oracle_sample(wl, data, n_pos, args.recur_block)
         cpu = {"value": wl.B * n_pos / t_cpu, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle",
-               "sample": f"first {n_pos} of {wl.N} positions, all {wl.B} sequences, one run ({t_cpu:.1f} s)"}
+               "sample": f"first {n_pos} of {wl.N} positions, all {wl.B} sequences, one warmed run ({t_cpu:.1f} s); "
+                         "`--impl reference` times the same positions"}
         launches = sum(v["launches"] for v in prof.values())
         # the pre-pass group is three kernels, every other group one
         gpu_launches = int(launches + 2 * prof["prepass"]["launches"])
@@ -397,10 +409,52 @@ def run_cuda(args):
                           "flops_tile": counters["flops_tile"], "flops_leaf": counters["flops_leaf"],
                           "flops_gemm": counters["flops_gemm"]},
                 "wall_s_timed_region": wall}
+        if world == 1 and args.also:
+            line["also"] = measure_also([n for n in args.also.split(",") if n and n != wl.name], 3, dev, stream, flush)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def measure_also(names, steps, dev, stream, flush):
+    """Tokens/s of other single-layer workloads in this process (few steps each; same timing rules as the main line)."""
+    import torch
+    from paper_2604_21215_b200 import inputs, rt
+    out = {}
+    for name in names:
+        wl = get_workload(name)
+        data = inputs.make_inputs(wl)
+        tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        layer = rt.Layer(wl.d_model, wl.n_heads, wl.d_ff, dtype=wl.dtype, device=str(dev), residual_scale=wl.residual_scale)
+        layer.set_weights(data["layers"][0])
+        layer.reserve(wl.B, wl.N)
+        x = torch.from_numpy(data["x"]).to(tdt).to(dev)
+        z = torch.empty_like(x)
+        for _ in range(3):
+            layer.prefill_device(x, z)
+        torch.cuda.synchronize(dev)
+        rt.rt_profile_enable(True)
+        rt.rt_profile_read()
+        evs = []
+        for _ in range(steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); layer.prefill_device(x, z); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        prof = rt.rt_profile_read()
+        rt.rt_profile_enable(False)
+        if layer.status() != rt.RT_OK:
+            out[name] = {"error": rt.rt_status_string(layer.status())}
+            continue
+        ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+        out[name] = {"tokens_per_s": wl.B * wl.N / (ms * 1e-3), "ms_per_step": ms, "steps": steps, "B": wl.B, "N": wl.N,
+                     "d_model": wl.d_model, "us_per_token_step": 1e3 * prof["leaf"]["ms"] / (wl.N * steps),
+                     "tile_ms_per_step": prof["tile"]["ms"] / steps}
+        del layer, x, z
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_tile_bench(args):
@@ -657,13 +711,28 @@ def run_backward_bench(args):
 BASE_TILE_SEED = 20260421
 
 
+def spawn_replicas(args):
+    """`python bench.py --gpus N` without a launcher: start one replica process per GPU (the launch line the contract
+    gives for N > 1) and pass rank 0's JSON line through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4",
+                    help="c4 (default: the 8-layer stack, the largest single-GPU configuration), c2, c3, c5_N<len>, p512")
+    ap.add_argument("--also", default="c2,c3",
+                    help="single-layer workloads also timed in the same process and reported under `also` ('' = none)")
     ap.add_argument("--sched", default="tiled", choices=["tiled", "naive"])
     ap.add_argument("--leaf", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
@@ -690,6 +759,8 @@ def main():
         return run_backward_bench(args)
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_replicas(args)
     return run_cuda(args)
 
 

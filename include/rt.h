@@ -11,18 +11,22 @@
  *
  * Conventions for every entry point
  *  - All tensor pointers are DEVICE pointers unless a comment says "host".  The caller owns
- *    every buffer, including the workspace; the library allocates no device memory and keeps
- *    no global mutable state.  Pointers must be 16-byte aligned.
+ *    every buffer, including the workspace; the library allocates no device memory.  Its only
+ *    state outside the caller's buffers: the profiling switch (rt_profile_enable), the built-in
+ *    scratch array of rt_layer_decode_step_static, and per-thread caches of encoded tensor maps
+ *    and kernel attributes (pure functions of their arguments).  It reads no environment
+ *    variables.  Pointers must be 16-byte aligned.
  *  - Storage type (rt_dtype) applies to x, weights, gains, z, the K/V caches and the
  *    embedding.  Accumulation is always fp32.  Logits are fp32.
  *  - Weights are row-major [out, in]:  y = W u.
- *  - x and z are [B, N, d_model] row-major.  z must not alias x.
+ *  - x and z are [B, N, d_model] row-major.  z must not overlap x (checked: RT_ERR_INVALID_ARG).
  *  - A K/V cache is POSITION-MAJOR [N_max, B, d_model] (Sec. 6, "Cache locality"): row t
  *    holds the persistent pair of position t for all sequences.  Prefill writes rows [0, N),
  *    decode appends row pos.  All sequences of a batch share the same length.
  *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
  *    stream) and return without synchronising.  Argument, shape, alignment and workspace
- *    errors are detected on the host before anything is enqueued.  A device-side bounded
+ *    errors, and configurations an entry point does not support, are detected on the host
+ *    before anything is enqueued.  A device-side bounded
  *    wait that runs out is recorded in the workspace and read with rt_get_status after the
  *    caller has synchronised the stream.  Nothing aborts, traps or throws.
  *  - The same workspace must not be used by two calls that overlap in time.
@@ -54,11 +58,18 @@ typedef enum { RT_F32 = 0, RT_BF16 = 1 } rt_dtype;
  * as the comparison path.  Both give the same result up to rounding order. */
 typedef enum { RT_SCHED_TILED = 0, RT_SCHED_NAIVE = 1 } rt_sched;
 
-enum {                      /* rt_config.norm_flags */
+enum {                      /* rt_config.norm_flags (bit 2 is not used: Sec. 2.2 normalises queries and keys "independently
+                               per head", and a full-width variant would need a reduction across all heads inside every
+                               token step of the leaf kernel; any other bit is RT_ERR_INVALID_ARG) */
   RT_NORM_PRE = 1,          /* RMS(x_i), RMS before the MLP and RMS(z_i) are applied (Sec. 2.2) */
   RT_NORM_QK = 2,           /* qkRMS on queries and keys, per head */
-  RT_NORM_QK_FULL = 4,      /* qkRMS over the full width: oracle only, RT_ERR_UNSUPPORTED here */
   RT_NORM_SKIP_Z = 8        /* persistent pair from z_i itself (the RMSNorm-ablation appendix) */
+};
+
+enum {                      /* rt_config.flags */
+  RT_FLAG_BACKWARD_STEP_LAUNCHES = 1   /* rt_layer_backward: run the reverse loop as one launch per step instead of one
+                                          cooperative launch per leaf (the form a device without cooperative launch gets
+                                          anyway; same device code, used by tests to compare the two) */
 };
 
 typedef struct {
@@ -75,6 +86,7 @@ typedef struct {
                                of all positions in earlier blocks and to the temporary pairs of the positions j <= i of its own
                                block, so a block is computed in one parallel sweep; S >= N is an ordinary pre-LN Transformer
                                layer).  Prefill entry points only, tiled schedule; decode returns RT_ERR_UNSUPPORTED */
+  int32_t flags;            /* RT_FLAG_*; 0 for the defaults */
 } rt_config;
 
 typedef struct {            /* device pointers; read-only */
@@ -106,7 +118,9 @@ rt_status rt_layer_prefill(const rt_config *cfg, const rt_layer_weights *w,
 /* A stack of n_layers RT layers with token embedding and tied output head:
  * x^0 = emb[ids], x^l = layer_l(x^{l-1}), logits = emb . RMS_{g_final}(x^L at the last position).
  * `layers`, `k_caches`, `v_caches` are HOST arrays of n_layers entries (device pointers inside).
- * hidden [B,N,d] (storage type) and logits_last [B,vocab] (fp32) may each be NULL. */
+ * hidden [B,N,d] (storage type) and logits_last [B,vocab] (fp32) may each be NULL.
+ * The head keeps one fp32 row of d_model per sequence in shared memory: B * d_model * 4 bytes must not exceed 200 KB
+ * (RT_ERR_UNSUPPORTED otherwise; the same holds for rt_decode_step). */
 rt_status rt_stack_prefill(const rt_config *cfg, int32_t n_layers, const rt_layer_weights *layers,
                            const void *emb, const void *g_final, int32_t vocab,
                            const int32_t *ids, int32_t B, int32_t N,
@@ -146,13 +160,18 @@ rt_status rt_layer_decode_step(const rt_config *cfg, const rt_layer_weights *w,
  *  - All calls on a device share the one array, which keeps the previous call's contents; the
  *    words that must start from zero are cleared on the stream at the start of each call.  Two
  *    calls that overlap on the GPU (different streams, no dependency) race on it: serialise them.
- *  - The device status word of such a call lives in the built-in scratch and cannot be read
- *    back through rt_get_status; use the workspace variant where that matters. */
+ *  - The device status word of such a call lives in the built-in scratch: read it with
+ *    rt_static_get_status() (below) after synchronising the stream. */
 #define RT_STATIC_SCRATCH_BYTES (8u << 20)
 rt_status rt_layer_decode_step_static(const rt_config *cfg, const rt_layer_weights *w,
                                       const void *x, int32_t B, int32_t pos,
                                       void *z, void *k_cache, void *v_cache, int32_t N_max,
                                       void *cuda_stream);
+
+/* rt_get_status for the built-in scratch of rt_layer_decode_step_static on the current device (the paper has no
+ * counterpart): after the caller synchronised the stream, copies back the status word of the last such call
+ * (a blocking 4-byte copy): RT_OK, or RT_ERR_TIMEOUT when a bounded device-side wait ran out.  Allocates nothing. */
+rt_status rt_static_get_status(void);
 
 /* After the caller synchronised the stream: copies the device status word of `workspace`
  * back (a blocking 4-byte copy) and returns it (RT_OK or RT_ERR_TIMEOUT). */

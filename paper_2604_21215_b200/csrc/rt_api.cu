@@ -14,6 +14,7 @@ using namespace rt;
 namespace {
 
 constexpr int kMaxChunks = 32;
+constexpr int kSmallBatchMax = 64;      // above this the per-token chain runs as dense products (tiled prefill only)
 constexpr int kAutoLeaf = 64;
 
 struct WsLayout {
@@ -31,16 +32,14 @@ bool config_ok(const rt_config* c) {
   if (c->sched != RT_SCHED_TILED && c->sched != RT_SCHED_NAIVE) return false;
   if (c->leaf != 0 && (c->leaf < 16 || c->leaf > 256 || (c->leaf & (c->leaf - 1)))) return false;
   if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
-  if (c->norm_flags & ~15) return false;
+  if (c->norm_flags & ~(RT_NORM_PRE | RT_NORM_QK | RT_NORM_SKIP_Z)) return false;
   if (c->recur_block < 0) return false;
+  if (c->flags & ~RT_FLAG_BACKWARD_STEP_LAUNCHES) return false;
   return true;
 }
 
-constexpr int kSmallBatchMax = 64;      // above this the per-token chain runs as dense products (tiled prefill only)
-
 rt_status config_supported(const rt_config* c, int B, bool wide_ok = false) {
   if (c->head_dim != kHeadDim) return RT_ERR_UNSUPPORTED;
-  if (c->norm_flags & RT_NORM_QK_FULL) return RT_ERR_UNSUPPORTED;
   if (c->d_ff % 4) return RT_ERR_UNSUPPORTED;
   if (B > kSmallBatchMax && !(wide_ok && c->sched == RT_SCHED_TILED)) return RT_ERR_UNSUPPORTED;
   return RT_OK;
@@ -85,6 +84,10 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b);
+  return pa < pb + nb && pb < pa + na;
+}
 
 bool weights_ok(const rt_layer_weights* w) {
   if (!w) return false;
@@ -96,6 +99,26 @@ bool weights_ok(const rt_layer_weights* w) {
 }
 
 int leaf_size(const rt_config* c) { return c->leaf ? c->leaf : kAutoLeaf; }
+
+// Which form of the per-token chain a prefill with this configuration and batch runs, and the granularity of
+// Algorithm 1's tiles that goes with it.  Used by run_layer and by rt_plan_counters, so that the modelled schedule is
+// the one that runs (the tensor-core leaf kernel's leaf depends on the shared memory of the part; the planner assumes
+// a B200).
+enum ChainPath { kPathGeneric = 0, kPathMma = 1, kPathWide = 2, kPathBlocks = 3 };
+struct Schedule { ChainPath path; int leaf; };
+Schedule effective_schedule(const rt_config* c, int B) {
+  if (c->recur_block > 1) return {kPathBlocks, c->recur_block};
+  if (c->sched == RT_SCHED_TILED) {
+    // bf16 batches the persistent tensor-core leaf kernel does not take (B > 16) are faster as dense products from
+    // about 24 sequences on (measured at d = 1024: 68 us per token step at B = 32 and 64 against 99 and 191 us for the
+    // generic kernel); fp32 keeps the generic kernel up to its limit
+    if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : 32};
+    LeafMmaLaunch ml;
+    if (c->dtype == RT_BF16 && leaf_mma_shape(B, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
+      return {kPathMma, ml.leaf};
+  }
+  return {kPathGeneric, leaf_size(c)};
+}
 
 // ---- optional per-kernel-class timing (rt_profile_enable / rt_profile_read) -----------------
 enum ProfClass { kProfPrepass = 0, kProfLeaf = 1, kProfTile = 2, kProfOther = 3, kProfClasses = 4 };
@@ -235,11 +258,8 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     return RT_OK;
   }
 
-  // bf16 batches the persistent tensor-core leaf kernel does not take (B > 16) are faster as dense products from
-  // about 24 sequences on (measured at d = 1024: 68 us per token step at B = 32 and 64 against 99 and 191 us for the
-  // generic kernel); fp32 keeps the generic kernel up to its limit
-  const bool wide = B > kSmallBatchMax ||
-                    (c->dtype == RT_BF16 && c->sched == RT_SCHED_TILED && pos0 == 0 && B >= 24);
+  const Schedule plan = effective_schedule(c, B);
+  const bool wide = B > kSmallBatchMax || (plan.path == kPathWide && pos0 == 0);
   if (wide) {
     // Wide batches (the regime of the paper's own experiments, Sec. 6: B in the hundreds): a token step is a chain
     // of dense products with M = B rows, so it runs on the tensor cores through the same kernels as the parallel
@@ -274,7 +294,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     dp.partial = (float*)(ws + L.ex_part); dp.partial_bytes = (size_t)B * c->n_heads * kMaxChunks * 68 * 4;
     // in-leaf attention re-reads the leaf's pairs for every position (leaf^2 * B * d bytes per leaf), so wide
     // batches default to a shorter leaf
-    const int Lf = c->leaf ? c->leaf : 32, N = n_rows;
+    const int Lf = plan.path == kPathWide ? plan.leaf : (c->leaf ? c->leaf : 32), N = n_rows;
     for (int s0 = 0; s0 < N; s0 += Lf) {
       const int e0 = s0 + Lf < N ? s0 + Lf : N;
       {
@@ -393,6 +413,8 @@ rt_status common_checks(const rt_config* c, int B, int N, int n_layers, void* ws
   if (!config_ok(c) || B <= 0 || N <= 0 || n_layers <= 0 || !ws || !aligned16(ws)) return RT_ERR_INVALID_ARG;
   const rt_status st = config_supported(c, B, wide_ok);
   if (st != RT_OK) return st;
+  // the recurrence over blocks exists for tiled prefill only (wide_ok marks the prefill entry points)
+  if (c->recur_block > 1 && !(wide_ok && c->sched == RT_SCHED_TILED)) return RT_ERR_UNSUPPORTED;
   if (ws_bytes < ws_layout(c, B, N).total) return RT_ERR_WORKSPACE;
   return RT_OK;
 }
@@ -416,8 +438,10 @@ rt_status rt_layer_prefill(const rt_config* cfg, const rt_layer_weights* w, cons
                            size_t workspace_bytes, void* cuda_stream) {
   rt_status st = common_checks(cfg, B, N, 1, workspace, workspace_bytes, true);
   if (st != RT_OK) return st;
-  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || x == z || N_max < N) return RT_ERR_INVALID_ARG;
+  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || N_max < N) return RT_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(z) || !aligned16(k_cache) || !aligned16(v_cache)) return RT_ERR_INVALID_ARG;
+  const size_t xz_bytes = (size_t)B * N * cfg->d_model * esize_of(cfg->dtype);
+  if (overlaps(x, xz_bytes, z, xz_bytes)) return RT_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, N);
@@ -540,8 +564,12 @@ rt_status rt_layer_decode_step(const rt_config* cfg, const rt_layer_weights* w, 
                                size_t workspace_bytes, void* cuda_stream) {
   rt_status st = common_checks(cfg, B, 1, 1, workspace, workspace_bytes);
   if (st != RT_OK) return st;
-  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || x == z || pos < 0 || pos >= N_max) return RT_ERR_INVALID_ARG;
+  if (!weights_ok(w) || !x || !z || !k_cache || !v_cache || pos < 0 || pos >= N_max) return RT_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(z) || !aligned16(k_cache) || !aligned16(v_cache)) return RT_ERR_INVALID_ARG;
+  {
+    const size_t xz_bytes = (size_t)B * cfg->d_model * esize_of(cfg->dtype);
+    if (overlaps(x, xz_bytes, z, xz_bytes)) return RT_ERR_INVALID_ARG;
+  }
   cudaStream_t s = (cudaStream_t)cuda_stream;
   unsigned char* ws = (unsigned char*)workspace;
   const WsLayout L = ws_layout(cfg, B, 1);
@@ -747,15 +775,20 @@ rt_status rt_plan_counters(const rt_config* cfg, int32_t B, int32_t N, int32_t n
     kv = b * d * e * n * (n - 1);                        // K and V rows of the whole prefix, every position
     fl_leaf += 4 * d * b * (n * (n - 1) / 2);
   } else {
-    const uint64_t Lf = leaf_size(cfg);
+    // the schedule that runs: leaf (or block) granularity of the chain form this shape takes
+    const Schedule plan = effective_schedule(cfg, B);
+    const uint64_t Lf = plan.leaf;
     for (uint64_t s0 = 0; s0 < n; s0 += Lf) {
       const uint64_t e0 = s0 + Lf < n ? s0 + Lf : n, len = e0 - s0;
       ++leaves;
-      rd += chain_w;                                     // each launch stages its weight rows once
+      // persistent kernels stage their weight rows once per leaf launch; dense products (wide batches, block sweeps)
+      // stream them once per position resp. once per block
+      rd += chain_w * (plan.path == kPathWide ? len : 1);
       kv_leaf += 2 * b * d * e * (len * (len - 1) / 2);  // in-leaf pairs: written a few steps earlier, L2-resident
       fl_leaf += 4 * d * b * (len * (len - 1) / 2);
       if (e0 < n) {
-        const uint64_t P = e0 & (~e0 + 1);
+        const uint64_t blocks = e0 / Lf;
+        const uint64_t P = Lf * (blocks & (~blocks + 1));
         const uint64_t nq = (e0 + P < n ? e0 + P : n) - e0;
         ++tiles;
         kv += 2 * P * b * d * e;

@@ -1209,7 +1209,8 @@ bool bwd_config_ok(const rt_config* c) {
   if (c->d_model <= 0 || c->n_heads <= 0 || c->d_ff <= 0 || (long long)c->n_heads * c->head_dim != c->d_model) return false;
   if (c->dtype != RT_F32 && c->dtype != RT_BF16) return false;
   if (!(c->rms_eps >= 0.f) || !isfinite(c->softmax_scale) || !isfinite(c->residual_scale)) return false;
-  if (c->norm_flags & ~15) return false;
+  if (c->norm_flags & ~(RT_NORM_PRE | RT_NORM_QK | RT_NORM_SKIP_Z)) return false;
+  if (c->flags & ~RT_FLAG_BACKWARD_STEP_LAUNCHES) return false;
   return true;
 }
 
@@ -1372,10 +1373,9 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
   };
   RT_TRY(cudaFuncSetAttribute(loop_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
   RT_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_loop_kernel<T, 4>, kRmThreads, smem_max));
-  // RT_BACKWARD_STEP_LAUNCHES=1 in the environment forces the one-launch-per-step form (kept for devices without
-  // cooperative launch; the tests run both forms)
-  const char* force_steps = getenv("RT_BACKWARD_STEP_LAUNCHES");
-  bool use_coop = coop && per_sm >= 1 && !(force_steps && force_steps[0] == '1');
+  // RT_FLAG_BACKWARD_STEP_LAUNCHES in the configuration forces the one-launch-per-step form (what a device without
+  // cooperative launch gets; the tests run both forms)
+  bool use_coop = coop && per_sm >= 1 && !(c->flags & RT_FLAG_BACKWARD_STEP_LAUNCHES);
   // weight slices resident in shared memory when every step has at most one task per CTA and they fit beside the staging
   const size_t slice_bytes = ((size_t)d * cols_pair + (size_t)d * cols_down + (size_t)(f / up_split) * cols_up + (size_t)d * cols_out) * sizeof(T);
   const bool one_task = (d / cols_pair) * chunks * 2 <= sms && (f / cols_down) * chunks <= sms && (d / cols_up) * chunks * up_split <= sms &&
@@ -1581,7 +1581,7 @@ rt_status rt_layer_backward(const rt_config* cfg, const rt_layer_weights* w, con
                             size_t workspace_bytes, void* cuda_stream) {
   using namespace rt;
   if (!bwd_config_ok(cfg) || B <= 0 || N <= 0 || !workspace || ((uintptr_t)workspace & 15)) return RT_ERR_INVALID_ARG;
-  if (cfg->head_dim != kHeadDim || (cfg->norm_flags & RT_NORM_QK_FULL) || cfg->d_ff % 32 || cfg->recur_block > 1)
+  if (cfg->head_dim != kHeadDim || cfg->d_ff % 32 || cfg->recur_block > 1)
     return RT_ERR_UNSUPPORTED;
   if (!w || !w->w_q || !w->w_k || !w->w_v || !w->w_o || !w->w_up || !w->w_down || !x || !z || !dz || !dx || !grads)
     return RT_ERR_INVALID_ARG;

@@ -51,6 +51,10 @@ cudaError_t wait_expiry_selftest_launch(SyncArea* sync, cudaStream_t s);
 struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
 struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [16,d/2] words x3, packed bf16 [B,dff], [B,2d] words
 bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out);
+// the same decision for a device with `sms` multiprocessors and `max_smem` bytes of shared memory per CTA (no CUDA call)
+bool leaf_mma_shape(int B, int d, int H, int dff, int want_leaf, int sms, size_t max_smem, LeafMmaLaunch* out);
+constexpr int kB200Sms = 148;                    // the part this library is written for: what the pure-host planner assumes
+constexpr size_t kB200SmemPerCta = 232448;
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s);
 
 // Pre-pass (Algorithm 1, line 1 and the temporary pair of line 7, hoisted out of the loop).

@@ -610,24 +610,30 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
 
 // ------------------------------------------------------------------------------------ host
 
-// Picks the leaf capacity and the launch shape; returns false when this kernel does not take
-// the shape (the generic leaf kernel does).
-bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out) {
-  int dev = 0, sms = 0, max_smem = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+// Picks the leaf capacity and the launch shape for a device with `sms` multiprocessors and `max_smem` bytes of shared
+// memory per CTA (pure host arithmetic); returns false when this kernel does not take the shape (the generic leaf
+// kernel does).
+bool leaf_mma_shape(int B, int d, int H, int dff, int want_leaf, int sms, size_t max_smem, LeafMmaLaunch* out) {
   if (B > 16 || (d % 64) || (dff % 16) || B * H > kAttnSlots * sms) return false;
   const int cands[3] = {64, 32, 16};
   for (int lf : cands) {
     if (want_leaf && lf != want_leaf) continue;
     const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms));
-    if (L.total <= (size_t)max_smem) {
+    if (L.total <= max_smem) {
       out->grid = sms; out->block = kLeafMmaThreads; out->smem = L.total; out->leaf = lf;
       return true;
     }
   }
   return false;
+}
+
+// The same for the current device.
+bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out) {
+  int dev = 0, sms = 0, max_smem = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+  return leaf_mma_shape(B, d, H, dff, want_leaf, sms, (size_t)max_smem, out);
 }
 
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {

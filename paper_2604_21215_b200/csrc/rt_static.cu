@@ -54,3 +54,10 @@ extern "C" rt_status rt_layer_decode_step_static(const rt_config* cfg, const rt_
   if (st != RT_OK) return st;
   return rt_layer_decode_step(cfg, w, x, B, pos, z, k_cache, v_cache, N_max, scratch, kStaticScratchBytes, cuda_stream);
 }
+
+extern "C" rt_status rt_static_get_status(void) {
+  void* scratch = nullptr;
+  const rt_status st = scratch_for_current_device(&scratch);
+  if (st != RT_OK) return st;
+  return rt_get_status(scratch);      // the status word is the first word of the scratch, as in any workspace
+}

@@ -303,8 +303,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 // ------------------------------------------------------------------------------------ host
 
-// [rows, B, H, 64] bf16 viewed as a 4-D tensor; a box is `box_rows` rows of one head of one sequence.
-static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H, int box_rows) {
+static bool make_map_uncached(CUtensorMap* map, const void* base, int rows, int B, int H, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)H, (cuuint64_t)B, (cuuint64_t)rows};
@@ -314,6 +313,25 @@ static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H,
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [rows, B, H, 64] bf16 viewed as a 4-D tensor; a box is `box_rows` rows of one head of one sequence.  An encoded
+// map is a pure function of these arguments, so each thread remembers the ones it made: a prefill launches a tile
+// after every leaf, always on the same three buffers.
+static bool make_map(CUtensorMap* map, const void* base, int rows, int B, int H, int box_rows) {
+  struct Entry { const void* base; int rows, B, H, box_rows; CUtensorMap map; };
+  constexpr int kEntries = 64;
+  thread_local Entry tab[kEntries];
+  thread_local int used = 0, next = 0;
+  for (int i = 0; i < used; ++i)
+    if (tab[i].base == base && tab[i].rows == rows && tab[i].B == B && tab[i].H == H && tab[i].box_rows == box_rows) {
+      *map = tab[i].map;
+      return true;
+    }
+  if (!make_map_uncached(map, base, rows, B, H, box_rows)) return false;
+  const int slot = used < kEntries ? used++ : (next++ % kEntries);
+  tab[slot].base = base; tab[slot].rows = rows; tab[slot].B = B; tab[slot].H = H; tab[slot].box_rows = box_rows; tab[slot].map = *map;
+  return true;
 }
 
 // rows_q / rows_kv: number of rows the query buffer / caches hold (bounds for the tensor maps).
@@ -327,7 +345,7 @@ cudaError_t tile_tc_launch(const TileParams& p, int rows_q, int rows_kv, SyncAre
   const size_t smem = TcCfg::total + 1024;
   dim3 grid(ceil_div(nq, kBM), p.B * p.H, p.batch > 1 ? p.batch : 1);
   auto go = [&](auto kernel) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
     kernel<<<grid, TcCfg::threads, smem, s>>>(mq, mk, mv, p, sync);
     return cudaGetLastError();

@@ -21,12 +21,14 @@ LIB_PATH = os.path.join(_HERE, "librt_b200.so")
 RT_OK, RT_ERR_INVALID_ARG, RT_ERR_UNSUPPORTED, RT_ERR_WORKSPACE, RT_ERR_CUDA, RT_ERR_TIMEOUT = range(6)
 RT_F32, RT_BF16 = 0, 1
 RT_SCHED_TILED, RT_SCHED_NAIVE = 0, 1
-RT_NORM_PRE, RT_NORM_QK, RT_NORM_QK_FULL, RT_NORM_SKIP_Z = 1, 2, 4, 8
+RT_NORM_PRE, RT_NORM_QK, RT_NORM_SKIP_Z = 1, 2, 8
+RT_FLAG_BACKWARD_STEP_LAUNCHES = 1
 
 EXPORTS = ("rt_workspace_bytes", "rt_layer_prefill", "rt_stack_prefill", "rt_decode_step",
            "rt_layer_decode_step", "rt_get_status", "rt_status_string", "rt_plan_counters", "rt_plan_tiles",
            "rt_profile_enable", "rt_profile_read", "rt_layer_decode_step_static", "rt_update_tile", "rt_selftest_wait_expiry",
-           "rt_recompute_workspace_bytes", "rt_layer_recompute", "rt_backward_workspace_bytes", "rt_layer_backward")
+           "rt_recompute_workspace_bytes", "rt_layer_recompute", "rt_backward_workspace_bytes", "rt_layer_backward",
+           "rt_static_get_status")
 RT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -34,7 +36,7 @@ class RtConfig(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32),
                 ("dtype", C.c_int32), ("sched", C.c_int32), ("leaf", C.c_int32), ("norm_flags", C.c_int32),
                 ("rms_eps", C.c_float), ("softmax_scale", C.c_float), ("residual_scale", C.c_float),
-                ("recur_block", C.c_int32)]
+                ("recur_block", C.c_int32), ("flags", C.c_int32)]
 
 
 class RtLayerWeights(C.Structure):
@@ -76,6 +78,8 @@ def _load():
     lib.rt_layer_decode_step.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P, Z, P]
     lib.rt_layer_decode_step_static.restype = C.c_int
     lib.rt_layer_decode_step_static.argtypes = [C.POINTER(RtConfig), C.POINTER(RtLayerWeights), P, I, I, P, P, P, I, P]
+    lib.rt_static_get_status.restype = C.c_int
+    lib.rt_static_get_status.argtypes = []
     lib.rt_selftest_wait_expiry.restype = C.c_int
     lib.rt_selftest_wait_expiry.argtypes = [P, P]
     lib.rt_recompute_workspace_bytes.restype = Z
@@ -149,6 +153,11 @@ def rt_layer_decode_step_static(cfg, w, x, B, pos, z, k_cache, v_cache, N_max, s
     return _lib.rt_layer_decode_step_static(C.byref(cfg), C.byref(w), x, B, pos, z, k_cache, v_cache, N_max, stream)
 
 
+def rt_static_get_status() -> int:
+    """Device status word of the last rt_layer_decode_step_static call on the current device (after a synchronise)."""
+    return _lib.rt_static_get_status()
+
+
 def rt_stack_prefill(cfg, n_layers, layers, emb, g_final, vocab, ids, B, N, hidden, logits_last, k_caches, v_caches,
                      N_max, workspace, workspace_bytes, stream) -> int:
     return _lib.rt_stack_prefill(C.byref(cfg), n_layers, layers, emb, g_final, vocab, ids, B, N, hidden, logits_last,
@@ -219,10 +228,10 @@ def rt_profile_read() -> Dict[str, Dict[str, float]]:
 def make_config(d_model: int, n_heads: int, d_ff: int, dtype: str = "bf16", sched: str = "tiled", leaf: int = 0,
                 norm_flags: int = RT_NORM_PRE | RT_NORM_QK, rms_eps: float = 1e-6,
                 softmax_scale: Optional[float] = None, residual_scale: float = 1.0, head_dim: int = 64,
-                recur_block: int = 0) -> RtConfig:
+                recur_block: int = 0, flags: int = 0) -> RtConfig:
     return RtConfig(d_model, n_heads, head_dim, d_ff, {"f32": RT_F32, "bf16": RT_BF16}[dtype],
                     {"tiled": RT_SCHED_TILED, "naive": RT_SCHED_NAIVE}[sched], leaf, norm_flags, rms_eps,
-                    (1.0 / math.sqrt(head_dim)) if softmax_scale is None else softmax_scale, residual_scale, recur_block)
+                    (1.0 / math.sqrt(head_dim)) if softmax_scale is None else softmax_scale, residual_scale, recur_block, flags)
 
 
 # ------------------------------------------------------------------ conveniences on torch tensors

@@ -79,7 +79,7 @@ def test_backward_from_the_prefill_outputs_and_determinism():
         assert rel_err(g1[n], g_ref[n]) <= TOL["f32"], n
 
 
-def test_backward_one_launch_per_step_form_agrees(monkeypatch):
+def test_backward_one_launch_per_step_form_agrees():
     # the same device code as one launch per step (the form for devices without cooperative launch)
     from paper_2604_21215_b200 import rt
     for dtype, B in (("f32", 3), ("bf16", 6)):
@@ -88,11 +88,10 @@ def test_backward_one_launch_per_step_form_agrees(monkeypatch):
         layer = rt.Layer(d, H, dff, dtype=dtype)
         layer.set_weights(lw)
         z, _, _ = layer.prefill(x)
-        monkeypatch.delenv("RT_BACKWARD_STEP_LAUNCHES", raising=False)
         dx1, g1 = layer.backward(x, z, dz)
-        monkeypatch.setenv("RT_BACKWARD_STEP_LAUNCHES", "1")
+        layer.cfg.flags = rt.RT_FLAG_BACKWARD_STEP_LAUNCHES
         dx2, g2 = layer.backward(x, z, dz)
-        monkeypatch.delenv("RT_BACKWARD_STEP_LAUNCHES")
+        layer.cfg.flags = 0
         # same arithmetic, separately compiled: equal up to the contraction of multiply-adds
         tol = 1e-5 if dtype == "f32" else 1e-3             # bf16: a last-bit change can flip an operand's bf16 rounding
         assert rel_err(dx2, dx1) <= tol and all(rel_err(g2[n], g1[n]) <= tol for n in g1)

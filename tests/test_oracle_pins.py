@@ -506,3 +506,96 @@ def test_blocked_recurrence_blocks_see_outputs_of_earlier_blocks_only():
     # of every block only when that block's predecessors agree -- here simply: first block of S = 4 equals S >= N on it
     zf, _, _ = layer_blockrec(cfg, w, x, 100)
     assert np.allclose(z0[:, :4], zf[:, :4], rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ pin: every norm flag and every gain, two positions by hand
+
+def _by_hand_two_positions(x, W, g, flags, alpha, s, eps, H):
+    """Sec. 2.2 for N = 2, written out with Python scalars only (math.sqrt / exp / erf, explicit loops): the
+    first position sees its temporary pair alone, the second one the persistent pair of the first (Eqs. 1-2;
+    with the flag of the RMSNorm-ablation appendix that pair comes from z_1 itself, without RMS) and its own
+    temporary pair.  Returns z_1, z_2, k_1, v_1 as lists."""
+    import math
+    d = len(x[0])
+    dh = d // H
+
+    def matvec(M, u):
+        return [sum(M[i][j] * u[j] for j in range(len(u))) for i in range(len(M))]
+
+    def rms_gain(u, gain):                      # u_j g_j / sqrt(mean(u^2) + eps)
+        ms = sum(t * t for t in u) / len(u)
+        return [u[j] * gain[j] / math.sqrt(ms + eps) for j in range(len(u))]
+
+    def pre(u, gain):
+        return rms_gain(u, gain) if flags & NORM_PRE else list(u)
+
+    def qk(u, gain):
+        if not flags & NORM_QK:
+            return list(u)
+        if flags & NORM_QK_FULL:
+            return rms_gain(u, gain)
+        out = []
+        for h in range(H):
+            out += rms_gain(u[h * dh:(h + 1) * dh], gain[h * dh:(h + 1) * dh])
+        return out
+
+    def gelu_s(t):
+        return 0.5 * t * (1.0 + math.erf(t / math.sqrt(2.0)))
+
+    def finish(xi, c):
+        a = matvec(W["w_o"], c)
+        hres = [xi[j] + alpha * a[j] for j in range(d)]
+        u = pre(hres, g["g_mlp"])
+        f = matvec(W["w_down"], [gelu_s(t) for t in matvec(W["w_up"], u)])
+        return [hres[j] + alpha * f[j] for j in range(d)]
+
+    # position 1
+    n1 = pre(x[0], g["g_attn"])
+    vt1 = matvec(W["w_v"], n1)
+    z1 = finish(x[0], vt1)                       # softmax over one logit: c_1 is the temporary value
+    r1 = list(z1) if flags & NORM_SKIP_Z else pre(z1, g["g_kv"])
+    k1 = qk(matvec(W["w_k"], r1), g["g_k"])
+    v1 = matvec(W["w_v"], r1)
+    # position 2
+    n2 = pre(x[1], g["g_attn"])
+    q2 = qk(matvec(W["w_q"], n2), g["g_q"])
+    kt2 = qk(matvec(W["w_k"], n2), g["g_k"])
+    vt2 = matvec(W["w_v"], n2)
+    c2 = []
+    for h in range(H):
+        sl = range(h * dh, (h + 1) * dh)
+        l1 = s * sum(q2[j] * k1[j] for j in sl)
+        l2 = s * sum(q2[j] * kt2[j] for j in sl)
+        m = max(l1, l2)
+        e1, e2 = math.exp(l1 - m), math.exp(l2 - m)
+        c2 += [(e1 * v1[j] + e2 * vt2[j]) / (e1 + e2) for j in sl]
+    z2 = finish(x[1], c2)
+    return z1, z2, k1, v1
+
+
+@pytest.mark.parametrize("flags", [0, NORM_PRE, NORM_QK, NORM_PRE | NORM_QK, NORM_PRE | NORM_QK | NORM_QK_FULL,
+                                   NORM_PRE | NORM_QK | NORM_SKIP_Z, NORM_PRE | NORM_SKIP_Z])
+def test_two_positions_by_hand_every_flag_and_gain(flags):
+    # Non-zero W_down and five distinct gains, so a swapped or dropped gain, a norm applied in the wrong place
+    # (before instead of after the projection, per head instead of full width, RMS(z) under the ablation flag)
+    # or a missing MLP term changes the result.
+    rng = np.random.default_rng(1234 + flags)
+    d, H, dff, alpha, s, eps = 4, 2, 3, 0.7, 0.6, 1e-5
+    W = {n: rng.standard_normal(shape) for n, shape in
+         (("w_q", (d, d)), ("w_k", (d, d)), ("w_v", (d, d)), ("w_o", (d, d)), ("w_up", (dff, d)), ("w_down", (d, dff)))}
+    g = {n: 1.0 + 0.3 * rng.standard_normal(d) for n in ("g_attn", "g_mlp", "g_kv", "g_q", "g_k")}
+    x = rng.standard_normal((2, d))
+    z1, z2, k1, v1 = _by_hand_two_positions([list(map(float, r)) for r in x],
+                                            {n: [list(map(float, r)) for r in M] for n, M in W.items()},
+                                            {n: list(map(float, v)) for n, v in g.items()}, flags, alpha, s, eps, H)
+    cfg = RTConfig(d, H, d // H, dff, norm_flags=flags, rms_eps=eps, softmax_scale=s, residual_scale=alpha)
+    w = RTWeights(**W, **g)
+    z, k, v = layer_seq(cfg, w, x[None])
+    assert np.allclose(z[0, 0], z1, rtol=1e-12, atol=1e-13) and np.allclose(z[0, 1], z2, rtol=1e-12, atol=1e-13)
+    assert np.allclose(k[0, 0], k1, rtol=1e-12, atol=1e-13) and np.allclose(v[0, 0], v1, rtol=1e-12, atol=1e-13)
+    # the flags and gains really matter on this input: the next flag set / a uniform gain gives another result
+    for other in ("g_mlp", "g_kv"):
+        w2 = RTWeights(**W, **{**g, other: np.ones(d)})
+        z_o, k_o, _ = layer_seq(cfg, w2, x[None])
+        if flags & NORM_PRE and not (other == "g_kv" and flags & NORM_SKIP_Z):
+            assert np.abs(z_o - z).max() + np.abs(k_o - k).max() > 1e-6, other
