@@ -18,7 +18,7 @@ constexpr int kSmallBatchMax = 64;      // above this the per-token chain runs a
 constexpr int kAutoLeaf = 64;
 
 struct WsLayout {
-  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, ll, ll_bytes, hid0, hid1,
+  size_t sync, q, kt, vt, n, st_o, st_m, st_l, ex_h, ex_g, ex_z, ex_k, ex_part, dec_part, ll, ll_bytes, hid0, hid1,
       blk_h, blk_u, blk_c, blk_g, total;
 };
 
@@ -64,6 +64,7 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_z = take((size_t)B * d * 4);
   L.ex_k = take((size_t)B * d * 4);
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
+  L.dec_part = take((size_t)B * H * kDecodeMaxChunks * 66 * 4);      // chunk partials of the decode-step attention
   // exchange buffers of the tensor-core leaf kernel: c, h, z as flag-carrying words (16 sequence slots each),
   // g as packed bf16 in fragment order (16 sequence slots), raw k|v as flag-carrying fp32 words
   L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)16 * (f / 4) + (size_t)B * 2 * d) * 8;
@@ -385,6 +386,26 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     return true;
   };
 
+  if (n_rows == 1 && pos0 > 0 && c->dtype == RT_BF16 &&
+      leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml)) {
+    // decode step on the fast path: the new position's query attends to the whole cache in chunks (Algorithm 2,
+    // partial states merged into the seeded state), then the tensor-core leaf kernel runs the one token step
+    DecodeAttnParams da;
+    memset(&da, 0, sizeof(da));
+    da.B = B; da.d = c->d_model; da.H = c->n_heads; da.scale_log2 = scale_log2; da.alibi = w->alibi_slopes;
+    da.q = ws + L.q; da.k_cache = k_cache; da.v_cache = v_cache; da.pos = pos0;
+    da.part = (float*)(ws + L.dec_part); da.st_o = pp.st_o; da.st_m = pp.st_m; da.st_l = pp.st_l;
+    {
+      ProfScope ps(s, kProfTile);
+      if (decode_attn_launch(da, s) != cudaSuccess) return RT_ERR_CUDA;
+    }
+    lp.t0 = pos0; lp.t1 = pos0 + 1; lp.attn_begin = pos0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
+    ProfScope ps(s, kProfLeaf);
+    if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return RT_ERR_CUDA;
+    ctx.seq_base += 1u;
+    ctx.bar_base += (unsigned)ml.grid;
+    return RT_OK;
+  }
   if (c->sched == RT_SCHED_NAIVE || pos0 > 0) {
     // token-sequential: every position reads its whole prefix from the cache
     return leaf(pos0, pos0 + n_rows, 0) ? RT_OK : RT_ERR_CUDA;

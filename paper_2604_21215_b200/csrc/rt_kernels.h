@@ -102,6 +102,22 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s);
 // one query row (position q0) per (sequence, head) against the pairs [k0, k1): the in-leaf step of wide batches
 cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s);
 
+// Attention of one decode step over the whole cache (bf16): query row q [B, d] of the new position against the pairs
+// [0, pos), chunk partials in `part` ([B*H][kDecodeMaxChunks][66] floats), merged into the seeded state row (st_*).
+constexpr int kDecodeMaxChunks = 64;
+struct DecodeAttnParams {
+  int B, d, H;
+  float scale_log2;
+  const float* alibi;                            // [H] slopes or NULL
+  const void* q;                                 // [B, d] bf16
+  const void *k_cache, *v_cache;                 // [N_max, B, d] bf16
+  int pos;                                       // positions in the cache
+  int chunk, n_chunks;                           // set by the launcher
+  float* part;
+  float *st_o, *st_m, *st_l;                     // state row of the new position: o [B, d], m, l [B, H]
+};
+cudaError_t decode_attn_launch(const DecodeAttnParams& p, cudaStream_t s);
+
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,
                          void* x, cudaStream_t s);

@@ -193,14 +193,14 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
 
   // queries and carried stats of the leaf (written by earlier kernels of this call)
   for (int i = 0; i < n; ++i) {
-    const size_t row = (size_t)(p.t0 + i) * B + b;
+    const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
     *reinterpret_cast<unsigned*>(qs + i * kQStride + 2 * lane) =
         *reinterpret_cast<const unsigned*>(q + row * d + h * kHeadDim + 2 * lane);
     os[i * kOStride + lane] = p.st_o[row * d + h * kHeadDim + lane];
     os[i * kOStride + lane + 32] = p.st_o[row * d + h * kHeadDim + lane + 32];
   }
   for (int i = lane; i < n; i += 32) {
-    const size_t row = (size_t)(p.t0 + i) * B + b;
+    const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
     ms[i] = p.st_m[row * H + h];
     ls[i] = p.st_l[row * H + h];
   }
@@ -399,8 +399,8 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
         const bool mine = warp < n_tiles && rl < nrows;
         unsigned xw0 = 0, xw1 = 0;
         if (ph == 0 && mine) {                                     // x_t for the residual, fetched before the wait
-          if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
-          if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)t * p.x_ts + d_lo + rl);
+          if (has0) xw0 = *reinterpret_cast<const unsigned*>(x + (size_t)g * p.x_bs + (size_t)(t - p.row_off) * p.x_ts + d_lo + rl);
+          if (has1) xw1 = *reinterpret_cast<const unsigned*>(x + (size_t)(g + 8) * p.x_bs + (size_t)(t - p.row_off) * p.x_ts + d_lo + rl);
         }
 
         // The loops below are written without branches around the loads and the products (indices
@@ -577,12 +577,12 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
           } else if (ph == 2) {                                     // z_t = h + alpha W_down g   (layer output)
             if (has0) {
               const unsigned zw = pack_bf2(hown[g * L.max_nd + rl] + p.alpha * y0, hown[g * L.max_nd + rl + 1] + p.alpha * y1);
-              *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              *reinterpret_cast<unsigned*>(z + (size_t)g * p.z_bs + (size_t)(t - p.row_off) * p.z_ts + d_lo + rl) = zw;
               st_relaxed_u64(ll_z + ll_word(g, d_lo + rl), zw, seq);
             }
             if (has1) {
               const unsigned zw = pack_bf2(hown[(g + 8) * L.max_nd + rl] + p.alpha * y2, hown[(g + 8) * L.max_nd + rl + 1] + p.alpha * y3);
-              *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)t * p.z_ts + d_lo + rl) = zw;
+              *reinterpret_cast<unsigned*>(z + (size_t)(g + 8) * p.z_bs + (size_t)(t - p.row_off) * p.z_ts + d_lo + rl) = zw;
               st_relaxed_u64(ll_z + ll_word(g + 8, d_lo + rl), zw, seq);
             }
           } else {                                                  // raw k_t, v_t from RMS(z_t): Eqs. (1)-(2) before qkRMS

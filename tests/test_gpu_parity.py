@@ -193,7 +193,8 @@ def test_c3_full_size_bf16_prefix_and_fixed_point():
 
 # ---------------------------------------------------------------- Algorithm 2 on its own (tensor-core and SIMT tile kernels)
 
-@pytest.mark.parametrize("dtype,nq,nk", [("bf16", 200, 128), ("bf16", 128, 320), ("bf16", 77, 96), ("f32", 40, 50)])
+@pytest.mark.parametrize("dtype,nq,nk", [("bf16", 200, 128), ("bf16", 128, 320), ("bf16", 77, 96), ("f32", 40, 50),
+                                          ("bf16", 130, 384), ("bf16", 256, 1024)])
 def test_update_tile_matches_algorithm_2(dtype, nq, nk):
     import torch
     from oracle import update_tile
