@@ -169,6 +169,11 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   pp.n = ws + L.n; pp.q = ws + L.q; pp.kt = ws + L.kt; pp.vt = ws + L.vt;
   pp.st_o = (float*)(ws + L.st_o); pp.st_m = (float*)(ws + L.st_m); pp.st_l = (float*)(ws + L.st_l);
   pp.sync = (SyncArea*)(ws + L.sync);
+  // decode step on the fast path (bf16 shapes the tensor-core leaf kernel takes): its attention warps seed the state
+  LeafMmaLaunch ml;
+  const bool dec_fast = n_rows == 1 && pos0 > 0 && c->dtype == RT_BF16 && c->recur_block <= 1 &&
+                        leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
+  if (dec_fast) pp.no_seed = 1;
   {
     ProfScope ps(s, kProfPrepass);
     if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
@@ -367,7 +372,6 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   };
 
   // bf16 tiled prefill takes the tensor-core leaf kernel when the shape fits it
-  LeafMmaLaunch ml;
   const bool use_mma = c->dtype == RT_BF16 && c->sched == RT_SCHED_TILED && pos0 == 0 &&
                        leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
   LeafMmaBuffers mb;
@@ -386,19 +390,20 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     return true;
   };
 
-  if (n_rows == 1 && pos0 > 0 && c->dtype == RT_BF16 &&
-      leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml)) {
-    // decode step on the fast path: the new position's query attends to the whole cache in chunks (Algorithm 2,
-    // partial states merged into the seeded state), then the tensor-core leaf kernel runs the one token step
+  if (dec_fast) {
+    // decode step on the fast path: the new position's query attends to the whole cache in chunks (Algorithm 2 per
+    // chunk), then the tensor-core leaf kernel merges the partial states and runs the one token step
     DecodeAttnParams da;
     memset(&da, 0, sizeof(da));
     da.B = B; da.d = c->d_model; da.H = c->n_heads; da.scale_log2 = scale_log2; da.alibi = w->alibi_slopes;
     da.q = ws + L.q; da.k_cache = k_cache; da.v_cache = v_cache; da.pos = pos0;
-    da.part = (float*)(ws + L.dec_part); da.st_o = pp.st_o; da.st_m = pp.st_m; da.st_l = pp.st_l;
+    da.part = (float*)(ws + L.dec_part);
+    int n_chunks = 0;
     {
       ProfScope ps(s, kProfTile);
-      if (decode_attn_launch(da, s) != cudaSuccess) return RT_ERR_CUDA;
+      if (decode_attn_launch(da, &n_chunks, s) != cudaSuccess) return RT_ERR_CUDA;
     }
+    lp.kt = ws + L.kt; lp.vt = ws + L.vt; lp.dec_part = da.part; lp.dec_chunks = n_chunks;
     lp.t0 = pos0; lp.t1 = pos0 + 1; lp.attn_begin = pos0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
     ProfScope ps(s, kProfLeaf);
     if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return RT_ERR_CUDA;

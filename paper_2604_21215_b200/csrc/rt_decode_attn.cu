@@ -1,13 +1,13 @@
 // Attention of one decode step over the whole cache (bf16 storage): the new position's query of every (sequence, head)
 // against the persistent pairs [0, pos), as Algorithm 2 applied to chunks of the cache whose partial states (m, l, o) are
-// merged, in chunk order, into the state the pre-pass seeded with the temporary pair.  A forward pass is a sequence of
-// such steps (Sec. 5); with a long cache the step is bound by streaming K and V once (2 pos B d e bytes per layer).
+// merged, in chunk order, into the state seeded with the temporary pair (by the attention warps of the leaf kernel that
+// runs the token step).  A forward pass is a sequence of such steps (Sec. 5); with a long cache the step is bound by
+// streaming K and V once (2 pos B d e bytes per layer).
 //
 // partial kernel: a CTA takes one chunk of positions of one sequence, a warp one head.  Scores: lane = key (the lane reads
 // its key's 128-byte row; the query sits in shared memory, read as broadcasts), no shuffles per product.  Values:
 // lane = two dimensions (the warp reads a V row as one coalesced 128-byte line, the key's weight comes by shuffle), so a
 // lane keeps two accumulators.  All 40 loads of a group of 32 keys are issued before the first product.
-// merge kernel: one warp per (sequence, head) folds the chunks' partial states into the running state in a fixed order.
 #include <cuda_bf16.h>
 
 #include "rt_kernels.h"
@@ -99,28 +99,6 @@ __global__ void __launch_bounds__(kDecWarps * 32, 2) decode_attn_partial_kernel(
   if (lane == 0) { out[64] = m_run; out[65] = l; }
 }
 
-__global__ void decode_attn_merge_kernel(const DecodeAttnParams p) {
-  const int lane = threadIdx.x & 31;
-  const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);    // (sequence, head)
-  if (u >= p.B * p.H) return;
-  const int b = u / p.H, h = u % p.H;
-  const size_t off = (size_t)b * p.d + h * kHeadDim + 2 * lane;
-  float m = p.st_m[u], l = p.st_l[u];                       // seeded with the temporary pair by the pre-pass
-  float2 o = *reinterpret_cast<const float2*>(p.st_o + off);
-  const float* part = p.part + (size_t)u * p.n_chunks * 66;
-  for (int c = 0; c < p.n_chunks; ++c) {
-    const float mc = part[c * 66 + 64], lc = part[c * 66 + 65];
-    const float2 oc = *reinterpret_cast<const float2*>(part + c * 66 + 2 * lane);
-    const float m_new = fmaxf(m, mc);
-    const float a = ex2f(m - m_new), bb = ex2f(mc - m_new);
-    o.x = o.x * a + oc.x * bb; o.y = o.y * a + oc.y * bb;
-    l = l * a + lc * bb;
-    m = m_new;
-  }
-  *reinterpret_cast<float2*>(p.st_o + off) = o;
-  if (lane == 0) { p.st_m[u] = m; p.st_l[u] = l; }
-}
-
 }  // namespace
 
 // Chunking of a cache of `pos` positions: whole groups of 32 keys, at most kDecodeMaxChunks chunks.
@@ -130,16 +108,15 @@ int decode_attn_chunk(int pos) {
   return chunk;
 }
 
-cudaError_t decode_attn_launch(const DecodeAttnParams& p0, cudaStream_t s) {
+cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, cudaStream_t s) {
   DecodeAttnParams p = p0;
+  *n_chunks = 0;
   if (p.pos <= 0) return cudaSuccess;
   p.chunk = decode_attn_chunk(p.pos);
   p.n_chunks = (p.pos + p.chunk - 1) / p.chunk;
+  *n_chunks = p.n_chunks;
   dim3 grid(p.n_chunks, p.B, ceil_div(p.H, kDecWarps));
   decode_attn_partial_kernel<<<grid, kDecWarps * 32, 0, s>>>(p);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  decode_attn_merge_kernel<<<ceil_div(p.B * p.H, 8), 256, 0, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -32,6 +32,12 @@ struct LeafParams {
   unsigned bar_base;                             // arrivals counted by earlier launches of the same call (bar_count is
                                                  // zeroed once per API call and only ever grows)
   unsigned seq_base;                             // token steps enqueued before this launch in the same call (flag values)
+  // decode step through the tensor-core leaf kernel (one position): the attention warps build the position's state
+  // themselves -- seeded with the temporary pair (kt, vt rows [B, d]), then the cache's chunk partials
+  // ([B*H][dec_chunks][66] floats: o, m, l) folded in chunk order; dec_chunks = 0 otherwise
+  const void *kt, *vt;
+  const float* dec_part;
+  int dec_chunks;
   int timers;                                    // 1: CTA 0 accumulates per-phase times in the sync area (costs a few per cent)
   SyncArea* sync;
 };
@@ -103,7 +109,8 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s);
 cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s);
 
 // Attention of one decode step over the whole cache (bf16): query row q [B, d] of the new position against the pairs
-// [0, pos), chunk partials in `part` ([B*H][kDecodeMaxChunks][66] floats), merged into the seeded state row (st_*).
+// [0, pos), chunk partials (o, m, l) in `part` ([B*H][n_chunks][66] floats, n_chunks <= kDecodeMaxChunks); the leaf
+// kernel's attention warps fold them, in chunk order, into the state seeded with the temporary pair.
 constexpr int kDecodeMaxChunks = 64;
 struct DecodeAttnParams {
   int B, d, H;
@@ -114,9 +121,9 @@ struct DecodeAttnParams {
   int pos;                                       // positions in the cache
   int chunk, n_chunks;                           // set by the launcher
   float* part;
-  float *st_o, *st_m, *st_l;                     // state row of the new position: o [B, d], m, l [B, H]
 };
-cudaError_t decode_attn_launch(const DecodeAttnParams& p, cudaStream_t s);
+// Launches the partial kernel; returns the number of chunks it wrote per (sequence, head) in *n_chunks.
+cudaError_t decode_attn_launch(const DecodeAttnParams& p, int* n_chunks, cudaStream_t s);
 
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,

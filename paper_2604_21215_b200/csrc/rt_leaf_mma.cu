@@ -191,6 +191,31 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   const bool qkn = (p.norm_flags & RT_NORM_QK) != 0;
   const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;     // ALiBi distances, in log2 units
 
+  if (p.dec_chunks > 0) {
+    // Decode step (one position): build the position's state here.  Seed: its temporary pair (logit s<q, k~>, l = 1,
+    // o = v~); then the partial states of the cache's chunks (Algorithm 2 per chunk, written by the decode attention
+    // kernel) are folded in chunk order.  Lane = dimensions 2 lane, 2 lane + 1.
+    const size_t roff = (size_t)b * d + h * kHeadDim + 2 * lane;
+    const unsigned qw = *reinterpret_cast<const unsigned*>(q + roff);
+    const unsigned kw = *reinterpret_cast<const unsigned*>(reinterpret_cast<const __nv_bfloat16*>(p.kt) + roff);
+    const unsigned vw = *reinterpret_cast<const unsigned*>(reinterpret_cast<const __nv_bfloat16*>(p.vt) + roff);
+    float m = warp_sum(bf_lo(qw) * bf_lo(kw) + bf_hi(qw) * bf_hi(kw)) * p.scale_log2, l = 1.0f;
+    float o0 = bf_lo(vw), o1 = bf_hi(vw);
+    const float* part = p.dec_part + (size_t)pair * p.dec_chunks * 66;
+#pragma unroll 4
+    for (int ch = 0; ch < p.dec_chunks; ++ch) {
+      const float mc = __ldcg(part + ch * 66 + 64), lc = __ldcg(part + ch * 66 + 65);
+      const float2 oc = __ldcg(reinterpret_cast<const float2*>(part + ch * 66 + 2 * lane));
+      const float m_new = fmaxf(m, mc);
+      const float a = exp2f(m - m_new), bb = exp2f(mc - m_new);
+      o0 = o0 * a + oc.x * bb; o1 = o1 * a + oc.y * bb;
+      l = l * a + lc * bb;
+      m = m_new;
+    }
+    *reinterpret_cast<unsigned*>(qs + 2 * lane) = qw;
+    os[2 * lane] = o0; os[2 * lane + 1] = o1;
+    if (lane == 0) { ms[0] = m; ls[0] = l; }
+  } else {
   // queries and carried stats of the leaf (written by earlier kernels of this call)
   for (int i = 0; i < n; ++i) {
     const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
@@ -203,6 +228,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
     ms[i] = p.st_m[row * H + h];
     ls[i] = p.st_l[row * H + h];
+  }
   }
   __syncwarp();
   const float gk0 = qkn ? gain_at(g_k, h * kHeadDim + 2 * lane) : 1.0f;
