@@ -64,7 +64,7 @@ WsLayout ws_layout(const rt_config* c, int B, int N) {
   L.ex_z = take((size_t)B * d * 4);
   L.ex_k = take((size_t)B * d * 4);
   L.ex_part = take((size_t)B * H * kMaxChunks * 68 * 4);
-  L.dec_part = take((size_t)B * H * kDecodeMaxChunks * 66 * 4);      // chunk partials of the decode-step attention
+  L.dec_part = take((size_t)B * H * kDecodeMaxRowChunks * 66 * 4);   // chunk partials of the decode-step attention
   // exchange buffers of the tensor-core leaf kernel: c, h, z as flag-carrying words (16 sequence slots each),
   // g as packed bf16 in fragment order (16 sequence slots), raw k|v as flag-carrying fp32 words
   L.ll_bytes = ((size_t)16 * 3 * (d / 2) + (size_t)16 * (f / 4) + (size_t)B * 2 * d) * 8;
@@ -398,12 +398,12 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     da.B = B; da.d = c->d_model; da.H = c->n_heads; da.scale_log2 = scale_log2; da.alibi = w->alibi_slopes;
     da.q = ws + L.q; da.k_cache = k_cache; da.v_cache = v_cache; da.pos = pos0;
     da.part = (float*)(ws + L.dec_part);
-    int n_chunks = 0;
+    int n_chunks = 0, chunk_stride = 0;
     {
       ProfScope ps(s, kProfTile);
-      if (decode_attn_launch(da, &n_chunks, s) != cudaSuccess) return RT_ERR_CUDA;
+      if (decode_attn_launch(da, &n_chunks, &chunk_stride, s) != cudaSuccess) return RT_ERR_CUDA;
     }
-    lp.kt = ws + L.kt; lp.vt = ws + L.vt; lp.dec_part = da.part; lp.dec_chunks = n_chunks;
+    lp.kt = ws + L.kt; lp.vt = ws + L.vt; lp.dec_part = da.part; lp.dec_chunks = n_chunks; lp.dec_stride = chunk_stride;
     lp.t0 = pos0; lp.t1 = pos0 + 1; lp.attn_begin = pos0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
     ProfScope ps(s, kProfLeaf);
     if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return RT_ERR_CUDA;

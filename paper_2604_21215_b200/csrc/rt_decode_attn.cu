@@ -17,6 +17,17 @@ namespace rt {
 namespace {
 
 constexpr int kDecWarps = 8;
+constexpr int kDecodeRowsFrom = 2048;            // cache lengths from which the lane = pair kernel streams the cache
+
+int sm_count_cached() {
+  thread_local int dev_cached = -1, sms = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev != dev_cached) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) { sms = n; dev_cached = dev; }
+  }
+  return sms;
+}
 
 __device__ __forceinline__ float bf_lo_f(unsigned u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi_f(unsigned u) { return __uint_as_float(u & 0xffff0000u); }
@@ -26,7 +37,7 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(kDecWarps * 32, 2) decode_attn_partial_kernel(const DecodeAttnParams p) {
+__global__ void __launch_bounds__(kDecWarps * 32) decode_attn_partial_kernel(const DecodeAttnParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = blockIdx.x, b = blockIdx.y, h = blockIdx.z * kDecWarps + warp;
   if (h >= p.H) return;
@@ -99,6 +110,119 @@ __global__ void __launch_bounds__(kDecWarps * 32, 2) decode_attn_partial_kernel(
   if (lane == 0) { out[64] = m_run; out[65] = l; }
 }
 
+
+// ---- long caches: lane = (sequence, head) ---------------------------------------------------------------------------
+// With many positions per chunk the cache is read fastest when consecutive lanes read consecutive segments of the same
+// position-major row: a pair of lanes owns a (sequence, head) pair, a warp reads 2 KB of a K row and 2 KB of a V row per
+// key, each lane pair runs Algorithm 2 for its pair key by key (one shuffle per key, no shared memory) with the next
+// key's rows in flight while it works on the current one.  A second kernel merges the chunk partials of a pair in parallel.
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ void load_half(const __nv_bfloat16* p, uint4 (&r)[4]) {
+  const uint4* q = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) r[i] = q[i];
+}
+__device__ __forceinline__ float dot_half(const uint4 (&k)[4], const uint4 (&q)[4]) {
+  float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    d0 = fmaf(bf_lo_f(k[i].x), bf_lo_f(q[i].x), d0); d1 = fmaf(bf_hi_f(k[i].x), bf_hi_f(q[i].x), d1);
+    d2 = fmaf(bf_lo_f(k[i].y), bf_lo_f(q[i].y), d2); d3 = fmaf(bf_hi_f(k[i].y), bf_hi_f(q[i].y), d3);
+    d0 = fmaf(bf_lo_f(k[i].z), bf_lo_f(q[i].z), d0); d1 = fmaf(bf_hi_f(k[i].z), bf_hi_f(q[i].z), d1);
+    d2 = fmaf(bf_lo_f(k[i].w), bf_lo_f(q[i].w), d2); d3 = fmaf(bf_hi_f(k[i].w), bf_hi_f(q[i].w), d3);
+  }
+  return (d0 + d1) + (d2 + d3);
+}
+
+// Two lanes per pair, 32 dimensions (64 bytes of a row) each: half the registers of one lane per pair, so two CTAs share
+// an SM and twice as many loads are in flight; the two halves of a logit meet through one shuffle per key.
+__global__ void __launch_bounds__(kRowThreads, 2) decode_attn_rows_kernel(const DecodeAttnParams p) {
+  const int seg = blockIdx.y * kRowThreads + threadIdx.x;     // 32-element segment of a row
+  const int u = seg >> 1, half = seg & 1;                     // (sequence, head) pair and which half of its 64 dimensions
+  const bool live = u < p.B * p.H;
+  const int uu = live ? u : 0;                                // lanes beyond the last pair shadow pair 0 (their shuffles are needed)
+  const int chunk = blockIdx.x;
+  const int j0 = chunk * p.chunk, j1 = min(j0 + p.chunk, p.pos);
+  float* out = p.part + ((size_t)uu * p.n_chunks + chunk) * 66;
+  const int h = uu % p.H;
+  const size_t row_stride = (size_t)p.B * p.d;
+  const __nv_bfloat16* kc = reinterpret_cast<const __nv_bfloat16*>(p.k_cache) + (size_t)uu * kHeadDim + half * 32;
+  const __nv_bfloat16* vc = reinterpret_cast<const __nv_bfloat16*>(p.v_cache) + (size_t)uu * kHeadDim + half * 32;
+  uint4 q[4];                                                  // this lane's half of the query as packed bf16
+  load_half(reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)uu * kHeadDim + half * 32, q);
+  const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
+  float o[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) o[e] = 0.f;
+  float m = -INFINITY, l = 0.f;
+  uint4 kr[4], vr[4], kn[4], vn[4];
+  if (j0 < j1) { load_half(kc + (size_t)j0 * row_stride, kr); load_half(vc + (size_t)j0 * row_stride, vr); }
+  for (int j = j0; j < j1; ++j) {
+    const int jn = j + 1 < j1 ? j + 1 : j;                    // next key's rows in flight meanwhile (the last one re-read)
+    load_half(kc + (size_t)jn * row_stride, kn);
+    load_half(vc + (size_t)jn * row_stride, vn);
+    float dt = dot_half(kr, q);
+    dt += __shfl_xor_sync(0xffffffffu, dt, 1);
+    const float s = dt * p.scale_log2 - slope_l2 * (float)(p.pos - j);
+    const float m_new = fmaxf(m, s);
+    const float corr = ex2f(m - m_new), w = ex2f(s - m_new);
+    l = l * corr + w;
+    m = m_new;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      o[8 * i] = fmaf(o[8 * i], corr, w * bf_lo_f(vr[i].x));         o[8 * i + 1] = fmaf(o[8 * i + 1], corr, w * bf_hi_f(vr[i].x));
+      o[8 * i + 2] = fmaf(o[8 * i + 2], corr, w * bf_lo_f(vr[i].y)); o[8 * i + 3] = fmaf(o[8 * i + 3], corr, w * bf_hi_f(vr[i].y));
+      o[8 * i + 4] = fmaf(o[8 * i + 4], corr, w * bf_lo_f(vr[i].z)); o[8 * i + 5] = fmaf(o[8 * i + 5], corr, w * bf_hi_f(vr[i].z));
+      o[8 * i + 6] = fmaf(o[8 * i + 6], corr, w * bf_lo_f(vr[i].w)); o[8 * i + 7] = fmaf(o[8 * i + 7], corr, w * bf_hi_f(vr[i].w));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { kr[i] = kn[i]; vr[i] = vn[i]; }
+  }
+  if (!live) return;
+#pragma unroll
+  for (int e = 0; e < 32; e += 2) *reinterpret_cast<float2*>(out + half * 32 + e) = make_float2(o[e], o[e + 1]);
+  if (half == 0) { out[64] = m; out[65] = l; }
+}
+
+// Merges the n_chunks partial states of every pair into ONE partial state (written over the pair's first slot): a CTA
+// per pair, lanes over chunks for the maximum and the weights, then lanes over the 64 dimensions with the chunks
+// strided over the warps, combined through shared memory in warp order (a fixed order: bit-reproducible).
+__global__ void __launch_bounds__(256) decode_attn_merge_kernel(const DecodeAttnParams p) {
+  __shared__ float s_w[kDecodeMaxRowChunks];
+  __shared__ float s_red[8][68];
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float* part = p.part + (size_t)u * p.n_chunks * 66;
+  float mx = -INFINITY;
+  for (int c = tid; c < p.n_chunks; c += 256) mx = fmaxf(mx, part[c * 66 + 64]);
+  mx = warp_max(mx);
+  if (lane == 0) s_red[warp][0] = mx;
+  __syncthreads();
+  float M = s_red[0][0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) M = fmaxf(M, s_red[w][0]);
+  __syncthreads();
+  for (int c = tid; c < p.n_chunks; c += 256) s_w[c] = ex2f(part[c * 66 + 64] - M);
+  __syncthreads();
+  float o0 = 0.f, o1 = 0.f, lsum = 0.f;
+  for (int c = warp; c < p.n_chunks; c += 8) {                // lane = dimensions 2 lane, 2 lane + 1
+    const float w = s_w[c];
+    const float2 oc = *reinterpret_cast<const float2*>(part + c * 66 + 2 * lane);
+    o0 = fmaf(w, oc.x, o0); o1 = fmaf(w, oc.y, o1);
+    if (lane == 0) lsum = fmaf(w, part[c * 66 + 65], lsum);
+  }
+  s_red[warp][2 * lane] = o0; s_red[warp][2 * lane + 1] = o1;
+  if (lane == 0) s_red[warp][64] = lsum;
+  __syncthreads();
+  if (warp == 0) {
+    float a0 = 0.f, a1 = 0.f, ll = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { a0 += s_red[w][2 * lane]; a1 += s_red[w][2 * lane + 1]; ll += s_red[w][64]; }
+    *reinterpret_cast<float2*>(part + 2 * lane) = make_float2(a0, a1);
+    if (lane == 0) { part[64] = M; part[65] = ll; }
+  }
+}
+
 }  // namespace
 
 // Chunking of a cache of `pos` positions: whole groups of 32 keys, at most kDecodeMaxChunks chunks.
@@ -108,13 +232,28 @@ int decode_attn_chunk(int pos) {
   return chunk;
 }
 
-cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, cudaStream_t s) {
+cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, int* chunk_stride, cudaStream_t s) {
   DecodeAttnParams p = p0;
-  *n_chunks = 0;
+  *n_chunks = 0; *chunk_stride = 0;
   if (p.pos <= 0) return cudaSuccess;
+  if (p.pos >= kDecodeRowsFrom) {
+    // long cache: lane = pair, about two chunks per multiprocessor, then a parallel merge into one partial per pair
+    int target = 2 * sm_count_cached();
+    if (target > kDecodeMaxRowChunks) target = kDecodeMaxRowChunks;
+    p.chunk = (p.pos + target - 1) / target;
+    if (p.chunk < 8) p.chunk = 8;
+    p.n_chunks = (p.pos + p.chunk - 1) / p.chunk;
+    dim3 grid(p.n_chunks, ceil_div(2 * p.B * p.H, kRowThreads));
+    decode_attn_rows_kernel<<<grid, kRowThreads, 0, s>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    decode_attn_merge_kernel<<<p.B * p.H, 256, 0, s>>>(p);
+    *n_chunks = 1; *chunk_stride = p.n_chunks;                // the merged state sits in the pair's first slot
+    return cudaGetLastError();
+  }
   p.chunk = decode_attn_chunk(p.pos);
   p.n_chunks = (p.pos + p.chunk - 1) / p.chunk;
-  *n_chunks = p.n_chunks;
+  *n_chunks = p.n_chunks; *chunk_stride = p.n_chunks;
   dim3 grid(p.n_chunks, p.B, ceil_div(p.H, kDecWarps));
   decode_attn_partial_kernel<<<grid, kDecWarps * 32, 0, s>>>(p);
   return cudaGetLastError();

@@ -37,7 +37,7 @@ struct LeafParams {
   // ([B*H][dec_chunks][66] floats: o, m, l) folded in chunk order; dec_chunks = 0 otherwise
   const void *kt, *vt;
   const float* dec_part;
-  int dec_chunks;
+  int dec_chunks, dec_stride;
   int timers;                                    // 1: CTA 0 accumulates per-phase times in the sync area (costs a few per cent)
   SyncArea* sync;
 };
@@ -112,6 +112,7 @@ cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s);
 // [0, pos), chunk partials (o, m, l) in `part` ([B*H][n_chunks][66] floats, n_chunks <= kDecodeMaxChunks); the leaf
 // kernel's attention warps fold them, in chunk order, into the state seeded with the temporary pair.
 constexpr int kDecodeMaxChunks = 64;
+constexpr int kDecodeMaxRowChunks = 320;         // chunks of the long-cache kernel (its partials are merged to one per pair)
 struct DecodeAttnParams {
   int B, d, H;
   float scale_log2;
@@ -122,8 +123,9 @@ struct DecodeAttnParams {
   int chunk, n_chunks;                           // set by the launcher
   float* part;
 };
-// Launches the partial kernel; returns the number of chunks it wrote per (sequence, head) in *n_chunks.
-cudaError_t decode_attn_launch(const DecodeAttnParams& p, int* n_chunks, cudaStream_t s);
+// Launches the partial kernel(s); *n_chunks = partial states per (sequence, head) left for the leaf kernel to fold in,
+// *chunk_stride = slots per pair in `part` (the leaf kernel reads slots 0 .. n_chunks-1 of pair u at u * chunk_stride).
+cudaError_t decode_attn_launch(const DecodeAttnParams& p, int* n_chunks, int* chunk_stride, cudaStream_t s);
 
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,

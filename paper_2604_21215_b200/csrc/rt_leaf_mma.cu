@@ -201,7 +201,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     const unsigned vw = *reinterpret_cast<const unsigned*>(reinterpret_cast<const __nv_bfloat16*>(p.vt) + roff);
     float m = warp_sum(bf_lo(qw) * bf_lo(kw) + bf_hi(qw) * bf_hi(kw)) * p.scale_log2, l = 1.0f;
     float o0 = bf_lo(vw), o1 = bf_hi(vw);
-    const float* part = p.dec_part + (size_t)pair * p.dec_chunks * 66;
+    const float* part = p.dec_part + (size_t)pair * p.dec_stride * 66;
 #pragma unroll 4
     for (int ch = 0; ch < p.dec_chunks; ++ch) {
       const float mc = __ldcg(part + ch * 66 + 64), lc = __ldcg(part + ch * 66 + 65);

@@ -449,3 +449,30 @@ def test_blocked_recurrence_stack_matches_oracle():
     st.set_weights(data["layers"], data["emb"])
     hid, logits = st.prefill(data["ids"])
     assert rel_err(hid, x) <= TOL["f32"] and rel_err(logits, logits_ref) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("alibi", [False, True])
+def test_decode_over_a_long_cache_matches_oracle(alibi):
+    # From 2048 cached positions on the decode step streams the cache with one lane per (sequence, head) and merges
+    # the chunk partials in a second kernel; two steps after a prefill of 2200 positions against the oracle.
+    from oracle import RTConfig, RTWeights, layer_seq
+    from parity_metrics import check_tensor
+    from paper_2604_21215_b200 import inputs, rt
+    d, H, dff, B, N = 128, 2, 256, 3, 2200
+    wl = inputs.Workload("longdec", 1, B, N + 2, d, H, dff, "bf16")
+    data = inputs.make_inputs(wl, seed=77)
+    lw = data["layers"][0]
+    slopes = [2.0 ** (-8.0 * (h + 1) / H) for h in range(H)] if alibi else None
+    ref = layer_seq(RTConfig(d, H, 64, dff, alibi_slopes=slopes), RTWeights(**lw), data["x"])
+    lw_gpu = dict(lw, alibi_slopes=slopes) if alibi else lw
+    layer = rt.Layer(d, H, dff, dtype="bf16")
+    layer.set_weights(lw_gpu)
+    layer.prefill(data["x"][:, :N], N_max=N + 2)
+    for step in range(2):
+        zn = layer.decode(data["x"][:, N + step], N + step)
+        check_tensor(f"long-cache decode step {step}", "z", zn, ref[0][:, N + step], TOL["bf16"], curve=False)
+    import torch
+    k = layer.k_cache.permute(1, 0, 2).to(torch.float64).cpu().numpy()
+    v = layer.v_cache.permute(1, 0, 2).to(torch.float64).cpu().numpy()
+    check_tensor("long-cache decode", "k", k, ref[1], TOL["bf16"])
+    check_tensor("long-cache decode", "v", v, ref[2], TOL["bf16"])
