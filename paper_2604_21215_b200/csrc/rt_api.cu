@@ -173,8 +173,18 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   LeafMmaLaunch ml;
   const bool dec_fast = n_rows == 1 && pos0 > 0 && c->dtype == RT_BF16 && c->recur_block <= 1 &&
                         leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
-  if (dec_fast) pp.no_seed = 1;
-  {
+  if (dec_fast && (size_t)16 * (c->d_model + 16) * 2 <= 190 * 1024) {
+    // the decode step's pre-pass in one launch (the leaf kernel's attention warps seed the state)
+    DecodePrepassParams dp;
+    memset(&dp, 0, sizeof(dp));
+    dp.B = B; dp.d = c->d_model; dp.H = c->n_heads; dp.norm_flags = c->norm_flags; dp.eps = c->rms_eps;
+    dp.x = x; dp.x_bs = x_bs;
+    dp.w_q = w->w_q; dp.w_k = w->w_k; dp.w_v = w->w_v; dp.g_attn = w->g_attn; dp.g_q = w->g_q; dp.g_k = w->g_k;
+    dp.q = pp.q; dp.kt = pp.kt; dp.vt = pp.vt;
+    ProfScope ps(s, kProfPrepass);
+    if (decode_prepass_launch(dp, s) != cudaSuccess) return RT_ERR_CUDA;
+  } else {
+    if (dec_fast) pp.no_seed = 1;
     ProfScope ps(s, kProfPrepass);
     if (prepass_launch(c->dtype, pp, s) != cudaSuccess) return RT_ERR_CUDA;
   }

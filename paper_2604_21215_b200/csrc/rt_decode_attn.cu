@@ -223,6 +223,108 @@ __global__ void __launch_bounds__(256) decode_attn_merge_kernel(const DecodeAttn
   }
 }
 
+
+// ---- pre-pass of a decode step in one launch -------------------------------------------------------------------------
+// The one new row per sequence: n = RMS(x), q = qkRMS(W_q n), k~ = qkRMS(W_k n), v~ = W_v n (first display of Sec. 2.2).
+// A CTA owns one head of one of the three projections (64 output columns); every CTA first normalises the B <= 16 rows
+// into shared memory (they are small), then its 8 warps take 8 columns each and run the product as m16n8k16 MMAs with
+// the sequences as rows, weights read straight from global memory (each weight is used once), and the head's
+// normalisation is finished through shared memory.
+constexpr int kPreThreads = 256;
+
+__device__ __forceinline__ void mma_16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// a weight word that is used once: asm, so that a run of these stays a run of loads in flight
+__device__ __forceinline__ uint2 ldg_stream_v2(const void* p) {
+  uint2 w;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w.x), "=r"(w.y) : "l"(p));
+  return w;
+}
+__device__ __forceinline__ unsigned pack2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const unsigned*>(&v);
+}
+
+__global__ void __launch_bounds__(kPreThreads) decode_prepass_kernel(const DecodePrepassParams p) {
+  extern __shared__ __align__(16) unsigned char dsm[];
+  const int d = p.d, stride = d + 16;                          // row stride in elements: 8-byte fragment loads without conflicts
+  __nv_bfloat16* n_s = reinterpret_cast<__nv_bfloat16*>(dsm);                   // [16][d + 16]
+  float* ssq_s = reinterpret_cast<float*>(dsm + (size_t)16 * stride * 2);       // [8 warps][16 sequences]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool pre = (p.norm_flags & RT_NORM_PRE) != 0, qkn = (p.norm_flags & RT_NORM_QK) != 0;
+  const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(p.x);
+  const __nv_bfloat16* g_attn = reinterpret_cast<const __nv_bfloat16*>(p.g_attn);
+  // ---- n = RMS_g(x) for the B rows (two per warp), rounded to the storage type; rows beyond B are zero ----
+  for (int b = warp * 2; b < warp * 2 + 2; ++b) {
+    unsigned* dst = reinterpret_cast<unsigned*>(n_s + (size_t)b * stride);
+    if (b >= p.B) {
+      for (int k = lane; k < d / 2; k += 32) dst[k] = 0u;
+      continue;
+    }
+    const unsigned* xr = reinterpret_cast<const unsigned*>(x + (size_t)b * p.x_bs);
+    float ss = 0.f;
+    for (int k = lane; k < d / 2; k += 32) { const unsigned w = xr[k]; ss += bf_lo_f(w) * bf_lo_f(w) + bf_hi_f(w) * bf_hi_f(w); }
+    ss = warp_sum(ss);
+    const float rs = pre ? rsqrtf(ss / (float)d + p.eps) : 1.0f;
+    for (int k = lane; k < d / 2; k += 32) {
+      const unsigned w = xr[k];
+      const float g0 = (pre && g_attn) ? __bfloat162float(g_attn[2 * k]) : 1.0f, g1 = (pre && g_attn) ? __bfloat162float(g_attn[2 * k + 1]) : 1.0f;
+      dst[k] = pack2(bf_lo_f(w) * rs * g0, bf_hi_f(w) * rs * g1);
+    }
+  }
+  __syncthreads();
+  // ---- this warp's 8 columns of the head: sequences as MMA rows, this thread reads weight row g at k = 4c ----
+  const int which = blockIdx.x / p.H, h = blockIdx.x % p.H;    // 0: q, 1: k~, 2: v~
+  const __nv_bfloat16* W = reinterpret_cast<const __nv_bfloat16*>(which == 0 ? p.w_q : (which == 1 ? p.w_k : p.w_v));
+  const int g = lane >> 2, c = lane & 3;
+  const int col0 = h * kHeadDim + warp * 8;
+  const unsigned char* wrow = reinterpret_cast<const unsigned char*>(W + (size_t)(col0 + g) * d + 4 * c);
+  const unsigned char* a_lo = reinterpret_cast<const unsigned char*>(n_s + (size_t)g * stride + 4 * c);
+  const unsigned char* a_hi = reinterpret_cast<const unsigned char*>(n_s + (size_t)(g + 8) * stride + 4 * c);
+  float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  const int n_ks = d / 16;
+  for (int ks0 = 0; ks0 < n_ks; ks0 += 16) {
+    uint2 bw[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) bw[i] = ldg_stream_v2(wrow + (size_t)(ks0 + i < n_ks ? ks0 + i : ks0) * 32);   // all 16 in flight
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (ks0 + i < n_ks) {
+        const size_t off = (size_t)(ks0 + i) * 32;
+        const uint2 lo = *reinterpret_cast<const uint2*>(a_lo + off), hi = *reinterpret_cast<const uint2*>(a_hi + off);
+        mma_16816(acc[i & 1], lo.x, hi.x, lo.y, hi.y, bw[i].x, bw[i].y);
+      }
+    }
+  }
+  float y[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) y[j] = acc[0][j] + acc[1][j];    // y0, y1: sequence g, columns col0 + 2c, + 1; y2, y3: sequence g + 8
+  // ---- qkRMS over the head's 64 columns (q and k~ only), gain, storage rounding ----
+  const bool norm = qkn && which < 2;
+  if (norm) {
+    float s_lo = y[0] * y[0] + y[1] * y[1], s_hi = y[2] * y[2] + y[3] * y[3];
+    s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 1); s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 2);
+    s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 1); s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 2);
+    if (c == 0) { ssq_s[warp * 16 + g] = s_lo; ssq_s[warp * 16 + 8 + g] = s_hi; }
+  }
+  __syncthreads();
+  float rs_lo = 1.0f, rs_hi = 1.0f;
+  if (norm) {
+    float t_lo = 0.f, t_hi = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { t_lo += ssq_s[w * 16 + g]; t_hi += ssq_s[w * 16 + 8 + g]; }
+    rs_lo = rsqrtf(t_lo * (1.0f / kHeadDim) + p.eps); rs_hi = rsqrtf(t_hi * (1.0f / kHeadDim) + p.eps);
+  }
+  const __nv_bfloat16* gain = reinterpret_cast<const __nv_bfloat16*>(which == 0 ? p.g_q : (which == 1 ? p.g_k : nullptr));
+  const int col = col0 + 2 * c;
+  const float ga = (norm && gain) ? __bfloat162float(gain[col]) : 1.0f, gb = (norm && gain) ? __bfloat162float(gain[col + 1]) : 1.0f;
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.q : (which == 1 ? p.kt : p.vt));
+  if (g < p.B) *reinterpret_cast<unsigned*>(out + (size_t)g * d + col) = pack2(y[0] * rs_lo * ga, y[1] * rs_lo * gb);
+  if (g + 8 < p.B) *reinterpret_cast<unsigned*>(out + (size_t)(g + 8) * d + col) = pack2(y[2] * rs_hi * ga, y[3] * rs_hi * gb);
+}
+
 }  // namespace
 
 // Chunking of a cache of `pos` positions: whole groups of 32 keys, at most kDecodeMaxChunks chunks.
@@ -256,6 +358,23 @@ cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, int* c
   *n_chunks = p.n_chunks; *chunk_stride = p.n_chunks;
   dim3 grid(p.n_chunks, p.B, ceil_div(p.H, kDecWarps));
   decode_attn_partial_kernel<<<grid, kDecWarps * 32, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t decode_prepass_launch(const DecodePrepassParams& p, cudaStream_t s) {
+  const size_t smem = (size_t)16 * (p.d + 16) * 2 + 8 * 16 * 4;
+  if (smem > 48 * 1024) {
+    thread_local int set_for = -1;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (set_for != dev) {
+      e = cudaFuncSetAttribute(decode_prepass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      set_for = dev;
+    }
+  }
+  decode_prepass_kernel<<<3 * p.H, kPreThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 

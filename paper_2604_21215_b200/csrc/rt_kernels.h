@@ -127,6 +127,18 @@ struct DecodeAttnParams {
 // *chunk_stride = slots per pair in `part` (the leaf kernel reads slots 0 .. n_chunks-1 of pair u at u * chunk_stride).
 cudaError_t decode_attn_launch(const DecodeAttnParams& p, int* n_chunks, int* chunk_stride, cudaStream_t s);
 
+// Pre-pass of a decode step (bf16, B <= 16, d a multiple of 16 with 16 (d + 16) 2 bytes of shared memory available):
+// n = RMS(x), q, k~, v~ of the one new row per sequence in one launch; x [B, d] with row stride x_bs, outputs [B, d].
+struct DecodePrepassParams {
+  int B, d, H;
+  int norm_flags;
+  float eps;
+  const void* x; long long x_bs;
+  const void *w_q, *w_k, *w_v, *g_attn, *g_q, *g_k;
+  void *q, *kt, *vt;
+};
+cudaError_t decode_prepass_launch(const DecodePrepassParams& p, cudaStream_t s);
+
 // Stack helpers.
 cudaError_t embed_launch(int dtype, const void* emb, const int32_t* ids, int B, int N, int d, int vocab,
                          void* x, cudaStream_t s);

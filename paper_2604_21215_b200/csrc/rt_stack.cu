@@ -71,11 +71,103 @@ __global__ void __launch_bounds__(256) head_kernel(const T* emb, const T* g_fina
   }
 }
 
+// bf16, B <= 16: the head as tensor-core mat-vecs.  The B normalised hidden rows sit in shared memory as TWO bf16 arrays
+// (value = hi + lo, so the fp32 activations lose nothing that matters), the sequences are the 16 rows of an m16n8k16 MMA
+// and 8 vocabulary rows its columns; a warp walks whole rows of E (each read once, 8 bytes per lane and k-step, 16 loads
+// in flight) and writes 8 x B logits.  The kernel is bound by streaming E once.
+__device__ __forceinline__ uint2 ldg_stream_v2(const void* p) {
+  uint2 w;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w.x), "=r"(w.y) : "l"(p));
+  return w;
+}
+__global__ void __launch_bounds__(256) head_mma_kernel(const __nv_bfloat16* emb, const __nv_bfloat16* g_final, const __nv_bfloat16* hidden,
+                                                       long long h_bs, int B, int d, int vocab, int norm_flags, float eps, float* logits) {
+  extern __shared__ __align__(16) unsigned char hsm[];
+  const int stride = d + 16;
+  __nv_bfloat16* hi_s = reinterpret_cast<__nv_bfloat16*>(hsm);                 // [16][d + 16]
+  __nv_bfloat16* lo_s = hi_s + (size_t)16 * stride;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool pre = (norm_flags & RT_NORM_PRE) != 0;
+  for (int b = warp * 2; b < warp * 2 + 2; ++b) {
+    __nv_bfloat16* hr_hi = hi_s + (size_t)b * stride;
+    __nv_bfloat16* hr_lo = lo_s + (size_t)b * stride;
+    if (b >= B) {
+      for (int k = lane; k < d; k += 32) { hr_hi[k] = __float2bfloat16_rn(0.f); hr_lo[k] = __float2bfloat16_rn(0.f); }
+      continue;
+    }
+    const __nv_bfloat16* hr = hidden + (size_t)b * h_bs;
+    float ss = 0.f;
+    for (int k = lane; k < d; k += 32) { const float v = __bfloat162float(hr[k]); ss += v * v; }
+    ss = warp_sum(ss);
+    const float rs = pre ? rsqrtf(ss / (float)d + eps) : 1.0f;
+    for (int k = lane; k < d; k += 32) {
+      const float v = __bfloat162float(hr[k]) * rs * (pre ? gain_at(g_final, k) : 1.0f);
+      const __nv_bfloat16 h = __float2bfloat16_rn(v);
+      hr_hi[k] = h;
+      hr_lo[k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+  }
+  __syncthreads();
+  const int g = lane >> 2, c = lane & 3;
+  const unsigned char* a_hi0 = reinterpret_cast<const unsigned char*>(hi_s + (size_t)g * stride + 4 * c);
+  const unsigned char* a_hi1 = reinterpret_cast<const unsigned char*>(hi_s + (size_t)(g + 8) * stride + 4 * c);
+  const unsigned char* a_lo0 = reinterpret_cast<const unsigned char*>(lo_s + (size_t)g * stride + 4 * c);
+  const unsigned char* a_lo1 = reinterpret_cast<const unsigned char*>(lo_s + (size_t)(g + 8) * stride + 4 * c);
+  const int n_ks = d / 16, n_groups = (vocab + 7) / 8;
+  for (int grp = blockIdx.x * 8 + warp; grp < n_groups; grp += gridDim.x * 8) {
+    const int v0 = grp * 8;
+    const int vr = v0 + g < vocab ? v0 + g : vocab - 1;                        // rows beyond the vocabulary repeat the last one (not stored)
+    const unsigned char* erow = reinterpret_cast<const unsigned char*>(emb + (size_t)vr * d + 4 * c);
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    for (int ks0 = 0; ks0 < n_ks; ks0 += 16) {
+      uint2 bw[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) bw[i] = ldg_stream_v2(erow + (size_t)(ks0 + i < n_ks ? ks0 + i : ks0) * 32);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        if (ks0 + i < n_ks) {
+          const size_t off = (size_t)(ks0 + i) * 32;
+          const uint2 h0 = *reinterpret_cast<const uint2*>(a_hi0 + off), h1 = *reinterpret_cast<const uint2*>(a_hi1 + off);
+          const uint2 l0 = *reinterpret_cast<const uint2*>(a_lo0 + off), l1 = *reinterpret_cast<const uint2*>(a_lo1 + off);
+          asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                       : "+f"(acc[0][0]), "+f"(acc[0][1]), "+f"(acc[0][2]), "+f"(acc[0][3])
+                       : "r"(h0.x), "r"(h1.x), "r"(h0.y), "r"(h1.y), "r"(bw[i].x), "r"(bw[i].y));
+          asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                       : "+f"(acc[1][0]), "+f"(acc[1][1]), "+f"(acc[1][2]), "+f"(acc[1][3])
+                       : "r"(l0.x), "r"(l1.x), "r"(l0.y), "r"(l1.y), "r"(bw[i].x), "r"(bw[i].y));
+        }
+      }
+    }
+    // acc[.][0], [1]: sequence g, vocabulary rows v0 + 2c, + 1; [2], [3]: sequence g + 8
+    const int v = v0 + 2 * c;
+    if (g < B) {
+      if (v < vocab) logits[(size_t)g * vocab + v] = acc[0][0] + acc[1][0];
+      if (v + 1 < vocab) logits[(size_t)g * vocab + v + 1] = acc[0][1] + acc[1][1];
+    }
+    if (g + 8 < B) {
+      if (v < vocab) logits[(size_t)(g + 8) * vocab + v] = acc[0][2] + acc[1][2];
+      if (v + 1 < vocab) logits[(size_t)(g + 8) * vocab + v + 1] = acc[0][3] + acc[1][3];
+    }
+  }
+}
+
 cudaError_t head_launch(int dtype, const void* emb, const void* g_final, const void* hidden, long long h_bs, int B,
                         int d, int vocab, int norm_flags, float eps, float* logits, cudaStream_t s) {
   const size_t smem = sizeof(float) * (size_t)B * d;
   const int blocks = ceil_div(vocab, 8) < 1184 ? ceil_div(vocab, 8) : 1184;
   cudaError_t e;
+  if (dtype == RT_BF16 && B <= 16 && d % 16 == 0 && (size_t)2 * 16 * (d + 16) * 2 <= 200 * 1024) {
+    const size_t sm2 = (size_t)2 * 16 * (d + 16) * 2;
+    e = cudaFuncSetAttribute(head_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int groups = ceil_div(vocab, 8);
+    const int nblk = ceil_div(groups, 8) < 2 * sms ? ceil_div(groups, 8) : 2 * sms;
+    head_mma_kernel<<<nblk, 256, sm2, s>>>((const __nv_bfloat16*)emb, (const __nv_bfloat16*)g_final, (const __nv_bfloat16*)hidden, h_bs,
+                                           B, d, vocab, norm_flags, eps, logits);
+    return cudaGetLastError();
+  }
   if (dtype == RT_BF16) {
     e = cudaFuncSetAttribute(head_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
