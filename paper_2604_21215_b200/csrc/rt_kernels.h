@@ -54,7 +54,7 @@ inline unsigned leaf_barrier_arrivals(int t0, int t1, int grid) { return (unsign
 cudaError_t wait_expiry_selftest_launch(SyncArea* sync, cudaStream_t s);
 
 // bf16 / tiled-schedule leaf kernel (tensor-core mat-vecs, flag-carrying exchange words).
-struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; };
+struct LeafMmaLaunch { int grid, block; size_t smem; int leaf; int q_smem; };
 struct LeafMmaBuffers { unsigned long long *ll_c, *ll_h, *ll_g, *ll_z, *ll_kv; };   // [16,d/2] words x3, packed bf16 [B,dff], [B,2d] words
 bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* out);
 // the same decision for a device with `sms` multiprocessors and `max_smem` bytes of shared memory per CTA (no CUDA call)

@@ -39,21 +39,24 @@ struct LeafMmaLayout {
   int max_nd, max_nf;          // weight rows per CTA (upper bounds): d-row matrices, W_up
   int stride_d, stride_f;      // shared-memory row strides in elements (K + 16)
   int lf;                      // leaf capacity of the attention state
+  int q_smem;                  // 1: the attention warps keep a copy of the leaf's queries in shared memory; 0: they read
+                               // them from global memory (what lets a 64-position leaf fit when an SM owns two pairs)
   size_t off_wo, off_wup, off_wdn, off_wk, off_wv, off_red, off_ssq, off_hown, off_attn, attn_bytes, total;
 };
 
-LeafMmaLayout leaf_mma_layout(int d, int dff, int grid, int lf, int slots) {
+LeafMmaLayout leaf_mma_layout(int d, int dff, int grid, int lf, int slots, int q_smem) {
   LeafMmaLayout L;
   L.max_nd = 2 * ceil_div(d / 2, grid);
   L.max_nf = 2 * ceil_div(dff / 2, grid);
   L.stride_d = d + 16;
   L.stride_f = dff + 16;
   L.lf = lf;
+  L.q_smem = q_smem;
   size_t o = 64;                                             // abort flag
   L.off_red = o;   o += sizeof(float4) * kMmaWarps * kNT * 32;
   L.off_ssq = o;   o += sizeof(float) * kMmaWarps * 16;
   L.off_hown = o;  o += align_up(sizeof(float) * 16 * (size_t)L.max_nd, 16);
-  L.attn_bytes = align_up((size_t)lf * kQStride * 2 + (size_t)lf * kOStride * 4 + (size_t)lf * 8 + 2 * kHeadDim * 4, 16);
+  L.attn_bytes = align_up((q_smem ? (size_t)lf * kQStride * 2 : 0) + (size_t)lf * kOStride * 4 + (size_t)lf * 8 + 2 * kHeadDim * 4, 16);
   L.off_attn = o;  o += L.attn_bytes * slots;
   o = align_up(o, 128);
   L.off_wo = o;    o += (size_t)L.max_nd * L.stride_d * 2;
@@ -171,7 +174,8 @@ __device__ __forceinline__ bool mma_grid_barrier(SyncArea* sync, volatile int* s
 }
 
 // ---- attention warp: one (sequence, head) pair for the whole leaf ----------------------------
-template <bool TIMERS>
+// QSMEM (compile-time, like the other switches: see the kernel): the leaf's queries are copied to shared memory.
+template <bool TIMERS, bool QSMEM>
 __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsigned char* smem_slot, int pair,
                                const unsigned long long* ll_kv, unsigned long long* ll_c) {
   const int lane = threadIdx.x & 31;
@@ -179,7 +183,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   const int b = pair / H, h = pair % H;
   const int n = p.t1 - p.t0;
   __nv_bfloat16* qs = reinterpret_cast<__nv_bfloat16*>(smem_slot);
-  float* os = reinterpret_cast<float*>(smem_slot + (size_t)L.lf * kQStride * 2);
+  float* os = reinterpret_cast<float*>(smem_slot + (QSMEM ? (size_t)L.lf * kQStride * 2 : 0));
   float* ms = os + (size_t)L.lf * kOStride;
   float* ls = ms + L.lf;
   float* kbuf = ls + L.lf;
@@ -212,15 +216,15 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
       l = l * a + lc * bb;
       m = m_new;
     }
-    *reinterpret_cast<unsigned*>(qs + 2 * lane) = qw;
     os[2 * lane] = o0; os[2 * lane + 1] = o1;
     if (lane == 0) { ms[0] = m; ls[0] = l; }
   } else {
   // queries and carried stats of the leaf (written by earlier kernels of this call)
   for (int i = 0; i < n; ++i) {
     const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
-    *reinterpret_cast<unsigned*>(qs + i * kQStride + 2 * lane) =
-        *reinterpret_cast<const unsigned*>(q + row * d + h * kHeadDim + 2 * lane);
+    if (QSMEM)
+      *reinterpret_cast<unsigned*>(qs + i * kQStride + 2 * lane) =
+          *reinterpret_cast<const unsigned*>(q + row * d + h * kHeadDim + 2 * lane);
     os[i * kOStride + lane] = p.st_o[row * d + h * kHeadDim + lane];
     os[i * kOStride + lane + 32] = p.st_o[row * d + h * kHeadDim + lane + 32];
   }
@@ -245,6 +249,9 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   unsigned long long a_work = 0, a_wait = 0, t_mark = timing ? globaltimer_ns() : 0ull;
   for (int j = 0; j < n; ++j) {
     const unsigned seq = p.seq_base + (unsigned)j + 1u;      // step that reveals position t0 + j
+    unsigned q_next = 0u;                                    // this lane's two values of query j + 1 (fetched ahead of the wait)
+    if (!QSMEM && j + 1 < n)
+      q_next = *reinterpret_cast<const unsigned*>(q + ((size_t)(p.t0 - p.row_off + j + 1) * B + b) * d + h * kHeadDim + 2 * lane);
     uint4 kw, vw;
     if (timing) { const unsigned long long now = globaltimer_ns(); a_work += now - t_mark; t_mark = now; }
     unsigned spins = 0;
@@ -275,7 +282,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     {
       // critical path: finish query j+1 and publish c_{j+1}
       const int i = j + 1;
-      const unsigned qw = *reinterpret_cast<const unsigned*>(qs + i * kQStride + 2 * lane);
+      const unsigned qw = QSMEM ? *reinterpret_cast<const unsigned*>(qs + i * kQStride + 2 * lane) : q_next;
       const float s = warp_sum(bf_lo(qw) * kf0 + bf_hi(qw) * kf1) * p.scale_log2 - slope_l2;      // distance (j+1) - j = 1
       const float m_old = ms[i], l_old = ls[i];
       const float m_new = fmaxf(m_old, s);
@@ -290,12 +297,24 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     vbuf[2 * lane] = vf0; vbuf[2 * lane + 1] = vf1;
     __syncwarp();
     for (int i = j + 2 + lane; i < n; i += 32) {
-      const __nv_bfloat16* qi = qs + i * kQStride;
       float s = 0.f;
+      if (QSMEM) {
+        const __nv_bfloat16* qi = qs + i * kQStride;
 #pragma unroll 8
-      for (int e = 0; e < kHeadDim; e += 2) {
-        const unsigned qw = *reinterpret_cast<const unsigned*>(qi + e);
-        s += bf_lo(qw) * kbuf[e] + bf_hi(qw) * kbuf[e + 1];
+        for (int e = 0; e < kHeadDim; e += 2) {
+          const unsigned qw = *reinterpret_cast<const unsigned*>(qi + e);
+          s += bf_lo(qw) * kbuf[e] + bf_hi(qw) * kbuf[e + 1];
+        }
+      } else {
+        const uint4* qg = reinterpret_cast<const uint4*>(q + ((size_t)(p.t0 - p.row_off + i) * B + b) * d + h * kHeadDim);
+        uint4 qv[8];
+#pragma unroll
+        for (int v = 0; v < 8; ++v) qv[v] = qg[v];
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          s += bf_lo(qv[v].x) * kbuf[8 * v] + bf_hi(qv[v].x) * kbuf[8 * v + 1] + bf_lo(qv[v].y) * kbuf[8 * v + 2] + bf_hi(qv[v].y) * kbuf[8 * v + 3] +
+               bf_lo(qv[v].z) * kbuf[8 * v + 4] + bf_hi(qv[v].z) * kbuf[8 * v + 5] + bf_lo(qv[v].w) * kbuf[8 * v + 6] + bf_hi(qv[v].w) * kbuf[8 * v + 7];
+        }
       }
       s = s * p.scale_log2 - slope_l2 * (float)(i - j);
       const float m_old = ms[i];
@@ -314,7 +333,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
 
 // TIMERS and GAINS are compile-time: the token step is a latency chain of code that runs once per token, and every
 // instruction and live register that is compiled in costs time even when its branch is not taken.
-template <int MB, bool TIMERS, bool GAINS>
+template <int MB, bool TIMERS, bool GAINS, bool QSMEM>
 __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const LeafParams p, const LeafMmaLayout L,
                                                                       unsigned long long* ll_c, unsigned long long* ll_h,
                                                                       unsigned long long* ll_g, unsigned long long* ll_z,
@@ -360,7 +379,7 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   if (warp >= kMmaWarps) {
     const int slot = warp - kMmaWarps;
     const int pair = cta + slot * G;
-    if (pair < B * H) attention_role<TIMERS>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
+    if (pair < B * H) attention_role<TIMERS, QSMEM>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
     return;
   }
 
@@ -644,10 +663,12 @@ bool leaf_mma_shape(int B, int d, int H, int dff, int want_leaf, int sms, size_t
   const int cands[3] = {64, 32, 16};
   for (int lf : cands) {
     if (want_leaf && lf != want_leaf) continue;
-    const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms));
-    if (L.total <= max_smem) {
-      out->grid = sms; out->block = kLeafMmaThreads; out->smem = L.total; out->leaf = lf;
-      return true;
+    for (int q_smem = 1; q_smem >= 0; --q_smem) {              // a longer leaf without the query copy beats a shorter one with it
+      const LeafMmaLayout L = leaf_mma_layout(d, dff, sms, lf, ceil_div(B * H, sms), q_smem);
+      if (L.total <= max_smem) {
+        out->grid = sms; out->block = kLeafMmaThreads; out->smem = L.total; out->leaf = lf; out->q_smem = q_smem;
+        return true;
+      }
     }
   }
   return false;
@@ -663,15 +684,19 @@ bool leaf_mma_plan(int B, int d, int H, int dff, int want_leaf, LeafMmaLaunch* o
 }
 
 cudaError_t leaf_mma_launch(const LeafParams& p, const LeafMmaLaunch& l, const LeafMmaBuffers& buf, cudaStream_t s) {
-  LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid));
+  LeafMmaLayout L = leaf_mma_layout(p.d, p.dff, l.grid, l.leaf, ceil_div(p.B * p.H, l.grid), l.q_smem);
   // compile-time variants: row blocks (B > 8), per-phase timers, RMS gains present
   const bool gains = p.g_mlp != nullptr || p.g_kv != nullptr;
-  auto pick = [&](auto mb) -> const void* {
+  auto pick2 = [&](auto mb, auto qs) -> const void* {
     constexpr int MB = decltype(mb)::value;
-    if (p.timers) return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, true>)
-                               : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, false>);
-    return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, true>)
-                 : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, false>);
+    constexpr bool QS = decltype(qs)::value;
+    if (p.timers) return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, true, QS>)
+                               : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, true, false, QS>);
+    return gains ? reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, true, QS>)
+                 : reinterpret_cast<const void*>(&leaf_mma_kernel<MB, false, false, QS>);
+  };
+  auto pick = [&](auto mb) -> const void* {
+    return l.q_smem ? pick2(mb, std::true_type{}) : pick2(mb, std::false_type{});
   };
   const void* fn = p.B > 8 ? pick(std::integral_constant<int, 2>{}) : pick(std::integral_constant<int, 1>{});
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.smem);

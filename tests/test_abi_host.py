@@ -99,14 +99,14 @@ def test_plan_counters_follow_the_n_log_n_model():
 
 def test_plan_counters_model_the_schedule_that_runs():
     # The counters follow the chain form a shape takes: wide batches use leaves of 32 positions, the tensor-core
-    # leaf kernel halves its leaf when an SM owns two (sequence, head) pairs, blocked recurrence tiles by blocks.
+    # leaf kernel keeps 64-position leaves also when an SM owns two (sequence, head) pairs, blocked recurrence tiles by blocks.
     N = 2048
     wide = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 32, N)
     assert wide["n_leaves"] == N // 32 and wide["n_tiles"] == len(rt.rt_plan_tiles(N, 32))
     c3 = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 8, N)
     assert c3["n_leaves"] == N // 64 and c3["n_tiles"] == len(rt.rt_plan_tiles(N, 64))
     c4 = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 16, N)
-    assert c4["n_leaves"] == N // 32 and c4["n_tiles"] == len(rt.rt_plan_tiles(N, 32))
+    assert c4["n_leaves"] == N // 64 and c4["n_tiles"] == len(rt.rt_plan_tiles(N, 64))
     blk = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16", recur_block=128), 8, N)
     assert blk["n_leaves"] == N // 128 and blk["n_tiles"] == N // 128 - 1
     f32 = rt.rt_plan_counters(rt.make_config(128, 2, 512, dtype="f32"), 4, 256)
