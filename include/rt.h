@@ -106,9 +106,11 @@ size_t rt_workspace_bytes(const rt_config *cfg, int32_t B, int32_t N, int32_t n_
 
 /* One RT layer over x[B,N,d] (Sec. 2.2; Algorithm 1).  Writes z[B,N,d] and rows [0,N) of
  * k_cache / v_cache [N_max,B,d] (Eqs. 1-2).  N_max >= N.
- * Batch sizes: B <= 16 in bf16 takes the persistent tensor-core leaf kernel; larger batches run each token step as
- * dense products over the batch (bf16 from B = 24, fp32 from B = 65: the regime of the paper's own experiments,
- * Sec. 6), tiled schedule only; in between, and for the naive schedule and decode up to B = 64, a generic kernel.
+ * Batch sizes (tiled schedule): B <= 16 in bf16 takes the persistent tensor-core leaf kernel; 17 <= B <= 48 in bf16
+ * runs as 2 or 3 slices of at most 16 sequences through that kernel, leaf by leaf (the sequences are independent),
+ * sharing the pre-pass and the cross tiles; larger batches run each token step as dense products over the batch
+ * (bf16 from B = 49, fp32 from B = 65: the regime of the paper's own experiments, Sec. 6).  fp32 up to B = 64, the
+ * naive schedule and decode up to B = 64 take a generic kernel.
  * The naive schedule and the decode entry points return RT_ERR_UNSUPPORTED for B > 64. */
 rt_status rt_layer_prefill(const rt_config *cfg, const rt_layer_weights *w,
                            const void *x, int32_t B, int32_t N,

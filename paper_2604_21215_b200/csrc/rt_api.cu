@@ -105,20 +105,29 @@ int leaf_size(const rt_config* c) { return c->leaf ? c->leaf : kAutoLeaf; }
 // Algorithm 1's tiles that goes with it.  Used by run_layer and by rt_plan_counters, so that the modelled schedule is
 // the one that runs (the tensor-core leaf kernel's leaf depends on the shared memory of the part; the planner assumes
 // a B200).
-enum ChainPath { kPathGeneric = 0, kPathMma = 1, kPathWide = 2, kPathBlocks = 3 };
-struct Schedule { ChainPath path; int leaf; };
+enum ChainPath { kPathGeneric = 0, kPathMma = 1, kPathWide = 2, kPathBlocks = 3, kPathMmaSplit = 4 };
+struct Schedule { ChainPath path; int leaf; int sub; };      // sub: sequences per launch of the tensor-core leaf kernel (kPathMmaSplit)
+constexpr int kMmaSplitMax = 48;         // largest batch that runs as slices of at most 16 sequences through the tensor-core leaf kernel
 Schedule effective_schedule(const rt_config* c, int B) {
-  if (c->recur_block > 1) return {kPathBlocks, c->recur_block};
+  if (c->recur_block > 1) return {kPathBlocks, c->recur_block, 0};
   if (c->sched == RT_SCHED_TILED) {
     // bf16 batches the persistent tensor-core leaf kernel does not take (B > 16) are faster as dense products from
     // about 24 sequences on (measured at d = 1024: 68 us per token step at B = 32 and 64 against 99 and 191 us for the
     // generic kernel); fp32 keeps the generic kernel up to its limit
-    if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : 32};
     LeafMmaLaunch ml;
+    if (c->dtype == RT_BF16 && B > 16 && B <= kMmaSplitMax) {
+      // Sequences are independent (Sec. 2.2 states the layer per sequence) and a token step of the tensor-core leaf
+      // kernel costs 10 - 14 us whatever its batch, against 53 us for the dense-product step at B = 32: up to 48
+      // sequences run as 2 or 3 slices of at most 16 through that kernel, leaf by leaf, and share the cross tiles.
+      const int n_sub = (B + 15) / 16, sub = (B + n_sub - 1) / n_sub;
+      if (leaf_mma_shape(sub, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
+        return {kPathMmaSplit, ml.leaf, sub};
+    }
+    if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : 32, 0};
     if (c->dtype == RT_BF16 && leaf_mma_shape(B, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
-      return {kPathMma, ml.leaf};
+      return {kPathMma, ml.leaf, B};
   }
-  return {kPathGeneric, leaf_size(c)};
+  return {kPathGeneric, leaf_size(c), 0};
 }
 
 // ---- optional per-kernel-class timing (rt_profile_enable / rt_profile_read) -----------------
@@ -382,8 +391,10 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
   };
 
   // bf16 tiled prefill takes the tensor-core leaf kernel when the shape fits it
+  // (batches of 17 .. 48 sequences: in slices of at most 16, see effective_schedule)
+  const int b_sub = (plan.path == kPathMmaSplit && pos0 == 0) ? plan.sub : B;
   const bool use_mma = c->dtype == RT_BF16 && c->sched == RT_SCHED_TILED && pos0 == 0 &&
-                       leaf_mma_plan(B, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
+                       leaf_mma_plan(b_sub, c->d_model, c->n_heads, c->d_ff, c->leaf, &ml);
   LeafMmaBuffers mb;
   {
     unsigned long long* w = (unsigned long long*)(ws + L.ll);
@@ -392,11 +403,17 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     mb.ll_kv = mb.ll_g + (size_t)16 * (c->d_ff / 4);
   }
   auto leaf_mma = [&](int t0, int t1) -> bool {
-    lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
     ProfScope ps(s, kProfLeaf);
-    if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return false;
-    ctx.seq_base += (unsigned)(t1 - t0);
-    ctx.bar_base += (unsigned)(t1 - t0) * (unsigned)ml.grid;      // one grid barrier per token step
+    const size_t e = esize_of(c->dtype);
+    for (int b0 = 0; b0 < B; b0 += b_sub) {
+      lp.B = B - b0 < b_sub ? B - b0 : b_sub; lp.Bs = B; lp.b0 = b0;
+      lp.x = (const unsigned char*)x + (size_t)b0 * x_bs * e;
+      lp.z = (unsigned char*)z + (size_t)b0 * z_bs * e;
+      lp.t0 = t0; lp.t1 = t1; lp.attn_begin = t0; lp.seq_base = ctx.seq_base; lp.bar_base = ctx.bar_base;
+      if (leaf_mma_launch(lp, ml, mb, s) != cudaSuccess) return false;
+      ctx.seq_base += (unsigned)(t1 - t0);
+      ctx.bar_base += (unsigned)(t1 - t0) * (unsigned)ml.grid;    // one grid barrier per token step
+    }
     return true;
   };
 
@@ -819,7 +836,7 @@ rt_status rt_plan_counters(const rt_config* cfg, int32_t B, int32_t N, int32_t n
       ++leaves;
       // persistent kernels stage their weight rows once per leaf launch; dense products (wide batches, block sweeps)
       // stream them once per position resp. once per block
-      rd += chain_w * (plan.path == kPathWide ? len : 1);
+      rd += chain_w * (plan.path == kPathWide ? len : (plan.path == kPathMmaSplit ? (b + plan.sub - 1) / plan.sub : 1));
       kv_leaf += 2 * b * d * e * (len * (len - 1) / 2);  // in-leaf pairs: written a few steps earlier, L2-resident
       fl_leaf += 4 * d * b * (len * (len - 1) / 2);
       if (e0 < n) {

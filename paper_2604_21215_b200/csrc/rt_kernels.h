@@ -24,6 +24,9 @@ struct LeafParams {
   float *st_o, *st_m, *st_l;                     // online-softmax state: o [rows,B,d], m,l [rows,B,H] (m in log2 units)
   int t0, t1;                                    // positions [t0, t1) are processed by this launch
   int row_off;
+  // tensor-core leaf kernel on a slice of the batch: the rows of q, the state and the caches are [row][Bs][...] and this
+  // launch's sequence b is column b0 + b of them (x and z are passed already offset); Bs = 0 means Bs = B, b0 = 0
+  int Bs, b0;
   int attn_begin;                                // first key position the in-launch attention covers (0 = whole prefix)
   float *ex_h, *ex_g, *ex_z, *ex_k;              // exchange vectors [B,d], [B,dff], [B,d], [B,d]
   float* ex_part;                                // partial attention states [B*H, max_chunks, 66]

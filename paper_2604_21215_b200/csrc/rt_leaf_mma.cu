@@ -181,6 +181,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   const int lane = threadIdx.x & 31;
   const int B = p.B, d = p.d, H = p.H;
   const int b = pair / H, h = pair % H;
+  const int Bs = p.Bs ? p.Bs : B, bc = p.b0 + b;               // row stride and column of this sequence in q / state / caches
   const int n = p.t1 - p.t0;
   __nv_bfloat16* qs = reinterpret_cast<__nv_bfloat16*>(smem_slot);
   float* os = reinterpret_cast<float*>(smem_slot + (QSMEM ? (size_t)L.lf * kQStride * 2 : 0));
@@ -221,7 +222,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
   } else {
   // queries and carried stats of the leaf (written by earlier kernels of this call)
   for (int i = 0; i < n; ++i) {
-    const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
+    const size_t row = (size_t)(p.t0 - p.row_off + i) * Bs + bc;
     if (QSMEM)
       *reinterpret_cast<unsigned*>(qs + i * kQStride + 2 * lane) =
           *reinterpret_cast<const unsigned*>(q + row * d + h * kHeadDim + 2 * lane);
@@ -229,7 +230,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     os[i * kOStride + lane + 32] = p.st_o[row * d + h * kHeadDim + lane + 32];
   }
   for (int i = lane; i < n; i += 32) {
-    const size_t row = (size_t)(p.t0 - p.row_off + i) * B + b;
+    const size_t row = (size_t)(p.t0 - p.row_off + i) * Bs + bc;
     ms[i] = p.st_m[row * H + h];
     ls[i] = p.st_l[row * H + h];
   }
@@ -251,7 +252,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     const unsigned seq = p.seq_base + (unsigned)j + 1u;      // step that reveals position t0 + j
     unsigned q_next = 0u;                                    // this lane's two values of query j + 1 (fetched ahead of the wait)
     if (!QSMEM && j + 1 < n)
-      q_next = *reinterpret_cast<const unsigned*>(q + ((size_t)(p.t0 - p.row_off + j + 1) * B + b) * d + h * kHeadDim + 2 * lane);
+      q_next = *reinterpret_cast<const unsigned*>(q + ((size_t)(p.t0 - p.row_off + j + 1) * Bs + bc) * d + h * kHeadDim + 2 * lane);
     uint4 kw, vw;
     if (timing) { const unsigned long long now = globaltimer_ns(); a_work += now - t_mark; t_mark = now; }
     unsigned spins = 0;
@@ -274,7 +275,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
     const float rs = qkn ? rsqrtf(ss * (1.0f / kHeadDim) + p.eps) : 1.0f;
     const unsigned kq = pack_bf2(k0 * rs * gk0, k1 * rs * gk1);
     const unsigned vq = pack_bf2(__uint_as_float(vw.x), __uint_as_float(vw.z));
-    const size_t crow = ((size_t)(p.t0 + j) * B + b) * d + h * kHeadDim + 2 * lane;
+    const size_t crow = ((size_t)(p.t0 + j) * Bs + bc) * d + h * kHeadDim + 2 * lane;
     *reinterpret_cast<unsigned*>(kc + crow) = kq;
     *reinterpret_cast<unsigned*>(vc + crow) = vq;
     if (j + 1 >= n) break;
@@ -306,7 +307,7 @@ __device__ void attention_role(const LeafParams& p, const LeafMmaLayout& L, unsi
           s += bf_lo(qw) * kbuf[e] + bf_hi(qw) * kbuf[e + 1];
         }
       } else {
-        const uint4* qg = reinterpret_cast<const uint4*>(q + ((size_t)(p.t0 - p.row_off + i) * B + b) * d + h * kHeadDim);
+        const uint4* qg = reinterpret_cast<const uint4*>(q + ((size_t)(p.t0 - p.row_off + i) * Bs + bc) * d + h * kHeadDim);
         uint4 qv[8];
 #pragma unroll
         for (int v = 0; v < 8; ++v) qv[v] = qg[v];

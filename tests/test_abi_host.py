@@ -101,8 +101,16 @@ def test_plan_counters_model_the_schedule_that_runs():
     # The counters follow the chain form a shape takes: wide batches use leaves of 32 positions, the tensor-core
     # leaf kernel keeps 64-position leaves also when an SM owns two (sequence, head) pairs, blocked recurrence tiles by blocks.
     N = 2048
-    wide = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 32, N)
+    wide = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 96, N)
     assert wide["n_leaves"] == N // 32 and wide["n_tiles"] == len(rt.rt_plan_tiles(N, 32))
+    # 17 .. 48 sequences run as slices of at most 16 through the tensor-core leaf kernel: its leaves, and the chain
+    # weights staged once per slice and leaf
+    split = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 32, N)
+    assert split["n_leaves"] == N // 64 and split["n_tiles"] == len(rt.rt_plan_tiles(N, 64))
+    one = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 16, N)
+    chain_w = (3 * 1024 * 1024 + 2 * 1024 * 4096) * 2
+    assert split["model_bytes_read"] - 2 * one["model_bytes_read"] == -(3 * 1024 * 1024 * 2)    # the pre-pass weights once, not twice
+    assert one["model_bytes_read"] > (N // 64) * chain_w
     c3 = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 8, N)
     assert c3["n_leaves"] == N // 64 and c3["n_tiles"] == len(rt.rt_plan_tiles(N, 64))
     c4 = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 16, N)

@@ -334,7 +334,8 @@ def test_alibi_stack_prefill_and_decode_match_oracle(dtype):
     ("bf16", 128, 2, 512, 96, 33, 16, False), ("bf16", 256, 4, 768, 40, 50, 0, False),
     ("bf16", 192, 3, 208, 30, 40, 16, True)])
 def test_wide_batch_prefill_matches_oracle(dtype, d, H, dff, B, N, leaf, alibi):
-    # B > 64 (bf16: B >= 24): every token step runs as dense products over the B rows (tensor cores for bf16)
+    # B > 64 (bf16: B > 48): every token step runs as dense products over the B rows (tensor cores for bf16); the bf16
+    # cases with B = 30 and 40 run as slices through the small-batch kernel
     from oracle import RTConfig, RTWeights, layer_seq
     from paper_2604_21215_b200 import inputs
     wl = inputs.Workload("wide", 1, B, N, d, H, dff, dtype)
@@ -347,6 +348,30 @@ def test_wide_batch_prefill_matches_oracle(dtype, d, H, dff, B, N, leaf, alibi):
     for name, g_, r_ in zip(("z", "k", "v"), got, ref):
         assert np.isfinite(g_).all(), name
         assert rel_err(g_, r_) <= TOL[dtype], (name, rel_err(g_, r_))
+
+
+@pytest.mark.parametrize("d,H,dff,B,N,leaf", [(256, 4, 1024, 17, 150, 16), (128, 2, 512, 33, 200, 0), (256, 4, 768, 48, 90, 32)])
+def test_batches_of_17_to_48_run_as_slices_of_the_small_batch_kernel(d, H, dff, B, N, leaf):
+    # bf16, tiled: the sequences are independent (Sec. 2.2), so such a batch runs as 2 or 3 slices of at most 16
+    # sequences through the tensor-core leaf kernel and shares the pre-pass and the cross tiles.  Checked against the
+    # oracle, and bit for bit against the same slices run as batches of their own.
+    from oracle import RTConfig, RTWeights, layer_seq
+    from paper_2604_21215_b200 import inputs
+    wl = inputs.Workload("split", 1, B, N, d, H, dff, "bf16")
+    data = inputs.make_inputs(wl, seed=8550 + B)
+    lw = data["layers"][0]
+    ref = layer_seq(RTConfig(d, H, 64, dff, residual_scale=0.8), RTWeights(**lw), data["x"])
+    layer = _layer(d, H, dff, "bf16", lw, leaf=leaf, residual_scale=0.8)
+    got = layer.prefill(data["x"])
+    for name, g_, r_ in zip(("z", "k", "v"), got, ref):
+        assert np.isfinite(g_).all(), name
+        assert rel_err(g_, r_) <= TOL["bf16"], (name, rel_err(g_, r_))
+    n_sub = (B + 15) // 16
+    sub = (B + n_sub - 1) // n_sub
+    for b0 in range(0, B, sub):
+        part = _layer(d, H, dff, "bf16", lw, leaf=leaf, residual_scale=0.8).prefill(data["x"][b0:b0 + sub])
+        for name, g_, p_ in zip(("z", "k", "v"), got, part):
+            assert np.array_equal(g_[b0:b0 + sub], p_), (name, b0)
 
 
 def test_wide_batch_unsupported_paths_say_so():
