@@ -111,9 +111,6 @@ constexpr int kMmaSplitMax = 48;         // largest batch that runs as slices of
 Schedule effective_schedule(const rt_config* c, int B) {
   if (c->recur_block > 1) return {kPathBlocks, c->recur_block, 0};
   if (c->sched == RT_SCHED_TILED) {
-    // bf16 batches the persistent tensor-core leaf kernel does not take (B > 16) are faster as dense products from
-    // about 24 sequences on (measured at d = 1024: 68 us per token step at B = 32 and 64 against 99 and 191 us for the
-    // generic kernel); fp32 keeps the generic kernel up to its limit
     LeafMmaLaunch ml;
     if (c->dtype == RT_BF16 && B > 16 && B <= kMmaSplitMax) {
       // Sequences are independent (Sec. 2.2 states the layer per sequence) and a token step of the tensor-core leaf
@@ -123,6 +120,9 @@ Schedule effective_schedule(const rt_config* c, int B) {
       if (leaf_mma_shape(sub, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
         return {kPathMmaSplit, ml.leaf, sub};
     }
+    // bf16 batches beyond that (or whose slices the tensor-core leaf kernel does not take) run as dense products from
+    // 24 sequences on, where they overtake the generic kernel (measured at d = 1024: 53 us per token step at B = 32
+    // against 99 us); fp32 keeps the generic kernel up to its limit
     if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : 32, 0};
     if (c->dtype == RT_BF16 && leaf_mma_shape(B, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
       return {kPathMma, ml.leaf, B};
