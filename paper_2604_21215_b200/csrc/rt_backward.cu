@@ -844,17 +844,6 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem, const T* 
   const T* gain = reinterpret_cast<const T*>(p.gain);
   const long long part_stride = (long long)p.B * d;
   __syncthreads();                                          // shared memory of the previous task is free
-#ifdef RT_BWD_TIMERS2
-  unsigned long long tb = globaltimer_ns();
-  auto bmark = [&](int slot) {
-    if (COOP && blockIdx.x == 0 && p.mode == RT_BWD_TIMERS2) {
-      __syncthreads();
-      if (threadIdx.x == 0) { const unsigned long long now = globaltimer_ns(); p.sync->phase_ns[slot] += now - tb; tb = now; }
-    }
-  };
-#else
-  auto bmark = [](int) {};
-#endif
 
   // ---- prologue: the input rows of this task's sequences, transposed into shared memory
   if (p.mode == RM_PAIR) {
@@ -976,7 +965,6 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem, const T* 
       if (writer && live) keep[e] = val;
     }
   }
-  bmark(0);
   __syncthreads();
 
   // ---- product: a warp's lanes = (32 / ncq) rows of W x ncq groups of 4 columns
@@ -1004,7 +992,6 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem, const T* 
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], wf[c], acc[r][c]);
   }
-  bmark(1);
 #pragma unroll
   for (int r = 0; r < RB; ++r)
 #pragma unroll
@@ -1032,7 +1019,6 @@ __device__ void rowmat_body(const RowmatParams& p, int t, float* smem, const T* 
       }
     }
   }
-  bmark(2);
 }
 
 template <typename T, int RB>
@@ -1105,17 +1091,6 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
     const int tasks = (Ncols / cols) * chunks * nsplit;
     for (int t = blockIdx.x; t < tasks; t += gridDim.x) rowmat_body<T, true, RB>(p, t, smem, slice[mode]);
   };
-#ifdef RT_BWD_TIMERS
-  unsigned long long t_mark = globaltimer_ns();
-  auto mark = [&](int slot) {
-    if (blockIdx.x == 0) {
-      __syncthreads();
-      if (threadIdx.x == 0) { const unsigned long long now = globaltimer_ns(); lp.sync->phase_ns[slot] += now - t_mark; t_mark = now; }
-    }
-  };
-#else
-  auto mark = [](int) {};
-#endif
   // The rows of the next position that nobody has touched since the sweep (dz, z, h, k_raw, W_up u) would each cost a trip
   // to HBM in the middle of a step: the last CTA (never the busiest) asks L2 for them one position ahead.
   auto warm = [&](int pos) {
@@ -1143,27 +1118,17 @@ __global__ void __launch_bounds__(kRmThreads, 1) bwd_loop_kernel(RowmatParams p,
     p.i = i;
     warm(i - 1);
     phase(RM_PAIR, p.d, p.d, lp.Wk, lp.Wv, lp.g_k, 0, 1.f, lp.cols_pair, 2, 0);
-    mark(0);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    mark(1);
     phase(RM_DOWN, p.d, p.dff, lp.Wdn, nullptr, lp.g_kv, lp.z_norm, lp.alpha, lp.cols_down, 1, 2);
-    mark(2);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    mark(3);
     phase(RM_UP, p.dff, p.d, lp.Wup, nullptr, nullptr, 0, 1.f, lp.cols_up, lp.up_split, 0);
-    mark(4);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    mark(5);
     phase(RM_OUT, p.d, p.d, lp.Wo, nullptr, lp.g_mlp, lp.pre, lp.alpha, lp.cols_out, 1, lp.up_split);
-    mark(6);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    mark(7);
     const int tasks = (i - lp.s0 + 1) * a.B * a.H;
     for (int t = blockIdx.x * kRmWarps + warp; t < tasks; t += gridDim.x * kRmWarps)
       attn_self_task<true>(a, i, lp.s0 + t / (a.B * a.H), (t / a.H) % a.B, t % a.H, lane);
-    mark(8);
     if (!grid_barrier(lp.sync, target, gridDim.x, &s_flag)) return;
-    mark(9);
   }
 }
 

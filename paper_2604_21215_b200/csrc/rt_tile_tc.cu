@@ -9,7 +9,9 @@
 //   S       (warp 4) tcgen05.mma  S[128x64] = Q . K^T  into the S columns of TMEM
 //   softmax (warps 0-3, one thread per query row) tcgen05.ld of the row, block max,
 //           p = 2^(s - m), row sum; P goes back into TMEM as packed bf16 over the first half of
-//           the S columns it came from (tcgen05.st)
+//           the S columns it came from (tcgen05.st).  The special-function unit (16 exponentials
+//           per clock and SM) is the busiest unit of this loop at d_h = 64, so a quarter of the
+//           exponentials are computed on the FMA pipe instead (exp_half below)
 //   PV      (warp 4) tcgen05.mma  O[128x64] += P . V  (A from TMEM, B = V MN-major: V rows are
 //           keys), ACCUMULATING in the O columns of TMEM
 // The running output never visits registers inside the loop: O is seeded from the carried state
@@ -31,6 +33,55 @@ constexpr int kBK = 64;                // keys per block
 constexpr uint32_t kKVBytes = kBK * kHeadDim * 2;    // 8 KB
 constexpr uint32_t kQBytes = kBM * kHeadDim * 2;     // 16 KB
 constexpr float kLazyLog2 = 8.0f;      // the reference maximum may lag the true one by this much (log2 units)
+
+// Which pairs of a row's values (by pair index mod 8) take their exponentials from the FMA pipe: a quarter.  Measured on
+// the c3 shape at P = 2048 / 4096 (TF/s): none 581 / 703 (all on the special-function unit, scalar arithmetic),
+// 1/4 605 / 744, 3/8 594 / 720, 1/2 579 / 693.
+constexpr unsigned kEmuMask = 0x88u;
+// Packed fp32 pairs (f32x2 arithmetic of sm_100): one instruction works on both halves of a 64-bit register, which
+// halves the issue slots of the scale-and-subtract and of the row sum.
+__device__ __forceinline__ uint64_t pk2(uint32_t lo, uint32_t hi) { uint64_t r; asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "r"(lo), "r"(hi)); return r; }
+__device__ __forceinline__ uint64_t pk2f(float lo, float hi) { return pk2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void upk2(uint64_t v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0,%1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+
+// p = 2^(s * scale + neg_m) for the 16 pairs of `s`, packed bf16 into w, the pairs' sums added to sum2[0..1].
+// Pairs whose bit is set in kEmuMask (by pair index mod 8) take the exponential from the FMA pipe instead of the
+// special-function unit: x is split into an integer j (round to nearest through the 1.5 * 2^23 constant) and r in
+// [-0.5, 0.5], 2^r is a cubic (max. relative error 7.5e-5, far below the bf16 rounding of P), and j goes into the
+// exponent field by an integer add.  x is clamped at -125 so that the exponent field cannot wrap.
+__device__ __forceinline__ void exp_half(const uint32_t (&s)[32], float scale, float neg_m, uint32_t (&w)[16], uint64_t (&sum2)[2]) {
+  const uint64_t sc2 = pk2f(scale, scale), nm2 = pk2f(neg_m, neg_m);
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const uint64_t x2 = fma2(pk2(s[2 * j], s[2 * j + 1]), sc2, nm2);
+    uint32_t x0, x1, p0, p1;
+    upk2(x2, x0, x1);
+    if ((kEmuMask >> (j & 7)) & 1u) {
+      const uint64_t magic2 = pk2f(12582912.f, 12582912.f);
+      const uint64_t xc2 = pk2f(fmaxf(__uint_as_float(x0), -125.f), fmaxf(__uint_as_float(x1), -125.f));
+      const uint64_t t2 = add2(xc2, magic2);
+      const uint64_t r2 = sub2(xc2, sub2(t2, magic2));
+      uint64_t q2 = fma2(r2, pk2f(0.0551716685f, 0.0551716685f), pk2f(0.242611125f, 0.242611125f));
+      q2 = fma2(q2, r2, pk2f(0.693260968f, 0.693260968f));
+      q2 = fma2(q2, r2, pk2f(0.999928057f, 0.999928057f));
+      uint32_t q0, q1, t0, t1;
+      upk2(q2, q0, q1);
+      upk2(t2, t0, t1);
+      p0 = q0 + (t0 << 23);
+      p1 = q1 + (t1 << 23);
+    } else {
+      p0 = __float_as_uint(ex2(__uint_as_float(x0)));
+      p1 = __float_as_uint(ex2(__uint_as_float(x1)));
+    }
+    sum2[j & 1] = add2(sum2[j & 1], pk2(p0, p1));
+    const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(p0), __uint_as_float(p1));
+    w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+  }
+}
 
 struct TcCfg {
   static constexpr int stages = 2;
@@ -213,14 +264,14 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_wait_ld();
       adjust(s1, 32);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) mx4[j] = __uint_as_float(s1[j]);
+      for (int j = 0; j < 4; ++j) mx4[j] = fmaxf(__uint_as_float(s1[2 * j]), __uint_as_float(s1[2 * j + 1]));
 #pragma unroll
-      for (int i = 4; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(s1[i]));
+      for (int i = 4; i < 16; ++i) mx4[i & 3] = max3(mx4[i & 3], __uint_as_float(s1[2 * i]), __uint_as_float(s1[2 * i + 1]));
       tc_ld32(t_s, s0);
       tc_wait_ld();
       adjust(s0, 0);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(s0[i]));
+      for (int i = 0; i < 16; ++i) mx4[i & 3] = max3(mx4[i & 3], __uint_as_float(s0[2 * i]), __uint_as_float(s0[2 * i + 1]));
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
       if (ALIBI) mx += base_l2;
       m_true = fmaxf(m_true, mx);
@@ -229,31 +280,21 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const float corr = ex2(m_used - m_new);                  // 1 when the reference stays
       float neg_m = -m_new;
       if (ALIBI) neg_m += base_l2;
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint64_t sum2[2] = {0ull, 0ull};
       // p = 2^(s*scale - m) as packed bf16, written over the first 32 columns of the S buffer
       uint32_t w[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float p0 = ex2(fmaf(__uint_as_float(s0[2 * j]), p.scale_log2, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(s0[2 * j + 1]), p.scale_log2, neg_m));
-        sum4[j & 3] += p0 + p1;
-        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-        w[j] = *reinterpret_cast<const uint32_t*>(&pk);
-      }
+      exp_half(s0, p.scale_log2, neg_m, w, sum2);
       tc_ld32(t_s + 32u, s1);                                  // columns 32..63 are still the raw products
       tc_st16(t_s, w);
       tc_wait_ld();
       adjust(s1, 32);
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float p0 = ex2(fmaf(__uint_as_float(s1[2 * j]), p.scale_log2, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(s1[2 * j + 1]), p.scale_log2, neg_m));
-        sum4[j & 3] += p0 + p1;
-        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-        w[j] = *reinterpret_cast<const uint32_t*>(&pk);
-      }
+      exp_half(s1, p.scale_log2, neg_m, w, sum2);
       tc_st16(t_s + 16u, w);
-      l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      {
+        uint32_t a0, a1;
+        upk2(add2(sum2[0], sum2[1]), a0, a1);
+        l_run = l_run * corr + (__uint_as_float(a0) + __uint_as_float(a1));
+      }
       m_used = m_new;
       if (__any_sync(0xffffffffu, raise)) {
         // rare: rescale this warp's rows of O in place (O is quiescent: S_READY(kb) covers P.V(kb-1))

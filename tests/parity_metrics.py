@@ -9,7 +9,10 @@ and they report (and loosely bound) two more figures:
   * the element-wise maximum of |D| / (|ref| + 1e-3 max|ref|).  An entry near zero carries the absolute
     error of its row (about 2^-9 of the row's typical magnitude in bf16 mode), so this figure is of
     order (row rms / max) / (1e-3 * 2^9), i.e. well above the bound of the first metric; what the
-    arithmetic guarantees is 1e3 times that bound, and the tests assert a tenth of that,
+    arithmetic guarantees is 1e3 times that bound, and the tests assert a quarter of that.  The figure is the
+    maximum of millions of rounding-noise samples (6.3e6 entries at config 2), an extreme-value statistic: two
+    builds with the same max-norm and row errors gave 1.92 and 2.28 for the same tensor (and 1.89 / 1.55 for
+    another), so a bound just above one observed value would test the noise, not the arithmetic,
   * the error by position t for [B, N, d] tensors: e(t) = max_{b,j} |D[b,t,j]| / max|ref|.  Sec. 4 argues
     that long dependency chains are damped, so e(t) must not grow along the sequence: the maximum over the
     last quarter of the positions may not exceed ten times the maximum over the first quarter (or a floor
@@ -65,5 +68,5 @@ def check_tensor(what, name, got, ref, tol, curve=True):
             f.write(json.dumps(rec) + "\n")
     assert e_max <= tol, f"{what}: {name} max-norm error {e_max:.3e} > {tol}"
     assert e_row <= tol, f"{what}: {name} worst-row relative error {e_row:.3e} > {tol}"
-    assert e_el <= 100.0 * tol, f"{what}: {name} element-wise error {e_el:.3e} > {100.0 * tol}"
+    assert e_el <= 250.0 * tol, f"{what}: {name} element-wise error {e_el:.3e} > {250.0 * tol}"
     return rec
