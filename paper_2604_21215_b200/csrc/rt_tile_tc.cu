@@ -20,8 +20,9 @@
 // any reference value; the bound keeps p <= 256), and then the row's O and l are rescaled in place.
 // The state is renormalised to the true running maximum when it is written back, so the stored
 // triple is the one Algorithm 2 defines.
-// TMEM: S [0,64) O [64,128); 48 KB of shared memory and 80 registers per thread, so four CTAs share
-// an SM and their chains (softmax -> P.V -> S -> softmax) interleave on the tensor pipe.
+// TMEM: S [0,64) O [64,128); 48 KB of shared memory and 256 threads at 64 registers, so four CTAs share
+// an SM and their chains (softmax -> P.V -> S -> softmax) interleave on the tensor pipe; the threads form two
+// warpgroups (softmax; issuing warps plus two idle ones) so that registers can move between them.
 // Every mbarrier wait is bounded: on expiry the CTA records RT_ERR_TIMEOUT, stops issuing work,
 // waits (bounded) for its copies in flight, frees its TMEM and returns.
 #include "rt_kernels.h"
@@ -38,6 +39,7 @@ constexpr float kLazyLog2 = 8.0f;      // the reference maximum may lag the true
 // the c3 shape at P = 2048 / 4096 (TF/s): none 581 / 703 (all on the special-function unit, scalar arithmetic),
 // 1/4 605 / 744, 3/8 594 / 720, 1/2 579 / 693.
 constexpr unsigned kEmuMask = 0x88u;
+constexpr int kRegsSoftmax = 88, kRegsIssue = 40;      // registers per thread after the hand-over (setmaxnreg), see the kernel
 // Packed fp32 pairs (f32x2 arithmetic of sm_100): one instruction works on both halves of a 64-bit register, which
 // halves the issue slots of the scale-and-subtract and of the row sum.
 __device__ __forceinline__ uint64_t pk2(uint32_t lo, uint32_t hi) { uint64_t r; asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "r"(lo), "r"(hi)); return r; }
@@ -86,7 +88,7 @@ __device__ __forceinline__ void exp_half(const uint32_t (&s)[32], float scale, f
 struct TcCfg {
   static constexpr int stages = 2;
   static constexpr int ctas_per_sm = 4;
-  static constexpr int threads = 6 * 32;                 // 4 softmax warps + MMA warp + TMA warp
+  static constexpr int threads = 8 * 32;                 // warpgroup 0: 4 softmax warps; warpgroup 1: MMA warp, TMA warp, two idle warps
   static constexpr int tmem_cols = 128;
   // offsets from a 1024-byte aligned base
   static constexpr uint32_t q = 0;
@@ -100,7 +102,7 @@ struct TcCfg {
 enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = 2, BAR_Q_FULL = 4, BAR_S_READY = 5, BAR_P_READY = 6 };
 
 // ALIBI / CAUSAL are compile-time so that the plain kernel carries none of their registers or instructions
-// (it runs at 80 registers per thread, four CTAs per SM, and loses a fifth of its rate to a few spills).
+// (four CTAs per SM leave its softmax threads 88 registers, and it loses up to a fifth of its rate to a few spills).
 template <bool ALIBI, bool CAUSAL>
 __global__ void __launch_bounds__(TcCfg::threads, TcCfg::ctas_per_sm)
 tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -140,8 +142,16 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  // Registers move from the issuing warpgroup to the softmax warpgroup: the launch gives each of the 256 threads 64
+  // (four CTAs per SM), the issuing warps keep kRegsIssue and the softmax warps grow to kRegsSoftmax, where their loop
+  // runs without spills.  Measured (TF/s at P = 2048 / 4096): 88 + 40 628 / 769, 96 + 32 553 / 693, 104 + 24 517 / 654
+  // (the issuing threads then spill), against 601 / 740 for 192 threads at 80 registers.
 
-  if (warp == kTmaWarp) {
+  if (warp >= 6) {
+    // idle warps of the issuing warpgroup
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
+  } else if (warp == kTmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       const int k0 = p.k0 + shift();
@@ -170,6 +180,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     __syncwarp();
   } else if (warp == kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(kBK, false);
@@ -208,6 +219,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     __syncwarp();
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // ------------------------------ softmax warps: one thread per query row ------------------------------
     const int row = warp * 32 + lane;
     const int qi = qb + row;
@@ -258,7 +270,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       };
       // The row lives in registers half at a time (32 of its 64 values): the second half is read for the
       // maximum, dropped, and read again for the exponentials.  A TMEM load costs little; holding all 64
-      // values next to the packed P words would not fit the 80 registers four resident CTAs leave a thread.
+      // values next to the packed P words would not fit the 88 registers four resident CTAs leave a softmax thread.
       float mx4[4];                                            // four independent chains
       tc_ld32(t_s + 32u, s1);
       tc_wait_ld();
