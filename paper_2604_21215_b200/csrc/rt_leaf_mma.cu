@@ -19,6 +19,9 @@
 //     j+1 (the only one on the critical path) and publishes c_{j+1} = o/l, and only then folds
 //     the new pair into the later queries of the leaf, while the rest of the chip is busy with
 //     the mat-vecs of step j+1.  These warps also apply qkRMS to k_j and write the caches.
+//   * a CTA is 384 threads = three warpgroups (MMA warps 0-3, MMA warps 4-7, the attention warps plus two idle
+//     warps): once the weights are staged, setmaxnreg moves registers from the last group to the MMA warps, which
+//     then hold all of a phase's fragments (up to 64 loads in flight per thread) without spilling.
 #include <cuda_bf16.h>
 
 #include <type_traits>
@@ -30,7 +33,10 @@ namespace rt {
 constexpr int kMmaWarps = 8;
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kAttnSlots = 2;
-constexpr int kLeafMmaThreads = kMmaThreads + 32 * kAttnSlots;
+// Three warpgroups: MMA warps 0-3, MMA warps 4-7, and the two attention warps with two idle ones, so that registers can
+// move from the last group to the MMA warps after the weights are staged (setmaxnreg works on whole warpgroups).
+constexpr int kLeafMmaThreads = kMmaThreads + 128;
+constexpr int kRegsMma = 216, kRegsAttn = 72;           // 2 * 128 * 216 + 128 * 72 <= 65536
 constexpr int kNT = 4;                  // n-tiles (8 weight rows each) per pass
 constexpr int kQStride = kHeadDim + 2;  // bf16 elements per query row in shared memory
 constexpr int kOStride = kHeadDim + 1;  // floats per o row in shared memory
@@ -378,13 +384,15 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   __syncthreads();
 
   if (warp >= kMmaWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsAttn));
     const int slot = warp - kMmaWarps;
     const int pair = cta + slot * G;
-    if (pair < B * H) attention_role<TIMERS, QSMEM>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
+    if (slot < kAttnSlots && pair < B * H) attention_role<TIMERS, QSMEM>(p, L, smem + L.off_attn + (size_t)slot * L.attn_bytes, pair, ll_kv, ll_c);
     return;
   }
 
   // ------------------------------ MMA warps ------------------------------
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsMma));
   // The four mat-vec phases of a token step run through ONE inlined copy of the code below (a loop
   // over the phase index): the step executes once per token, so four straight-line copies would
   // only thrash the instruction cache, and calls through a real function would put the fragments
@@ -458,9 +466,9 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
         const unsigned keep0 = has0 ? 0xffffffffu : 0u, keep1 = has1 ? 0xffffffffu : 0u;
         if (ph == 2) {
           // W_down reads g as packed bf16 after the barrier: plain loads, and ALL of this warp's
-          // k-steps are in flight before the first product (two rounds when B > 8).  One tile per
+          // k-steps are in flight before the first product (at d_ff = 4096: 32 k-steps, 64 loads when B > 8).  One tile per
           // pass keeps this at 32 products; the two accumulators halve the dependent chain.
-          constexpr int KD = 32 / MB;
+          constexpr int KD = 32;
           float acc[2][4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) { acc[0][j] = acc[1][j] = 0.f; }
