@@ -38,6 +38,7 @@ __device__ __forceinline__ float ex2f(float x) {
 }
 
 __global__ void __launch_bounds__(kDecWarps * 32) decode_attn_partial_kernel(const DecodeAttnParams p) {
+  grid_dep_sync();                                           // the launches of a decode step are chained (programmatic dependent launches)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = blockIdx.x, b = blockIdx.y, h = blockIdx.z * kDecWarps + warp;
   if (h >= p.H) return;
@@ -138,6 +139,7 @@ __device__ __forceinline__ float dot_half(const uint4 (&k)[4], const uint4 (&q)[
 // Two lanes per pair, 32 dimensions (64 bytes of a row) each: half the registers of one lane per pair, so two CTAs share
 // an SM and twice as many loads are in flight; the two halves of a logit meet through one shuffle per key.
 __global__ void __launch_bounds__(kRowThreads, 2) decode_attn_rows_kernel(const DecodeAttnParams p) {
+  grid_dep_sync();                                           // the launches of a decode step are chained (programmatic dependent launches)
   const int seg = blockIdx.y * kRowThreads + threadIdx.x;     // 32-element segment of a row
   const int u = seg >> 1, half = seg & 1;                     // (sequence, head) pair and which half of its 64 dimensions
   const bool live = u < p.B * p.H;
@@ -189,6 +191,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_attn_rows_kernel(const 
 // per pair, lanes over chunks for the maximum and the weights, then lanes over the 64 dimensions with the chunks
 // strided over the warps, combined through shared memory in warp order (a fixed order: bit-reproducible).
 __global__ void __launch_bounds__(256) decode_attn_merge_kernel(const DecodeAttnParams p) {
+  grid_dep_sync();                                           // the launches of a decode step are chained (programmatic dependent launches)
   __shared__ float s_w[kDecodeMaxRowChunks];
   __shared__ float s_red[8][68];
   const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -248,6 +251,7 @@ __device__ __forceinline__ unsigned pack2(float lo, float hi) {
 }
 
 __global__ void __launch_bounds__(kPreThreads) decode_prepass_kernel(const DecodePrepassParams p) {
+  grid_dep_sync();                                           // the launches of a decode step are chained (programmatic dependent launches)
   extern __shared__ __align__(16) unsigned char dsm[];
   const int d = p.d, stride = d + 16;                          // row stride in elements: 8-byte fragment loads without conflicts
   __nv_bfloat16* n_s = reinterpret_cast<__nv_bfloat16*>(dsm);                   // [16][d + 16]
@@ -346,10 +350,8 @@ cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, int* c
     if (p.chunk < 8) p.chunk = 8;
     p.n_chunks = (p.pos + p.chunk - 1) / p.chunk;
     dim3 grid(p.n_chunks, ceil_div(2 * p.B * p.H, kRowThreads));
-    decode_attn_rows_kernel<<<grid, kRowThreads, 0, s>>>(p);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    decode_attn_merge_kernel<<<p.B * p.H, 256, 0, s>>>(p);
+    { const cudaError_t el = launch_chained(decode_attn_rows_kernel, grid, dim3(kRowThreads), 0, s, true, p); if (el != cudaSuccess) return el; }
+    { const cudaError_t el = launch_chained(decode_attn_merge_kernel, dim3(p.B * p.H), dim3(256), 0, s, true, p); if (el != cudaSuccess) return el; }
     *n_chunks = 1; *chunk_stride = p.n_chunks;                // the merged state sits in the pair's first slot
     return cudaGetLastError();
   }
@@ -357,7 +359,7 @@ cudaError_t decode_attn_launch(const DecodeAttnParams& p0, int* n_chunks, int* c
   p.n_chunks = (p.pos + p.chunk - 1) / p.chunk;
   *n_chunks = p.n_chunks; *chunk_stride = p.n_chunks;
   dim3 grid(p.n_chunks, p.B, ceil_div(p.H, kDecWarps));
-  decode_attn_partial_kernel<<<grid, kDecWarps * 32, 0, s>>>(p);
+  { const cudaError_t el = launch_chained(decode_attn_partial_kernel, grid, dim3(kDecWarps * 32), 0, s, true, p); if (el != cudaSuccess) return el; }
   return cudaGetLastError();
 }
 
@@ -374,7 +376,7 @@ cudaError_t decode_prepass_launch(const DecodePrepassParams& p, cudaStream_t s) 
       set_for = dev;
     }
   }
-  decode_prepass_kernel<<<3 * p.H, kPreThreads, smem, s>>>(p);
+  { const cudaError_t el = launch_chained(decode_prepass_kernel, dim3(3 * p.H), dim3(kPreThreads), smem, s, true, p); if (el != cudaSuccess) return el; }
   return cudaGetLastError();
 }
 

@@ -82,6 +82,7 @@ __device__ __forceinline__ uint2 ldg_stream_v2(const void* p) {
 }
 __global__ void __launch_bounds__(256) head_mma_kernel(const __nv_bfloat16* emb, const __nv_bfloat16* g_final, const __nv_bfloat16* hidden,
                                                        long long h_bs, int B, int d, int vocab, int norm_flags, float eps, float* logits) {
+  grid_dep_sync();                                           // chained to the last layer's kernel (programmatic dependent launch)
   extern __shared__ __align__(16) unsigned char hsm[];
   const int stride = d + 16;
   __nv_bfloat16* hi_s = reinterpret_cast<__nv_bfloat16*>(hsm);                 // [16][d + 16]
@@ -164,9 +165,8 @@ cudaError_t head_launch(int dtype, const void* emb, const void* g_final, const v
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int groups = ceil_div(vocab, 8);
     const int nblk = ceil_div(groups, 8) < 2 * sms ? ceil_div(groups, 8) : 2 * sms;
-    head_mma_kernel<<<nblk, 256, sm2, s>>>((const __nv_bfloat16*)emb, (const __nv_bfloat16*)g_final, (const __nv_bfloat16*)hidden, h_bs,
-                                           B, d, vocab, norm_flags, eps, logits);
-    return cudaGetLastError();
+    return launch_chained(head_mma_kernel, dim3(nblk), dim3(256), sm2, s, true, (const __nv_bfloat16*)emb, (const __nv_bfloat16*)g_final,
+                          (const __nv_bfloat16*)hidden, h_bs, B, d, vocab, norm_flags, eps, logits);
   }
   if (dtype == RT_BF16) {
     e = cudaFuncSetAttribute(head_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
