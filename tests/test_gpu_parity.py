@@ -193,16 +193,18 @@ def test_c3_full_size_bf16_prefix_and_fixed_point():
 
 # ---------------------------------------------------------------- Algorithm 2 on its own (tensor-core and SIMT tile kernels)
 
-@pytest.mark.parametrize("dtype,nq,nk", [("bf16", 200, 128), ("bf16", 128, 320), ("bf16", 77, 96), ("f32", 40, 50),
-                                          ("bf16", 130, 384), ("bf16", 256, 1024)])
-def test_update_tile_matches_algorithm_2(dtype, nq, nk):
+@pytest.mark.parametrize("dtype,nq,nk,scale", [("bf16", 200, 128, 0.125), ("bf16", 128, 320, 0.125), ("bf16", 77, 96, 0.125),
+                                                ("f32", 40, 50, 0.125), ("bf16", 130, 384, 0.125), ("bf16", 256, 1024, 0.125),
+                                                ("bf16", 200, 448, 2.0), ("bf16", 128, 256, 6.0), ("f32", 40, 50, 2.0)])
+def test_update_tile_matches_algorithm_2(dtype, nq, nk, scale):
+    # scale 0.125: logits of order one; scale 2 and 6: logits of order +-16 and +-50, so that block maxima exceed the
+    # running reference maximum by far more than the lazy-rescale threshold of the tensor-core kernel again and again
     import torch
     from oracle import update_tile
     from paper_2604_21215_b200 import inputs, rt
     B, H, dh = 2, 3, 64
     d = H * dh
     rng = np.random.default_rng(600 + nq + nk)
-    scale = 0.125
     rows_q, rows_kv = nq + 8, nk + 24
     q = inputs.round_to(rng.standard_normal((rows_q, B, d)), dtype)
     k = inputs.round_to(rng.standard_normal((rows_kv, B, d)), dtype)
