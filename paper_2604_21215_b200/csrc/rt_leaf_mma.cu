@@ -27,6 +27,7 @@
 #include <type_traits>
 
 #include "rt_kernels.h"
+#include "rt_tc.cuh"
 
 namespace rt {
 
@@ -118,6 +119,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const unsigned (&a)[4], 
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// One weight row, global -> shared memory, as an asynchronous bulk copy that reports its bytes to an mbarrier (both
+// addresses 16-byte aligned, the size a multiple of 16 bytes).
+__device__ __forceinline__ void bulk_row(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory"); }
 
@@ -365,15 +372,22 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   const int f_lo = 2 * (int)((long long)(dff / 2) * cta / G), f_hi = 2 * (int)((long long)(dff / 2) * (cta + 1) / G);
   const int nd = d_hi - d_lo, nf = f_hi - f_lo;
 
-  if (tid == 0) *s_abort = 0;
-  {
+  // The CTA's weight rows go to shared memory as asynchronous bulk copies, one per row, issued by the threads of warp 0
+  // and counted by an mbarrier; the attention warps, which never read the weights, do not wait for them and build the
+  // leaf's state meanwhile; the MMA warps wait before their first token step.
+  const uint32_t w_bar = smem_u32(smem + 8);
+  if (tid == 0) {
+    *s_abort = 0;
+    mbar_init(w_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(w_bar, (uint32_t)(((size_t)3 * nd * d + (size_t)nf * d + (size_t)nd * dff) * 2));      // W_o, W_k, W_v; W_up; W_down
+  }
+  __syncthreads();
+  if (warp == 0) {
     auto stage = [&](__nv_bfloat16* dst, int dst_stride, const void* src_base, int row_lo, int nrows, int K) {
-      const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(src_base) + (size_t)row_lo * K);
-      const int per_row = K / 8;
-      for (int i = tid; i < nrows * per_row; i += kLeafMmaThreads) {
-        const int r = i / per_row, v = i % per_row;
-        *reinterpret_cast<uint4*>(dst + (size_t)r * dst_stride + v * 8) = src[(size_t)r * per_row + v];
-      }
+      const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(src_base) + (size_t)row_lo * K;
+      for (int r = lane; r < nrows; r += 32)
+        bulk_row(smem_u32(dst + (size_t)r * dst_stride), src + (size_t)r * K, (uint32_t)K * 2u, w_bar);
     };
     stage(s_wo, L.stride_d, p.w_o, d_lo, nd, d);
     stage(s_wup, L.stride_d, p.w_up, f_lo, nf, d);
@@ -381,7 +395,6 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
     stage(s_wk, L.stride_d, p.w_k, d_lo, nd, d);
     stage(s_wv, L.stride_d, p.w_v, d_lo, nd, d);
   }
-  __syncthreads();
 
   if (warp >= kMmaWarps) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsAttn));
@@ -413,6 +426,12 @@ __global__ void __launch_bounds__(kLeafMmaThreads, 1) leaf_mma_kernel(const Leaf
   unsigned bar_target = p.bar_base;
   const bool timing = TIMERS && (cta == 0 && tid == 0);
   unsigned long long t_ph = timing ? globaltimer_ns() : 0ull;
+
+  // the weight rows must have landed (the attention warps have been at work since the copies were issued); warp 0 waits
+  // for the copies, the other MMA warps for warp 0
+  if (warp == 0 && !mbar_wait(w_bar, 0, s_abort, p.sync)) *s_abort = 1;
+  mma_warps_sync();
+  if (*s_abort) return;
 
   for (int t = p.t0; t < p.t1; ++t) {
     const unsigned seq = p.seq_base + (unsigned)(t - p.t0) + 1u;
