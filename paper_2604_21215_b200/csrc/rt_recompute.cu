@@ -313,6 +313,69 @@ __global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) 
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
   const int b = m % p.B, r = m / p.B;
+  const T* g = reinterpret_cast<const T*>(p.norm_gain);
+  if (p.N % 4 == 0 && p.N <= 4096) {
+    // rows of up to 4096 entries: a thread owns up to four groups of four consecutive columns, fetched as 16-byte
+    // loads (all of a thread's loads are independent) and kept in registers for the normalisation
+    float v[4][4];
+    float ss = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int n = 4 * (tid + 256 * c);
+      if (n >= p.N) break;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int z = 0; z < p.splits; ++z) {
+        const float4 a = *reinterpret_cast<const float4*>(p.partial + ((size_t)z * p.M + m) * p.N + n);
+        acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+      }
+      const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+      if (p.epi == DENSE_RES_X) {
+        const T* xs = reinterpret_cast<const T*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[c][j] = to_f(xs[j]) + p.alpha * a4[j];
+        *reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n) = make_float4(v[c][0], v[c][1], v[c][2], v[c][3]);
+      } else if (p.epi == DENSE_GELU) {
+        T* o = reinterpret_cast<T*>(p.out) + (size_t)m * p.N + n;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { v[c][j] = gelu_exact(a4[j]); o[j] = from_f<T>(v[c][j]); }
+      } else if (p.epi == DENSE_F32) {
+        float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
+        const float4 old = p.accumulate ? *dst : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[c][0] = old.x + p.alpha * a4[0]; v[c][1] = old.y + p.alpha * a4[1];
+        v[c][2] = old.z + p.alpha * a4[2]; v[c][3] = old.w + p.alpha * a4[3];
+        *dst = make_float4(v[c][0], v[c][1], v[c][2], v[c][3]);
+      } else {
+        const float4 hv = *reinterpret_cast<const float4*>(p.h + (size_t)m * p.N + n);
+        const float h4[4] = {hv.x, hv.y, hv.z, hv.w};
+        T* o = reinterpret_cast<T*>(p.out) + (size_t)b * p.o_bs + (size_t)r * p.o_ts + n;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const T zr = from_f<T>(h4[j] + p.alpha * a4[j]);
+          o[j] = zr;
+          v[c][j] = to_f(zr);                                  // the next product sees the stored (rounded) z
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ss += v[c][j] * v[c][j];
+    }
+    if (!p.norm_out) return;
+    ss = warp_sum(ss);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float rs = p.norm_pre ? rsqrtf(tot / (float)p.N + p.norm_eps) : 1.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int n = 4 * (tid + 256 * c);
+      if (n >= p.N) break;
+      T* o = reinterpret_cast<T*>(p.norm_out) + (size_t)m * p.N + n;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[j] = from_f<T>(v[c][j] * rs * (p.norm_pre ? gain_at(g, n + j) : 1.0f));
+    }
+    return;
+  }
   float ss = 0.f;
   for (int n = tid; n < p.N; n += 256) {
     float acc = 0.f;
@@ -343,13 +406,12 @@ __global__ void __launch_bounds__(256) dense_reduce_kernel(const DenseParams p) 
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float rs = p.norm_pre ? rsqrtf(tot / (float)p.N + p.norm_eps) : 1.0f;
-  const T* g = reinterpret_cast<const T*>(p.norm_gain);
   for (int n = tid; n < p.N; n += 256) {
     float v;
     if (p.epi == DENSE_RES_X) v = p.h[(size_t)m * p.N + n];
     else if (p.epi == DENSE_GELU) v = to_f(reinterpret_cast<const T*>(p.out)[(size_t)m * p.N + n]);
     else v = to_f(reinterpret_cast<const T*>(p.out)[(size_t)b * p.o_bs + (size_t)r * p.o_ts + n]);
-    reinterpret_cast<T*>(p.norm_out)[(size_t)m * p.N + n] = from_f<T>(v * rs * (p.norm_pre ? gain_at(g, n) : 1.0f));
+    reinterpret_cast<T*>(p.norm_out)[(size_t)m * p.N + n] = from_f<T>(v * rs * (p.norm_pre ? gain_at(g, n + 0) : 1.0f));
   }
 }
 
