@@ -106,8 +106,9 @@ cudaError_t tile_simt_launch(int dtype, const TileParams& p, cudaStream_t s) {
 // Used by the wide-batch token step: position t attends to the pairs of its own leaf revealed so far,
 // [k0, k1) with k1 = t.  One warp per (sequence, head): each K and V row is one coalesced load (lanes over
 // the head's dimensions), the 32 per-lane partial products become per-key scores by a transposed reduction.
-template <typename T>
+template <typename T, int G>
 __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
+  // G: groups of 8 keys fetched per batch of 32 (the launcher picks the smallest that covers k1 - k0 when that is at most 32)
   grid_dep_sync();
   const int lane = threadIdx.x & 31;
   const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -130,10 +131,14 @@ __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
     float2 vv[32];
 #pragma unroll
     for (int jj = 0; jj < 32; ++jj) {
-      const int j = jb + (jj < cnt ? jj : 0);
-      const float2 k2 = ldcg_T2(Kc + (size_t)j * rstride + col);
-      vv[jj] = ldcg_T2(Vc + (size_t)j * rstride + col);
-      prod[jj] = q0 * k2.x + q1 * k2.y;
+      if (jj < 8 * G) {
+        const int j = jb + (jj < cnt ? jj : 0);
+        const float2 k2 = ldcg_T2(Kc + (size_t)j * rstride + col);
+        vv[jj] = ldcg_T2(Vc + (size_t)j * rstride + col);
+        prod[jj] = q0 * k2.x + q1 * k2.y;
+      } else {
+        prod[jj] = 0.f;
+      }
     }
     warp_transpose_sum32(prod, lane);
     const bool valid = lane < cnt;
@@ -144,7 +149,7 @@ __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
     l_run = l_run * corr + warp_sum(pj);
     o.x *= corr; o.y *= corr;
 #pragma unroll
-    for (int jj = 0; jj < 32; ++jj) {
+    for (int jj = 0; jj < 8 * G; ++jj) {
       const float pw = __shfl_sync(0xffffffffu, pj, jj);
       o.x += pw * vv[jj].x; o.y += pw * vv[jj].y;
     }
@@ -162,8 +167,23 @@ __global__ void __launch_bounds__(256) row_attn_kernel(const TileParams p) {
 cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s) {
   if (p.k1 <= p.k0 && !p.c_out) return cudaSuccess;
   const int blocks = ceil_div(p.B * p.H, 8);
-  if (dtype == RT_BF16) return launch_chained(row_attn_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, s, p.chained != 0, p);
-  return launch_chained(row_attn_kernel<float>, dim3(blocks), dim3(256), 0, s, p.chained != 0, p);
+  const int nk = p.k1 - p.k0;
+  const int groups = nk > 32 ? 4 : (nk > 24 ? 4 : (nk > 16 ? 3 : (nk > 8 ? 2 : 1)));
+  auto go = [&](auto kern) { return launch_chained(kern, dim3(blocks), dim3(256), 0, s, p.chained != 0, p); };
+  if (dtype == RT_BF16) {
+    switch (groups) {
+      case 1: return go(row_attn_kernel<__nv_bfloat16, 1>);
+      case 2: return go(row_attn_kernel<__nv_bfloat16, 2>);
+      case 3: return go(row_attn_kernel<__nv_bfloat16, 3>);
+      default: return go(row_attn_kernel<__nv_bfloat16, 4>);
+    }
+  }
+  switch (groups) {
+    case 1: return go(row_attn_kernel<float, 1>);
+    case 2: return go(row_attn_kernel<float, 2>);
+    case 3: return go(row_attn_kernel<float, 3>);
+    default: return go(row_attn_kernel<float, 4>);
+  }
 }
 
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
