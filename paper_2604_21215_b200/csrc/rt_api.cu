@@ -107,6 +107,8 @@ int leaf_size(const rt_config* c) { return c->leaf ? c->leaf : kAutoLeaf; }
 // a B200).
 enum ChainPath { kPathGeneric = 0, kPathMma = 1, kPathWide = 2, kPathBlocks = 3, kPathMmaSplit = 4 };
 struct Schedule { ChainPath path; int leaf; int sub; };      // sub: sequences per launch of the tensor-core leaf kernel (kPathMmaSplit)
+constexpr int kWideLeafDefault = 16;    // leaf of the dense-product token steps: the in-leaf attention re-reads the leaf's pairs for every position,
+                                        // so short leaves win (p512: 16 -> 41.6 ms, 32 -> 42.3, 64 -> 45.9 per layer)
 constexpr int kMmaSplitMax = 48;         // largest batch that runs as slices of at most 16 sequences through the tensor-core leaf kernel
 Schedule effective_schedule(const rt_config* c, int B) {
   if (c->recur_block > 1) return {kPathBlocks, c->recur_block, 0};
@@ -123,7 +125,7 @@ Schedule effective_schedule(const rt_config* c, int B) {
     // bf16 batches beyond that (or whose slices the tensor-core leaf kernel does not take) run as dense products from
     // 24 sequences on, where they overtake the generic kernel (measured at d = 1024: 53 us per token step at B = 32
     // against 99 us); fp32 keeps the generic kernel up to its limit
-    if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : 32, 0};
+    if (B > kSmallBatchMax || (c->dtype == RT_BF16 && B >= 24)) return {kPathWide, c->leaf ? c->leaf : kWideLeafDefault, 0};
     if (c->dtype == RT_BF16 && leaf_mma_shape(B, c->d_model, c->n_heads, c->d_ff, c->leaf, kB200Sms, kB200SmemPerCta, &ml))
       return {kPathMma, ml.leaf, B};
   }
@@ -319,7 +321,7 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
     dp.partial = (float*)(ws + L.ex_part); dp.partial_bytes = (size_t)B * c->n_heads * kMaxChunks * 68 * 4;
     // in-leaf attention re-reads the leaf's pairs for every position (leaf^2 * B * d bytes per leaf), so wide
     // batches default to a shorter leaf
-    const int Lf = plan.path == kPathWide ? plan.leaf : (c->leaf ? c->leaf : 32), N = n_rows;
+    const int Lf = plan.path == kPathWide ? plan.leaf : (c->leaf ? c->leaf : kWideLeafDefault), N = n_rows;
     for (int s0 = 0; s0 < N; s0 += Lf) {
       const int e0 = s0 + Lf < N ? s0 + Lf : N;
       {

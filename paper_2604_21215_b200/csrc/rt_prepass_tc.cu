@@ -14,22 +14,25 @@
 
 namespace rt {
 
-constexpr int kGemmBN = 128;
 constexpr int kGemmBK = 64;
-constexpr int kGemmStages = 3;
 constexpr int kGemmThreads = 192;
 constexpr uint32_t kGemmABytes = kBM * kGemmBK * 2;        // 16 KB
-constexpr uint32_t kGemmBBytes = kGemmBN * kGemmBK * 2;    // 16 KB
 
-struct GemmSmem {
+// BN: output columns per CTA.  128 with a 3-stage ring (two CTAs per SM) for the sweep over all positions; 64 (one head)
+// with a 6-stage ring for launches over few rows (one position of a wide batch), which then fill twice as many SMs.
+template <int BN>
+struct GemmSmemT {
+  static constexpr int stages = BN == 64 ? 6 : 3;
+  static constexpr uint32_t b_bytes = BN * kGemmBK * 2;
   static constexpr uint32_t a = 0;
-  static constexpr uint32_t b = a + kGemmStages * kGemmABytes;
-  static constexpr uint32_t bars = b + kGemmStages * kGemmBBytes;      // full[3], empty[3], acc_ready
-  static constexpr uint32_t tmem_ptr = bars + 64;
+  static constexpr uint32_t b = a + stages * kGemmABytes;
+  static constexpr uint32_t bars = b + stages * b_bytes;               // full[], empty[], acc_ready
+  static constexpr uint32_t tmem_ptr = bars + 128;
   static constexpr uint32_t abort_flag = tmem_ptr + 8;
   static constexpr uint32_t total = abort_flag + 8;
 };
 
+template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 2)
 qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_constant__ CUtensorMap map_wq,
                    const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv,
@@ -38,6 +41,9 @@ qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_const
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
+  using GemmSmem = GemmSmemT<BN>;
+  constexpr int kGemmBN = BN, kGemmStages = GemmSmem::stages;
+  constexpr uint32_t kGemmBBytes = GemmSmem::b_bytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int M = p.N * p.B, d = p.d;
   const int tiles_per_mat = d / kGemmBN;
@@ -168,19 +174,26 @@ qkv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_n, const __grid_const
 
 static_assert(kGemmBK == 64, "tensor_map_rows_bf16 encodes 64-column boxes");
 
-bool qkv_gemm_tc_supported(const PrepassParams& p) { return p.d % kGemmBN == 0 && p.d >= kGemmBN; }
+bool qkv_gemm_tc_supported(const PrepassParams& p) { return p.d % 128 == 0 && p.d >= 128; }
 
 cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStream_t s) {
   const int M = p.N * p.B;
+  int mats = 0;
+  for (int w = 0; w < 3; ++w) mats += (!p.mats || ((p.mats >> w) & 1)) ? 1 : 0;
+  // few rows: one head per CTA, so that the launch fills the multiprocessors
+  const int bn = ceil_div(M, kBM) * mats * (p.d / 128) < sm_count() / 2 ? 64 : 128;
   CUtensorMap mn, mq, mk, mv;
-  if (!tensor_map_rows_bf16(&mn, p.n, M, p.d, kBM) || !tensor_map_rows_bf16(&mq, p.w_q, p.d, p.d, kGemmBN) ||
-      !tensor_map_rows_bf16(&mk, p.w_k, p.d, p.d, kGemmBN) || !tensor_map_rows_bf16(&mv, p.w_v, p.d, p.d, kGemmBN))
+  if (!tensor_map_rows_bf16(&mn, p.n, M, p.d, kBM) || !tensor_map_rows_bf16(&mq, p.w_q, p.d, p.d, bn) ||
+      !tensor_map_rows_bf16(&mk, p.w_k, p.d, p.d, bn) || !tensor_map_rows_bf16(&mv, p.w_v, p.d, p.d, bn))
     return cudaErrorInvalidValue;
-  const size_t smem = GemmSmem::total + 1024;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&qkv_gemm_tc_kernel), (int)smem);
-  if (e != cudaSuccess) return e;
-  dim3 grid(ceil_div(M, kBM), 3 * (p.d / kGemmBN));
-  return launch_chained(qkv_gemm_tc_kernel, grid, dim3(kGemmThreads), smem, s, p.chained != 0, mn, mq, mk, mv, p, sync);
+  dim3 grid(ceil_div(M, kBM), 3 * (p.d / bn));
+  auto run = [&](auto kern, size_t smem) -> cudaError_t {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_chained(kern, grid, dim3(kGemmThreads), smem, s, p.chained != 0, mn, mq, mk, mv, p, sync);
+  };
+  if (bn == 64) return run(qkv_gemm_tc_kernel<64>, GemmSmemT<64>::total + 1024);
+  return run(qkv_gemm_tc_kernel<128>, GemmSmemT<128>::total + 1024);
 }
 
 }  // namespace rt

@@ -98,11 +98,11 @@ def test_plan_counters_follow_the_n_log_n_model():
 
 
 def test_plan_counters_model_the_schedule_that_runs():
-    # The counters follow the chain form a shape takes: wide batches use leaves of 32 positions, the tensor-core
+    # The counters follow the chain form a shape takes: wide batches use leaves of 16 positions, the tensor-core
     # leaf kernel keeps 64-position leaves also when an SM owns two (sequence, head) pairs, blocked recurrence tiles by blocks.
     N = 2048
     wide = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 96, N)
-    assert wide["n_leaves"] == N // 32 and wide["n_tiles"] == len(rt.rt_plan_tiles(N, 32))
+    assert wide["n_leaves"] == N // 16 and wide["n_tiles"] == len(rt.rt_plan_tiles(N, 16))
     # 17 .. 48 sequences run as slices of at most 16 through the tensor-core leaf kernel: its leaves, and the chain
     # weights staged once per slice and leaf
     split = rt.rt_plan_counters(rt.make_config(1024, 16, 4096, dtype="bf16"), 32, N)
