@@ -732,7 +732,7 @@ rt_status rt_update_tile(const rt_config* cfg, const void* q, const void* k_cach
   if (q0 < 0 || q1 < q0 || q1 > rows_q || k0 < 0 || k1 < k0 || k1 > rows_kv) return RT_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(st_o) || !aligned16(workspace))
     return RT_ERR_INVALID_ARG;
-  const rt_status sup = config_supported(cfg, B);
+  const rt_status sup = config_supported(cfg, B, true);        // a tile takes any batch
   if (sup != RT_OK) return sup;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (cudaMemsetAsync(workspace, 0, sizeof(SyncArea), s) != cudaSuccess) return RT_ERR_CUDA;

@@ -186,7 +186,85 @@ cudaError_t row_attn_launch(int dtype, const TileParams& p, cudaStream_t s) {
   }
 }
 
+// ---- small tiles: at most 16 pairs against a short run of queries ---------------------------------------
+// Algorithm 2 for the lowest levels of a short-leaf schedule (wide batches: leaves of 16).  One warp per (sequence,
+// head) and kSmallTileQueries queries: the K and V rows of the tile are fetched once (one coalesced load per row, lanes
+// over the head's dimensions) and stay in registers, and the warp's query rows, output rows and statistics are all
+// requested before the first product; every query then costs one transposed reduction for its scores and one pass over
+// the values.  G = groups of 8 pairs (1 or 2).
+constexpr int kSmallTileQueries = 4;      // queries per warp
+template <typename T, int G>
+__global__ void __launch_bounds__(128) tile_rows_kernel(const TileParams p) {
+  grid_dep_sync();
+  const int lane = threadIdx.x & 31;
+  const int u = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (u >= p.B * p.H) return;
+  const int b = u / p.H, h = u % p.H;
+  const int qa = p.q0 + (int)blockIdx.y * kSmallTileQueries;
+  const int cnt = p.k1 - p.k0;
+  const T* Kc = reinterpret_cast<const T*>(p.k_cache);
+  const T* Vc = reinterpret_cast<const T*>(p.v_cache);
+  const size_t col = (size_t)b * p.d + h * kHeadDim + 2 * lane;
+  const size_t rstride = (size_t)p.B * p.d;
+  const float slope_l2 = p.alibi ? p.alibi[h] * kLog2e : 0.f;
+  float2 qq[kSmallTileQueries], oo[kSmallTileQueries];
+  float mm[kSmallTileQueries], ll[kSmallTileQueries];
+#pragma unroll
+  for (int i = 0; i < kSmallTileQueries; ++i) {
+    const int t = qa + i < p.q1 ? qa + i : p.q1 - 1;              // (rows beyond the tile repeat its last query and are not stored)
+    const size_t sidx = (size_t)t * p.B + b;
+    qq[i] = ldcg_T2(reinterpret_cast<const T*>(p.q) + (size_t)t * rstride + col);
+    oo[i] = __ldcg(reinterpret_cast<const float2*>(p.st_o + sidx * p.d + h * kHeadDim + 2 * lane));
+    mm[i] = __ldcg(p.st_m + sidx * p.H + h);
+    ll[i] = __ldcg(p.st_l + sidx * p.H + h);
+  }
+  float2 kk[8 * G], vv[8 * G];
+#pragma unroll
+  for (int jj = 0; jj < 8 * G; ++jj) {
+    const int j = p.k0 + (jj < cnt ? jj : 0);
+    kk[jj] = ldcg_T2(Kc + (size_t)j * rstride + col);
+    vv[jj] = ldcg_T2(Vc + (size_t)j * rstride + col);
+  }
+  const bool valid = lane < cnt;
+#pragma unroll
+  for (int i = 0; i < kSmallTileQueries; ++i) {
+    const int t = qa + i;
+    float prod[32];
+#pragma unroll
+    for (int jj = 0; jj < 32; ++jj) prod[jj] = jj < 8 * G ? qq[i].x * kk[jj].x + qq[i].y * kk[jj].y : 0.f;
+    warp_transpose_sum32(prod, lane);
+    const float s2 = valid ? prod[0] * p.scale_log2 - slope_l2 * (float)(t - (p.k0 + lane)) : -INFINITY;
+    const float m_new = fmaxf(mm[i], warp_max(s2));
+    const float pj = valid ? exp2f(s2 - m_new) : 0.f;
+    const float corr = exp2f(mm[i] - m_new);
+    const float l_new = ll[i] * corr + warp_sum(pj);
+    float2 o = make_float2(oo[i].x * corr, oo[i].y * corr);
+#pragma unroll
+    for (int jj = 0; jj < 8 * G; ++jj) {
+      const float pw = __shfl_sync(0xffffffffu, pj, jj);
+      o.x += pw * vv[jj].x; o.y += pw * vv[jj].y;
+    }
+    if (t < p.q1) {
+      const size_t sidx = (size_t)t * p.B + b;
+      if (lane == 0) { p.st_m[sidx * p.H + h] = m_new; p.st_l[sidx * p.H + h] = l_new; }
+      *reinterpret_cast<float2*>(p.st_o + sidx * p.d + h * kHeadDim + 2 * lane) = o;
+    }
+  }
+}
+
+cudaError_t tile_rows_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  const int nk = p.k1 - p.k0, nq = p.q1 - p.q0;
+  dim3 grid(ceil_div(p.B * p.H, 4), ceil_div(nq, kSmallTileQueries));
+  auto go = [&](auto kern) { return launch_chained(kern, grid, dim3(128), 0, s, p.chained != 0, p); };
+  if (dtype == RT_BF16) return nk > 8 ? go(tile_rows_kernel<__nv_bfloat16, 2>) : go(tile_rows_kernel<__nv_bfloat16, 1>);
+  return nk > 8 ? go(tile_rows_kernel<float, 2>) : go(tile_rows_kernel<float, 1>);
+}
+
 cudaError_t tile_launch(int dtype, const TileParams& p, cudaStream_t s) {
+  // at most 16 pairs, a plain tile (no causal mask, one copy): the small-tile kernel (measured on B = 512, H = 16: 16 pairs
+  // x 16 queries 78 us against 127 us; with 32 pairs the registers it needs leave too few warps per SM: 260 against 254 us)
+  if (p.k1 - p.k0 <= 16 && p.k1 > p.k0 && p.q1 > p.q0 && !p.causal && p.batch <= 1 && p.q_limit == 0)
+    return tile_rows_launch(dtype, p, s);
   // Whole 64-key blocks only on the tensor-core path: a partial block would bring cache rows that
   // are not revealed yet (arbitrary bits) into the P.V product.
   if (dtype == RT_BF16 && (p.k1 - p.k0) % 64 == 0 && p.d % kHeadDim == 0)
