@@ -133,6 +133,85 @@ struct DenseSmem {
   static constexpr uint32_t total = abort_flag + 8;
 };
 
+// Epilogue of one thread's output row: its BN accumulator columns from TMEM (lane = row), 32 at a time.
+template <int BN>
+__device__ __forceinline__ void dense_epilogue_row(const DenseParams& p, uint32_t tmem, int warp, int m, int n0, int splits, int zsplit) {
+  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+  const int b = m % p.B, r = m / p.B;
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    uint32_t v[32];
+    tc_ld32(t_row + (uint32_t)c0, v);
+    tc_wait_ld();
+    if (m >= p.M) continue;
+    const int n = n0 + c0;
+    if (splits > 1) {                                          // raw partial sums; dense_reduce_kernel finishes
+      float4* dst = reinterpret_cast<float4*>(p.partial + ((size_t)zsplit * p.M + m) * p.N + n);
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+      continue;
+    }
+    if (p.epi == DENSE_F32) {
+      float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        float4 o = make_float4(p.alpha * __uint_as_float(v[4 * q]), p.alpha * __uint_as_float(v[4 * q + 1]),
+                               p.alpha * __uint_as_float(v[4 * q + 2]), p.alpha * __uint_as_float(v[4 * q + 3]));
+        if (p.accumulate) { const float4 old = dst[q]; o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+        dst[q] = o;
+      }
+      continue;
+    }
+    if (p.epi == DENSE_RES_X) {
+      const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n);
+      float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {                           // 8 columns per 16-byte load of x
+        const uint4 xw = xs[q];
+        const unsigned w4[4] = {xw.x, xw.y, xw.z, xw.w};
+        float o[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          o[2 * j] = __uint_as_float(w4[j] << 16) + p.alpha * __uint_as_float(v[8 * q + 2 * j]);
+          o[2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u) + p.alpha * __uint_as_float(v[8 * q + 2 * j + 1]);
+        }
+        dst[2 * q] = make_float4(o[0], o[1], o[2], o[3]);
+        dst[2 * q + 1] = make_float4(o[4], o[5], o[6], o[7]);
+      }
+    } else {
+      float o[32];
+      if (p.epi == DENSE_GELU) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[j] = gelu_exact(__uint_as_float(v[j]));
+      } else {
+        const float4* hs = reinterpret_cast<const float4*>(p.h + (size_t)m * p.N + n);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float4 hv = hs[q];
+          o[4 * q] = hv.x + p.alpha * __uint_as_float(v[4 * q]);
+          o[4 * q + 1] = hv.y + p.alpha * __uint_as_float(v[4 * q + 1]);
+          o[4 * q + 2] = hv.z + p.alpha * __uint_as_float(v[4 * q + 2]);
+          o[4 * q + 3] = hv.w + p.alpha * __uint_as_float(v[4 * q + 3]);
+        }
+      }
+      __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                          (p.epi == DENSE_GELU ? (size_t)m * p.N + n : (size_t)b * p.o_bs + (size_t)r * p.o_ts + n);
+      uint4* dst = reinterpret_cast<uint4*>(ob);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const __nv_bfloat162 pk = __floats2bfloat162_rn(o[8 * q + 2 * j], o[8 * q + 2 * j + 1]);
+          w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+        }
+        dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kTThreads, 2)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
@@ -221,80 +300,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int m = m0 + warp * 32 + lane;
     if (mbar_wait(acc_ready, 0, s_abort, sync)) {
       tc_fence_after();
-      const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-      const int b = m % p.B, r = m / p.B;
-#pragma unroll 1
-      for (int c0 = 0; c0 < kTBN; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(t_row + (uint32_t)c0, v);
-        tc_wait_ld();
-        if (m >= p.M) continue;
-        const int n = n0 + c0;
-        if (splits > 1) {                                          // raw partial sums; dense_reduce_kernel finishes
-          float4* dst = reinterpret_cast<float4*>(p.partial + ((size_t)blockIdx.z * p.M + m) * p.N + n);
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
-          continue;
-        }
-        if (p.epi == DENSE_F32) {
-          float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 o = make_float4(p.alpha * __uint_as_float(v[4 * q]), p.alpha * __uint_as_float(v[4 * q + 1]),
-                                   p.alpha * __uint_as_float(v[4 * q + 2]), p.alpha * __uint_as_float(v[4 * q + 3]));
-            if (p.accumulate) { const float4 old = dst[q]; o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
-            dst[q] = o;
-          }
-          continue;
-        }
-        if (p.epi == DENSE_RES_X) {
-          const uint4* xs = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.x) + (size_t)b * p.x_bs + (size_t)r * p.x_ts + n);
-          float4* dst = reinterpret_cast<float4*>(p.h + (size_t)m * p.N + n);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {                           // 8 columns per 16-byte load of x
-            const uint4 xw = xs[q];
-            const unsigned w4[4] = {xw.x, xw.y, xw.z, xw.w};
-            float o[8];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              o[2 * j] = __uint_as_float(w4[j] << 16) + p.alpha * __uint_as_float(v[8 * q + 2 * j]);
-              o[2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u) + p.alpha * __uint_as_float(v[8 * q + 2 * j + 1]);
-            }
-            dst[2 * q] = make_float4(o[0], o[1], o[2], o[3]);
-            dst[2 * q + 1] = make_float4(o[4], o[5], o[6], o[7]);
-          }
-        } else {
-          float o[32];
-          if (p.epi == DENSE_GELU) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = gelu_exact(__uint_as_float(v[j]));
-          } else {
-            const float4* hs = reinterpret_cast<const float4*>(p.h + (size_t)m * p.N + n);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 hv = hs[q];
-              o[4 * q] = hv.x + p.alpha * __uint_as_float(v[4 * q]);
-              o[4 * q + 1] = hv.y + p.alpha * __uint_as_float(v[4 * q + 1]);
-              o[4 * q + 2] = hv.z + p.alpha * __uint_as_float(v[4 * q + 2]);
-              o[4 * q + 3] = hv.w + p.alpha * __uint_as_float(v[4 * q + 3]);
-            }
-          }
-          __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) +
-                              (p.epi == DENSE_GELU ? (size_t)m * p.N + n : (size_t)b * p.o_bs + (size_t)r * p.o_ts + n);
-          uint4* dst = reinterpret_cast<uint4*>(ob);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const __nv_bfloat162 pk = __floats2bfloat162_rn(o[8 * q + 2 * j], o[8 * q + 2 * j + 1]);
-              w[j] = *reinterpret_cast<const uint32_t*>(&pk);
-            }
-            dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-      }
+      dense_epilogue_row<kTBN>(p, tmem, warp, m, n0, splits, (int)blockIdx.z);
     }
   }
   tc_fence_before();
@@ -302,6 +308,137 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (warp == 4) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTBN) : "memory");
+  }
+}
+
+// ---- the same product on CTA pairs (cta_group::2) -----------------------------------------------------------
+// Two CTAs of a cluster share a 256 x BN output tile: each fetches its own 128 rows of A and HALF of the BN weight rows,
+// the leader's thread issues tcgen05.mma.cta_group::2 (M = 256), which reads A and W from both CTAs' shared memory and
+// accumulates each CTA's 128 rows in that CTA's TMEM.  Per CTA and 64-wide k-block that is 16 KB + BN * 64 bytes from L2
+// instead of 16 KB + BN * 128: the products here are bound by that stream.  Copies are plain TMA loads (no multicast)
+// that report to the leader's barrier; the leader's commits reach both CTAs' barriers.
+template <int BN>
+struct PairSmem {
+  static constexpr int stages = BN == 256 ? 3 : 4;
+  static constexpr uint32_t b_bytes = (BN / 2) * kTBK * 2;
+  static constexpr uint32_t a = 0;
+  static constexpr uint32_t b = a + stages * kTABytes;
+  static constexpr uint32_t bars = b + stages * b_bytes;         // full[], empty[], acc_ready
+  static constexpr uint32_t tmem_ptr = bars + 128;
+  static constexpr uint32_t abort_flag = tmem_ptr + 8;
+  static constexpr uint32_t total = abort_flag + 8;
+};
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load of this CTA's tile whose bytes are reported to the LEADER's barrier at the same offset (bit 24 of a
+// shared::cluster address selects the CTA of the pair)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar & 0xFEFFFFFFu), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {           // arrives on the barrier at this offset in BOTH CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
+template <int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTThreads, 2)
+dense_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
+                  SyncArea* sync) {
+  grid_dep_sync();
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  using PS = PairSmem<BN>;
+  constexpr int kSt = PS::stages;
+  const int rank = (int)cluster_rank();                         // 0: leader (issues the products)
+  const int m0 = ((int)blockIdx.x >> 1) * 2 * kBM + rank * kBM, n0 = blockIdx.y * BN;
+  const int splits = p.splits > 1 ? p.splits : 1;
+  const int kb_all = p.K / kTBK;
+  const int kb0 = (int)((long long)kb_all * blockIdx.z / splits);
+  const int n_kb = (int)((long long)kb_all * (blockIdx.z + 1) / splits) - kb0;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + PS::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + PS::tmem_ptr);
+  auto full = [&](int s) { return sbase + PS::bars + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return sbase + PS::bars + 8u * (uint32_t)(kSt + s); };
+  const uint32_t acc_ready = sbase + PS::bars + 8u * (2 * kSt);
+
+  if (tid == 0) {
+    *s_abort = 0;
+    for (int s = 0; s < kSt; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    mbar_init(acc_ready, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + PS::tmem_ptr), "n"(BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                           // both CTAs' barriers exist before anything is signalled
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  // No role returns early: every thread of both CTAs reaches the cluster barrier at the end.
+  if (warp == 4) {
+    // ---------------- TMA producer (each CTA: its 128 rows of A, its half of the weight rows) ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kSt;
+        if (kb >= kSt) ok = mbar_wait(empty(s), ((kb / kSt) - 1) & 1, s_abort, sync);
+        if (!ok) break;
+        if (rank == 0) mbar_expect_tx(full(s), 2u * (kTABytes + PS::b_bytes));      // the bytes of both CTAs
+        tma_load_2d_pair(sbase + PS::a + s * kTABytes, &map_a, full(s), (kb0 + kb) * kTBK, m0);
+        tma_load_2d_pair(sbase + PS::b + s * PS::b_bytes, &map_w, full(s), (kb0 + kb) * kTBK, n0 + rank * (BN / 2));
+        ++issued;
+      }
+      (void)issued;
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ---------------- MMA issuer (leader only) ----------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
+      bool ok = true;
+      for (int kb = 0; kb < n_kb && ok; ++kb) {
+        const int s = kb % kSt;
+        ok = mbar_wait(full(s), (kb / kSt) & 1, s_abort, sync);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t a0 = make_desc(sbase + PS::a + s * kTABytes, 16, 1024);
+        const uint64_t b0 = make_desc(sbase + PS::b + s * PS::b_bytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < kTBK / 16; ++ks)
+          tc_mma_pair(tmem, a0 + 2u * ks, b0 + 2u * ks, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+        tc_commit_pair(empty(s));
+      }
+      if (ok) tc_commit_pair(acc_ready);
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue: one output row per thread ----------------
+    const int m = m0 + warp * 32 + lane;
+    if (mbar_wait(acc_ready, 0, s_abort, sync)) {
+      tc_fence_after();
+      dense_epilogue_row<BN>(p, tmem, warp, m, n0, splits, (int)blockIdx.z);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                           // the partner is done with this CTA's shared memory and TMEM
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(BN) : "memory");
   }
 }
 
@@ -438,22 +575,21 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       while (want > 1 && kb_all / want < 4) --want;               // at least 4 k blocks per split
       if ((size_t)want * p.M * p.N * sizeof(float) <= p.partial_bytes) q.splits = want;
     }
+    // CTA pairs on 256-row tiles (each CTA fetches half of the weight tile) for products of at least a wave of CTAs:
+    // c3's chain products 0.892 -> 0.850 ms; the few-row products of a wide-batch token step are 3 % slower as pairs
+    const bool pair = q.splits == 1 && ctas >= sms;
     CUtensorMap ma, mw;
-    if (!tensor_map_rows_bf16(&ma, p.A, p.M, p.K, kBM) || !tensor_map_rows_bf16(&mw, p.W, p.N, p.K, bn)) return cudaErrorInvalidValue;
-    dim3 grid(m_tiles, p.N / bn, q.splits);
-    if (bn == 256) {
-      const size_t smem = DenseSmem<256>::total + 1024;
-      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_tc_kernel<256>), (int)smem);
+    if (!tensor_map_rows_bf16(&ma, p.A, p.M, p.K, kBM) || !tensor_map_rows_bf16(&mw, p.W, p.N, p.K, pair ? bn / 2 : bn)) return cudaErrorInvalidValue;
+    dim3 grid(pair ? 2 * ceil_div(p.M, 2 * kBM) : m_tiles, p.N / bn, q.splits);
+    auto run = [&](auto kern, size_t smem) -> cudaError_t {
+      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), (int)smem);
       if (e != cudaSuccess) return e;
-      e = launch_chained(dense_tc_kernel<256>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
-      if (e != cudaSuccess) return e;
-    } else {
-      const size_t smem = DenseSmem<128>::total + 1024;
-      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_tc_kernel<128>), (int)smem);
-      if (e != cudaSuccess) return e;
-      e = launch_chained(dense_tc_kernel<128>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
-      if (e != cudaSuccess) return e;
-    }
+      return launch_chained(kern, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
+    };
+    cudaError_t e;
+    if (pair) e = bn == 256 ? run(dense_pair_kernel<256>, PairSmem<256>::total + 1024) : run(dense_pair_kernel<128>, PairSmem<128>::total + 1024);
+    else e = bn == 256 ? run(dense_tc_kernel<256>, DenseSmem<256>::total + 1024) : run(dense_tc_kernel<128>, DenseSmem<128>::total + 1024);
+    if (e != cudaSuccess) return e;
     if (q.splits > 1) {
       cudaError_t er = launch_chained(dense_reduce_kernel<__nv_bfloat16>, dim3(p.M), dim3(256), 0, s, p.chained != 0, q);
       if (er != cudaSuccess) return er;
