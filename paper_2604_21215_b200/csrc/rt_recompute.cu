@@ -442,6 +442,136 @@ dense_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
+// ---- CTA pairs, persistent: one pair per two SMs walks over the 256 x 256 output tiles ----------------------------
+// Same products as dense_pair_kernel, but a pair stays resident (one CTA per SM, all 512 TMEM columns = two accumulator
+// buffers of 256) and takes tile after tile: while the epilogue warps of both CTAs drain buffer b, the leader already
+// accumulates the next tile into buffer b ^ 1, and the operand ring never runs dry between tiles.
+struct PersistSmem {
+  static constexpr int stages = 6;
+  static constexpr uint32_t b_bytes = 128 * kTBK * 2;            // half of a 256-column weight tile
+  static constexpr uint32_t a = 0;
+  static constexpr uint32_t b = a + stages * kTABytes;
+  static constexpr uint32_t bars = b + stages * b_bytes;         // full[6], empty[6], acc_full[2], acc_empty[2]
+  static constexpr uint32_t tmem_ptr = bars + 192;
+  static constexpr uint32_t abort_flag = tmem_ptr + 8;
+  static constexpr uint32_t total = abort_flag + 8;
+};
+// arrive on the barrier at this offset in the LEADER's shared memory (from either CTA of the pair)
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(0u));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTThreads, 1)
+dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
+                          SyncArea* sync) {
+  grid_dep_sync();
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  using PS = PersistSmem;
+  constexpr int kSt = PS::stages, BN = 256;
+  const int rank = (int)cluster_rank();
+  const int m_pairs = (p.M + 2 * kBM - 1) / (2 * kBM), n_tiles = p.N / BN;
+  const int T = m_pairs * n_tiles;                              // tiles; pair c takes c, c + pairs, ...
+  const int pairs = (int)gridDim.x >> 1, pair_id = (int)blockIdx.x >> 1;
+  const int n_kb = p.K / kTBK;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + PS::abort_flag);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + PS::tmem_ptr);
+  auto full = [&](int s) { return sbase + PS::bars + 8u * (uint32_t)s; };
+  auto empty = [&](int s) { return sbase + PS::bars + 8u * (uint32_t)(kSt + s); };
+  auto acc_full = [&](int b) { return sbase + PS::bars + 8u * (uint32_t)(2 * kSt + b); };
+  auto acc_empty = [&](int b) { return sbase + PS::bars + 8u * (uint32_t)(2 * kSt + 2 + b); };
+
+  if (tid == 0) {
+    *s_abort = 0;
+    for (int s = 0; s < kSt; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }   // 4 epilogue warps of each CTA
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + PS::tmem_ptr), "n"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  // No role returns early: every thread of both CTAs reaches the cluster barrier at the end.
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int t = pair_id; t < T && ok; t += pairs) {
+        const int m0 = (t % m_pairs) * 2 * kBM + rank * kBM, n0 = (t / m_pairs) * BN;
+        for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+          const int s = it % kSt;
+          if (it >= kSt) ok = mbar_wait(empty(s), ((it / kSt) - 1) & 1, s_abort, sync);
+          if (!ok) break;
+          if (rank == 0) mbar_expect_tx(full(s), 2u * (kTABytes + PS::b_bytes));
+          tma_load_2d_pair(sbase + PS::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
+          tma_load_2d_pair(sbase + PS::b + s * PS::b_bytes, &map_w, full(s), kb * kTBK, n0 + rank * (BN / 2));
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ---------------- MMA issuer (leader only) ----------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
+      int it = 0, i = 0;
+      bool ok = true;
+      for (int t = pair_id; t < T && ok; t += pairs, ++i) {
+        const int b = i & 1;
+        if (i >= 2) ok = mbar_wait(acc_empty(b), ((i >> 1) - 1) & 1, s_abort, sync);     // both CTAs have drained this buffer
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+          const int s = it % kSt;
+          ok = mbar_wait(full(s), (it / kSt) & 1, s_abort, sync);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t a0 = make_desc(sbase + PS::a + s * kTABytes, 16, 1024);
+          const uint64_t b0 = make_desc(sbase + PS::b + s * PS::b_bytes, 16, 1024);
+#pragma unroll
+          for (int ks = 0; ks < kTBK / 16; ++ks)
+            tc_mma_pair(tmem + (uint32_t)(b * BN), a0 + 2u * ks, b0 + 2u * ks, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+          tc_commit_pair(empty(s));
+        }
+        if (ok) tc_commit_pair(acc_full(b));
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue: one output row per thread, tile after tile ----------------
+    int i = 0;
+    bool ok = true;
+    for (int t = pair_id; t < T && ok; t += pairs, ++i) {
+      const int b = i & 1;
+      const int m = (t % m_pairs) * 2 * kBM + rank * kBM + warp * 32 + lane, n0 = (t / m_pairs) * BN;
+      ok = __all_sync(0xffffffffu, mbar_wait(acc_full(b), (i >> 1) & 1, s_abort, sync));
+      if (!ok) break;
+      tc_fence_after();
+      dense_epilogue_row<BN>(p, tmem + (uint32_t)(b * BN), warp, m, n0, 1, 0);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(acc_empty(b));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(512) : "memory");
+  }
+}
+
 // Sums the partial products of a split contraction in a fixed order and applies the epilogue; one CTA per
 // output row, so it can also leave RMS_g(row) of the result for the product that follows.
 template <typename T>
@@ -587,7 +717,15 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       return launch_chained(kern, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, mw, q, sync);
     };
     cudaError_t e;
-    if (pair) e = bn == 256 ? run(dense_pair_kernel<256>, PairSmem<256>::total + 1024) : run(dense_pair_kernel<128>, PairSmem<128>::total + 1024);
+#ifndef RT_DENSE_PERSIST
+#define RT_DENSE_PERSIST 1
+#endif
+    if (pair && bn == 256 && RT_DENSE_PERSIST) {
+      // resident pairs (one CTA per SM) walking over the tiles, two accumulator buffers
+      const int tiles = ceil_div(p.M, 2 * kBM) * (p.N / 256), max_pairs = sms / 2;
+      grid = dim3(2 * (tiles < max_pairs ? tiles : max_pairs), 1, 1);
+      e = run(dense_pair_persist_kernel, PersistSmem::total + 1024);
+    } else if (pair) e = bn == 256 ? run(dense_pair_kernel<256>, PairSmem<256>::total + 1024) : run(dense_pair_kernel<128>, PairSmem<128>::total + 1024);
     else e = bn == 256 ? run(dense_tc_kernel<256>, DenseSmem<256>::total + 1024) : run(dense_tc_kernel<128>, DenseSmem<128>::total + 1024);
     if (e != cudaSuccess) return e;
     if (q.splits > 1) {
