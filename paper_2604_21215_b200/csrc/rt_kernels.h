@@ -167,7 +167,18 @@ struct DenseParams {
   // optional: also write RMS_g(row) of the epilogue's result (h or z) for the next product.  Only a split
   // contraction does this (its reduction kernel owns whole rows); `normed` tells the caller whether it happened.
   void* norm_out; const void* norm_gain; float norm_eps; int norm_pre;
+  // DENSE_QKV (persistent CTA pairs only): three products A W_q^T, A W_k^T, A W_v^T in one launch, N = d columns each;
+  // qkRMS over each head's 64 columns of q and k (qk_norm), bf16 outputs [M, d]
+  const void *W2, *W3;                           // W = W_q, W2 = W_k, W3 = W_v
+  void *q_out, *k_out, *v_out;
+  const void *g_q, *g_k;
+  int qk_norm; float qk_eps;
 };
+constexpr int DENSE_QKV = 100;
+// The q / k~ / v~ projections of the pre-pass as one launch of persistent CTA pairs (bf16, d a multiple of 256, at least a
+// wave of tiles); false when the shape does not qualify (the caller then takes qkv_gemm_tc_launch's own kernel).
+bool dense_qkv_pair_supported(int M, int d);
+cudaError_t dense_qkv_pair_launch(const DenseParams& p, SyncArea* sync, cudaStream_t s);
 cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaStream_t s, bool* normed = nullptr);
 cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s,
                               bool chained = false);

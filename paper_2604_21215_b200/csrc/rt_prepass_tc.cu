@@ -9,6 +9,8 @@
 // accumulator, warps 0-3 own one output row per thread: tcgen05.ld, sum of squares per head,
 // gain, bf16, 16-byte stores.  Two CTAs per SM, so one tile's epilogue overlaps the other's
 // main loop.  All waits are bounded (see rt_tc.cuh).
+#include <cstring>
+
 #include "rt_kernels.h"
 #include "rt_tc.cuh"
 
@@ -178,6 +180,16 @@ bool qkv_gemm_tc_supported(const PrepassParams& p) { return p.d % 128 == 0 && p.
 
 cudaError_t qkv_gemm_tc_launch(const PrepassParams& p, SyncArea* sync, cudaStream_t s) {
   const int M = p.N * p.B;
+  if (!p.mats && dense_qkv_pair_supported(M, p.d)) {
+    // all three projections over many rows: persistent CTA pairs
+    DenseParams dp;
+    memset(&dp, 0, sizeof(dp));
+    dp.M = M; dp.N = p.d; dp.K = p.d; dp.B = p.B; dp.epi = DENSE_QKV; dp.chained = p.chained;
+    dp.A = p.n; dp.W = p.w_q; dp.W2 = p.w_k; dp.W3 = p.w_v;
+    dp.q_out = p.q; dp.k_out = p.kt; dp.v_out = p.vt; dp.g_q = p.g_q; dp.g_k = p.g_k;
+    dp.qk_norm = (p.norm_flags & RT_NORM_QK) ? 1 : 0; dp.qk_eps = p.eps;
+    return dense_qkv_pair_launch(dp, sync, s);
+  }
   int mats = 0;
   for (int w = 0; w < 3; ++w) mats += (!p.mats || ((p.mats >> w) & 1)) ? 1 : 0;
   // few rows: one head per CTA, so that the launch fills the multiprocessors

@@ -463,8 +463,54 @@ __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
+// One thread's row of a q / k~ / v~ tile: 64 columns (one head) at a time, qkRMS over the head for q and k, bf16 out.
+__device__ __forceinline__ void qkv_epilogue_row(const DenseParams& p, uint32_t tmem, int warp, int m, int which, int col0) {
+  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+  const bool qkn = p.qk_norm != 0 && which < 2;
+  const __nv_bfloat16* gain = reinterpret_cast<const __nv_bfloat16*>(which == 0 ? p.g_q : p.g_k);
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.q_out : (which == 1 ? p.k_out : p.v_out));
+#pragma unroll 1
+  for (int hh = 0; hh < 256 / kHeadDim; ++hh) {
+    uint32_t v0[32], v1[32];
+    tc_ld32(t_row + (uint32_t)(hh * kHeadDim), v0);
+    tc_ld32(t_row + (uint32_t)(hh * kHeadDim + 32), v1);
+    tc_wait_ld();
+    float rs = 1.0f;
+    if (qkn) {
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float a = __uint_as_float(v0[i]), b = __uint_as_float(v1[i]);
+        ss += a * a + b * b;
+      }
+      rs = rsqrtf(ss * (1.0f / kHeadDim) + p.qk_eps);
+    }
+    if (m >= p.M) continue;
+    const int c_head = col0 + hh * kHeadDim;
+    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)m * p.N + c_head);
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {                           // 8 columns = 16 bytes per store
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int e = c8 * 8 + 2 * j;
+        float x0 = __uint_as_float(e < 32 ? v0[e & 31] : v1[e & 31]) * rs;
+        float x1 = __uint_as_float(e + 1 < 32 ? v0[(e + 1) & 31] : v1[(e + 1) & 31]) * rs;
+        if (qkn && gain) { x0 *= __bfloat162float(gain[c_head + e]); x1 *= __bfloat162float(gain[c_head + e + 1]); }
+        const __nv_bfloat162 pk = __floats2bfloat162_rn(x0, x1);
+        w[j] = *reinterpret_cast<const uint32_t*>(&pk);
+      }
+      dst[c8] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+// QKV: the three projections of the pre-pass (p.epi == DENSE_QKV; tiles walk over q, then k~, then v~ columns, each
+// with its own weight map); otherwise one product with map_w (map_w2, map_w3 unused).
+template <bool QKV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTThreads, 1)
-dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const DenseParams p,
+dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                          const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_w3, const DenseParams p,
                           SyncArea* sync) {
   grid_dep_sync();
   extern __shared__ unsigned char smem_raw[];
@@ -474,7 +520,7 @@ dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __gri
   using PS = PersistSmem;
   constexpr int kSt = PS::stages, BN = 256;
   const int rank = (int)cluster_rank();
-  const int m_pairs = (p.M + 2 * kBM - 1) / (2 * kBM), n_tiles = p.N / BN;
+  const int m_pairs = (p.M + 2 * kBM - 1) / (2 * kBM), n_per_mat = p.N / BN, n_tiles = (QKV ? 3 : 1) * n_per_mat;
   const int T = m_pairs * n_tiles;                              // tiles; pair c takes c, c + pairs, ...
   const int pairs = (int)gridDim.x >> 1, pair_id = (int)blockIdx.x >> 1;
   const int n_kb = p.K / kTBK;
@@ -508,14 +554,16 @@ dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __gri
       int it = 0;
       bool ok = true;
       for (int t = pair_id; t < T && ok; t += pairs) {
-        const int m0 = (t % m_pairs) * 2 * kBM + rank * kBM, n0 = (t / m_pairs) * BN;
+        const int nt = t / m_pairs, which = QKV ? nt / n_per_mat : 0;
+        const int m0 = (t % m_pairs) * 2 * kBM + rank * kBM, n0 = (QKV ? nt % n_per_mat : nt) * BN;
+        const CUtensorMap* mw = which == 0 ? &map_w : (which == 1 ? &map_w2 : &map_w3);
         for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
           const int s = it % kSt;
           if (it >= kSt) ok = mbar_wait(empty(s), ((it / kSt) - 1) & 1, s_abort, sync);
           if (!ok) break;
           if (rank == 0) mbar_expect_tx(full(s), 2u * (kTABytes + PS::b_bytes));
           tma_load_2d_pair(sbase + PS::a + s * kTABytes, &map_a, full(s), kb * kTBK, m0);
-          tma_load_2d_pair(sbase + PS::b + s * PS::b_bytes, &map_w, full(s), kb * kTBK, n0 + rank * (BN / 2));
+          tma_load_2d_pair(sbase + PS::b + s * PS::b_bytes, mw, full(s), kb * kTBK, n0 + rank * (BN / 2));
         }
       }
     }
@@ -553,11 +601,13 @@ dense_pair_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __gri
     bool ok = true;
     for (int t = pair_id; t < T && ok; t += pairs, ++i) {
       const int b = i & 1;
-      const int m = (t % m_pairs) * 2 * kBM + rank * kBM + warp * 32 + lane, n0 = (t / m_pairs) * BN;
+      const int nt = t / m_pairs, which = QKV ? nt / n_per_mat : 0;
+      const int m = (t % m_pairs) * 2 * kBM + rank * kBM + warp * 32 + lane, n0 = (QKV ? nt % n_per_mat : nt) * BN;
       ok = __all_sync(0xffffffffu, mbar_wait(acc_full(b), (i >> 1) & 1, s_abort, sync));
       if (!ok) break;
       tc_fence_after();
-      dense_epilogue_row<BN>(p, tmem + (uint32_t)(b * BN), warp, m, n0, 1, 0);
+      if (QKV) qkv_epilogue_row(p, tmem + (uint32_t)(b * BN), warp, m, which, n0);
+      else dense_epilogue_row<BN>(p, tmem + (uint32_t)(b * BN), warp, m, n0, 1, 0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(acc_empty(b));
@@ -724,7 +774,9 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
       // resident pairs (one CTA per SM) walking over the tiles, two accumulator buffers
       const int tiles = ceil_div(p.M, 2 * kBM) * (p.N / 256), max_pairs = sms / 2;
       grid = dim3(2 * (tiles < max_pairs ? tiles : max_pairs), 1, 1);
-      e = run(dense_pair_persist_kernel, PersistSmem::total + 1024);
+      e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_pair_persist_kernel<false>), (int)(PersistSmem::total + 1024));
+      if (e == cudaSuccess)
+        e = launch_chained(dense_pair_persist_kernel<false>, grid, dim3(kTThreads), PersistSmem::total + 1024, s, p.chained != 0, ma, mw, mw, mw, q, sync);
     } else if (pair) e = bn == 256 ? run(dense_pair_kernel<256>, PairSmem<256>::total + 1024) : run(dense_pair_kernel<128>, PairSmem<128>::total + 1024);
     else e = bn == 256 ? run(dense_tc_kernel<256>, DenseSmem<256>::total + 1024) : run(dense_tc_kernel<128>, DenseSmem<128>::total + 1024);
     if (e != cudaSuccess) return e;
@@ -739,6 +791,23 @@ cudaError_t dense_launch(int dtype, const DenseParams& p, SyncArea* sync, cudaSt
   if (dtype == RT_BF16) dense_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(p);
   else dense_simt_kernel<float><<<grid, 256, 0, s>>>(p);
   return cudaGetLastError();
+}
+
+bool dense_qkv_pair_supported(int M, int d) {
+  return d % 256 == 0 && ceil_div(M, 2 * kBM) * 3 * (d / 256) >= sm_count() / 2;
+}
+
+cudaError_t dense_qkv_pair_launch(const DenseParams& p, SyncArea* sync, cudaStream_t s) {
+  CUtensorMap ma, m1, m2, m3;
+  if (!tensor_map_rows_bf16(&ma, p.A, p.M, p.K, kBM) || !tensor_map_rows_bf16(&m1, p.W, p.N, p.K, 128) ||
+      !tensor_map_rows_bf16(&m2, p.W2, p.N, p.K, 128) || !tensor_map_rows_bf16(&m3, p.W3, p.N, p.K, 128))
+    return cudaErrorInvalidValue;
+  const int tiles = ceil_div(p.M, 2 * kBM) * 3 * (p.N / 256), max_pairs = sm_count() / 2;
+  dim3 grid(2 * (tiles < max_pairs ? tiles : max_pairs), 1, 1);
+  const size_t smem = PersistSmem::total + 1024;
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&dense_pair_persist_kernel<true>), (int)smem);
+  if (e != cudaSuccess) return e;
+  return launch_chained(dense_pair_persist_kernel<true>, grid, dim3(kTThreads), smem, s, p.chained != 0, ma, m1, m2, m3, p, sync);
 }
 
 cudaError_t attn_value_launch(int dtype, const float* st_o, const float* st_l, void* c, long long rows, int d, int H, cudaStream_t s,
