@@ -576,6 +576,14 @@ rt_status rt_layer_recompute(const rt_config* cfg, const rt_layer_weights* w, co
     const int Lb = cfg->dtype == RT_BF16 ? 2 * kAutoLeaf : kAutoLeaf;
     const int full = N / Lb;
     tp.causal = 1;
+    if (cfg->dtype == RT_BF16 && N % Lb == 0 && N >= 4 * Lb) {
+      // whole blocks only, tensor cores: every query's causal prefix in ONE launch (a CTA walks over the key blocks up to
+      // its own query tile) instead of diagonal blocks plus one launch per level of short tiles
+      tp.q0 = 0; tp.q1 = N; tp.k0 = 0; tp.k1 = N; tp.batch = 0; tp.batch_stride = 0; tp.causal_full = 1;
+      if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+      tp.causal_full = 0; tp.causal = 0;
+      goto attention_done;
+    }
     if (full > 0) {
       tp.q0 = 0; tp.q1 = Lb; tp.k0 = 0; tp.k1 = Lb; tp.batch = full; tp.batch_stride = Lb;
       if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
@@ -590,6 +598,7 @@ rt_status rt_layer_recompute(const rt_config* cfg, const rt_layer_weights* w, co
       tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
       if (tile_launch(cfg->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
     }
+  attention_done:;
   }
   // 4. position-wise chain over all rows at once
   ProfScope ps(s, kProfOther);

@@ -99,6 +99,8 @@ struct TileParams {
   int batch, batch_stride, q_limit;              // batch > 1: blockIdx.z-th copy of the tile, shifted by z * batch_stride rows
                                                  // (one level of Algorithm 1 in one launch); q_limit > 0 clips the queries
   int causal;                                    // 1: only pairs with key position < query position
+  int causal_full;                               // with causal (tensor-core kernel): a CTA's key blocks end at its own query tile, so one
+                                                 // launch over [q0,q1) x [k0,k1) covers every query's whole causal prefix; heavy tiles first
   int chained;                                   // row_attn only: launch as a programmatic dependent launch
   void* c_out;                                   // row_attn only: also write the attention value o/l of the row, [B, d] storage type
   int rows_q, rows_kv;                           // rows held by the query buffer / the caches (tensor-map bounds)

@@ -119,9 +119,15 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // recomputed where they are used rather than kept in registers across the roles
   auto shift = [&]() { return (int)blockIdx.z * p.batch_stride; };
   auto q_end = [&]() { const int q1 = p.q1 + shift(); return (p.q_limit > 0 && q1 > p.q_limit) ? p.q_limit : q1; };
-  const int qb = p.q0 + shift() + blockIdx.x * kBM;       // first query row of this CTA
+  // (whole causal prefix in one launch: the CTAs with the most key blocks come first)
+  const int bx = (CAUSAL && p.causal_full) ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+  const int qb = p.q0 + shift() + bx * kBM;               // first query row of this CTA
   if (qb >= q_end()) return;                              // nothing left of this copy (uniform per CTA)
-  const int n_blocks = (p.k1 - p.k0) / kBK;               // whole blocks only (checked by the launcher)
+  int n_blocks = (p.k1 - p.k0) / kBK;                     // whole blocks only (checked by the launcher)
+  if (CAUSAL && p.causal_full) {                          // no key block beyond this CTA's own queries
+    const int own = (qb + kBM - (p.k0 + shift())) / kBK;
+    n_blocks = own < n_blocks ? own : n_blocks;
+  }
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::abort_flag);
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + C::tmem_ptr);
   auto bar = [&](int i) { return sbase + C::bars + 8u * (uint32_t)i; };
@@ -261,7 +267,7 @@ tile_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaf(step_raw, (float)(i + col0), __uint_as_float(v[i])));
         }
-        if (CAUSAL) {
+        if (CAUSAL && p.k0 + shift() + (kb + 1) * kBK > qb) {          // (blocks wholly before the tile's first query need no mask)
           const int n_valid = qi - (p.k0 + shift() + kb * kBK);
 #pragma unroll
           for (int i = 0; i < 32; ++i)
