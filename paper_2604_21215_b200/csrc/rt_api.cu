@@ -234,21 +234,28 @@ rt_status run_layer(const rt_config* c, const rt_layer_weights* w, const void* x
         tp.k_cache = ws + L.kt; tp.v_cache = ws + L.vt; tp.rows_kv = n_rows; tp.q_limit = e0;
         const int full = rows / Lb;
         tp.causal = 1;
-        if (full > 0) {
-          tp.q0 = s0; tp.q1 = s0 + Lb; tp.k0 = s0; tp.k1 = s0 + Lb; tp.batch = full; tp.batch_stride = Lb;
+        if (c->dtype == RT_BF16 && rows % Lb == 0 && rows >= 4 * Lb) {
+          // whole blocks of 128, tensor cores: every query's causal prefix inside the block in one launch
+          tp.q0 = s0; tp.q1 = e0; tp.k0 = s0; tp.k1 = e0; tp.batch = 0; tp.batch_stride = 0; tp.causal_full = 1;
           if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          tp.causal_full = 0;
+        } else {
+          if (full > 0) {
+            tp.q0 = s0; tp.q1 = s0 + Lb; tp.k0 = s0; tp.k1 = s0 + Lb; tp.batch = full; tp.batch_stride = Lb;
+            if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          }
+          if (full * Lb < rows) {
+            tp.q0 = s0 + full * Lb; tp.q1 = e0; tp.k0 = tp.q0; tp.k1 = e0; tp.batch = 1; tp.batch_stride = 0;
+            if (tile_simt_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          }
+          tp.causal = 0;
+          for (long long P = Lb; P < rows; P *= 2) {
+            tp.q0 = s0 + (int)P; tp.q1 = s0 + (int)(2 * P); tp.k0 = s0; tp.k1 = s0 + (int)P;
+            tp.batch = (int)((rows - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
+            if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
+          }
         }
-        if (full * Lb < rows) {
-          tp.q0 = s0 + full * Lb; tp.q1 = e0; tp.k0 = tp.q0; tp.k1 = e0; tp.batch = 1; tp.batch_stride = 0;
-          if (tile_simt_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
-        }
-        tp.causal = 0;
-        for (long long P = Lb; P < rows; P *= 2) {
-          tp.q0 = s0 + (int)P; tp.q1 = s0 + (int)(2 * P); tp.k0 = s0; tp.k1 = s0 + (int)P;
-          tp.batch = (int)((rows - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
-          if (tile_launch(c->dtype, tp, s) != cudaSuccess) return RT_ERR_CUDA;
-        }
-        tp.batch = 0; tp.batch_stride = 0; tp.q_limit = 0;
+        tp.causal = 0; tp.batch = 0; tp.batch_stride = 0; tp.q_limit = 0;
       }
       {
         // 2. position-wise chain over the block's rows, 3. its persistent pairs
