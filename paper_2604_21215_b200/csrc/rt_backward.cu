@@ -1275,19 +1275,26 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     const int Lb = 128;                                         // diagonal blocks under the causal mask, then Algorithm 1's levels
     const int full = N / Lb;
     tp.causal = 1;
-    if (full > 0) {
-      tp.q0 = 0; tp.q1 = Lb; tp.k0 = 0; tp.k1 = Lb; tp.batch = full; tp.batch_stride = Lb;
+    if (N % Lb == 0 && N >= 4 * Lb) {
+      // whole blocks: every query's causal prefix in one launch (a CTA walks over the key blocks up to its own query tile)
+      tp.q0 = 0; tp.q1 = N; tp.k0 = 0; tp.k1 = N; tp.causal_full = 1;
       RT_TRY(tile_launch(RT_BF16, tp, s));
-    }
-    if (full * Lb < N) {
-      tp.q0 = full * Lb; tp.q1 = N; tp.k0 = full * Lb; tp.k1 = N; tp.batch = 1; tp.batch_stride = 0;
-      RT_TRY(tile_simt_launch(RT_BF16, tp, s));
-    }
-    tp.causal = 0;
-    for (long long P = Lb; P < N; P *= 2) {
-      tp.q0 = (int)P; tp.q1 = (int)(2 * P); tp.k0 = 0; tp.k1 = (int)P;
-      tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
-      RT_TRY(tile_launch(RT_BF16, tp, s));
+      tp.causal_full = 0;
+    } else {
+      if (full > 0) {
+        tp.q0 = 0; tp.q1 = Lb; tp.k0 = 0; tp.k1 = Lb; tp.batch = full; tp.batch_stride = Lb;
+        RT_TRY(tile_launch(RT_BF16, tp, s));
+      }
+      if (full * Lb < N) {
+        tp.q0 = full * Lb; tp.q1 = N; tp.k0 = full * Lb; tp.k1 = N; tp.batch = 1; tp.batch_stride = 0;
+        RT_TRY(tile_simt_launch(RT_BF16, tp, s));
+      }
+      tp.causal = 0;
+      for (long long P = Lb; P < N; P *= 2) {
+        tp.q0 = (int)P; tp.q1 = (int)(2 * P); tp.k0 = 0; tp.k1 = (int)P;
+        tp.batch = (int)((N - P + 2 * P - 1) / (2 * P)); tp.batch_stride = (int)(2 * P);
+        RT_TRY(tile_launch(RT_BF16, tp, s));
+      }
     }
     stats_finish_kernel<<<warps_grid(rows * H), tpb, 0, s>>>(ab, st_o, st_m, st_l);
   } else {
