@@ -241,13 +241,18 @@ __device__ __forceinline__ float gelu_f(float a) { return 0.5f * a * (1.f + erff
 __device__ __forceinline__ float gelu_grad_f(float a) {
   return 0.5f * (1.f + erff(a * 0.70710678118654752f)) + a * 0.3989422804014327f * __expf(-0.5f * a * a);
 }
+// four consecutive entries per thread (n a multiple of 4: d_ff is)
 __global__ void gelu_bwd_kernel(float* __restrict__ dg, const float* __restrict__ a, long long n, __nv_bfloat16* out_bf) {
   grid_dep_sync();
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long idx = 4 * ((long long)blockIdx.x * blockDim.x + threadIdx.x);
   if (idx < n) {
-    const float v = dg[idx] * gelu_grad_f(a[idx]);
-    dg[idx] = v;
-    if (out_bf) out_bf[idx] = __float2bfloat16_rn(v);
+    const float4 g = *reinterpret_cast<const float4*>(dg + idx), x = *reinterpret_cast<const float4*>(a + idx);
+    const float4 v = make_float4(g.x * gelu_grad_f(x.x), g.y * gelu_grad_f(x.y), g.z * gelu_grad_f(x.z), g.w * gelu_grad_f(x.w));
+    *reinterpret_cast<float4*>(dg + idx) = v;
+    if (out_bf) {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+      *reinterpret_cast<uint2*>(out_bf + idx) = make_uint2(*reinterpret_cast<const unsigned*>(&lo), *reinterpret_cast<const unsigned*>(&hi));
+    }
   }
 }
 __global__ void gelu_kernel(const float* __restrict__ a, float* __restrict__ out, long long n) {
@@ -1411,7 +1416,7 @@ rt_status backward_impl(const rt_config* c, const rt_layer_weights* w, const T* 
     RT_TRY(launch_chained(norm_bwd_row_kernel<T, T>, dim3(B), dim3(256), 0, s, true, (const float*)(F(L.dr) + od), z + (size_t)i * xts, xbs, xts, B,
                           g_kv, (const float*)(F(L.dzp) + od), F(L.Gz) + od, d, eps, z_norm ? 1 : 0, tc ? SA : (__nv_bfloat16*)nullptr, alpha));
     RT_TRY(step_product(F(L.Gz) + od, SA, d, Wdn, WdnT, f, F(L.dpre) + of, alpha, false));
-    RT_TRY(launch_chained(gelu_bwd_kernel, dim3(elems_grid((long long)pos_f)), blk, 0, s, true, F(L.dpre) + of, (const float*)(F(L.act) + of),
+    RT_TRY(launch_chained(gelu_bwd_kernel, dim3(elems_grid(((long long)pos_f + 3) / 4)), blk, 0, s, true, F(L.dpre) + of, (const float*)(F(L.act) + of),
                           (long long)pos_f, tc ? SA : (__nv_bfloat16*)nullptr));
     // du = dpre W_up;  dh = Gz + RMS backward of du;  dc = alpha dh W_o
     RT_TRY(step_product(F(L.dpre) + of, SA, f, Wup, WupT, d, F(L.du) + od, 1.f, false));
