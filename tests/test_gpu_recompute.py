@@ -32,7 +32,11 @@ def _case(dtype, d, H, dff, B, N, seed, gains=False, alibi=False):
     ("bf16", 256, 4, 1024, 3, 333, 3, True, False, 1.0),
     ("bf16", 768, 12, 3072, 2, 300, 3, False, True, 0.6),
     ("bf16", 320, 5, 384, 5, 129, 1, False, False, 1.0),
-    ("bf16", 128, 2, 512, 16, 1, 3, False, False, 1.0)])
+    ("bf16", 128, 2, 512, 16, 1, 3, False, False, 1.0),
+    # 9950 rows (not a multiple of the 256-row pair tiles) and 10240 rows with N a multiple of 128: the products and the
+    # projections run on persistent CTA pairs, the second case's attention as one causal launch with ALiBi distances
+    ("bf16", 256, 4, 1024, 5, 1990, 3, True, False, 1.0),
+    ("bf16", 256, 4, 1024, 5, 2048, 3, False, True, 0.7)])
 def test_recompute_matches_fixed_point_sweep(dtype, d, H, dff, B, N, flags, gains, alibi, alpha):
     # z_claim is NOT the true output (random): the sweep must still reproduce the oracle's one-sweep map
     # z_claim -> (z', k, v), which exercises every product and every attention pair without relying on
