@@ -165,6 +165,19 @@ def test_c2_full_size_bf16_matches_oracle():
     check(got, ref, TOL["bf16"], "c2")
 
 
+def test_prefill_with_a_ragged_row_count_on_the_pair_kernels():
+    # 5 x 1990 = 9950 rows: the pre-pass projections run on persistent CTA pairs (256-row tiles, the last one ragged),
+    # N is not a multiple of the leaf, B = 5 leaves three of the eight sequence slots of the leaf kernel empty
+    from paper_2604_21215_b200 import inputs
+    d, H, dff, B, N = 256, 4, 1024, 5, 1990
+    wl = inputs.Workload("ragged_rows", 1, B, N, d, H, dff, "bf16")
+    data = inputs.make_inputs(wl, seed=4242)
+    lw = data["layers"][0]
+    ref = oracle_layer(data["x"], lw, d, H, dff)
+    _, got = run_layer(data["x"], lw, d, H, dff, "bf16")
+    check(got, ref, TOL["bf16"], "ragged rows")
+
+
 def test_c3_full_size_bf16_prefix_and_fixed_point():
     # The oracle replays the first 384 positions (causality makes them independent of the
     # rest); the whole length is checked with the fixed-point property on one sequence: feeding
