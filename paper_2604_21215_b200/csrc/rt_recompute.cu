@@ -315,8 +315,8 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // Two CTAs of a cluster share a 256 x BN output tile: each fetches its own 128 rows of A and HALF of the BN weight rows,
 // the leader's thread issues tcgen05.mma.cta_group::2 (M = 256), which reads A and W from both CTAs' shared memory and
 // accumulates each CTA's 128 rows in that CTA's TMEM.  Per CTA and 64-wide k-block that is 16 KB + BN * 64 bytes from L2
-// instead of 16 KB + BN * 128: the products here are bound by that stream.  Copies are plain TMA loads (no multicast)
-// that report to the leader's barrier; the leader's commits reach both CTAs' barriers.
+// instead of 16 KB + BN * 128: the products here are bound by that stream.  Copies are plain TMA loads, one per CTA,
+// that report to the leader's barrier; the leader's commits arrive on both CTAs' barriers.
 template <int BN>
 struct PairSmem {
   static constexpr int stages = BN == 256 ? 3 : 4;
@@ -343,9 +343,13 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
                ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {           // arrives on the barrier at this offset in BOTH CTAs
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"((unsigned short)3) : "memory");
+// Issued by the leader: arrives on the barrier at this offset in BOTH CTAs once the pair's products so far are done
+// (one commit per CTA's barrier; the partner's address comes from mapa).
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  uint32_t peer;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer) : "r"(bar), "r"(1u));
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 
 template <int BN>
